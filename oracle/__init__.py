@@ -1,0 +1,173 @@
+"""fp64 CPU oracle for RoCo KV-constrained inference (test infrastructure only).
+
+Thin ctypes/numpy marshalling around ``roco_oracle.c``; all arithmetic is in the C file.
+Only the test suite, the smoke check and the benchmark's CPU-baseline leg may import this
+package; the CUDA library never does.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+
+from .build import build as build_library
+
+EXCLUDE_TOP_R, LOWEST_R = 0, 1
+EVICT_FIRST, ATTEND_FIRST = 0, 1
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build_library())
+        _lib.roco_oracle_threads.restype = C.c_int
+        _lib.roco_oracle_select.restype = C.c_int
+        _lib.roco_oracle_select_to_budget_onepass.restype = C.c_int
+        _lib.roco_oracle_prefill_unit.restype = C.c_int
+        _lib.roco_oracle_prefill_batch.restype = C.c_int
+    return _lib
+
+
+def threads() -> int:
+    return int(lib().roco_oracle_threads())
+
+
+def _f64(a):
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def prefill_stats(Q, K, scale, count_self=1, want_P=False):
+    """Column statistics of the causal softmax of one unit.  Q, K: [L][d].
+    Returns lse [L], s [L], q [L], n [L] (and P [L][L] if asked)."""
+    Q, K = _f64(Q), _f64(K)
+    L, d = Q.shape
+    lse = np.zeros(L); s = np.zeros(L); q = np.zeros(L); n = np.zeros(L, np.int32)
+    P = np.zeros((L, L)) if want_P else None
+    lib().roco_oracle_prefill_stats(_p(Q), _p(K), C.c_int(L), C.c_int(d), C.c_double(scale),
+                                    C.c_int(count_self), _p(lse), _p(s), _p(q), _p(n), _p(P))
+    return (lse, s, q, n, P) if want_P else (lse, s, q, n)
+
+
+def select(s, q, n, pos, r, mode, delta=1e-5):
+    """Victim slot among slots 0..len-1.  Returns (slot, near_tie, scope_size)."""
+    s, q, n, pos = _f64(s), _f64(q), _i32(n), _i32(pos)
+    near, m = C.c_int(0), C.c_int(0)
+    slot = lib().roco_oracle_select(_p(s), _p(q), _p(n), _p(pos), C.c_int(len(s)), C.c_int(r), C.c_int(mode),
+                                    C.c_double(delta), C.byref(near), C.byref(m))
+    return int(slot), bool(near.value), int(m.value)
+
+
+def select_to_budget_iterated(s, q, n, B, r, mode):
+    s, q, n = _f64(s), _f64(q), _i32(n)
+    keep = np.zeros(len(s), np.int32)
+    lib().roco_oracle_select_to_budget_iterated(_p(s), _p(q), _p(n), C.c_int(len(s)), C.c_int(B), C.c_int(r),
+                                                C.c_int(mode), _p(keep))
+    return keep.astype(bool)
+
+
+def select_to_budget_onepass(s, q, n, B, r, delta=1e-5):
+    s, q, n = _f64(s), _f64(q), _i32(n)
+    keep = np.zeros(len(s), np.int32); unc = np.zeros(len(s), np.int32)
+    rc = lib().roco_oracle_select_to_budget_onepass(_p(s), _p(q), _p(n), C.c_int(len(s)), C.c_int(B), C.c_int(r),
+                                                    C.c_double(delta), _p(keep), _p(unc))
+    if rc:
+        raise ValueError(f"one-pass select-to-budget precondition failed ({rc})")
+    return keep.astype(bool), unc.astype(bool)
+
+
+@dataclass
+class State:
+    """Budgeted cache of U units, everything fp64/int32 numpy, unit-major."""
+    K: np.ndarray      # [U][B][d]
+    V: np.ndarray      # [U][B][d]
+    s: np.ndarray      # [U][B]
+    q: np.ndarray      # [U][B]
+    n: np.ndarray      # [U][B] int32
+    pos: np.ndarray    # [U][B] int32, -1 = empty
+    live: np.ndarray   # [U] int32
+    t_next: np.ndarray  # [U] int32
+
+    @property
+    def U(self): return self.K.shape[0]
+    @property
+    def B(self): return self.K.shape[1]
+    @property
+    def d(self): return self.K.shape[2]
+
+    def copy(self) -> "State":
+        return State(*(a.copy() for a in (self.K, self.V, self.s, self.q, self.n, self.pos, self.live, self.t_next)))
+
+
+def empty_state(U, B, d) -> State:
+    return State(np.zeros((U, B, d)), np.zeros((U, B, d)), np.zeros((U, B)), np.zeros((U, B)),
+                 np.zeros((U, B), np.int32), np.full((U, B), -1, np.int32), np.zeros(U, np.int32),
+                 np.zeros(U, np.int32))
+
+
+@dataclass
+class PrefillResult:
+    state: State
+    lse: np.ndarray        # [U][Lmax]
+    s_full: np.ndarray     # [U][Lmax]
+    q_full: np.ndarray
+    n_full: np.ndarray
+    keep: np.ndarray       # [U][Lmax] bool
+    uncertain: np.ndarray  # [U][Lmax] bool
+
+
+def prefill(Q, K, V, lens, B, r, mode, scale, count_self=1, delta=1e-5, force_keep=None) -> PrefillResult:
+    """Q, K, V: [U][Lmax][d]; lens: [U] per-unit prompt length."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    U, Lmax, d = Q.shape
+    lens = _i32(lens)
+    st = empty_state(U, B, d)
+    lse = np.zeros((U, Lmax)); sf = np.zeros((U, Lmax)); qf = np.zeros((U, Lmax)); nf = np.zeros((U, Lmax), np.int32)
+    keep = np.zeros((U, Lmax), np.int32) if force_keep is None else _i32(force_keep).copy()
+    unc = np.zeros((U, Lmax), np.int32)
+    rc = lib().roco_oracle_prefill_batch(C.c_int(U), _p(Q), _p(K), _p(V), _p(lens), C.c_int(Lmax), C.c_int(d),
+                                         C.c_int(B), C.c_int(r), C.c_int(mode), C.c_double(scale),
+                                         C.c_int(count_self), C.c_double(delta), _p(st.K), _p(st.V), _p(st.s),
+                                         _p(st.q), _p(st.n), _p(st.pos), _p(st.live), _p(lse), _p(sf), _p(qf),
+                                         _p(nf), _p(keep), C.c_int(0 if force_keep is None else 1), _p(unc))
+    if rc:
+        raise ValueError(f"oracle prefill failed ({rc})")
+    st.t_next[:] = lens
+    return PrefillResult(st, lse, sf, qf, nf, keep.astype(bool), unc.astype(bool))
+
+
+@dataclass
+class StepResult:
+    out: np.ndarray           # [U][d]
+    lse: np.ndarray           # [U]
+    evicted_slot: np.ndarray  # [U], -1 = nothing evicted
+    evicted_pos: np.ndarray   # [U]
+    choice: np.ndarray        # [U] the policy's own victim (differs from evicted_slot only when forced)
+    near_tie: np.ndarray      # [U] bool
+
+
+def decode_step(st: State, qv, k_new, v_new, r, mode, order, scale, count_self=1, delta=1e-5,
+                force_victim: Optional[np.ndarray] = None) -> StepResult:
+    """One decode step of every unit, in place on `st`.  qv, k_new, v_new: [U][d]."""
+    qv, k_new, v_new = _f64(qv), _f64(k_new), _f64(v_new)
+    U, B, d = st.U, st.B, st.d
+    out = np.zeros((U, d)); lse = np.zeros(U)
+    es = np.zeros(U, np.int32); ep = np.zeros(U, np.int32); ch = np.zeros(U, np.int32); nt = np.zeros(U, np.int32)
+    fv = None if force_victim is None else _i32(force_victim)
+    lib().roco_oracle_decode_step_batch(C.c_int(U), _p(st.K), _p(st.V), _p(st.s), _p(st.q), _p(st.n), _p(st.pos),
+                                        _p(st.live), _p(st.t_next), C.c_int(B), C.c_int(d), _p(qv), _p(k_new),
+                                        _p(v_new), C.c_int(r), C.c_int(mode), C.c_int(order), C.c_double(scale),
+                                        C.c_int(count_self), C.c_double(delta), _p(fv), _p(out), _p(lse), _p(es),
+                                        _p(ep), _p(ch), _p(nt))
+    return StepResult(out, lse, es, ep, ch, nt.astype(bool))

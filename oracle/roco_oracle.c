@@ -1,0 +1,411 @@
+/*
+ * CPU oracle for KV-constrained inference with the RoCo eviction policy.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain restatement of the
+ * paper's definitions that the CUDA library is checked against.  It shares no
+ * code with the CUDA path and must never be called from it: only the test
+ * suite, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * Everything is fp64.  Inputs are the exact fp32/bf16 input values widened to
+ * double by the caller.  One "unit" = one (sequence, layer, head); units are
+ * independent (Fig. 1: heads evict at different positions), and the only
+ * parallelism here is an OpenMP loop over units in the *_batch drivers.
+ *
+ * What each function follows:
+ *   softmax / attention ............ Eq. 1 (scaled dot-product attention, one head)
+ *   causal prefill ................. Sec. 2.1 "Key-Value Cache": a token sees itself and earlier tokens
+ *   Acc, Acc^square, Count ......... Sec. 4.3: three B-sized arrays per head
+ *   mean attention score (MAS) ..... Sec. 4.3: Acc / Count
+ *   Std ............................ Sec. 4.3: sqrt(Acc^square/Count - (Acc/Count)^2); ranking uses the
+ *                                    variance (sqrt is monotone), population form (divide by Count)
+ *   eviction scope ................. Sec. 4.3: exclude the r tokens of highest Std (EXCLUDE_TOP_R);
+ *                                    Sec. 1: "tokens with the lowest variance" read as the r lowest
+ *                                    (LOWEST_R).  Both are "the m lowest-variance tokens" with
+ *                                    m = live - r or m = r.
+ *   victim ......................... Sec. 4.3: the in-scope token of lowest mean attention score
+ *   fixed buffer, evict when full .. Sec. 3 (n <= B at every step), Sec. 4 first paragraph
+ *   evict before appending ......... Fig. 1 caption (EVICT_FIRST step order)
+ *   prefill-stage eviction to B .... Sec. 4.3 last paragraph / Sec. 5.1 "Other Details" (B = len x rate)
+ *
+ * Readings where the paper is silent (stated once here, in words):
+ *   - ties: scope membership by (variance asc, position asc); victim by (mean asc, position asc);
+ *   - a token's own query counts (count_self = 1) unless asked otherwise; with count_self = 0 tokens
+ *     whose Count is still 0 are not evictable;
+ *   - statistics are raw accumulations: no reset or renormalisation after an eviction;
+ *   - a freed slot is overwritten in place; while the buffer is not full the new token goes to slot
+ *     `live`; after prefill the survivors sit in increasing position order;
+ *   - select-to-budget at prefill = the per-step rule applied L-B times on frozen statistics.
+ *
+ * Parity pins: every function here is pinned by tests that do not call it to produce their expected
+ * values (hand-worked rationals, harmonic-number closed forms, library softmax/logsumexp, brute-force
+ * history recomputation, invariants).  No function is "parity unpinned".
+ */
+#include <float.h>
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ROCO_ORACLE_EXCLUDE_TOP_R = 0, ROCO_ORACLE_LOWEST_R = 1 };
+enum { ROCO_ORACLE_EVICT_FIRST = 0, ROCO_ORACLE_ATTEND_FIRST = 1 };
+
+int roco_oracle_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/* ---------------------------------------------------------------- Eq. 1 -- */
+
+/* p = Softmax(scale * qv . K[j]) over j = 0..count-1, with max subtraction.
+ * Returns log-sum-exp of the scaled scores (-inf when count == 0). */
+static double softmax_row(const double *qv, const double *K, int count, int d, double scale, double *p) {
+  if (count <= 0) return -INFINITY;
+  double zmax = -INFINITY;
+  for (int j = 0; j < count; ++j) {
+    double z = 0.0;
+    for (int c = 0; c < d; ++c) z += qv[c] * K[(size_t)j * d + c];
+    z *= scale;
+    p[j] = z;
+    if (z > zmax) zmax = z;
+  }
+  double Z = 0.0;
+  for (int j = 0; j < count; ++j) {
+    p[j] = exp(p[j] - zmax);
+    Z += p[j];
+  }
+  for (int j = 0; j < count; ++j) p[j] /= Z;
+  return zmax + log(Z);
+}
+
+/* Causal prefill statistics of one unit (Eq. 1 with the causal mask; Sec. 4.3 arrays).
+ * Q, K: [L][d].  lse: [L] (may be NULL).  s, q: [L] doubles; n: [L] ints.
+ * P_out: [L][L] row-major full probability matrix (may be NULL; zeros above the diagonal). */
+void roco_oracle_prefill_stats(const double *Q, const double *K, int L, int d, double scale, int count_self,
+                               double *lse, double *s, double *q, int *n, double *P_out) {
+  double *p = (double *)malloc(sizeof(double) * (size_t)(L > 0 ? L : 1));
+  for (int j = 0; j < L; ++j) { s[j] = 0.0; q[j] = 0.0; n[j] = 0; }
+  if (P_out) memset(P_out, 0, sizeof(double) * (size_t)L * L);
+  for (int i = 0; i < L; ++i) {
+    double l = softmax_row(Q + (size_t)i * d, K, i + 1, d, scale, p);   /* row i sees keys 0..i */
+    if (lse) lse[i] = l;
+    for (int j = 0; j <= i; ++j) {
+      if (P_out) P_out[(size_t)i * L + j] = p[j];
+      if (j == i && !count_self) continue;
+      s[j] += p[j];
+      q[j] += p[j] * p[j];
+      n[j] += 1;
+    }
+  }
+  free(p);
+}
+
+/* ------------------------------------------------- scope and victim (4.3) -- */
+
+typedef struct {
+  double var, mean, ab; /* ab = Acc^square/Count + mean^2: the uncancelled magnitude of the variance */
+  int pos, slot;
+} cand_t;
+
+static int cmp_var_pos(const void *a, const void *b) {
+  const cand_t *x = (const cand_t *)a, *y = (const cand_t *)b;
+  if (x->var < y->var) return -1;
+  if (x->var > y->var) return 1;
+  return (x->pos > y->pos) - (x->pos < y->pos);
+}
+
+static int before_mean_pos(const cand_t *x, const cand_t *y) {
+  if (x->mean < y->mean) return 1;
+  if (x->mean > y->mean) return 0;
+  return x->pos < y->pos;
+}
+
+/* Victim among slots 0..live-1.  Returns the slot; *near_tie is set when the decision margin is
+ * below delta (relative): the runner-up's mean is within delta*(sum of the two means); or the victim,
+ * or a lower-mean outsider, sits within delta*(uncancelled variance terms) of the scope boundary.
+ * *scope_size receives m. */
+int roco_oracle_select(const double *s, const double *q, const int *n, const int *pos, int live, int r,
+                       int mode, double delta, int *near_tie, int *scope_size) {
+  if (near_tie) *near_tie = 0;
+  if (scope_size) *scope_size = 0;
+  if (live <= 0) return -1;
+  cand_t *c = (cand_t *)malloc(sizeof(cand_t) * (size_t)live);
+  int nc = 0;
+  for (int j = 0; j < live; ++j) {
+    if (n[j] <= 0) continue; /* never attended yet (count_self = 0 only): not evictable */
+    double mean = s[j] / n[j];
+    double a = q[j] / n[j];
+    double var = a - mean * mean;
+    if (var < 0.0) var = 0.0;
+    c[nc].mean = mean; c[nc].var = var; c[nc].ab = a + mean * mean;
+    c[nc].pos = pos[j]; c[nc].slot = j;
+    ++nc;
+  }
+  if (nc == 0) { /* nothing has statistics: fall back to the oldest token */
+    int best = 0;
+    for (int j = 1; j < live; ++j) if (pos[j] < pos[best]) best = j;
+    free(c);
+    return best;
+  }
+  qsort(c, (size_t)nc, sizeof(cand_t), cmp_var_pos);
+  int m = (mode == ROCO_ORACLE_EXCLUDE_TOP_R) ? nc - r : r;
+  if (m < 1) m = 1;
+  if (m > nc) m = nc;
+  if (scope_size) *scope_size = m;
+  int v = 0;
+  for (int k = 1; k < m; ++k) if (before_mean_pos(&c[k], &c[v])) v = k;
+  if (near_tie) {
+    int near = 0;
+    /* (i) runner-up in scope */
+    int u = -1;
+    for (int k = 0; k < m; ++k) {
+      if (k == v) continue;
+      if (u < 0 || before_mean_pos(&c[k], &c[u])) u = k;
+    }
+    if (u >= 0 && c[u].mean - c[v].mean <= delta * (c[u].mean + c[v].mean)) near = 1;
+    if (m < nc) {
+      /* (ii) the victim could drop out of the scope */
+      double lo_out = INFINITY; /* lowest reachable variance of any outsider */
+      for (int k = m; k < nc; ++k) {
+        double t = c[k].var - delta * c[k].ab;
+        if (t < lo_out) lo_out = t;
+      }
+      if (lo_out <= c[v].var + delta * c[v].ab) near = 1;
+      /* (iii) an outsider that would win on mean could enter the scope */
+      double hi_in = -INFINITY; /* highest reachable variance of any insider */
+      for (int k = 0; k < m; ++k) {
+        double t = c[k].var + delta * c[k].ab;
+        if (t > hi_in) hi_in = t;
+      }
+      for (int k = m; k < nc && !near; ++k) {
+        if (c[k].mean <= c[v].mean + delta * (c[k].mean + c[v].mean) && c[k].var - delta * c[k].ab <= hi_in)
+          near = 1;
+      }
+    }
+    *near_tie = near;
+  }
+  int slot = c[v].slot;
+  free(c);
+  return slot;
+}
+
+/* Select-to-budget, literal form: apply the per-step rule L-B times on frozen statistics, removing the
+ * victim each time.  keep[j] = 1 for survivors.  Works for both scope modes. */
+void roco_oracle_select_to_budget_iterated(const double *s, const double *q, const int *n, int L, int B, int r,
+                                           int mode, int *keep) {
+  for (int j = 0; j < L; ++j) keep[j] = 1;
+  if (L <= B) return;
+  double *cs = (double *)malloc(sizeof(double) * (size_t)L), *cq = (double *)malloc(sizeof(double) * (size_t)L);
+  int *cn = (int *)malloc(sizeof(int) * (size_t)L), *cp = (int *)malloc(sizeof(int) * (size_t)L);
+  for (int alive = L; alive > B; --alive) {
+    int k = 0;
+    for (int j = 0; j < L; ++j)
+      if (keep[j]) { cs[k] = s[j]; cq[k] = q[j]; cn[k] = n[j]; cp[k] = j; ++k; }
+    int slot = roco_oracle_select(cs, cq, cn, cp, alive, r, mode, 0.0, NULL, NULL);
+    keep[cp[slot]] = 0;
+  }
+  free(cs); free(cq); free(cn); free(cp);
+}
+
+typedef struct { double key; double eps; int pos; } rank_t;
+static int cmp_key_pos(const void *a, const void *b) {
+  const rank_t *x = (const rank_t *)a, *y = (const rank_t *)b;
+  if (x->key < y->key) return -1;
+  if (x->key > y->key) return 1;
+  return (x->pos > y->pos) - (x->pos < y->pos);
+}
+
+/* Select-to-budget, one pass (EXCLUDE_TOP_R only, every Count > 0, r <= B): protect the r tokens last in
+ * (variance, position) order; of the others evict the L-B first in (mean, position) order.  Equal to the
+ * iterated form because a protected token is never in scope, so the protected set never changes.
+ * uncertain[j] = 1 where token j's fate could flip within the relative margin delta (near either
+ * boundary; if any token is near the protection boundary, the tokens around the eviction boundary that
+ * a one-token shift per such token could reach are marked too).  Returns 0, or -1 on a precondition. */
+int roco_oracle_select_to_budget_onepass(const double *s, const double *q, const int *n, int L, int B, int r,
+                                         double delta, int *keep, int *uncertain) {
+  for (int j = 0; j < L; ++j) { keep[j] = 1; if (uncertain) uncertain[j] = 0; }
+  if (L <= B) return 0;
+  if (r > B || r < 0) return -1;
+  for (int j = 0; j < L; ++j) if (n[j] <= 0) return -1;
+  rank_t *v = (rank_t *)malloc(sizeof(rank_t) * (size_t)L);
+  for (int j = 0; j < L; ++j) {
+    double mean = s[j] / n[j], a = q[j] / n[j];
+    double var = a - mean * mean;
+    if (var < 0.0) var = 0.0;
+    v[j].key = var; v[j].eps = delta * (a + mean * mean); v[j].pos = j;
+  }
+  qsort(v, (size_t)L, sizeof(rank_t), cmp_key_pos);
+  int nu = L - r; /* unprotected: v[0..nu) */
+  int shaky = 0;  /* tokens that could cross the protection boundary */
+  if (r > 0 && nu > 0 && uncertain) {
+    double lo_prot = INFINITY, hi_unprot = -INFINITY;
+    for (int k = nu; k < L; ++k) if (v[k].key - v[k].eps < lo_prot) lo_prot = v[k].key - v[k].eps;
+    for (int k = 0; k < nu; ++k) if (v[k].key + v[k].eps > hi_unprot) hi_unprot = v[k].key + v[k].eps;
+    for (int k = 0; k < L; ++k) {
+      int crosses = (k < nu) ? (v[k].key + v[k].eps >= lo_prot) : (v[k].key - v[k].eps <= hi_unprot);
+      if (crosses) { uncertain[v[k].pos] = 1; ++shaky; }
+    }
+  }
+  rank_t *m = (rank_t *)malloc(sizeof(rank_t) * (size_t)(nu > 0 ? nu : 1));
+  for (int k = 0; k < nu; ++k) {
+    int j = v[k].pos;
+    m[k].key = s[j] / n[j]; m[k].eps = delta * m[k].key; m[k].pos = j;
+  }
+  qsort(m, (size_t)nu, sizeof(rank_t), cmp_key_pos);
+  int E = L - B;
+  for (int k = 0; k < E; ++k) keep[m[k].pos] = 0;
+  if (uncertain && E < nu) {
+    double last_out = m[E - 1].key + m[E - 1].eps, first_in = m[E].key - m[E].eps;
+    for (int k = 0; k < nu; ++k) {
+      int near = (k < E) ? (m[k].key + m[k].eps >= first_in) : (m[k].key - m[k].eps <= last_out);
+      if (near) uncertain[m[k].pos] = 1;
+    }
+    int lo = E - shaky, hi = E + shaky;
+    if (lo < 0) lo = 0;
+    if (hi > nu) hi = nu;
+    for (int k = lo; k < hi; ++k) uncertain[m[k].pos] = 1;
+  }
+  free(v); free(m);
+  return 0;
+}
+
+/* ------------------------------------------------------------ prefill ---- */
+
+/* Whole prefill of one unit: statistics, select-to-budget, survivors copied in increasing position
+ * order.  Q,K,V: [L][d].  Cache outputs: Kc,Vc [B][d]; sc,qc [B]; nc,posc [B] (pos = -1 for empty);
+ * *live = min(L,B).  s_full,q_full,n_full: [L] pre-eviction statistics (required).  keep_io [L]:
+ * if force_keep != 0 it is read as the survivor set to use; otherwise it receives the oracle's own.
+ * uncertain [L] may be NULL.  LOWEST_R uses the iterated form (no margin analysis). */
+int roco_oracle_prefill_unit(const double *Q, const double *K, const double *V, int L, int d, int B, int r,
+                             int mode, double scale, int count_self, double delta, double *Kc, double *Vc,
+                             double *sc, double *qc, int *nc, int *posc, int *live, double *lse, double *s_full,
+                             double *q_full, int *n_full, int *keep_io, int force_keep, int *uncertain) {
+  roco_oracle_prefill_stats(Q, K, L, d, scale, count_self, lse, s_full, q_full, n_full, NULL);
+  if (!force_keep) {
+    int rc = 0;
+    if (mode == ROCO_ORACLE_EXCLUDE_TOP_R && count_self)
+      rc = roco_oracle_select_to_budget_onepass(s_full, q_full, n_full, L, B, r, delta, keep_io, uncertain);
+    else {
+      roco_oracle_select_to_budget_iterated(s_full, q_full, n_full, L, B, r, mode, keep_io);
+      if (uncertain) for (int j = 0; j < L; ++j) uncertain[j] = 0;
+    }
+    if (rc) return rc;
+  }
+  int k = 0;
+  for (int j = 0; j < L; ++j) {
+    if (!keep_io[j]) continue;
+    if (k >= B) return -2;
+    memcpy(Kc + (size_t)k * d, K + (size_t)j * d, sizeof(double) * (size_t)d);
+    memcpy(Vc + (size_t)k * d, V + (size_t)j * d, sizeof(double) * (size_t)d);
+    sc[k] = s_full[j]; qc[k] = q_full[j]; nc[k] = n_full[j]; posc[k] = j;
+    ++k;
+  }
+  *live = k;
+  for (; k < B; ++k) {
+    memset(Kc + (size_t)k * d, 0, sizeof(double) * (size_t)d);
+    memset(Vc + (size_t)k * d, 0, sizeof(double) * (size_t)d);
+    sc[k] = 0.0; qc[k] = 0.0; nc[k] = 0; posc[k] = -1;
+  }
+  return 0;
+}
+
+/* ------------------------------------------------------------- decode ---- */
+
+static void insert_token(double *K, double *V, double *s, double *q, int *n, int *pos, int slot, int d,
+                         const double *k_new, const double *v_new, int t) {
+  memcpy(K + (size_t)slot * d, k_new, sizeof(double) * (size_t)d);
+  memcpy(V + (size_t)slot * d, v_new, sizeof(double) * (size_t)d);
+  s[slot] = 0.0; q[slot] = 0.0; n[slot] = 0; pos[slot] = t;
+}
+
+static double attend(const double *K, const double *V, double *s, double *q, int *n, int live, int d,
+                     const double *qv, double scale, int skip_slot, double *out, double *p) {
+  double lse = softmax_row(qv, K, live, d, scale, p);
+  for (int c = 0; c < d; ++c) out[c] = 0.0;
+  for (int j = 0; j < live; ++j) {
+    for (int c = 0; c < d; ++c) out[c] += p[j] * V[(size_t)j * d + c];
+    if (j == skip_slot) continue; /* count_self = 0: the new token's own query is not a "future" query */
+    s[j] += p[j];
+    q[j] += p[j] * p[j];
+    n[j] += 1;
+  }
+  return lse;
+}
+
+/* One decode step of one unit.  Cache K,V [B][d]; s,q [B]; n,pos [B]; *live; *t_next = position of the
+ * new token (incremented on return).  force_victim >= 0 replaces the policy's choice when the buffer is
+ * full (used to continue from a common state after a logged near-tie).
+ * Outputs: out [d]; *lse; *evicted_slot (-1 when nothing was evicted); *evicted_pos; *choice = the
+ * policy's own victim (-1 if none); *near_tie.  p_out [B] may be NULL. */
+void roco_oracle_decode_step_unit(double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
+                                  int *t_next, int B, int d, const double *qv, const double *k_new,
+                                  const double *v_new, int r, int mode, int order, double scale,
+                                  int count_self, double delta, int force_victim, double *out, double *lse,
+                                  int *evicted_slot, int *evicted_pos, int *choice, int *near_tie,
+                                  double *p_out) {
+  double *p = p_out ? p_out : (double *)malloc(sizeof(double) * (size_t)B);
+  int t = *t_next, slot, near = 0, own = -1;
+  *evicted_slot = -1;
+  *evicted_pos = -1;
+  if (order == ROCO_ORACLE_ATTEND_FIRST)
+    *lse = attend(K, V, s, q, n, *live, d, qv, scale, -1, out, p); /* the new token is not in the cache yet */
+  if (*live == B) { /* buffer full: run the policy (Sec. 4) */
+    own = roco_oracle_select(s, q, n, pos, *live, r, mode, delta, &near, NULL);
+    slot = (force_victim >= 0) ? force_victim : own;
+    *evicted_slot = slot;
+    *evicted_pos = pos[slot];
+  } else {
+    slot = (*live)++;
+  }
+  insert_token(K, V, s, q, n, pos, slot, d, k_new, v_new, t);
+  if (order == ROCO_ORACLE_EVICT_FIRST)
+    *lse = attend(K, V, s, q, n, *live, d, qv, scale, count_self ? -1 : slot, out, p);
+  *choice = own;
+  *near_tie = near;
+  *t_next = t + 1;
+  if (!p_out) free(p);
+}
+
+/* ------------------------------------------------- batch drivers (OpenMP) -- */
+
+void roco_oracle_decode_step_batch(int U, double *K, double *V, double *s, double *q, int *n, int *pos,
+                                   int *live, int *t_next, int B, int d, const double *qv,
+                                   const double *k_new, const double *v_new, int r, int mode, int order,
+                                   double scale, int count_self, double delta, const int *force_victim,
+                                   double *out, double *lse, int *evicted_slot, int *evicted_pos, int *choice,
+                                   int *near_tie) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int u = 0; u < U; ++u) {
+    size_t kb = (size_t)u * B * d, sb = (size_t)u * B, vb = (size_t)u * d;
+    roco_oracle_decode_step_unit(K + kb, V + kb, s + sb, q + sb, n + sb, pos + sb, live + u, t_next + u, B, d,
+                                 qv + vb, k_new + vb, v_new + vb, r, mode, order, scale, count_self, delta,
+                                 force_victim ? force_victim[u] : -1, out + vb, lse + u, evicted_slot + u,
+                                 evicted_pos + u, choice + u, near_tie + u, NULL);
+  }
+}
+
+/* Units may have different prompt lengths: unit u uses rows 0..lens[u]-1 of its [Lmax][d] block. */
+int roco_oracle_prefill_batch(int U, const double *Q, const double *K, const double *V, const int *lens,
+                              int Lmax, int d, int B, int r, int mode, double scale, int count_self,
+                              double delta, double *Kc, double *Vc, double *sc, double *qc, int *nc, int *posc,
+                              int *live, double *lse, double *s_full, double *q_full, int *n_full, int *keep_io,
+                              int force_keep, int *uncertain) {
+  int bad = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int u = 0; u < U; ++u) {
+    size_t ib = (size_t)u * Lmax * d, cb = (size_t)u * B * d, sb = (size_t)u * B, fb = (size_t)u * Lmax;
+    int rc = roco_oracle_prefill_unit(Q + ib, K + ib, V + ib, lens[u], d, B, r, mode, scale, count_self, delta,
+                                      Kc + cb, Vc + cb, sc + sb, qc + sb, nc + sb, posc + sb, live + u,
+                                      lse + fb, s_full + fb, q_full + fb, n_full + fb, keep_io + fb, force_keep,
+                                      uncertain ? uncertain + fb : NULL);
+    if (rc) {
+#pragma omp atomic write
+      bad = rc;
+    }
+  }
+  return bad;
+}
