@@ -1,0 +1,159 @@
+/*
+ * libroco -- KV-constrained attention with the RoCo eviction policy on one GPU (sm_100a).
+ *
+ * Notation follows the paper.  A *unit* is one (sequence, layer, head); units are independent
+ * (Fig. 1: heads evict at different positions).  d is the head dimension d', B the per-head token
+ * budget of Sec. 3 (the cache of a unit never holds more than B tokens), r the eviction-scope
+ * parameter of Sec. 4.2/4.3.  Per cached token the library keeps the three B-sized arrays of
+ * Sec. 4.3 -- Acc (s), Acc^square (q), Count (n) -- plus the token's original position (pos), which
+ * the paper's rule needs once heads have evicted at different positions and which breaks ties.
+ *
+ *     mean attention score  = s / n                         (Sec. 4.3, "MAS")
+ *     variance              = max(0, q / n - (s / n)^2)      (Sec. 4.3, Std formula; sqrt is monotone)
+ *     eviction scope        = the m lowest-variance cached tokens, order (variance, position):
+ *                             m = live - r  (EXCLUDE_TOP_R, Sec. 4.3: exclude the r highest-Std tokens)
+ *                             m = r         (LOWEST_R, Sec. 1: "tokens with the lowest variance")
+ *                             m is clipped to [1, live]
+ *     victim                = the in-scope token of lowest mean, order (mean, position)   (Sec. 4.3)
+ *
+ * Conventions for every entry point
+ *   - All array arguments are DEVICE pointers owned by the caller unless the name ends in _host.
+ *     The library allocates no device memory and keeps no state between calls.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls enqueue work
+ *     and return; outputs are valid once the stream reaches that point.  The *_host variants
+ *     synchronise the stream before returning.
+ *   - Argument errors are detected on the host before anything is launched and reported by the
+ *     return value; nothing throws or aborts.  Device-side anomalies (a wait that ran out, a
+ *     corrupt `live`) set bits in the caller-owned status word `roco_cache.status` and the kernel
+ *     returns normally; read it with roco_device_status().
+ *   - Q/K/V element type is roco_cache.kv_dtype (fp32 or bf16); statistics are fp32, counts int32.
+ *   - Supported shapes: d in {64, 128}; 1 <= B <= 8192; K, V, Q pointers 16-byte aligned.
+ */
+#ifndef ROCO_H_
+#define ROCO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ROCO_OK = 0,
+  ROCO_ERR_INVALID_ARG = 1, /* null/misaligned pointer, r or B out of range, bad lens          */
+  ROCO_ERR_UNSUPPORTED = 2, /* d, dtype, B or option outside what the kernels are built for     */
+  ROCO_ERR_WORKSPACE = 3,   /* workspace missing or smaller than roco_*_workspace_bytes()       */
+  ROCO_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch, copy)                        */
+  ROCO_ERR_STATE = 5        /* the device status word is non-zero                               */
+} roco_status;
+
+typedef enum { ROCO_F32 = 0, ROCO_BF16 = 1 } roco_dtype;
+
+typedef enum {
+  ROCO_SCOPE_EXCLUDE_TOP_R = 0, /* Sec. 4.3: scope = cached tokens minus the r of highest variance  */
+  ROCO_SCOPE_LOWEST_R = 1       /* Sec. 1:   scope = the r cached tokens of lowest variance         */
+} roco_scope_mode;
+
+typedef enum {
+  ROCO_EVICT_FIRST = 0, /* Fig. 1: evict, write the new K/V, then attend (the query sees its own key) */
+  ROCO_ATTEND_FIRST = 1 /* attend over the cache, update statistics, then evict and write the new K/V */
+} roco_step_order;
+
+/* Bits of the device status word. */
+enum {
+  ROCO_DEV_WAIT_TIMEOUT = 1, /* a bounded wait on a shared-memory barrier ran out */
+  ROCO_DEV_BAD_LIVE = 2,     /* live[u] outside [0, B]                            */
+  ROCO_DEV_BAD_VICTIM = 4    /* the selection produced no slot (NaN statistics)   */
+};
+
+/* The budgeted cache of Sec. 3/4 for S sequences x G (= layers*heads) units each; U = S*G.
+ * Slot order inside a unit is not position order once eviction has happened: pos[] says what a
+ * slot holds.  Slots live[u]..B-1 are empty (pos = -1). */
+typedef struct {
+  int32_t kv_dtype;  /* roco_dtype of K and V                                      */
+  int32_t S, G, d, B;
+  void *K, *V;       /* [S][G][B][d]                                               */
+  float *s, *q;      /* [S][G][B]   Acc and Acc^square                             */
+  int32_t *n, *pos;  /* [S][G][B]   Count; original position (-1 = empty slot)     */
+  int32_t *live;     /* [S][G]      occupied slots, always <= B                    */
+  int32_t *t_next;   /* [S][G]      position the next token of this unit will get  */
+  int32_t *status;   /* [1]         device status word, zeroed by the caller       */
+} roco_cache;
+
+/* Library version (major*100 + minor). */
+int roco_version(void);
+const char *roco_status_string(int st);
+
+/* Bytes of device workspace roco_prefill needs for prompts of up to Lmax tokens (host function). */
+size_t roco_prefill_workspace_bytes(const roco_cache *cache, int Lmax);
+
+/*
+ * Prefill with eviction to budget (Sec. 4.3 last paragraph; Sec. 5.1 "Other Details": the budget is
+ * fixed from the prompt length and eviction happens once, at the prefilling stage).
+ *
+ * For every unit: causal attention probabilities P (Eq. 1 with the mask of Sec. 2.1: row i sees
+ * keys 0..i), without storing P; column statistics n_j = lens - j, s_j = sum_i P_ij,
+ * q_j = sum_i P_ij^2 over rows i >= j; then, if lens > B, tokens are evicted down to B by applying
+ * the per-step rule lens - B times on these frozen statistics, and the survivors' K, V, s, q, n, pos
+ * are written to the cache in increasing position order.  live = min(lens, B); t_next = lens.
+ *
+ *   Q, K, V        [S][G][Lmax][d], cache->kv_dtype; rows >= lens_host[b] are ignored
+ *   lens_host      [S] HOST array, 1 <= lens <= Lmax (all units of a sequence share the length)
+ *   B              must equal cache->B;   r: 0 <= r <= B
+ *   scope_mode     ROCO_SCOPE_EXCLUDE_TOP_R (ROCO_SCOPE_LOWEST_R: ROCO_ERR_UNSUPPORTED when lens > B)
+ *   count_self     1: a token's own query counts towards its statistics (0: ROCO_ERR_UNSUPPORTED)
+ *   scale          multiplies Q.K (1/sqrt(d) in Eq. 1)
+ *   lse_out        [S][G][Lmax] row log-sum-exp, or NULL
+ *   s_full, q_full [S][G][Lmax] pre-eviction column statistics, or NULL
+ *   workspace      >= roco_prefill_workspace_bytes(cache, Lmax), 256-byte aligned
+ */
+roco_status roco_prefill(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax,
+                         int B, int r, int scope_mode, int count_self, float scale, roco_cache *cache,
+                         float *lse_out, float *s_full, float *q_full, void *workspace,
+                         size_t workspace_bytes, void *stream);
+
+/*
+ * One decode step for every unit (Sec. 3 constrained inference; Sec. 4 "when the buffer is full, an
+ * eviction policy is executed"; Sec. 4.3 RoCo rule; Fig. 1 ordering).
+ *
+ * EVICT_FIRST: if live == B the victim's slot is freed, else slot `live` is taken; the new token's
+ * K/V are written there with empty statistics and pos = t_next; the query attends over all occupied
+ * slots (Eq. 1); every occupied slot gets n += 1, s += p, q += p^2.  ATTEND_FIRST: attention and the
+ * statistics update run over the cache as it stands, then the eviction and the in-place write.
+ * The cache is never compacted: only the freed slot is overwritten.
+ *
+ *   q, k_new, v_new  [S][G][d], cache->kv_dtype
+ *   r                EXCLUDE_TOP_R: 0 <= r < B;  LOWEST_R: 1 <= r <= B
+ *   attn_out         [S][G][d], cache->kv_dtype
+ *   lse_out          [S][G] fp32 log-sum-exp of the scaled scores, or NULL
+ *   evicted_slot     [S][G] int32, -1 where nothing was evicted
+ *   evicted_pos      [S][G] int32 original position of the evicted token (-1 if none), or NULL
+ */
+roco_status roco_decode_step(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,
+                             int scope_mode, int step_order, float scale, void *attn_out, float *lse_out,
+                             int32_t *evicted_slot, int32_t *evicted_pos, void *stream);
+
+/* Bytes of device staging roco_decode_step_host needs (host function). */
+size_t roco_decode_host_staging_bytes(const roco_cache *cache);
+
+/*
+ * The same step for callers whose per-step tensors live in (pinned) HOST memory: copies q, k_new,
+ * v_new to `staging`, runs roco_decode_step, copies attn_out / evicted_slot / evicted_pos back and
+ * synchronises the stream.  The cache stays on the device.  *_host arguments are host pointers with
+ * the shapes above; evicted_pos_host may be NULL.  staging: device,
+ * >= roco_decode_host_staging_bytes(cache), 256-byte aligned.
+ */
+roco_status roco_decode_step_host(roco_cache *cache, const void *q_host, const void *k_new_host,
+                                  const void *v_new_host, int r, int scope_mode, int step_order, float scale,
+                                  void *attn_out_host, int32_t *evicted_slot_host, int32_t *evicted_pos_host,
+                                  void *staging, size_t staging_bytes, void *stream);
+
+/* Copies the device status word to *flags_host (synchronises the stream).  Returns ROCO_ERR_STATE
+ * when it is non-zero. */
+roco_status roco_device_status(const roco_cache *cache, void *stream, int32_t *flags_host);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ROCO_H_ */

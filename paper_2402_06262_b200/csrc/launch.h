@@ -1,0 +1,27 @@
+// Internal launch functions behind the C ABI (one per kernel family).  Arguments are validated by the
+// callers in api.cu; these only pick a template instance and enqueue.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "../../include/roco.h"
+
+namespace roco {
+
+roco_status launch_decode_step(const roco_cache &c, const void *q, const void *k_new, const void *v_new, int r,
+                               int scope_mode, int step_order, float scale, void *out, float *lse, int32_t *ev_slot,
+                               int32_t *ev_pos, cudaStream_t stream);
+
+// Row log-sum-exp and column statistics of the causal softmax, CUDA-core path (any supported dtype/d).
+// lens_dev: [S] device copy of the prompt lengths.  lse, s_full, q_full: [U][Lmax].
+roco_status launch_prefill_stats_simt(int kv_dtype, int d, int S, int G, int Lmax, const int *lens_dev, int maxlen,
+                                      const void *Q, const void *K, float scale, float *lse, float *s_full,
+                                      float *q_full, cudaStream_t stream);
+
+// Select-to-budget on frozen statistics and gather of the survivors into the cache.
+// dst: [U][Lmax] int32 scratch (destination slot per token, -1 = evicted).
+roco_status launch_budget_select_gather(const roco_cache &c, int Lmax, const int *lens_dev, int maxlen, int r,
+                                        const void *K, const void *V, const float *s_full, const float *q_full,
+                                        int *dst, cudaStream_t stream);
+
+}  // namespace roco

@@ -1,0 +1,147 @@
+// Per-unit eviction-scope construction and victim choice (Sec. 4.3), done by one thread group on
+// statistics that already sit in shared memory.
+//
+//   scope   = the m cached tokens first in (variance asc, position asc)
+//   victim  = the in-scope token first in (mean asc, position asc)
+//
+// The rank-m threshold comes from a most-significant-digit radix select over 32-bit keys (the variance
+// rounded to fp32, whose bit pattern orders like the value for non-negative floats); ties on the
+// threshold variance are resolved by a second radix select over the tied tokens' positions, only when
+// not all of them fit in the scope.  Mean and variance are formed in fp64 from the fp32 sums so that the
+// only error in the decision is the accumulated rounding of s and q themselves.
+#pragma once
+
+#include "common.cuh"
+
+namespace roco {
+
+struct SelectScratch {
+  uint32_t hist[256];
+  uint32_t digit, rank, count, pad;
+  double red_mean[32];
+  int red_pos[32];
+  int red_slot[32];
+};
+
+// k-th smallest (0-based) of key(j) over the j in [0, n) with pred(j); keys are unsigned integers of type
+// KeyT (32 or 64 bits).  Called by all `nthreads` threads that synchronise on named barrier `bar_id`.
+// *rank_in_ties: how many elements equal to the result precede the k-th in a stable order (so
+// rank_in_ties + 1 of them are among the k+1 smallest); *n_ties: how many elements equal the result.
+template <typename KeyT, typename KeyF, typename PredF>
+__device__ __forceinline__ KeyT radix_select(KeyF key, PredF pred, int n, uint32_t k, SelectScratch &sc, int tid,
+                                             int nthreads, int bar_id, uint32_t *rank_in_ties, uint32_t *n_ties) {
+  KeyT prefix = 0, mask = 0;
+  uint32_t kk = k;
+  const int lane = tid & 31;
+#pragma unroll 1
+  for (int shift = (int)sizeof(KeyT) * 8 - 8; shift >= 0; shift -= 8) {
+    for (int i = tid; i < 256; i += nthreads) sc.hist[i] = 0;
+    named_bar_sync(bar_id, nthreads);
+    for (int j = tid; j < n; j += nthreads) {
+      if (pred(j)) {
+        KeyT x = key(j);
+        if ((x & mask) == prefix) atomicAdd(&sc.hist[(uint32_t)(x >> shift) & 255u], 1u);
+      }
+    }
+    named_bar_sync(bar_id, nthreads);
+    if (tid < 32) {
+      uint32_t c[8], total = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { c[i] = sc.hist[lane * 8 + i]; total += c[i]; }
+      uint32_t incl = total;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      uint32_t excl = incl - total;
+      if (kk >= excl && kk < incl) {
+        uint32_t rem = kk - excl;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (rem < c[i]) { sc.digit = lane * 8 + i; sc.rank = rem; sc.count = c[i]; break; }
+          rem -= c[i];
+        }
+      }
+    }
+    named_bar_sync(bar_id, nthreads);
+    prefix |= (KeyT)sc.digit << shift;
+    mask |= (KeyT)255u << shift;
+    kk = sc.rank;
+  }
+  *rank_in_ties = kk;
+  *n_ties = sc.count;
+  named_bar_sync(bar_id, nthreads);  // sc.* may be reused by the caller right away
+  return prefix;
+}
+
+__device__ __forceinline__ double mean_f64(float s, int n) { return (double)s / (double)n; }
+
+__device__ __forceinline__ double variance_f64(float s, float q, int n) {
+  double mean = (double)s / (double)n;
+  double var = (double)q / (double)n - mean * mean;
+  return fmax(var, 0.0);  // also maps NaN to 0
+}
+
+__device__ __forceinline__ uint32_t variance_key(float s, float q, int n) {
+  return __float_as_uint((float)variance_f64(s, q, n));
+}
+
+// Victim slot among slots [0, live) given scope size m (1 <= m <= live).  s, q, n, pos and vkey are
+// shared-memory arrays; vkey[live] is scratch.  Returns -1 if no slot qualifies (NaN statistics).
+// Every one of the `nthreads` threads gets the same return value.
+__device__ __forceinline__ int block_select_victim(const float *s, const float *q, const int *n, const int *pos,
+                                                   int live, int m, uint32_t *vkey, SelectScratch &sc, int tid,
+                                                   int nthreads, int bar_id) {
+  for (int j = tid; j < live; j += nthreads) vkey[j] = variance_key(s[j], q[j], n[j]);
+  named_bar_sync(bar_id, nthreads);
+  uint32_t T = 0xffffffffu;
+  int P = 0x7fffffff;
+  if (m < live) {
+    uint32_t rank, ties;
+    T = radix_select<uint32_t>([&](int j) { return vkey[j]; }, [&](int) { return true; }, live, (uint32_t)(m - 1),
+                               sc, tid, nthreads, bar_id, &rank, &ties);
+    if (ties != rank + 1) {  // only some of the tokens tied at the threshold are in scope: lowest positions
+      uint32_t r2, t2;
+      P = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)pos[j]; }, [&](int j) { return vkey[j] == T; },
+                                      live, rank, sc, tid, nthreads, bar_id, &r2, &t2);
+    }
+  }
+  double bm = INFINITY;
+  int bp = 0x7fffffff, bs = -1;
+  for (int j = tid; j < live; j += nthreads) {
+    uint32_t k = vkey[j];
+    bool in_scope = (k < T) || (k == T && pos[j] <= P);
+    if (!in_scope) continue;
+    double mean = mean_f64(s[j], n[j]);
+    if (mean < bm || (mean == bm && pos[j] < bp)) { bm = mean; bp = pos[j]; bs = j; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    double om = __shfl_xor_sync(0xffffffffu, bm, o);
+    int op = __shfl_xor_sync(0xffffffffu, bp, o);
+    int os = __shfl_xor_sync(0xffffffffu, bs, o);
+    if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+  }
+  const int warp = tid >> 5, nwarps = nthreads >> 5;
+  if ((tid & 31) == 0) { sc.red_mean[warp] = bm; sc.red_pos[warp] = bp; sc.red_slot[warp] = bs; }
+  named_bar_sync(bar_id, nthreads);
+  bm = sc.red_mean[0]; bp = sc.red_pos[0]; bs = sc.red_slot[0];
+  for (int w = 1; w < nwarps; ++w) {
+    double om = sc.red_mean[w];
+    int op = sc.red_pos[w], os = sc.red_slot[w];
+    if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+  }
+  named_bar_sync(bar_id, nthreads);
+  return bs;
+}
+
+// Scope size for `live` cached tokens (Sec. 4.3 / Sec. 1 readings), clipped to [1, live].
+__device__ __host__ __forceinline__ int scope_size(int live, int r, int scope_mode) {
+  int m = (scope_mode == ROCO_SCOPE_EXCLUDE_TOP_R) ? live - r : r;
+  if (m < 1) m = 1;
+  if (m > live) m = live;
+  return m;
+}
+
+}  // namespace roco
