@@ -1,0 +1,166 @@
+// The C ABI of libroco: argument validation on the host, workspace carving, launches.
+#include <cstring>
+
+#include "common.cuh"
+#include "launch.h"
+
+using namespace roco;
+
+namespace {
+
+constexpr int kMaxB = 8192;
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+roco_status check_cache(const roco_cache *c) {
+  if (!c) return ROCO_ERR_INVALID_ARG;
+  if (!c->K || !c->V || !c->s || !c->q || !c->n || !c->pos || !c->live || !c->t_next || !c->status)
+    return ROCO_ERR_INVALID_ARG;
+  if (c->S < 1 || c->G < 1 || c->B < 1) return ROCO_ERR_INVALID_ARG;
+  if (!aligned16(c->K) || !aligned16(c->V)) return ROCO_ERR_INVALID_ARG;
+  if (c->kv_dtype != ROCO_F32 && c->kv_dtype != ROCO_BF16) return ROCO_ERR_UNSUPPORTED;
+  if (c->d != 64 && c->d != 128) return ROCO_ERR_UNSUPPORTED;
+  if (c->B > kMaxB) return ROCO_ERR_UNSUPPORTED;
+  if ((long long)c->S * c->G > 0x7fffffffLL / 64) return ROCO_ERR_UNSUPPORTED;
+  return ROCO_OK;
+}
+
+roco_status check_scope(int r, int scope_mode, int B, bool decode) {
+  if (scope_mode == ROCO_SCOPE_EXCLUDE_TOP_R) return (r >= 0 && (decode ? r < B : r <= B)) ? ROCO_OK : ROCO_ERR_INVALID_ARG;
+  if (scope_mode == ROCO_SCOPE_LOWEST_R) return (r >= 1 && r <= B) ? ROCO_OK : ROCO_ERR_INVALID_ARG;
+  return ROCO_ERR_INVALID_ARG;
+}
+
+struct PrefillWs {
+  size_t lens_off, lse_off, s_off, q_off, dst_off, total;
+};
+
+PrefillWs prefill_ws(int S, int G, int Lmax) {
+  PrefillWs w;
+  const size_t per = align_up((size_t)S * G * (size_t)Lmax * 4, 256);
+  w.lens_off = 0;
+  w.lse_off = align_up((size_t)S * 4, 256);
+  w.s_off = w.lse_off + per;
+  w.q_off = w.s_off + per;
+  w.dst_off = w.q_off + per;
+  w.total = w.dst_off + per;
+  return w;
+}
+
+}  // namespace
+
+extern "C" {
+
+int roco_version(void) { return 100; }
+
+const char *roco_status_string(int st) {
+  switch (st) {
+    case ROCO_OK: return "ok";
+    case ROCO_ERR_INVALID_ARG: return "invalid argument";
+    case ROCO_ERR_UNSUPPORTED: return "unsupported shape, dtype or option";
+    case ROCO_ERR_WORKSPACE: return "workspace missing or too small";
+    case ROCO_ERR_CUDA: return "CUDA runtime error";
+    case ROCO_ERR_STATE: return "device status word is set";
+    default: return "unknown status";
+  }
+}
+
+size_t roco_prefill_workspace_bytes(const roco_cache *cache, int Lmax) {
+  if (!cache || Lmax < 1 || cache->S < 1 || cache->G < 1) return 0;
+  return prefill_ws(cache->S, cache->G, Lmax).total;
+}
+
+roco_status roco_prefill(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax, int B,
+                         int r, int scope_mode, int count_self, float scale, roco_cache *cache, float *lse_out,
+                         float *s_full, float *q_full, void *workspace, size_t workspace_bytes, void *stream) {
+  roco_status st = check_cache(cache);
+  if (st != ROCO_OK) return st;
+  if (!Q || !K || !V || !lens_host || Lmax < 1 || B != cache->B) return ROCO_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V)) return ROCO_ERR_INVALID_ARG;
+  if ((st = check_scope(r, scope_mode, B, false)) != ROCO_OK) return st;
+  if (count_self != 1) return ROCO_ERR_UNSUPPORTED;
+  int maxlen = 0;
+  for (int b = 0; b < cache->S; ++b) {
+    if (lens_host[b] < 1 || lens_host[b] > Lmax) return ROCO_ERR_INVALID_ARG;
+    if (lens_host[b] > maxlen) maxlen = lens_host[b];
+  }
+  if (scope_mode == ROCO_SCOPE_LOWEST_R && maxlen > B) return ROCO_ERR_UNSUPPORTED;
+  if ((long long)cache->S * cache->G * ((maxlen + 63) / 64 + 1) > 0x7fffffffLL) return ROCO_ERR_UNSUPPORTED;
+  const PrefillWs w = prefill_ws(cache->S, cache->G, Lmax);
+  if (!workspace || workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return ROCO_ERR_WORKSPACE;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  char *ws = static_cast<char *>(workspace);
+  int *lens_dev = reinterpret_cast<int *>(ws + w.lens_off);
+  float *lse = lse_out ? lse_out : reinterpret_cast<float *>(ws + w.lse_off);
+  float *sf = s_full ? s_full : reinterpret_cast<float *>(ws + w.s_off);
+  float *qf = q_full ? q_full : reinterpret_cast<float *>(ws + w.q_off);
+  int *dst = reinterpret_cast<int *>(ws + w.dst_off);
+  if (cudaMemcpyAsync(lens_dev, lens_host, (size_t)cache->S * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess)
+    return ROCO_ERR_CUDA;
+  st = launch_prefill_stats_simt(cache->kv_dtype, cache->d, cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, scale,
+                                 lse, sf, qf, cs);
+  if (st != ROCO_OK) return st;
+  return launch_budget_select_gather(*cache, Lmax, lens_dev, maxlen, r, K, V, sf, qf, dst, cs);
+}
+
+roco_status roco_decode_step(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,
+                             int scope_mode, int step_order, float scale, void *attn_out, float *lse_out,
+                             int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {
+  roco_status st = check_cache(cache);
+  if (st != ROCO_OK) return st;
+  if (!q || !k_new || !v_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
+  if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
+  if (step_order != ROCO_EVICT_FIRST && step_order != ROCO_ATTEND_FIRST) return ROCO_ERR_INVALID_ARG;
+  return launch_decode_step(*cache, q, k_new, v_new, r, scope_mode, step_order, scale, attn_out, lse_out,
+                            evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
+}
+
+size_t roco_decode_host_staging_bytes(const roco_cache *cache) {
+  if (!cache || cache->S < 1 || cache->G < 1) return 0;
+  const size_t U = (size_t)cache->S * cache->G;
+  const size_t vec = align_up(U * cache->d * (cache->kv_dtype == ROCO_BF16 ? 2 : 4), 256);
+  return 4 * vec + 2 * align_up(U * 4, 256);
+}
+
+roco_status roco_decode_step_host(roco_cache *cache, const void *q_host, const void *k_new_host,
+                                  const void *v_new_host, int r, int scope_mode, int step_order, float scale,
+                                  void *attn_out_host, int32_t *evicted_slot_host, int32_t *evicted_pos_host,
+                                  void *staging, size_t staging_bytes, void *stream) {
+  roco_status st = check_cache(cache);
+  if (st != ROCO_OK) return st;
+  if (!q_host || !k_new_host || !v_new_host || !attn_out_host || !evicted_slot_host) return ROCO_ERR_INVALID_ARG;
+  if (!staging || staging_bytes < roco_decode_host_staging_bytes(cache) ||
+      (reinterpret_cast<uintptr_t>(staging) & 255u))
+    return ROCO_ERR_WORKSPACE;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const size_t U = (size_t)cache->S * cache->G;
+  const size_t vbytes = U * cache->d * (cache->kv_dtype == ROCO_BF16 ? 2 : 4);
+  const size_t vec = align_up(vbytes, 256), ivec = align_up(U * 4, 256);
+  char *p = static_cast<char *>(staging);
+  char *dq = p, *dk = p + vec, *dv = p + 2 * vec, *dout = p + 3 * vec;
+  int32_t *dslot = reinterpret_cast<int32_t *>(p + 4 * vec), *dpos = reinterpret_cast<int32_t *>(p + 4 * vec + ivec);
+  if (cudaMemcpyAsync(dq, q_host, vbytes, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+      cudaMemcpyAsync(dk, k_new_host, vbytes, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+      cudaMemcpyAsync(dv, v_new_host, vbytes, cudaMemcpyHostToDevice, cs) != cudaSuccess)
+    return ROCO_ERR_CUDA;
+  st = roco_decode_step(cache, dq, dk, dv, r, scope_mode, step_order, scale, dout, nullptr, dslot, dpos, stream);
+  if (st != ROCO_OK) return st;
+  if (cudaMemcpyAsync(attn_out_host, dout, vbytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
+      cudaMemcpyAsync(evicted_slot_host, dslot, U * 4, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+    return ROCO_ERR_CUDA;
+  if (evicted_pos_host && cudaMemcpyAsync(evicted_pos_host, dpos, U * 4, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+    return ROCO_ERR_CUDA;
+  return cudaStreamSynchronize(cs) == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
+}
+
+roco_status roco_device_status(const roco_cache *cache, void *stream, int32_t *flags_host) {
+  if (!cache || !cache->status || !flags_host) return ROCO_ERR_INVALID_ARG;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(flags_host, cache->status, 4, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return ROCO_ERR_CUDA;
+  if (cudaStreamSynchronize(cs) != cudaSuccess) return ROCO_ERR_CUDA;
+  return *flags_host ? ROCO_ERR_STATE : ROCO_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,148 @@
+// Prefill-stage eviction to budget (Sec. 4.3 last paragraph, Sec. 5.1 "Other Details") on frozen column
+// statistics, then the gather of the survivors into the cache in increasing position order.
+//
+// Under EXCLUDE_TOP_R, applying the per-step rule L-B times on frozen statistics equals one pass: the r
+// tokens last in (variance, position) order are never in scope, so the scope's complement never changes;
+// of the other tokens the L-B first in (mean, position) order leave.  Both thresholds come from radix
+// selects over the fp64 bit patterns of variance and mean (non-negative doubles order like their bits).
+#include "common.cuh"
+#include "launch.h"
+#include "select.cuh"
+
+namespace roco {
+
+constexpr int kBudgetThreads = 512;
+constexpr int kBarAll = 1;
+
+// One CTA per unit.  dst[u][j] = cache slot of token j, or -1 if it is evicted.
+__global__ void __launch_bounds__(kBudgetThreads) budget_select_kernel(const float *s_full, const float *q_full,
+                                                                       const int *lens, int G, int Lmax, int B, int r,
+                                                                       int *dst, int *live, int *t_next) {
+  __shared__ SelectScratch sc;
+  __shared__ int warp_tot[kBudgetThreads / 32];
+  __shared__ int base_sh;
+  const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int L = lens[u / G];
+  const float *s = s_full + (size_t)u * Lmax, *q = q_full + (size_t)u * Lmax;
+  int *du = dst + (size_t)u * Lmax;
+  if (tid == 0) { live[u] = L < B ? L : B; t_next[u] = L; }
+  if (L <= B) {
+    for (int j = tid; j < L; j += kBudgetThreads) du[j] = j;
+    return;
+  }
+  const int E = L - B;  // tokens to evict
+  auto vkey = [&](int j) { return (uint64_t)__double_as_longlong(variance_f64(s[j], q[j], L - j)); };
+  auto mkey = [&](int j) { return (uint64_t)__double_as_longlong(mean_f64(s[j], L - j)); };
+  uint64_t Tv = ~0ull;
+  int Pv = 0x7fffffff;
+  if (r > 0) {  // the L-r tokens first in (variance, position) order may be evicted
+    uint32_t rank, ties;
+    Tv = radix_select<uint64_t>(vkey, [&](int) { return true; }, L, (uint32_t)(L - r - 1), sc, tid, kBudgetThreads,
+                                kBarAll, &rank, &ties);
+    if (ties != rank + 1) {
+      uint32_t r2, t2;
+      Pv = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)j; }, [&](int j) { return vkey(j) == Tv; }, L,
+                                       rank, sc, tid, kBudgetThreads, kBarAll, &r2, &t2);
+    }
+  }
+  auto unprot = [&](int j) {
+    if (r == 0) return true;
+    const uint64_t k = vkey(j);
+    return k < Tv || (k == Tv && j <= Pv);
+  };
+  uint32_t rank, ties;
+  const uint64_t Tm = radix_select<uint64_t>(mkey, unprot, L, (uint32_t)(E - 1), sc, tid, kBudgetThreads, kBarAll,
+                                             &rank, &ties);
+  int Pm = 0x7fffffff;
+  if (ties != rank + 1) {
+    uint32_t r2, t2;
+    Pm = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)j; },
+                                     [&](int j) { return unprot(j) && mkey(j) == Tm; }, L, rank, sc, tid,
+                                     kBudgetThreads, kBarAll, &r2, &t2);
+  }
+  // survivors keep their order: exclusive prefix sum of the keep flags
+  if (tid == 0) base_sh = 0;
+  __syncthreads();
+  for (int j0 = 0; j0 < L; j0 += kBudgetThreads) {
+    const int j = j0 + tid;
+    bool keep = false;
+    if (j < L) {
+      const uint64_t k = mkey(j);
+      keep = !(unprot(j) && (k < Tm || (k == Tm && j <= Pm)));
+    }
+    const uint32_t bal = __ballot_sync(0xffffffffu, keep);
+    const int before = __popc(bal & ((1u << lane) - 1u));
+    if (lane == 0) warp_tot[warp] = __popc(bal);
+    __syncthreads();
+    int off = base_sh;
+    for (int w = 0; w < warp; ++w) off += warp_tot[w];
+    if (j < L) du[j] = keep ? off + before : -1;
+    __syncthreads();
+    if (tid == 0) {
+      int t = 0;
+      for (int w = 0; w < kBudgetThreads / 32; ++w) t += warp_tot[w];
+      base_sh += t;
+    }
+    __syncthreads();
+  }
+}
+
+// grid U * chunks (unit-major); each CTA moves up to 64 tokens.  Also clears the slots past `live`.
+template <int ROWB>
+__global__ void __launch_bounds__(256) gather_kernel(const char *K, const char *V, const float *s_full,
+                                                     const float *q_full, const int *dst, const int *lens, int G,
+                                                     int Lmax, int B, int chunks, char *Kc, char *Vc, float *sc,
+                                                     float *qc, int *nc, int *posc) {
+  constexpr int kChunksPerRow = ROWB / 16;
+  const int u = blockIdx.x / chunks, c0 = (int)(blockIdx.x % chunks) * 64;
+  const int L = lens[u / G], tid = threadIdx.x;
+  const int live = L < B ? L : B;
+  const size_t in_off = (size_t)u * Lmax, out_off = (size_t)u * B;
+  for (int w = tid; w < 64 * 2 * kChunksPerRow; w += 256) {
+    const int k = w / (2 * kChunksPerRow), rem = w % (2 * kChunksPerRow);
+    const int j = c0 + k;
+    if (j >= L) continue;
+    const int slot = dst[in_off + j];
+    if (slot < 0) continue;
+    const bool isv = rem >= kChunksPerRow;
+    const int c = isv ? rem - kChunksPerRow : rem;
+    const uint4 val = *((const uint4 *)((isv ? V : K) + (in_off + j) * ROWB) + c);
+    *((uint4 *)((isv ? Vc : Kc) + (out_off + slot) * ROWB) + c) = val;
+  }
+  if (tid < 64) {
+    const int j = c0 + tid;
+    if (j < L) {
+      const int slot = dst[in_off + j];
+      if (slot >= 0) {
+        sc[out_off + slot] = s_full[in_off + j];
+        qc[out_off + slot] = q_full[in_off + j];
+        nc[out_off + slot] = L - j;  // Count: queries j..L-1 have attended token j
+        posc[out_off + slot] = j;
+      }
+    }
+    if (j >= live && j < B) { sc[out_off + j] = 0.f; qc[out_off + j] = 0.f; nc[out_off + j] = 0; posc[out_off + j] = -1; }
+  }
+}
+
+roco_status launch_budget_select_gather(const roco_cache &c, int Lmax, const int *lens_dev, int maxlen, int r,
+                                        const void *K, const void *V, const float *s_full, const float *q_full,
+                                        int *dst, cudaStream_t stream) {
+  const int U = c.S * c.G;
+  budget_select_kernel<<<U, kBudgetThreads, 0, stream>>>(s_full, q_full, lens_dev, c.G, Lmax, c.B, r, dst, c.live,
+                                                         c.t_next);
+  const int span = maxlen > c.B ? maxlen : c.B;
+  const int chunks = (span + 63) / 64;
+  const unsigned grid = (unsigned)U * (unsigned)chunks;
+  const int rowb = c.d * (c.kv_dtype == ROCO_BF16 ? 2 : 4);
+#define ROCO_GATHER(RB)                                                                                         \
+  gather_kernel<RB><<<grid, 256, 0, stream>>>((const char *)K, (const char *)V, s_full, q_full, dst, lens_dev, c.G, \
+                                              Lmax, c.B, chunks, (char *)c.K, (char *)c.V, c.s, c.q, c.n, c.pos)
+  if (rowb == 128) ROCO_GATHER(128);
+  else if (rowb == 256) ROCO_GATHER(256);
+  else if (rowb == 512) ROCO_GATHER(512);
+  else return ROCO_ERR_UNSUPPORTED;
+#undef ROCO_GATHER
+  return cudaGetLastError() == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
+}
+
+}  // namespace roco

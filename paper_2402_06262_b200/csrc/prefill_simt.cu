@@ -40,14 +40,14 @@ __device__ __forceinline__ void score_tile(const float *Qs, const float *Ks, int
   }
 }
 
-// grid (row tiles, U).  lse[u][i] = log sum_{j<=i} exp(scale * Q_i.K_j)
+// grid U * tiles, unit-major; heavy (late) row tiles first.  lse[u][i] = log sum_{j<=i} exp(scale * Q_i.K_j)
 template <typename T, int D>
 __global__ void __launch_bounds__(kPThreads) prefill_lse_kernel(const T *Q, const T *K, const int *lens, int G,
-                                                                int Lmax, float scale, float *lse) {
+                                                                int Lmax, int tiles, float scale, float *lse) {
   extern __shared__ float psm[];
   float *Qs = psm, *Ks = psm + kPT * (D + 1);
-  const int u = blockIdx.y, L = lens[u / G];
-  const int row0 = blockIdx.x * kPT;
+  const int u = blockIdx.x / tiles, L = lens[u / G];
+  const int row0 = (tiles - 1 - (int)(blockIdx.x % tiles)) * kPT;
   if (row0 >= L) return;
   const int tid = threadIdx.x, ty = tid / 16, tx = tid % 16;
   const T *Qu = Q + (size_t)u * Lmax * D, *Ku = K + (size_t)u * Lmax * D;
@@ -95,15 +95,15 @@ __global__ void __launch_bounds__(kPThreads) prefill_lse_kernel(const T *Q, cons
   }
 }
 
-// grid (column tiles, U).  s[u][j] = sum_{i>=j} P_ij, q[u][j] = sum_{i>=j} P_ij^2 with P_ij = exp(z_ij - lse_i)
+// grid U * tiles, unit-major; heavy (early) column tiles first.  s[u][j] = sum_{i>=j} P_ij, q[u][j] = sum_{i>=j} P_ij^2 with P_ij = exp(z_ij - lse_i)
 template <typename T, int D>
 __global__ void __launch_bounds__(kPThreads) prefill_colstats_kernel(const T *Q, const T *K, const int *lens, int G,
-                                                                     int Lmax, float scale, const float *lse,
+                                                                     int Lmax, int tiles, float scale, const float *lse,
                                                                      float *s_full, float *q_full) {
   extern __shared__ float psm[];
   float *Qs = psm, *Ks = psm + kPT * (D + 1), *lse2 = Ks + kPT * (D + 1), *red = lse2 + kPT;
-  const int u = blockIdx.y, L = lens[u / G];
-  const int col0 = blockIdx.x * kPT;
+  const int u = blockIdx.x / tiles, L = lens[u / G];
+  const int col0 = (int)(blockIdx.x % tiles) * kPT;
   if (col0 >= L) return;
   const int tid = threadIdx.x, ty = tid / 16, tx = tid % 16;
   const T *Qu = Q + (size_t)u * Lmax * D, *Ku = K + (size_t)u * Lmax * D;
@@ -163,10 +163,12 @@ static cudaError_t launch_t(int S, int G, int Lmax, const int *lens, int maxlen,
   err = cudaFuncSetAttribute(prefill_colstats_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem2);
   if (err != cudaSuccess) return err;
-  dim3 grid((maxlen + kPT - 1) / kPT, S * G);
-  prefill_lse_kernel<T, D><<<grid, kPThreads, smem1, stream>>>((const T *)Q, (const T *)K, lens, G, Lmax, scale, lse);
-  prefill_colstats_kernel<T, D><<<grid, kPThreads, smem2, stream>>>((const T *)Q, (const T *)K, lens, G, Lmax, scale,
-                                                                    lse, s_full, q_full);
+  const int tiles = (maxlen + kPT - 1) / kPT;
+  const unsigned grid = (unsigned)(S * G) * (unsigned)tiles;
+  prefill_lse_kernel<T, D><<<grid, kPThreads, smem1, stream>>>((const T *)Q, (const T *)K, lens, G, Lmax, tiles, scale,
+                                                               lse);
+  prefill_colstats_kernel<T, D><<<grid, kPThreads, smem2, stream>>>((const T *)Q, (const T *)K, lens, G, Lmax, tiles,
+                                                                    scale, lse, s_full, q_full);
   return cudaGetLastError();
 }
 
