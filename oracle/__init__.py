@@ -158,8 +158,9 @@ class StepResult:
 
 
 def decode_step(st: State, qv, k_new, v_new, r, mode, order, scale, count_self=1, delta=1e-5,
-                force_victim: Optional[np.ndarray] = None) -> StepResult:
-    """One decode step of every unit, in place on `st`.  qv, k_new, v_new: [U][d]."""
+                force_victim: Optional[np.ndarray] = None, force_only_near: bool = False) -> StepResult:
+    """One decode step of every unit, in place on `st`.  qv, k_new, v_new: [U][d].
+    force_victim[u] >= 0 replaces the policy's victim (only at near-ties if force_only_near)."""
     qv, k_new, v_new = _f64(qv), _f64(k_new), _f64(v_new)
     U, B, d = st.U, st.B, st.d
     out = np.zeros((U, d)); lse = np.zeros(U)
@@ -168,6 +169,6 @@ def decode_step(st: State, qv, k_new, v_new, r, mode, order, scale, count_self=1
     lib().roco_oracle_decode_step_batch(C.c_int(U), _p(st.K), _p(st.V), _p(st.s), _p(st.q), _p(st.n), _p(st.pos),
                                         _p(st.live), _p(st.t_next), C.c_int(B), C.c_int(d), _p(qv), _p(k_new),
                                         _p(v_new), C.c_int(r), C.c_int(mode), C.c_int(order), C.c_double(scale),
-                                        C.c_int(count_self), C.c_double(delta), _p(fv), _p(out), _p(lse), _p(es),
+                                        C.c_int(count_self), C.c_double(delta), _p(fv), C.c_int(int(force_only_near)), _p(out), _p(lse), _p(es),
                                         _p(ep), _p(ch), _p(nt))
     return StepResult(out, lse, es, ep, ch, nt.astype(bool))

@@ -338,15 +338,16 @@ static double attend(const double *K, const double *V, double *s, double *q, int
 
 /* One decode step of one unit.  Cache K,V [B][d]; s,q [B]; n,pos [B]; *live; *t_next = position of the
  * new token (incremented on return).  force_victim >= 0 replaces the policy's choice when the buffer is
- * full (used to continue from a common state after a logged near-tie).
+ * full (used to continue from a common state after a logged near-tie); with force_only_near != 0 it does
+ * so only at steps the margin analysis flags as near-ties.
  * Outputs: out [d]; *lse; *evicted_slot (-1 when nothing was evicted); *evicted_pos; *choice = the
  * policy's own victim (-1 if none); *near_tie.  p_out [B] may be NULL. */
 void roco_oracle_decode_step_unit(double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
                                   int *t_next, int B, int d, const double *qv, const double *k_new,
                                   const double *v_new, int r, int mode, int order, double scale,
-                                  int count_self, double delta, int force_victim, double *out, double *lse,
-                                  int *evicted_slot, int *evicted_pos, int *choice, int *near_tie,
-                                  double *p_out) {
+                                  int count_self, double delta, int force_victim, int force_only_near,
+                                  double *out, double *lse, int *evicted_slot, int *evicted_pos, int *choice,
+                                  int *near_tie, double *p_out) {
   double *p = p_out ? p_out : (double *)malloc(sizeof(double) * (size_t)B);
   int t = *t_next, slot, near = 0, own = -1;
   *evicted_slot = -1;
@@ -355,7 +356,7 @@ void roco_oracle_decode_step_unit(double *K, double *V, double *s, double *q, in
     *lse = attend(K, V, s, q, n, *live, d, qv, scale, -1, out, p); /* the new token is not in the cache yet */
   if (*live == B) { /* buffer full: run the policy (Sec. 4) */
     own = roco_oracle_select(s, q, n, pos, *live, r, mode, delta, &near, NULL);
-    slot = (force_victim >= 0) ? force_victim : own;
+    slot = (force_victim >= 0 && force_victim < B && (near || !force_only_near)) ? force_victim : own;
     *evicted_slot = slot;
     *evicted_pos = pos[slot];
   } else {
@@ -376,15 +377,15 @@ void roco_oracle_decode_step_batch(int U, double *K, double *V, double *s, doubl
                                    int *live, int *t_next, int B, int d, const double *qv,
                                    const double *k_new, const double *v_new, int r, int mode, int order,
                                    double scale, int count_self, double delta, const int *force_victim,
-                                   double *out, double *lse, int *evicted_slot, int *evicted_pos, int *choice,
-                                   int *near_tie) {
+                                   int force_only_near, double *out, double *lse, int *evicted_slot,
+                                   int *evicted_pos, int *choice, int *near_tie) {
 #pragma omp parallel for schedule(dynamic, 1)
   for (int u = 0; u < U; ++u) {
     size_t kb = (size_t)u * B * d, sb = (size_t)u * B, vb = (size_t)u * d;
     roco_oracle_decode_step_unit(K + kb, V + kb, s + sb, q + sb, n + sb, pos + sb, live + u, t_next + u, B, d,
                                  qv + vb, k_new + vb, v_new + vb, r, mode, order, scale, count_self, delta,
-                                 force_victim ? force_victim[u] : -1, out + vb, lse + u, evicted_slot + u,
-                                 evicted_pos + u, choice + u, near_tie + u, NULL);
+                                 force_victim ? force_victim[u] : -1, force_only_near, out + vb, lse + u,
+                                 evicted_slot + u, evicted_pos + u, choice + u, near_tie + u, NULL);
   }
 }
 

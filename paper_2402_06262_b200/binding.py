@@ -1,0 +1,161 @@
+"""ctypes binding of libroco's C ABI (argument marshalling only; every step runs in the CUDA kernels).
+
+PyTorch is used for device memory and streams.  There is no CPU path: loading fails loudly when the
+compiled library is missing.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libroco.so")
+
+ROCO_OK = 0
+ROCO_F32, ROCO_BF16 = 0, 1
+ROCO_SCOPE_EXCLUDE_TOP_R, ROCO_SCOPE_LOWEST_R = 0, 1
+ROCO_EVICT_FIRST, ROCO_ATTEND_FIRST = 0, 1
+
+EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes", "roco_prefill",
+           "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status")
+
+
+class RocoError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: status {code} ({status_string(code)})")
+        self.code = code
+
+
+class roco_cache(C.Structure):
+    _fields_ = [("kv_dtype", C.c_int32), ("S", C.c_int32), ("G", C.c_int32), ("d", C.c_int32), ("B", C.c_int32),
+                ("K", C.c_void_p), ("V", C.c_void_p), ("s", C.c_void_p), ("q", C.c_void_p),
+                ("n", C.c_void_p), ("pos", C.c_void_p), ("live", C.c_void_p), ("t_next", C.c_void_p),
+                ("status", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2402_06262_b200.build` "
+                               "(there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        L.roco_version.restype = C.c_int
+        L.roco_status_string.restype = C.c_char_p
+        L.roco_status_string.argtypes = [C.c_int]
+        L.roco_prefill_workspace_bytes.restype = C.c_size_t
+        L.roco_prefill_workspace_bytes.argtypes = [C.POINTER(roco_cache), C.c_int]
+        L.roco_decode_host_staging_bytes.restype = C.c_size_t
+        L.roco_decode_host_staging_bytes.argtypes = [C.POINTER(roco_cache)]
+        L.roco_prefill.restype = C.c_int
+        L.roco_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
+                                   C.c_int, C.c_float, C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p,
+                                   C.c_void_p, C.c_size_t, C.c_void_p]
+        L.roco_decode_step.restype = C.c_int
+        L.roco_decode_step.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                       C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.roco_decode_step_host.restype = C.c_int
+        L.roco_decode_step_host.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                            C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
+                                            C.c_void_p, C.c_size_t, C.c_void_p]
+        L.roco_device_status.restype = C.c_int
+        L.roco_device_status.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().roco_status_string(int(code)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Cache:
+    """Device tensors of the budgeted cache for S sequences x G units, plus the C struct over them."""
+
+    def __init__(self, S: int, G: int, B: int, d: int, dtype: torch.dtype, device="cuda"):
+        assert dtype in (torch.float32, torch.bfloat16)
+        self.S, self.G, self.B, self.d, self.dtype = S, G, B, d, dtype
+        self.K = torch.zeros(S, G, B, d, dtype=dtype, device=device)
+        self.V = torch.zeros(S, G, B, d, dtype=dtype, device=device)
+        self.s = torch.zeros(S, G, B, dtype=torch.float32, device=device)
+        self.q = torch.zeros(S, G, B, dtype=torch.float32, device=device)
+        self.n = torch.zeros(S, G, B, dtype=torch.int32, device=device)
+        self.pos = torch.full((S, G, B), -1, dtype=torch.int32, device=device)
+        self.live = torch.zeros(S, G, dtype=torch.int32, device=device)
+        self.t_next = torch.zeros(S, G, dtype=torch.int32, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.c = roco_cache(ROCO_F32 if dtype == torch.float32 else ROCO_BF16, S, G, d, B,
+                            self.K.data_ptr(), self.V.data_ptr(), self.s.data_ptr(), self.q.data_ptr(),
+                            self.n.data_ptr(), self.pos.data_ptr(), self.live.data_ptr(), self.t_next.data_ptr(),
+                            self.status.data_ptr())
+
+    @property
+    def U(self) -> int:
+        return self.S * self.G
+
+
+def roco_prefill_workspace_bytes(cache: Cache, Lmax: int) -> int:
+    return int(lib().roco_prefill_workspace_bytes(C.byref(cache.c), Lmax))
+
+
+def roco_prefill(Q, K, V, lens: Sequence[int], B: int, r: int, cache: Cache, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R,
+                 count_self=1, scale: Optional[float] = None, lse_out=None, s_full=None, q_full=None,
+                 workspace: Optional[torch.Tensor] = None):
+    """Q, K, V: [S][G][Lmax][d] device tensors.  Fills `cache`."""
+    Lmax = Q.shape[2]
+    scale = cache.d ** -0.5 if scale is None else scale
+    if workspace is None:
+        workspace = torch.empty(roco_prefill_workspace_bytes(cache, Lmax), dtype=torch.uint8, device=Q.device)
+    lens_arr = (C.c_int32 * len(lens))(*[int(x) for x in lens])
+    rc = lib().roco_prefill(_ptr(Q), _ptr(K), _ptr(V), C.cast(lens_arr, C.c_void_p), Lmax, B, r, scope_mode,
+                            count_self, scale, C.byref(cache.c), _ptr(lse_out), _ptr(s_full), _ptr(q_full),
+                            _ptr(workspace), workspace.numel(), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_prefill")
+    return workspace
+
+
+def roco_decode_step(cache: Cache, q, k_new, v_new, r: int, attn_out, evicted_slot, evicted_pos=None, lse_out=None,
+                     scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R, step_order=ROCO_EVICT_FIRST, scale: Optional[float] = None):
+    scale = cache.d ** -0.5 if scale is None else scale
+    rc = lib().roco_decode_step(C.byref(cache.c), _ptr(q), _ptr(k_new), _ptr(v_new), r, scope_mode, step_order,
+                                scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot), _ptr(evicted_pos), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_decode_step")
+
+
+def roco_decode_host_staging_bytes(cache: Cache) -> int:
+    return int(lib().roco_decode_host_staging_bytes(C.byref(cache.c)))
+
+
+def roco_decode_step_host(cache: Cache, q_host, k_new_host, v_new_host, r: int, attn_out_host, evicted_slot_host,
+                          evicted_pos_host, staging, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R,
+                          step_order=ROCO_EVICT_FIRST, scale: Optional[float] = None):
+    """Same step with host (pinned) per-step tensors; synchronises the stream."""
+    scale = cache.d ** -0.5 if scale is None else scale
+    rc = lib().roco_decode_step_host(C.byref(cache.c), _ptr(q_host), _ptr(k_new_host), _ptr(v_new_host), r,
+                                     scope_mode, step_order, scale, _ptr(attn_out_host), _ptr(evicted_slot_host),
+                                     _ptr(evicted_pos_host), _ptr(staging), staging.numel(), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_decode_step_host")
+
+
+def roco_device_status(cache: Cache) -> int:
+    flags = C.c_int32(0)
+    rc = lib().roco_device_status(C.byref(cache.c), _stream(), C.byref(flags))
+    if rc not in (ROCO_OK, 5):
+        raise RocoError(rc, "roco_device_status")
+    return int(flags.value)
