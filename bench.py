@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the RoCo decode hot path on B200 (one JSON line on stdout).
+
+A *step* is one decode step of every (sequence, layer, head) unit of the Llama-2-7B-shape workload:
+attention over the budgeted cache, statistics update, scope/victim selection and in-place overwrite, all
+in one kernel launch per step.  The cache is first built by the library's own prefill (2048-token prompts
+evicted to B = 1024).  `value` is decode tokens/s of the attention path (one step yields S tokens and needs
+all layers*heads units of each sequence).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+N > 1 (under torch.distributed.run): every rank runs the same-sized workload on its own GPU with its own
+seed (units are independent; no data-path collective) and the aggregate is reported: weak scaling.
+`--impl reference` times the fp64 CPU oracle instead (rank 0 only), on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import workloads as W
+
+METRIC = "decode_tokens_per_s"
+UNIT = "tokens/s"
+
+
+# ----------------------------------------------------------------------------------------- helpers
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), float(p["bf16_tflops"]), "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+def algorithmic_bytes_per_unit_step(B: int, d: int, elem: int) -> int:
+    """K and V read once (2*B*d elements) plus s, q, n read and written (24*B bytes)."""
+    return 2 * B * d * elem + 24 * B
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.perf_counter(), [x.strip() for x in line.split(",")]))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for t, r in self.rows if t0 <= t <= t1 + 0.1] or [r for _, r in self.rows[-3:]]
+        sm, reasons, mx = [], set(), None
+        for r in rows:
+            try:
+                sm.append(float(r[1])); mx = float(r[2])
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def aggregate(tokens_per_rank: float, seconds_this_rank: float, world: int, backend_device=None) -> tuple:
+    """Whole-job throughput: tokens of all ranks / max over ranks of the elapsed time."""
+    if world == 1:
+        return tokens_per_rank / seconds_this_rank, seconds_this_rank
+    import torch.distributed as dist
+    t = torch.tensor([seconds_this_rank], dtype=torch.float64, device=backend_device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    tmax = float(t.item())
+    return world * tokens_per_rank / tmax, tmax
+
+
+# ----------------------------------------------------------------------------------------- workload
+
+def build_cache(w, device, R, seed_offset=0):
+    """Prefill every unit with the library (prompt -> budget B), layer-chunk by layer-chunk."""
+    w = W.scaled(w, seed=w.seed + 1000 * seed_offset)
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, device)
+    lens = W.prompt_lens(w)
+    chunk = min(w.G, 256)
+    ws = None
+    for b in range(w.S):
+        for g0 in range(0, w.G, chunk):
+            Q, K, V = (t[None] for t in W.prompt_chunk(w, b, g0, g0 + chunk, lens[b], device))
+            sub = R.Cache(1, chunk, w.B, w.d, w.torch_dtype, device)
+            ws = R.roco_prefill(Q, K, V, [lens[b]], w.B, w.r, sub, scale=w.scale, workspace=ws)
+            for name in ("K", "V", "s", "q", "n", "pos", "live", "t_next"):
+                getattr(cache, name)[b, g0:g0 + chunk].copy_(getattr(sub, name)[0])
+            if R.roco_device_status(sub) != 0:
+                raise RuntimeError("device status set during prefill")
+    return w, cache, lens
+
+
+def oracle_sample(w, cache, sample_units, n_steps, first_step, t_pos):
+    """Times the fp64 oracle (as it stands) on `sample_units` of the cache for n_steps decode steps."""
+    import oracle
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from harness import unit_view, widen
+    st = oracle.State(widen(unit_view(cache.K, sample_units)), widen(unit_view(cache.V, sample_units)),
+                      widen(unit_view(cache.s, sample_units)), widen(unit_view(cache.q, sample_units)),
+                      unit_view(cache.n, sample_units).cpu().numpy().copy(),
+                      unit_view(cache.pos, sample_units).cpu().numpy().copy(),
+                      unit_view(cache.live, sample_units).cpu().numpy().copy(),
+                      unit_view(cache.t_next, sample_units).cpu().numpy().copy())
+    toks = []
+    tp = list(t_pos)
+    for i in range(n_steps):
+        q, k, v = W.decode_tokens(w, first_step + i, tp, cache.K.device)
+        toks.append(tuple(widen(unit_view(x, sample_units)) for x in (q, k, v)))
+        tp = [t + 1 for t in tp]
+    per_step = []
+    for q, k, v in toks:
+        t0 = time.perf_counter()
+        oracle.decode_step(st, q, k, v, w.r, oracle.EXCLUDE_TOP_R, oracle.EVICT_FIRST, w.scale)
+        per_step.append(time.perf_counter() - t0)
+    return per_step, oracle.threads()
+
+
+def describe(w, world):
+    elem = 2 if w.dtype == "bf16" else 4
+    return {"workload": f"{w.name}: S={w.S} x {w.layers} layers x {w.heads} heads, d={w.d}, {w.dtype}, "
+                        f"prompt {w.prompt_lo}" + (f"-{w.prompt_hi}" if w.prompt_hi != w.prompt_lo else "") +
+                        f" -> B={w.B}, r={w.r}, EXCLUDE_TOP_R, EVICT_FIRST",
+            "units": w.U, "budget": w.B, "scope_r": w.r,
+            "l2": "inputs larger than L2 (K+V cache per step %.2f GB)" % (w.U * 2 * w.B * w.d * elem / 1e9),
+            "parallelism": f"units sharded over {world} GPU(s), no collective" if world > 1 else "1 GPU"}
+
+
+def reference_arm(args, steps, warmup):
+    """The fp64 oracle as it stands, on the host cores only (no GPU): a sample of units of the same workload is
+    prefilled and stepped by the oracle; its time is scaled by U / sample (units are independent)."""
+    import oracle
+    w = W.ALL[args.workload]
+    n_units = min(w.G, 32)
+    lens = W.prompt_lens(w)
+    Q, K, V = (x[None].to(torch.float64).numpy() for x in W.prompt_chunk(w, 0, 0, n_units, lens[0], "cpu"))
+    res = oracle.prefill(Q[0], K[0], V[0], [lens[0]] * n_units, w.B, w.r, oracle.EXCLUDE_TOP_R, w.scale)
+    st = res.state
+    per_step = []
+    tp = list(lens)
+    for i in range(warmup + steps):
+        q, k, v = (x[0, :n_units].to(torch.float64).numpy() for x in W.decode_tokens(w, i, tp, "cpu"))
+        t0 = time.perf_counter()
+        oracle.decode_step(st, q, k, v, w.r, oracle.EXCLUDE_TOP_R, oracle.EVICT_FIRST, w.scale)
+        per_step.append(time.perf_counter() - t0)
+        tp = [t + 1 for t in tp]
+    timed = per_step[warmup:]
+    sec = sum(timed)
+    value = (n_units * len(timed) / sec) * w.S / w.U
+    cores = oracle.threads()
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+            "warmup": warmup, "ms_per_step": 1e3 * sec / len(timed) * w.U / n_units, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": describe(w, 1),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{n_units} of {w.U} units, every step; time scaled by U/sample"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ----------------------------------------------------------------------------------------- main
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="roco", choices=["roco", "reference"])
+    ap.add_argument("--workload", default="llama7b_decode")
+    ap.add_argument("--small", action="store_true", help="1/16 of the units (for profiler captures)")
+    args = ap.parse_args()
+    rank, local_rank, world = dist_env()
+    if args.impl == "reference" and rank != 0:
+        return 0
+    steps, warmup = args.steps, max(args.warmup, 3)
+
+    if args.impl == "reference":
+        return reference_arm(args, steps, warmup)
+
+    import paper_2402_06262_b200 as R
+    torch.cuda.set_device(local_rank)
+    device = f"cuda:{local_rank}"
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(device))
+
+    w0 = W.ALL[args.workload]
+    if args.small:
+        w0 = W.scaled(w0, layers=max(1, w0.layers // 16))
+    w, cache, lens = build_cache(w0, device, R, seed_offset=rank)
+    elem = 2 if w.dtype == "bf16" else 4
+    config = describe(w, world)
+
+    total = warmup + steps
+    t_pos = list(lens)
+
+    # ---- decode inputs for every step, resident on the device before the timed region
+    toks = []
+    tp = list(t_pos)
+    for i in range(total):
+        toks.append(W.decode_tokens(w, i, tp, device))
+        tp = [t + 1 for t in tp]
+    out = torch.zeros(w.S, w.G, w.d, dtype=w.torch_dtype, device=device)
+    ev_slot = torch.zeros(w.S, w.G, dtype=torch.int32, device=device)
+    ev_pos = torch.zeros_like(ev_slot)
+
+    def step(i):
+        q, k, v = toks[i]
+        R.roco_decode_step(cache, q, k, v, w.r, out, ev_slot, ev_pos, scale=w.scale)
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+    visible = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
+    sampler = ClockSampler(visible[local_rank] if local_rank < len(visible) else local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    torch.cuda.synchronize()
+    t_wall0 = time.perf_counter()
+    evs[0].record()
+    for i in range(steps):
+        step(warmup + i)
+        evs[i + 1].record()
+    torch.cuda.synchronize()
+    t_wall1 = time.perf_counter()
+    if world > 1:
+        torch.distributed.barrier()
+    clocks = sampler.stop(t_wall0, t_wall1)
+    launch_ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
+    sec = evs[0].elapsed_time(evs[steps]) / 1e3
+    if R.roco_device_status(cache) != 0:
+        raise RuntimeError("device status word set during the timed region")
+    value, tmax = aggregate(w.S * steps, sec, world, device)
+
+    # ---- end to end through the host-buffer entry point (pinned host tensors in, results out, every step)
+    e2e_steps = min(steps, 32)
+    staging = torch.empty(R.roco_decode_host_staging_bytes(cache), dtype=torch.uint8, device=device)
+    h_toks = [tuple(x.cpu().pin_memory() for x in W.decode_tokens(w, total + i, [t + total + i for t in t_pos], device))
+              for i in range(e2e_steps)]
+    h_out = torch.zeros(w.S, w.G, w.d, dtype=w.torch_dtype).pin_memory()
+    h_slot = torch.zeros(w.S, w.G, dtype=torch.int32).pin_memory()
+    h_pos = torch.zeros(w.S, w.G, dtype=torch.int32).pin_memory()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for q, k, v in h_toks:
+        R.roco_decode_step_host(cache, q, k, v, w.r, h_out, h_slot, h_pos, staging, scale=w.scale)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_sec = e0.elapsed_time(e1) / 1e3
+    e2e_value, _ = aggregate(w.S * e2e_steps, e2e_sec, world, device)
+    vec = w.U * w.d * elem
+    e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 3 * vec, "d2h_bytes_per_step": vec + 8 * w.U,
+           "steps": e2e_steps}
+
+    # ---- roofline of the decode kernel (the only kernel in a step)
+    hbm_peak, _, which = peaks()
+    alg = algorithmic_bytes_per_unit_step(w.B, w.d, elem) * w.U
+    avg_launch = sum(launch_ms) / len(launch_ms) / 1e3
+    roofline = {"bound": "hbm", "achieved": alg / avg_launch / 1e9, "peak": hbm_peak, "unit": "GB/s",
+                "frac": alg / avg_launch / 1e9 / hbm_peak, "traffic": None, "peak_source": f"of {which}",
+                "kernel": "decode_step_kernel", "algorithmic_bytes_per_launch": alg,
+                "avg_launch_ms": avg_launch * 1e3, "frac_of_nominal_8TBs": alg / avg_launch / 8e12}
+    traffic_file = os.path.join(ROOT, "profiles", "decode_traffic.json")
+    if os.path.exists(traffic_file):
+        tr = json.load(open(traffic_file))
+        if tr.get("kernel_hash") == kernel_hash():
+            roofline["traffic"] = tr["dram_bytes_per_unit"] * w.U
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": 1e3 * tmax / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 K/V, fp32 softmax and statistics" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": config, "clocks": clocks, "e2e": e2e, "gpu_launches": steps, "roofline": roofline}
+
+    if rank == 0:
+        n_units, n_steps = min(w.U, 256), 64
+        sample = sorted(np.random.default_rng(0).choice(w.U, n_units, replace=False).tolist())
+        per_step, cores = oracle_sample(w, cache, sample, n_steps, total + e2e_steps,
+                                        [t + total + e2e_steps for t in t_pos])
+        osec = sum(per_step)
+        line["cpu_baseline"] = {"value": (n_units * n_steps / osec) * w.S / w.U, "unit": UNIT, "cores": cores,
+                                "kind": "oracle", "seconds": osec,
+                                "sample": f"{n_units} of {w.U} units x {n_steps} decode steps; scaled by U/sample"}
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+def kernel_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for fn in ("decode.cu", "select.cuh", "common.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_2402_06262_b200", "csrc", fn), "rb").read())
+    return h.hexdigest()[:16]
+
+
+if __name__ == "__main__":
+    sys.exit(main())
