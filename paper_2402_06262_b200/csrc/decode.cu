@@ -1,9 +1,15 @@
 // One decode step of KV-constrained inference with RoCo eviction (Sec. 3, Sec. 4.3, Fig. 1), one CTA per
-// unit.  The step is bound by HBM traffic: each unit's K and V blocks are streamed exactly once through a
-// shared-memory ring filled by bulk asynchronous copies (TMA, one producer warp), the B scores stay in
-// shared memory (no online softmax needed), the statistics update rides between the two passes, and the
-// scope / victim selection and the in-place slot overwrite happen in the same launch while the ring is
-// being filled -- so the per-unit traffic is 2*B*d elements of K/V plus the B-sized statistics arrays.
+// unit.  The step is bound by HBM traffic, so the kernel is organised around keeping each SM's share of the
+// memory system busy:
+//   - a producer warp streams the unit's K block, then its V block, exactly once, through a shared-memory
+//     ring filled by bulk asynchronous copies (TMA, non-multicast); the four statistics arrays arrive the
+//     same way;
+//   - eight consumer warps turn K tiles into scores (kept in shared memory: B floats, no online softmax),
+//     normalise, update Acc / Acc^square / Count and write them back, then turn V tiles into the output;
+//   - four policy warps build the eviction scope and pick the victim (Sec. 4.3) *while* the consumers stream:
+//     under EVICT_FIRST they work during the K pass (the new token's score and value are patched in
+//     afterwards, so the stream never waits for the decision), under ATTEND_FIRST during the V pass.
+// The freed slot is overwritten in place; the cache is never compacted.
 #include "common.cuh"
 #include "launch.h"
 #include "select.cuh"
@@ -12,9 +18,13 @@ namespace roco {
 
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumers = kConsumerWarps * 32;
-constexpr int kDecodeThreads = kConsumers + 32;  // + one producer warp
-constexpr int kTileBytes = 16384;
-constexpr int kBarConsumers = 1;  // named barrier id used by the consumer warps
+constexpr int kProducerWarp = kConsumerWarps;
+constexpr int kPolicyWarp0 = kConsumerWarps + 1;
+constexpr int kPolicyWarps = 4;
+constexpr int kPolicyThreads = kPolicyWarps * 32;
+constexpr int kDecodeThreads = kConsumers + 32 + kPolicyThreads;
+constexpr int kBarConsumers = 1;  // named barrier ids
+constexpr int kBarPolicy = 2;
 
 struct DecodeParams {
   const char *K, *V;
@@ -29,52 +39,59 @@ struct DecodeParams {
 };
 
 struct DecodeSmem {
-  // carve-up of dynamic shared memory; `stages` ring buffers come first (128-byte aligned)
-  char *ring;
-  uint64_t *full, *empty;
-  float *z;  // scores, then probabilities; doubles as the selection's key array
+  char *ring;  // `stages` tiles, 128-byte aligned
   float *s, *q;
-  int *n, *pos;
+  int *n, *pos;       // the unit's statistics (16-byte aligned: bulk-copy destinations)
+  float *z;           // scores, then probabilities
+  uint32_t *vkey;     // policy warps: variance keys
+  SelectScratch *sel; // policy warps: histogram and reduction scratch
   float *qf, *knew, *vnew, *outred, *red;
-  SelectScratch *sel;
-  int *flags;  // [0] abort flag
+  uint64_t *full, *empty;  // ring barriers
+  uint64_t *stats_full;    // statistics have landed in shared memory
+  uint64_t *stats_done;    // consumers have updated the statistics (ATTEND_FIRST: policy warp may start)
+  uint64_t *policy_done;   // victim chosen, slot reset, new K/V written
+  int *ctl;                // [0] abort flag, [1] slot of the new token, [2] evicted position
+  float *znew;             // score of the new token (EVICT_FIRST)
 };
 
+template <int TILE>
 __host__ __device__ inline size_t decode_smem_bytes(int B, int d, int stages) {
-  size_t Bp = align_up((size_t)B, 4);
-  size_t b = (size_t)stages * kTileBytes;
-  b += 2 * (size_t)stages * sizeof(uint64_t);
-  b = align_up(b, 16);
-  b += 5 * Bp * 4;                            // z, s, q, n, pos
+  const size_t Bp = align_up((size_t)B, 4);
+  size_t b = (size_t)stages * TILE;
+  b += 6 * Bp * 4;                            // s, q, n, pos, z, vkey
+  b += sizeof(SelectScratch);
   b += (size_t)(3 + kConsumerWarps) * d * 4;  // qf, knew, vnew, outred
   b += 64 * 4;                                // red
-  b = align_up(b, 16);
-  b += sizeof(SelectScratch);
-  b += 16;
+  b += (2 * (size_t)stages + 3) * sizeof(uint64_t);
+  b += 8 * 4;
   return b + 128;  // slack for aligning the base
 }
 
+template <int TILE>
 __device__ inline DecodeSmem carve(char *raw, int B, int d, int stages) {
   DecodeSmem m;
   char *p = (char *)align_up((size_t)raw, 128);
-  m.ring = p; p += (size_t)stages * kTileBytes;
-  m.full = (uint64_t *)p; p += stages * sizeof(uint64_t);
-  m.empty = (uint64_t *)p; p += stages * sizeof(uint64_t);
-  p = (char *)align_up((size_t)p, 16);
-  size_t Bp = align_up((size_t)B, 4);
-  m.z = (float *)p; p += Bp * 4;
+  const size_t Bp = align_up((size_t)B, 4);
+  m.ring = p; p += (size_t)stages * TILE;
   m.s = (float *)p; p += Bp * 4;
   m.q = (float *)p; p += Bp * 4;
   m.n = (int *)p; p += Bp * 4;
   m.pos = (int *)p; p += Bp * 4;
+  m.z = (float *)p; p += Bp * 4;
+  m.vkey = (uint32_t *)p; p += Bp * 4;
+  m.sel = (SelectScratch *)p; p += sizeof(SelectScratch);
   m.qf = (float *)p; p += d * 4;
   m.knew = (float *)p; p += d * 4;
   m.vnew = (float *)p; p += d * 4;
   m.outred = (float *)p; p += (size_t)kConsumerWarps * d * 4;
   m.red = (float *)p; p += 64 * 4;
-  p = (char *)align_up((size_t)p, 16);
-  m.sel = (SelectScratch *)p; p += sizeof(SelectScratch);
-  m.flags = (int *)p;
+  m.full = (uint64_t *)p; p += stages * sizeof(uint64_t);
+  m.empty = (uint64_t *)p; p += stages * sizeof(uint64_t);
+  m.stats_full = (uint64_t *)p; p += sizeof(uint64_t);
+  m.stats_done = (uint64_t *)p; p += sizeof(uint64_t);
+  m.policy_done = (uint64_t *)p; p += sizeof(uint64_t);
+  m.ctl = (int *)p; p += 4 * 4;
+  m.znew = (float *)p;
   return m;
 }
 
@@ -85,42 +102,49 @@ __device__ __forceinline__ float consumers_max(float v, float *red, int tid) {
   float r = red[0];
 #pragma unroll
   for (int w = 1; w < kConsumerWarps; ++w) r = fmaxf(r, red[w]);
-  named_bar_sync(kBarConsumers, kConsumers);
   return r;
 }
 
 __device__ __forceinline__ float consumers_sum(float v, float *red, int tid) {
   v = warp_sum(v);
-  if ((tid & 31) == 0) red[tid >> 5] = v;
+  if ((tid & 31) == 0) red[16 + (tid >> 5)] = v;
   named_bar_sync(kBarConsumers, kConsumers);
-  float r = red[0];
+  float r = red[16];
 #pragma unroll
-  for (int w = 1; w < kConsumerWarps; ++w) r += red[w];
-  named_bar_sync(kBarConsumers, kConsumers);
+  for (int w = 1; w < kConsumerWarps; ++w) r += red[16 + w];
   return r;
 }
 
-template <typename T, int D>
+template <typename T, int D, int TILE>
 __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const DecodeParams p) {
   constexpr int kRowBytes = D * (int)sizeof(T);
   constexpr int kLanesPerRow = kRowBytes / 16;
   constexpr int kRowsPerLoad = 32 / kLanesPerRow;
-  constexpr int kTileRows = kTileBytes / kRowBytes;
+  constexpr int kTileRows = TILE / kRowBytes;
   constexpr int kRowsPerWarp = kTileRows / kConsumerWarps;
   constexpr int kLoads = kRowsPerWarp / kRowsPerLoad;
   constexpr int kEPC = Elem<T>::kPerChunk;
   static_assert(kLanesPerRow <= 32 && kLoads >= 1, "tile shape");
 
   extern __shared__ char smem_raw[];
-  const DecodeSmem sm = carve(smem_raw, p.B, D, p.stages);
-  volatile int *abort_flag = sm.flags;
+  const DecodeSmem sm = carve<TILE>(smem_raw, p.B, D, p.stages);
+  volatile int *abort_flag = sm.ctl;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int u = blockIdx.x;
   const int B = p.B;
   const size_t unit_kv = (size_t)u * B * kRowBytes;
   const size_t unit_st = (size_t)u * B;
+  const int stages = p.stages;
 
+  if (tid == 0) {
+    for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kConsumerWarps); }
+    mbar_init(sm.stats_full, 1);
+    mbar_init(sm.stats_done, kConsumerWarps);
+    mbar_init(sm.policy_done, 1);
+    sm.ctl[0] = 0;
+    mbar_init_fence();
+  }
   int live0 = p.live[u];
   if (live0 < 0 || live0 > B) {
     if (tid == 0) atomicOr(p.status, ROCO_DEV_BAD_LIVE);
@@ -131,82 +155,105 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
   const int live_att = evict_first ? (full ? B : live0 + 1) : live0;  // slots the query attends over
   const int live_new = full ? B : live0 + 1;
   const int n_tiles = (live_att + kTileRows - 1) / kTileRows;
-  const int stages = p.stages;
-
-  if (tid == 0) {
-    for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kConsumerWarps); }
-    sm.flags[0] = 0;
-    mbar_init_fence();
-  }
+  const bool stats_by_tma = (B % 4) == 0;  // bulk copies need 16-byte aligned sources
   __syncthreads();
 
-  if (warp == kConsumerWarps) {
-    // ------------------------------------------------------------ producer: K tiles, then V tiles
+  if (warp == kProducerWarp) {
+    // ------------------------------------------------------------ producer: statistics, K tiles, V tiles
     if (lane == 0) {
+      if (stats_by_tma) {
+        const uint32_t bytes = (uint32_t)align_up((size_t)live0, 4) * 4;
+        if (bytes > 0) {
+          mbar_expect_tx(sm.stats_full, 4 * bytes);
+          bulk_g2s(sm.s, p.s + unit_st, bytes, sm.stats_full);
+          bulk_g2s(sm.q, p.q + unit_st, bytes, sm.stats_full);
+          bulk_g2s(sm.n, p.n + unit_st, bytes, sm.stats_full);
+          bulk_g2s(sm.pos, p.pos + unit_st, bytes, sm.stats_full);
+        } else {
+          mbar_arrive(sm.stats_full);
+        }
+      }
       for (int g = 0; g < 2 * n_tiles; ++g) {
         const int st = g % stages;
         if (g >= stages) mbar_wait(&sm.empty[st], ((g / stages) - 1) & 1, abort_flag, p.status);
         const int it = (g < n_tiles) ? g : g - n_tiles;
-        const char *src = ((g < n_tiles) ? p.K : p.V) + unit_kv + (size_t)it * kTileBytes;
+        const char *src = ((g < n_tiles) ? p.K : p.V) + unit_kv + (size_t)it * TILE;
         int rows = live_att - it * kTileRows;
         if (rows > kTileRows) rows = kTileRows;
         const uint32_t bytes = (uint32_t)rows * kRowBytes;
         mbar_expect_tx(&sm.full[st], bytes);
-        bulk_g2s(sm.ring + (size_t)st * kTileBytes, src, bytes, &sm.full[st]);
+        bulk_g2s(sm.ring + (size_t)st * TILE, src, bytes, &sm.full[st]);
       }
     }
     return;
   }
 
-  // -------------------------------------------------------------- consumers
-  const int t_new = p.t_next[u];
-  for (int j = tid; j < live0; j += kConsumers) {
-    sm.s[j] = p.s[unit_st + j];
-    sm.q[j] = p.q[unit_st + j];
-    sm.n[j] = p.n[unit_st + j];
-    sm.pos[j] = p.pos[unit_st + j];
-  }
-  if (tid < D) {
-    const size_t o = (size_t)u * D + tid;
-    sm.qf[tid] = Elem<T>::load((const T *)p.qv + o);
-    sm.knew[tid] = Elem<T>::load((const T *)p.k_new + o);
-    sm.vnew[tid] = Elem<T>::load((const T *)p.v_new + o);
-  }
-  named_bar_sync(kBarConsumers, kConsumers);
-
-  int e = -1;  // slot the new token goes to
-  int ev_slot = -1, ev_pos = -1;
-
-  // Frees a slot if the buffer is full (Sec. 4: "when the buffer is full, an eviction policy is
-  // executed"), writes the new token there with empty statistics.
-  auto evict_and_insert = [&]() {
+  if (warp >= kPolicyWarp0) {
+    // ------------------------------------------------------------ policy: scope, victim, in-place overwrite
+    const int ptid = tid - kPolicyWarp0 * 32;
+    const int t_new = p.t_next[u];  // read by these warps only: they also write the incremented value
+    if (!stats_by_tma) {            // odd budgets: plain loads
+      for (int j = ptid; j < live0; j += kPolicyThreads) {
+        sm.s[j] = p.s[unit_st + j]; sm.q[j] = p.q[unit_st + j];
+        sm.n[j] = p.n[unit_st + j]; sm.pos[j] = p.pos[unit_st + j];
+      }
+    }
+    named_bar_sync(kBarPolicy, kPolicyThreads);
+    if (!stats_by_tma && ptid == 0) mbar_arrive(sm.stats_full);
+    mbar_wait(sm.stats_full, 0, abort_flag, p.status);
+    if (!evict_first) mbar_wait(sm.stats_done, 0, abort_flag, p.status);  // select on the updated statistics
+    int e = live0, ev_slot = -1, ev_pos = -1;
     if (full) {
+      // Sec. 4: "when the buffer is full, an eviction policy is executed"
       const int m = scope_size(B, p.r, p.scope_mode);
-      e = block_select_victim(sm.s, sm.q, sm.n, sm.pos, B, m, (uint32_t *)sm.z, *sm.sel, tid, kConsumers,
-                              kBarConsumers);
+      e = group_select_victim(sm.s, sm.q, sm.n, sm.pos, B, m, sm.vkey, *sm.sel, ptid, kPolicyThreads, kBarPolicy);
       if (e < 0) {
-        if (tid == 0) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
+        if (ptid == 0) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
         e = 0;
       }
       ev_slot = e;
       ev_pos = sm.pos[e];
-    } else {
-      e = live0;
     }
-    named_bar_sync(kBarConsumers, kConsumers);  // everyone has read pos[e]
-    if (tid == 0) { sm.s[e] = 0.f; sm.q[e] = 0.f; sm.n[e] = 0; sm.pos[e] = t_new; }
-    if (tid < 2 * kLanesPerRow) {  // in-place overwrite of the freed slot, 16 bytes per thread
-      const bool isv = tid >= kLanesPerRow;
-      const int c = isv ? tid - kLanesPerRow : tid;
-      const uint4 val = *((const uint4 *)((isv ? p.v_new : p.k_new) + (size_t)u * kRowBytes) + c);
+    named_bar_sync(kBarPolicy, kPolicyThreads);  // everyone has read pos[e]
+    // the new token takes the slot with empty statistics
+    if (ptid == 0) {
+      sm.s[e] = 0.f; sm.q[e] = 0.f; sm.n[e] = 0; sm.pos[e] = t_new;
+      sm.ctl[1] = e;
+      p.pos[unit_st + e] = t_new;
+      p.ev_slot[u] = ev_slot;
+      if (p.ev_pos) p.ev_pos[u] = ev_pos;
+      p.live[u] = live_new;
+      p.t_next[u] = t_new + 1;
+      if (!evict_first) { p.s[unit_st + e] = 0.f; p.q[unit_st + e] = 0.f; p.n[unit_st + e] = 0; }
+    }
+    if (ptid >= 32 && ptid < 32 + 2 * kLanesPerRow) {  // in-place overwrite, 16 bytes per thread
+      const int c = ptid - 32;
+      const bool isv = c >= kLanesPerRow;
+      const int cc = isv ? c - kLanesPerRow : c;
+      const uint4 val = *((const uint4 *)((isv ? p.v_new : p.k_new) + (size_t)u * kRowBytes) + cc);
       char *dst = const_cast<char *>(isv ? p.V : p.K) + unit_kv + (size_t)e * kRowBytes;
-      *((uint4 *)dst + c) = val;
+      *((uint4 *)dst + cc) = val;
     }
-    named_bar_sync(kBarConsumers, kConsumers);
-  };
+    if (evict_first && ptid >= 96) {  // the new token's own score, from k_new directly
+      float acc = 0.f;
+      for (int c = lane; c < D; c += 32)
+        acc = fmaf(Elem<T>::load((const T *)p.qv + (size_t)u * D + c),
+                   Elem<T>::load((const T *)p.k_new + (size_t)u * D + c), acc);
+      acc = warp_sum(acc);
+      if (lane == 0) *sm.znew = acc * (p.scale * kLog2e);
+    }
+    named_bar_sync(kBarPolicy, kPolicyThreads);
+    if (ptid == 0) mbar_arrive(sm.policy_done);
+    return;
+  }
 
-  if (evict_first) evict_and_insert();
-  const int e_sub = evict_first ? e : -1;  // slot whose K/V come from k_new/v_new rather than the stream
+  // -------------------------------------------------------------- consumers
+  if (tid < D) {
+    const size_t o = (size_t)u * D + tid;
+    sm.qf[tid] = Elem<T>::load((const T *)p.qv + o);
+    if (evict_first) sm.vnew[tid] = Elem<T>::load((const T *)p.v_new + o);
+  }
+  named_bar_sync(kBarConsumers, kConsumers);
 
   // ---- scores: z_j = scale * q.K[j]  (Eq. 1), kept in base 2
   const float zscale = p.scale * kLog2e;
@@ -218,7 +265,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
   for (int it = 0; it < n_tiles; ++it) {
     const int st = it % stages;
     mbar_wait(&sm.full[st], (it / stages) & 1, abort_flag, p.status);
-    const char *tile = sm.ring + (size_t)st * kTileBytes;
+    const char *tile = sm.ring + (size_t)st * TILE;
 #pragma unroll
     for (int l = 0; l < kLoads; ++l) {
       const int row = warp * kRowsPerWarp + l * kRowsPerLoad + lane_row;
@@ -236,14 +283,19 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.empty[st]);
   }
-  if (e_sub >= 0 && warp == 0) {  // the new token's own score, from k_new directly
-    float acc = 0.f;
-    for (int c = lane; c < D; c += 32) acc = fmaf(sm.qf[c], sm.knew[c], acc);
-    acc = warp_sum(acc);
-    if (lane == 0) sm.red[32] = acc * zscale;
+
+  // EVICT_FIRST: the slot the policy warp has freed holds the new token; its score and value come from
+  // k_new / v_new, not from the stream (which may have read the slot before or after the overwrite).
+  int e_sub = -1;
+  if (evict_first) {
+    mbar_wait(sm.policy_done, 0, abort_flag, p.status);
+    e_sub = sm.ctl[1];
+    if (e_sub < 0 || e_sub >= B) e_sub = 0;  // only after an aborted wait
+  } else {
+    mbar_wait(sm.stats_full, 0, abort_flag, p.status);
   }
-  named_bar_sync(kBarConsumers, kConsumers);
-  if (e_sub >= 0 && tid == 0) sm.z[e_sub] = sm.red[32];
+  named_bar_sync(kBarConsumers, kConsumers);  // all scores are in shared memory
+  if (tid == 0 && e_sub >= 0) sm.z[e_sub] = *sm.znew;
   named_bar_sync(kBarConsumers, kConsumers);
 
   // ---- softmax over the occupied slots
@@ -262,11 +314,19 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     const float pj = sm.z[j] * inv;
     sm.z[j] = pj;
     // statistics of Sec. 4.3: Acc, Acc^square, Count
-    sm.s[j] += pj;
-    sm.q[j] = fmaf(pj, pj, sm.q[j]);
-    sm.n[j] += 1;
+    const float sj = sm.s[j] + pj, qj = fmaf(pj, pj, sm.q[j]);
+    const int nj = sm.n[j] + 1;
+    p.s[unit_st + j] = sj;
+    p.q[unit_st + j] = qj;
+    p.n[unit_st + j] = nj;
+    if (!evict_first) { sm.s[j] = sj; sm.q[j] = qj; sm.n[j] = nj; }
   }
-  named_bar_sync(kBarConsumers, kConsumers);
+  if (!evict_first) {  // hand the updated statistics to the policy warp
+    __syncwarp();
+    if (lane == 0) mbar_arrive(sm.stats_done);
+  }
+  if (tid == 0 && p.lse) p.lse[u] = (live_att > 0) ? (zmax + log2f(zsum)) * kLn2 : -INFINITY;
+  named_bar_sync(kBarConsumers, kConsumers);  // all probabilities are in shared memory
 
   // ---- out = sum_j p_j V[j]
   float acc[kEPC];
@@ -276,7 +336,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     const int g = n_tiles + it;
     const int st = g % stages;
     mbar_wait(&sm.full[st], (g / stages) & 1, abort_flag, p.status);
-    const char *tile = sm.ring + (size_t)st * kTileBytes;
+    const char *tile = sm.ring + (size_t)st * TILE;
 #pragma unroll
     for (int l = 0; l < kLoads; ++l) {
       const int row = warp * kRowsPerWarp + l * kRowsPerLoad + lane_row;
@@ -310,46 +370,35 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     if (e_sub >= 0) o = fmaf(sm.z[e_sub], sm.vnew[tid], o);
     Elem<T>::store((T *)p.out + (size_t)u * D + tid, o);
   }
-
-  if (!evict_first) {
-    named_bar_sync(kBarConsumers, kConsumers);  // sm.z (probabilities) no longer needed
-    evict_and_insert();
-  }
-
-  // ---- write the statistics back; only the freed slot's position changes
-  for (int j = tid; j < live_new; j += kConsumers) {
-    p.s[unit_st + j] = sm.s[j];
-    p.q[unit_st + j] = sm.q[j];
-    p.n[unit_st + j] = sm.n[j];
-  }
-  if (tid == 0) {
-    p.pos[unit_st + e] = t_new;
-    p.live[u] = live_new;
-    p.t_next[u] = t_new + 1;
-    p.ev_slot[u] = ev_slot;
-    if (p.ev_pos) p.ev_pos[u] = ev_pos;
-    if (p.lse) p.lse[u] = (live_att > 0) ? (zmax + log2f(zsum)) * kLn2 : -INFINITY;
-  }
 }
 
-template <typename T, int D>
+template <typename T, int D, int TILE>
 static cudaError_t launch_decode_t(const DecodeParams &p, int U, cudaStream_t stream) {
-  const size_t smem = decode_smem_bytes(p.B, D, p.stages);
-  cudaError_t err = cudaFuncSetAttribute(decode_step_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+  const size_t smem = decode_smem_bytes<TILE>(p.B, D, p.stages);
+  cudaError_t err = cudaFuncSetAttribute(decode_step_kernel<T, D, TILE>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
-  decode_step_kernel<T, D><<<U, kDecodeThreads, smem, stream>>>(p);
+  decode_step_kernel<T, D, TILE><<<U, kDecodeThreads, smem, stream>>>(p);
   return cudaGetLastError();
 }
 
-// Ring depth: the deepest ring (3..6 stages of 16 KiB) that still lets the most CTAs share an SM.
+// Tile size and ring depth: 16 KiB tiles and the deepest ring (3..6 stages) that still lets the most CTAs
+// share an SM; budgets too large for that fall back to 8 KiB tiles.
+template <int TILE>
 static int pick_stages(int B, int d) {
   const size_t per_sm = 227 * 1024;
   for (int ctas = 3; ctas >= 1; --ctas) {
     for (int st = 6; st >= 3; --st)
-      if ((decode_smem_bytes(B, d, st) + 1024) * ctas <= per_sm) return st;
+      if ((decode_smem_bytes<TILE>(B, d, st) + 1024) * ctas <= per_sm) return st;
   }
   return 0;
+}
+
+template <typename T, int D>
+static cudaError_t launch_decode_td(DecodeParams &p, int U, cudaStream_t stream) {
+  if ((p.stages = pick_stages<16384>(p.B, D)) > 0) return launch_decode_t<T, D, 16384>(p, U, stream);
+  if ((p.stages = pick_stages<8192>(p.B, D)) > 0) return launch_decode_t<T, D, 8192>(p, U, stream);
+  return cudaErrorInvalidConfiguration;
 }
 
 roco_status launch_decode_step(const roco_cache &c, const void *q, const void *k_new, const void *v_new, int r,
@@ -361,14 +410,12 @@ roco_status launch_decode_step(const roco_cache &c, const void *q, const void *k
   p.qv = (const char *)q; p.k_new = (const char *)k_new; p.v_new = (const char *)v_new;
   p.out = (char *)out; p.lse = lse; p.ev_slot = ev_slot; p.ev_pos = ev_pos;
   p.B = c.B; p.r = r; p.scope_mode = scope_mode; p.order = step_order; p.scale = scale;
-  p.stages = pick_stages(c.B, c.d);
-  if (p.stages == 0) return ROCO_ERR_UNSUPPORTED;
   const int U = c.S * c.G;
   cudaError_t err;
-  if (c.kv_dtype == ROCO_BF16 && c.d == 128) err = launch_decode_t<__nv_bfloat16, 128>(p, U, stream);
-  else if (c.kv_dtype == ROCO_BF16 && c.d == 64) err = launch_decode_t<__nv_bfloat16, 64>(p, U, stream);
-  else if (c.kv_dtype == ROCO_F32 && c.d == 128) err = launch_decode_t<float, 128>(p, U, stream);
-  else if (c.kv_dtype == ROCO_F32 && c.d == 64) err = launch_decode_t<float, 64>(p, U, stream);
+  if (c.kv_dtype == ROCO_BF16 && c.d == 128) err = launch_decode_td<__nv_bfloat16, 128>(p, U, stream);
+  else if (c.kv_dtype == ROCO_BF16 && c.d == 64) err = launch_decode_td<__nv_bfloat16, 64>(p, U, stream);
+  else if (c.kv_dtype == ROCO_F32 && c.d == 128) err = launch_decode_td<float, 128>(p, U, stream);
+  else if (c.kv_dtype == ROCO_F32 && c.d == 64) err = launch_decode_td<float, 64>(p, U, stream);
   else return ROCO_ERR_UNSUPPORTED;
   return err == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
 }

@@ -4,11 +4,10 @@
 //   scope   = the m cached tokens first in (variance asc, position asc)
 //   victim  = the in-scope token first in (mean asc, position asc)
 //
-// The rank-m threshold comes from a most-significant-digit radix select over 32-bit keys (the variance
-// rounded to fp32, whose bit pattern orders like the value for non-negative floats); ties on the
-// threshold variance are resolved by a second radix select over the tied tokens' positions, only when
-// not all of them fit in the scope.  Mean and variance are formed in fp64 from the fp32 sums so that the
-// only error in the decision is the accumulated rounding of s and q themselves.
+// The rank-m threshold comes from a most-significant-digit radix select over unsigned keys (the bit
+// pattern of a non-negative float or double orders like its value); ties on the threshold variance are
+// resolved by a second radix select over the tied tokens' positions, only when not all of them fit in the
+// scope.
 #pragma once
 
 #include "common.cuh"
@@ -18,7 +17,7 @@ namespace roco {
 struct SelectScratch {
   uint32_t hist[256];
   uint32_t digit, rank, count, pad;
-  double red_mean[32];
+  float red_mean[32];
   int red_pos[32];
   int red_slot[32];
 };
@@ -37,6 +36,7 @@ __device__ __forceinline__ KeyT radix_select(KeyF key, PredF pred, int n, uint32
   for (int shift = (int)sizeof(KeyT) * 8 - 8; shift >= 0; shift -= 8) {
     for (int i = tid; i < 256; i += nthreads) sc.hist[i] = 0;
     named_bar_sync(bar_id, nthreads);
+#pragma unroll 4
     for (int j = tid; j < n; j += nthreads) {
       if (pred(j)) {
         KeyT x = key(j);
@@ -83,17 +83,28 @@ __device__ __forceinline__ double variance_f64(float s, float q, int n) {
   return fmax(var, 0.0);  // also maps NaN to 0
 }
 
-__device__ __forceinline__ uint32_t variance_key(float s, float q, int n) {
-  return __float_as_uint((float)variance_f64(s, q, n));
+// Decode-step keys avoid fp64 division: the variance numerator q*n - s*s is formed in fp64 (both products
+// of fp32 values are exact there, so the cancellation costs nothing), then rounded to fp32 and divided by
+// n*n; the mean is the fp32 quotient s/n.  Both carry a relative error of a few 1e-7 of the value itself,
+// far inside the 1e-5 decision margin; equal (s, q, n) always give equal keys, so exact ties still fall to
+// the position rule.
+__device__ __forceinline__ uint32_t variance_key_fast(float s, float q, int n) {
+  const double num = fmax((double)q * (double)n - (double)s * (double)s, 0.0);  // NaN -> 0
+  const float nf = (float)n;
+  return __float_as_uint(__fdiv_rn((float)num, nf * nf));
 }
+
+__device__ __forceinline__ float mean_fast(float s, int n) { return __fdiv_rn(s, (float)n); }
 
 // Victim slot among slots [0, live) given scope size m (1 <= m <= live).  s, q, n, pos and vkey are
 // shared-memory arrays; vkey[live] is scratch.  Returns -1 if no slot qualifies (NaN statistics).
-// Every one of the `nthreads` threads gets the same return value.
-__device__ __forceinline__ int block_select_victim(const float *s, const float *q, const int *n, const int *pos,
+// Called by the `nthreads` threads (a multiple of 32) that synchronise on named barrier `bar_id`; every one
+// of them gets the same return value.
+__device__ __forceinline__ int group_select_victim(const float *s, const float *q, const int *n, const int *pos,
                                                    int live, int m, uint32_t *vkey, SelectScratch &sc, int tid,
                                                    int nthreads, int bar_id) {
-  for (int j = tid; j < live; j += nthreads) vkey[j] = variance_key(s[j], q[j], n[j]);
+#pragma unroll 4
+  for (int j = tid; j < live; j += nthreads) vkey[j] = variance_key_fast(s[j], q[j], n[j]);
   named_bar_sync(bar_id, nthreads);
   uint32_t T = 0xffffffffu;
   int P = 0x7fffffff;
@@ -107,20 +118,21 @@ __device__ __forceinline__ int block_select_victim(const float *s, const float *
                                       live, rank, sc, tid, nthreads, bar_id, &r2, &t2);
     }
   }
-  double bm = INFINITY;
+  float bm = INFINITY;
   int bp = 0x7fffffff, bs = -1;
+#pragma unroll 4
   for (int j = tid; j < live; j += nthreads) {
-    uint32_t k = vkey[j];
-    bool in_scope = (k < T) || (k == T && pos[j] <= P);
+    const uint32_t k = vkey[j];
+    const bool in_scope = (k < T) || (k == T && pos[j] <= P);
     if (!in_scope) continue;
-    double mean = mean_f64(s[j], n[j]);
+    const float mean = mean_fast(s[j], n[j]);
     if (mean < bm || (mean == bm && pos[j] < bp)) { bm = mean; bp = pos[j]; bs = j; }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
-    double om = __shfl_xor_sync(0xffffffffu, bm, o);
-    int op = __shfl_xor_sync(0xffffffffu, bp, o);
-    int os = __shfl_xor_sync(0xffffffffu, bs, o);
+    const float om = __shfl_xor_sync(0xffffffffu, bm, o);
+    const int op = __shfl_xor_sync(0xffffffffu, bp, o);
+    const int os = __shfl_xor_sync(0xffffffffu, bs, o);
     if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
   }
   const int warp = tid >> 5, nwarps = nthreads >> 5;
@@ -128,8 +140,8 @@ __device__ __forceinline__ int block_select_victim(const float *s, const float *
   named_bar_sync(bar_id, nthreads);
   bm = sc.red_mean[0]; bp = sc.red_pos[0]; bs = sc.red_slot[0];
   for (int w = 1; w < nwarps; ++w) {
-    double om = sc.red_mean[w];
-    int op = sc.red_pos[w], os = sc.red_slot[w];
+    const float om = sc.red_mean[w];
+    const int op = sc.red_pos[w], os = sc.red_slot[w];
     if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
   }
   named_bar_sync(bar_id, nthreads);
