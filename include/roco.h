@@ -88,6 +88,10 @@ const char *roco_status_string(int st);
 /* Bytes of device workspace roco_prefill needs for prompts of up to Lmax tokens (host function). */
 size_t roco_prefill_workspace_bytes(const roco_cache *cache, int Lmax);
 
+/* 1 if roco_prefill will run the score contraction of Eq. 1 on the tensor cores for this cache's dtype and
+ * head dimension (bf16, d = 128), 0 if it will use the CUDA-core path (host function). */
+int roco_prefill_uses_tensor_cores(const roco_cache *cache);
+
 /*
  * Prefill with eviction to budget (Sec. 4.3 last paragraph; Sec. 5.1 "Other Details": the budget is
  * fixed from the prompt length and eviction happens once, at the prefilling stage).

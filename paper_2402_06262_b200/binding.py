@@ -20,6 +20,7 @@ ROCO_SCOPE_EXCLUDE_TOP_R, ROCO_SCOPE_LOWEST_R = 0, 1
 ROCO_EVICT_FIRST, ROCO_ATTEND_FIRST = 0, 1
 
 EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes", "roco_prefill",
+           "roco_prefill_uses_tensor_cores",
            "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status")
 
 
@@ -51,6 +52,8 @@ def lib() -> C.CDLL:
         L.roco_status_string.argtypes = [C.c_int]
         L.roco_prefill_workspace_bytes.restype = C.c_size_t
         L.roco_prefill_workspace_bytes.argtypes = [C.POINTER(roco_cache), C.c_int]
+        L.roco_prefill_uses_tensor_cores.restype = C.c_int
+        L.roco_prefill_uses_tensor_cores.argtypes = [C.POINTER(roco_cache)]
         L.roco_decode_host_staging_bytes.restype = C.c_size_t
         L.roco_decode_host_staging_bytes.argtypes = [C.POINTER(roco_cache)]
         L.roco_prefill.restype = C.c_int
@@ -109,6 +112,10 @@ class Cache:
 
 def roco_prefill_workspace_bytes(cache: Cache, Lmax: int) -> int:
     return int(lib().roco_prefill_workspace_bytes(C.byref(cache.c), Lmax))
+
+
+def roco_prefill_uses_tensor_cores(cache: Cache) -> bool:
+    return bool(lib().roco_prefill_uses_tensor_cores(C.byref(cache.c)))
 
 
 def roco_prefill(Q, K, V, lens: Sequence[int], B: int, r: int, cache: Cache, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R,

@@ -70,6 +70,10 @@ size_t roco_prefill_workspace_bytes(const roco_cache *cache, int Lmax) {
   return prefill_ws(cache->S, cache->G, Lmax).total;
 }
 
+int roco_prefill_uses_tensor_cores(const roco_cache *cache) {
+  return (cache && prefill_tc_supported(cache->kv_dtype, cache->d)) ? 1 : 0;
+}
+
 roco_status roco_prefill(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax, int B,
                          int r, int scope_mode, int count_self, float scale, roco_cache *cache, float *lse_out,
                          float *s_full, float *q_full, void *workspace, size_t workspace_bytes, void *stream) {
@@ -98,8 +102,12 @@ roco_status roco_prefill(const void *Q, const void *K, const void *V, const int3
   int *dst = reinterpret_cast<int *>(ws + w.dst_off);
   if (cudaMemcpyAsync(lens_dev, lens_host, (size_t)cache->S * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess)
     return ROCO_ERR_CUDA;
-  st = launch_prefill_stats_simt(cache->kv_dtype, cache->d, cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, scale,
-                                 lse, sf, qf, cs);
+  if (prefill_tc_supported(cache->kv_dtype, cache->d))
+    st = launch_prefill_stats_tc(cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, scale, lse, sf, qf, cache->status,
+                                 cs);
+  else
+    st = launch_prefill_stats_simt(cache->kv_dtype, cache->d, cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, scale,
+                                   lse, sf, qf, cs);
   if (st != ROCO_OK) return st;
   return launch_budget_select_gather(*cache, Lmax, lens_dev, maxlen, r, K, V, sf, qf, dst, cs);
 }

@@ -18,6 +18,12 @@ roco_status launch_prefill_stats_simt(int kv_dtype, int d, int S, int G, int Lma
                                       const void *Q, const void *K, float scale, float *lse, float *s_full,
                                       float *q_full, cudaStream_t stream);
 
+// The same two passes on tcgen05 tensor cores with TMA-fed operands (bf16, d = 128 only).
+bool prefill_tc_supported(int kv_dtype, int d);
+roco_status launch_prefill_stats_tc(int S, int G, int Lmax, const int *lens_dev, int maxlen, const void *Q,
+                                    const void *K, float scale, float *lse, float *s_full, float *q_full, int *status,
+                                    cudaStream_t stream);
+
 // Select-to-budget on frozen statistics and gather of the survivors into the cache.
 // dst: [U][Lmax] int32 scratch (destination slot per token, -1 = evicted).
 roco_status launch_budget_select_gather(const roco_cache &c, int Lmax, const int *lens_dev, int maxlen, int r,

@@ -1,0 +1,384 @@
+// Prefill statistics on the 5th-generation tensor cores (bf16, d = 128): the causal score matrix of Eq. 1 is
+// a dense contraction, computed 128 x 128 tiles at a time by tcgen05.mma with fp32 accumulators in tensor
+// memory, operands staged in shared memory by TMA (128-byte swizzle, non-multicast).  Two passes, neither
+// of which ever stores the L x L matrix:
+//   pass 0 (row LSE):      S   = Q_a K_j^T  (a query row per TMEM lane): each thread keeps the running
+//                          (max, sum) of one row, lse_i = log sum_{j<=i} exp(scale * Q_i.K_j);
+//   pass 1 (column stats): S^T = K_a Q_i^T  (a key per TMEM lane): each thread recomputes
+//                          P_ij = exp(z_ij - lse_i) for one key column and keeps running fp32 sums
+//                          s_j = sum_i P_ij and q_j = sum_i P_ij^2 (Sec. 4.3) over all query tiles i >= a.
+// A CTA owns a pair of stationary tiles (a, T-1-a), so every CTA does the same number of tile products
+// under the causal mask.  Warp roles: warps 0-3 read the accumulators (TMEM lane quarter = warp id) and do
+// the softmax arithmetic, warp 4 issues TMA, warp 5 issues the MMAs; two accumulators alternate so that
+// the contraction of one tile overlaps the exponentials of the previous one.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "launch.h"
+
+namespace roco {
+
+constexpr int kTcTile = 128;                       // rows of a stationary / streamed tile
+constexpr int kTcD = 128;                          // head dimension
+constexpr int kTcTileBytes = kTcTile * kTcD * 2;   // 32 KiB: two 64-column halves of 16 KiB
+constexpr int kTcHalfBytes = kTcTileBytes / 2;
+constexpr int kTcStages = 2;                       // streamed-tile ring
+constexpr int kTcAccs = 2;                         // accumulators in tensor memory
+constexpr int kTcTmemCols = kTcAccs * kTcTile;     // 256 columns
+constexpr int kTcComputeWarps = 4;
+constexpr int kTcComputeThreads = kTcComputeWarps * 32;
+constexpr int kTcThreads = kTcComputeThreads + 64; // + TMA warp + MMA warp
+constexpr int kTcBarCompute = 1;
+
+// ------------------------------------------------------------------ PTX wrappers (tcgen05, TMA tensor)
+
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int c0, int c1, int c2, uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, M = 128, N = 128, K = 16.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// mbarrier arrives once all MMAs issued so far by this thread have completed
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base + t)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 operand tile stored as rows of 128 bytes with the
+// 128-byte swizzle (what TMA writes for a 64-column box): 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(const void *p) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_u32(p) >> 4) & 0x3fffu);  // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                         // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                         // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                         // 128-byte swizzle
+  return d;
+}
+
+// kind::f16 instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = 128
+constexpr uint32_t kIdescBf16M128N128 = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+
+struct TcSmem {
+  char *stat;                 // stationary operand tile
+  char *ring;                 // kTcStages streamed operand tiles
+  float *lse2;                // [2][128] log2-domain row LSE of the current query tile (pass 1)
+  uint64_t *stat_full, *stat_empty;
+  uint64_t *ring_full, *ring_empty;  // [kTcStages]
+  uint64_t *acc_full, *acc_empty;    // [kTcAccs]
+  uint32_t *tmem_base;
+  int *abort_flag;
+};
+
+constexpr size_t kTcSmemBytes = 1024 /*align*/ + (size_t)(1 + kTcStages) * kTcTileBytes + 2 * 128 * 4 +
+                                (2 + 2 * kTcStages + 2 * kTcAccs) * 8 + 16;
+
+__device__ inline TcSmem tc_carve(char *raw) {
+  TcSmem m;
+  char *p = (char *)align_up((size_t)raw, 1024);  // swizzle atoms are 1024-byte aligned
+  m.stat = p; p += kTcTileBytes;
+  m.ring = p; p += (size_t)kTcStages * kTcTileBytes;
+  m.lse2 = (float *)p; p += 2 * 128 * 4;
+  m.stat_full = (uint64_t *)p; p += 8;
+  m.stat_empty = (uint64_t *)p; p += 8;
+  m.ring_full = (uint64_t *)p; p += 8 * kTcStages;
+  m.ring_empty = (uint64_t *)p; p += 8 * kTcStages;
+  m.acc_full = (uint64_t *)p; p += 8 * kTcAccs;
+  m.acc_empty = (uint64_t *)p; p += 8 * kTcAccs;
+  m.tmem_base = (uint32_t *)p; p += 8;
+  m.abort_flag = (int *)p;
+  return m;
+}
+
+// PASS 0: stationary = Q tile a, streamed = K tiles 0..a, output lse.
+// PASS 1: stationary = K tile a, streamed = Q tiles a..T-1, input lse, output s_full / q_full.
+template <int PASS>
+__global__ void __launch_bounds__(kTcThreads) prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ,
+                                                                const __grid_constant__ CUtensorMap mapK,
+                                                                const int *lens, int G, int Lmax, int npairs,
+                                                                float scale, float *lse, float *s_full, float *q_full,
+                                                                int *status) {
+  extern __shared__ char tc_smem_raw[];
+  const TcSmem sm = tc_carve(tc_smem_raw);
+  volatile int *abort_flag = sm.abort_flag;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int u = blockIdx.x / npairs, pair = blockIdx.x % npairs;
+  const int L = lens[u / G];
+  const int T = (L + kTcTile - 1) / kTcTile;
+  // stationary tiles of this CTA: `pair` and its mirror (same total work for every CTA)
+  const int a0 = pair, a1 = T - 1 - pair;
+  const int n_tasks = (a0 > a1) ? 0 : (a0 == a1 ? 1 : 2);
+  if (n_tasks == 0) return;
+
+  if (tid == 0) {
+    mbar_init(sm.stat_full, 1);
+    mbar_init(sm.stat_empty, 1);
+    for (int i = 0; i < kTcStages; ++i) { mbar_init(&sm.ring_full[i], 1); mbar_init(&sm.ring_empty[i], 1); }
+    for (int i = 0; i < kTcAccs; ++i) { mbar_init(&sm.acc_full[i], 1); mbar_init(&sm.acc_empty[i], kTcComputeWarps); }
+    *sm.abort_flag = 0;
+    mbar_init_fence();
+  }
+  if (warp == 0) {
+    tmem_alloc(sm.tmem_base, kTcTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *sm.tmem_base;
+
+  // streamed tiles of task k: first index and count
+  auto task_tile = [&](int k) { return k == 0 ? a0 : a1; };
+  auto task_first = [&](int a) { return PASS == 0 ? 0 : a; };
+  auto task_count = [&](int a) { return PASS == 0 ? a + 1 : T - a; };
+
+  if (warp == kTcComputeWarps) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      const CUtensorMap *map_stat = PASS == 0 ? &mapQ : &mapK;
+      const CUtensorMap *map_ring = PASS == 0 ? &mapK : &mapQ;
+      int g = 0;  // streamed tiles issued so far
+      for (int k = 0; k < n_tasks; ++k) {
+        const int a = task_tile(k);
+        if (k > 0) mbar_wait(sm.stat_empty, (k - 1) & 1, abort_flag, status);
+        mbar_expect_tx(sm.stat_full, kTcTileBytes);
+        tma_load_3d(sm.stat, map_stat, 0, a * kTcTile, u, sm.stat_full);
+        tma_load_3d(sm.stat + kTcHalfBytes, map_stat, 64, a * kTcTile, u, sm.stat_full);
+        const int first = task_first(a), cnt = task_count(a);
+        for (int t = 0; t < cnt; ++t, ++g) {
+          const int st = g % kTcStages;
+          if (g >= kTcStages) mbar_wait(&sm.ring_empty[st], ((g / kTcStages) - 1) & 1, abort_flag, status);
+          char *dst = sm.ring + (size_t)st * kTcTileBytes;
+          mbar_expect_tx(&sm.ring_full[st], kTcTileBytes);
+          tma_load_3d(dst, map_ring, 0, (first + t) * kTcTile, u, &sm.ring_full[st]);
+          tma_load_3d(dst + kTcHalfBytes, map_ring, 64, (first + t) * kTcTile, u, &sm.ring_full[st]);
+        }
+      }
+    }
+  } else if (warp == kTcComputeWarps + 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int g = 0;
+      for (int k = 0; k < n_tasks; ++k) {
+        const int a = task_tile(k);
+        mbar_wait(sm.stat_full, k & 1, abort_flag, status);
+        const int cnt = task_count(a);
+        for (int t = 0; t < cnt; ++t, ++g) {
+          const int st = g % kTcStages, ac = g % kTcAccs;
+          mbar_wait(&sm.ring_full[st], (g / kTcStages) & 1, abort_flag, status);
+          if (g >= kTcAccs) mbar_wait(&sm.acc_empty[ac], ((g / kTcAccs) - 1) & 1, abort_flag, status);
+          tc_fence_after();
+          const char *bt = sm.ring + (size_t)st * kTcTileBytes;
+#pragma unroll
+          for (int kk = 0; kk < kTcD / 16; ++kk) {
+            const int off = (kk / 4) * kTcHalfBytes + (kk % 4) * 32;  // 16 bf16 = 32 bytes inside the swizzle row
+            umma_bf16(tmem + (uint32_t)(ac * kTcTile), smem_desc_sw128(sm.stat + off), smem_desc_sw128(bt + off),
+                      kIdescBf16M128N128, kk > 0 ? 1u : 0u);
+          }
+          umma_commit(&sm.ring_empty[st]);  // the streamed stage may be refilled once these MMAs are done
+          umma_commit(&sm.acc_full[ac]);
+        }
+        umma_commit(sm.stat_empty);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax / statistics warps
+    const float zscale = scale * kLog2e;
+    const int row = warp * 32 + lane;  // TMEM lane of this thread
+    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+    int g = 0;
+    for (int k = 0; k < n_tasks; ++k) {
+      const int a = task_tile(k);
+      const int first = task_first(a), cnt = task_count(a);
+      const int grow = a * kTcTile + row;  // global index of this thread's row (query in pass 0, key in pass 1)
+      float run0 = PASS == 0 ? -INFINITY : 0.f;  // pass 0: running max;  pass 1: running sum of p
+      float run1 = 0.f;                          // pass 0: running sum;  pass 1: running sum of p^2
+      float lse_next = 0.f;
+      if (PASS == 1) {
+        const int qi = first * kTcTile + tid;
+        lse_next = (qi < L) ? lse[(size_t)u * Lmax + qi] : 0.f;
+      }
+      for (int t = 0; t < cnt; ++t, ++g) {
+        const int ac = g % kTcAccs;
+        const int j = first + t;  // streamed tile index
+        if (PASS == 1) {
+          sm.lse2[(g & 1) * 128 + tid] = lse_next * kLog2e;
+          named_bar_sync(kTcBarCompute, kTcComputeThreads);
+          const int qn = (j + 1) * kTcTile + tid;
+          lse_next = (t + 1 < cnt && qn < L) ? lse[(size_t)u * Lmax + qn] : 0.f;
+        }
+        mbar_wait(&sm.acc_full[ac], (g / kTcAccs) & 1, abort_flag, status);
+        tc_fence_after();
+        const uint32_t taddr = tmem + lane_addr + (uint32_t)(ac * kTcTile);
+        const int col0 = j * kTcTile;  // global index of column 0 (key in pass 0, query in pass 1)
+        if (PASS == 0) {
+          const bool diag = (j == a);
+          float tmax = -INFINITY;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            float v[32];
+            tmem_ld32(taddr + c * 32, v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const bool ok = !diag || (col0 + c * 32 + i <= grow);
+              tmax = fmaxf(tmax, ok ? v[i] : -INFINITY);
+            }
+          }
+          const float m_new = fmaxf(run0, tmax * zscale);
+          float part = 0.f;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            float v[32];
+            tmem_ld32(taddr + c * 32, v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const bool ok = !diag || (col0 + c * 32 + i <= grow);
+              const float ex = ex2_approx(fmaf(v[i], zscale, -m_new));
+              part += ok ? ex : 0.f;
+            }
+          }
+          run1 = run1 * ex2_approx(run0 - m_new) + part;
+          run0 = m_new;
+        } else {
+          const bool edge = (j == a) || ((j + 1) * kTcTile > L);
+          const float *l2 = sm.lse2 + (g & 1) * 128;
+          float ts = 0.f, tq = 0.f;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            float v[32];
+            tmem_ld32(taddr + c * 32, v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int qi = col0 + c * 32 + i;
+              const float pij = ex2_approx(fmaf(v[i], zscale, -l2[c * 32 + i]));
+              const bool ok = !edge || (qi >= grow && qi < L);
+              const float pm = ok ? pij : 0.f;
+              ts += pm;
+              tq = fmaf(pm, pm, tq);
+            }
+          }
+          run0 += ts;
+          run1 += tq;
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.acc_empty[ac]);
+      }
+      if (grow < L) {
+        if (PASS == 0) {
+          lse[(size_t)u * Lmax + grow] = (run0 + log2f(run1)) * kLn2;
+        } else {
+          s_full[(size_t)u * Lmax + grow] = run0;
+          q_full[(size_t)u * Lmax + grow] = run1;
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, kTcTmemCols);
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [U][Lmax][128] bf16 as a 3-D tensor; box = 64 columns x 128 rows x 1 unit, 128-byte swizzle, zero fill
+static bool make_map(CUtensorMap *map, const void *base, int U, int Lmax) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)kTcD, (cuuint64_t)Lmax, (cuuint64_t)U};
+  const cuuint64_t strides[2] = {(cuuint64_t)kTcD * 2, (cuuint64_t)Lmax * kTcD * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)kTcTile, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool prefill_tc_supported(int kv_dtype, int d) { return kv_dtype == ROCO_BF16 && d == kTcD && encode_fn() != nullptr; }
+
+roco_status launch_prefill_stats_tc(int S, int G, int Lmax, const int *lens_dev, int maxlen, const void *Q,
+                                    const void *K, float scale, float *lse, float *s_full, float *q_full, int *status,
+                                    cudaStream_t stream) {
+  CUtensorMap mapQ, mapK;
+  const int U = S * G;
+  if (!make_map(&mapQ, Q, U, Lmax) || !make_map(&mapK, K, U, Lmax)) return ROCO_ERR_CUDA;
+  const int T = (maxlen + kTcTile - 1) / kTcTile;
+  const int npairs = (T + 1) / 2;
+  const unsigned grid = (unsigned)U * (unsigned)npairs;
+  cudaError_t err = cudaFuncSetAttribute(prefill_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kTcSmemBytes);
+  if (err == cudaSuccess)
+    err = cudaFuncSetAttribute(prefill_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes);
+  if (err != cudaSuccess) return ROCO_ERR_CUDA;
+  prefill_tc_kernel<0><<<grid, kTcThreads, kTcSmemBytes, stream>>>(mapQ, mapK, lens_dev, G, Lmax, npairs, scale, lse,
+                                                                  s_full, q_full, status);
+  prefill_tc_kernel<1><<<grid, kTcThreads, kTcSmemBytes, stream>>>(mapQ, mapK, lens_dev, G, Lmax, npairs, scale, lse,
+                                                                  s_full, q_full, status);
+  return cudaGetLastError() == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
+}
+
+}  // namespace roco
