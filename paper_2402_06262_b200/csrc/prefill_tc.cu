@@ -8,10 +8,14 @@
 //                          P_ij = exp(z_ij - lse_i) for one key column and keeps running fp32 sums
 //                          s_j = sum_i P_ij and q_j = sum_i P_ij^2 (Sec. 4.3) over all query tiles i >= a.
 // A CTA owns a pair of stationary tiles (a, T-1-a), so every CTA does the same number of tile products
-// under the causal mask.  Warp roles: warps 0-3 read the accumulators (TMEM lane quarter = warp id) and do
-// the softmax arithmetic, warp 4 issues TMA, warp 5 issues the MMAs; two accumulators alternate so that
-// the contraction of one tile overlaps the exponentials of the previous one.
+// under the causal mask.  Warp roles: warps 0-7 read the accumulators (TMEM lane quarter = warp id mod 4) and
+// do the softmax arithmetic -- two groups of four warps, each owning one of the two accumulators, so that
+// the contraction of one tile overlaps the exponentials of the previous one and the exponential unit always
+// has a second group to serve -- warp 8 issues TMA, warp 9 issues the MMAs.  The exponentials, not the
+// tensor pipe, are the practical limit of both passes (16384 per tile against 512 MMA cycles).
 #include <cuda.h>
+
+#include <type_traits>
 
 #include "common.cuh"
 #include "launch.h"
@@ -25,10 +29,12 @@ constexpr int kTcHalfBytes = kTcTileBytes / 2;
 constexpr int kTcStages = 2;                       // streamed-tile ring
 constexpr int kTcAccs = 2;                         // accumulators in tensor memory
 constexpr int kTcTmemCols = kTcAccs * kTcTile;     // 256 columns
-constexpr int kTcComputeWarps = 4;
+constexpr int kTcComputeWarps = 8;                 // two groups of four, one per accumulator
+constexpr int kTcGroupThreads = 128;
 constexpr int kTcComputeThreads = kTcComputeWarps * 32;
 constexpr int kTcThreads = kTcComputeThreads + 64; // + TMA warp + MMA warp
-constexpr int kTcBarCompute = 1;
+constexpr int kTcBarGroup0 = 1;                    // named barriers: 1, 2 = the two groups; 3 = both
+constexpr int kTcBarBoth = 3;
 
 // ------------------------------------------------------------------ PTX wrappers (tcgen05, TMA tensor)
 
@@ -68,9 +74,9 @@ __device__ __forceinline__ void umma_commit(uint64_t *bar) {
                : "memory");
 }
 
-// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base + t)
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base + t).  The load is
+// asynchronous: the registers are valid only after tmem_ld_wait on the same array.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -81,9 +87,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Waits for this thread's outstanding tensor-memory loads.  The array is an in/out operand so that no use
+// of its registers can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]),
+                 "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]),
+                 "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
 }
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -110,7 +126,8 @@ constexpr uint32_t kIdescBf16M128N128 = (1u << 4) | (1u << 7) | (1u << 10) | ((1
 struct TcSmem {
   char *stat;                 // stationary operand tile
   char *ring;                 // kTcStages streamed operand tiles
-  float *lse2;                // [2][128] log2-domain row LSE of the current query tile (pass 1)
+  float *lse2;                // [2 groups][2][128] log2-domain row LSE of a group's current query tile (pass 1)
+  float *merge;               // [2 tasks][2][128] partial running values handed from group 1 to group 0
   uint64_t *stat_full, *stat_empty;
   uint64_t *ring_full, *ring_empty;  // [kTcStages]
   uint64_t *acc_full, *acc_empty;    // [kTcAccs]
@@ -118,7 +135,7 @@ struct TcSmem {
   int *abort_flag;
 };
 
-constexpr size_t kTcSmemBytes = 1024 /*align*/ + (size_t)(1 + kTcStages) * kTcTileBytes + 2 * 128 * 4 +
+constexpr size_t kTcSmemBytes = 1024 /*align*/ + (size_t)(1 + kTcStages) * kTcTileBytes + 8 * 128 * 4 +
                                 (2 + 2 * kTcStages + 2 * kTcAccs) * 8 + 16;
 
 __device__ inline TcSmem tc_carve(char *raw) {
@@ -126,7 +143,8 @@ __device__ inline TcSmem tc_carve(char *raw) {
   char *p = (char *)align_up((size_t)raw, 1024);  // swizzle atoms are 1024-byte aligned
   m.stat = p; p += kTcTileBytes;
   m.ring = p; p += (size_t)kTcStages * kTcTileBytes;
-  m.lse2 = (float *)p; p += 2 * 128 * 4;
+  m.lse2 = (float *)p; p += 4 * 128 * 4;
+  m.merge = (float *)p; p += 4 * 128 * 4;
   m.stat_full = (uint64_t *)p; p += 8;
   m.stat_empty = (uint64_t *)p; p += 8;
   m.ring_full = (uint64_t *)p; p += 8 * kTcStages;
@@ -162,7 +180,7 @@ __global__ void __launch_bounds__(kTcThreads) prefill_tc_kernel(const __grid_con
     mbar_init(sm.stat_full, 1);
     mbar_init(sm.stat_empty, 1);
     for (int i = 0; i < kTcStages; ++i) { mbar_init(&sm.ring_full[i], 1); mbar_init(&sm.ring_empty[i], 1); }
-    for (int i = 0; i < kTcAccs; ++i) { mbar_init(&sm.acc_full[i], 1); mbar_init(&sm.acc_empty[i], kTcComputeWarps); }
+    for (int i = 0; i < kTcAccs; ++i) { mbar_init(&sm.acc_full[i], 1); mbar_init(&sm.acc_empty[i], 4); }
     *sm.abort_flag = 0;
     mbar_init_fence();
   }
@@ -232,92 +250,117 @@ __global__ void __launch_bounds__(kTcThreads) prefill_tc_kernel(const __grid_con
   } else {
     // ------------------------------------------------------------------ softmax / statistics warps
     const float zscale = scale * kLog2e;
-    const int row = warp * 32 + lane;  // TMEM lane of this thread
-    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-    int g = 0;
+    const int group = warp >> 2;                 // which accumulator this warp serves
+    const int gtid = tid & (kTcGroupThreads - 1);
+    const int row = (warp & 3) * 32 + lane;      // TMEM lane of this thread
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t taddr = tmem + lane_addr + (uint32_t)(group * kTcTile);
+    int g0 = 0;     // streamed tiles of earlier tasks
+    int mine = 0;   // tiles this group has processed so far (parity of its accumulator barrier, lse2 buffer)
     for (int k = 0; k < n_tasks; ++k) {
       const int a = task_tile(k);
       const int first = task_first(a), cnt = task_count(a);
       const int grow = a * kTcTile + row;  // global index of this thread's row (query in pass 0, key in pass 1)
       float run0 = PASS == 0 ? -INFINITY : 0.f;  // pass 0: running max;  pass 1: running sum of p
       float run1 = 0.f;                          // pass 0: running sum;  pass 1: running sum of p^2
+      const int t0 = ((g0 & 1) == group) ? 0 : 1;  // this group's first tile of the task
       float lse_next = 0.f;
-      if (PASS == 1) {
-        const int qi = first * kTcTile + tid;
+      if (PASS == 1 && t0 < cnt) {
+        const int qi = (first + t0) * kTcTile + gtid;
         lse_next = (qi < L) ? lse[(size_t)u * Lmax + qi] : 0.f;
       }
-      for (int t = 0; t < cnt; ++t, ++g) {
-        const int ac = g % kTcAccs;
+      for (int t = t0; t < cnt; t += 2, ++mine) {
         const int j = first + t;  // streamed tile index
+        float *l2 = sm.lse2 + (group * 2 + (mine & 1)) * 128;
         if (PASS == 1) {
-          sm.lse2[(g & 1) * 128 + tid] = lse_next * kLog2e;
-          named_bar_sync(kTcBarCompute, kTcComputeThreads);
-          const int qn = (j + 1) * kTcTile + tid;
-          lse_next = (t + 1 < cnt && qn < L) ? lse[(size_t)u * Lmax + qn] : 0.f;
+          l2[gtid] = lse_next * kLog2e;
+          if (group == 0) named_bar_sync(kTcBarGroup0, kTcGroupThreads);
+          else named_bar_sync(kTcBarGroup0 + 1, kTcGroupThreads);
+          const int qn = (j + 2) * kTcTile + gtid;
+          lse_next = (t + 2 < cnt && qn < L) ? lse[(size_t)u * Lmax + qn] : 0.f;
         }
-        mbar_wait(&sm.acc_full[ac], (g / kTcAccs) & 1, abort_flag, status);
+        mbar_wait(&sm.acc_full[group], mine & 1, abort_flag, status);
         tc_fence_after();
-        const uint32_t taddr = tmem + lane_addr + (uint32_t)(ac * kTcTile);
         const int col0 = j * kTcTile;  // global index of column 0 (key in pass 0, query in pass 1)
-        if (PASS == 0) {
-          const bool diag = (j == a);
-          float tmax = -INFINITY;
-#pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            float v[32];
-            tmem_ld32(taddr + c * 32, v);
+        uint32_t ra[32], rb[32];
+
+        // one 32-column chunk of the accumulator row of this thread
+        auto chunk = [&](const uint32_t (&r)[32], int c, auto masked_tag) {
+          constexpr bool kMasked = decltype(masked_tag)::value;
+          if (PASS == 0) {
+            // online softmax, one rescale per chunk
+            float cmax = -INFINITY;
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-              const bool ok = !diag || (col0 + c * 32 + i <= grow);
-              tmax = fmaxf(tmax, ok ? v[i] : -INFINITY);
+              const bool ok = !kMasked || (col0 + c * 32 + i <= grow);
+              cmax = fmaxf(cmax, ok ? __uint_as_float(r[i]) : -INFINITY);
             }
-          }
-          const float m_new = fmaxf(run0, tmax * zscale);
-          float part = 0.f;
-#pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            float v[32];
-            tmem_ld32(taddr + c * 32, v);
+            const float m_new = fmaxf(run0, cmax * zscale);
+            float part = 0.f;
+            if (m_new > -INFINITY) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const bool ok = !diag || (col0 + c * 32 + i <= grow);
-              const float ex = ex2_approx(fmaf(v[i], zscale, -m_new));
-              part += ok ? ex : 0.f;
+              for (int i = 0; i < 32; ++i) {
+                const bool ok = !kMasked || (col0 + c * 32 + i <= grow);
+                const float ex = ex2_approx(fmaf(__uint_as_float(r[i]), zscale, -m_new));
+                part += ok ? ex : 0.f;
+              }
+              run1 = run1 * ex2_approx(run0 - m_new) + part;
+              run0 = m_new;
             }
-          }
-          run1 = run1 * ex2_approx(run0 - m_new) + part;
-          run0 = m_new;
-        } else {
-          const bool edge = (j == a) || ((j + 1) * kTcTile > L);
-          const float *l2 = sm.lse2 + (g & 1) * 128;
-          float ts = 0.f, tq = 0.f;
-#pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            float v[32];
-            tmem_ld32(taddr + c * 32, v);
+          } else {
+            float ts = 0.f, tq = 0.f;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const int qi = col0 + c * 32 + i;
-              const float pij = ex2_approx(fmaf(v[i], zscale, -l2[c * 32 + i]));
-              const bool ok = !edge || (qi >= grow && qi < L);
-              const float pm = ok ? pij : 0.f;
-              ts += pm;
-              tq = fmaf(pm, pm, tq);
+            for (int i = 0; i < 32; i += 4) {
+              const float4 lv = *reinterpret_cast<const float4 *>(l2 + c * 32 + i);
+              const float lvv[4] = {lv.x, lv.y, lv.z, lv.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int qi = col0 + c * 32 + i + e;
+                float pij = ex2_approx(fmaf(__uint_as_float(r[i + e]), zscale, -lvv[e]));
+                if (kMasked) pij = (qi >= grow && qi < L) ? pij : 0.f;
+                ts += pij;
+                tq = fmaf(pij, pij, tq);
+              }
             }
+            run0 += ts;
+            run1 += tq;
           }
-          run0 += ts;
-          run1 += tq;
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.acc_empty[ac]);
+        };
+        auto tile = [&](auto masked_tag) {
+          tmem_ld32_issue(taddr, ra);
+          tmem_ld_wait(ra);
+          tmem_ld32_issue(taddr + 32, rb);
+          chunk(ra, 0, masked_tag);
+          tmem_ld_wait(rb);
+          tmem_ld32_issue(taddr + 64, ra);
+          chunk(rb, 1, masked_tag);
+          tmem_ld_wait(ra);
+          tmem_ld32_issue(taddr + 96, rb);
+          chunk(ra, 2, masked_tag);
+          tmem_ld_wait(rb);
+          // the accumulator has been read completely: hand it back before the last chunk's arithmetic
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.acc_empty[group]);
+          chunk(rb, 3, masked_tag);
+        };
+        const bool edge = PASS == 0 ? (j == a) : ((j == a) || ((j + 1) * kTcTile > L));
+        if (edge) tile(std::true_type{}); else tile(std::false_type{});
       }
-      if (grow < L) {
+      g0 += cnt;
+      // group 1 hands its partial running values to group 0, which merges and stores
+      float *mg = sm.merge + k * 256;
+      if (group == 1) { mg[row] = run0; mg[128 + row] = run1; }
+      named_bar_sync(kTcBarBoth, kTcComputeThreads);
+      if (group == 0 && grow < L) {
+        const float o0 = mg[row], o1 = mg[128 + row];
         if (PASS == 0) {
-          lse[(size_t)u * Lmax + grow] = (run0 + log2f(run1)) * kLn2;
+          const float m = fmaxf(run0, o0);
+          const float l = run1 * ex2_approx(run0 - m) + o1 * ex2_approx(o0 - m);
+          lse[(size_t)u * Lmax + grow] = (m + log2f(l)) * kLn2;
         } else {
-          s_full[(size_t)u * Lmax + grow] = run0;
-          q_full[(size_t)u * Lmax + grow] = run1;
+          s_full[(size_t)u * Lmax + grow] = run0 + o0;
+          q_full[(size_t)u * Lmax + grow] = run1 + o1;
         }
       }
     }
