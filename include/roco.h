@@ -118,6 +118,27 @@ roco_status roco_prefill(const void *Q, const void *K, const void *V, const int3
                          size_t workspace_bytes, void *stream);
 
 /*
+ * roco_prefill without a caller-provided workspace.  The paper has no counterpart: this exists for callers
+ * that cannot allocate device memory at call time -- code running inside a serving runtime whose memory
+ * pool already owns the GPU (cudaMalloc fails there), or a latency-critical loop that must not call
+ * cudaMalloc/cudaFree because they synchronise the device.  Same arguments, results and errors as
+ * roco_prefill, minus `workspace`; the scratch is an array of ROCO_PREFILL_STATIC_SCRATCH_BYTES built into
+ * the library (every GPU that loads the library holds it until the process exits).  The call allocates
+ * nothing.
+ *   - Limit: roco_prefill_workspace_bytes(cache, Lmax) must not exceed ROCO_PREFILL_STATIC_SCRATCH_BYTES
+ *     (S*G*Lmax up to about 524 000 tokens, e.g. 64 units x 8192); larger problems get ROCO_ERR_WORKSPACE.
+ *   - The first call on a device looks up the array's device address (with that device current); make that
+ *     first call before starting any stream capture on the device.
+ *   - All calls on a device share the one array, which keeps the previous call's contents (no buffer in it
+ *     needs to start at zero).  Two calls that overlap on the GPU -- different streams, or another host
+ *     thread -- race on it: issue them on one stream or order them yourself.
+ */
+#define ROCO_PREFILL_STATIC_SCRATCH_BYTES (8u << 20)
+roco_status roco_prefill_static(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax,
+                                int B, int r, int scope_mode, int count_self, float scale, roco_cache *cache,
+                                float *lse_out, float *s_full, float *q_full, void *stream);
+
+/*
  * One decode step for every unit (Sec. 3 constrained inference; Sec. 4 "when the buffer is full, an
  * eviction policy is executed"; Sec. 4.3 RoCo rule; Fig. 1 ordering).
  *

@@ -20,7 +20,7 @@ ROCO_SCOPE_EXCLUDE_TOP_R, ROCO_SCOPE_LOWEST_R = 0, 1
 ROCO_EVICT_FIRST, ROCO_ATTEND_FIRST = 0, 1
 
 EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes", "roco_prefill",
-           "roco_prefill_uses_tensor_cores",
+           "roco_prefill_uses_tensor_cores", "roco_prefill_static",
            "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status")
 
 
@@ -60,6 +60,10 @@ def lib() -> C.CDLL:
         L.roco_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
                                    C.c_int, C.c_float, C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_void_p, C.c_size_t, C.c_void_p]
+        L.roco_prefill_static.restype = C.c_int
+        L.roco_prefill_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                          C.c_int, C.c_int, C.c_float, C.POINTER(roco_cache), C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p]
         L.roco_decode_step.restype = C.c_int
         L.roco_decode_step.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                                        C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -133,6 +137,25 @@ def roco_prefill(Q, K, V, lens: Sequence[int], B: int, r: int, cache: Cache, sco
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_prefill")
     return workspace
+
+
+PREFILL_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def roco_prefill_static(Q, K, V, lens: Sequence[int], B: int, r: int, cache: Cache,
+                        scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R, count_self=1, scale: Optional[float] = None,
+                        lse_out=None, s_full=None, q_full=None):
+    """roco_prefill for callers that cannot allocate a workspace: the scratch is an 8 MiB array built into the
+    library (so S*G*Lmax is limited; larger problems raise RocoError with the workspace status).  Calls on one
+    device share that array: keep them on one stream."""
+    Lmax = Q.shape[2]
+    scale = cache.d ** -0.5 if scale is None else scale
+    lens_arr = (C.c_int32 * len(lens))(*[int(x) for x in lens])
+    rc = lib().roco_prefill_static(_ptr(Q), _ptr(K), _ptr(V), C.cast(lens_arr, C.c_void_p), Lmax, B, r, scope_mode,
+                                   count_self, scale, C.byref(cache.c), _ptr(lse_out), _ptr(s_full), _ptr(q_full),
+                                   _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_prefill_static")
 
 
 def roco_decode_step(cache: Cache, q, k_new, v_new, r: int, attn_out, evicted_slot, evicted_pos=None, lse_out=None,
