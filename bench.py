@@ -158,6 +158,43 @@ def oracle_sample(w, cache, sample_units, n_steps, first_step, t_pos):
     return per_step, oracle.threads()
 
 
+def prefill_bench(R, device, small=False, reps=3):
+    """Prefill-stage statistics + eviction to budget on the Llama-2-7B-shape prompt workload (8192-token causal
+    prompt, 32 x 32 heads, evicted to B = 2048 with r = 256): best of `reps` calls of roco_prefill."""
+    w = W.LLAMA7B_PREFILL
+    if small:
+        w = W.scaled(w, layers=1)
+    L = w.prompt_lo
+    _, bf16_peak, which = peaks()
+    chunk = min(w.G, 256)
+    Q, K, V = (torch.cat(x)[None] for x in zip(*[W.prompt_chunk(w, 0, g0, g0 + chunk, L, device)
+                                                  for g0 in range(0, w.G, chunk)]))
+    cache = R.Cache(1, w.G, w.B, w.d, w.torch_dtype, device)
+    ws = R.roco_prefill(Q, K, V, [L], w.B, w.r, cache, scale=w.scale)
+    torch.cuda.synchronize()
+    best = float("inf")
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        R.roco_prefill(Q, K, V, [L], w.B, w.r, cache, scale=w.scale, workspace=ws)
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1) / 1e3)
+    if R.roco_device_status(cache) != 0:
+        raise RuntimeError("device status word set during prefill")
+    T = (L + 127) // 128
+    executed = 2 * w.U * (T * (T + 1) // 2) * 2 * 128 ** 3          # two passes of 128^3 tile products
+    algorithmic = w.U * L * (L + 1) * w.d                            # one causal Q K^T
+    tc = R.roco_prefill_uses_tensor_cores(cache)
+    return {"workload": f"{w.name}: {w.layers} layers x {w.heads} heads, d={w.d}, {w.dtype}, causal prompt {L} -> "
+                        f"B={w.B}, r={w.r}, EXCLUDE_TOP_R", "ms": best * 1e3, "tokens_per_s": w.S * L / best,
+            "tensor_cores": tc, "tflops_executed": executed / best / 1e12,
+            "tflops_algorithmic": algorithmic / best / 1e12, "peak_tflops": bf16_peak, "peak_source": f"of {which}",
+            "frac_executed": executed / best / 1e12 / bf16_peak,
+            "frac_algorithmic": algorithmic / best / 1e12 / bf16_peak,
+            "launches_per_call": 4, "timing": f"best of {reps} whole roco_prefill calls (both passes, select, gather)"}
+
+
 def describe(w, world):
     elem = 2 if w.dtype == "bf16" else 4
     return {"workload": f"{w.name}: S={w.S} x {w.layers} layers x {w.heads} heads, d={w.d}, {w.dtype}, "
@@ -211,6 +248,7 @@ def main():
     ap.add_argument("--impl", default="roco", choices=["roco", "reference"])
     ap.add_argument("--workload", default="llama7b_decode")
     ap.add_argument("--small", action="store_true", help="1/16 of the units (for profiler captures)")
+    ap.add_argument("--prefill-only", action="store_true", help="run only the prefill measurement")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
     if args.impl == "reference" and rank != 0:
@@ -227,6 +265,9 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(device))
 
+    if args.prefill_only:
+        print(json.dumps({"prefill": prefill_bench(R, device, small=args.small)}))
+        return 0
     w0 = W.ALL[args.workload]
     if args.small:
         w0 = W.scaled(w0, layers=max(1, w0.layers // 16))
@@ -316,6 +357,10 @@ def main():
             "ms_per_step": 1e3 * tmax / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 K/V, fp32 softmax and statistics" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": config, "clocks": clocks, "e2e": e2e, "gpu_launches": steps, "roofline": roofline}
+
+    del toks, h_toks
+    torch.cuda.empty_cache()
+    line["prefill"] = prefill_bench(R, device, small=args.small)
 
     if rank == 0:
         n_units, n_steps = min(w.U, 512), 128
