@@ -26,6 +26,7 @@ def lib():
         _lib = C.CDLL(build_library())
         _lib.roco_oracle_threads.restype = C.c_int
         _lib.roco_oracle_select.restype = C.c_int
+        _lib.roco_oracle_attention_row.restype = C.c_double
         _lib.roco_oracle_select_to_budget_onepass.restype = C.c_int
         _lib.roco_oracle_prefill_unit.restype = C.c_int
         _lib.roco_oracle_prefill_batch.restype = C.c_int
@@ -58,6 +59,15 @@ def prefill_stats(Q, K, scale, count_self=1, want_P=False):
     lib().roco_oracle_prefill_stats(_p(Q), _p(K), C.c_int(L), C.c_int(d), C.c_double(scale),
                                     C.c_int(count_self), _p(lse), _p(s), _p(q), _p(n), _p(P))
     return (lse, s, q, n, P) if want_P else (lse, s, q, n)
+
+
+def attention_row(qv, K, scale):
+    """Eq. 1 for one query over the rows of K: returns (p [count], lse)."""
+    qv, K = _f64(qv), _f64(K)
+    p = np.zeros(K.shape[0])
+    lse = lib().roco_oracle_attention_row(_p(qv), _p(K), C.c_int(K.shape[0]), C.c_int(K.shape[1]), C.c_double(scale),
+                                          _p(p))
+    return p, float(lse)
 
 
 def select(s, q, n, pos, r, mode, delta=1e-5):

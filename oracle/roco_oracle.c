@@ -82,6 +82,11 @@ static double softmax_row(const double *qv, const double *K, int count, int d, d
   return zmax + log(Z);
 }
 
+/* Eq. 1 for one query over `count` keys: probabilities p[count]; returns the log-sum-exp of the scaled scores. */
+double roco_oracle_attention_row(const double *qv, const double *K, int count, int d, double scale, double *p) {
+  return softmax_row(qv, K, count, d, scale, p);
+}
+
 /* Causal prefill statistics of one unit (Eq. 1 with the causal mask; Sec. 4.3 arrays).
  * Q, K: [L][d].  lse: [L] (may be NULL).  s, q: [L] doubles; n: [L] ints.
  * P_out: [L][L] row-major full probability matrix (may be NULL; zeros above the diagonal). */

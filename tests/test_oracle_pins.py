@@ -483,3 +483,11 @@ def test_ragged_prompts_in_one_batch():
         np.testing.assert_array_equal(res.state.pos[u], solo.state.pos[0])
         np.testing.assert_array_equal(res.state.s[u], solo.state.s[0])
         assert res.state.live[u] == min(L, B) and res.state.t_next[u] == L
+
+
+def test_attention_row_is_library_softmax():
+    rng = np.random.default_rng(21)
+    K = rng.normal(size=(37, 8)); qv = rng.normal(size=8)
+    p, lse = oracle.attention_row(qv, K, 0.4)
+    np.testing.assert_allclose(p, softmax(0.4 * K @ qv), rtol=1e-13)
+    assert lse == pytest.approx(logsumexp(0.4 * K @ qv), rel=1e-13)
