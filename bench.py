@@ -123,11 +123,15 @@ def build_cache(w, device, R, seed_offset=0):
     ws = None
     for b in range(w.S):
         for g0 in range(0, w.G, chunk):
-            Q, K, V = (t[None] for t in W.prompt_chunk(w, b, g0, g0 + chunk, lens[b], device))
-            sub = R.Cache(1, chunk, w.B, w.d, w.torch_dtype, device)
-            ws = R.roco_prefill(Q, K, V, [lens[b]], w.B, w.r, sub, scale=w.scale, workspace=ws)
+            g1 = min(g0 + chunk, w.G)
+            Q, K, V = (t[None] for t in W.prompt_chunk(w, b, g0, g1, lens[b], device))
+            sub = R.Cache(1, g1 - g0, w.B, w.d, w.torch_dtype, device)
+            need = R.roco_prefill_workspace_bytes(sub, lens[b])
+            if ws is None or ws.numel() < need:
+                ws = torch.empty(need, dtype=torch.uint8, device=device)
+            R.roco_prefill(Q, K, V, [lens[b]], w.B, w.r, sub, scale=w.scale, workspace=ws)
             for name in ("K", "V", "s", "q", "n", "pos", "live", "t_next"):
-                getattr(cache, name)[b, g0:g0 + chunk].copy_(getattr(sub, name)[0])
+                getattr(cache, name)[b, g0:g1].copy_(getattr(sub, name)[0])
             if R.roco_device_status(sub) != 0:
                 raise RuntimeError("device status set during prefill")
     return w, cache, lens

@@ -2,10 +2,10 @@
 // unit.  The step is bound by HBM traffic, so the kernel is organised around keeping each SM's share of the
 // memory system busy:
 //   - a producer warp streams the unit's K block, then its V block, exactly once, through a shared-memory
-//     ring filled by bulk asynchronous copies (TMA, non-multicast); the four statistics arrays arrive the
-//     same way;
+//     ring filled by bulk asynchronous copies (TMA, non-multicast);
 //   - eight consumer warps turn K tiles into scores (kept in shared memory: B floats, no online softmax),
-//     normalise, update Acc / Acc^square / Count and write them back, then turn V tiles into the output;
+//     normalise, update Acc / Acc^square / Count in global memory (read once, written once), then turn V
+//     tiles into the output;
 //   - four policy warps build the eviction scope and pick the victim (Sec. 4.3) *while* the consumers stream:
 //     under EVICT_FIRST they work during the K pass (the new token's score and value are patched in
 //     afterwards, so the stream never waits for the decision), under ATTEND_FIRST during the V pass.
@@ -39,18 +39,16 @@ struct DecodeParams {
 };
 
 struct DecodeSmem {
-  char *ring;  // `stages` tiles, 128-byte aligned
-  float *s, *q;
-  int *n, *pos;       // the unit's statistics (16-byte aligned: bulk-copy destinations)
-  float *z;           // scores, then probabilities
-  uint32_t *vkey;     // policy warps: variance keys
-  SelectScratch *sel; // policy warps: histogram and reduction scratch
-  float *qf, *knew, *vnew, *outred, *red;
+  char *ring;          // `stages` tiles, 128-byte aligned
+  float *z;            // scores, then probabilities
+  uint32_t *vkey;      // policy warps: variance keys
+  float *mkey;         // policy warps: mean keys
+  SelectScratch *sel;  // policy warps: histogram and reduction scratch
+  float *qf, *vnew, *outred, *red;
   uint64_t *full, *empty;  // ring barriers
-  uint64_t *stats_full;    // statistics have landed in shared memory
-  uint64_t *stats_done;    // consumers have updated the statistics (ATTEND_FIRST: policy warp may start)
-  uint64_t *policy_done;   // victim chosen, slot reset, new K/V written
-  int *ctl;                // [0] abort flag, [1] slot of the new token, [2] evicted position
+  uint64_t *stats_done;    // consumers have written the updated statistics (ATTEND_FIRST: policy may start)
+  uint64_t *policy_done;   // victim chosen, new K/V written
+  int *ctl;                // [0] abort flag, [1] slot of the new token
   float *znew;             // score of the new token (EVICT_FIRST)
 };
 
@@ -58,11 +56,11 @@ template <int TILE>
 __host__ __device__ inline size_t decode_smem_bytes(int B, int d, int stages) {
   const size_t Bp = align_up((size_t)B, 4);
   size_t b = (size_t)stages * TILE;
-  b += 6 * Bp * 4;                            // s, q, n, pos, z, vkey
+  b += 3 * Bp * 4;  // z, vkey, mkey
   b += sizeof(SelectScratch);
-  b += (size_t)(3 + kConsumerWarps) * d * 4;  // qf, knew, vnew, outred
+  b += (size_t)(2 + kConsumerWarps) * d * 4;  // qf, vnew, outred
   b += 64 * 4;                                // red
-  b += (2 * (size_t)stages + 3) * sizeof(uint64_t);
+  b += (2 * (size_t)stages + 2) * sizeof(uint64_t);
   b += 8 * 4;
   return b + 128;  // slack for aligning the base
 }
@@ -73,21 +71,16 @@ __device__ inline DecodeSmem carve(char *raw, int B, int d, int stages) {
   char *p = (char *)align_up((size_t)raw, 128);
   const size_t Bp = align_up((size_t)B, 4);
   m.ring = p; p += (size_t)stages * TILE;
-  m.s = (float *)p; p += Bp * 4;
-  m.q = (float *)p; p += Bp * 4;
-  m.n = (int *)p; p += Bp * 4;
-  m.pos = (int *)p; p += Bp * 4;
   m.z = (float *)p; p += Bp * 4;
   m.vkey = (uint32_t *)p; p += Bp * 4;
+  m.mkey = (float *)p; p += Bp * 4;
   m.sel = (SelectScratch *)p; p += sizeof(SelectScratch);
   m.qf = (float *)p; p += d * 4;
-  m.knew = (float *)p; p += d * 4;
   m.vnew = (float *)p; p += d * 4;
   m.outred = (float *)p; p += (size_t)kConsumerWarps * d * 4;
   m.red = (float *)p; p += 64 * 4;
   m.full = (uint64_t *)p; p += stages * sizeof(uint64_t);
   m.empty = (uint64_t *)p; p += stages * sizeof(uint64_t);
-  m.stats_full = (uint64_t *)p; p += sizeof(uint64_t);
   m.stats_done = (uint64_t *)p; p += sizeof(uint64_t);
   m.policy_done = (uint64_t *)p; p += sizeof(uint64_t);
   m.ctl = (int *)p; p += 4 * 4;
@@ -139,7 +132,6 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
 
   if (tid == 0) {
     for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kConsumerWarps); }
-    mbar_init(sm.stats_full, 1);
     mbar_init(sm.stats_done, kConsumerWarps);
     mbar_init(sm.policy_done, 1);
     sm.ctl[0] = 0;
@@ -155,24 +147,11 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
   const int live_att = evict_first ? (full ? B : live0 + 1) : live0;  // slots the query attends over
   const int live_new = full ? B : live0 + 1;
   const int n_tiles = (live_att + kTileRows - 1) / kTileRows;
-  const bool stats_by_tma = (B % 4) == 0;  // bulk copies need 16-byte aligned sources
   __syncthreads();
 
   if (warp == kProducerWarp) {
-    // ------------------------------------------------------------ producer: statistics, K tiles, V tiles
+    // ------------------------------------------------------------ producer: K tiles, then V tiles
     if (lane == 0) {
-      if (stats_by_tma) {
-        const uint32_t bytes = (uint32_t)align_up((size_t)live0, 4) * 4;
-        if (bytes > 0) {
-          mbar_expect_tx(sm.stats_full, 4 * bytes);
-          bulk_g2s(sm.s, p.s + unit_st, bytes, sm.stats_full);
-          bulk_g2s(sm.q, p.q + unit_st, bytes, sm.stats_full);
-          bulk_g2s(sm.n, p.n + unit_st, bytes, sm.stats_full);
-          bulk_g2s(sm.pos, p.pos + unit_st, bytes, sm.stats_full);
-        } else {
-          mbar_arrive(sm.stats_full);
-        }
-      }
       for (int g = 0; g < 2 * n_tiles; ++g) {
         const int st = g % stages;
         if (g >= stages) mbar_wait(&sm.empty[st], ((g / stages) - 1) & 1, abort_flag, p.status);
@@ -192,32 +171,23 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     // ------------------------------------------------------------ policy: scope, victim, in-place overwrite
     const int ptid = tid - kPolicyWarp0 * 32;
     const int t_new = p.t_next[u];  // read by these warps only: they also write the incremented value
-    if (!stats_by_tma) {            // odd budgets: plain loads
-      for (int j = ptid; j < live0; j += kPolicyThreads) {
-        sm.s[j] = p.s[unit_st + j]; sm.q[j] = p.q[unit_st + j];
-        sm.n[j] = p.n[unit_st + j]; sm.pos[j] = p.pos[unit_st + j];
-      }
-    }
     named_bar_sync(kBarPolicy, kPolicyThreads);
-    if (!stats_by_tma && ptid == 0) mbar_arrive(sm.stats_full);
-    mbar_wait(sm.stats_full, 0, abort_flag, p.status);
     if (!evict_first) mbar_wait(sm.stats_done, 0, abort_flag, p.status);  // select on the updated statistics
     int e = live0, ev_slot = -1, ev_pos = -1;
     if (full) {
       // Sec. 4: "when the buffer is full, an eviction policy is executed"
       const int m = scope_size(B, p.r, p.scope_mode);
-      e = group_select_victim(sm.s, sm.q, sm.n, sm.pos, B, m, sm.vkey, *sm.sel, ptid, kPolicyThreads, kBarPolicy);
+      e = group_select_victim(p.s + unit_st, p.q + unit_st, p.n + unit_st, p.pos + unit_st, B, m, sm.vkey, sm.mkey,
+                              *sm.sel, ptid, kPolicyThreads, kBarPolicy);
       if (e < 0) {
         if (ptid == 0) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
         e = 0;
       }
       ev_slot = e;
-      ev_pos = sm.pos[e];
+      if (ptid == 0) ev_pos = p.pos[unit_st + e];
     }
-    named_bar_sync(kBarPolicy, kPolicyThreads);  // everyone has read pos[e]
     // the new token takes the slot with empty statistics
     if (ptid == 0) {
-      sm.s[e] = 0.f; sm.q[e] = 0.f; sm.n[e] = 0; sm.pos[e] = t_new;
       sm.ctl[1] = e;
       p.pos[unit_st + e] = t_new;
       p.ev_slot[u] = ev_slot;
@@ -252,6 +222,12 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     const size_t o = (size_t)u * D + tid;
     sm.qf[tid] = Elem<T>::load((const T *)p.qv + o);
     if (evict_first) sm.vnew[tid] = Elem<T>::load((const T *)p.v_new + o);
+  }
+  // the statistics are needed after the K pass: pull their lines into L2 now (32 floats per line)
+  for (int j = tid * 32; j < live0; j += kConsumers * 32) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.s + unit_st + j));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.q + unit_st + j));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.n + unit_st + j));
   }
   named_bar_sync(kBarConsumers, kConsumers);
 
@@ -291,8 +267,6 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     mbar_wait(sm.policy_done, 0, abort_flag, p.status);
     e_sub = sm.ctl[1];
     if (e_sub < 0 || e_sub >= B) e_sub = 0;  // only after an aborted wait
-  } else {
-    mbar_wait(sm.stats_full, 0, abort_flag, p.status);
   }
   named_bar_sync(kBarConsumers, kConsumers);  // all scores are in shared memory
   if (tid == 0 && e_sub >= 0) sm.z[e_sub] = *sm.znew;
@@ -313,15 +287,15 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
   for (int j = tid; j < live_att; j += kConsumers) {
     const float pj = sm.z[j] * inv;
     sm.z[j] = pj;
-    // statistics of Sec. 4.3: Acc, Acc^square, Count
-    const float sj = sm.s[j] + pj, qj = fmaf(pj, pj, sm.q[j]);
-    const int nj = sm.n[j] + 1;
-    p.s[unit_st + j] = sj;
-    p.q[unit_st + j] = qj;
-    p.n[unit_st + j] = nj;
-    if (!evict_first) { sm.s[j] = sj; sm.q[j] = qj; sm.n[j] = nj; }
+    // statistics of Sec. 4.3: Acc, Acc^square, Count (the slot of the new token starts from zero)
+    const bool fresh = (j == e_sub) || (j >= live0);
+    const float s0 = fresh ? 0.f : p.s[unit_st + j], q0 = fresh ? 0.f : p.q[unit_st + j];
+    const int n0 = fresh ? 0 : p.n[unit_st + j];
+    p.s[unit_st + j] = s0 + pj;
+    p.q[unit_st + j] = fmaf(pj, pj, q0);
+    p.n[unit_st + j] = n0 + 1;
   }
-  if (!evict_first) {  // hand the updated statistics to the policy warp
+  if (!evict_first) {  // hand the updated statistics to the policy warps
     __syncwarp();
     if (lane == 0) mbar_arrive(sm.stats_done);
   }
@@ -384,10 +358,12 @@ static cudaError_t launch_decode_t(const DecodeParams &p, int U, cudaStream_t st
 
 // Tile size and ring depth: 16 KiB tiles and the deepest ring (3..6 stages) that still lets the most CTAs
 // share an SM; budgets too large for that fall back to 8 KiB tiles.
+constexpr int kMaxCtasPerSm = 3;
+
 template <int TILE>
 static int pick_stages(int B, int d) {
   const size_t per_sm = 227 * 1024;
-  for (int ctas = 3; ctas >= 1; --ctas) {
+  for (int ctas = kMaxCtasPerSm; ctas >= 1; --ctas) {
     for (int st = 6; st >= 3; --st)
       if ((decode_smem_bytes<TILE>(B, d, st) + 1024) * ctas <= per_sm) return st;
   }

@@ -96,15 +96,21 @@ __device__ __forceinline__ uint32_t variance_key_fast(float s, float q, int n) {
 
 __device__ __forceinline__ float mean_fast(float s, int n) { return __fdiv_rn(s, (float)n); }
 
-// Victim slot among slots [0, live) given scope size m (1 <= m <= live).  s, q, n, pos and vkey are
-// shared-memory arrays; vkey[live] is scratch.  Returns -1 if no slot qualifies (NaN statistics).
+// Victim slot among slots [0, live) given scope size m (1 <= m <= live).  s, q, n, pos are the unit's
+// statistics in GLOBAL memory (each read once, coalesced; positions only where a tie has to be broken);
+// vkey[live] and mkey[live] are shared-memory scratch.  Returns -1 if no slot qualifies (NaN statistics).
 // Called by the `nthreads` threads (a multiple of 32) that synchronise on named barrier `bar_id`; every one
 // of them gets the same return value.
 __device__ __forceinline__ int group_select_victim(const float *s, const float *q, const int *n, const int *pos,
-                                                   int live, int m, uint32_t *vkey, SelectScratch &sc, int tid,
-                                                   int nthreads, int bar_id) {
+                                                   int live, int m, uint32_t *vkey, float *mkey, SelectScratch &sc,
+                                                   int tid, int nthreads, int bar_id) {
 #pragma unroll 4
-  for (int j = tid; j < live; j += nthreads) vkey[j] = variance_key_fast(s[j], q[j], n[j]);
+  for (int j = tid; j < live; j += nthreads) {
+    const float sj = s[j], qj = q[j];
+    const int nj = n[j];
+    vkey[j] = variance_key_fast(sj, qj, nj);
+    mkey[j] = mean_fast(sj, nj);
+  }
   named_bar_sync(bar_id, nthreads);
   uint32_t T = 0xffffffffu;
   int P = 0x7fffffff;
@@ -119,15 +125,17 @@ __device__ __forceinline__ int group_select_victim(const float *s, const float *
     }
   }
   float bm = INFINITY;
-  int bp = 0x7fffffff, bs = -1;
+  int bs = -1;
 #pragma unroll 4
   for (int j = tid; j < live; j += nthreads) {
     const uint32_t k = vkey[j];
-    const bool in_scope = (k < T) || (k == T && pos[j] <= P);
-    if (!in_scope) continue;
-    const float mean = mean_fast(s[j], n[j]);
-    if (mean < bm || (mean == bm && pos[j] < bp)) { bm = mean; bp = pos[j]; bs = j; }
+    if (k > T) continue;
+    if (k == T && P != 0x7fffffff && pos[j] > P) continue;
+    const float mean = mkey[j];
+    if (mean < bm) { bm = mean; bs = j; }
+    else if (mean == bm && bs >= 0 && pos[j] < pos[bs]) bs = j;
   }
+  int bp = (bs >= 0) ? pos[bs] : 0x7fffffff;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     const float om = __shfl_xor_sync(0xffffffffu, bm, o);
