@@ -4,11 +4,12 @@
 //   - a producer warp streams the unit's K block, then its V block, exactly once, through a shared-memory
 //     ring filled by bulk asynchronous copies (TMA, non-multicast);
 //   - eight consumer warps turn K tiles into scores (kept in shared memory: B floats, no online softmax),
-//     normalise, update Acc / Acc^square / Count in global memory (read once, written once), then turn V
-//     tiles into the output;
-//   - four policy warps build the eviction scope and pick the victim (Sec. 4.3) *while* the consumers stream:
-//     under EVICT_FIRST they work during the K pass (the new token's score and value are patched in
-//     afterwards, so the stream never waits for the decision), under ATTEND_FIRST during the V pass.
+//     normalise, then turn V tiles into the output;
+//   - four policy warps build the eviction scope and pick the victim (Sec. 4.3) and update Acc / Acc^square /
+//     Count in global memory (read once, written once) *while* the consumers stream: under EVICT_FIRST the
+//     selection runs during the K pass (the new token's score and value are patched in afterwards, so the
+//     stream never waits for the decision) and the statistics update during the V pass; under ATTEND_FIRST
+//     both run during the V pass.
 // The freed slot is overwritten in place; the cache is never compacted.
 #include "common.cuh"
 #include "launch.h"
@@ -46,7 +47,7 @@ struct DecodeSmem {
   SelectScratch *sel;  // policy warps: histogram and reduction scratch
   float *qf, *vnew, *outred, *red;
   uint64_t *full, *empty;  // ring barriers
-  uint64_t *stats_done;    // consumers have written the updated statistics (ATTEND_FIRST: policy may start)
+  uint64_t *p_ready;       // consumers have left the probabilities in shared memory
   uint64_t *policy_done;   // victim chosen, new K/V written
   int *ctl;                // [0] abort flag, [1] slot of the new token
   float *znew;             // score of the new token (EVICT_FIRST)
@@ -81,7 +82,7 @@ __device__ inline DecodeSmem carve(char *raw, int B, int d, int stages) {
   m.red = (float *)p; p += 64 * 4;
   m.full = (uint64_t *)p; p += stages * sizeof(uint64_t);
   m.empty = (uint64_t *)p; p += stages * sizeof(uint64_t);
-  m.stats_done = (uint64_t *)p; p += sizeof(uint64_t);
+  m.p_ready = (uint64_t *)p; p += sizeof(uint64_t);
   m.policy_done = (uint64_t *)p; p += sizeof(uint64_t);
   m.ctl = (int *)p; p += 4 * 4;
   m.znew = (float *)p;
@@ -132,7 +133,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
 
   if (tid == 0) {
     for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kConsumerWarps); }
-    mbar_init(sm.stats_done, kConsumerWarps);
+    mbar_init(sm.p_ready, kConsumerWarps);
     mbar_init(sm.policy_done, 1);
     sm.ctl[0] = 0;
     mbar_init_fence();
@@ -172,7 +173,25 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     const int ptid = tid - kPolicyWarp0 * 32;
     const int t_new = p.t_next[u];  // read by these warps only: they also write the incremented value
     named_bar_sync(kBarPolicy, kPolicyThreads);
-    if (!evict_first) mbar_wait(sm.stats_done, 0, abort_flag, p.status);  // select on the updated statistics
+    // statistics of Sec. 4.3 for the slots the query attended over: Acc += p, Acc^square += p^2, Count += 1
+    // (a slot that has just received the new token starts from zero)
+    auto update_statistics = [&](int fresh_slot) {
+      mbar_wait(sm.p_ready, 0, abort_flag, p.status);
+#pragma unroll 4
+      for (int j = ptid; j < live_att; j += kPolicyThreads) {
+        const bool fresh = (j == fresh_slot) || (j >= live0);
+        const float pj = sm.z[j];
+        const float s0 = fresh ? 0.f : p.s[unit_st + j], q0 = fresh ? 0.f : p.q[unit_st + j];
+        const int n0 = fresh ? 0 : p.n[unit_st + j];
+        p.s[unit_st + j] = s0 + pj;
+        p.q[unit_st + j] = fmaf(pj, pj, q0);
+        p.n[unit_st + j] = n0 + 1;
+      }
+    };
+    if (!evict_first) {  // select on the updated statistics
+      update_statistics(-1);
+      named_bar_sync(kBarPolicy, kPolicyThreads);
+    }
     int e = live0, ev_slot = -1, ev_pos = -1;
     if (full) {
       // Sec. 4: "when the buffer is full, an eviction policy is executed"
@@ -214,6 +233,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     }
     named_bar_sync(kBarPolicy, kPolicyThreads);
     if (ptid == 0) mbar_arrive(sm.policy_done);
+    if (evict_first) update_statistics(e);
     return;
   }
 
@@ -222,12 +242,6 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     const size_t o = (size_t)u * D + tid;
     sm.qf[tid] = Elem<T>::load((const T *)p.qv + o);
     if (evict_first) sm.vnew[tid] = Elem<T>::load((const T *)p.v_new + o);
-  }
-  // the statistics are needed after the K pass: pull their lines into L2 now (32 floats per line)
-  for (int j = tid * 32; j < live0; j += kConsumers * 32) {
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.s + unit_st + j));
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.q + unit_st + j));
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.n + unit_st + j));
   }
   named_bar_sync(kBarConsumers, kConsumers);
 
@@ -287,18 +301,10 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
   for (int j = tid; j < live_att; j += kConsumers) {
     const float pj = sm.z[j] * inv;
     sm.z[j] = pj;
-    // statistics of Sec. 4.3: Acc, Acc^square, Count (the slot of the new token starts from zero)
-    const bool fresh = (j == e_sub) || (j >= live0);
-    const float s0 = fresh ? 0.f : p.s[unit_st + j], q0 = fresh ? 0.f : p.q[unit_st + j];
-    const int n0 = fresh ? 0 : p.n[unit_st + j];
-    p.s[unit_st + j] = s0 + pj;
-    p.q[unit_st + j] = fmaf(pj, pj, q0);
-    p.n[unit_st + j] = n0 + 1;
   }
-  if (!evict_first) {  // hand the updated statistics to the policy warps
-    __syncwarp();
-    if (lane == 0) mbar_arrive(sm.stats_done);
-  }
+  // hand the probabilities to the policy warps (statistics update) before streaming V
+  __syncwarp();
+  if (lane == 0) mbar_arrive(sm.p_ready);
   if (tid == 0 && p.lse) p.lse[u] = (live_att > 0) ? (zmax + log2f(zsum)) * kLn2 : -INFINITY;
   named_bar_sync(kBarConsumers, kConsumers);  // all probabilities are in shared memory
 
