@@ -88,6 +88,10 @@ const char *roco_status_string(int st);
 /* Bytes of device workspace roco_prefill needs for prompts of up to Lmax tokens (host function). */
 size_t roco_prefill_workspace_bytes(const roco_cache *cache, int Lmax);
 
+/* The same for ROCO_SCOPE_LOWEST_R when a prompt is longer than the budget: that mode replays the evictions one
+ * by one on a sorted order and needs 8 more bytes per token, rounded up to a power of two (host function). */
+size_t roco_prefill_workspace_bytes_lowest_r(const roco_cache *cache, int Lmax);
+
 /* 1 if roco_prefill will run the score contraction of Eq. 1 on the tensor cores for this cache's dtype and
  * head dimension (bf16, d = 128), 0 if it will use the CUDA-core path (host function). */
 int roco_prefill_uses_tensor_cores(const roco_cache *cache);
@@ -105,7 +109,8 @@ int roco_prefill_uses_tensor_cores(const roco_cache *cache);
  *   Q, K, V        [S][G][Lmax][d], cache->kv_dtype; rows >= lens_host[b] are ignored
  *   lens_host      [S] HOST array, 1 <= lens <= Lmax (all units of a sequence share the length)
  *   B              must equal cache->B;   r: 0 <= r <= B
- *   scope_mode     ROCO_SCOPE_EXCLUDE_TOP_R (ROCO_SCOPE_LOWEST_R: ROCO_ERR_UNSUPPORTED when lens > B)
+ *   scope_mode     ROCO_SCOPE_EXCLUDE_TOP_R, or ROCO_SCOPE_LOWEST_R (then, when lens > B: r <= 2048, else
+ *                  ROCO_ERR_UNSUPPORTED, and the workspace of roco_prefill_workspace_bytes_lowest_r)
  *   count_self     1: a token's own query counts towards its statistics (0: ROCO_ERR_UNSUPPORTED)
  *   scale          multiplies Q.K (1/sqrt(d) in Eq. 1)
  *   lse_out        [S][G][Lmax] row log-sum-exp, or NULL

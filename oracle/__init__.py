@@ -26,6 +26,7 @@ def lib():
         _lib = C.CDLL(build_library())
         _lib.roco_oracle_threads.restype = C.c_int
         _lib.roco_oracle_select.restype = C.c_int
+        _lib.roco_oracle_select_to_budget_iterated.restype = C.c_int
         _lib.roco_oracle_attention_row.restype = C.c_double
         _lib.roco_oracle_select_to_budget_onepass.restype = C.c_int
         _lib.roco_oracle_prefill_unit.restype = C.c_int
@@ -79,11 +80,11 @@ def select(s, q, n, pos, r, mode, delta=1e-5):
     return int(slot), bool(near.value), int(m.value)
 
 
-def select_to_budget_iterated(s, q, n, B, r, mode):
+def select_to_budget_iterated(s, q, n, B, r, mode, delta=0.0):
     s, q, n = _f64(s), _f64(q), _i32(n)
     keep = np.zeros(len(s), np.int32)
     lib().roco_oracle_select_to_budget_iterated(_p(s), _p(q), _p(n), C.c_int(len(s)), C.c_int(B), C.c_int(r),
-                                                C.c_int(mode), _p(keep))
+                                                C.c_int(mode), C.c_double(delta), _p(keep))
     return keep.astype(bool)
 
 

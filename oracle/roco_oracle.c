@@ -199,21 +199,26 @@ int roco_oracle_select(const double *s, const double *q, const int *n, const int
 }
 
 /* Select-to-budget, literal form: apply the per-step rule L-B times on frozen statistics, removing the
- * victim each time.  keep[j] = 1 for survivors.  Works for both scope modes. */
-void roco_oracle_select_to_budget_iterated(const double *s, const double *q, const int *n, int L, int B, int r,
-                                           int mode, int *keep) {
+ * victim each time.  keep[j] = 1 for survivors.  Works for both scope modes.  Returns how many of the
+ * iterations were near-ties at relative margin delta (after one, later iterations may legitimately differ). */
+int roco_oracle_select_to_budget_iterated(const double *s, const double *q, const int *n, int L, int B, int r,
+                                          int mode, double delta, int *keep) {
+  int n_near = 0;
   for (int j = 0; j < L; ++j) keep[j] = 1;
-  if (L <= B) return;
+  if (L <= B) return 0;
   double *cs = (double *)malloc(sizeof(double) * (size_t)L), *cq = (double *)malloc(sizeof(double) * (size_t)L);
   int *cn = (int *)malloc(sizeof(int) * (size_t)L), *cp = (int *)malloc(sizeof(int) * (size_t)L);
   for (int alive = L; alive > B; --alive) {
     int k = 0;
     for (int j = 0; j < L; ++j)
       if (keep[j]) { cs[k] = s[j]; cq[k] = q[j]; cn[k] = n[j]; cp[k] = j; ++k; }
-    int slot = roco_oracle_select(cs, cq, cn, cp, alive, r, mode, 0.0, NULL, NULL);
+    int near = 0;
+    int slot = roco_oracle_select(cs, cq, cn, cp, alive, r, mode, delta, &near, NULL);
+    n_near += near;
     keep[cp[slot]] = 0;
   }
   free(cs); free(cq); free(cn); free(cp);
+  return n_near;
 }
 
 typedef struct { double key; double eps; int pos; } rank_t;
@@ -284,7 +289,8 @@ int roco_oracle_select_to_budget_onepass(const double *s, const double *q, const
  * order.  Q,K,V: [L][d].  Cache outputs: Kc,Vc [B][d]; sc,qc [B]; nc,posc [B] (pos = -1 for empty);
  * *live = min(L,B).  s_full,q_full,n_full: [L] pre-eviction statistics (required).  keep_io [L]:
  * if force_keep != 0 it is read as the survivor set to use; otherwise it receives the oracle's own.
- * uncertain [L] may be NULL.  LOWEST_R uses the iterated form (no margin analysis). */
+ * uncertain [L] may be NULL.  LOWEST_R uses the iterated form; there every token is marked uncertain as
+ * soon as one iteration was a near-tie. */
 int roco_oracle_prefill_unit(const double *Q, const double *K, const double *V, int L, int d, int B, int r,
                              int mode, double scale, int count_self, double delta, double *Kc, double *Vc,
                              double *sc, double *qc, int *nc, int *posc, int *live, double *lse, double *s_full,
@@ -295,8 +301,8 @@ int roco_oracle_prefill_unit(const double *Q, const double *K, const double *V, 
     if (mode == ROCO_ORACLE_EXCLUDE_TOP_R && count_self)
       rc = roco_oracle_select_to_budget_onepass(s_full, q_full, n_full, L, B, r, delta, keep_io, uncertain);
     else {
-      roco_oracle_select_to_budget_iterated(s_full, q_full, n_full, L, B, r, mode, keep_io);
-      if (uncertain) for (int j = 0; j < L; ++j) uncertain[j] = 0;
+      int n_near = roco_oracle_select_to_budget_iterated(s_full, q_full, n_full, L, B, r, mode, delta, keep_io);
+      if (uncertain) for (int j = 0; j < L; ++j) uncertain[j] = n_near > 0; /* no finer analysis for this form */
     }
     if (rc) return rc;
   }

@@ -20,7 +20,7 @@ ROCO_SCOPE_EXCLUDE_TOP_R, ROCO_SCOPE_LOWEST_R = 0, 1
 ROCO_EVICT_FIRST, ROCO_ATTEND_FIRST = 0, 1
 
 EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes", "roco_prefill",
-           "roco_prefill_uses_tensor_cores", "roco_prefill_static",
+           "roco_prefill_uses_tensor_cores", "roco_prefill_static", "roco_prefill_workspace_bytes_lowest_r",
            "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status")
 
 
@@ -52,6 +52,8 @@ def lib() -> C.CDLL:
         L.roco_status_string.argtypes = [C.c_int]
         L.roco_prefill_workspace_bytes.restype = C.c_size_t
         L.roco_prefill_workspace_bytes.argtypes = [C.POINTER(roco_cache), C.c_int]
+        L.roco_prefill_workspace_bytes_lowest_r.restype = C.c_size_t
+        L.roco_prefill_workspace_bytes_lowest_r.argtypes = [C.POINTER(roco_cache), C.c_int]
         L.roco_prefill_uses_tensor_cores.restype = C.c_int
         L.roco_prefill_uses_tensor_cores.argtypes = [C.POINTER(roco_cache)]
         L.roco_decode_host_staging_bytes.restype = C.c_size_t
@@ -118,6 +120,10 @@ def roco_prefill_workspace_bytes(cache: Cache, Lmax: int) -> int:
     return int(lib().roco_prefill_workspace_bytes(C.byref(cache.c), Lmax))
 
 
+def roco_prefill_workspace_bytes_lowest_r(cache: Cache, Lmax: int) -> int:
+    return int(lib().roco_prefill_workspace_bytes_lowest_r(C.byref(cache.c), Lmax))
+
+
 def roco_prefill_uses_tensor_cores(cache: Cache) -> bool:
     return bool(lib().roco_prefill_uses_tensor_cores(C.byref(cache.c)))
 
@@ -129,7 +135,9 @@ def roco_prefill(Q, K, V, lens: Sequence[int], B: int, r: int, cache: Cache, sco
     Lmax = Q.shape[2]
     scale = cache.d ** -0.5 if scale is None else scale
     if workspace is None:
-        workspace = torch.empty(roco_prefill_workspace_bytes(cache, Lmax), dtype=torch.uint8, device=Q.device)
+        nbytes = (roco_prefill_workspace_bytes_lowest_r if scope_mode == ROCO_SCOPE_LOWEST_R
+                  else roco_prefill_workspace_bytes)(cache, Lmax)
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=Q.device)
     lens_arr = (C.c_int32 * len(lens))(*[int(x) for x in lens])
     rc = lib().roco_prefill(_ptr(Q), _ptr(K), _ptr(V), C.cast(lens_arr, C.c_void_p), Lmax, B, r, scope_mode,
                             count_self, scale, C.byref(cache.c), _ptr(lse_out), _ptr(s_full), _ptr(q_full),

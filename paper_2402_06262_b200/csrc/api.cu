@@ -47,6 +47,12 @@ PrefillWs prefill_ws(int S, int G, int Lmax) {
   return w;
 }
 
+int pow2_at_least(int x) {
+  int p = 1;
+  while (p < x) p <<= 1;
+  return p;
+}
+
 }  // namespace
 
 extern "C" {
@@ -70,6 +76,11 @@ size_t roco_prefill_workspace_bytes(const roco_cache *cache, int Lmax) {
   return prefill_ws(cache->S, cache->G, Lmax).total;
 }
 
+size_t roco_prefill_workspace_bytes_lowest_r(const roco_cache *cache, int Lmax) {
+  if (!cache || Lmax < 1 || cache->S < 1 || cache->G < 1) return 0;
+  return prefill_ws(cache->S, cache->G, Lmax).total + (size_t)cache->S * cache->G * pow2_at_least(Lmax) * 8;
+}
+
 int roco_prefill_uses_tensor_cores(const roco_cache *cache) {
   return (cache && prefill_tc_supported(cache->kv_dtype, cache->d)) ? 1 : 0;
 }
@@ -88,10 +99,12 @@ roco_status roco_prefill(const void *Q, const void *K, const void *V, const int3
     if (lens_host[b] < 1 || lens_host[b] > Lmax) return ROCO_ERR_INVALID_ARG;
     if (lens_host[b] > maxlen) maxlen = lens_host[b];
   }
-  if (scope_mode == ROCO_SCOPE_LOWEST_R && maxlen > B) return ROCO_ERR_UNSUPPORTED;
+  const bool lowest_evicts = scope_mode == ROCO_SCOPE_LOWEST_R && maxlen > B;
+  if (lowest_evicts && r > budget_lowest_max_r()) return ROCO_ERR_UNSUPPORTED;
   if ((long long)cache->S * cache->G * ((maxlen + 63) / 64 + 1) > 0x7fffffffLL) return ROCO_ERR_UNSUPPORTED;
   const PrefillWs w = prefill_ws(cache->S, cache->G, Lmax);
-  if (!workspace || workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+  const size_t need = lowest_evicts ? roco_prefill_workspace_bytes_lowest_r(cache, Lmax) : w.total;
+  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
     return ROCO_ERR_WORKSPACE;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   char *ws = static_cast<char *>(workspace);
@@ -109,7 +122,8 @@ roco_status roco_prefill(const void *Q, const void *K, const void *V, const int3
     st = launch_prefill_stats_simt(cache->kv_dtype, cache->d, cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, scale,
                                    lse, sf, qf, cs);
   if (st != ROCO_OK) return st;
-  return launch_budget_select_gather(*cache, Lmax, lens_dev, maxlen, r, K, V, sf, qf, dst, cs);
+  return launch_budget_select_gather(*cache, Lmax, lens_dev, maxlen, r, scope_mode, K, V, sf, qf, dst,
+                                     reinterpret_cast<unsigned long long *>(ws + w.total), pow2_at_least(Lmax), cs);
 }
 
 roco_status roco_decode_step(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,

@@ -87,6 +87,118 @@ __global__ void __launch_bounds__(kBudgetThreads) budget_select_kernel(const flo
   }
 }
 
+// LOWEST_R has no one-pass form: the scope (the r lowest-variance tokens still alive) gains a member every time
+// the victim leaves it.  With frozen statistics the members enter in (variance, position) order, so the kernel
+// sorts the tokens once by that order (bitonic sort of 64-bit keys = variance bits : position, in the caller's
+// scratch) and then one warp replays the L-B evictions on a scope held in shared memory: pop the lowest
+// (mean, position), admit the next token of the sorted order.  One CTA per unit.
+constexpr int kLowestMaxR = 2048;
+
+__global__ void __launch_bounds__(kBudgetThreads) budget_lowest_kernel(const float *s_full, const float *q_full,
+                                                                       const int *lens, int G, int Lmax, int Lp2max,
+                                                                       int B, int r, unsigned long long *sortbuf,
+                                                                       int *dst, int *live, int *t_next) {
+  __shared__ float sc_mean[kLowestMaxR];
+  __shared__ int sc_idx[kLowestMaxR];
+  __shared__ int warp_tot[kBudgetThreads / 32];
+  __shared__ int base_sh;
+  const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int L = lens[u / G];
+  const float *s = s_full + (size_t)u * Lmax, *q = q_full + (size_t)u * Lmax;
+  int *du = dst + (size_t)u * Lmax;
+  unsigned long long *keys = sortbuf + (size_t)u * Lp2max;
+  if (tid == 0) { live[u] = L < B ? L : B; t_next[u] = L; }
+  if (L <= B) {
+    for (int j = tid; j < L; j += kBudgetThreads) du[j] = j;
+    return;
+  }
+  int Lp2 = 1;
+  while (Lp2 < L) Lp2 <<= 1;
+  for (int j = tid; j < Lp2; j += kBudgetThreads) {
+    unsigned long long k = ~0ull;
+    if (j < L) {
+      k = ((unsigned long long)__float_as_uint((float)variance_f64(s[j], q[j], L - j)) << 32) | (unsigned)j;
+      du[j] = 0;  // 0 = alive, -1 = evicted (turned into slots at the end)
+    }
+    keys[j] = k;
+  }
+  __syncthreads();
+  for (int k = 2; k <= Lp2; k <<= 1) {
+    for (int jj = k >> 1; jj > 0; jj >>= 1) {
+      for (int i = tid; i < Lp2; i += kBudgetThreads) {
+        const int p = i ^ jj;
+        if (p > i) {
+          const unsigned long long a = keys[i], b = keys[p];
+          const bool up = (i & k) == 0;
+          if ((a > b) == up) { keys[i] = b; keys[p] = a; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  if (warp == 0) {
+    const int rs = r < L ? r : L;
+    for (int k = lane; k < rs; k += 32) {
+      const int j = (int)(keys[k] & 0xffffffffu);
+      sc_idx[k] = j;
+      sc_mean[k] = mean_fast(s[j], L - j);
+    }
+    __syncwarp();
+    int cursor = rs;
+    for (int it = 0; it < L - B; ++it) {
+      float bm = INFINITY;
+      int bi = 0x7fffffff, bk = -1;
+      for (int k = lane; k < rs; k += 32) {
+        const float m = sc_mean[k];
+        const int j = sc_idx[k];
+        if (m < bm || (m == bm && j < bi)) { bm = m; bi = j; bk = k; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, bm, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        const int ok = __shfl_xor_sync(0xffffffffu, bk, o);
+        if (ok >= 0 && (bk < 0 || om < bm || (om == bm && oi < bi))) { bm = om; bi = oi; bk = ok; }
+      }
+      if (bk < 0) break;  // NaN statistics everywhere: nothing left to pop
+      if (lane == 0) {
+        du[bi] = -1;
+        if (cursor < L) {
+          const int j = (int)(keys[cursor] & 0xffffffffu);
+          sc_idx[bk] = j;
+          sc_mean[bk] = mean_fast(s[j], L - j);
+        } else {
+          sc_idx[bk] = 0x7fffffff;
+          sc_mean[bk] = INFINITY;
+        }
+      }
+      ++cursor;
+      __syncwarp();
+    }
+  }
+  // survivors keep their order: exclusive prefix sum of the keep flags
+  if (tid == 0) base_sh = 0;
+  __syncthreads();
+  for (int j0 = 0; j0 < L; j0 += kBudgetThreads) {
+    const int j = j0 + tid;
+    const bool keep = j < L && du[j] == 0;
+    const uint32_t bal = __ballot_sync(0xffffffffu, keep);
+    const int before = __popc(bal & ((1u << lane) - 1u));
+    if (lane == 0) warp_tot[warp] = __popc(bal);
+    __syncthreads();
+    int off = base_sh;
+    for (int w = 0; w < warp; ++w) off += warp_tot[w];
+    if (j < L) du[j] = keep ? off + before : -1;
+    __syncthreads();
+    if (tid == 0) {
+      int t = 0;
+      for (int w = 0; w < kBudgetThreads / 32; ++w) t += warp_tot[w];
+      base_sh += t;
+    }
+    __syncthreads();
+  }
+}
+
 // grid U * chunks (unit-major); each CTA moves up to 64 tokens.  Also clears the slots past `live`.
 template <int ROWB>
 __global__ void __launch_bounds__(256) gather_kernel(const char *K, const char *V, const float *s_full,
@@ -124,12 +236,19 @@ __global__ void __launch_bounds__(256) gather_kernel(const char *K, const char *
   }
 }
 
+int budget_lowest_max_r() { return kLowestMaxR; }
+
 roco_status launch_budget_select_gather(const roco_cache &c, int Lmax, const int *lens_dev, int maxlen, int r,
-                                        const void *K, const void *V, const float *s_full, const float *q_full,
-                                        int *dst, cudaStream_t stream) {
+                                        int scope_mode, const void *K, const void *V, const float *s_full,
+                                        const float *q_full, int *dst, unsigned long long *sortbuf, int Lp2max,
+                                        cudaStream_t stream) {
   const int U = c.S * c.G;
-  budget_select_kernel<<<U, kBudgetThreads, 0, stream>>>(s_full, q_full, lens_dev, c.G, Lmax, c.B, r, dst, c.live,
-                                                         c.t_next);
+  if (scope_mode == ROCO_SCOPE_LOWEST_R && maxlen > c.B)
+    budget_lowest_kernel<<<U, kBudgetThreads, 0, stream>>>(s_full, q_full, lens_dev, c.G, Lmax, Lp2max, c.B, r,
+                                                           sortbuf, dst, c.live, c.t_next);
+  else
+    budget_select_kernel<<<U, kBudgetThreads, 0, stream>>>(s_full, q_full, lens_dev, c.G, Lmax, c.B, r, dst, c.live,
+                                                           c.t_next);
   const int span = maxlen > c.B ? maxlen : c.B;
   const int chunks = (span + 63) / 64;
   const unsigned grid = (unsigned)U * (unsigned)chunks;

@@ -25,9 +25,12 @@ roco_status launch_prefill_stats_tc(int S, int G, int Lmax, const int *lens_dev,
                                     cudaStream_t stream);
 
 // Select-to-budget on frozen statistics and gather of the survivors into the cache.
-// dst: [U][Lmax] int32 scratch (destination slot per token, -1 = evicted).
+// dst: [U][Lmax] int32 scratch (destination slot per token, -1 = evicted).  LOWEST_R with eviction also needs
+// sortbuf: [U][Lp2max] 64-bit scratch, Lp2max = Lmax rounded up to a power of two, and r <= budget_lowest_max_r().
+int budget_lowest_max_r();
 roco_status launch_budget_select_gather(const roco_cache &c, int Lmax, const int *lens_dev, int maxlen, int r,
-                                        const void *K, const void *V, const float *s_full, const float *q_full,
-                                        int *dst, cudaStream_t stream);
+                                        int scope_mode, const void *K, const void *V, const float *s_full,
+                                        const float *q_full, int *dst, unsigned long long *sortbuf, int Lp2max,
+                                        cudaStream_t stream);
 
 }  // namespace roco

@@ -99,7 +99,8 @@ def test_prefill_rejects_bad_arguments_on_the_host():
     lens[0] = 0
     assert call() == 1
     lens[0] = 32
-    assert call(Lmax=32, mode=R.ROCO_SCOPE_LOWEST_R, wsb=1 << 30) == 2   # LOWEST_R cannot evict at prefill
+    assert call(Lmax=32, mode=R.ROCO_SCOPE_LOWEST_R, wsb=need) == 3      # LOWEST_R eviction needs the larger workspace
+    assert L.roco_prefill_workspace_bytes_lowest_r(C.byref(c), 32) > L.roco_prefill_workspace_bytes(C.byref(c), 32)
     assert L.roco_prefill_workspace_bytes(None, 8) == 0
     assert L.roco_decode_host_staging_bytes(C.byref(c)) >= 4 * 2 * 128 * 2
 

@@ -29,8 +29,7 @@ def run_workload(w, units, mode, order, steps, lens=None, check_every=8, Lmax=No
     Lmax = max(lens) if Lmax is None else Lmax
     Q, K, V = prompt_tensors(w, Lmax)
     cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
-    pmode = mode if max(lens) <= w.B else R.ROCO_SCOPE_EXCLUDE_TOP_R   # LOWEST_R cannot evict at prefill
-    st = prefill_parity(cache, Q, K, V, lens, w.r, pmode, units, tally, scale=w.scale)
+    st = prefill_parity(cache, Q, K, V, lens, w.r, mode, units, tally, scale=w.scale)
     par = DecodeParity(cache, st, units, w.r, mode, order, tally, scale=w.scale)
     t_pos = list(lens)
     for i in range(steps):
@@ -68,6 +67,13 @@ def test_prefill_eviction_structured(kind):
     t = run_workload(w, range(w.U), R.ROCO_SCOPE_EXCLUDE_TOP_R, R.ROCO_EVICT_FIRST, 12, lens=[700, 333, 65],
                      check_every=4)
     assert t.prefill_swapped <= 4, t
+
+
+@pytest.mark.parametrize("r", [1, 31, 200])
+def test_prefill_eviction_lowest_r(r):
+    """LOWEST_R at prefill: the evictions are replayed one by one on frozen statistics (sorted scope order)."""
+    w = W.scaled(W.LLAMA7B_PREFILL, S=3, layers=1, heads=3, prompt_lo=700, prompt_hi=700, B=200, r=r, kind="sink")
+    run_workload(w, range(w.U), R.ROCO_SCOPE_LOWEST_R, R.ROCO_EVICT_FIRST, 6, lens=[700, 333, 65], check_every=3)
 
 
 def test_prefill_keeps_everything_when_budget_not_binding():
