@@ -108,6 +108,75 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// ---- packed fp32x2 arithmetic (two lanes per instruction) and exp2 on the FMA pipe
+typedef unsigned long long f32x2;
+
+__device__ __forceinline__ f32x2 pack2(float a, float b) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 pack2u(uint32_t a, uint32_t b) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float &a, float &b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// 2^x for a pair of x <= 0 without the exponential unit: x = n + f with n the nearest integer (magic-number
+// rounding) and f in [-1/2, 1/2]; 2^f by a degree-4 polynomial (max relative error 2.7e-6, mean error 4e-8);
+// the integer n is then added to the exponent field.  x is clamped at -125 (results below 2^-125 are noise
+// for the sums they enter).
+__device__ __forceinline__ f32x2 exp2_poly2(f32x2 x2) {
+  float xa, xb;
+  unpack2(x2, xa, xb);
+  x2 = pack2(fmaxf(xa, -125.f), fmaxf(xb, -125.f));
+  const f32x2 magic = pack2(12582912.f, 12582912.f);  // 1.5 * 2^23: the low mantissa bits hold n
+  const f32x2 t2 = add2(x2, magic);
+  const f32x2 n2 = add2(t2, pack2(-12582912.f, -12582912.f));
+  const f32x2 f2 = fma2(n2, pack2(-1.f, -1.f), x2);
+  f32x2 p2 = fma2(f2, pack2(0.009570101276040077f, 0.009570101276040077f),
+                  pack2(0.05591785907745361f, 0.05591785907745361f));
+  p2 = fma2(p2, f2, pack2(0.240247443318367f, 0.240247443318367f));
+  p2 = fma2(p2, f2, pack2(0.6931217908859253f, 0.6931217908859253f));
+  p2 = fma2(p2, f2, pack2(0.9999992847442627f, 0.9999992847442627f));
+  float ta, tb, pa, pb;
+  unpack2(t2, ta, tb);
+  unpack2(p2, pa, pb);
+  const uint32_t ra = __float_as_uint(pa) + (__float_as_uint(ta) << 23);
+  const uint32_t rb = __float_as_uint(pb) + (__float_as_uint(tb) << 23);
+  return pack2u(ra, rb);
+}
+
+__device__ __forceinline__ f32x2 exp2_mufu2(f32x2 x2) {
+  float xa, xb;
+  unpack2(x2, xa, xb);
+  return pack2(ex2_approx(xa), ex2_approx(xb));
+}
+
+// Of every 8 pairs, how many take the polynomial instead of the exponential unit (which is the bottleneck
+// of both passes: 16 results per cycle per SM against 128 FMA lanes).
+#ifndef ROCO_POLY_PAIRS_PER_8
+#define ROCO_POLY_PAIRS_PER_8 3
+#endif
+constexpr int kPolyPairsPer8 = ROCO_POLY_PAIRS_PER_8;
+
+__device__ __forceinline__ f32x2 exp2_pair(f32x2 x2, int pair_index) {
+  return ((pair_index & 7) < kPolyPairsPer8) ? exp2_poly2(x2) : exp2_mufu2(x2);
+}
+
 // Shared-memory matrix descriptor of a K-major bf16 operand tile stored as rows of 128 bytes with the
 // 128-byte swizzle (what TMA writes for a 64-column box): 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw128(const void *p) {
@@ -126,7 +195,7 @@ constexpr uint32_t kIdescBf16M128N128 = (1u << 4) | (1u << 7) | (1u << 10) | ((1
 struct TcSmem {
   char *stat;                 // stationary operand tile
   char *ring;                 // kTcStages streamed operand tiles
-  float *lse2;                // [2 groups][2][128] log2-domain row LSE of a group's current query tile (pass 1)
+  float *lse2;                // [2 groups][2][128] minus the log2-domain row LSE of a group's query tile (pass 1)
   float *merge;               // [2 tasks][2][128] partial running values handed from group 1 to group 0
   uint64_t *stat_full, *stat_empty;
   uint64_t *ring_full, *ring_empty;  // [kTcStages]
@@ -159,7 +228,7 @@ __device__ inline TcSmem tc_carve(char *raw) {
 // PASS 0: stationary = Q tile a, streamed = K tiles 0..a, output lse.
 // PASS 1: stationary = K tile a, streamed = Q tiles a..T-1, input lse, output s_full / q_full.
 template <int PASS>
-__global__ void __launch_bounds__(kTcThreads) prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ,
+__global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_constant__ CUtensorMap mapQ,
                                                                 const __grid_constant__ CUtensorMap mapK,
                                                                 const int *lens, int G, int Lmax, int npairs,
                                                                 float scale, float *lse, float *s_full, float *q_full,
@@ -273,7 +342,7 @@ __global__ void __launch_bounds__(kTcThreads) prefill_tc_kernel(const __grid_con
         const int j = first + t;  // streamed tile index
         float *l2 = sm.lse2 + (group * 2 + (mine & 1)) * 128;
         if (PASS == 1) {
-          l2[gtid] = lse_next * kLog2e;
+          l2[gtid] = -lse_next * kLog2e;
           if (group == 0) named_bar_sync(kTcBarGroup0, kTcGroupThreads);
           else named_bar_sync(kTcBarGroup0 + 1, kTcGroupThreads);
           const int qn = (j + 2) * kTcTile + gtid;
@@ -287,6 +356,7 @@ __global__ void __launch_bounds__(kTcThreads) prefill_tc_kernel(const __grid_con
         // one 32-column chunk of the accumulator row of this thread
         auto chunk = [&](const uint32_t (&r)[32], int c, auto masked_tag) {
           constexpr bool kMasked = decltype(masked_tag)::value;
+          const f32x2 zs2 = pack2(zscale, zscale);
           if (PASS == 0) {
             // online softmax, one rescale per chunk
             float cmax = -INFINITY;
@@ -296,34 +366,44 @@ __global__ void __launch_bounds__(kTcThreads) prefill_tc_kernel(const __grid_con
               cmax = fmaxf(cmax, ok ? __uint_as_float(r[i]) : -INFINITY);
             }
             const float m_new = fmaxf(run0, cmax * zscale);
-            float part = 0.f;
             if (m_new > -INFINITY) {
+              const f32x2 nm2 = pack2(-m_new, -m_new);
+              f32x2 part2 = pack2(0.f, 0.f);
 #pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                const bool ok = !kMasked || (col0 + c * 32 + i <= grow);
-                const float ex = ex2_approx(fmaf(__uint_as_float(r[i]), zscale, -m_new));
-                part += ok ? ex : 0.f;
+              for (int i = 0; i < 32; i += 2) {
+                f32x2 e2 = exp2_pair(fma2(pack2u(r[i], r[i + 1]), zs2, nm2), i >> 1);
+                if (kMasked) {
+                  float ea, eb;
+                  unpack2(e2, ea, eb);
+                  e2 = pack2((col0 + c * 32 + i <= grow) ? ea : 0.f, (col0 + c * 32 + i + 1 <= grow) ? eb : 0.f);
+                }
+                part2 = add2(part2, e2);
               }
-              run1 = run1 * ex2_approx(run0 - m_new) + part;
+              float pa, pb;
+              unpack2(part2, pa, pb);
+              run1 = run1 * ex2_approx(run0 - m_new) + (pa + pb);
               run0 = m_new;
             }
           } else {
-            float ts = 0.f, tq = 0.f;
+            f32x2 ts2 = pack2(0.f, 0.f), tq2 = pack2(0.f, 0.f);
+            const f32x2 *l2p = reinterpret_cast<const f32x2 *>(l2 + c * 32);  // holds -lse * log2(e)
 #pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              const float4 lv = *reinterpret_cast<const float4 *>(l2 + c * 32 + i);
-              const float lvv[4] = {lv.x, lv.y, lv.z, lv.w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int qi = col0 + c * 32 + i + e;
-                float pij = ex2_approx(fmaf(__uint_as_float(r[i + e]), zscale, -lvv[e]));
-                if (kMasked) pij = (qi >= grow && qi < L) ? pij : 0.f;
-                ts += pij;
-                tq = fmaf(pij, pij, tq);
+            for (int i = 0; i < 32; i += 2) {
+              f32x2 p2 = exp2_pair(fma2(pack2u(r[i], r[i + 1]), zs2, l2p[i >> 1]), i >> 1);
+              if (kMasked) {
+                const int qi = col0 + c * 32 + i;
+                float pa, pb;
+                unpack2(p2, pa, pb);
+                p2 = pack2((qi >= grow && qi < L) ? pa : 0.f, (qi + 1 >= grow && qi + 1 < L) ? pb : 0.f);
               }
+              ts2 = add2(ts2, p2);
+              tq2 = fma2(p2, p2, tq2);
             }
-            run0 += ts;
-            run1 += tq;
+            float a0, a1, b0, b1;
+            unpack2(ts2, a0, a1);
+            unpack2(tq2, b0, b1);
+            run0 += a0 + a1;
+            run1 += b0 + b1;
           }
         };
         auto tile = [&](auto masked_tag) {
