@@ -169,7 +169,7 @@ __device__ __forceinline__ f32x2 exp2_mufu2(f32x2 x2) {
 // Of every 8 pairs, how many take the polynomial instead of the exponential unit (which is the bottleneck
 // of both passes: 16 results per cycle per SM against 128 FMA lanes).
 #ifndef ROCO_POLY_PAIRS_PER_8
-#define ROCO_POLY_PAIRS_PER_8 3
+#define ROCO_POLY_PAIRS_PER_8 2
 #endif
 constexpr int kPolyPairsPer8 = ROCO_POLY_PAIRS_PER_8;
 
