@@ -183,3 +183,43 @@ def decode_step(st: State, qv, k_new, v_new, r, mode, order, scale, count_self=1
                                         C.c_int(count_self), C.c_double(delta), _p(fv), C.c_int(int(force_only_near)), _p(out), _p(lse), _p(es),
                                         _p(ep), _p(ch), _p(nt))
     return StepResult(out, lse, es, ep, ch, nt.astype(bool))
+
+
+@dataclass
+class BlockResult:
+    out: np.ndarray           # [U][b][d]
+    lse: np.ndarray           # [U][b]
+    evicted_slot: np.ndarray  # [U][b] ascending slots, -1 padded
+    evicted_pos: np.ndarray   # [U][b]
+    choice: np.ndarray        # [U][b] the policy's own set (differs from evicted_slot only when forced)
+    near_tie: np.ndarray      # [U] number of eviction iterations inside the decision margin
+
+
+def block_step(st: State, Q, K_new, V_new, r, mode, scale, delta=1e-5, force_slots=None) -> BlockResult:
+    """Block-wise evict-and-encode of b tokens per unit, in place on `st`.  Q, K_new, V_new: [U][b][d]."""
+    Q, K_new, V_new = _f64(Q), _f64(K_new), _f64(V_new)
+    U, b, d = Q.shape
+    out = np.zeros((U, b, d)); lse = np.zeros((U, b))
+    es = np.zeros((U, b), np.int32); ep = np.zeros((U, b), np.int32); ch = np.zeros((U, b), np.int32)
+    nt = np.zeros(U, np.int32)
+    fs = None if force_slots is None else _i32(force_slots)
+    lib().roco_oracle_block_step_batch(C.c_int(U), _p(st.K), _p(st.V), _p(st.s), _p(st.q), _p(st.n), _p(st.pos),
+                                       _p(st.live), _p(st.t_next), C.c_int(st.B), C.c_int(d), C.c_int(b), _p(Q),
+                                       _p(K_new), _p(V_new), C.c_int(r), C.c_int(mode), C.c_double(scale),
+                                       C.c_double(delta), _p(fs), _p(out), _p(lse), _p(es), _p(ep), _p(ch), _p(nt))
+    return BlockResult(out, lse, es, ep, ch, nt)
+
+
+def gqa_step(st: State, Q, k_new, v_new, r, mode, scale, delta=1e-5, force_victim=None) -> StepResult:
+    """One decode step of U key-value heads, each shared by `group` query heads.  Q: [U][group][d];
+    k_new, v_new: [U][d].  Returns out [U][group][d], lse [U][group]."""
+    Q, k_new, v_new = _f64(Q), _f64(k_new), _f64(v_new)
+    U, group, d = Q.shape
+    out = np.zeros((U, group, d)); lse = np.zeros((U, group))
+    es = np.zeros(U, np.int32); ep = np.zeros(U, np.int32); ch = np.zeros(U, np.int32); nt = np.zeros(U, np.int32)
+    fv = None if force_victim is None else _i32(force_victim)
+    lib().roco_oracle_gqa_step_batch(C.c_int(U), _p(st.K), _p(st.V), _p(st.s), _p(st.q), _p(st.n), _p(st.pos),
+                                     _p(st.live), _p(st.t_next), C.c_int(st.B), C.c_int(d), C.c_int(group), _p(Q),
+                                     _p(k_new), _p(v_new), C.c_int(r), C.c_int(mode), C.c_double(scale),
+                                     C.c_double(delta), _p(fv), _p(out), _p(lse), _p(es), _p(ep), _p(ch), _p(nt))
+    return StepResult(out, lse, es, ep, ch, nt.astype(bool))

@@ -26,6 +26,8 @@
  *   fixed buffer, evict when full .. Sec. 3 (n <= B at every step), Sec. 4 first paragraph
  *   evict before appending ......... Fig. 1 caption (EVICT_FIRST step order)
  *   prefill-stage eviction to B .... Sec. 4.3 last paragraph / Sec. 5.1 "Other Details" (B = len x rate)
+ *   block-wise evict-and-encode .... Sec. 5.3 "Overhead", App. B (b tokens freed and encoded per eviction step)
+ *   grouped-query attention ........ Sec. 5.3 / App. A (group-wise averaged attention score updates the statistics)
  *
  * Readings where the paper is silent (stated once here, in words):
  *   - ties: scope membership by (variance asc, position asc); victim by (mean asc, position asc);
@@ -34,7 +36,11 @@
  *   - statistics are raw accumulations: no reset or renormalisation after an eviction;
  *   - a freed slot is overwritten in place; while the buffer is not full the new token goes to slot
  *     `live`; after prefill the survivors sit in increasing position order;
- *   - select-to-budget at prefill = the per-step rule applied L-B times on frozen statistics.
+ *   - select-to-budget at prefill = the per-step rule applied L-B times on frozen statistics;
+ *   - a block step frees its slots the same way (rule applied on frozen statistics), the b new tokens take the
+ *     freed / free slots in increasing slot order, and attention inside the block is causal;
+ *   - grouped queries: the probabilities are averaged over the group first, then the mean enters Acc and its
+ *     square Acc^square, with one Count per step.
  *
  * Parity pins: every function here is pinned by tests that do not call it to produce their expected
  * values (hand-worked rationals, harmonic-number closed forms, library softmax/logsumexp, brute-force
@@ -420,4 +426,166 @@ int roco_oracle_prefill_batch(int U, const double *Q, const double *K, const dou
     }
   }
   return bad;
+}
+
+/* ------------------------------------------------ block-wise evict-and-encode (Sec. 5.3 "Overhead", App. B) -- */
+
+/* One eviction step that frees and encodes b tokens (Sec. 5.3: "The block size b controls the number of tokens
+ * being freed and encoded within one eviction step").  Order as in Fig. 1: evict, insert, attend.
+ *   1. need = live + b - B tokens (if positive) leave the cache: the per-step rule of Sec. 4.3 applied `need`
+ *      times on the frozen statistics, each time on the tokens still alive.
+ *   2. The b new tokens (positions t_next .. t_next+b-1) take, in order, the target slots sorted by slot index:
+ *      the freed slots and, while the buffer is not full, slots live, live+1, ...
+ *   3. Query i attends over the remaining old tokens and the new tokens 0..i (causal inside the block, Sec. 2.1);
+ *      every attended token gets Count += 1, Acc += p, Acc^square += p^2 (Sec. 4.3).
+ * Q, Kn, Vn: [b][d].  out: [b][d]; lse: [b].  evicted_slot / evicted_pos: [b], ascending slot order, -1 padded.
+ * force_slots (may be NULL): [b] slots to evict instead of the policy's, -1 padded (used only when *near_tie).
+ * *near_tie counts the eviction iterations inside the decision margin delta. */
+void roco_oracle_block_step_unit(double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
+                                 int *t_next, int B, int d, int b, const double *Q, const double *Kn,
+                                 const double *Vn, int r, int mode, double scale, double delta,
+                                 const int *force_slots, double *out, double *lse, int *evicted_slot,
+                                 int *evicted_pos, int *choice, int *near_tie) {
+  const int live0 = *live, t0 = *t_next;
+  int need = live0 + b - B;
+  if (need < 0) need = 0;
+  int *gone = (int *)calloc((size_t)B, sizeof(int));
+  int n_near = 0;
+  /* 1. policy on frozen statistics */
+  double *cs = (double *)malloc(sizeof(double) * (size_t)B), *cq = (double *)malloc(sizeof(double) * (size_t)B);
+  int *cn = (int *)malloc(sizeof(int) * (size_t)B), *cp = (int *)malloc(sizeof(int) * (size_t)B);
+  int *cslot = (int *)malloc(sizeof(int) * (size_t)B);
+  for (int it = 0; it < need; ++it) {
+    int k = 0;
+    for (int j = 0; j < live0; ++j)
+      if (!gone[j]) { cs[k] = s[j]; cq[k] = q[j]; cn[k] = n[j]; cp[k] = pos[j]; cslot[k] = j; ++k; }
+    int near = 0;
+    int c = roco_oracle_select(cs, cq, cn, cp, k, r, mode, delta, &near, NULL);
+    n_near += near;
+    gone[cslot[c]] = 1;
+  }
+  for (int i = 0; i < b; ++i) { choice[i] = -1; evicted_slot[i] = -1; evicted_pos[i] = -1; }
+  {
+    int k = 0;
+    for (int j = 0; j < live0; ++j) if (gone[j]) choice[k++] = j;
+  }
+  if (force_slots && n_near > 0) { /* continue from the other side's (in-margin) choice */
+    memset(gone, 0, sizeof(int) * (size_t)B);
+    for (int i = 0; i < b; ++i) if (force_slots[i] >= 0 && force_slots[i] < live0) gone[force_slots[i]] = 1;
+  }
+  {
+    int k = 0;
+    for (int j = 0; j < live0; ++j) if (gone[j]) { evicted_slot[k] = j; evicted_pos[k] = pos[j]; ++k; }
+  }
+  /* 2. insert: target slots in increasing slot order */
+  int *slot_of_new = (int *)malloc(sizeof(int) * (size_t)b);
+  {
+    int k = 0;
+    for (int j = 0; j < B && k < b; ++j)
+      if (j >= live0 || gone[j]) slot_of_new[k++] = j;
+  }
+  int live1 = live0 - need + b;
+  for (int i = 0; i < b; ++i)
+    insert_token(K, V, s, q, n, pos, slot_of_new[i], d, Kn + (size_t)i * d, Vn + (size_t)i * d, t0 + i);
+  /* 3. attention of query i over the old survivors and the new tokens 0..i */
+  double *p = (double *)malloc(sizeof(double) * (size_t)B);
+  double *Kc = (double *)malloc(sizeof(double) * (size_t)B * d);
+  int *members = (int *)malloc(sizeof(int) * (size_t)B);
+  for (int i = 0; i < b; ++i) {
+    int m = 0;
+    for (int j = 0; j < live1; ++j) {
+      int newer = 0;
+      for (int i2 = i + 1; i2 < b; ++i2) if (slot_of_new[i2] == j) newer = 1;
+      if (!newer) members[m++] = j;
+    }
+    for (int k = 0; k < m; ++k) memcpy(Kc + (size_t)k * d, K + (size_t)members[k] * d, sizeof(double) * (size_t)d);
+    lse[i] = softmax_row(Q + (size_t)i * d, Kc, m, d, scale, p);
+    for (int c = 0; c < d; ++c) out[(size_t)i * d + c] = 0.0;
+    for (int k = 0; k < m; ++k) {
+      const int j = members[k];
+      for (int c = 0; c < d; ++c) out[(size_t)i * d + c] += p[k] * V[(size_t)j * d + c];
+      s[j] += p[k];
+      q[j] += p[k] * p[k];
+      n[j] += 1;
+    }
+  }
+  *live = live1;
+  *t_next = t0 + b;
+  *near_tie = n_near;
+  free(gone); free(cs); free(cq); free(cn); free(cp); free(cslot); free(slot_of_new); free(p); free(Kc); free(members);
+}
+
+/* --------------------------------------------------- grouped-query attention (Sec. 5.3, App. A "Extension") -- */
+
+/* One decode step of a key-value head shared by `group` query heads (Sec. 5.3: the group-wise averaged attention
+ * score updates the importance score).  Order as in Fig. 1 (evict, insert, attend).  Every query head g attends
+ * over the same cache: p_g = Softmax(scale * q_g K^T), out_g = p_g V (Eq. 1); the statistics of Sec. 4.3 receive
+ * the group mean pbar = (1/group) sum_g p_g: Count += 1, Acc += pbar, Acc^square += pbar^2.
+ * Q: [group][d]; out: [group][d]; lse: [group]. */
+void roco_oracle_gqa_step_unit(double *K, double *V, double *s, double *q, int *n, int *pos, int *live, int *t_next,
+                               int B, int d, int group, const double *Q, const double *k_new, const double *v_new,
+                               int r, int mode, double scale, double delta, int force_victim, double *out,
+                               double *lse, int *evicted_slot, int *evicted_pos, int *choice, int *near_tie) {
+  int t = *t_next, slot, near = 0, own = -1;
+  *evicted_slot = -1;
+  *evicted_pos = -1;
+  if (*live == B) {
+    own = roco_oracle_select(s, q, n, pos, *live, r, mode, delta, &near, NULL);
+    slot = (force_victim >= 0 && force_victim < B && near) ? force_victim : own;
+    *evicted_slot = slot;
+    *evicted_pos = pos[slot];
+  } else {
+    slot = (*live)++;
+  }
+  insert_token(K, V, s, q, n, pos, slot, d, k_new, v_new, t);
+  const int m = *live;
+  double *p = (double *)malloc(sizeof(double) * (size_t)m), *pbar = (double *)calloc((size_t)m, sizeof(double));
+  for (int g = 0; g < group; ++g) {
+    lse[g] = softmax_row(Q + (size_t)g * d, K, m, d, scale, p);
+    for (int c = 0; c < d; ++c) out[(size_t)g * d + c] = 0.0;
+    for (int j = 0; j < m; ++j) {
+      for (int c = 0; c < d; ++c) out[(size_t)g * d + c] += p[j] * V[(size_t)j * d + c];
+      pbar[j] += p[j];
+    }
+  }
+  for (int j = 0; j < m; ++j) {
+    const double pb = pbar[j] / group;
+    s[j] += pb;
+    q[j] += pb * pb;
+    n[j] += 1;
+  }
+  *choice = own;
+  *near_tie = near;
+  *t_next = t + 1;
+  free(p); free(pbar);
+}
+
+void roco_oracle_block_step_batch(int U, double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
+                                  int *t_next, int B, int d, int b, const double *Q, const double *Kn,
+                                  const double *Vn, int r, int mode, double scale, double delta,
+                                  const int *force_slots, double *out, double *lse, int *evicted_slot,
+                                  int *evicted_pos, int *choice, int *near_tie) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int u = 0; u < U; ++u) {
+    size_t kb = (size_t)u * B * d, sb = (size_t)u * B, vb = (size_t)u * b * d, ib = (size_t)u * b;
+    roco_oracle_block_step_unit(K + kb, V + kb, s + sb, q + sb, n + sb, pos + sb, live + u, t_next + u, B, d, b,
+                                Q + vb, Kn + vb, Vn + vb, r, mode, scale, delta,
+                                force_slots ? force_slots + ib : NULL, out + vb, lse + ib, evicted_slot + ib,
+                                evicted_pos + ib, choice + ib, near_tie + u);
+  }
+}
+
+void roco_oracle_gqa_step_batch(int U, double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
+                                int *t_next, int B, int d, int group, const double *Q, const double *k_new,
+                                const double *v_new, int r, int mode, double scale, double delta,
+                                const int *force_victim, double *out, double *lse, int *evicted_slot,
+                                int *evicted_pos, int *choice, int *near_tie) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int u = 0; u < U; ++u) {
+    size_t kb = (size_t)u * B * d, sb = (size_t)u * B, qb = (size_t)u * group * d, vb = (size_t)u * d;
+    roco_oracle_gqa_step_unit(K + kb, V + kb, s + sb, q + sb, n + sb, pos + sb, live + u, t_next + u, B, d, group,
+                              Q + qb, k_new + vb, v_new + vb, r, mode, scale, delta,
+                              force_victim ? force_victim[u] : -1, out + qb, lse + (size_t)u * group,
+                              evicted_slot + u, evicted_pos + u, choice + u, near_tie + u);
+  }
 }
