@@ -164,6 +164,41 @@ roco_status roco_decode_step(roco_cache *cache, const void *q, const void *k_new
                              int scope_mode, int step_order, float scale, void *attn_out, float *lse_out,
                              int32_t *evicted_slot, int32_t *evicted_pos, void *stream);
 
+/*
+ * Block-wise evict-and-encode (Sec. 5.3 "Overhead", App. B: "the block size b controls the number of tokens being
+ * freed and encoded within one eviction step"): b new tokens per unit in one pass over the cache.
+ *   1. live + b - B tokens (if positive) leave: the rule of Sec. 4.3 applied that many times on the statistics as
+ *      they stand (frozen), each time on the tokens still cached.
+ *   2. The new tokens (positions t_next .. t_next + b - 1) take, in order, the freed slots and -- while the buffer
+ *      is not full -- slots live, live + 1, ..., all in increasing slot order.
+ *   3. Query i attends over the remaining old tokens and the new tokens 0..i (causal inside the block); every
+ *      attended token gets Count += 1, Acc += p, Acc^square += p^2.
+ * b = 1 is roco_decode_step with ROCO_EVICT_FIRST.
+ *
+ *   Q, K_new, V_new  [S][G][b][d], cache->kv_dtype
+ *   b                1..16; b > 1 needs ROCO_SCOPE_EXCLUDE_TOP_R (else ROCO_ERR_UNSUPPORTED) and r + b <= B;
+ *                    b * B floats of scores must fit in shared memory (else ROCO_ERR_UNSUPPORTED)
+ *   attn_out         [S][G][b][d];   lse_out [S][G][b] or NULL
+ *   evicted_slot     [S][G][b] freed slots in increasing order, padded with -1;  evicted_pos likewise, or NULL
+ */
+roco_status roco_block_step(roco_cache *cache, const void *Q, const void *K_new, const void *V_new, int b, int r,
+                            int scope_mode, float scale, void *attn_out, float *lse_out, int32_t *evicted_slot,
+                            int32_t *evicted_pos, void *stream);
+
+/*
+ * Decode step for grouped-query attention (Sec. 5.3 "Extension to Grouped-Query Attention", App. A): the cache
+ * belongs to a key-value head that `group` query heads share.  Order as ROCO_EVICT_FIRST.  Each query head g
+ * attends over the same cache, out_g = Softmax(scale * q_g K^T) V; the statistics receive the group-wise
+ * averaged probability pbar = (1/group) sum_g p_g: Count += 1, Acc += pbar, Acc^square += pbar^2.
+ *
+ *   Q            [S][G][group][d]  (G counts key-value heads);  k_new, v_new [S][G][d]
+ *   group        1..16 (group * B floats of scores must fit in shared memory)
+ *   attn_out     [S][G][group][d];  lse_out [S][G][group] or NULL;  evicted_slot, evicted_pos [S][G]
+ */
+roco_status roco_gqa_decode_step(roco_cache *cache, const void *Q, const void *k_new, const void *v_new, int group,
+                                 int r, int scope_mode, float scale, void *attn_out, float *lse_out,
+                                 int32_t *evicted_slot, int32_t *evicted_pos, void *stream);
+
 /* Bytes of device staging roco_decode_step_host needs (host function). */
 size_t roco_decode_host_staging_bytes(const roco_cache *cache);
 

@@ -21,6 +21,7 @@ ROCO_EVICT_FIRST, ROCO_ATTEND_FIRST = 0, 1
 
 EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes", "roco_prefill",
            "roco_prefill_uses_tensor_cores", "roco_prefill_static", "roco_prefill_workspace_bytes_lowest_r",
+           "roco_block_step", "roco_gqa_decode_step",
            "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status")
 
 
@@ -69,6 +70,10 @@ def lib() -> C.CDLL:
         L.roco_decode_step.restype = C.c_int
         L.roco_decode_step.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                                        C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        for fn in (L.roco_block_step, L.roco_gqa_decode_step):
+            fn.restype = C.c_int
+            fn.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                           C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.roco_decode_step_host.restype = C.c_int
         L.roco_decode_step_host.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                             C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -173,6 +178,27 @@ def roco_decode_step(cache: Cache, q, k_new, v_new, r: int, attn_out, evicted_sl
                                 scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot), _ptr(evicted_pos), _stream())
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_decode_step")
+
+
+def roco_block_step(cache: Cache, Q, K_new, V_new, r: int, attn_out, evicted_slot, evicted_pos=None, lse_out=None,
+                    scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R, scale: Optional[float] = None):
+    """Block-wise evict-and-encode of b = Q.shape[2] tokens per unit.  Q, K_new, V_new: [S][G][b][d]."""
+    scale = cache.d ** -0.5 if scale is None else scale
+    rc = lib().roco_block_step(C.byref(cache.c), _ptr(Q), _ptr(K_new), _ptr(V_new), int(Q.shape[2]), r, scope_mode,
+                               scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot), _ptr(evicted_pos), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_block_step")
+
+
+def roco_gqa_decode_step(cache: Cache, Q, k_new, v_new, r: int, attn_out, evicted_slot, evicted_pos=None,
+                         lse_out=None, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R, scale: Optional[float] = None):
+    """Decode step of key-value heads shared by group = Q.shape[2] query heads.  Q: [S][G][group][d]."""
+    scale = cache.d ** -0.5 if scale is None else scale
+    rc = lib().roco_gqa_decode_step(C.byref(cache.c), _ptr(Q), _ptr(k_new), _ptr(v_new), int(Q.shape[2]), r,
+                                    scope_mode, scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot),
+                                    _ptr(evicted_pos), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_gqa_decode_step")
 
 
 def roco_decode_host_staging_bytes(cache: Cache) -> int:

@@ -139,6 +139,37 @@ roco_status roco_decode_step(roco_cache *cache, const void *q, const void *k_new
                             evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
 }
 
+roco_status roco_block_step(roco_cache *cache, const void *Q, const void *K_new, const void *V_new, int b, int r,
+                            int scope_mode, float scale, void *attn_out, float *lse_out, int32_t *evicted_slot,
+                            int32_t *evicted_pos, void *stream) {
+  roco_status st = check_cache(cache);
+  if (st != ROCO_OK) return st;
+  if (!Q || !K_new || !V_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K_new) || !aligned16(V_new) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
+  if (b < 1) return ROCO_ERR_INVALID_ARG;
+  if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
+  if (b > multi_max_queries()) return ROCO_ERR_UNSUPPORTED;
+  if (b > 1 && scope_mode != ROCO_SCOPE_EXCLUDE_TOP_R) return ROCO_ERR_UNSUPPORTED;  // the scope would refill
+  if (b > 1 && r + b > cache->B) return ROCO_ERR_INVALID_ARG;  // the scope must hold the b victims
+  if (!multi_fits(cache->B, cache->d, b, b)) return ROCO_ERR_UNSUPPORTED;
+  return launch_multi_step(*cache, 0, b, b, Q, K_new, V_new, r, scope_mode, scale, attn_out, lse_out, evicted_slot,
+                           evicted_pos, static_cast<cudaStream_t>(stream));
+}
+
+roco_status roco_gqa_decode_step(roco_cache *cache, const void *Q, const void *k_new, const void *v_new, int group,
+                                 int r, int scope_mode, float scale, void *attn_out, float *lse_out,
+                                 int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {
+  roco_status st = check_cache(cache);
+  if (st != ROCO_OK) return st;
+  if (!Q || !k_new || !v_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
+  if (group < 1) return ROCO_ERR_INVALID_ARG;
+  if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
+  if (group > multi_max_queries() || !multi_fits(cache->B, cache->d, group, 1)) return ROCO_ERR_UNSUPPORTED;
+  return launch_multi_step(*cache, 1, group, 1, Q, k_new, v_new, r, scope_mode, scale, attn_out, lse_out,
+                           evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
+}
+
 size_t roco_decode_host_staging_bytes(const roco_cache *cache) {
   if (!cache || cache->S < 1 || cache->G < 1) return 0;
   const size_t U = (size_t)cache->S * cache->G;

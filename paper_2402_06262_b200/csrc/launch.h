@@ -33,4 +33,11 @@ roco_status launch_budget_select_gather(const roco_cache &c, int Lmax, const int
                                         const float *q_full, int *dst, unsigned long long *sortbuf, int Lp2max,
                                         cudaStream_t stream);
 
+// Multi-query steps (block-wise evict-and-encode: kind 0, nb == M; grouped-query decode: kind 1, nb == 1).
+int multi_max_queries();
+bool multi_fits(int B, int d, int M, int nb);
+roco_status launch_multi_step(const roco_cache &c, int kind, int M, int nb, const void *Q, const void *k_new,
+                              const void *v_new, int r, int scope_mode, float scale, void *out, float *lse,
+                              int32_t *ev_slot, int32_t *ev_pos, cudaStream_t stream);
+
 }  // namespace roco

@@ -1,0 +1,474 @@
+// Multi-query steps over the budgeted cache: several queries share one pass over a unit's K and V blocks.
+//   - block-wise evict-and-encode (Sec. 5.3 "Overhead", App. B): b new tokens per unit and step; b slots are
+//     freed by the rule of Sec. 4.3 applied on frozen statistics, the new tokens take the freed / free slots in
+//     increasing slot order, query i attends over the old survivors and the new tokens 0..i, and every attended
+//     token gets Count += 1, Acc += p, Acc^square += p^2 per query;
+//   - grouped-query attention (Sec. 5.3, App. A): `group` query heads share a key-value head; one new token;
+//     the statistics receive the group mean of the probabilities.
+// Same organisation as the single-query decode step (producer warp + TMA ring, eight consumer warps, four
+// policy warps that select, insert and update the statistics while the consumers stream), with the M x B score
+// matrix in shared memory.  Each consumer warp owns four queries and a share of every tile's rows, so the
+// per-row arithmetic grows with M while the HBM traffic per unit stays that of one decode step.
+#include "common.cuh"
+#include "launch.h"
+#include "select.cuh"
+
+namespace roco {
+
+constexpr int kMqConsumerWarps = 8;
+constexpr int kMqConsumers = kMqConsumerWarps * 32;
+constexpr int kMqProducerWarp = kMqConsumerWarps;
+constexpr int kMqPolicyWarp0 = kMqConsumerWarps + 1;
+constexpr int kMqPolicyThreads = 128;
+constexpr int kMqThreads = kMqConsumers + 32 + kMqPolicyThreads;
+constexpr int kMqBarConsumers = 1;
+constexpr int kMqBarPolicy = 2;
+constexpr int kMqTile = 16384;
+constexpr int kMqMaxQ = 16;  // queries per step
+constexpr int kMqQPW = 4;    // queries per consumer warp
+
+enum { kMqBlock = 0, kMqGqa = 1 };
+
+struct MultiParams {
+  const char *K, *V;
+  float *s, *q;
+  int *n, *pos, *live, *t_next, *status;
+  const char *Q, *k_new, *v_new;
+  char *out;
+  float *lse;
+  int *ev_slot, *ev_pos;
+  int B, r, scope_mode, stages, M, nb, kind;
+  float scale;
+};
+
+struct MultiSmem {
+  char *ring;
+  float *z;  // [M][Bp] scores, then probabilities
+  uint32_t *vkey;
+  float *mkey;
+  signed char *newtok;  // [Bp] index of the new token a slot holds, -1 for an old token
+  SelectScratch *sel;
+  float *qf;      // [M][D]
+  float *knew;    // [nb][D]
+  float *vnew;    // [nb][D]
+  float *zn;      // [M][nb] scores of the queries against the new tokens
+  float *outred;  // [8 warps][4][D]
+  uint64_t *full, *empty, *p_ready, *policy_done;
+  int *ctl;  // [0] abort flag, [1..16] target slots of the new tokens, [17] warp_tot scratch base
+};
+
+__host__ __device__ inline size_t multi_smem_bytes(int B, int d, int stages, int M, int nb) {
+  const size_t Bp = align_up((size_t)B, 16);
+  size_t b = (size_t)stages * kMqTile;
+  b += (size_t)M * Bp * 4 + 2 * Bp * 4 + Bp;
+  b += sizeof(SelectScratch);
+  b += ((size_t)M + 2 * (size_t)nb) * d * 4 + (size_t)M * nb * 4;
+  b += (size_t)kMqConsumerWarps * kMqQPW * d * 4;
+  b = align_up(b, 8) + (2 * (size_t)stages + 2) * 8 + 64 * 4;
+  return b + 128;
+}
+
+__device__ inline MultiSmem multi_carve(char *raw, int B, int d, int stages, int M, int nb) {
+  MultiSmem m;
+  char *p = (char *)align_up((size_t)raw, 128);
+  const size_t Bp = align_up((size_t)B, 16);
+  m.ring = p; p += (size_t)stages * kMqTile;
+  m.z = (float *)p; p += (size_t)M * Bp * 4;
+  m.vkey = (uint32_t *)p; p += Bp * 4;
+  m.mkey = (float *)p; p += Bp * 4;
+  m.newtok = (signed char *)p; p += Bp;
+  m.sel = (SelectScratch *)p; p += sizeof(SelectScratch);
+  m.qf = (float *)p; p += (size_t)M * d * 4;
+  m.knew = (float *)p; p += (size_t)nb * d * 4;
+  m.vnew = (float *)p; p += (size_t)nb * d * 4;
+  m.zn = (float *)p; p += (size_t)M * nb * 4;
+  m.outred = (float *)p; p += (size_t)kMqConsumerWarps * kMqQPW * d * 4;
+  p = (char *)align_up((size_t)p, 8);
+  m.full = (uint64_t *)p; p += stages * 8;
+  m.empty = (uint64_t *)p; p += stages * 8;
+  m.p_ready = (uint64_t *)p; p += 8;
+  m.policy_done = (uint64_t *)p; p += 8;
+  m.ctl = (int *)p;
+  return m;
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParams p) {
+  constexpr int kRowBytes = D * (int)sizeof(T);
+  constexpr int kLanesPerRow = kRowBytes / 16;
+  constexpr int kRowsPerLoad = 32 / kLanesPerRow;
+  constexpr int kTileRows = kMqTile / kRowBytes;
+  constexpr int kEPC = Elem<T>::kPerChunk;
+
+  extern __shared__ char mq_smem_raw[];
+  const int M = p.M, nb = p.nb, B = p.B, stages = p.stages;
+  const MultiSmem sm = multi_carve(mq_smem_raw, B, D, stages, M, nb);
+  volatile int *abort_flag = sm.ctl;
+  const size_t Bp = align_up((size_t)B, 16);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int u = blockIdx.x;
+  const size_t unit_kv = (size_t)u * B * kRowBytes;
+  const size_t unit_st = (size_t)u * B;
+
+  if (tid == 0) {
+    for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kMqConsumerWarps); }
+    mbar_init(sm.p_ready, kMqConsumerWarps);
+    mbar_init(sm.policy_done, 1);
+    sm.ctl[0] = 0;
+    mbar_init_fence();
+  }
+  int live0 = p.live[u];
+  if (live0 < 0 || live0 > B) {
+    if (tid == 0) atomicOr(p.status, ROCO_DEV_BAD_LIVE);
+    live0 = live0 < 0 ? 0 : B;
+  }
+  int need = live0 + nb - B;  // tokens that have to leave
+  if (need < 0) need = 0;
+  const int live1 = live0 - need + nb;  // occupied slots after the insertion = slots every query streams over
+  const int n_tiles = (live1 + kTileRows - 1) / kTileRows;
+  __syncthreads();
+
+  if (warp == kMqProducerWarp) {
+    if (lane == 0) {
+      for (int g = 0; g < 2 * n_tiles; ++g) {
+        const int st = g % stages;
+        if (g >= stages) mbar_wait(&sm.empty[st], ((g / stages) - 1) & 1, abort_flag, p.status);
+        const int it = (g < n_tiles) ? g : g - n_tiles;
+        const char *src = ((g < n_tiles) ? p.K : p.V) + unit_kv + (size_t)it * kMqTile;
+        int rows = live1 - it * kTileRows;
+        if (rows > kTileRows) rows = kTileRows;
+        const uint32_t bytes = (uint32_t)rows * kRowBytes;
+        mbar_expect_tx(&sm.full[st], bytes);
+        bulk_g2s(sm.ring + (size_t)st * kMqTile, src, bytes, &sm.full[st]);
+      }
+    }
+    return;
+  }
+
+  if (warp >= kMqPolicyWarp0) {
+    // ---------------------------------------------------------- policy: free slots, insert, statistics
+    const int ptid = tid - kMqPolicyWarp0 * 32, plane = ptid & 31, pwarp = ptid >> 5;
+    const int t_new = p.t_next[u];
+    const float *gs = p.s + unit_st, *gq = p.q + unit_st;
+    const int *gn = p.n + unit_st;
+    int *gpos = p.pos + unit_st;
+    for (int j = ptid; j < live1; j += kMqPolicyThreads) sm.newtok[j] = -1;
+    for (int i = ptid; i < nb * D; i += kMqPolicyThreads) {
+      sm.knew[i] = Elem<T>::load((const T *)p.k_new + (size_t)u * nb * D + i);
+      sm.vnew[i] = Elem<T>::load((const T *)p.v_new + (size_t)u * nb * D + i);
+    }
+    named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+    int *tgt = sm.ctl + 1;  // [nb] target slots, ascending
+    if (need > 0) {
+      // the rule of Sec. 4.3 applied `need` times on frozen statistics = one pass: the tokens outside the scope
+      // (the live0 - m last in (variance, position) order) never enter it, so the `need` first of the scope in
+      // (mean, position) order leave
+      for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+        const float sj = gs[j], qj = gq[j];
+        const int nj = gn[j];
+        sm.vkey[j] = variance_key_fast(sj, qj, nj);
+        sm.mkey[j] = mean_fast(sj, nj);
+      }
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      const int m = scope_size(live0, p.r, p.scope_mode);
+      uint32_t Tv = 0xffffffffu;
+      int Pv = 0x7fffffff;
+      uint32_t rank, ties;
+      if (m < live0) {
+        Tv = radix_select<uint32_t>([&](int j) { return sm.vkey[j]; }, [&](int) { return true; }, live0,
+                                    (uint32_t)(m - 1), *sm.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &rank, &ties);
+        if (ties != rank + 1) {
+          uint32_t r2, t2;
+          Pv = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)gpos[j]; },
+                                           [&](int j) { return sm.vkey[j] == Tv; }, live0, rank, *sm.sel, ptid,
+                                           kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
+        }
+      }
+      auto in_scope = [&](int j) {
+        const uint32_t k = sm.vkey[j];
+        return k < Tv || (k == Tv && (Pv == 0x7fffffff || gpos[j] <= Pv));
+      };
+      const uint32_t Tm = radix_select<uint32_t>([&](int j) { return __float_as_uint(sm.mkey[j]); }, in_scope, live0,
+                                                 (uint32_t)(need - 1), *sm.sel, ptid, kMqPolicyThreads, kMqBarPolicy,
+                                                 &rank, &ties);
+      int Pm = 0x7fffffff;
+      if (ties != rank + 1) {
+        uint32_t r2, t2;
+        Pm = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)gpos[j]; },
+                                         [&](int j) { return in_scope(j) && __float_as_uint(sm.mkey[j]) == Tm; },
+                                         live0, rank, *sm.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
+      }
+      // freed slots in increasing slot order: ballot prefix over chunks of 128 slots
+      int *wtot = sm.ctl + 20;  // [4] per-warp counts, [4] = running base
+      if (ptid == 0) wtot[4] = 0;
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      for (int j0 = 0; j0 < live0; j0 += kMqPolicyThreads) {
+        const int j = j0 + ptid;
+        bool ev = false;
+        if (j < live0 && in_scope(j)) {
+          const uint32_t k = __float_as_uint(sm.mkey[j]);
+          ev = k < Tm || (k == Tm && (Pm == 0x7fffffff || gpos[j] <= Pm));
+        }
+        const uint32_t bal = __ballot_sync(0xffffffffu, ev);
+        if (plane == 0) wtot[pwarp] = __popc(bal);
+        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+        int off = wtot[4];
+        for (int w = 0; w < pwarp; ++w) off += wtot[w];
+        const int rk = off + __popc(bal & ((1u << plane) - 1u));
+        if (ev && rk < nb) tgt[rk] = j;
+        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+        if (ptid == 0) wtot[4] += wtot[0] + wtot[1] + wtot[2] + wtot[3];
+        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      }
+      if (ptid == 0 && wtot[4] != need) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
+    }
+    if (ptid < nb - need) tgt[need + ptid] = live0 + ptid;  // free slots behind the occupied ones
+    named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+    // the new tokens take the target slots: evicted positions out, new K/V and positions in
+    if (ptid < nb) {
+      int slot = tgt[ptid];
+      if (slot < 0 || slot >= B) slot = 0;  // only after corrupt statistics (status bit set above)
+      p.ev_slot[(size_t)u * nb + ptid] = ptid < need ? slot : -1;
+      if (p.ev_pos) p.ev_pos[(size_t)u * nb + ptid] = ptid < need ? gpos[slot] : -1;
+      sm.newtok[slot] = (signed char)ptid;
+      gpos[slot] = t_new + ptid;
+    }
+    for (int w = ptid; w < nb * 2 * kLanesPerRow; w += kMqPolicyThreads) {  // in-place overwrite, 16 bytes each
+      const int i = w / (2 * kLanesPerRow), c = w % (2 * kLanesPerRow);
+      const bool isv = c >= kLanesPerRow;
+      const int cc = isv ? c - kLanesPerRow : c;
+      int slot = tgt[i];
+      if (slot < 0 || slot >= B) slot = 0;
+      const uint4 val = *((const uint4 *)((isv ? p.v_new : p.k_new) + ((size_t)u * nb + i) * kRowBytes) + cc);
+      *((uint4 *)(const_cast<char *>(isv ? p.V : p.K) + unit_kv + (size_t)slot * kRowBytes) + cc) = val;
+    }
+    // scores of every query against every new token, from k_new directly (log2 domain)
+    const float zscale = p.scale * kLog2e;
+    for (int w = ptid; w < M * nb; w += kMqPolicyThreads) {
+      const int i = w / nb, jn = w % nb;
+      const T *qrow = (const T *)p.Q + ((size_t)u * M + i) * D;
+      float acc = 0.f;
+      for (int c = 0; c < D; ++c) acc = fmaf(Elem<T>::load(qrow + c), sm.knew[jn * D + c], acc);
+      sm.zn[w] = acc * zscale;
+    }
+    if (ptid == 0) { p.live[u] = live1; p.t_next[u] = t_new + nb; }
+    named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+    if (ptid == 0) mbar_arrive(sm.policy_done);
+
+    // statistics of Sec. 4.3 once the probabilities are in shared memory
+    mbar_wait(sm.p_ready, 0, abort_flag, p.status);
+    for (int j = ptid; j < live1; j += kMqPolicyThreads) {
+      const int jn = sm.newtok[j];
+      const bool fresh = jn >= 0;
+      float ds = 0.f, dq = 0.f;
+      int dn;
+      if (p.kind == kMqGqa) {
+        for (int i = 0; i < M; ++i) ds += sm.z[(size_t)i * Bp + j];
+        ds /= (float)M;  // group-wise averaged attention score
+        dq = ds * ds;
+        dn = 1;
+      } else {
+        const int i0 = fresh ? jn : 0;  // query i sees new token jn only if i >= jn
+        for (int i = i0; i < M; ++i) {
+          const float pij = sm.z[(size_t)i * Bp + j];
+          ds += pij;
+          dq = fmaf(pij, pij, dq);
+        }
+        dn = M - i0;
+      }
+      const float s0 = fresh ? 0.f : gs[j], q0 = fresh ? 0.f : gq[j];
+      const int n0 = fresh ? 0 : gn[j];
+      p.s[unit_st + j] = s0 + ds;
+      p.q[unit_st + j] = q0 + dq;
+      p.n[unit_st + j] = n0 + dn;
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------- consumers
+  const int QG = M <= 4 ? 1 : (M <= 8 ? 2 : 4);  // query groups of four
+  const int RG = kMqConsumerWarps / QG;          // row groups
+  const int qg = warp % QG, rg = warp / QG;
+  const int rows_per_warp = kTileRows / RG;
+  const int loads = rows_per_warp / kRowsPerLoad;
+  for (int i = tid; i < M * D; i += kMqConsumers)
+    sm.qf[i] = Elem<T>::load((const T *)p.Q + (size_t)u * M * D + i);
+  named_bar_sync(kMqBarConsumers, kMqConsumers);
+
+  const float zscale = p.scale * kLog2e;
+  const int lane_chunk = lane % kLanesPerRow, lane_row = lane / kLanesPerRow;
+  float qreg[kMqQPW][kEPC];
+#pragma unroll
+  for (int i = 0; i < kMqQPW; ++i) {
+    const int qi = qg * kMqQPW + i;
+#pragma unroll
+    for (int e = 0; e < kEPC; ++e) qreg[i][e] = qi < M ? sm.qf[qi * D + lane_chunk * kEPC + e] : 0.f;
+  }
+
+  // ---- scores of four queries per warp: z_i[j] = scale * q_i.K[j]  (Eq. 1), log2 domain
+  for (int it = 0; it < n_tiles; ++it) {
+    const int st = it % stages;
+    mbar_wait(&sm.full[st], (it / stages) & 1, abort_flag, p.status);
+    const char *tile = sm.ring + (size_t)st * kMqTile;
+    for (int l = 0; l < loads; ++l) {
+      const int row = rg * rows_per_warp + l * kRowsPerLoad + lane_row;
+      const uint4 c = *(const uint4 *)(tile + (size_t)row * kRowBytes + lane_chunk * 16);
+      float f[kEPC];
+      Elem<T>::unpack(c, f);
+      float acc[kMqQPW];
+#pragma unroll
+      for (int i = 0; i < kMqQPW; ++i) {
+        acc[i] = 0.f;
+#pragma unroll
+        for (int e = 0; e < kEPC; ++e) acc[i] = fmaf(f[e], qreg[i][e], acc[i]);
+#pragma unroll
+        for (int o = kLanesPerRow / 2; o > 0; o >>= 1) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], o);
+      }
+      const int j = it * kTileRows + row;
+      if (lane_chunk < kMqQPW && j < live1) {
+        const int qi = qg * kMqQPW + lane_chunk;
+        float v = acc[0];
+        if (lane_chunk == 1) v = acc[1];
+        if (lane_chunk == 2) v = acc[2];
+        if (lane_chunk == 3) v = acc[3];
+        if (qi < M) sm.z[(size_t)qi * Bp + j] = v * zscale;
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.empty[st]);
+  }
+
+  // the slots the policy warps have filled hold the new tokens: their scores come from k_new, with the causal
+  // mask inside a block (query i does not see the tokens after it)
+  mbar_wait(sm.policy_done, 0, abort_flag, p.status);
+  named_bar_sync(kMqBarConsumers, kMqConsumers);
+  for (int w = tid; w < M * nb; w += kMqConsumers) {
+    const int i = w / nb, jn = w % nb;
+    int slot = sm.ctl[1 + jn];
+    if (slot < 0 || slot >= B) slot = 0;
+    sm.z[(size_t)i * Bp + slot] = (p.kind == kMqBlock && jn > i) ? -INFINITY : sm.zn[w];
+  }
+  named_bar_sync(kMqBarConsumers, kMqConsumers);
+
+  // ---- one softmax per query, each by one warp
+  for (int i = warp; i < M; i += kMqConsumerWarps) {
+    float *zi = sm.z + (size_t)i * Bp;
+    float zmax = -INFINITY;
+    for (int j = lane; j < live1; j += 32) zmax = fmaxf(zmax, zi[j]);
+    zmax = warp_max(zmax);
+    float zsum = 0.f;
+    for (int j = lane; j < live1; j += 32) {
+      const float ex = exp2f(zi[j] - zmax);
+      zi[j] = ex;
+      zsum += ex;
+    }
+    zsum = warp_sum(zsum);
+    const float inv = 1.f / zsum;
+    for (int j = lane; j < live1; j += 32) zi[j] *= inv;
+    if (lane == 0 && p.lse) p.lse[(size_t)u * M + i] = (zmax + log2f(zsum)) * kLn2;
+  }
+  __syncwarp();
+  if (lane == 0) mbar_arrive(sm.p_ready);
+  named_bar_sync(kMqBarConsumers, kMqConsumers);
+
+  // ---- out_i = sum_j p_i[j] V[j]; the new tokens' values come from v_new at the end
+  float oacc[kMqQPW][kEPC];
+#pragma unroll
+  for (int i = 0; i < kMqQPW; ++i)
+#pragma unroll
+    for (int e = 0; e < kEPC; ++e) oacc[i][e] = 0.f;
+  for (int it = 0; it < n_tiles; ++it) {
+    const int g = n_tiles + it;
+    const int st = g % stages;
+    mbar_wait(&sm.full[st], (g / stages) & 1, abort_flag, p.status);
+    const char *tile = sm.ring + (size_t)st * kMqTile;
+    for (int l = 0; l < loads; ++l) {
+      const int row = rg * rows_per_warp + l * kRowsPerLoad + lane_row;
+      const int j = it * kTileRows + row;
+      if (j < live1 && sm.newtok[j] < 0) {
+        const uint4 c = *(const uint4 *)(tile + (size_t)row * kRowBytes + lane_chunk * 16);
+        float f[kEPC];
+        Elem<T>::unpack(c, f);
+#pragma unroll
+        for (int i = 0; i < kMqQPW; ++i) {
+          const int qi = qg * kMqQPW + i;
+          const float pj = qi < M ? sm.z[(size_t)qi * Bp + j] : 0.f;
+#pragma unroll
+          for (int e = 0; e < kEPC; ++e) oacc[i][e] = fmaf(pj, f[e], oacc[i][e]);
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.empty[st]);
+  }
+#pragma unroll
+  for (int i = 0; i < kMqQPW; ++i)
+#pragma unroll
+    for (int e = 0; e < kEPC; ++e) {
+#pragma unroll
+      for (int o = kLanesPerRow; o < 32; o <<= 1) oacc[i][e] += __shfl_xor_sync(0xffffffffu, oacc[i][e], o);
+    }
+  if (lane_row == 0) {
+#pragma unroll
+    for (int i = 0; i < kMqQPW; ++i)
+#pragma unroll
+      for (int e = 0; e < kEPC; ++e) sm.outred[((size_t)warp * kMqQPW + i) * D + lane_chunk * kEPC + e] = oacc[i][e];
+  }
+  named_bar_sync(kMqBarConsumers, kMqConsumers);
+  for (int w = tid; w < M * D; w += kMqConsumers) {
+    const int qi = w / D, c = w % D;
+    float o = 0.f;
+    for (int r2 = 0; r2 < RG; ++r2) o += sm.outred[((size_t)(r2 * QG + qi / kMqQPW) * kMqQPW + qi % kMqQPW) * D + c];
+    for (int jn = 0; jn < nb; ++jn) {
+      int slot = sm.ctl[1 + jn];
+      if (slot < 0 || slot >= B) slot = 0;
+      o = fmaf(sm.z[(size_t)qi * Bp + slot], sm.vnew[jn * D + c], o);
+    }
+    Elem<T>::store((T *)p.out + (size_t)u * M * D + w, o);
+  }
+}
+
+static int multi_pick_stages(int B, int d, int M, int nb) {
+  const size_t per_sm = 227 * 1024;
+  for (int ctas = 2; ctas >= 1; --ctas)
+    for (int st = 5; st >= 3; --st)
+      if ((multi_smem_bytes(B, d, st, M, nb) + 1024) * ctas <= per_sm) return st;
+  return 0;
+}
+
+template <typename T, int D>
+static cudaError_t launch_multi_t(MultiParams &p, int U, cudaStream_t stream) {
+  const size_t smem = multi_smem_bytes(p.B, D, p.stages, p.M, p.nb);
+  cudaError_t err = cudaFuncSetAttribute(multi_step_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  multi_step_kernel<T, D><<<U, kMqThreads, smem, stream>>>(p);
+  return cudaGetLastError();
+}
+
+int multi_max_queries() { return kMqMaxQ; }
+
+bool multi_fits(int B, int d, int M, int nb) { return multi_pick_stages(B, d, M, nb) > 0; }
+
+roco_status launch_multi_step(const roco_cache &c, int kind, int M, int nb, const void *Q, const void *k_new,
+                              const void *v_new, int r, int scope_mode, float scale, void *out, float *lse,
+                              int32_t *ev_slot, int32_t *ev_pos, cudaStream_t stream) {
+  MultiParams p;
+  p.K = (const char *)c.K; p.V = (const char *)c.V;
+  p.s = c.s; p.q = c.q; p.n = c.n; p.pos = c.pos; p.live = c.live; p.t_next = c.t_next; p.status = c.status;
+  p.Q = (const char *)Q; p.k_new = (const char *)k_new; p.v_new = (const char *)v_new;
+  p.out = (char *)out; p.lse = lse; p.ev_slot = ev_slot; p.ev_pos = ev_pos;
+  p.B = c.B; p.r = r; p.scope_mode = scope_mode; p.M = M; p.nb = nb; p.kind = kind; p.scale = scale;
+  p.stages = multi_pick_stages(c.B, c.d, M, nb);
+  if (p.stages == 0) return ROCO_ERR_UNSUPPORTED;
+  const int U = c.S * c.G;
+  cudaError_t err;
+  if (c.kv_dtype == ROCO_BF16 && c.d == 128) err = launch_multi_t<__nv_bfloat16, 128>(p, U, stream);
+  else if (c.kv_dtype == ROCO_BF16 && c.d == 64) err = launch_multi_t<__nv_bfloat16, 64>(p, U, stream);
+  else if (c.kv_dtype == ROCO_F32 && c.d == 128) err = launch_multi_t<float, 128>(p, U, stream);
+  else if (c.kv_dtype == ROCO_F32 && c.d == 64) err = launch_multi_t<float, 64>(p, U, stream);
+  else return ROCO_ERR_UNSUPPORTED;
+  return err == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
+}
+
+}  // namespace roco

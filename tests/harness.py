@@ -163,3 +163,82 @@ class DecodeParity:
         if check_state:
             compare_state(c, self.st, self.units, f"after step {self.tally.steps}", check_kv=True)
         return res
+
+
+class BlockParity:
+    """Steps the GPU cache and the oracle state of the sampled units together, b tokens per step."""
+
+    def __init__(self, cache: R.Cache, st: oracle.State, units: Sequence[int], b: int, r: int, scope_mode: int,
+                 tally: Tally, scale: Optional[float] = None):
+        self.cache, self.st, self.units, self.b = cache, st, list(units), b
+        self.r, self.mode, self.tally = r, scope_mode, tally
+        self.scale = cache.d ** -0.5 if scale is None else scale
+        dev = cache.K.device
+        self.out = torch.zeros(cache.S, cache.G, b, cache.d, dtype=cache.dtype, device=dev)
+        self.lse = torch.zeros(cache.S, cache.G, b, dtype=torch.float32, device=dev)
+        self.ev_slot = torch.zeros(cache.S, cache.G, b, dtype=torch.int32, device=dev)
+        self.ev_pos = torch.zeros(cache.S, cache.G, b, dtype=torch.int32, device=dev)
+
+    def step(self, Q, K_new, V_new, check_state=False):
+        c = self.cache
+        R.roco_block_step(c, Q, K_new, V_new, self.r, self.out, self.ev_slot, self.ev_pos, self.lse,
+                          scope_mode=self.mode, scale=self.scale)
+        torch.cuda.synchronize()
+        g_slot = unit_view(self.ev_slot, self.units).cpu().numpy()
+        g_pos = unit_view(self.ev_pos, self.units).cpu().numpy()
+        res = oracle.block_step(self.st, widen(unit_view(Q, self.units)), widen(unit_view(K_new, self.units)),
+                                widen(unit_view(V_new, self.units)), self.r, self.mode, self.scale, delta=DELTA,
+                                force_slots=g_slot)
+        firm = res.near_tie == 0
+        np.testing.assert_array_equal(g_slot[firm], res.choice[firm], err_msg="freed slots differ outside the margin")
+        self.tally.near_ties += int((~firm).sum())
+        self.tally.near_tie_disagreements += int((g_slot != res.choice).any(axis=1)[~firm].sum())
+        np.testing.assert_array_equal(g_slot, res.evicted_slot)
+        np.testing.assert_array_equal(g_pos, res.evicted_pos)
+        self.tally.steps += 1
+        self.tally.decisions += int((res.choice >= 0).sum())
+        g_out = widen(unit_view(self.out, self.units))
+        assert np.abs(g_out - res.out).max() <= out_tol(c.dtype), f"attention output off by {np.abs(g_out - res.out).max()}"
+        np.testing.assert_allclose(widen(unit_view(self.lse, self.units)), res.lse, rtol=0, atol=LSE_ATOL)
+        if check_state:
+            compare_state(c, self.st, self.units, f"after block step {self.tally.steps}")
+        return res
+
+
+class GqaParity:
+    """Steps key-value-head caches shared by `group` query heads on the GPU and in the oracle."""
+
+    def __init__(self, cache: R.Cache, st: oracle.State, units: Sequence[int], group: int, r: int, scope_mode: int,
+                 tally: Tally, scale: Optional[float] = None):
+        self.cache, self.st, self.units, self.group = cache, st, list(units), group
+        self.r, self.mode, self.tally = r, scope_mode, tally
+        self.scale = cache.d ** -0.5 if scale is None else scale
+        dev = cache.K.device
+        self.out = torch.zeros(cache.S, cache.G, group, cache.d, dtype=cache.dtype, device=dev)
+        self.lse = torch.zeros(cache.S, cache.G, group, dtype=torch.float32, device=dev)
+        self.ev_slot = torch.zeros(cache.S, cache.G, dtype=torch.int32, device=dev)
+        self.ev_pos = torch.zeros(cache.S, cache.G, dtype=torch.int32, device=dev)
+
+    def step(self, Q, k_new, v_new, check_state=False):
+        c = self.cache
+        R.roco_gqa_decode_step(c, Q, k_new, v_new, self.r, self.out, self.ev_slot, self.ev_pos, self.lse,
+                               scope_mode=self.mode, scale=self.scale)
+        torch.cuda.synchronize()
+        g_slot = unit_view(self.ev_slot, self.units).cpu().numpy()
+        g_pos = unit_view(self.ev_pos, self.units).cpu().numpy()
+        res = oracle.gqa_step(self.st, widen(unit_view(Q, self.units)), widen(unit_view(k_new, self.units)),
+                              widen(unit_view(v_new, self.units)), self.r, self.mode, self.scale, delta=DELTA,
+                              force_victim=g_slot)
+        firm = ~res.near_tie
+        np.testing.assert_array_equal(g_slot[firm], res.choice[firm], err_msg="victim differs outside the margin")
+        self.tally.near_ties += int(res.near_tie.sum())
+        np.testing.assert_array_equal(g_slot, res.evicted_slot)
+        np.testing.assert_array_equal(g_pos, res.evicted_pos)
+        self.tally.steps += 1
+        self.tally.decisions += int((res.choice >= 0).sum())
+        g_out = widen(unit_view(self.out, self.units))
+        assert np.abs(g_out - res.out).max() <= out_tol(c.dtype), f"attention output off by {np.abs(g_out - res.out).max()}"
+        np.testing.assert_allclose(widen(unit_view(self.lse, self.units)), res.lse, rtol=0, atol=LSE_ATOL)
+        if check_state:
+            compare_state(c, self.st, self.units, f"after gqa step {self.tally.steps}")
+        return res

@@ -1,0 +1,112 @@
+"""GPU parity of the multi-query steps: block-wise evict-and-encode (b tokens per step) and grouped-query decode
+(several query heads per key-value head), against the oracle on every unit."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2402_06262_b200 as R
+import workloads as W
+from harness import BlockParity, DecodeParity, GqaParity, Tally, prefill_parity, unit_view, widen
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def prompt_tensors(w, L):
+    qs, ks, vs = zip(*[W.prompt_chunk(w, b, 0, w.G, L, DEV) for b in range(w.S)])
+    return torch.stack(qs), torch.stack(ks), torch.stack(vs)
+
+
+def block_tokens(w, step0, b, t_pos):
+    toks = [W.decode_tokens(w, step0 + i, [t + i for t in t_pos], DEV) for i in range(b)]
+    return tuple(torch.stack([t[k] for t in toks], dim=2).contiguous() for k in range(3))   # [S][G][b][d]
+
+
+def prefilled(w, L, tally, units):
+    Q, K, V = prompt_tensors(w, L)
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    st = prefill_parity(cache, Q, K, V, [L] * w.S, w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, units, tally, scale=w.scale)
+    return cache, st
+
+
+@pytest.mark.parametrize("b", [1, 2, 4, 8, 16])
+@pytest.mark.parametrize("dtype,d,B", [("bf16", 128, 300), ("f32", 64, 128)])
+def test_block_steps_fill_then_evict(b, dtype, d, B):
+    """Short prompt: the first block steps only fill free slots (some mix freed and free slots), later ones evict
+    b tokens each."""
+    w = W.scaled(W.LLAMA7B_DECODE, S=2, layers=1, heads=3, d=d, dtype=dtype, prompt_lo=B - 21, prompt_hi=B - 21,
+                 B=B, r=9)
+    tally = Tally()
+    cache, st = prefilled(w, B - 21, tally, range(w.U))
+    par = BlockParity(cache, st, range(w.U), b, w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, tally, scale=w.scale)
+    t = B - 21
+    for i in range(max(4, 40 // b)):
+        par.step(*block_tokens(w, i * b, b, [t] * w.S), check_state=True)
+        t += b
+    assert R.roco_device_status(cache) == 0
+    assert tally.decisions > 0
+
+
+def test_block_step_after_eviction_prefill_llama_shape():
+    """Evict-and-encode with b = 16 on a cache built by prefill eviction (B = 1024, d = 128, bf16, sinks)."""
+    w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=8, prompt_lo=1500, prompt_hi=1500)
+    tally = Tally()
+    cache, st = prefilled(w, 1500, tally, range(w.U))
+    par = BlockParity(cache, st, range(w.U), 16, w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, tally, scale=w.scale)
+    for i in range(3):
+        par.step(*block_tokens(w, 16 * i, 16, [1500 + 16 * i]), check_state=(i == 2))
+    assert tally.decisions == 3 * 16 * w.U
+
+
+def test_block_of_one_equals_decode_step_bitwise():
+    w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=4, prompt_lo=200, prompt_hi=200, B=128, r=8)
+    Q, K, V = prompt_tensors(w, 200)
+    caches = [R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV) for _ in range(2)]
+    for c in caches:
+        R.roco_prefill(Q, K, V, [200], w.B, w.r, c, scale=w.scale)
+    out = torch.zeros(w.S, w.G, w.d, dtype=w.torch_dtype, device=DEV)
+    outb = torch.zeros(w.S, w.G, 1, w.d, dtype=w.torch_dtype, device=DEV)
+    ev = torch.zeros(w.S, w.G, dtype=torch.int32, device=DEV)
+    evb = torch.zeros(w.S, w.G, 1, dtype=torch.int32, device=DEV)
+    for i in range(6):
+        q, k, v = W.decode_tokens(w, i, [200 + i], DEV)
+        R.roco_decode_step(caches[0], q, k, v, w.r, out, ev, scale=w.scale)
+        R.roco_block_step(caches[1], q[:, :, None].contiguous(), k[:, :, None].contiguous(), v[:, :, None].contiguous(),
+                          w.r, outb, evb, scale=w.scale)
+        torch.cuda.synchronize()
+        assert torch.equal(ev, evb[..., 0])
+        assert (out.float() - outb[:, :, 0].float()).abs().max() <= 2e-2
+    assert torch.equal(caches[0].pos, caches[1].pos) and torch.equal(caches[0].n, caches[1].n)
+    np.testing.assert_allclose(caches[1].s.cpu().numpy(), caches[0].s.cpu().numpy(), rtol=1e-5)
+
+
+def test_block_step_argument_checks():
+    w = W.scaled(W.TOY, B=32, r=4)
+    cache = R.Cache(w.S, w.G, w.B, w.d, torch.float32, DEV)
+    mk = lambda b: torch.zeros(w.S, w.G, b, w.d, device=DEV)
+    out = lambda b: (torch.zeros(w.S, w.G, b, w.d, device=DEV), torch.zeros(w.S, w.G, b, dtype=torch.int32, device=DEV))
+    with pytest.raises(R.RocoError) as e:
+        R.roco_block_step(cache, mk(17), mk(17), mk(17), 4, *out(17))
+    assert e.value.code == 2
+    with pytest.raises(R.RocoError) as e:
+        R.roco_block_step(cache, mk(4), mk(4), mk(4), 4, *out(4), scope_mode=R.ROCO_SCOPE_LOWEST_R)
+    assert e.value.code == 2
+    with pytest.raises(R.RocoError) as e:
+        R.roco_block_step(cache, mk(8), mk(8), mk(8), 25, *out(8))        # r + b > B
+    assert e.value.code == 1
+
+
+@pytest.mark.parametrize("group", [1, 2, 4, 8])
+@pytest.mark.parametrize("mode", [R.ROCO_SCOPE_EXCLUDE_TOP_R, R.ROCO_SCOPE_LOWEST_R])
+def test_gqa_decode_steps(group, mode):
+    """Zephyr-like grouping: `group` query heads per key-value head, statistics from the group mean."""
+    w = W.scaled(W.LLAMA7B_DECODE, S=2, layers=1, heads=4, prompt_lo=260, prompt_hi=260, B=200, r=12)
+    tally = Tally()
+    cache, st = prefilled(w, 260, tally, range(w.U))
+    par = GqaParity(cache, st, range(w.U), group, w.r, mode, tally, scale=w.scale)
+    for i in range(10):
+        qs = [W.decode_tokens(w, 1000 * g + i, [260 + i] * w.S, DEV)[0] for g in range(group)]
+        _, k, v = W.decode_tokens(w, i, [260 + i] * w.S, DEV)
+        par.step(torch.stack(qs, dim=2).contiguous(), k, v, check_state=(i % 3 == 2))
+    assert R.roco_device_status(cache) == 0 and tally.decisions == 10 * w.U
