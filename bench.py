@@ -199,6 +199,44 @@ def prefill_bench(R, device, small=False, reps=3):
             "launches_per_call": 4, "timing": f"best of {reps} whole roco_prefill calls (both passes, select, gather)"}
 
 
+def multi_bench(R, cache, w, device, reps=6):
+    """Block-wise evict-and-encode (b tokens per pass over the cache) and grouped-query decode on the cache of the
+    decode workload: ms per step, tokens encoded per second, and the speed-up over token-wise eviction (b = 1)."""
+    hbm_peak, _, which = peaks()
+    elem = 2 if w.dtype == "bf16" else 4
+    alg = algorithmic_bytes_per_unit_step(w.B, w.d, elem) * w.U
+    res = {"block": [], "gqa": [], "peak_source": f"of {which}"}
+    dt = w.torch_dtype
+    gen = torch.Generator(device=device); gen.manual_seed(99)
+    def timed(fn):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts)
+    base = None
+    for b in (1, 2, 4, 8, 16):
+        Q, K, V = (torch.randn(w.S, w.G, b, w.d, device=device, generator=gen).to(dt) for _ in range(3))
+        out = torch.zeros(w.S, w.G, b, w.d, dtype=dt, device=device)
+        ev = torch.zeros(w.S, w.G, b, dtype=torch.int32, device=device)
+        ms = timed(lambda: R.roco_block_step(cache, Q, K, V, w.r, out, ev, scale=w.scale))
+        base = base or ms
+        res["block"].append({"b": b, "ms_per_step": ms, "tokens_per_s": w.S * b / ms * 1e3,
+                             "speedup_vs_b1_per_token": base * b / ms, "hbm_frac": alg / ms / 1e6 / hbm_peak})
+    for g in (4, 8):
+        Q = torch.randn(w.S, w.G, g, w.d, device=device, generator=gen).to(dt)
+        k, v = (torch.randn(w.S, w.G, w.d, device=device, generator=gen).to(dt) for _ in range(2))
+        out = torch.zeros(w.S, w.G, g, w.d, dtype=dt, device=device)
+        ev = torch.zeros(w.S, w.G, dtype=torch.int32, device=device)
+        ms = timed(lambda: R.roco_gqa_decode_step(cache, Q, k, v, w.r, out, ev, scale=w.scale))
+        res["gqa"].append({"group": g, "ms_per_step": ms, "hbm_frac": alg / ms / 1e6 / hbm_peak})
+    return res
+
+
 def describe(w, world):
     elem = 2 if w.dtype == "bf16" else 4
     return {"workload": f"{w.name}: S={w.S} x {w.layers} layers x {w.heads} heads, d={w.d}, {w.dtype}, "
@@ -253,6 +291,7 @@ def main():
     ap.add_argument("--workload", default="llama7b_decode")
     ap.add_argument("--small", action="store_true", help="1/16 of the units (for profiler captures)")
     ap.add_argument("--prefill-only", action="store_true", help="run only the prefill measurement")
+    ap.add_argument("--extras", action="store_true", help="also time the block-wise and grouped-query steps")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
     if args.impl == "reference" and rank != 0:
@@ -364,6 +403,10 @@ def main():
 
     del toks, h_toks
     torch.cuda.empty_cache()
+    if args.extras:
+        line["multi_query"] = multi_bench(R, cache, w, device)
+        if R.roco_device_status(cache) != 0:
+            raise RuntimeError("device status word set during the multi-query steps")
     line["prefill"] = prefill_bench(R, device, small=args.small)
 
     if rank == 0:
