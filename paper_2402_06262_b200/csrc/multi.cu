@@ -92,6 +92,169 @@ __device__ inline MultiSmem multi_carve(char *raw, int B, int d, int stages, int
   return m;
 }
 
+// What the policy warps of a multi-query step see of the CTA's shared memory.
+struct PolicyView {
+  float *z;  // [M][Bp] probabilities once p_ready has completed
+  size_t Bp;
+  uint32_t *vkey;
+  float *mkey;
+  signed char *newtok;
+  SelectScratch *sel;
+  float *knew, *vnew, *zn;
+  float *pn;  // [M][nb] probabilities of the new tokens when the consumers have zeroed them in z, else nullptr
+  int *ctl;
+  uint64_t *p_ready, *policy_done;
+};
+
+// The policy warps' part of a multi-query step: free `need` slots (Sec. 4.3 rule on frozen statistics), insert
+// the new tokens in increasing slot order, score the queries against the new keys, and -- once the consumers
+// have normalised -- apply the statistics update.  Called by the kMqPolicyThreads policy threads.
+template <typename T, int D>
+__device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyView &v, int u, int ptid, int live0,
+                                             int need, int live1) {
+  constexpr int kRowBytes = D * (int)sizeof(T);
+  constexpr int kLanesPerRow = kRowBytes / 16;
+  const int M = p.M, nb = p.nb, B = p.B;
+  const size_t Bp = v.Bp;
+  const size_t unit_kv = (size_t)u * B * kRowBytes, unit_st = (size_t)u * B;
+  volatile int *abort_flag = v.ctl;
+  const int plane = ptid & 31, pwarp = ptid >> 5;
+  const int t_new = p.t_next[u];
+  const float *gs = p.s + unit_st, *gq = p.q + unit_st;
+  const int *gn = p.n + unit_st;
+  int *gpos = p.pos + unit_st;
+  for (int j = ptid; j < live1; j += kMqPolicyThreads) v.newtok[j] = -1;
+  for (int i = ptid; i < nb * D; i += kMqPolicyThreads) {
+    v.knew[i] = Elem<T>::load((const T *)p.k_new + (size_t)u * nb * D + i);
+    v.vnew[i] = Elem<T>::load((const T *)p.v_new + (size_t)u * nb * D + i);
+  }
+  named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+  int *tgt = v.ctl + 1;  // [nb] target slots, ascending
+  if (need > 0) {
+    // the rule of Sec. 4.3 applied `need` times on frozen statistics = one pass: the tokens outside the scope
+    // (the live0 - m last in (variance, position) order) never enter it, so the `need` first of the scope in
+    // (mean, position) order leave
+    for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+      const float sj = gs[j], qj = gq[j];
+      const int nj = gn[j];
+      v.vkey[j] = variance_key_fast(sj, qj, nj);
+      v.mkey[j] = mean_fast(sj, nj);
+    }
+    named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+    const int m = scope_size(live0, p.r, p.scope_mode);
+    uint32_t Tv = 0xffffffffu;
+    int Pv = 0x7fffffff;
+    uint32_t rank, ties;
+    if (m < live0) {
+      Tv = radix_select<uint32_t>([&](int j) { return v.vkey[j]; }, [&](int) { return true; }, live0,
+                                  (uint32_t)(m - 1), *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &rank, &ties);
+      if (ties != rank + 1) {
+        uint32_t r2, t2;
+        Pv = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)gpos[j]; },
+                                         [&](int j) { return v.vkey[j] == Tv; }, live0, rank, *v.sel, ptid,
+                                         kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
+      }
+    }
+    auto in_scope = [&](int j) {
+      const uint32_t k = v.vkey[j];
+      return k < Tv || (k == Tv && (Pv == 0x7fffffff || gpos[j] <= Pv));
+    };
+    const uint32_t Tm = radix_select<uint32_t>([&](int j) { return __float_as_uint(v.mkey[j]); }, in_scope, live0,
+                                               (uint32_t)(need - 1), *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy,
+                                               &rank, &ties);
+    int Pm = 0x7fffffff;
+    if (ties != rank + 1) {
+      uint32_t r2, t2;
+      Pm = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)gpos[j]; },
+                                       [&](int j) { return in_scope(j) && __float_as_uint(v.mkey[j]) == Tm; },
+                                       live0, rank, *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
+    }
+    // freed slots in increasing slot order: ballot prefix over chunks of 128 slots
+    int *wtot = v.ctl + 20;  // [4] per-warp counts, [4] = running base
+    if (ptid == 0) wtot[4] = 0;
+    named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+    for (int j0 = 0; j0 < live0; j0 += kMqPolicyThreads) {
+      const int j = j0 + ptid;
+      bool ev = false;
+      if (j < live0 && in_scope(j)) {
+        const uint32_t k = __float_as_uint(v.mkey[j]);
+        ev = k < Tm || (k == Tm && (Pm == 0x7fffffff || gpos[j] <= Pm));
+      }
+      const uint32_t bal = __ballot_sync(0xffffffffu, ev);
+      if (plane == 0) wtot[pwarp] = __popc(bal);
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      int off = wtot[4];
+      for (int w = 0; w < pwarp; ++w) off += wtot[w];
+      const int rk = off + __popc(bal & ((1u << plane) - 1u));
+      if (ev && rk < nb) tgt[rk] = j;
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      if (ptid == 0) wtot[4] += wtot[0] + wtot[1] + wtot[2] + wtot[3];
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+    }
+    if (ptid == 0 && wtot[4] != need) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
+  }
+  if (ptid < nb - need) tgt[need + ptid] = live0 + ptid;  // free slots behind the occupied ones
+  named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+  // the new tokens take the target slots: evicted positions out, new K/V and positions in
+  if (ptid < nb) {
+    int slot = tgt[ptid];
+    if (slot < 0 || slot >= B) slot = 0;  // only after corrupt statistics (status bit set above)
+    p.ev_slot[(size_t)u * nb + ptid] = ptid < need ? slot : -1;
+    if (p.ev_pos) p.ev_pos[(size_t)u * nb + ptid] = ptid < need ? gpos[slot] : -1;
+    v.newtok[slot] = (signed char)ptid;
+    gpos[slot] = t_new + ptid;
+  }
+  for (int w = ptid; w < nb * 2 * kLanesPerRow; w += kMqPolicyThreads) {  // in-place overwrite, 16 bytes each
+    const int i = w / (2 * kLanesPerRow), c = w % (2 * kLanesPerRow);
+    const bool isv = c >= kLanesPerRow;
+    const int cc = isv ? c - kLanesPerRow : c;
+    int slot = tgt[i];
+    if (slot < 0 || slot >= B) slot = 0;
+    const uint4 val = *((const uint4 *)((isv ? p.v_new : p.k_new) + ((size_t)u * nb + i) * kRowBytes) + cc);
+    *((uint4 *)(const_cast<char *>(isv ? p.V : p.K) + unit_kv + (size_t)slot * kRowBytes) + cc) = val;
+  }
+  // scores of every query against every new token, from k_new directly (log2 domain)
+  const float zscale = p.scale * kLog2e;
+  for (int w = ptid; w < M * nb; w += kMqPolicyThreads) {
+    const int i = w / nb, jn = w % nb;
+    const T *qrow = (const T *)p.Q + ((size_t)u * M + i) * D;
+    float acc = 0.f;
+    for (int c = 0; c < D; ++c) acc = fmaf(Elem<T>::load(qrow + c), v.knew[jn * D + c], acc);
+    v.zn[w] = acc * zscale;
+  }
+  if (ptid == 0) { p.live[u] = live1; p.t_next[u] = t_new + nb; }
+  named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+  if (ptid == 0) mbar_arrive(v.policy_done);
+
+  // statistics of Sec. 4.3 once the probabilities are in shared memory
+  mbar_wait(v.p_ready, 0, abort_flag, p.status);
+  for (int j = ptid; j < live1; j += kMqPolicyThreads) {
+    const int jn = v.newtok[j];
+    const bool fresh = jn >= 0;
+    float ds = 0.f, dq = 0.f;
+    int dn;
+    if (p.kind == kMqGqa) {
+      for (int i = 0; i < M; ++i) ds += (fresh && v.pn) ? v.pn[i * nb + jn] : v.z[(size_t)i * Bp + j];
+      ds /= (float)M;  // group-wise averaged attention score
+      dq = ds * ds;
+      dn = 1;
+    } else {
+      const int i0 = fresh ? jn : 0;  // query i sees new token jn only if i >= jn
+      for (int i = i0; i < M; ++i) {
+        const float pij = (fresh && v.pn) ? v.pn[i * nb + jn] : v.z[(size_t)i * Bp + j];
+        ds += pij;
+        dq = fmaf(pij, pij, dq);
+      }
+      dn = M - i0;
+    }
+    const float s0 = fresh ? 0.f : gs[j], q0 = fresh ? 0.f : gq[j];
+    const int n0 = fresh ? 0 : gn[j];
+    p.s[unit_st + j] = s0 + ds;
+    p.q[unit_st + j] = q0 + dq;
+    p.n[unit_st + j] = n0 + dn;
+  }
+}
+
 template <typename T, int D>
 __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParams p) {
   constexpr int kRowBytes = D * (int)sizeof(T);
@@ -148,141 +311,11 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
 
   if (warp >= kMqPolicyWarp0) {
     // ---------------------------------------------------------- policy: free slots, insert, statistics
-    const int ptid = tid - kMqPolicyWarp0 * 32, plane = ptid & 31, pwarp = ptid >> 5;
-    const int t_new = p.t_next[u];
-    const float *gs = p.s + unit_st, *gq = p.q + unit_st;
-    const int *gn = p.n + unit_st;
-    int *gpos = p.pos + unit_st;
-    for (int j = ptid; j < live1; j += kMqPolicyThreads) sm.newtok[j] = -1;
-    for (int i = ptid; i < nb * D; i += kMqPolicyThreads) {
-      sm.knew[i] = Elem<T>::load((const T *)p.k_new + (size_t)u * nb * D + i);
-      sm.vnew[i] = Elem<T>::load((const T *)p.v_new + (size_t)u * nb * D + i);
-    }
-    named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-    int *tgt = sm.ctl + 1;  // [nb] target slots, ascending
-    if (need > 0) {
-      // the rule of Sec. 4.3 applied `need` times on frozen statistics = one pass: the tokens outside the scope
-      // (the live0 - m last in (variance, position) order) never enter it, so the `need` first of the scope in
-      // (mean, position) order leave
-      for (int j = ptid; j < live0; j += kMqPolicyThreads) {
-        const float sj = gs[j], qj = gq[j];
-        const int nj = gn[j];
-        sm.vkey[j] = variance_key_fast(sj, qj, nj);
-        sm.mkey[j] = mean_fast(sj, nj);
-      }
-      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      const int m = scope_size(live0, p.r, p.scope_mode);
-      uint32_t Tv = 0xffffffffu;
-      int Pv = 0x7fffffff;
-      uint32_t rank, ties;
-      if (m < live0) {
-        Tv = radix_select<uint32_t>([&](int j) { return sm.vkey[j]; }, [&](int) { return true; }, live0,
-                                    (uint32_t)(m - 1), *sm.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &rank, &ties);
-        if (ties != rank + 1) {
-          uint32_t r2, t2;
-          Pv = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)gpos[j]; },
-                                           [&](int j) { return sm.vkey[j] == Tv; }, live0, rank, *sm.sel, ptid,
-                                           kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
-        }
-      }
-      auto in_scope = [&](int j) {
-        const uint32_t k = sm.vkey[j];
-        return k < Tv || (k == Tv && (Pv == 0x7fffffff || gpos[j] <= Pv));
-      };
-      const uint32_t Tm = radix_select<uint32_t>([&](int j) { return __float_as_uint(sm.mkey[j]); }, in_scope, live0,
-                                                 (uint32_t)(need - 1), *sm.sel, ptid, kMqPolicyThreads, kMqBarPolicy,
-                                                 &rank, &ties);
-      int Pm = 0x7fffffff;
-      if (ties != rank + 1) {
-        uint32_t r2, t2;
-        Pm = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)gpos[j]; },
-                                         [&](int j) { return in_scope(j) && __float_as_uint(sm.mkey[j]) == Tm; },
-                                         live0, rank, *sm.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
-      }
-      // freed slots in increasing slot order: ballot prefix over chunks of 128 slots
-      int *wtot = sm.ctl + 20;  // [4] per-warp counts, [4] = running base
-      if (ptid == 0) wtot[4] = 0;
-      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      for (int j0 = 0; j0 < live0; j0 += kMqPolicyThreads) {
-        const int j = j0 + ptid;
-        bool ev = false;
-        if (j < live0 && in_scope(j)) {
-          const uint32_t k = __float_as_uint(sm.mkey[j]);
-          ev = k < Tm || (k == Tm && (Pm == 0x7fffffff || gpos[j] <= Pm));
-        }
-        const uint32_t bal = __ballot_sync(0xffffffffu, ev);
-        if (plane == 0) wtot[pwarp] = __popc(bal);
-        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-        int off = wtot[4];
-        for (int w = 0; w < pwarp; ++w) off += wtot[w];
-        const int rk = off + __popc(bal & ((1u << plane) - 1u));
-        if (ev && rk < nb) tgt[rk] = j;
-        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-        if (ptid == 0) wtot[4] += wtot[0] + wtot[1] + wtot[2] + wtot[3];
-        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      }
-      if (ptid == 0 && wtot[4] != need) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
-    }
-    if (ptid < nb - need) tgt[need + ptid] = live0 + ptid;  // free slots behind the occupied ones
-    named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-    // the new tokens take the target slots: evicted positions out, new K/V and positions in
-    if (ptid < nb) {
-      int slot = tgt[ptid];
-      if (slot < 0 || slot >= B) slot = 0;  // only after corrupt statistics (status bit set above)
-      p.ev_slot[(size_t)u * nb + ptid] = ptid < need ? slot : -1;
-      if (p.ev_pos) p.ev_pos[(size_t)u * nb + ptid] = ptid < need ? gpos[slot] : -1;
-      sm.newtok[slot] = (signed char)ptid;
-      gpos[slot] = t_new + ptid;
-    }
-    for (int w = ptid; w < nb * 2 * kLanesPerRow; w += kMqPolicyThreads) {  // in-place overwrite, 16 bytes each
-      const int i = w / (2 * kLanesPerRow), c = w % (2 * kLanesPerRow);
-      const bool isv = c >= kLanesPerRow;
-      const int cc = isv ? c - kLanesPerRow : c;
-      int slot = tgt[i];
-      if (slot < 0 || slot >= B) slot = 0;
-      const uint4 val = *((const uint4 *)((isv ? p.v_new : p.k_new) + ((size_t)u * nb + i) * kRowBytes) + cc);
-      *((uint4 *)(const_cast<char *>(isv ? p.V : p.K) + unit_kv + (size_t)slot * kRowBytes) + cc) = val;
-    }
-    // scores of every query against every new token, from k_new directly (log2 domain)
-    const float zscale = p.scale * kLog2e;
-    for (int w = ptid; w < M * nb; w += kMqPolicyThreads) {
-      const int i = w / nb, jn = w % nb;
-      const T *qrow = (const T *)p.Q + ((size_t)u * M + i) * D;
-      float acc = 0.f;
-      for (int c = 0; c < D; ++c) acc = fmaf(Elem<T>::load(qrow + c), sm.knew[jn * D + c], acc);
-      sm.zn[w] = acc * zscale;
-    }
-    if (ptid == 0) { p.live[u] = live1; p.t_next[u] = t_new + nb; }
-    named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-    if (ptid == 0) mbar_arrive(sm.policy_done);
-
-    // statistics of Sec. 4.3 once the probabilities are in shared memory
-    mbar_wait(sm.p_ready, 0, abort_flag, p.status);
-    for (int j = ptid; j < live1; j += kMqPolicyThreads) {
-      const int jn = sm.newtok[j];
-      const bool fresh = jn >= 0;
-      float ds = 0.f, dq = 0.f;
-      int dn;
-      if (p.kind == kMqGqa) {
-        for (int i = 0; i < M; ++i) ds += sm.z[(size_t)i * Bp + j];
-        ds /= (float)M;  // group-wise averaged attention score
-        dq = ds * ds;
-        dn = 1;
-      } else {
-        const int i0 = fresh ? jn : 0;  // query i sees new token jn only if i >= jn
-        for (int i = i0; i < M; ++i) {
-          const float pij = sm.z[(size_t)i * Bp + j];
-          ds += pij;
-          dq = fmaf(pij, pij, dq);
-        }
-        dn = M - i0;
-      }
-      const float s0 = fresh ? 0.f : gs[j], q0 = fresh ? 0.f : gq[j];
-      const int n0 = fresh ? 0 : gn[j];
-      p.s[unit_st + j] = s0 + ds;
-      p.q[unit_st + j] = q0 + dq;
-      p.n[unit_st + j] = n0 + dn;
-    }
+    PolicyView v;
+    v.z = sm.z; v.Bp = Bp; v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok; v.sel = sm.sel;
+    v.knew = sm.knew; v.vnew = sm.vnew; v.zn = sm.zn; v.pn = nullptr; v.ctl = sm.ctl; v.p_ready = sm.p_ready;
+    v.policy_done = sm.policy_done;
+    multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
     return;
   }
 
