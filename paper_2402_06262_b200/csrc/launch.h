@@ -33,6 +33,10 @@ roco_status launch_budget_select_gather(const roco_cache &c, int Lmax, const int
                                         const float *q_full, int *dst, unsigned long long *sortbuf, int Lp2max,
                                         cudaStream_t stream);
 
+// Tensor map (CUtensorMap, 128 bytes, passed as void*) over a [rows][128] bf16 matrix with boxes of 64 columns x
+// box_rows rows and the 128-byte swizzle; false when the driver entry point is unavailable or the encode fails.
+bool make_tensor_map_rows128_bf16(void *map, const void *base, unsigned long long rows, unsigned box_rows);
+
 // Multi-query steps (block-wise evict-and-encode: kind 0, nb == M; grouped-query decode: kind 1, nb == 1).
 int multi_max_queries();
 bool multi_fits(int B, int d, int M, int nb);

@@ -9,6 +9,8 @@
 // policy warps that select, insert and update the statistics while the consumers stream), with the M x B score
 // matrix in shared memory.  Each consumer warp owns four queries and a share of every tile's rows, so the
 // per-row arithmetic grows with M while the HBM traffic per unit stays that of one decode step.
+#include <cuda.h>
+
 #include "common.cuh"
 #include "launch.h"
 #include "select.cuh"
@@ -272,7 +274,6 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int u = blockIdx.x;
   const size_t unit_kv = (size_t)u * B * kRowBytes;
-  const size_t unit_st = (size_t)u * B;
 
   if (tid == 0) {
     for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kMqConsumerWarps); }
@@ -462,6 +463,295 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
   }
 }
 
+// ------------------------------------------------------------------------------------------------------------
+// Tensor-core variant (bf16, d = 128): the M x 64 score block of a tile is one row of warp-level MMAs
+// (m16n8k16, queries on the M axis, padded to 16), and so is the 16 x 128 output update, which takes the per-row
+// arithmetic off the CUDA cores: the step stays HBM-bound for any M <= 16.  Tiles arrive through TMA tensor maps
+// with the 128-byte swizzle so that ldmatrix reads them without bank conflicts.
+
+struct MultiTcSmem {
+  char *ring;  // 1024-byte aligned, `stages` tiles of 64 rows x 128 bf16 (two 64-column halves of 8 KiB)
+  float *z;    // [M][Bp], Bp = B rounded up to 64
+  uint32_t *vkey;
+  float *mkey;
+  signed char *newtok;
+  SelectScratch *sel;
+  float *knew, *vnew, *zn, *pn;
+  uint64_t *full, *empty, *p_ready, *policy_done;
+  int *ctl;
+};
+
+__host__ __device__ inline size_t multi_tc_smem_bytes(int B, int stages, int M, int nb) {
+  const size_t Bp = align_up((size_t)B, 64);
+  size_t b = (size_t)stages * kMqTile;
+  b += (size_t)M * Bp * 4 + 2 * Bp * 4 + Bp;
+  b += sizeof(SelectScratch);
+  b += 2 * (size_t)nb * 128 * 4 + 2 * (size_t)M * nb * 4;
+  b = align_up(b, 8) + (2 * (size_t)stages + 2) * 8 + 64 * 4;
+  return b + 1024;
+}
+
+__device__ inline MultiTcSmem multi_tc_carve(char *raw, int B, int stages, int M, int nb) {
+  MultiTcSmem m;
+  char *p = (char *)align_up((size_t)raw, 1024);
+  const size_t Bp = align_up((size_t)B, 64);
+  m.ring = p; p += (size_t)stages * kMqTile;
+  m.z = (float *)p; p += (size_t)M * Bp * 4;
+  m.vkey = (uint32_t *)p; p += Bp * 4;
+  m.mkey = (float *)p; p += Bp * 4;
+  m.newtok = (signed char *)p; p += Bp;
+  m.sel = (SelectScratch *)p; p += sizeof(SelectScratch);
+  m.knew = (float *)p; p += (size_t)nb * 128 * 4;
+  m.vnew = (float *)p; p += (size_t)nb * 128 * 4;
+  m.zn = (float *)p; p += (size_t)M * nb * 4;
+  m.pn = (float *)p; p += (size_t)M * nb * 4;
+  p = (char *)align_up((size_t)p, 8);
+  m.full = (uint64_t *)p; p += stages * 8;
+  m.empty = (uint64_t *)p; p += stages * 8;
+  m.p_ready = (uint64_t *)p; p += 8;
+  m.policy_done = (uint64_t *)p; p += 8;
+  m.ctl = (int *)p;
+  return m;
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D (16 x 8, fp32) += A (16 x 16, bf16, row-major) * B (16 x 8, bf16, column-major)
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+               "{%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+// byte offset of the 16-byte chunk `chunk` (0..15 over the 128 columns) of row `row` inside a swizzled tile
+__device__ __forceinline__ uint32_t tile_chunk_offset(int row, int chunk) {
+  return (uint32_t)((chunk >> 3) * 8192 + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+}
+
+__global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_constant__ CUtensorMap mapK,
+                                                                   const __grid_constant__ CUtensorMap mapV,
+                                                                   const MultiParams p) {
+  using T = __nv_bfloat16;
+  constexpr int D = 128, kTileRows = 64;
+  extern __shared__ char mq_smem_raw[];
+  const int M = p.M, nb = p.nb, B = p.B, stages = p.stages;
+  const MultiTcSmem sm = multi_tc_carve(mq_smem_raw, B, stages, M, nb);
+  volatile int *abort_flag = sm.ctl;
+  const size_t Bp = align_up((size_t)B, 64);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int u = blockIdx.x;
+
+  if (tid == 0) {
+    for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kMqConsumerWarps); }
+    mbar_init(sm.p_ready, kMqConsumerWarps);
+    mbar_init(sm.policy_done, 1);
+    sm.ctl[0] = 0;
+    mbar_init_fence();
+  }
+  int live0 = p.live[u];
+  if (live0 < 0 || live0 > B) {
+    if (tid == 0) atomicOr(p.status, ROCO_DEV_BAD_LIVE);
+    live0 = live0 < 0 ? 0 : B;
+  }
+  int need = live0 + nb - B;
+  if (need < 0) need = 0;
+  const int live1 = live0 - need + nb;
+  const int n_tiles = (live1 + kTileRows - 1) / kTileRows;
+  __syncthreads();
+
+  if (warp == kMqProducerWarp) {
+    if (lane == 0) {
+      for (int g = 0; g < 2 * n_tiles; ++g) {
+        const int st = g % stages;
+        if (g >= stages) mbar_wait(&sm.empty[st], ((g / stages) - 1) & 1, abort_flag, p.status);
+        const int it = (g < n_tiles) ? g : g - n_tiles;
+        const CUtensorMap *map = (g < n_tiles) ? &mapK : &mapV;
+        char *dst = sm.ring + (size_t)st * kMqTile;
+        const int row = u * B + it * kTileRows;
+        mbar_expect_tx(&sm.full[st], kMqTile);
+        tma_load_2d(dst, map, 0, row, &sm.full[st]);
+        tma_load_2d(dst + 8192, map, 64, row, &sm.full[st]);
+      }
+    }
+    return;
+  }
+
+  if (warp >= kMqPolicyWarp0) {
+    PolicyView v;
+    v.z = sm.z; v.Bp = Bp; v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok; v.sel = sm.sel;
+    v.knew = sm.knew; v.vnew = sm.vnew; v.zn = sm.zn; v.pn = sm.pn; v.ctl = sm.ctl; v.p_ready = sm.p_ready;
+    v.policy_done = sm.policy_done;
+    multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
+    return;
+  }
+
+  // -------------------------------------------------------------- consumers
+  const float zscale = p.scale * kLog2e;
+  const int g = lane >> 2, tq = lane & 3;
+  const bool row_lo = g < M, row_hi = g + 8 < M;
+  // A fragments of Q (16 x 128, rows >= M are zero): a[s] covers k = 16 s .. 16 s + 15
+  uint32_t qa[8][4];
+  {
+    const T *Qu = (const T *)p.Q + (size_t)u * M * D;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      const int k0 = s * 16 + tq * 2;
+      qa[s][0] = row_lo ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)g * D + k0) : 0u;
+      qa[s][1] = row_hi ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)(g + 8) * D + k0) : 0u;
+      qa[s][2] = row_lo ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)g * D + k0 + 8) : 0u;
+      qa[s][3] = row_hi ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)(g + 8) * D + k0 + 8) : 0u;
+    }
+  }
+
+  // ---- scores: each warp takes 8 keys of every 64-key tile, all queries:  Z[16 x 8] = Q[16 x 128] K^T
+  for (int it = 0; it < n_tiles; ++it) {
+    const int st = it % stages;
+    mbar_wait(&sm.full[st], (it / stages) & 1, abort_flag, p.status);
+    const uint32_t tile = smem_u32(sm.ring + (size_t)st * kMqTile);
+    float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int sp = 0; sp < 4; ++sp) {
+      uint32_t kb[4];
+      ldmatrix_x4(tile + tile_chunk_offset(warp * 8 + (lane & 7), sp * 4 + (lane >> 3)), kb);
+      mma_bf16_16816(c, qa[2 * sp], kb[0], kb[1]);
+      mma_bf16_16816(c, qa[2 * sp + 1], kb[2], kb[3]);
+    }
+    const int j = it * kTileRows + warp * 8 + tq * 2;
+    if (row_lo) {
+      if (j < live1) sm.z[(size_t)g * Bp + j] = c[0] * zscale;
+      if (j + 1 < live1) sm.z[(size_t)g * Bp + j + 1] = c[1] * zscale;
+    }
+    if (row_hi) {
+      if (j < live1) sm.z[(size_t)(g + 8) * Bp + j] = c[2] * zscale;
+      if (j + 1 < live1) sm.z[(size_t)(g + 8) * Bp + j + 1] = c[3] * zscale;
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.empty[st]);
+  }
+
+  // scores of the new tokens from k_new, with the causal mask inside a block
+  mbar_wait(sm.policy_done, 0, abort_flag, p.status);
+  named_bar_sync(kMqBarConsumers, kMqConsumers);
+  for (int w = tid; w < M * nb; w += kMqConsumers) {
+    const int i = w / nb, jn = w % nb;
+    int slot = sm.ctl[1 + jn];
+    if (slot < 0 || slot >= B) slot = 0;
+    sm.z[(size_t)i * Bp + slot] = (p.kind == kMqBlock && jn > i) ? -INFINITY : sm.zn[w];
+  }
+  named_bar_sync(kMqBarConsumers, kMqConsumers);
+
+  // ---- one softmax per query, each by one warp; the tail of the last tile is cleared for the MMAs below
+  for (int i = warp; i < M; i += kMqConsumerWarps) {
+    float *zi = sm.z + (size_t)i * Bp;
+    float zmax = -INFINITY;
+    for (int j = lane; j < live1; j += 32) zmax = fmaxf(zmax, zi[j]);
+    zmax = warp_max(zmax);
+    float zsum = 0.f;
+    for (int j = lane; j < live1; j += 32) {
+      const float ex = exp2f(zi[j] - zmax);
+      zi[j] = ex;
+      zsum += ex;
+    }
+    zsum = warp_sum(zsum);
+    const float inv = 1.f / zsum;
+    for (int j = lane; j < live1; j += 32) zi[j] *= inv;
+    for (int j = live1 + lane; j < n_tiles * kTileRows; j += 32) zi[j] = 0.f;
+    if (lane == 0 && p.lse) p.lse[(size_t)u * M + i] = (zmax + log2f(zsum)) * kLn2;
+  }
+  named_bar_sync(kMqBarConsumers, kMqConsumers);
+  // the new tokens' values come from v_new: keep their probabilities aside and clear them in z, so that the
+  // streamed V rows of those slots (possibly read before the overwrite) contribute nothing
+  for (int w = tid; w < M * nb; w += kMqConsumers) {
+    const int i = w / nb, jn = w % nb;
+    int slot = sm.ctl[1 + jn];
+    if (slot < 0 || slot >= B) slot = 0;
+    sm.pn[w] = sm.z[(size_t)i * Bp + slot];
+    sm.z[(size_t)i * Bp + slot] = 0.f;
+  }
+  __syncwarp();
+  if (lane == 0) mbar_arrive(sm.p_ready);
+  named_bar_sync(kMqBarConsumers, kMqConsumers);
+
+  // ---- out[16 x 128] += P[16 x 64] V[64 x 128]: each warp owns 16 output columns
+  float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+  for (int it = 0; it < n_tiles; ++it) {
+    const int gg = n_tiles + it;
+    const int st = gg % stages;
+    mbar_wait(&sm.full[st], (gg / stages) & 1, abort_flag, p.status);
+    const uint32_t tile = smem_u32(sm.ring + (size_t)st * kMqTile);
+    // slots >= live0 were free before this step: whatever the stream brought for them (they may hold anything,
+    // NaN included, and 0 * NaN would poison the MMA) is cleared in the 16 columns this warp reads
+    if ((it + 1) * kTileRows > live0) {
+      const int r0 = live0 > it * kTileRows ? live0 - it * kTileRows : 0;
+      char *tp = sm.ring + (size_t)st * kMqTile;
+      for (int w = lane; w < (kTileRows - r0) * 2; w += 32) {
+        const int row = r0 + (w >> 1);
+        *reinterpret_cast<uint4 *>(tp + tile_chunk_offset(row, warp * 2 + (w & 1))) = make_uint4(0u, 0u, 0u, 0u);
+      }
+      __syncwarp();
+    }
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+      const int j = it * kTileRows + ks * 16 + tq * 2;
+      uint32_t pa[4];
+      const float *zl = sm.z + (size_t)g * Bp + j, *zh = sm.z + (size_t)(g + 8) * Bp + j;
+      pa[0] = row_lo ? pack_bf16x2(zl[0], zl[1]) : 0u;
+      pa[1] = row_hi ? pack_bf16x2(zh[0], zh[1]) : 0u;
+      pa[2] = row_lo ? pack_bf16x2(zl[8], zl[9]) : 0u;
+      pa[3] = row_hi ? pack_bf16x2(zh[8], zh[9]) : 0u;
+      uint32_t vb[4];
+      const int mi = lane >> 3;
+      ldmatrix_x4_trans(tile + tile_chunk_offset(ks * 16 + (mi & 1) * 8 + (lane & 7), warp * 2 + (mi >> 1)), vb);
+      mma_bf16_16816(o[0], pa, vb[0], vb[1]);
+      mma_bf16_16816(o[1], pa, vb[2], vb[3]);
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.empty[st]);
+  }
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    const int dcol = warp * 16 + nt * 8 + tq * 2;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int qi = g + 8 * h;
+      if (qi < M) {
+        float o0 = o[nt][2 * h], o1 = o[nt][2 * h + 1];
+        for (int jn = 0; jn < nb; ++jn) {
+          const float pj = sm.pn[qi * nb + jn];
+          o0 = fmaf(pj, sm.vnew[jn * D + dcol], o0);
+          o1 = fmaf(pj, sm.vnew[jn * D + dcol + 1], o1);
+        }
+        *reinterpret_cast<uint32_t *>((T *)p.out + ((size_t)u * M + qi) * D + dcol) = pack_bf16x2(o0, o1);
+      }
+    }
+  }
+}
+
+static int multi_tc_pick_stages(int B, int M, int nb) {
+  const size_t per_sm = 227 * 1024;
+  for (int ctas = 2; ctas >= 1; --ctas)
+    for (int st = 6; st >= 3; --st)
+      if ((multi_tc_smem_bytes(B, st, M, nb) + 1024) * ctas <= per_sm) return st;
+  return 0;
+}
+
 static int multi_pick_stages(int B, int d, int M, int nb) {
   const size_t per_sm = 227 * 1024;
   for (int ctas = 2; ctas >= 1; --ctas)
@@ -481,7 +771,9 @@ static cudaError_t launch_multi_t(MultiParams &p, int U, cudaStream_t stream) {
 
 int multi_max_queries() { return kMqMaxQ; }
 
-bool multi_fits(int B, int d, int M, int nb) { return multi_pick_stages(B, d, M, nb) > 0; }
+bool multi_fits(int B, int d, int M, int nb) {
+  return multi_pick_stages(B, d, M, nb) > 0 || (d == 128 && multi_tc_pick_stages(B, M, nb) > 0);
+}
 
 roco_status launch_multi_step(const roco_cache &c, int kind, int M, int nb, const void *Q, const void *k_new,
                               const void *v_new, int r, int scope_mode, float scale, void *out, float *lse,
@@ -492,10 +784,23 @@ roco_status launch_multi_step(const roco_cache &c, int kind, int M, int nb, cons
   p.Q = (const char *)Q; p.k_new = (const char *)k_new; p.v_new = (const char *)v_new;
   p.out = (char *)out; p.lse = lse; p.ev_slot = ev_slot; p.ev_pos = ev_pos;
   p.B = c.B; p.r = r; p.scope_mode = scope_mode; p.M = M; p.nb = nb; p.kind = kind; p.scale = scale;
-  p.stages = multi_pick_stages(c.B, c.d, M, nb);
-  if (p.stages == 0) return ROCO_ERR_UNSUPPORTED;
   const int U = c.S * c.G;
   cudaError_t err;
+  if (c.kv_dtype == ROCO_BF16 && c.d == 128 && (long long)U * c.B < 0x7fffffffLL) {
+    // tensor-core path; falls through to the CUDA-core path if the tensor maps cannot be built
+    CUtensorMap mapK, mapV;
+    p.stages = multi_tc_pick_stages(c.B, M, nb);
+    if (p.stages > 0 && make_tensor_map_rows128_bf16(&mapK, c.K, (unsigned long long)U * c.B, 64) &&
+        make_tensor_map_rows128_bf16(&mapV, c.V, (unsigned long long)U * c.B, 64)) {
+      const size_t smem = multi_tc_smem_bytes(c.B, p.stages, M, nb);
+      err = cudaFuncSetAttribute(multi_step_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (err != cudaSuccess) return ROCO_ERR_CUDA;
+      multi_step_tc_kernel<<<U, kMqThreads, smem, stream>>>(mapK, mapV, p);
+      return cudaGetLastError() == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
+    }
+  }
+  p.stages = multi_pick_stages(c.B, c.d, M, nb);
+  if (p.stages == 0) return ROCO_ERR_UNSUPPORTED;
   if (c.kv_dtype == ROCO_BF16 && c.d == 128) err = launch_multi_t<__nv_bfloat16, 128>(p, U, stream);
   else if (c.kv_dtype == ROCO_BF16 && c.d == 64) err = launch_multi_t<__nv_bfloat16, 64>(p, U, stream);
   else if (c.kv_dtype == ROCO_F32 && c.d == 128) err = launch_multi_t<float, 128>(p, U, stream);

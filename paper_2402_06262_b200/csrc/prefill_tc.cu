@@ -481,6 +481,19 @@ static bool make_map(CUtensorMap *map, const void *base, int U, int Lmax) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// [rows][128] bf16 as a 2-D tensor; box = 64 columns x box_rows rows, 128-byte swizzle, zero fill
+bool make_tensor_map_rows128_bf16(void *map, const void *base, unsigned long long rows, unsigned box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)kTcD, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)kTcD * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(static_cast<CUtensorMap *>(map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool prefill_tc_supported(int kv_dtype, int d) { return kv_dtype == ROCO_BF16 && d == kTcD && encode_fn() != nullptr; }
 
 roco_status launch_prefill_stats_tc(int S, int G, int Lmax, const int *lens_dev, int maxlen, const void *Q,
