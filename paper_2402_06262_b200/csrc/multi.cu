@@ -471,7 +471,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
 
 struct MultiTcSmem {
   char *ring;  // 1024-byte aligned, `stages` tiles of 64 rows x 128 bf16 (two 64-column halves of 8 KiB)
-  float *z;    // [M][Bp], Bp = B rounded up to 64
+  float *z;    // [M][Bp], Bp = multi_tc_row_stride(B)
   uint32_t *vkey;
   float *mkey;
   signed char *newtok;
@@ -481,8 +481,12 @@ struct MultiTcSmem {
   int *ctl;
 };
 
+// Row stride of the score matrix: the budget rounded up to a tile, plus 8 floats so that the eight query rows a
+// warp touches at once (MMA fragment rows) fall into different shared-memory banks.
+__host__ __device__ inline size_t multi_tc_row_stride(int B) { return align_up((size_t)B, 64) + 8; }
+
 __host__ __device__ inline size_t multi_tc_smem_bytes(int B, int stages, int M, int nb) {
-  const size_t Bp = align_up((size_t)B, 64);
+  const size_t Bp = multi_tc_row_stride(B);
   size_t b = (size_t)stages * kMqTile;
   b += (size_t)M * Bp * 4 + 2 * Bp * 4 + Bp;
   b += sizeof(SelectScratch);
@@ -494,7 +498,7 @@ __host__ __device__ inline size_t multi_tc_smem_bytes(int B, int stages, int M, 
 __device__ inline MultiTcSmem multi_tc_carve(char *raw, int B, int stages, int M, int nb) {
   MultiTcSmem m;
   char *p = (char *)align_up((size_t)raw, 1024);
-  const size_t Bp = align_up((size_t)B, 64);
+  const size_t Bp = multi_tc_row_stride(B);
   m.ring = p; p += (size_t)stages * kMqTile;
   m.z = (float *)p; p += (size_t)M * Bp * 4;
   m.vkey = (uint32_t *)p; p += Bp * 4;
@@ -554,7 +558,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
   const int M = p.M, nb = p.nb, B = p.B, stages = p.stages;
   const MultiTcSmem sm = multi_tc_carve(mq_smem_raw, B, stages, M, nb);
   volatile int *abort_flag = sm.ctl;
-  const size_t Bp = align_up((size_t)B, 64);
+  const size_t Bp = multi_tc_row_stride(B);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int u = blockIdx.x;
 
