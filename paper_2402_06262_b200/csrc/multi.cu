@@ -103,6 +103,7 @@ struct PolicyView {
   signed char *newtok;
   SelectScratch *sel;
   float *knew, *vnew, *zn;
+  float *qf;  // [M][D] queries as fp32, filled by the policy warps themselves (nullptr: read Q from global)
   float *pn;  // [M][nb] probabilities of the new tokens when the consumers have zeroed them in z, else nullptr
   int *ctl;
   uint64_t *p_ready, *policy_done;
@@ -126,9 +127,21 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
   const int *gn = p.n + unit_st;
   int *gpos = p.pos + unit_st;
   for (int j = ptid; j < live1; j += kMqPolicyThreads) v.newtok[j] = -1;
-  for (int i = ptid; i < nb * D; i += kMqPolicyThreads) {
-    v.knew[i] = Elem<T>::load((const T *)p.k_new + (size_t)u * nb * D + i);
-    v.vnew[i] = Elem<T>::load((const T *)p.v_new + (size_t)u * nb * D + i);
+  {  // new keys / values (and the queries) as fp32 in shared memory, 16-byte loads issued back to back
+    constexpr int kEPC = Elem<T>::kPerChunk;
+    const uint4 *gk = reinterpret_cast<const uint4 *>(p.k_new + (size_t)u * nb * kRowBytes);
+    const uint4 *gv = reinterpret_cast<const uint4 *>(p.v_new + (size_t)u * nb * kRowBytes);
+    const uint4 *gqr = reinterpret_cast<const uint4 *>(p.Q + (size_t)u * M * kRowBytes);
+    const int nkv = nb * D / kEPC, nq = v.qf ? M * D / kEPC : 0;
+#pragma unroll 4
+    for (int i = ptid; i < 2 * nkv + nq; i += kMqPolicyThreads) {
+      const uint4 c = i < nkv ? gk[i] : (i < 2 * nkv ? gv[i - nkv] : gqr[i - 2 * nkv]);
+      float *dst = i < nkv ? v.knew + i * kEPC : (i < 2 * nkv ? v.vnew + (i - nkv) * kEPC : v.qf + (i - 2 * nkv) * kEPC);
+      float f[kEPC];
+      Elem<T>::unpack(c, f);
+#pragma unroll
+      for (int e = 0; e < kEPC; ++e) dst[e] = f[e];
+    }
   }
   named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
   int *tgt = v.ctl + 1;  // [nb] target slots, ascending
@@ -136,6 +149,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     // the rule of Sec. 4.3 applied `need` times on frozen statistics = one pass: the tokens outside the scope
     // (the live0 - m last in (variance, position) order) never enter it, so the `need` first of the scope in
     // (mean, position) order leave
+#pragma unroll 4
     for (int j = ptid; j < live0; j += kMqPolicyThreads) {
       const float sj = gs[j], qj = gq[j];
       const int nj = gn[j];
@@ -161,39 +175,68 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
       const uint32_t k = v.vkey[j];
       return k < Tv || (k == Tv && (Pv == 0x7fffffff || gpos[j] <= Pv));
     };
-    const uint32_t Tm = radix_select<uint32_t>([&](int j) { return __float_as_uint(v.mkey[j]); }, in_scope, live0,
-                                               (uint32_t)(need - 1), *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy,
-                                               &rank, &ties);
-    int Pm = 0x7fffffff;
-    if (ties != rank + 1) {
-      uint32_t r2, t2;
-      Pm = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)gpos[j]; },
-                                       [&](int j) { return in_scope(j) && __float_as_uint(v.mkey[j]) == Tm; },
-                                       live0, rank, *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
-    }
-    // freed slots in increasing slot order: ballot prefix over chunks of 128 slots
-    int *wtot = v.ctl + 20;  // [4] per-warp counts, [4] = running base
-    if (ptid == 0) wtot[4] = 0;
-    named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-    for (int j0 = 0; j0 < live0; j0 += kMqPolicyThreads) {
-      const int j = j0 + ptid;
-      bool ev = false;
-      if (j < live0 && in_scope(j)) {
-        const uint32_t k = __float_as_uint(v.mkey[j]);
-        ev = k < Tm || (k == Tm && (Pm == 0x7fffffff || gpos[j] <= Pm));
+    int *cnt = v.ctl + 20, *list = v.ctl + 24;  // freed slots, unordered
+    if (need == 1) {
+      // one victim: the in-scope token first in (mean, position) order
+      float bm = INFINITY;
+      int bs = -1;
+      for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+        if (!in_scope(j)) continue;
+        const float mean = v.mkey[j];
+        if (mean < bm) { bm = mean; bs = j; }
+        else if (mean == bm && bs >= 0 && gpos[j] < gpos[bs]) bs = j;
       }
-      const uint32_t bal = __ballot_sync(0xffffffffu, ev);
-      if (plane == 0) wtot[pwarp] = __popc(bal);
+      int bp = bs >= 0 ? gpos[bs] : 0x7fffffff;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, bm, o);
+        const int op = __shfl_xor_sync(0xffffffffu, bp, o);
+        const int os = __shfl_xor_sync(0xffffffffu, bs, o);
+        if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+      }
+      if (plane == 0) { v.sel->red_mean[pwarp] = bm; v.sel->red_pos[pwarp] = bp; v.sel->red_slot[pwarp] = bs; }
       named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      int off = wtot[4];
-      for (int w = 0; w < pwarp; ++w) off += wtot[w];
-      const int rk = off + __popc(bal & ((1u << plane) - 1u));
-      if (ev && rk < nb) tgt[rk] = j;
+      if (ptid == 0) {
+        bm = v.sel->red_mean[0]; bp = v.sel->red_pos[0]; bs = v.sel->red_slot[0];
+        for (int w = 1; w < kMqPolicyThreads / 32; ++w) {
+          const float om = v.sel->red_mean[w];
+          const int op = v.sel->red_pos[w], os = v.sel->red_slot[w];
+          if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+        }
+        if (bs < 0) { atomicOr(p.status, ROCO_DEV_BAD_VICTIM); bs = 0; }
+        tgt[0] = bs;
+      }
+    } else {
+      const uint32_t Tm = radix_select<uint32_t>([&](int j) { return __float_as_uint(v.mkey[j]); }, in_scope, live0,
+                                                 (uint32_t)(need - 1), *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy,
+                                                 &rank, &ties);
+      int Pm = 0x7fffffff;
+      if (ties != rank + 1) {
+        uint32_t r2, t2;
+        Pm = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)gpos[j]; },
+                                         [&](int j) { return in_scope(j) && __float_as_uint(v.mkey[j]) == Tm; },
+                                         live0, rank, *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
+      }
+      // collect the freed slots (at most 16), then order them by slot index
+      if (ptid == 0) *cnt = 0;
       named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      if (ptid == 0) wtot[4] += wtot[0] + wtot[1] + wtot[2] + wtot[3];
+      for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+        if (!in_scope(j)) continue;
+        const uint32_t k = __float_as_uint(v.mkey[j]);
+        if (k < Tm || (k == Tm && (Pm == 0x7fffffff || gpos[j] <= Pm))) {
+          const int at = atomicAdd(cnt, 1);
+          if (at < kMqMaxQ) list[at] = j;
+        }
+      }
       named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      const int found = *cnt < kMqMaxQ ? *cnt : kMqMaxQ;
+      if (ptid == 0 && *cnt != need) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
+      if (ptid < found) {
+        int rk = 0;
+        for (int x = 0; x < found; ++x) rk += list[x] < list[ptid];
+        if (rk < nb) tgt[rk] = list[ptid];
+      }
     }
-    if (ptid == 0 && wtot[4] != need) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
   }
   if (ptid < nb - need) tgt[need + ptid] = live0 + ptid;  // free slots behind the occupied ones
   named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
@@ -206,6 +249,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     v.newtok[slot] = (signed char)ptid;
     gpos[slot] = t_new + ptid;
   }
+#pragma unroll 4
   for (int w = ptid; w < nb * 2 * kLanesPerRow; w += kMqPolicyThreads) {  // in-place overwrite, 16 bytes each
     const int i = w / (2 * kLanesPerRow), c = w % (2 * kLanesPerRow);
     const bool isv = c >= kLanesPerRow;
@@ -217,12 +261,17 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
   }
   // scores of every query against every new token, from k_new directly (log2 domain)
   const float zscale = p.scale * kLog2e;
-  for (int w = ptid; w < M * nb; w += kMqPolicyThreads) {
+  for (int w = pwarp; w < M * nb; w += kMqPolicyThreads / 32) {  // one dot product per warp and turn
     const int i = w / nb, jn = w % nb;
     const T *qrow = (const T *)p.Q + ((size_t)u * M + i) * D;
     float acc = 0.f;
-    for (int c = 0; c < D; ++c) acc = fmaf(Elem<T>::load(qrow + c), v.knew[jn * D + c], acc);
-    v.zn[w] = acc * zscale;
+    if (v.qf) {
+      for (int c = plane; c < D; c += 32) acc = fmaf(v.qf[i * D + c], v.knew[jn * D + c], acc);
+    } else {
+      for (int c = plane; c < D; c += 32) acc = fmaf(Elem<T>::load(qrow + c), v.knew[jn * D + c], acc);
+    }
+    acc = warp_sum(acc);
+    if (plane == 0) v.zn[w] = acc * zscale;
   }
   if (ptid == 0) { p.live[u] = live1; p.t_next[u] = t_new + nb; }
   named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
@@ -314,7 +363,8 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
     // ---------------------------------------------------------- policy: free slots, insert, statistics
     PolicyView v;
     v.z = sm.z; v.Bp = Bp; v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok; v.sel = sm.sel;
-    v.knew = sm.knew; v.vnew = sm.vnew; v.zn = sm.zn; v.pn = nullptr; v.ctl = sm.ctl; v.p_ready = sm.p_ready;
+    v.knew = sm.knew; v.vnew = sm.vnew; v.zn = sm.zn; v.qf = nullptr; v.pn = nullptr; v.ctl = sm.ctl;
+    v.p_ready = sm.p_ready;
     v.policy_done = sm.policy_done;
     multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
     return;
@@ -476,7 +526,7 @@ struct MultiTcSmem {
   float *mkey;
   signed char *newtok;
   SelectScratch *sel;
-  float *knew, *vnew, *zn, *pn;
+  float *knew, *vnew, *zn, *pn, *qf;
   uint64_t *full, *empty, *p_ready, *policy_done;
   int *ctl;
 };
@@ -490,7 +540,7 @@ __host__ __device__ inline size_t multi_tc_smem_bytes(int B, int stages, int M, 
   size_t b = (size_t)stages * kMqTile;
   b += (size_t)M * Bp * 4 + 2 * Bp * 4 + Bp;
   b += sizeof(SelectScratch);
-  b += 2 * (size_t)nb * 128 * 4 + 2 * (size_t)M * nb * 4;
+  b += (2 * (size_t)nb + (size_t)M) * 128 * 4 + 2 * (size_t)M * nb * 4;
   b = align_up(b, 8) + (2 * (size_t)stages + 2) * 8 + 64 * 4;
   return b + 1024;
 }
@@ -509,6 +559,7 @@ __device__ inline MultiTcSmem multi_tc_carve(char *raw, int B, int stages, int M
   m.vnew = (float *)p; p += (size_t)nb * 128 * 4;
   m.zn = (float *)p; p += (size_t)M * nb * 4;
   m.pn = (float *)p; p += (size_t)M * nb * 4;
+  m.qf = (float *)p; p += (size_t)M * 128 * 4;
   p = (char *)align_up((size_t)p, 8);
   m.full = (uint64_t *)p; p += stages * 8;
   m.empty = (uint64_t *)p; p += stages * 8;
@@ -600,7 +651,8 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
   if (warp >= kMqPolicyWarp0) {
     PolicyView v;
     v.z = sm.z; v.Bp = Bp; v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok; v.sel = sm.sel;
-    v.knew = sm.knew; v.vnew = sm.vnew; v.zn = sm.zn; v.pn = sm.pn; v.ctl = sm.ctl; v.p_ready = sm.p_ready;
+    v.knew = sm.knew; v.vnew = sm.vnew; v.zn = sm.zn; v.qf = sm.qf; v.pn = sm.pn; v.ctl = sm.ctl;
+    v.p_ready = sm.p_ready;
     v.policy_done = sm.policy_done;
     multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
     return;
