@@ -149,7 +149,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     // the rule of Sec. 4.3 applied `need` times on frozen statistics = one pass: the tokens outside the scope
     // (the live0 - m last in (variance, position) order) never enter it, so the `need` first of the scope in
     // (mean, position) order leave
-#pragma unroll 4
+#pragma unroll 8
     for (int j = ptid; j < live0; j += kMqPolicyThreads) {
       const float sj = gs[j], qj = gq[j];
       const int nj = gn[j];
@@ -261,17 +261,29 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
   }
   // scores of every query against every new token, from k_new directly (log2 domain)
   const float zscale = p.scale * kLog2e;
-  for (int w = pwarp; w < M * nb; w += kMqPolicyThreads / 32) {  // one dot product per warp and turn
-    const int i = w / nb, jn = w % nb;
-    const T *qrow = (const T *)p.Q + ((size_t)u * M + i) * D;
-    float acc = 0.f;
-    if (v.qf) {
-      for (int c = plane; c < D; c += 32) acc = fmaf(v.qf[i * D + c], v.knew[jn * D + c], acc);
-    } else {
-      for (int c = plane; c < D; c += 32) acc = fmaf(Elem<T>::load(qrow + c), v.knew[jn * D + c], acc);
+  if (v.qf) {
+    // one dot product per thread and turn, operands in shared memory; the element order is rotated by the lane
+    // so that the 32 lanes of a warp (different keys, same offset) hit different banks
+    for (int w = ptid; w < M * nb; w += kMqPolicyThreads) {
+      const int i = w / nb, jn = w % nb;
+      const float *qr = v.qf + i * D, *kr = v.knew + jn * D;
+      float acc = 0.f;
+#pragma unroll 8
+      for (int c = 0; c < D; ++c) {
+        const int cc = (c + plane) & (D - 1);
+        acc = fmaf(qr[cc], kr[cc], acc);
+      }
+      v.zn[w] = acc * zscale;
     }
-    acc = warp_sum(acc);
-    if (plane == 0) v.zn[w] = acc * zscale;
+  } else {
+    for (int w = pwarp; w < M * nb; w += kMqPolicyThreads / 32) {  // one dot product per warp and turn
+      const int i = w / nb, jn = w % nb;
+      const T *qrow = (const T *)p.Q + ((size_t)u * M + i) * D;
+      float acc = 0.f;
+      for (int c = plane; c < D; c += 32) acc = fmaf(Elem<T>::load(qrow + c), v.knew[jn * D + c], acc);
+      acc = warp_sum(acc);
+      if (plane == 0) v.zn[w] = acc * zscale;
+    }
   }
   if (ptid == 0) { p.live[u] = live1; p.t_next[u] = t_new + nb; }
   named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
