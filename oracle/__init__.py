@@ -16,6 +16,8 @@ from .build import build as build_library
 
 EXCLUDE_TOP_R, LOWEST_R = 0, 1
 EVICT_FIRST, ATTEND_FIRST = 0, 1
+(POLICY_ROCO, POLICY_RANDOM, POLICY_RECENCY, POLICY_STREAMLLM, POLICY_SCISSORHANDS, POLICY_H2O, POLICY_TOVA,
+ POLICY_MAS_WINDOW) = range(8)
 
 _lib = None
 
@@ -223,3 +225,21 @@ def gqa_step(st: State, Q, k_new, v_new, r, mode, scale, delta=1e-5, force_victi
                                      _p(k_new), _p(v_new), C.c_int(r), C.c_int(mode), C.c_double(scale),
                                      C.c_double(delta), _p(fv), _p(out), _p(lse), _p(es), _p(ep), _p(ch), _p(nt))
     return StepResult(out, lse, es, ep, ch, nt.astype(bool))
+
+
+def policy_step(st: State, qv, k_new, v_new, policy, r, scale, rnd=None, delta=1e-5, force_victim=None):
+    """One decode step (evict, insert, attend) under one of the Table 1 policies, in place on `st`.
+    Returns (StepResult, quant_near [U][B] bool).  rnd: [U] uint32 draws for POLICY_RANDOM."""
+    qv, k_new, v_new = _f64(qv), _f64(k_new), _f64(v_new)
+    U, B, d = st.U, st.B, st.d
+    out = np.zeros((U, d)); lse = np.zeros(U)
+    es = np.zeros(U, np.int32); ep = np.zeros(U, np.int32); ch = np.zeros(U, np.int32); nt = np.zeros(U, np.int32)
+    qn = np.zeros((U, B), np.int32)
+    fv = None if force_victim is None else _i32(force_victim)
+    rn = None if rnd is None else np.ascontiguousarray(rnd, dtype=np.uint32)
+    lib().roco_oracle_policy_step_batch(C.c_int(U), _p(st.K), _p(st.V), _p(st.s), _p(st.q), _p(st.n), _p(st.pos),
+                                        _p(st.live), _p(st.t_next), C.c_int(B), C.c_int(d), _p(qv), _p(k_new),
+                                        _p(v_new), C.c_int(policy), C.c_int(r), _p(rn), C.c_double(scale),
+                                        C.c_double(delta), _p(fv), _p(out), _p(lse), _p(es), _p(ep), _p(ch), _p(nt),
+                                        _p(qn))
+    return StepResult(out, lse, es, ep, ch, nt.astype(bool)), qn.astype(bool)

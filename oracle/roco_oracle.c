@@ -28,6 +28,7 @@
  *   prefill-stage eviction to B .... Sec. 4.3 last paragraph / Sec. 5.1 "Other Details" (B = len x rate)
  *   block-wise evict-and-encode .... Sec. 5.3 "Overhead", App. B (b tokens freed and encoded per eviction step)
  *   grouped-query attention ........ Sec. 5.3 / App. A (group-wise averaged attention score updates the statistics)
+ *   other policies ................. Table 1 with Sec. 4.1 (importance scores), Sec. 4.2 (local window), Sec. 5.1
  *
  * Readings where the paper is silent (stated once here, in words):
  *   - ties: scope membership by (variance asc, position asc); victim by (mean asc, position asc);
@@ -587,5 +588,111 @@ void roco_oracle_gqa_step_batch(int U, double *K, double *V, double *s, double *
                               Q + qb, k_new + vb, v_new + vb, r, mode, scale, delta,
                               force_victim ? force_victim[u] : -1, out + qb, lse + (size_t)u * group,
                               evicted_slot + u, evicted_pos + u, choice + u, near_tie + u);
+  }
+}
+
+/* ---------------------------------------------- the other eviction policies of Table 1 (Sec. 4.1, 4.2, 5.1) -- */
+
+enum {
+  ROCO_ORACLE_POLICY_ROCO = 0,         /* MAS + standard-deviation scope (Sec. 4.3), EXCLUDE_TOP_R reading        */
+  ROCO_ORACLE_POLICY_RANDOM = 1,       /* Sec. 4.1: a randomly chosen pair (the draw is an input)                  */
+  ROCO_ORACLE_POLICY_RECENCY = 2,      /* Sec. 4.1: the farthest token                                             */
+  ROCO_ORACLE_POLICY_STREAMLLM = 3,    /* Sec. 5.1: the first token after the 4 initial attention-sink tokens      */
+  ROCO_ORACLE_POLICY_SCISSORHANDS = 4, /* Sec. 4.1 AQAS (1 = above-average probability) + local window of size r   */
+  ROCO_ORACLE_POLICY_H2O = 5,          /* Sec. 4.1 AAS (accumulated probability) + local window of size r          */
+  ROCO_ORACLE_POLICY_TOVA = 6,         /* Sec. 4.1 LTAS (the last query's probability), no scope restriction       */
+  ROCO_ORACLE_POLICY_MAS_WINDOW = 7    /* Sec. 4.3 preliminary experiment: MAS + local window of size r            */
+};
+
+/* One decode step (evict, insert, attend: Fig. 1) under one of the policies above.
+ * State: s = accumulated probability (Acc), n = Count for every policy; q = Acc^square, except under
+ * SCISSORHANDS, where it accumulates the quantised score (1 if the token's probability exceeds the average
+ * 1/live of this query, else 0), and under TOVA, where it holds the last query's probability.
+ * Local window (Sec. 4.2): tokens outside a window of the r most recent positions are evictable, i.e. pos < t - r
+ * with t the position of the incoming token.  Ties: (score asc, position asc).
+ * rnd: the random draw for RANDOM (victim = rnd mod live).  quant_near [B] (may be NULL): set to 1 where a
+ * SCISSORHANDS quantisation falls within delta (relative) of the average. */
+void roco_oracle_policy_step_unit(double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
+                                  int *t_next, int B, int d, const double *qv, const double *k_new,
+                                  const double *v_new, int policy, int r, unsigned rnd, double scale, double delta,
+                                  int force_victim, double *out, double *lse, int *evicted_slot, int *evicted_pos,
+                                  int *choice, int *near_tie, int *quant_near) {
+  const int t = *t_next;
+  int slot, own = -1, near = 0;
+  *evicted_slot = -1;
+  *evicted_pos = -1;
+  if (*live == B) {
+    if (policy == ROCO_ORACLE_POLICY_ROCO) {
+      own = roco_oracle_select(s, q, n, pos, B, r, ROCO_ORACLE_EXCLUDE_TOP_R, delta, &near, NULL);
+    } else if (policy == ROCO_ORACLE_POLICY_RANDOM) {
+      own = (int)(rnd % (unsigned)B);
+    } else {
+      const int windowed = policy == ROCO_ORACLE_POLICY_SCISSORHANDS || policy == ROCO_ORACLE_POLICY_H2O ||
+                           policy == ROCO_ORACLE_POLICY_MAS_WINDOW;
+      int any = 0;
+      for (int j = 0; j < B; ++j) if (!windowed || pos[j] < t - r) any = 1;
+      double best = 0.0, second = INFINITY;
+      for (int j = 0; j < B; ++j) {
+        if (windowed && any && !(pos[j] < t - r)) continue;
+        if (policy == ROCO_ORACLE_POLICY_STREAMLLM && pos[j] < 4) continue;
+        double sc = 0.0; /* RECENCY, STREAMLLM: position alone decides */
+        if (policy == ROCO_ORACLE_POLICY_H2O) sc = s[j];
+        if (policy == ROCO_ORACLE_POLICY_SCISSORHANDS || policy == ROCO_ORACLE_POLICY_TOVA) sc = q[j];
+        if (policy == ROCO_ORACLE_POLICY_MAS_WINDOW) sc = s[j] / n[j];
+        if (own < 0 || sc < best || (sc == best && pos[j] < pos[own])) {
+          if (own >= 0) second = best < second ? best : second;
+          best = sc; own = j;
+        } else if (sc < second) {
+          second = sc;
+        }
+      }
+      if (own < 0) { own = 0; for (int j = 1; j < B; ++j) if (pos[j] < pos[own]) own = j; } /* all sinks */
+      const int real_valued = policy == ROCO_ORACLE_POLICY_H2O || policy == ROCO_ORACLE_POLICY_TOVA ||
+                              policy == ROCO_ORACLE_POLICY_MAS_WINDOW;
+      if (real_valued && second - best <= delta * (second + best)) near = 1;
+    }
+    slot = (force_victim >= 0 && force_victim < B && near) ? force_victim : own;
+    *evicted_slot = slot;
+    *evicted_pos = pos[slot];
+  } else {
+    slot = (*live)++;
+  }
+  insert_token(K, V, s, q, n, pos, slot, d, k_new, v_new, t);
+  const int m = *live;
+  double *p = (double *)malloc(sizeof(double) * (size_t)m);
+  *lse = softmax_row(qv, K, m, d, scale, p);
+  for (int c = 0; c < d; ++c) out[c] = 0.0;
+  for (int j = 0; j < m; ++j) {
+    for (int c = 0; c < d; ++c) out[c] += p[j] * V[(size_t)j * d + c];
+    s[j] += p[j];
+    n[j] += 1;
+    if (quant_near) quant_near[j] = 0;
+    if (policy == ROCO_ORACLE_POLICY_SCISSORHANDS) {
+      q[j] += (p[j] * m > 1.0) ? 1.0 : 0.0;
+      if (quant_near && fabs(p[j] * m - 1.0) <= delta) quant_near[j] = 1;
+    } else if (policy == ROCO_ORACLE_POLICY_TOVA) {
+      q[j] = p[j];
+    } else {
+      q[j] += p[j] * p[j];
+    }
+  }
+  free(p);
+  *choice = own;
+  *near_tie = near;
+  *t_next = t + 1;
+}
+
+void roco_oracle_policy_step_batch(int U, double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
+                                   int *t_next, int B, int d, const double *qv, const double *k_new,
+                                   const double *v_new, int policy, int r, const unsigned *rnd, double scale,
+                                   double delta, const int *force_victim, double *out, double *lse, int *evicted_slot,
+                                   int *evicted_pos, int *choice, int *near_tie, int *quant_near) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int u = 0; u < U; ++u) {
+    size_t kb = (size_t)u * B * d, sb = (size_t)u * B, vb = (size_t)u * d;
+    roco_oracle_policy_step_unit(K + kb, V + kb, s + sb, q + sb, n + sb, pos + sb, live + u, t_next + u, B, d, qv + vb,
+                                 k_new + vb, v_new + vb, policy, r, rnd ? rnd[u] : 0u, scale, delta,
+                                 force_victim ? force_victim[u] : -1, out + vb, lse + u, evicted_slot + u,
+                                 evicted_pos + u, choice + u, near_tie + u, quant_near ? quant_near + sb : NULL);
   }
 }
