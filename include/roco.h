@@ -164,6 +164,32 @@ roco_status roco_decode_step(roco_cache *cache, const void *q, const void *k_new
                              int scope_mode, int step_order, float scale, void *attn_out, float *lse_out,
                              int32_t *evicted_slot, int32_t *evicted_pos, void *stream);
 
+/* The eviction policies of Table 1 (importance score of Sec. 4.1 + eviction scope of Sec. 4.2 / 4.3). */
+typedef enum {
+  ROCO_POLICY_ROCO = 0,         /* mean attention score + standard-deviation scope (EXCLUDE_TOP_R)            */
+  ROCO_POLICY_RANDOM = 1,       /* a random cached pair: victim slot = rnd[unit] mod B                        */
+  ROCO_POLICY_RECENCY = 2,      /* the farthest token (lowest position)                                       */
+  ROCO_POLICY_STREAMLLM = 3,    /* the first token after the 4 initial attention-sink tokens                  */
+  ROCO_POLICY_SCISSORHANDS = 4, /* lowest accumulated quantised score outside the local window of size r      */
+  ROCO_POLICY_H2O = 5,          /* lowest accumulated attention score outside the local window of size r      */
+  ROCO_POLICY_TOVA = 6,         /* lowest attention score from the last query                                 */
+  ROCO_POLICY_MAS_WINDOW = 7    /* lowest mean attention score outside the local window (Sec. 4.3 experiment) */
+} roco_policy;
+
+/*
+ * roco_decode_step (order ROCO_EVICT_FIRST) under any policy of Table 1, on the same cache layout.
+ * The local window of Sec. 4.2 is the r most recent positions: a cached token is evictable if pos < t_next - r.
+ * Ties go to the lowest position.  s and n are Acc and Count for every policy; the q array holds Acc^square,
+ * except under ROCO_POLICY_SCISSORHANDS (accumulated quantised score: +1 when the token's probability exceeds
+ * the average 1/live of the step) and under ROCO_POLICY_TOVA (the last query's probability) -- so a cache should
+ * be stepped with one policy throughout.
+ *   rnd   [S][G] uint32 device array of random draws, read only by ROCO_POLICY_RANDOM (else may be NULL)
+ *   r     0 <= r < B: scope parameter of ROCO_POLICY_ROCO, window size of the windowed policies, else ignored
+ */
+roco_status roco_decode_step_policy(roco_cache *cache, const void *q, const void *k_new, const void *v_new,
+                                    int policy, int r, const uint32_t *rnd, float scale, void *attn_out,
+                                    float *lse_out, int32_t *evicted_slot, int32_t *evicted_pos, void *stream);
+
 /*
  * Block-wise evict-and-encode (Sec. 5.3 "Overhead", App. B: "the block size b controls the number of tokens being
  * freed and encoded within one eviction step"): b new tokens per unit in one pass over the cache.

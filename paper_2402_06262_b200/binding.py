@@ -18,10 +18,12 @@ ROCO_OK = 0
 ROCO_F32, ROCO_BF16 = 0, 1
 ROCO_SCOPE_EXCLUDE_TOP_R, ROCO_SCOPE_LOWEST_R = 0, 1
 ROCO_EVICT_FIRST, ROCO_ATTEND_FIRST = 0, 1
+(ROCO_POLICY_ROCO, ROCO_POLICY_RANDOM, ROCO_POLICY_RECENCY, ROCO_POLICY_STREAMLLM, ROCO_POLICY_SCISSORHANDS,
+ ROCO_POLICY_H2O, ROCO_POLICY_TOVA, ROCO_POLICY_MAS_WINDOW) = range(8)
 
 EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes", "roco_prefill",
            "roco_prefill_uses_tensor_cores", "roco_prefill_static", "roco_prefill_workspace_bytes_lowest_r",
-           "roco_block_step", "roco_gqa_decode_step",
+           "roco_block_step", "roco_gqa_decode_step", "roco_decode_step_policy",
            "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status")
 
 
@@ -74,6 +76,10 @@ def lib() -> C.CDLL:
             fn.restype = C.c_int
             fn.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                            C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.roco_decode_step_policy.restype = C.c_int
+        L.roco_decode_step_policy.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                              C.c_int, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
+                                              C.c_void_p, C.c_void_p]
         L.roco_decode_step_host.restype = C.c_int
         L.roco_decode_step_host.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                             C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -178,6 +184,17 @@ def roco_decode_step(cache: Cache, q, k_new, v_new, r: int, attn_out, evicted_sl
                                 scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot), _ptr(evicted_pos), _stream())
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_decode_step")
+
+
+def roco_decode_step_policy(cache: Cache, q, k_new, v_new, policy: int, r: int, attn_out, evicted_slot,
+                            evicted_pos=None, lse_out=None, rnd=None, scale: Optional[float] = None):
+    """Decode step (evict, insert, attend) under one of the Table 1 policies; rnd: [S][G] int32/uint32 draws."""
+    scale = cache.d ** -0.5 if scale is None else scale
+    rc = lib().roco_decode_step_policy(C.byref(cache.c), _ptr(q), _ptr(k_new), _ptr(v_new), policy, r, _ptr(rnd),
+                                       scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot), _ptr(evicted_pos),
+                                       _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_decode_step_policy")
 
 
 def roco_block_step(cache: Cache, Q, K_new, V_new, r: int, attn_out, evicted_slot, evicted_pos=None, lse_out=None,

@@ -135,8 +135,23 @@ roco_status roco_decode_step(roco_cache *cache, const void *q, const void *k_new
   if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
   if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
   if (step_order != ROCO_EVICT_FIRST && step_order != ROCO_ATTEND_FIRST) return ROCO_ERR_INVALID_ARG;
-  return launch_decode_step(*cache, q, k_new, v_new, r, scope_mode, step_order, scale, attn_out, lse_out,
-                            evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
+  return launch_decode_step(*cache, q, k_new, v_new, r, scope_mode, step_order, ROCO_POLICY_ROCO, nullptr, scale,
+                            attn_out, lse_out, evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
+}
+
+roco_status roco_decode_step_policy(roco_cache *cache, const void *q, const void *k_new, const void *v_new,
+                                    int policy, int r, const uint32_t *rnd, float scale, void *attn_out,
+                                    float *lse_out, int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {
+  roco_status st = check_cache(cache);
+  if (st != ROCO_OK) return st;
+  if (!q || !k_new || !v_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
+  if (policy < ROCO_POLICY_ROCO || policy > ROCO_POLICY_MAS_WINDOW) return ROCO_ERR_INVALID_ARG;
+  if (r < 0 || r >= cache->B) return ROCO_ERR_INVALID_ARG;
+  if (policy == ROCO_POLICY_RANDOM && !rnd) return ROCO_ERR_INVALID_ARG;
+  if (policy == ROCO_POLICY_STREAMLLM && cache->B <= 4) return ROCO_ERR_INVALID_ARG;  // room for the four sinks
+  return launch_decode_step(*cache, q, k_new, v_new, r, ROCO_SCOPE_EXCLUDE_TOP_R, ROCO_EVICT_FIRST, policy, rnd, scale,
+                            attn_out, lse_out, evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
 }
 
 roco_status roco_block_step(roco_cache *cache, const void *Q, const void *K_new, const void *V_new, int b, int r,

@@ -36,6 +36,8 @@ struct DecodeParams {
   float *lse;
   int *ev_slot, *ev_pos;
   int B, r, scope_mode, order, stages;
+  int policy;           // roco_policy
+  const unsigned *rnd;  // [U] random draws (ROCO_POLICY_RANDOM)
   float scale;
 };
 
@@ -184,7 +186,11 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
         const float s0 = fresh ? 0.f : p.s[unit_st + j], q0 = fresh ? 0.f : p.q[unit_st + j];
         const int n0 = fresh ? 0 : p.n[unit_st + j];
         p.s[unit_st + j] = s0 + pj;
-        p.q[unit_st + j] = fmaf(pj, pj, q0);
+        // Acc^square, except for the two policies of Table 1 that keep something else in this array
+        float q1 = fmaf(pj, pj, q0);
+        if (p.policy == ROCO_POLICY_SCISSORHANDS) q1 = q0 + (pj * (float)live_att > 1.f ? 1.f : 0.f);  // AQAS
+        if (p.policy == ROCO_POLICY_TOVA) q1 = pj;                                                    // LTAS
+        p.q[unit_st + j] = q1;
         p.n[unit_st + j] = n0 + 1;
       }
     };
@@ -195,9 +201,31 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     int e = live0, ev_slot = -1, ev_pos = -1;
     if (full) {
       // Sec. 4: "when the buffer is full, an eviction policy is executed"
-      const int m = scope_size(B, p.r, p.scope_mode);
-      e = group_select_victim(p.s + unit_st, p.q + unit_st, p.n + unit_st, p.pos + unit_st, B, m, sm.vkey, sm.mkey,
-                              *sm.sel, ptid, kPolicyThreads, kBarPolicy);
+      const float *gs = p.s + unit_st, *gq = p.q + unit_st;
+      const int *gn = p.n + unit_st, *gpos = p.pos + unit_st;
+      if (p.policy == ROCO_POLICY_ROCO) {
+        const int m = scope_size(B, p.r, p.scope_mode);
+        e = group_select_victim(gs, gq, gn, gpos, B, m, sm.vkey, sm.mkey, *sm.sel, ptid, kPolicyThreads, kBarPolicy);
+      } else if (p.policy == ROCO_POLICY_RANDOM) {
+        e = (int)(p.rnd[u] % (unsigned)B);
+      } else {
+        // Table 1: importance score (Sec. 4.1) and local window of the r most recent positions (Sec. 4.2)
+        const int pol = p.policy, horizon = t_new - p.r;
+        const bool windowed = pol == ROCO_POLICY_SCISSORHANDS || pol == ROCO_POLICY_H2O || pol == ROCO_POLICY_MAS_WINDOW;
+        e = group_argmin(
+            [&](int j) {
+              if (pol == ROCO_POLICY_H2O) return gs[j];
+              if (pol == ROCO_POLICY_SCISSORHANDS || pol == ROCO_POLICY_TOVA) return gq[j];
+              if (pol == ROCO_POLICY_MAS_WINDOW) return mean_fast(gs[j], gn[j]);
+              return 0.f;  // recency, StreamLLM: the position alone decides
+            },
+            [&](int j) {
+              if (windowed) return gpos[j] < horizon;
+              if (pol == ROCO_POLICY_STREAMLLM) return gpos[j] >= 4;
+              return true;
+            },
+            gpos, B, *sm.sel, ptid, kPolicyThreads, kBarPolicy);
+      }
       if (e < 0) {
         if (ptid == 0) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
         e = 0;
@@ -384,14 +412,15 @@ static cudaError_t launch_decode_td(DecodeParams &p, int U, cudaStream_t stream)
 }
 
 roco_status launch_decode_step(const roco_cache &c, const void *q, const void *k_new, const void *v_new, int r,
-                               int scope_mode, int step_order, float scale, void *out, float *lse, int32_t *ev_slot,
-                               int32_t *ev_pos, cudaStream_t stream) {
+                               int scope_mode, int step_order, int policy, const unsigned *rnd, float scale, void *out,
+                               float *lse, int32_t *ev_slot, int32_t *ev_pos, cudaStream_t stream) {
   DecodeParams p;
   p.K = (const char *)c.K; p.V = (const char *)c.V;
   p.s = c.s; p.q = c.q; p.n = c.n; p.pos = c.pos; p.live = c.live; p.t_next = c.t_next; p.status = c.status;
   p.qv = (const char *)q; p.k_new = (const char *)k_new; p.v_new = (const char *)v_new;
   p.out = (char *)out; p.lse = lse; p.ev_slot = ev_slot; p.ev_pos = ev_pos;
   p.B = c.B; p.r = r; p.scope_mode = scope_mode; p.order = step_order; p.scale = scale;
+  p.policy = policy; p.rnd = rnd;
   const int U = c.S * c.G;
   cudaError_t err;
   if (c.kv_dtype == ROCO_BF16 && c.d == 128) err = launch_decode_td<__nv_bfloat16, 128>(p, U, stream);

@@ -9,8 +9,8 @@
 namespace roco {
 
 roco_status launch_decode_step(const roco_cache &c, const void *q, const void *k_new, const void *v_new, int r,
-                               int scope_mode, int step_order, float scale, void *out, float *lse, int32_t *ev_slot,
-                               int32_t *ev_pos, cudaStream_t stream);
+                               int scope_mode, int step_order, int policy, const unsigned *rnd, float scale, void *out,
+                               float *lse, int32_t *ev_slot, int32_t *ev_pos, cudaStream_t stream);
 
 // Row log-sum-exp and column statistics of the causal softmax, CUDA-core path (any supported dtype/d).
 // lens_dev: [S] device copy of the prompt lengths.  lse, s_full, q_full: [U][Lmax].

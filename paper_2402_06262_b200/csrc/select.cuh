@@ -156,6 +156,40 @@ __device__ __forceinline__ int group_select_victim(const float *s, const float *
   return bs;
 }
 
+// Slot first in (score asc, position asc) order among the slots [0, live) with eligible(j); -1 if there is none.
+// Same calling convention as group_select_victim.  Used by the policies of Table 1 other than RoCo.
+template <typename ScoreF, typename EligF>
+__device__ __forceinline__ int group_argmin(ScoreF score, EligF eligible, const int *pos, int live, SelectScratch &sc,
+                                            int tid, int nthreads, int bar_id) {
+  float bm = INFINITY;
+  int bs = -1;
+  for (int j = tid; j < live; j += nthreads) {
+    if (!eligible(j)) continue;
+    const float v = score(j);
+    if (bs < 0 || v < bm) { bm = v; bs = j; }
+    else if (v == bm && pos[j] < pos[bs]) bs = j;
+  }
+  int bp = (bs >= 0) ? pos[bs] : 0x7fffffff;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, bm, o);
+    const int op = __shfl_xor_sync(0xffffffffu, bp, o);
+    const int os = __shfl_xor_sync(0xffffffffu, bs, o);
+    if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+  }
+  const int warp = tid >> 5, nwarps = nthreads >> 5;
+  if ((tid & 31) == 0) { sc.red_mean[warp] = bm; sc.red_pos[warp] = bp; sc.red_slot[warp] = bs; }
+  named_bar_sync(bar_id, nthreads);
+  bm = sc.red_mean[0]; bp = sc.red_pos[0]; bs = sc.red_slot[0];
+  for (int w = 1; w < nwarps; ++w) {
+    const float om = sc.red_mean[w];
+    const int op = sc.red_pos[w], os = sc.red_slot[w];
+    if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+  }
+  named_bar_sync(bar_id, nthreads);
+  return bs;
+}
+
 // Scope size for `live` cached tokens (Sec. 4.3 / Sec. 1 readings), clipped to [1, live].
 __device__ __host__ __forceinline__ int scope_size(int live, int r, int scope_mode) {
   int m = (scope_mode == ROCO_SCOPE_EXCLUDE_TOP_R) ? live - r : r;
