@@ -225,6 +225,20 @@ roco_status roco_gqa_decode_step(roco_cache *cache, const void *Q, const void *k
                                  int r, int scope_mode, float scale, void *attn_out, float *lse_out,
                                  int32_t *evicted_slot, int32_t *evicted_pos, void *stream);
 
+/*
+ * roco_decode_step (order ROCO_EVICT_FIRST) for calls with few units -- one layer of a small batch -- where one
+ * CTA per unit cannot fill the GPU: each unit's slots are divided among `splits` CTAs (Eq. 1 is merged from the
+ * partial (max, sum, sum of p*V) triples; the statistics of Sec. 4.3 are then accumulated in a second, cheap pass
+ * from the saved scores and the merged log-sum-exp).  Same arguments and results as roco_decode_step.
+ *   splits      1..64 CTAs per unit (a good value makes S*G*splits a few times the number of SMs)
+ *   workspace   >= roco_decode_split_workspace_bytes(cache, splits), 256-byte aligned, device; S*G <= 65535
+ */
+size_t roco_decode_split_workspace_bytes(const roco_cache *cache, int splits);
+roco_status roco_decode_step_split(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,
+                                   int scope_mode, int splits, float scale, void *attn_out, float *lse_out,
+                                   int32_t *evicted_slot, int32_t *evicted_pos, void *workspace,
+                                   size_t workspace_bytes, void *stream);
+
 /* Bytes of device staging roco_decode_step_host needs (host function). */
 size_t roco_decode_host_staging_bytes(const roco_cache *cache);
 

@@ -24,6 +24,7 @@ ROCO_EVICT_FIRST, ROCO_ATTEND_FIRST = 0, 1
 EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes", "roco_prefill",
            "roco_prefill_uses_tensor_cores", "roco_prefill_static", "roco_prefill_workspace_bytes_lowest_r",
            "roco_block_step", "roco_gqa_decode_step", "roco_decode_step_policy",
+           "roco_decode_split_workspace_bytes", "roco_decode_step_split",
            "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status")
 
 
@@ -76,6 +77,12 @@ def lib() -> C.CDLL:
             fn.restype = C.c_int
             fn.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                            C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.roco_decode_split_workspace_bytes.restype = C.c_size_t
+        L.roco_decode_split_workspace_bytes.argtypes = [C.POINTER(roco_cache), C.c_int]
+        L.roco_decode_step_split.restype = C.c_int
+        L.roco_decode_step_split.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                             C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.roco_decode_step_policy.restype = C.c_int
         L.roco_decode_step_policy.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                               C.c_int, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -184,6 +191,22 @@ def roco_decode_step(cache: Cache, q, k_new, v_new, r: int, attn_out, evicted_sl
                                 scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot), _ptr(evicted_pos), _stream())
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_decode_step")
+
+
+def roco_decode_split_workspace_bytes(cache: Cache, splits: int) -> int:
+    return int(lib().roco_decode_split_workspace_bytes(C.byref(cache.c), splits))
+
+
+def roco_decode_step_split(cache: Cache, q, k_new, v_new, r: int, splits: int, attn_out, evicted_slot, workspace,
+                           evicted_pos=None, lse_out=None, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R,
+                           scale: Optional[float] = None):
+    """roco_decode_step (evict, insert, attend) with every unit's slots divided among `splits` CTAs."""
+    scale = cache.d ** -0.5 if scale is None else scale
+    rc = lib().roco_decode_step_split(C.byref(cache.c), _ptr(q), _ptr(k_new), _ptr(v_new), r, scope_mode, splits,
+                                      scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot), _ptr(evicted_pos),
+                                      _ptr(workspace), workspace.numel(), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_decode_step_split")
 
 
 def roco_decode_step_policy(cache: Cache, q, k_new, v_new, policy: int, r: int, attn_out, evicted_slot,

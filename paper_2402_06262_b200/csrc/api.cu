@@ -139,6 +139,28 @@ roco_status roco_decode_step(roco_cache *cache, const void *q, const void *k_new
                             attn_out, lse_out, evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
 }
 
+size_t roco_decode_split_workspace_bytes(const roco_cache *cache, int splits) {
+  if (!cache || cache->S < 1 || cache->G < 1 || splits < 1 || splits > 64) return 0;
+  return decode_split_workspace_bytes(cache->S * cache->G, cache->B, cache->d, splits);
+}
+
+roco_status roco_decode_step_split(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,
+                                   int scope_mode, int splits, float scale, void *attn_out, float *lse_out,
+                                   int32_t *evicted_slot, int32_t *evicted_pos, void *workspace,
+                                   size_t workspace_bytes, void *stream) {
+  roco_status st = check_cache(cache);
+  if (st != ROCO_OK) return st;
+  if (!q || !k_new || !v_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
+  if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
+  if (splits < 1 || splits > 64) return ROCO_ERR_INVALID_ARG;
+  const size_t need = roco_decode_split_workspace_bytes(cache, splits);
+  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return ROCO_ERR_WORKSPACE;
+  return launch_decode_step_split(*cache, q, k_new, v_new, r, scope_mode, splits, scale, attn_out, lse_out,
+                                  evicted_slot, evicted_pos, workspace, static_cast<cudaStream_t>(stream));
+}
+
 roco_status roco_decode_step_policy(roco_cache *cache, const void *q, const void *k_new, const void *v_new,
                                     int policy, int r, const uint32_t *rnd, float scale, void *attn_out,
                                     float *lse_out, int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {

@@ -12,6 +12,13 @@ roco_status launch_decode_step(const roco_cache &c, const void *q, const void *k
                                int scope_mode, int step_order, int policy, const unsigned *rnd, float scale, void *out,
                                float *lse, int32_t *ev_slot, int32_t *ev_pos, cudaStream_t stream);
 
+// The same step (order evict, insert, attend) with each unit's slots divided among `splits` CTAs: three launches,
+// partial results and saved scores in `workspace` (decode_split_workspace_bytes).
+size_t decode_split_workspace_bytes(int U, int B, int d, int splits);
+roco_status launch_decode_step_split(const roco_cache &c, const void *q, const void *k_new, const void *v_new, int r,
+                                     int scope_mode, int splits, float scale, void *out, float *lse, int32_t *ev_slot,
+                                     int32_t *ev_pos, void *workspace, cudaStream_t stream);
+
 // Row log-sum-exp and column statistics of the causal softmax, CUDA-core path (any supported dtype/d).
 // lens_dev: [S] device copy of the prompt lengths.  lse, s_full, q_full: [U][Lmax].
 roco_status launch_prefill_stats_simt(int kv_dtype, int d, int S, int G, int Lmax, const int *lens_dev, int maxlen,

@@ -122,7 +122,10 @@ class DecodeParity:
     """Steps the GPU cache and the oracle state of the sampled units together."""
 
     def __init__(self, cache: R.Cache, st: oracle.State, units: Sequence[int], r: int, scope_mode: int, order: int,
-                 tally: Tally, scale: Optional[float] = None, strict: bool = False):
+                 tally: Tally, scale: Optional[float] = None, strict: bool = False, splits: int = 0):
+        self.splits = splits
+        self.ws = (torch.empty(R.roco_decode_split_workspace_bytes(cache, splits), dtype=torch.uint8,
+                               device=cache.K.device) if splits else None)
         self.cache, self.st, self.units = cache, st, list(units)
         self.r, self.mode, self.order, self.tally, self.strict = r, scope_mode, order, tally, strict
         self.scale = cache.d ** -0.5 if scale is None else scale
@@ -134,8 +137,12 @@ class DecodeParity:
 
     def step(self, q, k_new, v_new, check_state: bool = False):
         c = self.cache
-        R.roco_decode_step(c, q, k_new, v_new, self.r, self.out, self.ev_slot, self.ev_pos, self.lse,
-                           scope_mode=self.mode, step_order=self.order, scale=self.scale)
+        if self.splits:
+            R.roco_decode_step_split(c, q, k_new, v_new, self.r, self.splits, self.out, self.ev_slot, self.ws,
+                                     self.ev_pos, self.lse, scope_mode=self.mode, scale=self.scale)
+        else:
+            R.roco_decode_step(c, q, k_new, v_new, self.r, self.out, self.ev_slot, self.ev_pos, self.lse,
+                               scope_mode=self.mode, step_order=self.order, scale=self.scale)
         torch.cuda.synchronize()
         g_slot = unit_view(self.ev_slot, self.units).cpu().numpy()
         g_pos = unit_view(self.ev_pos, self.units).cpu().numpy()
