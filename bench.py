@@ -227,6 +227,39 @@ def multi_bench(R, cache, w, device, reps=6):
         base = base or ms
         res["block"].append({"b": b, "ms_per_step": ms, "tokens_per_s": w.S * b / ms * 1e3,
                              "speedup_vs_b1_per_token": base * b / ms, "hbm_frac": alg / ms / 1e6 / hbm_peak})
+    # calls with few units (one layer at a time, what a transformer's decode loop does): the same step with each
+    # unit's slots divided among several CTAs.  Two cases: one layer of the decode workload, and one layer of a
+    # single long-context sequence (32 units, B = 8192).  L2 is flushed between launches (the caches are small).
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    def timed_cold(fn):
+        ts = []
+        for _ in range(reps + 2):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts[2:])
+    sub = R.Cache(w.S, w.heads, w.B, w.d, dt, device)
+    for name in ("K", "V", "s", "q", "n", "pos", "live", "t_next"):
+        getattr(sub, name).copy_(getattr(cache, name)[:, :w.heads])
+    wl = W.scaled(W.LONG_CONTEXT, S=1, layers=1, prompt_lo=8192, prompt_hi=8192, B=8192)
+    _, long_cache, _ = build_cache(wl, device, R)
+    res["few_units"] = []
+    for label, cch, rr in ((f"{sub.U} units, B={sub.B}", sub, w.r), (f"{long_cache.U} units, B={long_cache.B}", long_cache, wl.r)):
+        algb = algorithmic_bytes_per_unit_step(cch.B, cch.d, elem) * cch.U
+        q1, k1, v1 = (torch.randn(cch.S, cch.G, cch.d, device=device, generator=gen).to(dt) for _ in range(3))
+        out1 = torch.zeros(cch.S, cch.G, cch.d, dtype=dt, device=device)
+        ev1 = torch.zeros(cch.S, cch.G, dtype=torch.int32, device=device)
+        rows = []
+        ms = timed_cold(lambda: R.roco_decode_step(cch, q1, k1, v1, rr, out1, ev1, scale=cch.d ** -0.5))
+        rows.append({"splits": 0, "us_per_step": ms * 1e3, "hbm_frac": algb / ms / 1e6 / hbm_peak})
+        for sp in (2, 4, 8):
+            ws = torch.empty(R.roco_decode_split_workspace_bytes(cch, sp), dtype=torch.uint8, device=device)
+            ms = timed_cold(lambda: R.roco_decode_step_split(cch, q1, k1, v1, rr, sp, out1, ev1, ws,
+                                                             scale=cch.d ** -0.5))
+            rows.append({"splits": sp, "us_per_step": ms * 1e3, "hbm_frac": algb / ms / 1e6 / hbm_peak})
+        res["few_units"].append({"case": label, "rows": rows})
+    del flush, long_cache
     for g in (4, 8):
         Q = torch.randn(w.S, w.G, g, w.d, device=device, generator=gen).to(dt)
         k, v = (torch.randn(w.S, w.G, w.d, device=device, generator=gen).to(dt) for _ in range(2))

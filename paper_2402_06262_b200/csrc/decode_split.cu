@@ -20,7 +20,8 @@ constexpr int kSpThreads = kSpConsumers + 32;
 constexpr int kSpTile = 16384;
 constexpr int kSpStages = 4;
 constexpr int kSpBar = 1;
-constexpr int kSpPolicyThreads = 128;
+constexpr int kSpPolicyThreads = 512;  // the selection is the serial part of a call with few units: go wide
+constexpr int kSpMergeThreads = 512;
 
 struct SplitParams {
   const char *K, *V;
@@ -38,7 +39,7 @@ struct SplitParams {
   int *slot_new; // [U]           slot that received the new token
 };
 
-// ---- 1. policy: one CTA of 128 threads per unit
+// ---- 1. policy: one CTA per unit
 template <typename T, int D>
 __global__ void __launch_bounds__(kSpPolicyThreads) split_policy_kernel(const SplitParams p) {
   constexpr int kRowBytes = D * (int)sizeof(T);
@@ -246,7 +247,7 @@ __global__ void __launch_bounds__(kSpThreads) split_attend_kernel(const SplitPar
 
 // ---- 3. merge of the partial results, output, and the statistics pass
 template <typename T, int D>
-__global__ void __launch_bounds__(256) split_merge_kernel(const SplitParams p) {
+__global__ void __launch_bounds__(kSpMergeThreads) split_merge_kernel(const SplitParams p) {
   __shared__ float w_sh[64];
   __shared__ float ml_sh[2];
   const int u = blockIdx.x, tid = threadIdx.x, B = p.B, splits = p.splits;
@@ -277,7 +278,7 @@ __global__ void __launch_bounds__(256) split_merge_kernel(const SplitParams p) {
   // statistics of Sec. 4.3 from the saved scores and the merged log-sum-exp
   const int e = p.slot_new[u];
 #pragma unroll 4
-  for (int j = tid; j < live; j += 256) {
+  for (int j = tid; j < live; j += kSpMergeThreads) {
     const float pj = exp2f(p.zbuf[unit_st + j] - M) * inv;
     const bool fresh = (j == e);
     const float s0 = fresh ? 0.f : p.s[unit_st + j], q0 = fresh ? 0.f : p.q[unit_st + j];
@@ -308,7 +309,7 @@ static cudaError_t launch_split_t(SplitParams &p, int U, cudaStream_t stream) {
   if (err != cudaSuccess) return err;
   split_policy_kernel<T, D><<<U, kSpPolicyThreads, smem1, stream>>>(p);
   split_attend_kernel<T, D><<<dim3(p.splits, U), kSpThreads, smem2, stream>>>(p);
-  split_merge_kernel<T, D><<<U, 256, 0, stream>>>(p);
+  split_merge_kernel<T, D><<<U, kSpMergeThreads, 0, stream>>>(p);
   return cudaGetLastError();
 }
 
