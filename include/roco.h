@@ -212,6 +212,24 @@ roco_status roco_block_step(roco_cache *cache, const void *Q, const void *K_new,
                             int32_t *evicted_pos, void *stream);
 
 /*
+ * Key-value constrained prompt encoding, block by block (Sec. 5.3 "Overhead": evict-and-encode "in a block-wise
+ * manner"; b = 1 is the token-wise scheme of the prior policies): the prompt of every sequence is fed through
+ * roco_block_step b tokens at a time (the last block may be shorter), so the cache never exceeds the budget while
+ * the prompt is encoded.  The cache is continued from its current state: start from live = 0, t_next = 0 for a
+ * fresh prompt.  Unlike roco_prefill no L x L work is done: each block attends over at most B cached tokens.
+ *
+ *   Q, K, V        [S][G][Lmax][d], cache->kv_dtype; rows >= lens_host[b] are ignored
+ *   lens_host      [S] HOST array, 1 <= lens <= Lmax
+ *   b              block size 1..16; r as for roco_block_step (EXCLUDE_TOP_R reading, r + b <= B)
+ *   attn_out       [S][G][Lmax][d] attention output of every prompt token over the budgeted cache
+ *   evicted_slot   [S][G][b] scratch; on return the slots the last block of each sequence freed (-1 padded)
+ * Launches sum_s ceil(lens[s] / b) kernels on the stream.
+ */
+roco_status roco_prefill_blockwise(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax,
+                                   int b, int r, float scale, roco_cache *cache, void *attn_out,
+                                   int32_t *evicted_slot, void *stream);
+
+/*
  * Decode step for grouped-query attention (Sec. 5.3 "Extension to Grouped-Query Attention", App. A): the cache
  * belongs to a key-value head that `group` query heads share.  Order as ROCO_EVICT_FIRST.  Each query head g
  * attends over the same cache, out_g = Softmax(scale * q_g K^T) V; the statistics receive the group-wise

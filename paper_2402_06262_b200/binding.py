@@ -24,7 +24,7 @@ ROCO_EVICT_FIRST, ROCO_ATTEND_FIRST = 0, 1
 EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes", "roco_prefill",
            "roco_prefill_uses_tensor_cores", "roco_prefill_static", "roco_prefill_workspace_bytes_lowest_r",
            "roco_block_step", "roco_gqa_decode_step", "roco_decode_step_policy",
-           "roco_decode_split_workspace_bytes", "roco_decode_step_split",
+           "roco_decode_split_workspace_bytes", "roco_decode_step_split", "roco_prefill_blockwise",
            "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status")
 
 
@@ -77,6 +77,9 @@ def lib() -> C.CDLL:
             fn.restype = C.c_int
             fn.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                            C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.roco_prefill_blockwise.restype = C.c_int
+        L.roco_prefill_blockwise.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                             C.c_float, C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p]
         L.roco_decode_split_workspace_bytes.restype = C.c_size_t
         L.roco_decode_split_workspace_bytes.argtypes = [C.POINTER(roco_cache), C.c_int]
         L.roco_decode_step_split.restype = C.c_int
@@ -191,6 +194,17 @@ def roco_decode_step(cache: Cache, q, k_new, v_new, r: int, attn_out, evicted_sl
                                 scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot), _ptr(evicted_pos), _stream())
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_decode_step")
+
+
+def roco_prefill_blockwise(Q, K, V, lens: Sequence[int], b: int, r: int, cache: Cache, attn_out, evicted_slot,
+                           scale: Optional[float] = None):
+    """Encode the prompts block by block (b tokens per evict-and-encode step) through the budgeted cache."""
+    scale = cache.d ** -0.5 if scale is None else scale
+    lens_arr = (C.c_int32 * len(lens))(*[int(x) for x in lens])
+    rc = lib().roco_prefill_blockwise(_ptr(Q), _ptr(K), _ptr(V), C.cast(lens_arr, C.c_void_p), int(Q.shape[2]), b, r,
+                                      scale, C.byref(cache.c), _ptr(attn_out), _ptr(evicted_slot), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_prefill_blockwise")
 
 
 def roco_decode_split_workspace_bytes(cache: Cache, splits: int) -> int:

@@ -193,6 +193,42 @@ roco_status roco_block_step(roco_cache *cache, const void *Q, const void *K_new,
                            evicted_pos, static_cast<cudaStream_t>(stream));
 }
 
+roco_status roco_prefill_blockwise(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax,
+                                   int b, int r, float scale, roco_cache *cache, void *attn_out,
+                                   int32_t *evicted_slot, void *stream) {
+  roco_status st = check_cache(cache);
+  if (st != ROCO_OK) return st;
+  if (!Q || !K || !V || !lens_host || !attn_out || !evicted_slot || Lmax < 1 || b < 1) return ROCO_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
+  if ((st = check_scope(r, ROCO_SCOPE_EXCLUDE_TOP_R, cache->B, true)) != ROCO_OK) return st;
+  if (b > multi_max_queries()) return ROCO_ERR_UNSUPPORTED;
+  if (b > 1 && r + b > cache->B) return ROCO_ERR_INVALID_ARG;
+  if (!multi_fits(cache->B, cache->d, b, b)) return ROCO_ERR_UNSUPPORTED;
+  for (int s = 0; s < cache->S; ++s)
+    if (lens_host[s] < 1 || lens_host[s] > Lmax) return ROCO_ERR_INVALID_ARG;
+  const size_t elem = cache->kv_dtype == ROCO_BF16 ? 2 : 4;
+  const size_t G = (size_t)cache->G, B = (size_t)cache->B, d = (size_t)cache->d;
+  for (int s = 0; s < cache->S; ++s) {
+    roco_cache sub = *cache;  // the units of sequence s
+    sub.S = 1;
+    sub.K = static_cast<char *>(cache->K) + s * G * B * d * elem;
+    sub.V = static_cast<char *>(cache->V) + s * G * B * d * elem;
+    sub.s = cache->s + s * G * B; sub.q = cache->q + s * G * B;
+    sub.n = cache->n + s * G * B; sub.pos = cache->pos + s * G * B;
+    sub.live = cache->live + s * G; sub.t_next = cache->t_next + s * G;
+    for (int t0 = 0; t0 < lens_host[s]; t0 += b) {
+      const int m = lens_host[s] - t0 < b ? lens_host[s] - t0 : b;
+      const size_t off = ((size_t)s * G * Lmax + t0) * d * elem;
+      st = launch_multi_step(sub, 0, m, m, static_cast<const char *>(Q) + off, static_cast<const char *>(K) + off,
+                             static_cast<const char *>(V) + off, r, ROCO_SCOPE_EXCLUDE_TOP_R, scale,
+                             static_cast<char *>(attn_out) + off, nullptr, evicted_slot + (size_t)s * G * b, nullptr,
+                             static_cast<cudaStream_t>(stream), Lmax);
+      if (st != ROCO_OK) return st;
+    }
+  }
+  return ROCO_OK;
+}
+
 roco_status roco_gqa_decode_step(roco_cache *cache, const void *Q, const void *k_new, const void *v_new, int group,
                                  int r, int scope_mode, float scale, void *attn_out, float *lse_out,
                                  int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {

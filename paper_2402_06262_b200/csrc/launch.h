@@ -49,6 +49,8 @@ int multi_max_queries();
 bool multi_fits(int B, int d, int M, int nb);
 roco_status launch_multi_step(const roco_cache &c, int kind, int M, int nb, const void *Q, const void *k_new,
                               const void *v_new, int r, int scope_mode, float scale, void *out, float *lse,
-                              int32_t *ev_slot, int32_t *ev_pos, cudaStream_t stream);
+                              int32_t *ev_slot, int32_t *ev_pos, cudaStream_t stream, long long unit_stride_rows = 0);
+// unit_stride_rows > 0: Q, k_new, v_new and out are slices of [U][rows][d] tensors with that many rows per unit
+// (used to step through a prompt block by block); 0: dense [U][M][d] / [U][nb][d].
 
 }  // namespace roco

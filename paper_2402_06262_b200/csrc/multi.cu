@@ -41,6 +41,7 @@ struct MultiParams {
   int *ev_slot, *ev_pos;
   int B, r, scope_mode, stages, M, nb, kind;
   float scale;
+  long long q_ustride, kv_ustride, out_ustride;  // rows (tokens) between consecutive units in Q, K_new/V_new, out
 };
 
 struct MultiSmem {
@@ -129,9 +130,9 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
   for (int j = ptid; j < live1; j += kMqPolicyThreads) v.newtok[j] = -1;
   {  // new keys / values (and the queries) as fp32 in shared memory, 16-byte loads issued back to back
     constexpr int kEPC = Elem<T>::kPerChunk;
-    const uint4 *gk = reinterpret_cast<const uint4 *>(p.k_new + (size_t)u * nb * kRowBytes);
-    const uint4 *gv = reinterpret_cast<const uint4 *>(p.v_new + (size_t)u * nb * kRowBytes);
-    const uint4 *gqr = reinterpret_cast<const uint4 *>(p.Q + (size_t)u * M * kRowBytes);
+    const uint4 *gk = reinterpret_cast<const uint4 *>(p.k_new + (size_t)u * p.kv_ustride * kRowBytes);
+    const uint4 *gv = reinterpret_cast<const uint4 *>(p.v_new + (size_t)u * p.kv_ustride * kRowBytes);
+    const uint4 *gqr = reinterpret_cast<const uint4 *>(p.Q + (size_t)u * p.q_ustride * kRowBytes);
     const int nkv = nb * D / kEPC, nq = v.qf ? M * D / kEPC : 0;
 #pragma unroll 4
     for (int i = ptid; i < 2 * nkv + nq; i += kMqPolicyThreads) {
@@ -256,7 +257,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     const int cc = isv ? c - kLanesPerRow : c;
     int slot = tgt[i];
     if (slot < 0 || slot >= B) slot = 0;
-    const uint4 val = *((const uint4 *)((isv ? p.v_new : p.k_new) + ((size_t)u * nb + i) * kRowBytes) + cc);
+    const uint4 val = *((const uint4 *)((isv ? p.v_new : p.k_new) + ((size_t)u * p.kv_ustride + i) * kRowBytes) + cc);
     *((uint4 *)(const_cast<char *>(isv ? p.V : p.K) + unit_kv + (size_t)slot * kRowBytes) + cc) = val;
   }
   // scores of every query against every new token, from k_new directly (log2 domain)
@@ -278,7 +279,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
   } else {
     for (int w = pwarp; w < M * nb; w += kMqPolicyThreads / 32) {  // one dot product per warp and turn
       const int i = w / nb, jn = w % nb;
-      const T *qrow = (const T *)p.Q + ((size_t)u * M + i) * D;
+      const T *qrow = (const T *)p.Q + ((size_t)u * p.q_ustride + i) * D;
       float acc = 0.f;
       for (int c = plane; c < D; c += 32) acc = fmaf(Elem<T>::load(qrow + c), v.knew[jn * D + c], acc);
       acc = warp_sum(acc);
@@ -389,7 +390,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
   const int rows_per_warp = kTileRows / RG;
   const int loads = rows_per_warp / kRowsPerLoad;
   for (int i = tid; i < M * D; i += kMqConsumers)
-    sm.qf[i] = Elem<T>::load((const T *)p.Q + (size_t)u * M * D + i);
+    sm.qf[i] = Elem<T>::load((const T *)p.Q + (size_t)u * p.q_ustride * D + i);
   named_bar_sync(kMqBarConsumers, kMqConsumers);
 
   const float zscale = p.scale * kLog2e;
@@ -521,7 +522,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
       if (slot < 0 || slot >= B) slot = 0;
       o = fmaf(sm.z[(size_t)qi * Bp + slot], sm.vnew[jn * D + c], o);
     }
-    Elem<T>::store((T *)p.out + (size_t)u * M * D + w, o);
+    Elem<T>::store((T *)p.out + (size_t)u * p.out_ustride * D + w, o);
   }
 }
 
@@ -677,7 +678,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
   // A fragments of Q (16 x 128, rows >= M are zero): a[s] covers k = 16 s .. 16 s + 15
   uint32_t qa[8][4];
   {
-    const T *Qu = (const T *)p.Q + (size_t)u * M * D;
+    const T *Qu = (const T *)p.Q + (size_t)u * p.q_ustride * D;
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
       const int k0 = s * 16 + tq * 2;
@@ -806,7 +807,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
           o0 = fmaf(pj, sm.vnew[jn * D + dcol], o0);
           o1 = fmaf(pj, sm.vnew[jn * D + dcol + 1], o1);
         }
-        *reinterpret_cast<uint32_t *>((T *)p.out + ((size_t)u * M + qi) * D + dcol) = pack_bf16x2(o0, o1);
+        *reinterpret_cast<uint32_t *>((T *)p.out + ((size_t)u * p.out_ustride + qi) * D + dcol) = pack_bf16x2(o0, o1);
       }
     }
   }
@@ -845,13 +846,16 @@ bool multi_fits(int B, int d, int M, int nb) {
 
 roco_status launch_multi_step(const roco_cache &c, int kind, int M, int nb, const void *Q, const void *k_new,
                               const void *v_new, int r, int scope_mode, float scale, void *out, float *lse,
-                              int32_t *ev_slot, int32_t *ev_pos, cudaStream_t stream) {
+                              int32_t *ev_slot, int32_t *ev_pos, cudaStream_t stream, long long unit_stride_rows) {
   MultiParams p;
   p.K = (const char *)c.K; p.V = (const char *)c.V;
   p.s = c.s; p.q = c.q; p.n = c.n; p.pos = c.pos; p.live = c.live; p.t_next = c.t_next; p.status = c.status;
   p.Q = (const char *)Q; p.k_new = (const char *)k_new; p.v_new = (const char *)v_new;
   p.out = (char *)out; p.lse = lse; p.ev_slot = ev_slot; p.ev_pos = ev_pos;
   p.B = c.B; p.r = r; p.scope_mode = scope_mode; p.M = M; p.nb = nb; p.kind = kind; p.scale = scale;
+  p.q_ustride = unit_stride_rows > 0 ? unit_stride_rows : M;
+  p.kv_ustride = unit_stride_rows > 0 ? unit_stride_rows : nb;
+  p.out_ustride = unit_stride_rows > 0 ? unit_stride_rows : M;
   const int U = c.S * c.G;
   cudaError_t err;
   if (c.kv_dtype == ROCO_BF16 && c.d == 128 && (long long)U * c.B < 0x7fffffffLL) {

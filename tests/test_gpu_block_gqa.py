@@ -110,3 +110,38 @@ def test_gqa_decode_steps(group, mode):
         _, k, v = W.decode_tokens(w, i, [260 + i] * w.S, DEV)
         par.step(torch.stack(qs, dim=2).contiguous(), k, v, check_state=(i % 3 == 2))
     assert R.roco_device_status(cache) == 0 and tally.decisions == 10 * w.U
+
+
+@pytest.mark.parametrize("b", [1, 4, 16])
+def test_blockwise_prompt_encoding(b):
+    """The paper's prefill scheme: the whole prompt goes through the budgeted cache b tokens at a time (ragged
+    prompt lengths, last block shorter).  The oracle replays the same sequence of block steps."""
+    w = W.scaled(W.LLAMA7B_DECODE, S=2, layers=1, heads=3, prompt_lo=150, prompt_hi=150, B=64, r=6)
+    lens = [150, 97]
+    Q, K, V = prompt_tensors(w, 150)
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    out = torch.zeros_like(Q)
+    ev = torch.zeros(w.S, w.G, b, dtype=torch.int32, device=DEV)
+    R.roco_prefill_blockwise(Q, K, V, lens, b, w.r, cache, out, ev, scale=w.scale)
+    torch.cuda.synchronize()
+    assert R.roco_device_status(cache) == 0
+    from harness import compare_state, out_tol
+    checked = 0
+    for s, L in enumerate(lens):
+        units = [s * w.G + g for g in range(w.G)]
+        st = oracle.empty_state(w.G, w.B, w.d)
+        Qs, Ks, Vs = (widen(x[s]) for x in (Q, K, V))
+        outs = np.zeros((w.G, L, w.d))
+        near = 0
+        for t0 in range(0, L, b):
+            m = min(b, L - t0)
+            res = oracle.block_step(st, Qs[:, t0:t0 + m], Ks[:, t0:t0 + m], Vs[:, t0:t0 + m], w.r,
+                                    R.ROCO_SCOPE_EXCLUDE_TOP_R, w.scale, delta=1e-5)
+            outs[:, t0:t0 + m] = res.out
+            near += int(res.near_tie.sum())
+        if near == 0:   # no decision inside the margin along the whole prompt: the final states must agree
+            compare_state(cache, st, units, f"sequence {s}")
+            assert np.abs(widen(out[s, :, :L]) - outs).max() <= out_tol(w.torch_dtype)
+            checked += 1
+        assert int(cache.live[s].min()) == min(L, w.B) and int(cache.t_next[s].max()) == L
+    assert checked >= 1, "every sequence hit a decision inside the margin: pick another seed"
