@@ -270,6 +270,29 @@ def multi_bench(R, cache, w, device, reps=6):
             rows.append({"splits": sp, "us_per_step": ms * 1e3, "hbm_frac": algb / ms / 1e6 / hbm_peak})
         res["few_units"].append({"case": label, "rows": rows})
     del flush, long_cache
+    # the paper's prefill scheme: the whole prompt through the budgeted cache, b tokens per evict-and-encode step
+    # (its Table "block-wise eviction" reports the speed-up over b = 1)
+    Lp = w.prompt_lo
+    Qp, Kp, Vp = (torch.randn(w.S, w.G, Lp, w.d, device=device, generator=gen, dtype=torch.float32).to(dt)
+                  for _ in range(3))
+    outp = torch.empty_like(Qp)
+    pc = R.Cache(w.S, w.G, w.B, w.d, dt, device)
+    res["blockwise_prefill"] = []
+    t_b1 = None
+    for b in (1, 4, 16):
+        evp = torch.zeros(w.S, w.G, b, dtype=torch.int32, device=device)
+        pc.live.zero_(); pc.t_next.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        R.roco_prefill_blockwise(Qp, Kp, Vp, [Lp] * w.S, b, w.r, pc, outp, evp, scale=w.scale)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        t_b1 = t_b1 or ms
+        res["blockwise_prefill"].append({"b": b, "prompt": Lp, "ms": ms, "prompt_tokens_per_s": w.S * Lp / ms * 1e3,
+                                         "speedup_vs_b1": t_b1 / ms})
+    del Qp, Kp, Vp, outp, pc
     for g in (4, 8):
         Q = torch.randn(w.S, w.G, g, w.d, device=device, generator=gen).to(dt)
         k, v = (torch.randn(w.S, w.G, w.d, device=device, generator=gen).to(dt) for _ in range(2))
