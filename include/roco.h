@@ -230,6 +230,25 @@ roco_status roco_prefill_blockwise(const void *Q, const void *K, const void *V, 
                                    int32_t *evicted_slot, void *stream);
 
 /*
+ * Attention output of the one-pass prompt encoding (Eq. 1 with the causal mask of Sec. 2.1), for callers that
+ * also need the layer's output and not only the budgeted cache:
+ *     out_i = sum_{j<=i} exp(scale * Q_i.K_j - lse_i) V_j,      i < lens
+ * where lse is the row log-sum-exp roco_prefill returned in lse_out for the same Q, K, lens, Lmax and scale
+ * (call roco_prefill first, on the same stream).  Tensor cores only: kv_dtype ROCO_BF16 and d = 128, else
+ * ROCO_ERR_UNSUPPORTED.  Only S, G, d, kv_dtype and status of `cache` are read.
+ *
+ *   Q, K, V      [S][G][Lmax][d] device; rows >= lens may hold anything
+ *   lens_host    [S] HOST array, 1 <= lens <= Lmax
+ *   lse          [S][G][Lmax] fp32 device
+ *   attn_out     [S][G][Lmax][d] device, cache->kv_dtype; rows >= lens are left untouched
+ *   workspace    >= roco_prefill_attend_workspace_bytes(cache) device bytes, 256-byte aligned
+ */
+size_t roco_prefill_attend_workspace_bytes(const roco_cache *cache);
+roco_status roco_prefill_attend(const roco_cache *cache, const void *Q, const void *K, const void *V,
+                                const int32_t *lens_host, int Lmax, float scale, const float *lse, void *attn_out,
+                                void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Decode step for grouped-query attention (Sec. 5.3 "Extension to Grouped-Query Attention", App. A): the cache
  * belongs to a key-value head that `group` query heads share.  Order as ROCO_EVICT_FIRST.  Each query head g
  * attends over the same cache, out_g = Softmax(scale * q_g K^T) V; the statistics receive the group-wise

@@ -73,6 +73,19 @@ def attention_row(qv, K, scale):
     return p, float(lse)
 
 
+def prompt_attention_rows(Q, K, V, rows, scale):
+    """Causal attention output of a prompt (Eq. 1 with the mask of Sec. 2.1) for the query rows listed:
+    out_i = sum_{j<=i} p_ij V_j.  Q, K, V: [L][d].  Returns (out [len(rows)][d], lse [len(rows)])."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    out = np.zeros((len(rows), V.shape[1]))
+    lse = np.zeros(len(rows))
+    for t, i in enumerate(rows):
+        p, lse[t] = attention_row(Q[i], K[: i + 1], scale)
+        for j in range(i + 1):
+            out[t] += p[j] * V[j]
+    return out, lse
+
+
 def select(s, q, n, pos, r, mode, delta=1e-5):
     """Victim slot among slots 0..len-1.  Returns (slot, near_tie, scope_size)."""
     s, q, n, pos = _f64(s), _f64(q), _i32(n), _i32(pos)

@@ -25,7 +25,8 @@ EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes",
            "roco_prefill_uses_tensor_cores", "roco_prefill_static", "roco_prefill_workspace_bytes_lowest_r",
            "roco_block_step", "roco_gqa_decode_step", "roco_decode_step_policy",
            "roco_decode_split_workspace_bytes", "roco_decode_step_split", "roco_prefill_blockwise",
-           "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status")
+           "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status",
+           "roco_prefill_attend_workspace_bytes", "roco_prefill_attend")
 
 
 class RocoError(RuntimeError):
@@ -70,6 +71,12 @@ def lib() -> C.CDLL:
         L.roco_prefill_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                           C.c_int, C.c_int, C.c_float, C.POINTER(roco_cache), C.c_void_p, C.c_void_p,
                                           C.c_void_p, C.c_void_p]
+        L.roco_prefill_attend_workspace_bytes.restype = C.c_size_t
+        L.roco_prefill_attend_workspace_bytes.argtypes = [C.POINTER(roco_cache)]
+        L.roco_prefill_attend.restype = C.c_int
+        L.roco_prefill_attend.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                          C.c_void_p]
         L.roco_decode_step.restype = C.c_int
         L.roco_decode_step.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                                        C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -185,6 +192,26 @@ def roco_prefill_static(Q, K, V, lens: Sequence[int], B: int, r: int, cache: Cac
                                    _stream())
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_prefill_static")
+
+
+def roco_prefill_attend_workspace_bytes(cache: Cache) -> int:
+    return int(lib().roco_prefill_attend_workspace_bytes(C.byref(cache.c)))
+
+
+def roco_prefill_attend(cache: Cache, Q, K, V, lens: Sequence[int], lse, attn_out, scale: Optional[float] = None,
+                        workspace: Optional[torch.Tensor] = None):
+    """Causal attention output of the prompt pass from the row log-sum-exp `lse` that roco_prefill returned.
+    Q, K, V, attn_out: [S][G][Lmax][d] bf16 device tensors (d = 128); lse: [S][G][Lmax] fp32."""
+    Lmax = Q.shape[2]
+    scale = cache.d ** -0.5 if scale is None else scale
+    if workspace is None:
+        workspace = torch.empty(roco_prefill_attend_workspace_bytes(cache), dtype=torch.uint8, device=Q.device)
+    lens_arr = (C.c_int32 * len(lens))(*[int(x) for x in lens])
+    rc = lib().roco_prefill_attend(C.byref(cache.c), _ptr(Q), _ptr(K), _ptr(V), C.cast(lens_arr, C.c_void_p), Lmax,
+                                   scale, _ptr(lse), _ptr(attn_out), _ptr(workspace), workspace.numel(), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_prefill_attend")
+    return workspace
 
 
 def roco_decode_step(cache: Cache, q, k_new, v_new, r: int, attn_out, evicted_slot, evicted_pos=None, lse_out=None,

@@ -126,6 +126,35 @@ roco_status roco_prefill(const void *Q, const void *K, const void *V, const int3
                                      reinterpret_cast<unsigned long long *>(ws + w.total), pow2_at_least(Lmax), cs);
 }
 
+size_t roco_prefill_attend_workspace_bytes(const roco_cache *cache) {
+  if (!cache || cache->S < 1) return 0;
+  return align_up((size_t)cache->S * 4, 256);
+}
+
+roco_status roco_prefill_attend(const roco_cache *cache, const void *Q, const void *K, const void *V,
+                                const int32_t *lens_host, int Lmax, float scale, const float *lse, void *attn_out,
+                                void *workspace, size_t workspace_bytes, void *stream) {
+  if (!cache || !cache->status || cache->S < 1 || cache->G < 1) return ROCO_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !lens_host || !lse || !attn_out || Lmax < 1) return ROCO_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
+  if (!prefill_tc_supported(cache->kv_dtype, cache->d)) return ROCO_ERR_UNSUPPORTED;
+  int maxlen = 0;
+  for (int b = 0; b < cache->S; ++b) {
+    if (lens_host[b] < 1 || lens_host[b] > Lmax) return ROCO_ERR_INVALID_ARG;
+    if (lens_host[b] > maxlen) maxlen = lens_host[b];
+  }
+  if ((long long)cache->S * cache->G * ((maxlen + 255) / 256 + 1) > 0x7fffffffLL) return ROCO_ERR_UNSUPPORTED;
+  if (!workspace || workspace_bytes < roco_prefill_attend_workspace_bytes(cache) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return ROCO_ERR_WORKSPACE;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  int *lens_dev = static_cast<int *>(workspace);
+  if (cudaMemcpyAsync(lens_dev, lens_host, (size_t)cache->S * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess)
+    return ROCO_ERR_CUDA;
+  return launch_prefill_attend_tc(cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, V, scale, lse, attn_out,
+                                  cache->status, cs);
+}
+
 roco_status roco_decode_step(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,
                              int scope_mode, int step_order, float scale, void *attn_out, float *lse_out,
                              int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {

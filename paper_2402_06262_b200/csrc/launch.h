@@ -31,6 +31,16 @@ roco_status launch_prefill_stats_tc(int S, int G, int Lmax, const int *lens_dev,
                                     const void *K, float scale, float *lse, float *s_full, float *q_full, int *status,
                                     cudaStream_t stream);
 
+// Tensor map (CUtensorMap, 128 bytes, passed as void*) over a [U][Lmax][128] bf16 prompt tensor with boxes of
+// 64 columns x 128 rows x 1 unit and the 128-byte swizzle; rows past Lmax read as zero.
+bool make_tensor_map_prompt_bf16(void *map, const void *base, int U, int Lmax);
+
+// Causal attention output of the prompt pass on the tensor cores (bf16, d = 128): out_i = sum_{j<=i}
+// exp(scale Q_i.K_j - lse_i) V_j with the row log-sum-exp `lse` the statistics pass produced.  out: [U][Lmax][128].
+roco_status launch_prefill_attend_tc(int S, int G, int Lmax, const int *lens_dev, int maxlen, const void *Q,
+                                     const void *K, const void *V, float scale, const float *lse, void *out,
+                                     int *status, cudaStream_t stream);
+
 // Select-to-budget on frozen statistics and gather of the survivors into the cache.
 // dst: [U][Lmax] int32 scratch (destination slot per token, -1 = evicted).  LOWEST_R with eviction also needs
 // sortbuf: [U][Lp2max] 64-bit scratch, Lp2max = Lmax rounded up to a power of two, and r <= budget_lowest_max_r().

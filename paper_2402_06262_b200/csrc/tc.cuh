@@ -1,0 +1,172 @@
+// tcgen05 / TMA-tensor PTX wrappers, packed fp32x2 arithmetic, the exponential helpers and the operand
+// descriptors shared by the tensor-core prefill kernels (bf16, 128 x 128 tiles, 128-byte swizzle).
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace roco {
+
+constexpr int kTcTile = 128;                       // rows of a stationary / streamed tile
+constexpr int kTcD = 128;                          // head dimension
+constexpr int kTcTileBytes = kTcTile * kTcD * 2;   // 32 KiB: two 64-column halves of 16 KiB
+constexpr int kTcHalfBytes = kTcTileBytes / 2;
+
+// ------------------------------------------------------------------ PTX wrappers (tcgen05, TMA tensor)
+
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int c0, int c1, int c2, uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, M = 128, N = 128, K = 16.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// mbarrier arrives once all MMAs issued so far by this thread have completed
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base + t).  The load is
+// asynchronous: the registers are valid only after tmem_ld_wait on the same array.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+
+// Waits for this thread's outstanding tensor-memory loads.  The array is an in/out operand so that no use
+// of its registers can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]),
+                 "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]),
+                 "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---- packed fp32x2 arithmetic (two lanes per instruction) and exp2 on the FMA pipe
+typedef unsigned long long f32x2;
+
+__device__ __forceinline__ f32x2 pack2(float a, float b) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 pack2u(uint32_t a, uint32_t b) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float &a, float &b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// 2^x for a pair of x <= 0 without the exponential unit: x = n + f with n the nearest integer (magic-number
+// rounding) and f in [-1/2, 1/2]; 2^f by a degree-4 polynomial (max relative error 2.7e-6, mean error 4e-8);
+// the integer n is then added to the exponent field.  x is clamped at -125 (results below 2^-125 are noise
+// for the sums they enter).
+__device__ __forceinline__ f32x2 exp2_poly2(f32x2 x2) {
+  float xa, xb;
+  unpack2(x2, xa, xb);
+  x2 = pack2(fmaxf(xa, -125.f), fmaxf(xb, -125.f));
+  const f32x2 magic = pack2(12582912.f, 12582912.f);  // 1.5 * 2^23: the low mantissa bits hold n
+  const f32x2 t2 = add2(x2, magic);
+  const f32x2 n2 = add2(t2, pack2(-12582912.f, -12582912.f));
+  const f32x2 f2 = fma2(n2, pack2(-1.f, -1.f), x2);
+  f32x2 p2 = fma2(f2, pack2(0.009570101276040077f, 0.009570101276040077f),
+                  pack2(0.05591785907745361f, 0.05591785907745361f));
+  p2 = fma2(p2, f2, pack2(0.240247443318367f, 0.240247443318367f));
+  p2 = fma2(p2, f2, pack2(0.6931217908859253f, 0.6931217908859253f));
+  p2 = fma2(p2, f2, pack2(0.9999992847442627f, 0.9999992847442627f));
+  float ta, tb, pa, pb;
+  unpack2(t2, ta, tb);
+  unpack2(p2, pa, pb);
+  const uint32_t ra = __float_as_uint(pa) + (__float_as_uint(ta) << 23);
+  const uint32_t rb = __float_as_uint(pb) + (__float_as_uint(tb) << 23);
+  return pack2u(ra, rb);
+}
+
+__device__ __forceinline__ f32x2 exp2_mufu2(f32x2 x2) {
+  float xa, xb;
+  unpack2(x2, xa, xb);
+  return pack2(ex2_approx(xa), ex2_approx(xb));
+}
+
+// Of every 8 pairs, how many take the polynomial instead of the exponential unit (which is the bottleneck
+// of both passes: 16 results per cycle per SM against 128 FMA lanes).
+#ifndef ROCO_POLY_PAIRS_PER_8
+#define ROCO_POLY_PAIRS_PER_8 2
+#endif
+constexpr int kPolyPairsPer8 = ROCO_POLY_PAIRS_PER_8;
+
+__device__ __forceinline__ f32x2 exp2_pair(f32x2 x2, int pair_index) {
+  return ((pair_index & 7) < kPolyPairsPer8) ? exp2_poly2(x2) : exp2_mufu2(x2);
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 operand tile stored as rows of 128 bytes with the
+// 128-byte swizzle (what TMA writes for a 64-column box): 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(const void *p) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_u32(p) >> 4) & 0x3fffu);  // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                         // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                         // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                         // 128-byte swizzle
+  return d;
+}
+
+// kind::f16 instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = 128
+constexpr uint32_t kIdescBf16M128N128 = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+
+}  // namespace roco

@@ -1,0 +1,82 @@
+"""GPU parity of the prompt pass's attention output (roco_prefill_attend, tensor cores) against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2402_06262_b200 as R
+import workloads as W
+from harness import unit_view, widen
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+OUT_TOL = 2e-2   # bf16 output: absolute + relative
+
+
+def prompt_tensors(w, L):
+    qs, ks, vs = zip(*[W.prompt_chunk(w, b, 0, w.G, L, DEV) for b in range(w.S)])
+    return torch.stack(qs), torch.stack(ks), torch.stack(vs)
+
+
+def run_attend(w, lens, Lmax, poison_padding=False):
+    Q, K, V = prompt_tensors(w, Lmax)
+    if poison_padding:   # rows past a prompt's length may hold anything
+        for b, L in enumerate(lens):
+            for X in (Q, K, V):
+                X[b, :, L:] = float("nan")
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    lse = torch.zeros(w.S, w.G, Lmax, dtype=torch.float32, device=DEV)
+    R.roco_prefill(Q, K, V, lens, w.B, w.r, cache, scale=w.scale, lse_out=lse)
+    out = torch.full((w.S, w.G, Lmax, w.d), 7.0, dtype=w.torch_dtype, device=DEV)
+    R.roco_prefill_attend(cache, Q, K, V, lens, lse, out, scale=w.scale)
+    torch.cuda.synchronize()
+    assert R.roco_device_status(cache) == 0
+    return Q, K, V, lse, out
+
+
+def check_rows(w, Q, K, V, lse, out, lens, units, rows_of):
+    for u in units:
+        L = lens[u // w.G]
+        q, k, v = (widen(unit_view(X, [u]))[0, :L] for X in (Q, K, V))
+        rows = rows_of(L)
+        want, want_lse = oracle.prompt_attention_rows(q, k, v, rows, w.scale)
+        got = widen(unit_view(out, [u]))[0]
+        np.testing.assert_allclose(widen(unit_view(lse, [u]))[0, rows], want_lse, rtol=0, atol=1e-4)
+        np.testing.assert_allclose(got[rows], want, rtol=OUT_TOL, atol=OUT_TOL, err_msg=f"unit {u}")
+        assert np.all(got[L:] == 7.0), "rows past the prompt must be left untouched"
+
+
+@pytest.mark.parametrize("kind", ["iid", "sink", "lowrank"])
+def test_attend_every_row_ragged(kind):
+    """Every row of every unit; lengths of one tile, a ragged multi-tile prompt and a short one (odd and even
+    tile counts, so both the paired and the unpaired query tile are exercised)."""
+    w = W.scaled(W.LLAMA7B_PREFILL, S=4, layers=1, heads=3, prompt_lo=520, prompt_hi=520, B=64, r=8, kind=kind)
+    lens = [520, 333, 128, 7]
+    Q, K, V, lse, out = run_attend(w, lens, 520)
+    check_rows(w, Q, K, V, lse, out, lens, range(w.U), lambda L: list(range(L)))
+
+
+def test_attend_ignores_rows_past_the_prompt():
+    """NaN in every padding row of Q, K and V changes nothing."""
+    w = W.scaled(W.LLAMA7B_PREFILL, S=3, layers=1, heads=2, prompt_lo=400, prompt_hi=400, B=64, r=8, kind="sink")
+    lens = [400, 257, 100]
+    Q, K, V, lse, out = run_attend(w, lens, 400, poison_padding=True)
+    check_rows(w, Q, K, V, lse, out, lens, range(w.U), lambda L: list(range(0, L, 3)) + [L - 1])
+
+
+def test_attend_long_prompt_sampled_rows():
+    """L = 4096 (32 key tiles): sampled rows of sampled units, including both ends of every tile pairing."""
+    w = W.scaled(W.LLAMA7B_PREFILL, S=1, layers=1, heads=8, prompt_lo=4096, prompt_hi=4096, B=1024, r=64)
+    lens = [4096]
+    Q, K, V, lse, out = run_attend(w, lens, 4096)
+    rows = [0, 1, 127, 128, 129, 2047, 2048, 3000, 3967, 3968, 4095]
+    check_rows(w, Q, K, V, lse, out, lens, [0, 3, 7], lambda L: rows)
+
+
+def test_attend_rejects_unsupported_shapes():
+    w = W.TOY   # fp32, d = 64
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    Q = torch.zeros(w.S, w.G, 128, w.d, device=DEV)
+    lse = torch.zeros(w.S, w.G, 128, device=DEV)
+    with pytest.raises(R.RocoError):
+        R.roco_prefill_attend(cache, Q, Q, Q, [128], lse, torch.zeros_like(Q))

@@ -491,3 +491,53 @@ def test_attention_row_is_library_softmax():
     p, lse = oracle.attention_row(qv, K, 0.4)
     np.testing.assert_allclose(p, softmax(0.4 * K @ qv), rtol=1e-13)
     assert lse == pytest.approx(logsumexp(0.4 * K @ qv), rel=1e-13)
+
+
+# ---------------------------------------------------------------- prompt attention output (Eq. 1, causal)
+
+def test_prompt_attention_constant_values_pass_through():
+    """Probabilities of a row sum to one, so identical value rows come back unchanged."""
+    rng = np.random.default_rng(31)
+    L, d = 23, 8
+    Q, K = rng.normal(size=(L, d)), rng.normal(size=(L, d))
+    v = rng.normal(size=d)
+    out, _ = oracle.prompt_attention_rows(Q, K, np.tile(v, (L, 1)), list(range(L)), 0.3)
+    np.testing.assert_allclose(out, np.tile(v, (L, 1)), rtol=1e-12, atol=1e-14)
+
+
+def test_prompt_attention_zero_queries_give_running_mean():
+    """Q = 0 makes every causal row uniform: out_i is the mean of V_0..V_i (a closed form that also pins the mask)."""
+    rng = np.random.default_rng(32)
+    L, d = 19, 4
+    K, V = rng.normal(size=(L, d)), rng.normal(size=(L, d))
+    out, lse = oracle.prompt_attention_rows(np.zeros((L, d)), K, V, list(range(L)), 1.0)
+    want = np.cumsum(V, axis=0) / np.arange(1, L + 1)[:, None]
+    np.testing.assert_allclose(out, want, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(lse, np.log(np.arange(1, L + 1)), rtol=1e-12, atol=1e-14)
+
+
+def test_prompt_attention_dominant_key_selects_its_value_and_future_is_masked():
+    """One key aligned with every query and far larger than the rest takes all the probability -- but only for
+    the rows at or after its position; earlier rows must not see it."""
+    L, d, hot = 12, 4, 5
+    Q = np.tile(np.array([1.0, 0, 0, 0]), (L, 1))
+    K = np.zeros((L, d)); K[hot, 0] = 60.0
+    V = np.arange(L * d, dtype=float).reshape(L, d)
+    out, _ = oracle.prompt_attention_rows(Q, K, V, list(range(L)), 1.0)
+    for i in range(L):
+        if i >= hot:
+            np.testing.assert_allclose(out[i], V[hot], rtol=1e-12)
+        else:
+            np.testing.assert_allclose(out[i], V[: i + 1].mean(axis=0), rtol=1e-12)
+
+
+def test_prompt_attention_last_row_equals_decode_attention_over_the_prompt():
+    """The last prompt row attends over the whole prompt: same output as one ATTEND_FIRST-style read of a cache
+    that holds every prompt token (cross-check against the decode-step oracle's attention)."""
+    rng = np.random.default_rng(33)
+    L, d = 17, 8
+    Q, K, V = rng.normal(size=(L, d)), rng.normal(size=(L, d)), rng.normal(size=(L, d))
+    out, lse = oracle.prompt_attention_rows(Q, K, V, [L - 1], 0.35)
+    p, l2 = oracle.attention_row(Q[L - 1], K, 0.35)
+    np.testing.assert_allclose(out[0], p @ V, rtol=1e-12)
+    assert lse[0] == pytest.approx(l2, rel=1e-14)
