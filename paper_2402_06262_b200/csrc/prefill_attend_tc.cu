@@ -1,13 +1,20 @@
 // Causal attention output of the prompt pass (Eq. 1 with the mask of Sec. 2.1) on the 5th-generation tensor
 // cores, bf16, d = 128:   out_i = sum_{j<=i} P_ij V_j,   P_ij = exp(scale Q_i.K_j - lse_i),
 // with the row log-sum-exp lse that the statistics pass produced, so that no running maximum and no rescaling
-// of the output accumulator is needed.  Per 128 x 128 tile two contractions:
-//   S = Q_a K_j^T       (both operands K-major, as TMA wrote them)           -> tensor memory, fp32
-//   O += P V_j          (P: bf16, written by the softmax warps into a swizzled K-major tile;
-//                        V_j: the TMA tile as it is, read as an MN-major operand) -> tensor memory, fp32
-// A CTA owns the query tiles (a, T-1-a) like the statistics passes.  Warps 0-7 turn S into P (two groups of four,
-// one per S accumulator), warp 8 issues TMA, warp 9 issues both contractions; the S product of tile j+1 is
-// issued before the P V product of tile j so that the tensor pipe works while the exponentials run.
+// of the output accumulator is needed.
+//
+// A CTA works on 256 query rows at a time (two 128-row query tiles h = 0, 1 that share every key/value tile it
+// streams, which halves the L2 traffic per product) and owns the 256-row blocks (a, T2-1-a), so that every CTA
+// does about the same number of tile products under the causal mask.  Per query tile and 128-key tile j:
+//   S_h  = Q_h K_j^T    operands in shared memory as TMA wrote them (K-major)       -> tensor memory, fp32
+//   P_h  = exp(...)     softmax group h (four warps, one query row per thread) reads S_h and writes P_h as
+//                       bf16 over the columns S_h occupied
+//   O_h += P_h V_j      A operand from tensor memory, V_j from shared memory as an MN-major operand
+// Tensor memory holds S_0 | S_1 | O_0 | O_1 (4 x 128 columns).  Warp 8 issues TMA (K ring and V ring), warp 9
+// issues the contractions in the order PV_0(j-1), S_0(j), PV_1(j-1), S_1(j): the products of one query tile
+// run while the other tile's exponentials are computed.  S_h(j) follows PV_h(j-1) in the issue order of one
+// thread, and the tensor pipe executes one thread's contractions in that order, so P_h(j-1) is read before S_h(j)
+// overwrites it.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -19,9 +26,9 @@
 
 namespace roco {
 
-constexpr int kAtStages = 2;                        // ring of (K_j, V_j) tile pairs
-constexpr int kAtStageBytes = 2 * kTcTileBytes;     // 64 KiB
-constexpr int kAtTmemCols = 512;                    // S0 | S1 | O | unused (allocations are powers of two)
+constexpr int kAtKStages = 2;                       // ring of K tiles
+constexpr int kAtVStages = 3;                       // ring of V tiles
+constexpr int kAtTmemCols = 512;                    // S0 | S1 | O0 | O1
 constexpr int kAtColO = 2 * kTcTile;
 constexpr int kAtComputeWarps = 8;
 constexpr int kAtThreads = kAtComputeWarps * 32 + 64;
@@ -42,38 +49,61 @@ __device__ __forceinline__ uint64_t smem_desc_sw128_mn(const void *p) {
 
 constexpr uint32_t kIdescPV = kIdescBf16M128N128 | (1u << 16);  // B operand MN-major
 
+// D[tmem] (+)= A[tmem] * B[smem]: A is 128 lanes (rows) x 8 columns of packed bf16 pairs (K = 16)
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// 32 lanes x 16 consecutive 32-bit columns: thread t of the warp writes lane (base + t)
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 struct AtSmem {
-  char *qt;     // query tile
-  char *ring;   // kAtStages x (K tile, V tile)
-  char *pt;     // probability tile, bf16, K-major, swizzled like a TMA tile
+  char *qt;     // two query tiles
+  char *kt;     // kAtKStages key tiles
+  char *vt;     // kAtVStages value tiles
   uint64_t *q_full, *q_empty;
-  uint64_t *ring_full, *ring_empty;  // [kAtStages]
-  uint64_t *acc_full, *acc_empty;    // [2]
-  uint64_t *p_full, *p_empty, *o_full, *o_empty;
+  uint64_t *k_full, *k_empty;  // [kAtKStages]
+  uint64_t *v_full, *v_empty;  // [kAtVStages]
+  uint64_t *s_full, *p_full;   // [2] per query tile
+  uint64_t *o_full, *o_empty;  // [2]
   uint32_t *tmem_base;
   int *abort_flag;
 };
 
-constexpr size_t kAtSmemBytes = 1024 + (size_t)kTcTileBytes * 2 + (size_t)kAtStages * kAtStageBytes + 16 * 8 + 16;
+constexpr int kAtBarriers = 2 + 2 * kAtKStages + 2 * kAtVStages + 8;
+constexpr size_t kAtSmemBytes = 1024 + (size_t)kTcTileBytes * (2 + kAtKStages + kAtVStages) + kAtBarriers * 8 + 16;
 
 __device__ inline AtSmem at_carve(char *raw) {
   AtSmem m;
   char *p = (char *)align_up((size_t)raw, 1024);
-  m.qt = p; p += kTcTileBytes;
-  m.ring = p; p += (size_t)kAtStages * kAtStageBytes;
-  m.pt = p; p += kTcTileBytes;
+  m.qt = p; p += 2 * kTcTileBytes;
+  m.kt = p; p += (size_t)kAtKStages * kTcTileBytes;
+  m.vt = p; p += (size_t)kAtVStages * kTcTileBytes;
   m.q_full = (uint64_t *)p; p += 8;
   m.q_empty = (uint64_t *)p; p += 8;
-  m.ring_full = (uint64_t *)p; p += 8 * kAtStages;
-  m.ring_empty = (uint64_t *)p; p += 8 * kAtStages;
-  m.acc_full = (uint64_t *)p; p += 16;
-  m.acc_empty = (uint64_t *)p; p += 16;
-  m.p_full = (uint64_t *)p; p += 8;
-  m.p_empty = (uint64_t *)p; p += 8;
-  m.o_full = (uint64_t *)p; p += 8;
-  m.o_empty = (uint64_t *)p; p += 8;
+  m.k_full = (uint64_t *)p; p += 8 * kAtKStages;
+  m.k_empty = (uint64_t *)p; p += 8 * kAtKStages;
+  m.v_full = (uint64_t *)p; p += 8 * kAtVStages;
+  m.v_empty = (uint64_t *)p; p += 8 * kAtVStages;
+  m.s_full = (uint64_t *)p; p += 16;
+  m.p_full = (uint64_t *)p; p += 16;
+  m.o_full = (uint64_t *)p; p += 16;
+  m.o_empty = (uint64_t *)p; p += 16;
   m.tmem_base = (uint32_t *)p; p += 8;
   m.abort_flag = (int *)p;
   return m;
@@ -94,20 +124,23 @@ __global__ void __launch_bounds__(kAtThreads, 1)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int u = blockIdx.x / npairs, pair = blockIdx.x % npairs;
   const int L = lens[u / G];
-  const int T = (L + kTcTile - 1) / kTcTile;
-  const int a0 = pair, a1 = T - 1 - pair;
+  const int T = (L + kTcTile - 1) / kTcTile;  // 128-row tiles
+  const int T2 = (T + 1) / 2;                 // 256-row blocks
+  const int a0 = pair, a1 = T2 - 1 - pair;
   const int n_tasks = (a0 > a1) ? 0 : (a0 == a1 ? 1 : 2);
   if (n_tasks == 0) return;
 
   if (tid == 0) {
     mbar_init(sm.q_full, 1);
     mbar_init(sm.q_empty, 1);
-    for (int i = 0; i < kAtStages; ++i) { mbar_init(&sm.ring_full[i], 1); mbar_init(&sm.ring_empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sm.acc_full[i], 1); mbar_init(&sm.acc_empty[i], 4); }
-    mbar_init(sm.p_full, 4);
-    mbar_init(sm.p_empty, 1);
-    mbar_init(sm.o_full, 1);
-    mbar_init(sm.o_empty, 4);
+    for (int i = 0; i < kAtKStages; ++i) { mbar_init(&sm.k_full[i], 1); mbar_init(&sm.k_empty[i], 1); }
+    for (int i = 0; i < kAtVStages; ++i) { mbar_init(&sm.v_full[i], 1); mbar_init(&sm.v_empty[i], 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sm.s_full[i], 1);
+      mbar_init(&sm.p_full[i], 4);
+      mbar_init(&sm.o_full[i], 1);
+      mbar_init(&sm.o_empty[i], 4);
+    }
     *sm.abort_flag = 0;
     mbar_init_fence();
   }
@@ -120,163 +153,163 @@ __global__ void __launch_bounds__(kAtThreads, 1)
   tc_fence_after();
   const uint32_t tmem = *sm.tmem_base;
 
-  auto task_tile = [&](int k) { return k == 0 ? a0 : a1; };  // query tile a streams key tiles 0..a
-  const int n_tiles = (a0 + 1) + (n_tasks == 2 ? a1 + 1 : 0);
+  // Task k works on the 256-row block A: query tiles 2A (h = 0) and 2A+1 (h = 1, if it exists); key tiles
+  // 0 .. 2A + nq - 1; query tile h takes part in key tile j while j <= 2A + h.
+  auto task_block = [&](int k) { return k == 0 ? a0 : a1; };
+  auto task_nq = [&](int A) { return (2 * A + 1 < T) ? 2 : 1; };
 
   if (warp == kAtComputeWarps) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int g = 0;
+      int gj = 0;  // key/value tiles issued so far
       for (int k = 0; k < n_tasks; ++k) {
-        const int a = task_tile(k);
+        const int A = task_block(k), nq = task_nq(A), nj = 2 * A + nq;
         if (k > 0) mbar_wait(sm.q_empty, (k - 1) & 1, abort_flag, status);
-        mbar_expect_tx(sm.q_full, kTcTileBytes);
-        tma_load_3d(sm.qt, &mapQ, 0, a * kTcTile, u, sm.q_full);
-        tma_load_3d(sm.qt + kTcHalfBytes, &mapQ, 64, a * kTcTile, u, sm.q_full);
-        for (int j = 0; j <= a; ++j, ++g) {
-          const int st = g % kAtStages;
-          if (g >= kAtStages) mbar_wait(&sm.ring_empty[st], ((g / kAtStages) - 1) & 1, abort_flag, status);
-          char *kd = sm.ring + (size_t)st * kAtStageBytes, *vd = kd + kTcTileBytes;
-          mbar_expect_tx(&sm.ring_full[st], kAtStageBytes);
-          tma_load_3d(kd, &mapK, 0, j * kTcTile, u, &sm.ring_full[st]);
-          tma_load_3d(kd + kTcHalfBytes, &mapK, 64, j * kTcTile, u, &sm.ring_full[st]);
-          tma_load_3d(vd, &mapV, 0, j * kTcTile, u, &sm.ring_full[st]);
-          tma_load_3d(vd + kTcHalfBytes, &mapV, 64, j * kTcTile, u, &sm.ring_full[st]);
+        mbar_expect_tx(sm.q_full, nq * kTcTileBytes);
+        for (int h = 0; h < nq; ++h) {
+          tma_load_3d(sm.qt + h * kTcTileBytes, &mapQ, 0, (2 * A + h) * kTcTile, u, sm.q_full);
+          tma_load_3d(sm.qt + h * kTcTileBytes + kTcHalfBytes, &mapQ, 64, (2 * A + h) * kTcTile, u, sm.q_full);
+        }
+        for (int j = 0; j < nj; ++j, ++gj) {
+          const int ks = gj % kAtKStages, vs = gj % kAtVStages;
+          if (gj >= kAtKStages) mbar_wait(&sm.k_empty[ks], ((gj / kAtKStages) - 1) & 1, abort_flag, status);
+          char *kd = sm.kt + (size_t)ks * kTcTileBytes;
+          mbar_expect_tx(&sm.k_full[ks], kTcTileBytes);
+          tma_load_3d(kd, &mapK, 0, j * kTcTile, u, &sm.k_full[ks]);
+          tma_load_3d(kd + kTcHalfBytes, &mapK, 64, j * kTcTile, u, &sm.k_full[ks]);
+          if (gj >= kAtVStages) mbar_wait(&sm.v_empty[vs], ((gj / kAtVStages) - 1) & 1, abort_flag, status);
+          char *vd = sm.vt + (size_t)vs * kTcTileBytes;
+          mbar_expect_tx(&sm.v_full[vs], kTcTileBytes);
+          tma_load_3d(vd, &mapV, 0, j * kTcTile, u, &sm.v_full[vs]);
+          tma_load_3d(vd + kTcHalfBytes, &mapV, 64, j * kTcTile, u, &sm.v_full[vs]);
         }
       }
     }
   } else if (warp == kAtComputeWarps + 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      // tile g of the CTA: its task and whether it opens / closes the task
-      auto first_of = [&](int g) { return g == 0 || g == a0 + 1; };
-      auto last_of = [&](int g) { return g == a0 || g == n_tiles - 1; };
-      auto task_of = [&](int g) { return g <= a0 ? 0 : 1; };
-      auto issue_s = [&](int g) {  // S = Q K_j^T into accumulator g & 1
-        const int st = g % kAtStages, ac = g & 1;
-        if (first_of(g)) mbar_wait(sm.q_full, task_of(g) & 1, abort_flag, status);
-        mbar_wait(&sm.ring_full[st], (g / kAtStages) & 1, abort_flag, status);
-        if (g >= 2) mbar_wait(&sm.acc_empty[ac], ((g >> 1) - 1) & 1, abort_flag, status);
-        tc_fence_after();
-        const char *kt = sm.ring + (size_t)st * kAtStageBytes;
+      int gj0 = 0;                 // key tiles of earlier tasks
+      int ns[2] = {0, 0};          // S products issued per query tile (= P tiles expected)
+      for (int k = 0; k < n_tasks; ++k) {
+        const int A = task_block(k), nq = task_nq(A), nj = 2 * A + nq;
+        auto active = [&](int h, int j) { return h < nq && j >= 0 && j < nj && j <= 2 * A + h; };
+        auto last_user = [&](int h, int j) { return !active(h + 1, j); };  // h is the last query tile using tile j
+        int np[2] = {ns[0], ns[1]};  // P tiles consumed per query tile
+        mbar_wait(sm.q_full, k & 1, abort_flag, status);
+        for (int j = 0; j <= nj; ++j) {
+          for (int h = 0; h < 2; ++h) {
+            if (active(h, j - 1)) {  // O_h += P_h V_{j-1}
+              const int gj = gj0 + j - 1, vs = gj % kAtVStages;
+              if (h == 0 || !active(0, j - 1)) mbar_wait(&sm.v_full[vs], (gj / kAtVStages) & 1, abort_flag, status);
+              mbar_wait(&sm.p_full[h], np[h] & 1, abort_flag, status);
+              ++np[h];
+              if (j - 1 == 0 && k > 0) mbar_wait(&sm.o_empty[h], (k - 1) & 1, abort_flag, status);
+              tc_fence_after();
+              const char *vt = sm.vt + (size_t)vs * kTcTileBytes;
 #pragma unroll
-        for (int kk = 0; kk < kTcD / 16; ++kk) {
-          const int off = (kk / 4) * kTcHalfBytes + (kk % 4) * 32;
-          umma_bf16(tmem + (uint32_t)(ac * kTcTile), smem_desc_sw128(sm.qt + off), smem_desc_sw128(kt + off),
-                    kIdescBf16M128N128, kk > 0 ? 1u : 0u);
-        }
-        umma_commit(&sm.acc_full[ac]);
-        if (last_of(g)) umma_commit(sm.q_empty);
-      };
-      auto issue_pv = [&](int g) {  // O += P V_j
-        const int st = g % kAtStages;
-        mbar_wait(sm.p_full, g & 1, abort_flag, status);
-        if (first_of(g) && task_of(g) > 0) mbar_wait(sm.o_empty, (task_of(g) - 1) & 1, abort_flag, status);
-        tc_fence_after();
-        const char *vt = sm.ring + (size_t)st * kAtStageBytes + kTcTileBytes;
+              for (int kk = 0; kk < kTcTile / 16; ++kk)  // 16 keys per instruction
+                umma_bf16_ts(tmem + (uint32_t)(kAtColO + h * kTcTile), tmem + (uint32_t)(h * kTcTile + kk * 8),
+                             smem_desc_sw128_mn(vt + kk * 2048), kIdescPV, (kk > 0 || j - 1 > 0) ? 1u : 0u);
+              if (last_user(h, j - 1)) umma_commit(&sm.v_empty[vs]);
+              if (!active(h, j)) umma_commit(&sm.o_full[h]);  // that was this query tile's last key tile
+            }
+            if (active(h, j)) {  // S_h = Q_h K_j^T
+              const int gj = gj0 + j, ks = gj % kAtKStages;
+              if (h == 0 || !active(0, j)) mbar_wait(&sm.k_full[ks], (gj / kAtKStages) & 1, abort_flag, status);
+              tc_fence_after();
+              const char *kt = sm.kt + (size_t)ks * kTcTileBytes;
+              const char *qt = sm.qt + h * kTcTileBytes;
 #pragma unroll
-        for (int kk = 0; kk < kTcTile / 16; ++kk) {  // 16 keys per instruction
-          const int poff = (kk / 4) * kTcHalfBytes + (kk % 4) * 32;
-          umma_bf16(tmem + (uint32_t)kAtColO, smem_desc_sw128(sm.pt + poff), smem_desc_sw128_mn(vt + kk * 2048),
-                    kIdescPV, (kk > 0 || !first_of(g)) ? 1u : 0u);
+              for (int kk = 0; kk < kTcD / 16; ++kk) {
+                const int off = (kk / 4) * kTcHalfBytes + (kk % 4) * 32;
+                umma_bf16(tmem + (uint32_t)(h * kTcTile), smem_desc_sw128(qt + off), smem_desc_sw128(kt + off),
+                          kIdescBf16M128N128, kk > 0 ? 1u : 0u);
+              }
+              umma_commit(&sm.s_full[h]);
+              ++ns[h];
+              if (last_user(h, j)) umma_commit(&sm.k_empty[ks]);
+              if (j == nj - 1 && last_user(h, j)) umma_commit(sm.q_empty);  // the task's last S product
+            }
+          }
         }
-        umma_commit(&sm.ring_empty[st]);
-        umma_commit(sm.p_empty);
-        if (last_of(g)) umma_commit(sm.o_full);
-      };
-      issue_s(0);
-      for (int g = 0; g < n_tiles; ++g) {
-        if (g + 1 < n_tiles) issue_s(g + 1);
-        issue_pv(g);
+        gj0 += nj;
       }
     }
   } else {
     // ------------------------------------------------------------------ softmax warps
     const float zscale = scale * kLog2e;
-    const int group = warp >> 2;
+    const int h = warp >> 2;                 // the query tile this group serves
     const int row = (warp & 3) * 32 + lane;  // TMEM lane = query row inside the tile
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t taddr = tmem + lane_addr + (uint32_t)(group * kTcTile);
-    char *prow = sm.pt + row * 128;
-    const int sw = row & 7;
-    int g0 = 0, mine = 0;
+    const uint32_t taddr = tmem + lane_addr + (uint32_t)(h * kTcTile);
+    int gj0 = 0, mine = 0;
     for (int k = 0; k < n_tasks; ++k) {
-      const int a = task_tile(k);
-      const int grow = a * kTcTile + row;
-      const float nl2 = (grow < L) ? -lse[(size_t)u * Lmax + grow] * kLog2e : 0.f;
-      const f32x2 nl22 = pack2(nl2, nl2), zs2 = pack2(zscale, zscale);
-      const int t0 = ((g0 & 1) == group) ? 0 : 1;
-      for (int j = t0; j <= a; j += 2, ++mine) {
-        const int g = g0 + j;
-        mbar_wait(&sm.acc_full[group], mine & 1, abort_flag, status);
-        tc_fence_after();
-        const int col0 = j * kTcTile;
-        uint32_t ra[32], rb[32];
-        bool p_free = (g == 0);
+      const int A = task_block(k), nq = task_nq(A), nj = 2 * A + nq;
+      if (h < nq) {
+        const int a = 2 * A + h;  // this group's 128-row query tile; its diagonal key tile
+        const int grow = a * kTcTile + row;
+        const float nl2 = (grow < L) ? -lse[(size_t)u * Lmax + grow] * kLog2e : 0.f;
+        const f32x2 nl22 = pack2(nl2, nl2), zs2 = pack2(zscale, zscale);
+        for (int j = 0; j <= a; ++j, ++mine) {
+          mbar_wait(&sm.s_full[h], mine & 1, abort_flag, status);
+          tc_fence_after();
+          const int col0 = j * kTcTile;
+          uint32_t ra[32], rb[32];
 
-        auto chunk = [&](const uint32_t (&r)[32], int c, auto masked_tag) {
-          constexpr bool kMasked = decltype(masked_tag)::value;
-          uint32_t pk[16];
+          auto chunk = [&](const uint32_t (&r)[32], int c, auto masked_tag) {
+            constexpr bool kMasked = decltype(masked_tag)::value;
+            uint32_t pk[16];
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            f32x2 p2 = exp2_pair(fma2(pack2u(r[i], r[i + 1]), zs2, nl22), i >> 1);
-            float pa, pb;
-            unpack2(p2, pa, pb);
-            if (kMasked) {
-              const int kj = col0 + c * 32 + i;
-              pa = (kj <= grow) ? pa : 0.f;
-              pb = (kj + 1 <= grow) ? pb : 0.f;
+            for (int i = 0; i < 32; i += 2) {
+              f32x2 p2 = exp2_pair(fma2(pack2u(r[i], r[i + 1]), zs2, nl22), i >> 1);
+              float pa, pb;
+              unpack2(p2, pa, pb);
+              if (kMasked) {
+                const int kj = col0 + c * 32 + i;
+                pa = (kj <= grow) ? pa : 0.f;
+                pb = (kj + 1 <= grow) ? pb : 0.f;
+              }
+              pk[i >> 1] = pack_bf16x2(pa, pb);
             }
-            pk[i >> 1] = pack_bf16x2(pa, pb);
-          }
-          if (!p_free) {  // the previous tile's P V product must have read the probability tile
-            mbar_wait(sm.p_empty, (g - 1) & 1, abort_flag, status);
-            p_free = true;
-          }
-          char *half = prow + (c >> 1) * kTcHalfBytes;
+            tmem_st16(taddr + c * 16, pk);  // behind the columns already read
+          };
+          auto tile = [&](auto masked_tag) {
+            tmem_ld32_issue(taddr, ra);
+            tmem_ld_wait(ra);
+            tmem_ld32_issue(taddr + 32, rb);
+            chunk(ra, 0, masked_tag);
+            tmem_ld_wait(rb);
+            tmem_ld32_issue(taddr + 64, ra);
+            chunk(rb, 1, masked_tag);
+            tmem_ld_wait(ra);
+            tmem_ld32_issue(taddr + 96, rb);
+            chunk(ra, 2, masked_tag);
+            tmem_ld_wait(rb);
+            chunk(rb, 3, masked_tag);
+          };
+          if (j == a) tile(std::true_type{}); else tile(std::false_type{});
+          // value rows past the prompt may hold anything (0 x NaN would poison every query): clear them.
+          // Only the last key tile of the prompt has such rows, and only one query tile ever reaches it.
+          if (j == T - 1 && col0 + row >= L) {
+            const int gj = gj0 + j, vs = gj % kAtVStages;
+            mbar_wait(&sm.v_full[vs], (gj / kAtVStages) & 1, abort_flag, status);
+            char *vrow = sm.vt + (size_t)vs * kTcTileBytes + row * 128;
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int cc = (c & 1) * 4 + i;
-            *reinterpret_cast<uint4 *>(half + ((cc ^ sw) << 4)) =
-                make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+            for (int i = 0; i < 8; ++i) {
+              *reinterpret_cast<uint4 *>(vrow + i * 16) = make_uint4(0, 0, 0, 0);
+              *reinterpret_cast<uint4 *>(vrow + kTcHalfBytes + i * 16) = make_uint4(0, 0, 0, 0);
+            }
+            fence_async_smem();  // generic-proxy writes -> visible to the tensor core's reads
           }
-        };
-        auto tile = [&](auto masked_tag) {
-          tmem_ld32_issue(taddr, ra);
-          tmem_ld_wait(ra);
-          tmem_ld32_issue(taddr + 32, rb);
-          chunk(ra, 0, masked_tag);
-          tmem_ld_wait(rb);
-          tmem_ld32_issue(taddr + 64, ra);
-          chunk(rb, 1, masked_tag);
-          tmem_ld_wait(ra);
-          tmem_ld32_issue(taddr + 96, rb);
-          chunk(ra, 2, masked_tag);
-          tmem_ld_wait(rb);
+          tmem_st_wait();
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&sm.acc_empty[group]);
-          chunk(rb, 3, masked_tag);
-        };
-        if (j == a) tile(std::true_type{}); else tile(std::false_type{});
-        // value rows past the prompt may hold anything (0 x NaN would poison every query): clear them
-        if (j == T - 1 && col0 + row >= L) {
-          char *vrow = sm.ring + (size_t)(g % kAtStages) * kAtStageBytes + kTcTileBytes + row * 128;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            *reinterpret_cast<uint4 *>(vrow + i * 16) = make_uint4(0, 0, 0, 0);
-            *reinterpret_cast<uint4 *>(vrow + kTcHalfBytes + i * 16) = make_uint4(0, 0, 0, 0);
-          }
+          if (lane == 0) mbar_arrive(&sm.p_full[h]);
         }
-        fence_async_smem();  // generic-proxy writes -> visible to the tensor core's reads
-        __syncwarp();
-        if (lane == 0) mbar_arrive(sm.p_full);
-      }
-      g0 += a + 1;
-      if (group == 0) {  // read the finished output accumulator: one query row per thread
-        mbar_wait(sm.o_full, k & 1, abort_flag, status);
+        // the finished output accumulator of this query tile: one row per thread
+        mbar_wait(&sm.o_full[h], k & 1, abort_flag, status);
         tc_fence_after();
-        const uint32_t oaddr = tmem + lane_addr + (uint32_t)kAtColO;
+        const uint32_t oaddr = tmem + lane_addr + (uint32_t)(kAtColO + h * kTcTile);
         uint32_t r[32];
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -294,8 +327,9 @@ __global__ void __launch_bounds__(kAtThreads, 1)
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(sm.o_empty);
+        if (lane == 0) mbar_arrive(&sm.o_empty[h]);
       }
+      gj0 += nj;
     }
   }
   tc_fence_before();
@@ -312,7 +346,8 @@ roco_status launch_prefill_attend_tc(int S, int G, int Lmax, const int *lens_dev
       !make_tensor_map_prompt_bf16(&mapV, V, U, Lmax))
     return ROCO_ERR_CUDA;
   const int T = (maxlen + kTcTile - 1) / kTcTile;
-  const int npairs = (T + 1) / 2;
+  const int T2 = (T + 1) / 2;
+  const int npairs = (T2 + 1) / 2;
   const unsigned grid = (unsigned)U * (unsigned)npairs;
   if (cudaFuncSetAttribute(prefill_attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)kAtSmemBytes) != cudaSuccess)
