@@ -32,6 +32,13 @@ constexpr int kAtTmemCols = 512;                    // S0 | S1 | O0 | O1
 constexpr int kAtColO = 2 * kTcTile;
 constexpr int kAtComputeWarps = 8;
 constexpr int kAtThreads = kAtComputeWarps * 32 + 64;
+// Of every 8 pairs of exponentials, how many run on the FMA pipe (polynomial) instead of the exponential unit.
+// Here two contractions stand against each tile's exponentials, so the exponential unit is not the limit and
+// the cheaper instruction sequence wins (measured: 0 -> 1043, 1 -> 1009, 2 -> 997 TFLOP/s executed).
+#ifndef ROCO_ATTEND_POLY_PAIRS_PER_8
+#define ROCO_ATTEND_POLY_PAIRS_PER_8 0
+#endif
+constexpr int kAtPolyPairsPer8 = ROCO_ATTEND_POLY_PAIRS_PER_8;
 
 // V_j as the B operand of O += P V_j: B[n][k] = V[key k][dim n] with the dimension index contiguous
 // (MN-major).  The tile sits as two halves of 64 dims, each 128 rows (keys) of 128 bytes, 128-byte swizzle:
@@ -261,7 +268,8 @@ __global__ void __launch_bounds__(kAtThreads, 1)
             uint32_t pk[16];
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
-              f32x2 p2 = exp2_pair(fma2(pack2u(r[i], r[i + 1]), zs2, nl22), i >> 1);
+              f32x2 p2 = ((i >> 1) & 7) < kAtPolyPairsPer8 ? exp2_poly2(fma2(pack2u(r[i], r[i + 1]), zs2, nl22))
+                                                         : exp2_mufu2(fma2(pack2u(r[i], r[i + 1]), zs2, nl22));
               float pa, pb;
               unpack2(p2, pa, pb);
               if (kMasked) {
