@@ -21,6 +21,11 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// Rounds a shared-memory pointer up to a multiple of `a` bytes by pointer arithmetic.  (A round trip through an
+// integer would hide the state space from the compiler, which then emits generic instead of shared-memory
+// loads, stores and atomics for everything carved from that pointer.)
+__device__ __forceinline__ char *smem_align(char *p, uint32_t a) { return p + ((a - (smem_u32(p) & (a - 1))) & (a - 1)); }
+
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
@@ -39,31 +44,42 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// One poll.  The hint lets the hardware keep the thread suspended (off the issue slots the other warps of the
+// SM need) until the phase completes or the hint runs out, instead of a short system-chosen limit.
+constexpr uint32_t kSuspendHintNs = 1000000u;
+
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendHintNs)
       : "memory");
   return ok != 0;
 }
 
-// Every wait is bounded: after kWaitPolls failed polls the thread records ROCO_DEV_WAIT_TIMEOUT in the
-// status word and in the CTA's abort flag and carries on along the *same* control flow (so that no
-// barrier is left short of arrivals); once the abort flag is up every later wait returns at once.
-// The CTA's results are then garbage and the status word says so.
-constexpr uint32_t kWaitPolls = 1u << 22;
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Every wait is bounded: once kWaitLimitNs have passed without the phase completing, the thread records
+// ROCO_DEV_WAIT_TIMEOUT in the status word and in the CTA's abort flag and carries on along the *same* control
+// flow (so that no barrier is left short of arrivals); once the abort flag is up every later wait returns at
+// once.  The CTA's results are then garbage and the status word says so.
+constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ void mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
                                           int32_t *status) {
   if (mbar_try_wait(bar, parity)) return;
-  for (uint32_t i = 0; i < kWaitPolls; ++i) {
+  const uint64_t t0 = global_timer_ns();
+  do {
     if (*abort_flag) return;
     if (mbar_try_wait(bar, parity)) return;
-  }
+  } while (global_timer_ns() - t0 < kWaitLimitNs);
   *abort_flag = 1;
   if (status) atomicOr(status, ROCO_DEV_WAIT_TIMEOUT);
 }

@@ -71,7 +71,7 @@ __host__ __device__ inline size_t decode_smem_bytes(int B, int d, int stages) {
 template <int TILE>
 __device__ inline DecodeSmem carve(char *raw, int B, int d, int stages) {
   DecodeSmem m;
-  char *p = (char *)align_up((size_t)raw, 128);
+  char *p = smem_align(raw, 128);
   const size_t Bp = align_up((size_t)B, 4);
   m.ring = p; p += (size_t)stages * TILE;
   m.z = (float *)p; p += Bp * 4;
@@ -179,19 +179,33 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     // (a slot that has just received the new token starts from zero)
     auto update_statistics = [&](int fresh_slot) {
       mbar_wait(sm.p_ready, 0, abort_flag, p.status);
-#pragma unroll 4
-      for (int j = ptid; j < live_att; j += kPolicyThreads) {
-        const bool fresh = (j == fresh_slot) || (j >= live0);
-        const float pj = sm.z[j];
-        const float s0 = fresh ? 0.f : p.s[unit_st + j], q0 = fresh ? 0.f : p.q[unit_st + j];
-        const int n0 = fresh ? 0 : p.n[unit_st + j];
-        p.s[unit_st + j] = s0 + pj;
-        // Acc^square, except for the two policies of Table 1 that keep something else in this array
-        float q1 = fmaf(pj, pj, q0);
-        if (p.policy == ROCO_POLICY_SCISSORHANDS) q1 = q0 + (pj * (float)live_att > 1.f ? 1.f : 0.f);  // AQAS
-        if (p.policy == ROCO_POLICY_TOVA) q1 = pj;                                                    // LTAS
-        p.q[unit_st + j] = q1;
-        p.n[unit_st + j] = n0 + 1;
+      // four slots per turn: all loads are issued before the first store (the compiler cannot move a load of
+      // one array above a store to another, and the arrays are read-modify-written in place)
+      constexpr int kBatch = 4;
+      for (int j0 = ptid; j0 < live_att; j0 += kBatch * kPolicyThreads) {
+        float s0[kBatch], q0[kBatch];
+        int n0[kBatch];
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+          const int j = j0 + k * kPolicyThreads;
+          const bool old = j < live_att && j != fresh_slot && j < live0;
+          s0[k] = old ? p.s[unit_st + j] : 0.f;
+          q0[k] = old ? p.q[unit_st + j] : 0.f;
+          n0[k] = old ? p.n[unit_st + j] : 0;
+        }
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+          const int j = j0 + k * kPolicyThreads;
+          if (j >= live_att) break;
+          const float pj = sm.z[j];
+          p.s[unit_st + j] = s0[k] + pj;
+          // Acc^square, except for the two policies of Table 1 that keep something else in this array
+          float q1 = fmaf(pj, pj, q0[k]);
+          if (p.policy == ROCO_POLICY_SCISSORHANDS) q1 = q0[k] + (pj * (float)live_att > 1.f ? 1.f : 0.f);  // AQAS
+          if (p.policy == ROCO_POLICY_TOVA) q1 = pj;                                                       // LTAS
+          p.q[unit_st + j] = q1;
+          p.n[unit_st + j] = n0[k] + 1;
+        }
       }
     };
     if (!evict_first) {  // select on the updated statistics

@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(kSpThreads) split_attend_kernel(const SplitPar
   constexpr int kEPC = Elem<T>::kPerChunk;
 
   extern __shared__ char sp_smem_raw[];
-  char *ring = (char *)align_up((size_t)sp_smem_raw, 128);
+  char *ring = smem_align(sp_smem_raw, 128);
   float *z = reinterpret_cast<float *>(ring + (size_t)kSpStages * kSpTile);   // [range rows]
   float *qf = z + align_up((size_t)p.B, 4);
   float *outred = qf + D;                                                     // [8][D]

@@ -73,7 +73,7 @@ __host__ __device__ inline size_t multi_smem_bytes(int B, int d, int stages, int
 
 __device__ inline MultiSmem multi_carve(char *raw, int B, int d, int stages, int M, int nb) {
   MultiSmem m;
-  char *p = (char *)align_up((size_t)raw, 128);
+  char *p = smem_align(raw, 128);
   const size_t Bp = align_up((size_t)B, 16);
   m.ring = p; p += (size_t)stages * kMqTile;
   m.z = (float *)p; p += (size_t)M * Bp * 4;
@@ -86,7 +86,7 @@ __device__ inline MultiSmem multi_carve(char *raw, int B, int d, int stages, int
   m.vnew = (float *)p; p += (size_t)nb * d * 4;
   m.zn = (float *)p; p += (size_t)M * nb * 4;
   m.outred = (float *)p; p += (size_t)kMqConsumerWarps * kMqQPW * d * 4;
-  p = (char *)align_up((size_t)p, 8);
+  p = smem_align(p, 8);
   m.full = (uint64_t *)p; p += stages * 8;
   m.empty = (uint64_t *)p; p += stages * 8;
   m.p_ready = (uint64_t *)p; p += 8;
@@ -292,30 +292,46 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
 
   // statistics of Sec. 4.3 once the probabilities are in shared memory
   mbar_wait(v.p_ready, 0, abort_flag, p.status);
-  for (int j = ptid; j < live1; j += kMqPolicyThreads) {
-    const int jn = v.newtok[j];
-    const bool fresh = jn >= 0;
-    float ds = 0.f, dq = 0.f;
-    int dn;
-    if (p.kind == kMqGqa) {
-      for (int i = 0; i < M; ++i) ds += (fresh && v.pn) ? v.pn[i * nb + jn] : v.z[(size_t)i * Bp + j];
-      ds /= (float)M;  // group-wise averaged attention score
-      dq = ds * ds;
-      dn = 1;
-    } else {
-      const int i0 = fresh ? jn : 0;  // query i sees new token jn only if i >= jn
-      for (int i = i0; i < M; ++i) {
-        const float pij = (fresh && v.pn) ? v.pn[i * nb + jn] : v.z[(size_t)i * Bp + j];
-        ds += pij;
-        dq = fmaf(pij, pij, dq);
-      }
-      dn = M - i0;
+  // four slots per turn, their old statistics loaded before the first store (the arrays are updated in place,
+  // so the compiler keeps loads behind earlier stores)
+  constexpr int kBatch = 4;
+  for (int j0 = ptid; j0 < live1; j0 += kBatch * kMqPolicyThreads) {
+    float s0v[kBatch], q0v[kBatch];
+    int n0v[kBatch];
+#pragma unroll
+    for (int k = 0; k < kBatch; ++k) {
+      const int j = j0 + k * kMqPolicyThreads;
+      const bool old = j < live1 && v.newtok[j] < 0;
+      s0v[k] = old ? gs[j] : 0.f;
+      q0v[k] = old ? gq[j] : 0.f;
+      n0v[k] = old ? gn[j] : 0;
     }
-    const float s0 = fresh ? 0.f : gs[j], q0 = fresh ? 0.f : gq[j];
-    const int n0 = fresh ? 0 : gn[j];
-    p.s[unit_st + j] = s0 + ds;
-    p.q[unit_st + j] = q0 + dq;
-    p.n[unit_st + j] = n0 + dn;
+#pragma unroll
+    for (int k = 0; k < kBatch; ++k) {
+      const int j = j0 + k * kMqPolicyThreads;
+      if (j >= live1) break;
+      const int jn = v.newtok[j];
+      const bool fresh = jn >= 0;
+      float ds = 0.f, dq = 0.f;
+      int dn;
+      if (p.kind == kMqGqa) {
+        for (int i = 0; i < M; ++i) ds += (fresh && v.pn) ? v.pn[i * nb + jn] : v.z[(size_t)i * Bp + j];
+        ds /= (float)M;  // group-wise averaged attention score
+        dq = ds * ds;
+        dn = 1;
+      } else {
+        const int i0 = fresh ? jn : 0;  // query i sees new token jn only if i >= jn
+        for (int i = i0; i < M; ++i) {
+          const float pij = (fresh && v.pn) ? v.pn[i * nb + jn] : v.z[(size_t)i * Bp + j];
+          ds += pij;
+          dq = fmaf(pij, pij, dq);
+        }
+        dn = M - i0;
+      }
+      p.s[unit_st + j] = s0v[k] + ds;
+      p.q[unit_st + j] = q0v[k] + dq;
+      p.n[unit_st + j] = n0v[k] + dn;
+    }
   }
 }
 
@@ -560,7 +576,7 @@ __host__ __device__ inline size_t multi_tc_smem_bytes(int B, int stages, int M, 
 
 __device__ inline MultiTcSmem multi_tc_carve(char *raw, int B, int stages, int M, int nb) {
   MultiTcSmem m;
-  char *p = (char *)align_up((size_t)raw, 1024);
+  char *p = smem_align(raw, 1024);
   const size_t Bp = multi_tc_row_stride(B);
   m.ring = p; p += (size_t)stages * kMqTile;
   m.z = (float *)p; p += (size_t)M * Bp * 4;
@@ -573,7 +589,7 @@ __device__ inline MultiTcSmem multi_tc_carve(char *raw, int B, int stages, int M
   m.zn = (float *)p; p += (size_t)M * nb * 4;
   m.pn = (float *)p; p += (size_t)M * nb * 4;
   m.qf = (float *)p; p += (size_t)M * 128 * 4;
-  p = (char *)align_up((size_t)p, 8);
+  p = smem_align(p, 8);
   m.full = (uint64_t *)p; p += stages * 8;
   m.empty = (uint64_t *)p; p += stages * 8;
   m.p_ready = (uint64_t *)p; p += 8;

@@ -97,7 +97,7 @@ constexpr size_t kAtSmemBytes = 1024 + (size_t)kTcTileBytes * (2 + kAtKStages + 
 
 __device__ inline AtSmem at_carve(char *raw) {
   AtSmem m;
-  char *p = (char *)align_up((size_t)raw, 1024);
+  char *p = smem_align(raw, 1024);
   m.qt = p; p += 2 * kTcTileBytes;
   m.kt = p; p += (size_t)kAtKStages * kTcTileBytes;
   m.vt = p; p += (size_t)kAtVStages * kTcTileBytes;

@@ -51,7 +51,7 @@ constexpr size_t kTcSmemBytes = 1024 /*align*/ + (size_t)(1 + kTcStages) * kTcTi
 
 __device__ inline TcSmem tc_carve(char *raw) {
   TcSmem m;
-  char *p = (char *)align_up((size_t)raw, 1024);  // swizzle atoms are 1024-byte aligned
+  char *p = smem_align(raw, 1024);  // swizzle atoms are 1024-byte aligned
   m.stat = p; p += kTcTileBytes;
   m.ring = p; p += (size_t)kTcStages * kTcTileBytes;
   m.lse2 = (float *)p; p += 4 * 128 * 4;

@@ -22,6 +22,12 @@ struct SelectScratch {
   int red_slot[32];
 };
 
+// Shared-memory reduction with the state space spelled out: the scratch is reached through pointers whose
+// provenance the compiler cannot see, and a generic-address atomic on shared memory is far slower.
+__device__ __forceinline__ void smem_red_add(uint32_t *addr, uint32_t v) {
+  asm volatile("red.shared::cta.add.u32 [%0], %1;" ::"r"(smem_u32(addr)), "r"(v) : "memory");
+}
+
 // k-th smallest (0-based) of key(j) over the j in [0, n) with pred(j); keys are unsigned integers of type
 // KeyT (32 or 64 bits).  Called by all `nthreads` threads that synchronise on named barrier `bar_id`.
 // *rank_in_ties: how many elements equal to the result precede the k-th in a stable order (so
@@ -39,8 +45,8 @@ __device__ __forceinline__ KeyT radix_select(KeyF key, PredF pred, int n, uint32
 #pragma unroll 4
     for (int j = tid; j < n; j += nthreads) {
       if (pred(j)) {
-        KeyT x = key(j);
-        if ((x & mask) == prefix) atomicAdd(&sc.hist[(uint32_t)(x >> shift) & 255u], 1u);
+        const KeyT x = key(j);
+        if ((x & mask) == prefix) smem_red_add(&sc.hist[(uint32_t)(x >> shift) & 255u], 1u);
       }
     }
     named_bar_sync(bar_id, nthreads);
