@@ -108,6 +108,12 @@ struct PolicyView {
   float *pn;  // [M][nb] probabilities of the new tokens when the consumers have zeroed them in z, else nullptr
   int *ctl;
   uint64_t *p_ready, *policy_done;
+  // Tensor-core kernel only (else nullptr / false): the producer copies the unit's s, q, n arrays into vkey, mkey,
+  // nbuf with bulk copies that complete on stats_full (the keys are then formed in place), and the consumer warps
+  // compute the new tokens' scores themselves, so the policy warps stage only the new values.
+  int *nbuf;
+  uint64_t *stats_full;
+  bool zn_by_consumers;
 };
 
 // The policy warps' part of a multi-query step: free `need` slots (Sec. 4.3 rule on frozen statistics), insert
@@ -134,14 +140,25 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     const uint4 *gv = reinterpret_cast<const uint4 *>(p.v_new + (size_t)u * p.kv_ustride * kRowBytes);
     const uint4 *gqr = reinterpret_cast<const uint4 *>(p.Q + (size_t)u * p.q_ustride * kRowBytes);
     const int nkv = nb * D / kEPC, nq = v.qf ? M * D / kEPC : 0;
+    if (v.zn_by_consumers) {
 #pragma unroll 4
-    for (int i = ptid; i < 2 * nkv + nq; i += kMqPolicyThreads) {
-      const uint4 c = i < nkv ? gk[i] : (i < 2 * nkv ? gv[i - nkv] : gqr[i - 2 * nkv]);
-      float *dst = i < nkv ? v.knew + i * kEPC : (i < 2 * nkv ? v.vnew + (i - nkv) * kEPC : v.qf + (i - 2 * nkv) * kEPC);
-      float f[kEPC];
-      Elem<T>::unpack(c, f);
+      for (int i = ptid; i < nkv; i += kMqPolicyThreads) {
+        float f[kEPC];
+        Elem<T>::unpack(gv[i], f);
 #pragma unroll
-      for (int e = 0; e < kEPC; ++e) dst[e] = f[e];
+        for (int e = 0; e < kEPC; ++e) v.vnew[i * kEPC + e] = f[e];
+      }
+    } else {
+#pragma unroll 4
+      for (int i = ptid; i < 2 * nkv + nq; i += kMqPolicyThreads) {
+        const uint4 c = i < nkv ? gk[i] : (i < 2 * nkv ? gv[i - nkv] : gqr[i - 2 * nkv]);
+        float *dst =
+            i < nkv ? v.knew + i * kEPC : (i < 2 * nkv ? v.vnew + (i - nkv) * kEPC : v.qf + (i - 2 * nkv) * kEPC);
+        float f[kEPC];
+        Elem<T>::unpack(c, f);
+#pragma unroll
+        for (int e = 0; e < kEPC; ++e) dst[e] = f[e];
+      }
     }
   }
   named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
@@ -150,12 +167,23 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     // the rule of Sec. 4.3 applied `need` times on frozen statistics = one pass: the tokens outside the scope
     // (the live0 - m last in (variance, position) order) never enter it, so the `need` first of the scope in
     // (mean, position) order leave
+    if (v.stats_full) {  // s, q, n sit in vkey, mkey, nbuf: form the keys in place
+      mbar_wait(v.stats_full, 0, abort_flag, p.status);
 #pragma unroll 8
-    for (int j = ptid; j < live0; j += kMqPolicyThreads) {
-      const float sj = gs[j], qj = gq[j];
-      const int nj = gn[j];
-      v.vkey[j] = variance_key_fast(sj, qj, nj);
-      v.mkey[j] = mean_fast(sj, nj);
+      for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+        const float sj = __uint_as_float(v.vkey[j]), qj = v.mkey[j];
+        const int nj = v.nbuf[j];
+        v.vkey[j] = variance_key_fast(sj, qj, nj);
+        v.mkey[j] = mean_fast(sj, nj);
+      }
+    } else {
+#pragma unroll 8
+      for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+        const float sj = gs[j], qj = gq[j];
+        const int nj = gn[j];
+        v.vkey[j] = variance_key_fast(sj, qj, nj);
+        v.mkey[j] = mean_fast(sj, nj);
+      }
     }
     named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
     const int m = scope_size(live0, p.r, p.scope_mode);
@@ -262,7 +290,9 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
   }
   // scores of every query against every new token, from k_new directly (log2 domain)
   const float zscale = p.scale * kLog2e;
-  if (v.qf) {
+  if (v.zn_by_consumers) {
+    // the consumer warps form these scores on the tensor cores
+  } else if (v.qf) {
     // one dot product per thread and turn, operands in shared memory; the element order is rotated by the lane
     // so that the 32 lanes of a warp (different keys, same offset) hit different banks
     for (int w = ptid; w < M * nb; w += kMqPolicyThreads) {
@@ -393,6 +423,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
     PolicyView v;
     v.z = sm.z; v.Bp = Bp; v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok; v.sel = sm.sel;
     v.knew = sm.knew; v.vnew = sm.vnew; v.zn = sm.zn; v.qf = nullptr; v.pn = nullptr; v.ctl = sm.ctl;
+    v.nbuf = nullptr; v.stats_full = nullptr; v.zn_by_consumers = false;
     v.p_ready = sm.p_ready;
     v.policy_done = sm.policy_done;
     multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
@@ -555,8 +586,9 @@ struct MultiTcSmem {
   float *mkey;
   signed char *newtok;
   SelectScratch *sel;
-  float *knew, *vnew, *zn, *pn, *qf;
-  uint64_t *full, *empty, *p_ready, *policy_done;
+  int *nbuf;   // [Bp] Count array of the unit (s and q are staged in vkey and mkey)
+  float *vnew, *zn, *pn;
+  uint64_t *full, *empty, *p_ready, *policy_done, *stats_full;
   int *ctl;
 };
 
@@ -567,10 +599,10 @@ __host__ __device__ inline size_t multi_tc_row_stride(int B) { return align_up((
 __host__ __device__ inline size_t multi_tc_smem_bytes(int B, int stages, int M, int nb) {
   const size_t Bp = multi_tc_row_stride(B);
   size_t b = (size_t)stages * kMqTile;
-  b += (size_t)M * Bp * 4 + 2 * Bp * 4 + Bp;
+  b += (size_t)M * Bp * 4 + 3 * Bp * 4 + Bp;
   b += sizeof(SelectScratch);
-  b += (2 * (size_t)nb + (size_t)M) * 128 * 4 + 2 * (size_t)M * nb * 4;
-  b = align_up(b, 8) + (2 * (size_t)stages + 2) * 8 + 64 * 4;
+  b += (size_t)nb * 128 * 4 + 2 * (size_t)M * nb * 4;
+  b = align_up(b, 8) + (2 * (size_t)stages + 3) * 8 + 64 * 4;
   return b + 1024;
 }
 
@@ -582,18 +614,18 @@ __device__ inline MultiTcSmem multi_tc_carve(char *raw, int B, int stages, int M
   m.z = (float *)p; p += (size_t)M * Bp * 4;
   m.vkey = (uint32_t *)p; p += Bp * 4;
   m.mkey = (float *)p; p += Bp * 4;
+  m.nbuf = (int *)p; p += Bp * 4;
   m.newtok = (signed char *)p; p += Bp;
   m.sel = (SelectScratch *)p; p += sizeof(SelectScratch);
-  m.knew = (float *)p; p += (size_t)nb * 128 * 4;
   m.vnew = (float *)p; p += (size_t)nb * 128 * 4;
   m.zn = (float *)p; p += (size_t)M * nb * 4;
   m.pn = (float *)p; p += (size_t)M * nb * 4;
-  m.qf = (float *)p; p += (size_t)M * 128 * 4;
   p = smem_align(p, 8);
   m.full = (uint64_t *)p; p += stages * 8;
   m.empty = (uint64_t *)p; p += stages * 8;
   m.p_ready = (uint64_t *)p; p += 8;
   m.policy_done = (uint64_t *)p; p += 8;
+  m.stats_full = (uint64_t *)p; p += 8;
   m.ctl = (int *)p;
   return m;
 }
@@ -646,6 +678,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
     for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kMqConsumerWarps); }
     mbar_init(sm.p_ready, kMqConsumerWarps);
     mbar_init(sm.policy_done, 1);
+    mbar_init(sm.stats_full, 1);
     sm.ctl[0] = 0;
     mbar_init_fence();
   }
@@ -658,10 +691,22 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
   if (need < 0) need = 0;
   const int live1 = live0 - need + nb;
   const int n_tiles = (live1 + kTileRows - 1) / kTileRows;
+  // The statistics the selection reads come in by bulk copy ahead of the K tiles (plain loads would queue behind
+  // the tile stream); needs 16-byte aligned unit offsets, i.e. B a multiple of 4 and aligned arrays.
+  const bool stats_by_tma =
+      need > 0 && (B & 3) == 0 &&
+      ((reinterpret_cast<uintptr_t>(p.s) | reinterpret_cast<uintptr_t>(p.q) | reinterpret_cast<uintptr_t>(p.n)) & 15) == 0;
   __syncthreads();
 
   if (warp == kMqProducerWarp) {
     if (lane == 0) {
+      if (stats_by_tma) {
+        const uint32_t bytes = (uint32_t)align_up((size_t)live0 * 4, 16);  // B % 4 == 0: stays inside the unit
+        mbar_expect_tx(sm.stats_full, 3 * bytes);
+        bulk_g2s(sm.vkey, p.s + (size_t)u * B, bytes, sm.stats_full);
+        bulk_g2s(sm.mkey, p.q + (size_t)u * B, bytes, sm.stats_full);
+        bulk_g2s(sm.nbuf, p.n + (size_t)u * B, bytes, sm.stats_full);
+      }
       for (int g = 0; g < 2 * n_tiles; ++g) {
         const int st = g % stages;
         if (g >= stages) mbar_wait(&sm.empty[st], ((g / stages) - 1) & 1, abort_flag, p.status);
@@ -680,7 +725,8 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
   if (warp >= kMqPolicyWarp0) {
     PolicyView v;
     v.z = sm.z; v.Bp = Bp; v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok; v.sel = sm.sel;
-    v.knew = sm.knew; v.vnew = sm.vnew; v.zn = sm.zn; v.qf = sm.qf; v.pn = sm.pn; v.ctl = sm.ctl;
+    v.knew = nullptr; v.vnew = sm.vnew; v.zn = sm.zn; v.qf = nullptr; v.pn = sm.pn; v.ctl = sm.ctl;
+    v.nbuf = sm.nbuf; v.stats_full = stats_by_tma ? sm.stats_full : nullptr; v.zn_by_consumers = true;
     v.p_ready = sm.p_ready;
     v.policy_done = sm.policy_done;
     multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
@@ -731,7 +777,29 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
     if (lane == 0) mbar_arrive(&sm.empty[st]);
   }
 
-  // scores of the new tokens from k_new, with the causal mask inside a block
+  // scores of the queries against the new tokens, from k_new: Zn[16 x 8] per warp, one warp per 8 new tokens
+  if (warp * 8 < nb) {
+    const T *Kn = (const T *)p.k_new + (size_t)u * p.kv_ustride * D;
+    const int jn = warp * 8 + g;  // the new token whose key this thread holds fragments of
+    float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      const int k0 = s * 16 + tq * 2;
+      const uint32_t b0 = jn < nb ? *reinterpret_cast<const uint32_t *>(Kn + (size_t)jn * D + k0) : 0u;
+      const uint32_t b1 = jn < nb ? *reinterpret_cast<const uint32_t *>(Kn + (size_t)jn * D + k0 + 8) : 0u;
+      mma_bf16_16816(c, qa[s], b0, b1);
+    }
+    const int j0 = warp * 8 + tq * 2;
+    if (row_lo) {
+      if (j0 < nb) sm.zn[g * nb + j0] = c[0] * zscale;
+      if (j0 + 1 < nb) sm.zn[g * nb + j0 + 1] = c[1] * zscale;
+    }
+    if (row_hi) {
+      if (j0 < nb) sm.zn[(g + 8) * nb + j0] = c[2] * zscale;
+      if (j0 + 1 < nb) sm.zn[(g + 8) * nb + j0 + 1] = c[3] * zscale;
+    }
+  }
+  // ... placed into the score matrix with the causal mask inside a block, once the target slots are known
   mbar_wait(sm.policy_done, 0, abort_flag, p.status);
   named_bar_sync(kMqBarConsumers, kMqConsumers);
   for (int w = tid; w < M * nb; w += kMqConsumers) {
