@@ -112,6 +112,7 @@ struct PolicyView {
   // nbuf with bulk copies that complete on stats_full (the keys are then formed in place), and the consumer warps
   // compute the new tokens' scores themselves, so the policy warps stage only the new values.
   int *nbuf;
+  int *posbuf;  // the unit's positions as they were before the step (with stats_full)
   uint64_t *stats_full;
   bool zn_by_consumers;
 };
@@ -133,6 +134,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
   const float *gs = p.s + unit_st, *gq = p.q + unit_st;
   const int *gn = p.n + unit_st;
   int *gpos = p.pos + unit_st;
+  const int *opos = v.stats_full ? v.posbuf : gpos;  // positions before the step (shared-memory copy if staged)
   for (int j = ptid; j < live1; j += kMqPolicyThreads) v.newtok[j] = -1;
   {  // new keys / values (and the queries) as fp32 in shared memory, 16-byte loads issued back to back
     constexpr int kEPC = Elem<T>::kPerChunk;
@@ -167,44 +169,52 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     // the rule of Sec. 4.3 applied `need` times on frozen statistics = one pass: the tokens outside the scope
     // (the live0 - m last in (variance, position) order) never enter it, so the `need` first of the scope in
     // (mean, position) order leave
+    uint32_t k_and = 0xffffffffu, k_or = 0u;
     if (v.stats_full) {  // s, q, n sit in vkey, mkey, nbuf: form the keys in place
       mbar_wait(v.stats_full, 0, abort_flag, p.status);
 #pragma unroll 8
       for (int j = ptid; j < live0; j += kMqPolicyThreads) {
         const float sj = __uint_as_float(v.vkey[j]), qj = v.mkey[j];
         const int nj = v.nbuf[j];
-        v.vkey[j] = variance_key_fast(sj, qj, nj);
+        const uint32_t vk = variance_key_fast(sj, qj, nj);
+        v.vkey[j] = vk;
         v.mkey[j] = mean_fast(sj, nj);
+        k_and &= vk;
+        k_or |= vk;
       }
     } else {
 #pragma unroll 8
       for (int j = ptid; j < live0; j += kMqPolicyThreads) {
         const float sj = gs[j], qj = gq[j];
         const int nj = gn[j];
-        v.vkey[j] = variance_key_fast(sj, qj, nj);
+        const uint32_t vk = variance_key_fast(sj, qj, nj);
+        v.vkey[j] = vk;
         v.mkey[j] = mean_fast(sj, nj);
+        k_and &= vk;
+        k_or |= vk;
       }
     }
-    named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+    group_and_or(k_and, k_or, *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy);  // publishes vkey / mkey too
     const int m = scope_size(live0, p.r, p.scope_mode);
     uint32_t Tv = 0xffffffffu;
     int Pv = 0x7fffffff;
     uint32_t rank, ties;
     if (m < live0) {
       Tv = radix_select<uint32_t>([&](int j) { return v.vkey[j]; }, [&](int) { return true; }, live0,
-                                  (uint32_t)(m - 1), *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &rank, &ties);
+                                  (uint32_t)(m - 1), *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &rank, &ties,
+                                  k_and, k_or);
       if (ties != rank + 1) {
         uint32_t r2, t2;
-        Pv = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)gpos[j]; },
+        Pv = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)opos[j]; },
                                          [&](int j) { return v.vkey[j] == Tv; }, live0, rank, *v.sel, ptid,
                                          kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
       }
     }
     auto in_scope = [&](int j) {
       const uint32_t k = v.vkey[j];
-      return k < Tv || (k == Tv && (Pv == 0x7fffffff || gpos[j] <= Pv));
+      return k < Tv || (k == Tv && (Pv == 0x7fffffff || opos[j] <= Pv));
     };
-    int *cnt = v.ctl + 20, *list = v.ctl + 24;  // freed slots, unordered
+    int *list = v.ctl + 24;  // freed slots, in the order they were chosen
     if (need == 1) {
       // one victim: the in-scope token first in (mean, position) order
       float bm = INFINITY;
@@ -213,9 +223,9 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
         if (!in_scope(j)) continue;
         const float mean = v.mkey[j];
         if (mean < bm) { bm = mean; bs = j; }
-        else if (mean == bm && bs >= 0 && gpos[j] < gpos[bs]) bs = j;
+        else if (mean == bm && bs >= 0 && opos[j] < opos[bs]) bs = j;
       }
-      int bp = bs >= 0 ? gpos[bs] : 0x7fffffff;
+      int bp = bs >= 0 ? opos[bs] : 0x7fffffff;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
         const float om = __shfl_xor_sync(0xffffffffu, bm, o);
@@ -236,33 +246,82 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
         tgt[0] = bs;
       }
     } else {
-      const uint32_t Tm = radix_select<uint32_t>([&](int j) { return __float_as_uint(v.mkey[j]); }, in_scope, live0,
-                                                 (uint32_t)(need - 1), *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy,
-                                                 &rank, &ties);
-      int Pm = 0x7fffffff;
-      if (ties != rank + 1) {
-        uint32_t r2, t2;
-        Pm = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)gpos[j]; },
-                                         [&](int j) { return in_scope(j) && __float_as_uint(v.mkey[j]) == Tm; },
-                                         live0, rank, *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
-      }
-      // collect the freed slots (at most 16), then order them by slot index
-      if (ptid == 0) *cnt = 0;
+      // the `need` (at most 16) in-scope tokens first in (mean, position) order; out-of-scope tokens are masked
+      // once, which leaves a plain selection over mkey
+      for (int j = ptid; j < live0; j += kMqPolicyThreads)
+        if (!in_scope(j)) v.mkey[j] = INFINITY;
       named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      for (int j = ptid; j < live0; j += kMqPolicyThreads) {
-        if (!in_scope(j)) continue;
-        const uint32_t k = __float_as_uint(v.mkey[j]);
-        if (k < Tm || (k == Tm && (Pm == 0x7fffffff || gpos[j] <= Pm))) {
-          const int at = atomicAdd(cnt, 1);
-          if (at < kMqMaxQ) list[at] = j;
+      if (need <= 4) {
+        // few victims: one argmin after the other (about 2 000 cycles each, against ~20 000 for the threshold
+        // search below); a chosen token is masked by the thread that scans it
+        for (int e = 0; e < need; ++e) {
+          float bm = INFINITY;
+          int bs = -1;
+#pragma unroll 4
+          for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+            const float mean = v.mkey[j];
+            if (mean < bm) { bm = mean; bs = j; }
+            else if (mean == bm && bs >= 0 && opos[j] < opos[bs]) bs = j;
+          }
+          // a thread's candidates come in increasing slot order but ties go to the lower *position*
+          int bp = bs >= 0 ? opos[bs] : 0x7fffffff;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, bm, o);
+            const int op = __shfl_xor_sync(0xffffffffu, bp, o);
+            const int os = __shfl_xor_sync(0xffffffffu, bs, o);
+            if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+          }
+          float *rm = v.sel->red_mean + (e & 1) * 4;  // double-buffered: one barrier per round
+          int *rp = v.sel->red_pos + (e & 1) * 4, *rs = v.sel->red_slot + (e & 1) * 4;
+          if (plane == 0) { rm[pwarp] = bm; rp[pwarp] = bp; rs[pwarp] = bs; }
+          named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+          bm = rm[0]; bp = rp[0]; bs = rs[0];
+#pragma unroll
+          for (int w = 1; w < kMqPolicyThreads / 32; ++w) {
+            const float om = rm[w];
+            const int op = rp[w], os = rs[w];
+            if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+          }
+          if (bs < 0) {
+            if (ptid == 0) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
+            bs = e;  // keeps the slots distinct; the step's results are void
+          }
+          if (ptid == 0) list[e] = bs;
+          if ((bs % kMqPolicyThreads) == ptid) v.mkey[bs] = INFINITY;  // only this thread ever scans slot bs
+        }
+      } else {
+        // many victims: the need-th smallest mean by radix select, then one pass that collects everything up to it
+        const uint32_t Tm = radix_select<uint32_t>([&](int j) { return __float_as_uint(v.mkey[j]); },
+                                                   [&](int) { return true; }, live0, (uint32_t)(need - 1), *v.sel, ptid,
+                                                   kMqPolicyThreads, kMqBarPolicy, &rank, &ties);
+        int Pm = 0x7fffffff;
+        if (ties != rank + 1) {
+          uint32_t r2, t2;
+          Pm = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)opos[j]; },
+                                           [&](int j) { return __float_as_uint(v.mkey[j]) == Tm; }, live0, rank,
+                                           *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
+        }
+        int *cnt = v.ctl + 20;
+        if (ptid == 0) *cnt = 0;
+        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+        for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+          const uint32_t k = __float_as_uint(v.mkey[j]);
+          if (k < 0x7f800000u && (k < Tm || (k == Tm && (Pm == 0x7fffffff || opos[j] <= Pm)))) {
+            const int at = atomicAdd(cnt, 1);
+            if (at < kMqMaxQ) list[at] = j;
+          }
+        }
+        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+        if (ptid == 0 && *cnt != need) {  // only after corrupt statistics
+          atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
+          for (int x = *cnt < 0 ? 0 : *cnt; x < need; ++x) list[x] = x;
         }
       }
       named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      const int found = *cnt < kMqMaxQ ? *cnt : kMqMaxQ;
-      if (ptid == 0 && *cnt != need) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
-      if (ptid < found) {
+      if (ptid < need) {  // order the freed slots by slot index
         int rk = 0;
-        for (int x = 0; x < found; ++x) rk += list[x] < list[ptid];
+        for (int x = 0; x < need; ++x) rk += list[x] < list[ptid];
         if (rk < nb) tgt[rk] = list[ptid];
       }
     }
@@ -274,7 +333,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     int slot = tgt[ptid];
     if (slot < 0 || slot >= B) slot = 0;  // only after corrupt statistics (status bit set above)
     p.ev_slot[(size_t)u * nb + ptid] = ptid < need ? slot : -1;
-    if (p.ev_pos) p.ev_pos[(size_t)u * nb + ptid] = ptid < need ? gpos[slot] : -1;
+    if (p.ev_pos) p.ev_pos[(size_t)u * nb + ptid] = ptid < need ? opos[slot] : -1;
     v.newtok[slot] = (signed char)ptid;
     gpos[slot] = t_new + ptid;
   }
@@ -423,7 +482,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
     PolicyView v;
     v.z = sm.z; v.Bp = Bp; v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok; v.sel = sm.sel;
     v.knew = sm.knew; v.vnew = sm.vnew; v.zn = sm.zn; v.qf = nullptr; v.pn = nullptr; v.ctl = sm.ctl;
-    v.nbuf = nullptr; v.stats_full = nullptr; v.zn_by_consumers = false;
+    v.nbuf = nullptr; v.posbuf = nullptr; v.stats_full = nullptr; v.zn_by_consumers = false;
     v.p_ready = sm.p_ready;
     v.policy_done = sm.policy_done;
     multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
@@ -587,6 +646,7 @@ struct MultiTcSmem {
   signed char *newtok;
   SelectScratch *sel;
   int *nbuf;   // [Bp] Count array of the unit (s and q are staged in vkey and mkey)
+  int *posbuf; // [Bp] positions of the unit before the step
   float *vnew, *zn, *pn;
   uint64_t *full, *empty, *p_ready, *policy_done, *stats_full;
   int *ctl;
@@ -599,7 +659,7 @@ __host__ __device__ inline size_t multi_tc_row_stride(int B) { return align_up((
 __host__ __device__ inline size_t multi_tc_smem_bytes(int B, int stages, int M, int nb) {
   const size_t Bp = multi_tc_row_stride(B);
   size_t b = (size_t)stages * kMqTile;
-  b += (size_t)M * Bp * 4 + 3 * Bp * 4 + Bp;
+  b += (size_t)M * Bp * 4 + 4 * Bp * 4 + Bp;
   b += sizeof(SelectScratch);
   b += (size_t)nb * 128 * 4 + 2 * (size_t)M * nb * 4;
   b = align_up(b, 8) + (2 * (size_t)stages + 3) * 8 + 64 * 4;
@@ -615,6 +675,7 @@ __device__ inline MultiTcSmem multi_tc_carve(char *raw, int B, int stages, int M
   m.vkey = (uint32_t *)p; p += Bp * 4;
   m.mkey = (float *)p; p += Bp * 4;
   m.nbuf = (int *)p; p += Bp * 4;
+  m.posbuf = (int *)p; p += Bp * 4;
   m.newtok = (signed char *)p; p += Bp;
   m.sel = (SelectScratch *)p; p += sizeof(SelectScratch);
   m.vnew = (float *)p; p += (size_t)nb * 128 * 4;
@@ -695,17 +756,19 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
   // the tile stream); needs 16-byte aligned unit offsets, i.e. B a multiple of 4 and aligned arrays.
   const bool stats_by_tma =
       need > 0 && (B & 3) == 0 &&
-      ((reinterpret_cast<uintptr_t>(p.s) | reinterpret_cast<uintptr_t>(p.q) | reinterpret_cast<uintptr_t>(p.n)) & 15) == 0;
+      ((reinterpret_cast<uintptr_t>(p.s) | reinterpret_cast<uintptr_t>(p.q) | reinterpret_cast<uintptr_t>(p.n) |
+        reinterpret_cast<uintptr_t>(p.pos)) & 15) == 0;
   __syncthreads();
 
   if (warp == kMqProducerWarp) {
     if (lane == 0) {
       if (stats_by_tma) {
         const uint32_t bytes = (uint32_t)align_up((size_t)live0 * 4, 16);  // B % 4 == 0: stays inside the unit
-        mbar_expect_tx(sm.stats_full, 3 * bytes);
+        mbar_expect_tx(sm.stats_full, 4 * bytes);
         bulk_g2s(sm.vkey, p.s + (size_t)u * B, bytes, sm.stats_full);
         bulk_g2s(sm.mkey, p.q + (size_t)u * B, bytes, sm.stats_full);
         bulk_g2s(sm.nbuf, p.n + (size_t)u * B, bytes, sm.stats_full);
+        bulk_g2s(sm.posbuf, p.pos + (size_t)u * B, bytes, sm.stats_full);
       }
       for (int g = 0; g < 2 * n_tiles; ++g) {
         const int st = g % stages;
@@ -726,7 +789,8 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
     PolicyView v;
     v.z = sm.z; v.Bp = Bp; v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok; v.sel = sm.sel;
     v.knew = nullptr; v.vnew = sm.vnew; v.zn = sm.zn; v.qf = nullptr; v.pn = sm.pn; v.ctl = sm.ctl;
-    v.nbuf = sm.nbuf; v.stats_full = stats_by_tma ? sm.stats_full : nullptr; v.zn_by_consumers = true;
+    v.nbuf = sm.nbuf; v.posbuf = sm.posbuf; v.stats_full = stats_by_tma ? sm.stats_full : nullptr;
+    v.zn_by_consumers = true;
     v.p_ready = sm.p_ready;
     v.policy_done = sm.policy_done;
     multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);

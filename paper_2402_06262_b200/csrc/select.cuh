@@ -32,14 +32,26 @@ __device__ __forceinline__ void smem_red_add(uint32_t *addr, uint32_t v) {
 // KeyT (32 or 64 bits).  Called by all `nthreads` threads that synchronise on named barrier `bar_id`.
 // *rank_in_ties: how many elements equal to the result precede the k-th in a stable order (so
 // rank_in_ties + 1 of them are among the k+1 smallest); *n_ties: how many elements equal the result.
+// `common` (optional): bits on which all selected keys are known to agree, as (AND of the keys, OR of the keys);
+// the digits above the first disagreeing one are then skipped.
 template <typename KeyT, typename KeyF, typename PredF>
 __device__ __forceinline__ KeyT radix_select(KeyF key, PredF pred, int n, uint32_t k, SelectScratch &sc, int tid,
-                                             int nthreads, int bar_id, uint32_t *rank_in_ties, uint32_t *n_ties) {
+                                             int nthreads, int bar_id, uint32_t *rank_in_ties, uint32_t *n_ties,
+                                             KeyT all_and = 0, KeyT all_or = ~(KeyT)0) {
   KeyT prefix = 0, mask = 0;
   uint32_t kk = k;
   const int lane = tid & 31;
+  int shift0 = (int)sizeof(KeyT) * 8 - 8;
+  {
+    const KeyT diff = all_and ^ all_or;  // a set bit: the keys may differ there
+    while (shift0 > 0 && (diff >> shift0) == 0) shift0 -= 8;
+    if (shift0 < (int)sizeof(KeyT) * 8 - 8) {
+      mask = ~(KeyT)0 << (shift0 + 8);
+      prefix = all_and & mask;
+    }
+  }
 #pragma unroll 1
-  for (int shift = (int)sizeof(KeyT) * 8 - 8; shift >= 0; shift -= 8) {
+  for (int shift = shift0; shift >= 0; shift -= 8) {
     for (int i = tid; i < 256; i += nthreads) sc.hist[i] = 0;
     named_bar_sync(bar_id, nthreads);
 #pragma unroll 4
@@ -102,6 +114,18 @@ __device__ __forceinline__ uint32_t variance_key_fast(float s, float q, int n) {
 
 __device__ __forceinline__ float mean_fast(float s, int n) { return __fdiv_rn(s, (float)n); }
 
+// AND and OR of a per-thread pair over the whole group (in place); every thread gets the group's values.
+__device__ __forceinline__ void group_and_or(uint32_t &k_and, uint32_t &k_or, SelectScratch &sc, int tid, int nthreads,
+                                             int bar_id) {
+  k_and = __reduce_and_sync(0xffffffffu, k_and);
+  k_or = __reduce_or_sync(0xffffffffu, k_or);
+  const int warp = tid >> 5, nwarps = nthreads >> 5;
+  if ((tid & 31) == 0) { sc.red_pos[warp] = (int)k_and; sc.red_slot[warp] = (int)k_or; }
+  named_bar_sync(bar_id, nthreads);
+  for (int w = 0; w < nwarps; ++w) { k_and &= (uint32_t)sc.red_pos[w]; k_or |= (uint32_t)sc.red_slot[w]; }
+  named_bar_sync(bar_id, nthreads);  // the scratch may be reused right away
+}
+
 // Victim slot among slots [0, live) given scope size m (1 <= m <= live).  s, q, n, pos are the unit's
 // statistics in GLOBAL memory (each read once, coalesced; positions only where a tie has to be broken);
 // vkey[live] and mkey[live] are shared-memory scratch.  Returns -1 if no slot qualifies (NaN statistics).
@@ -110,20 +134,24 @@ __device__ __forceinline__ float mean_fast(float s, int n) { return __fdiv_rn(s,
 __device__ __forceinline__ int group_select_victim(const float *s, const float *q, const int *n, const int *pos,
                                                    int live, int m, uint32_t *vkey, float *mkey, SelectScratch &sc,
                                                    int tid, int nthreads, int bar_id) {
+  uint32_t k_and = 0xffffffffu, k_or = 0u;
 #pragma unroll 4
   for (int j = tid; j < live; j += nthreads) {
     const float sj = s[j], qj = q[j];
     const int nj = n[j];
-    vkey[j] = variance_key_fast(sj, qj, nj);
+    const uint32_t vk = variance_key_fast(sj, qj, nj);
+    vkey[j] = vk;
     mkey[j] = mean_fast(sj, nj);
+    k_and &= vk;
+    k_or |= vk;
   }
-  named_bar_sync(bar_id, nthreads);
+  group_and_or(k_and, k_or, sc, tid, nthreads, bar_id);  // also the barrier that publishes vkey / mkey
   uint32_t T = 0xffffffffu;
   int P = 0x7fffffff;
   if (m < live) {
     uint32_t rank, ties;
     T = radix_select<uint32_t>([&](int j) { return vkey[j]; }, [&](int) { return true; }, live, (uint32_t)(m - 1),
-                               sc, tid, nthreads, bar_id, &rank, &ties);
+                               sc, tid, nthreads, bar_id, &rank, &ties, k_and, k_or);
     if (ties != rank + 1) {  // only some of the tokens tied at the threshold are in scope: lowest positions
       uint32_t r2, t2;
       P = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)pos[j]; }, [&](int j) { return vkey[j] == T; },
