@@ -36,6 +36,7 @@ struct DecodeParams {
   float *lse;
   int *ev_slot, *ev_pos;
   int B, r, scope_mode, order, stages;
+  int stage_stats;      // shared memory has room for a copy of the Count array (see stats_staged in the kernel)
   int policy;           // roco_policy
   const unsigned *rnd;  // [U] random draws (ROCO_POLICY_RANDOM)
   float scale;
@@ -51,25 +52,27 @@ struct DecodeSmem {
   uint64_t *full, *empty;  // ring barriers
   uint64_t *p_ready;       // consumers have left the probabilities in shared memory
   uint64_t *policy_done;   // victim chosen, new K/V written
+  uint64_t *stats_full;    // the unit's s, q, n have landed in vkey, mkey, nbuf (bulk copies ahead of the K tiles)
+  int *nbuf;
   int *ctl;                // [0] abort flag, [1] slot of the new token
   float *znew;             // score of the new token (EVICT_FIRST)
 };
 
 template <int TILE>
-__host__ __device__ inline size_t decode_smem_bytes(int B, int d, int stages) {
+__host__ __device__ inline size_t decode_smem_bytes(int B, int d, int stages, int stage_stats) {
   const size_t Bp = align_up((size_t)B, 4);
   size_t b = (size_t)stages * TILE;
-  b += 3 * Bp * 4;  // z, vkey, mkey
+  b += (stage_stats ? 4 : 3) * Bp * 4;  // z, vkey, mkey (, nbuf)
   b += sizeof(SelectScratch);
   b += (size_t)(2 + kConsumerWarps) * d * 4;  // qf, vnew, outred
   b += 64 * 4;                                // red
-  b += (2 * (size_t)stages + 2) * sizeof(uint64_t);
+  b += (2 * (size_t)stages + 3) * sizeof(uint64_t);
   b += 8 * 4;
   return b + 128;  // slack for aligning the base
 }
 
 template <int TILE>
-__device__ inline DecodeSmem carve(char *raw, int B, int d, int stages) {
+__device__ inline DecodeSmem carve(char *raw, int B, int d, int stages, int stage_stats) {
   DecodeSmem m;
   char *p = smem_align(raw, 128);
   const size_t Bp = align_up((size_t)B, 4);
@@ -77,6 +80,7 @@ __device__ inline DecodeSmem carve(char *raw, int B, int d, int stages) {
   m.z = (float *)p; p += Bp * 4;
   m.vkey = (uint32_t *)p; p += Bp * 4;
   m.mkey = (float *)p; p += Bp * 4;
+  m.nbuf = (int *)p; p += stage_stats ? Bp * 4 : 0;
   m.sel = (SelectScratch *)p; p += sizeof(SelectScratch);
   m.qf = (float *)p; p += d * 4;
   m.vnew = (float *)p; p += d * 4;
@@ -86,6 +90,7 @@ __device__ inline DecodeSmem carve(char *raw, int B, int d, int stages) {
   m.empty = (uint64_t *)p; p += stages * sizeof(uint64_t);
   m.p_ready = (uint64_t *)p; p += sizeof(uint64_t);
   m.policy_done = (uint64_t *)p; p += sizeof(uint64_t);
+  m.stats_full = (uint64_t *)p; p += sizeof(uint64_t);
   m.ctl = (int *)p; p += 4 * 4;
   m.znew = (float *)p;
   return m;
@@ -123,7 +128,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
   static_assert(kLanesPerRow <= 32 && kLoads >= 1, "tile shape");
 
   extern __shared__ char smem_raw[];
-  const DecodeSmem sm = carve<TILE>(smem_raw, p.B, D, p.stages);
+  const DecodeSmem sm = carve<TILE>(smem_raw, p.B, D, p.stages, p.stage_stats);
   volatile int *abort_flag = sm.ctl;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -137,6 +142,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kConsumerWarps); }
     mbar_init(sm.p_ready, kConsumerWarps);
     mbar_init(sm.policy_done, 1);
+    mbar_init(sm.stats_full, 1);
     sm.ctl[0] = 0;
     mbar_init_fence();
   }
@@ -150,11 +156,24 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
   const int live_att = evict_first ? (full ? B : live0 + 1) : live0;  // slots the query attends over
   const int live_new = full ? B : live0 + 1;
   const int n_tiles = (live_att + kTileRows - 1) / kTileRows;
+  // The statistics the selection reads are fetched by bulk copies issued ahead of the K tiles (plain loads would
+  // queue behind the tile stream for microseconds).  Only where the selection sees the statistics as they stand
+  // at the start of the step, and the unit's arrays start on 16-byte boundaries.
+  const bool stats_staged =
+      p.stage_stats && full && evict_first && p.policy == ROCO_POLICY_ROCO && (B & 3) == 0 &&
+      ((reinterpret_cast<uintptr_t>(p.s) | reinterpret_cast<uintptr_t>(p.q) | reinterpret_cast<uintptr_t>(p.n)) & 15) == 0;
   __syncthreads();
 
   if (warp == kProducerWarp) {
-    // ------------------------------------------------------------ producer: K tiles, then V tiles
+    // ------------------------------------------------------------ producer: statistics, K tiles, then V tiles
     if (lane == 0) {
+      if (stats_staged) {
+        const uint32_t bytes = (uint32_t)B * 4;
+        mbar_expect_tx(sm.stats_full, 3 * bytes);
+        bulk_g2s(sm.vkey, p.s + unit_st, bytes, sm.stats_full);
+        bulk_g2s(sm.mkey, p.q + unit_st, bytes, sm.stats_full);
+        bulk_g2s(sm.nbuf, p.n + unit_st, bytes, sm.stats_full);
+      }
       for (int g = 0; g < 2 * n_tiles; ++g) {
         const int st = g % stages;
         if (g >= stages) mbar_wait(&sm.empty[st], ((g / stages) - 1) & 1, abort_flag, p.status);
@@ -219,7 +238,24 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
       const int *gn = p.n + unit_st, *gpos = p.pos + unit_st;
       if (p.policy == ROCO_POLICY_ROCO) {
         const int m = scope_size(B, p.r, p.scope_mode);
-        e = group_select_victim(gs, gq, gn, gpos, B, m, sm.vkey, sm.mkey, *sm.sel, ptid, kPolicyThreads, kBarPolicy);
+        if (stats_staged) {  // s, q, n sit in vkey, mkey, nbuf: form the keys in place
+          mbar_wait(sm.stats_full, 0, abort_flag, p.status);
+          uint32_t k_and = 0xffffffffu, k_or = 0u;
+#pragma unroll 4
+          for (int j = ptid; j < B; j += kPolicyThreads) {
+            const float sj = __uint_as_float(sm.vkey[j]);
+            const uint32_t vk = variance_key_fast(sj, sm.mkey[j], sm.nbuf[j]);
+            sm.mkey[j] = mean_fast(sj, sm.nbuf[j]);
+            sm.vkey[j] = vk;
+            k_and &= vk;
+            k_or |= vk;
+          }
+          e = group_select_from_keys(gpos, B, m, sm.vkey, sm.mkey, k_and, k_or, *sm.sel, ptid, kPolicyThreads,
+                                     kBarPolicy);
+        } else {
+          e = group_select_victim(gs, gq, gn, gpos, B, m, sm.vkey, sm.mkey, *sm.sel, ptid, kPolicyThreads,
+                                  kBarPolicy);
+        }
       } else if (p.policy == ROCO_POLICY_RANDOM) {
         e = (int)(p.rnd[u] % (unsigned)B);
       } else {
@@ -396,7 +432,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
 
 template <typename T, int D, int TILE>
 static cudaError_t launch_decode_t(const DecodeParams &p, int U, cudaStream_t stream) {
-  const size_t smem = decode_smem_bytes<TILE>(p.B, D, p.stages);
+  const size_t smem = decode_smem_bytes<TILE>(p.B, D, p.stages, p.stage_stats);
   cudaError_t err = cudaFuncSetAttribute(decode_step_kernel<T, D, TILE>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
@@ -408,20 +444,39 @@ static cudaError_t launch_decode_t(const DecodeParams &p, int U, cudaStream_t st
 // share an SM; budgets too large for that fall back to 8 KiB tiles.
 constexpr int kMaxCtasPerSm = 3;
 
+// Stages of the tile ring (3..6, 0 = does not fit) for the largest number of CTAs per SM that fits; *ctas_out
+// gets that number.
 template <int TILE>
-static int pick_stages(int B, int d) {
+static int pick_stages(int B, int d, int stage_stats, int *ctas_out) {
   const size_t per_sm = 227 * 1024;
   for (int ctas = kMaxCtasPerSm; ctas >= 1; --ctas) {
     for (int st = 6; st >= 3; --st)
-      if ((decode_smem_bytes<TILE>(B, d, st) + 1024) * ctas <= per_sm) return st;
+      if ((decode_smem_bytes<TILE>(B, d, st, stage_stats) + 1024) * ctas <= per_sm) {
+        *ctas_out = ctas;
+        return st;
+      }
   }
+  *ctas_out = 0;
   return 0;
+}
+
+template <typename T, int D, int TILE>
+static bool try_launch(DecodeParams &p, int U, cudaStream_t stream, cudaError_t *err) {
+  // the copy of the Count array is kept only if it costs no CTA per SM
+  int ctas0, ctas1;
+  const int st0 = pick_stages<TILE>(p.B, D, 0, &ctas0), st1 = pick_stages<TILE>(p.B, D, 1, &ctas1);
+  if (st0 == 0) return false;
+  p.stage_stats = (st1 > 0 && ctas1 == ctas0) ? 1 : 0;
+  p.stages = p.stage_stats ? st1 : st0;
+  *err = launch_decode_t<T, D, TILE>(p, U, stream);
+  return true;
 }
 
 template <typename T, int D>
 static cudaError_t launch_decode_td(DecodeParams &p, int U, cudaStream_t stream) {
-  if ((p.stages = pick_stages<16384>(p.B, D)) > 0) return launch_decode_t<T, D, 16384>(p, U, stream);
-  if ((p.stages = pick_stages<8192>(p.B, D)) > 0) return launch_decode_t<T, D, 8192>(p, U, stream);
+  cudaError_t err;
+  if (try_launch<T, D, 16384>(p, U, stream, &err)) return err;
+  if (try_launch<T, D, 8192>(p, U, stream, &err)) return err;
   return cudaErrorInvalidConfiguration;
 }
 

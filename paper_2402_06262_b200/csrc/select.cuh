@@ -126,26 +126,15 @@ __device__ __forceinline__ void group_and_or(uint32_t &k_and, uint32_t &k_or, Se
   named_bar_sync(bar_id, nthreads);  // the scratch may be reused right away
 }
 
-// Victim slot among slots [0, live) given scope size m (1 <= m <= live).  s, q, n, pos are the unit's
-// statistics in GLOBAL memory (each read once, coalesced; positions only where a tie has to be broken);
-// vkey[live] and mkey[live] are shared-memory scratch.  Returns -1 if no slot qualifies (NaN statistics).
-// Called by the `nthreads` threads (a multiple of 32) that synchronise on named barrier `bar_id`; every one
-// of them gets the same return value.
-__device__ __forceinline__ int group_select_victim(const float *s, const float *q, const int *n, const int *pos,
-                                                   int live, int m, uint32_t *vkey, float *mkey, SelectScratch &sc,
-                                                   int tid, int nthreads, int bar_id) {
-  uint32_t k_and = 0xffffffffu, k_or = 0u;
-#pragma unroll 4
-  for (int j = tid; j < live; j += nthreads) {
-    const float sj = s[j], qj = q[j];
-    const int nj = n[j];
-    const uint32_t vk = variance_key_fast(sj, qj, nj);
-    vkey[j] = vk;
-    mkey[j] = mean_fast(sj, nj);
-    k_and &= vk;
-    k_or |= vk;
-  }
-  group_and_or(k_and, k_or, sc, tid, nthreads, bar_id);  // also the barrier that publishes vkey / mkey
+// Victim slot among slots [0, live) given scope size m (1 <= m <= live), from the keys in shared memory:
+// vkey[j] = variance key, mkey[j] = mean of slot j; (k_and, k_or) = each thread's AND / OR over the variance keys it
+// wrote (combined over the group here, which also publishes the keys).  pos: the unit's positions, read only
+// where a tie has to be broken.  Returns -1 if no slot qualifies (NaN statistics).  Called by the `nthreads`
+// threads (a multiple of 32) that synchronise on named barrier `bar_id`; every one of them gets the same value.
+__device__ __forceinline__ int group_select_from_keys(const int *pos, int live, int m, const uint32_t *vkey,
+                                                      const float *mkey, uint32_t k_and, uint32_t k_or,
+                                                      SelectScratch &sc, int tid, int nthreads, int bar_id) {
+  group_and_or(k_and, k_or, sc, tid, nthreads, bar_id);
   uint32_t T = 0xffffffffu;
   int P = 0x7fffffff;
   if (m < live) {
@@ -188,6 +177,25 @@ __device__ __forceinline__ int group_select_victim(const float *s, const float *
   }
   named_bar_sync(bar_id, nthreads);
   return bs;
+}
+
+// The same with the keys formed here from the unit's statistics s, q, n (any memory; each read once, coalesced).
+// vkey[live] and mkey[live] are shared-memory scratch.
+__device__ __forceinline__ int group_select_victim(const float *s, const float *q, const int *n, const int *pos,
+                                                   int live, int m, uint32_t *vkey, float *mkey, SelectScratch &sc,
+                                                   int tid, int nthreads, int bar_id) {
+  uint32_t k_and = 0xffffffffu, k_or = 0u;
+#pragma unroll 4
+  for (int j = tid; j < live; j += nthreads) {
+    const float sj = s[j], qj = q[j];
+    const int nj = n[j];
+    const uint32_t vk = variance_key_fast(sj, qj, nj);
+    vkey[j] = vk;
+    mkey[j] = mean_fast(sj, nj);
+    k_and &= vk;
+    k_or |= vk;
+  }
+  return group_select_from_keys(pos, live, m, vkey, mkey, k_and, k_or, sc, tid, nthreads, bar_id);
 }
 
 // Slot first in (score asc, position asc) order among the slots [0, live) with eligible(j); -1 if there is none.

@@ -31,10 +31,11 @@ def prefilled(w, L, tally, units):
 
 
 @pytest.mark.parametrize("b", [1, 2, 4, 8, 16])
-@pytest.mark.parametrize("dtype,d,B", [("bf16", 128, 300), ("f32", 64, 128)])
+@pytest.mark.parametrize("dtype,d,B", [("bf16", 128, 300), ("bf16", 128, 302), ("f32", 64, 128)])
 def test_block_steps_fill_then_evict(b, dtype, d, B):
     """Short prompt: the first block steps only fill free slots (some mix freed and free slots), later ones evict
-    b tokens each."""
+    b tokens each.  B = 300 takes the tensor-core kernel with the statistics staged by bulk copy, B = 302 (unit
+    offsets not 16-byte aligned) the same kernel with plain loads, fp32 / d = 64 the CUDA-core kernel."""
     w = W.scaled(W.LLAMA7B_DECODE, S=2, layers=1, heads=3, d=d, dtype=dtype, prompt_lo=B - 21, prompt_hi=B - 21,
                  B=B, r=9)
     tally = Tally()
