@@ -291,6 +291,16 @@ roco_status roco_decode_step_host(roco_cache *cache, const void *q_host, const v
                                   void *attn_out_host, int32_t *evicted_slot_host, int32_t *evicted_pos_host,
                                   void *staging, size_t staging_bytes, void *stream);
 
+/*
+ * Self-test of the bounded waits (the paper has no counterpart: this checks the library's own failure reporting).
+ * Every kernel here waits on shared-memory barriers with a time limit of about two seconds; a wait that runs out
+ * sets ROCO_DEV_WAIT_TIMEOUT in the status word and the kernel carries on to its end instead of hanging.  This
+ * call launches one small CTA that waits on a barrier nothing completes, so that limit is reached on purpose:
+ * afterwards *status has ROCO_DEV_WAIT_TIMEOUT set and *waited_ms (device, may be NULL) holds how long the wait
+ * took.  The kernel occupies one SM for that time and touches no other memory.
+ */
+roco_status roco_selftest_wait_timeout(int32_t *status, int32_t *waited_ms, void *stream);
+
 /* Copies the device status word to *flags_host (synchronises the stream).  Returns ROCO_ERR_STATE
  * when it is non-zero. */
 roco_status roco_device_status(const roco_cache *cache, void *stream, int32_t *flags_host);

@@ -26,7 +26,7 @@ EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes",
            "roco_block_step", "roco_gqa_decode_step", "roco_decode_step_policy",
            "roco_decode_split_workspace_bytes", "roco_decode_step_split", "roco_prefill_blockwise",
            "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status",
-           "roco_prefill_attend_workspace_bytes", "roco_prefill_attend")
+           "roco_prefill_attend_workspace_bytes", "roco_prefill_attend", "roco_selftest_wait_timeout")
 
 
 class RocoError(RuntimeError):
@@ -101,6 +101,8 @@ def lib() -> C.CDLL:
         L.roco_decode_step_host.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                             C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_size_t, C.c_void_p]
+        L.roco_selftest_wait_timeout.restype = C.c_int
+        L.roco_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.roco_device_status.restype = C.c_int
         L.roco_device_status.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p]
         _lib = L
@@ -212,6 +214,14 @@ def roco_prefill_attend(cache: Cache, Q, K, V, lens: Sequence[int], lse, attn_ou
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_prefill_attend")
     return workspace
+
+
+def roco_selftest_wait_timeout(status: torch.Tensor, waited_ms: Optional[torch.Tensor] = None):
+    """Launches the bounded-wait self-test: `status` (int32 [1], device) gets ROCO_DEV_WAIT_TIMEOUT once the
+    kernel's wait has run out (about two seconds); `waited_ms` (int32 [1], device) how long that took."""
+    rc = lib().roco_selftest_wait_timeout(_ptr(status), _ptr(waited_ms), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_selftest_wait_timeout")
 
 
 def roco_decode_step(cache: Cache, q, k_new, v_new, r: int, attn_out, evicted_slot, evicted_pos=None, lse_out=None,

@@ -1,4 +1,6 @@
 // The C ABI of libroco: argument validation on the host, workspace carving, launches.
+#include <nvtx3/nvToolsExt.h>
+
 #include <cstring>
 
 #include "common.cuh"
@@ -7,6 +9,12 @@
 using namespace roco;
 
 namespace {
+
+// A named range around every launching entry point, visible in the timeline of an attached profiler.
+struct NvtxRange {
+  explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+};
 
 constexpr int kMaxB = 8192;
 
@@ -88,6 +96,7 @@ int roco_prefill_uses_tensor_cores(const roco_cache *cache) {
 roco_status roco_prefill(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax, int B,
                          int r, int scope_mode, int count_self, float scale, roco_cache *cache, float *lse_out,
                          float *s_full, float *q_full, void *workspace, size_t workspace_bytes, void *stream) {
+  NvtxRange range("roco_prefill");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
   if (!Q || !K || !V || !lens_host || Lmax < 1 || B != cache->B) return ROCO_ERR_INVALID_ARG;
@@ -134,6 +143,7 @@ size_t roco_prefill_attend_workspace_bytes(const roco_cache *cache) {
 roco_status roco_prefill_attend(const roco_cache *cache, const void *Q, const void *K, const void *V,
                                 const int32_t *lens_host, int Lmax, float scale, const float *lse, void *attn_out,
                                 void *workspace, size_t workspace_bytes, void *stream) {
+  NvtxRange range("roco_prefill_attend");
   if (!cache || !cache->status || cache->S < 1 || cache->G < 1) return ROCO_ERR_INVALID_ARG;
   if (!Q || !K || !V || !lens_host || !lse || !attn_out || Lmax < 1) return ROCO_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
@@ -158,6 +168,7 @@ roco_status roco_prefill_attend(const roco_cache *cache, const void *Q, const vo
 roco_status roco_decode_step(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,
                              int scope_mode, int step_order, float scale, void *attn_out, float *lse_out,
                              int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {
+  NvtxRange range("roco_decode_step");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
   if (!q || !k_new || !v_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
@@ -177,6 +188,7 @@ roco_status roco_decode_step_split(roco_cache *cache, const void *q, const void 
                                    int scope_mode, int splits, float scale, void *attn_out, float *lse_out,
                                    int32_t *evicted_slot, int32_t *evicted_pos, void *workspace,
                                    size_t workspace_bytes, void *stream) {
+  NvtxRange range("roco_decode_step_split");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
   if (!q || !k_new || !v_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
@@ -193,6 +205,7 @@ roco_status roco_decode_step_split(roco_cache *cache, const void *q, const void 
 roco_status roco_decode_step_policy(roco_cache *cache, const void *q, const void *k_new, const void *v_new,
                                     int policy, int r, const uint32_t *rnd, float scale, void *attn_out,
                                     float *lse_out, int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {
+  NvtxRange range("roco_decode_step_policy");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
   if (!q || !k_new || !v_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
@@ -208,6 +221,7 @@ roco_status roco_decode_step_policy(roco_cache *cache, const void *q, const void
 roco_status roco_block_step(roco_cache *cache, const void *Q, const void *K_new, const void *V_new, int b, int r,
                             int scope_mode, float scale, void *attn_out, float *lse_out, int32_t *evicted_slot,
                             int32_t *evicted_pos, void *stream) {
+  NvtxRange range("roco_block_step");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
   if (!Q || !K_new || !V_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
@@ -225,6 +239,7 @@ roco_status roco_block_step(roco_cache *cache, const void *Q, const void *K_new,
 roco_status roco_prefill_blockwise(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax,
                                    int b, int r, float scale, roco_cache *cache, void *attn_out,
                                    int32_t *evicted_slot, void *stream) {
+  NvtxRange range("roco_prefill_blockwise");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
   if (!Q || !K || !V || !lens_host || !attn_out || !evicted_slot || Lmax < 1 || b < 1) return ROCO_ERR_INVALID_ARG;
@@ -261,6 +276,7 @@ roco_status roco_prefill_blockwise(const void *Q, const void *K, const void *V, 
 roco_status roco_gqa_decode_step(roco_cache *cache, const void *Q, const void *k_new, const void *v_new, int group,
                                  int r, int scope_mode, float scale, void *attn_out, float *lse_out,
                                  int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {
+  NvtxRange range("roco_gqa_decode_step");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
   if (!Q || !k_new || !v_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
@@ -283,6 +299,7 @@ roco_status roco_decode_step_host(roco_cache *cache, const void *q_host, const v
                                   const void *v_new_host, int r, int scope_mode, int step_order, float scale,
                                   void *attn_out_host, int32_t *evicted_slot_host, int32_t *evicted_pos_host,
                                   void *staging, size_t staging_bytes, void *stream) {
+  NvtxRange range("roco_decode_step_host");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
   if (!q_host || !k_new_host || !v_new_host || !attn_out_host || !evicted_slot_host) return ROCO_ERR_INVALID_ARG;

@@ -45,3 +45,16 @@ def test_nan_statistics_are_flagged_not_fatal():
     assert R.roco_device_status(cache) & 4           # ROCO_DEV_BAD_VICTIM
     assert 0 <= int(ev[0, 0]) < w.B and 0 <= int(ev[0, 1]) < w.B
     assert torch.isfinite(out.float()).all()         # the attention itself does not read the statistics
+
+
+def test_a_wait_that_nothing_ends_runs_out_and_is_reported():
+    """The self-test kernel waits on a barrier that nothing completes: the bounded wait gives up after about two
+    seconds, sets the time-out bit and the kernel returns; the context stays usable (a decode step runs after)."""
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    waited = torch.zeros(1, dtype=torch.int32, device=DEV)
+    R.roco_selftest_wait_timeout(status, waited)
+    torch.cuda.synchronize()
+    assert int(status.item()) & 1, "ROCO_DEV_WAIT_TIMEOUT must be set"
+    assert 1500 <= int(waited.item()) <= 4000, waited.item()
+    probe = torch.arange(8, device=DEV).sum().item()   # the device still answers
+    assert probe == 28
