@@ -285,6 +285,10 @@ size_t roco_decode_host_staging_bytes(const roco_cache *cache);
  * synchronises the stream.  The cache stays on the device.  *_host arguments are host pointers with
  * the shapes above; evicted_pos_host may be NULL.  staging: device,
  * >= roco_decode_host_staging_bytes(cache), 256-byte aligned.
+ * With 2048 units or more the step is cut into four unit ranges (units are independent) and the copies of one
+ * range overlap the kernel of another: the copies then run on a copy stream that the library creates, with a
+ * handful of events, at the first such call on a device and keeps until the process exits -- the one piece of
+ * state besides the scratch of roco_prefill_static.  Host buffers must be pinned for the overlap to happen.
  */
 roco_status roco_decode_step_host(roco_cache *cache, const void *q_host, const void *k_new_host,
                                   const void *v_new_host, int r, int scope_mode, int step_order, float scale,

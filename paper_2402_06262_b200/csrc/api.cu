@@ -2,6 +2,7 @@
 #include <nvtx3/nvToolsExt.h>
 
 #include <cstring>
+#include <mutex>
 
 #include "common.cuh"
 #include "launch.h"
@@ -53,6 +54,36 @@ PrefillWs prefill_ws(int S, int G, int Lmax) {
   w.dst_off = w.q_off + per;
   w.total = w.dst_off + per;
   return w;
+}
+
+// Copy stream and events of roco_decode_step_host, one set per device, created at the first call on that device
+// and kept until the process exits.
+constexpr int kHostChunks = 4;
+constexpr int kHostMaxDevices = 64;
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t copy = nullptr;
+  cudaEvent_t start = nullptr, done = nullptr, h2d[kHostChunks] = {}, ker[kHostChunks] = {};
+};
+
+HostPipe *host_pipe() {
+  static HostPipe pipes[kHostMaxDevices];
+  static std::mutex mu;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kHostMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  HostPipe &hp = pipes[dev];
+  if (!hp.ready) {
+    bool ok = cudaStreamCreateWithFlags(&hp.copy, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&hp.done, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < kHostChunks; ++i)
+      ok = cudaEventCreateWithFlags(&hp.h2d[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.ker[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return nullptr;
+    hp.ready = true;
+  }
+  return &hp;
 }
 
 int pow2_at_least(int x) {
@@ -308,23 +339,78 @@ roco_status roco_decode_step_host(roco_cache *cache, const void *q_host, const v
     return ROCO_ERR_WORKSPACE;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   const size_t U = (size_t)cache->S * cache->G;
-  const size_t vbytes = U * cache->d * (cache->kv_dtype == ROCO_BF16 ? 2 : 4);
+  const size_t esz = cache->kv_dtype == ROCO_BF16 ? 2 : 4;
+  const size_t row = (size_t)cache->d * esz;  // bytes of one unit's vector
+  const size_t vbytes = U * row;
   const size_t vec = align_up(vbytes, 256), ivec = align_up(U * 4, 256);
   char *p = static_cast<char *>(staging);
   char *dq = p, *dk = p + vec, *dv = p + 2 * vec, *dout = p + 3 * vec;
   int32_t *dslot = reinterpret_cast<int32_t *>(p + 4 * vec), *dpos = reinterpret_cast<int32_t *>(p + 4 * vec + ivec);
-  if (cudaMemcpyAsync(dq, q_host, vbytes, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
-      cudaMemcpyAsync(dk, k_new_host, vbytes, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
-      cudaMemcpyAsync(dv, v_new_host, vbytes, cudaMemcpyHostToDevice, cs) != cudaSuccess)
-    return ROCO_ERR_CUDA;
-  st = roco_decode_step(cache, dq, dk, dv, r, scope_mode, step_order, scale, dout, nullptr, dslot, dpos, stream);
+
+  HostPipe *hp = U >= 2048 ? host_pipe() : nullptr;
+  if (!hp) {  // few units (or no copy stream): copy in, one launch, copy out, all on the caller's stream
+    if (cudaMemcpyAsync(dq, q_host, vbytes, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+        cudaMemcpyAsync(dk, k_new_host, vbytes, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+        cudaMemcpyAsync(dv, v_new_host, vbytes, cudaMemcpyHostToDevice, cs) != cudaSuccess)
+      return ROCO_ERR_CUDA;
+    st = roco_decode_step(cache, dq, dk, dv, r, scope_mode, step_order, scale, dout, nullptr, dslot, dpos, stream);
+    if (st != ROCO_OK) return st;
+    if (cudaMemcpyAsync(attn_out_host, dout, vbytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
+        cudaMemcpyAsync(evicted_slot_host, dslot, U * 4, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+      return ROCO_ERR_CUDA;
+    if (evicted_pos_host &&
+        cudaMemcpyAsync(evicted_pos_host, dpos, U * 4, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+      return ROCO_ERR_CUDA;
+    return cudaStreamSynchronize(cs) == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
+  }
+
+  // Units are independent, so the step is cut into kHostChunks unit ranges: the copies of a range run on the copy
+  // stream while the kernel of the previous range runs on the caller's stream.
+  const char *hq = static_cast<const char *>(q_host), *hk = static_cast<const char *>(k_new_host),
+             *hv = static_cast<const char *>(v_new_host);
+  char *hout = static_cast<char *>(attn_out_host);
+  auto ok = [](cudaError_t e) { return e == cudaSuccess; };
+  if (!ok(cudaEventRecord(hp->start, cs)) || !ok(cudaStreamWaitEvent(hp->copy, hp->start, 0))) return ROCO_ERR_CUDA;
+  size_t lo[kHostChunks + 1];
+  for (int c = 0; c <= kHostChunks; ++c) lo[c] = U * c / kHostChunks;
+  for (int c = 0; c < kHostChunks && st == ROCO_OK; ++c) {  // inputs of range c in, then its kernel (launched early)
+    const size_t u0 = lo[c], nu = lo[c + 1] - lo[c], off = u0 * row, nb = nu * row;
+    if (!ok(cudaMemcpyAsync(dq + off, hq + off, nb, cudaMemcpyHostToDevice, hp->copy)) ||
+        !ok(cudaMemcpyAsync(dk + off, hk + off, nb, cudaMemcpyHostToDevice, hp->copy)) ||
+        !ok(cudaMemcpyAsync(dv + off, hv + off, nb, cudaMemcpyHostToDevice, hp->copy)) ||
+        !ok(cudaEventRecord(hp->h2d[c], hp->copy)) || !ok(cudaStreamWaitEvent(cs, hp->h2d[c], 0))) {
+      st = ROCO_ERR_CUDA;
+      break;
+    }
+    roco_cache view = *cache;  // the units u0 .. u0 + nu - 1 as a cache of their own
+    view.S = 1;
+    view.G = (int32_t)nu;
+    view.K = static_cast<char *>(cache->K) + u0 * cache->B * row;
+    view.V = static_cast<char *>(cache->V) + u0 * cache->B * row;
+    view.s = cache->s + u0 * cache->B;
+    view.q = cache->q + u0 * cache->B;
+    view.n = cache->n + u0 * cache->B;
+    view.pos = cache->pos + u0 * cache->B;
+    view.live = cache->live + u0;
+    view.t_next = cache->t_next + u0;
+    st = roco_decode_step(&view, dq + off, dk + off, dv + off, r, scope_mode, step_order, scale, dout + off, nullptr,
+                          dslot + u0, dpos + u0, stream);
+    if (st == ROCO_OK && !ok(cudaEventRecord(hp->ker[c], cs))) st = ROCO_ERR_CUDA;
+  }
+  for (int c = 0; c < kHostChunks && st == ROCO_OK; ++c) {  // results out, behind the last input copy
+    const size_t u0 = lo[c], nu = lo[c + 1] - lo[c];
+    if (!ok(cudaStreamWaitEvent(hp->copy, hp->ker[c], 0)) ||
+        !ok(cudaMemcpyAsync(hout + u0 * row, dout + u0 * row, nu * row, cudaMemcpyDeviceToHost, hp->copy)) ||
+        !ok(cudaMemcpyAsync(evicted_slot_host + u0, dslot + u0, nu * 4, cudaMemcpyDeviceToHost, hp->copy)) ||
+        (evicted_pos_host &&
+         !ok(cudaMemcpyAsync(evicted_pos_host + u0, dpos + u0, nu * 4, cudaMemcpyDeviceToHost, hp->copy))))
+      st = ROCO_ERR_CUDA;
+  }
+  // whatever was enqueued is drained before returning, also after an error
+  const bool drained = ok(cudaEventRecord(hp->done, hp->copy)) && ok(cudaStreamWaitEvent(cs, hp->done, 0)) &&
+                       ok(cudaStreamSynchronize(cs)) && ok(cudaStreamSynchronize(hp->copy));
   if (st != ROCO_OK) return st;
-  if (cudaMemcpyAsync(attn_out_host, dout, vbytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
-      cudaMemcpyAsync(evicted_slot_host, dslot, U * 4, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
-    return ROCO_ERR_CUDA;
-  if (evicted_pos_host && cudaMemcpyAsync(evicted_pos_host, dpos, U * 4, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
-    return ROCO_ERR_CUDA;
-  return cudaStreamSynchronize(cs) == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
+  return drained ? ROCO_OK : ROCO_ERR_CUDA;
 }
 
 roco_status roco_device_status(const roco_cache *cache, void *stream, int32_t *flags_host) {

@@ -158,8 +158,12 @@ def test_checkpoint_resume_is_bit_exact():
         assert torch.equal(a, b)
 
 
-def test_host_buffer_variant_matches_device_variant():
-    w = W.scaled(W.LLAMA7B_DECODE, S=2, layers=1, heads=4, prompt_lo=150, prompt_hi=150, B=128, r=8)
+@pytest.mark.parametrize("layers,heads,B", [(1, 4, 128), (32, 33, 32)])
+def test_host_buffer_variant_matches_device_variant(layers, heads, B):
+    """Host-buffer step against the device-buffer step, bit for bit: 8 units (one launch) and 2112 units (the
+    step is cut into four unit ranges whose copies overlap the kernels; 2112 is not a multiple of four ranges of
+    equal size times anything convenient, and 33 heads make the ranges straddle sequences)."""
+    w = W.scaled(W.LLAMA7B_DECODE, S=2, layers=layers, heads=heads, prompt_lo=150, prompt_hi=150, B=B, r=8)
     Q, K, V = prompt_tensors(w, 150)
     caches = [R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV) for _ in range(2)]
     for c in caches:
