@@ -289,6 +289,7 @@ size_t roco_decode_host_staging_bytes(const roco_cache *cache);
  * range overlap the kernel of another: the copies then run on a copy stream that the library creates, with a
  * handful of events, at the first such call on a device and keeps until the process exits -- the one piece of
  * state besides the scratch of roco_prefill_static.  Host buffers must be pinned for the overlap to happen.
+ * Large calls on one device share those events, so they must not be issued from several host threads at once.
  */
 roco_status roco_decode_step_host(roco_cache *cache, const void *q_host, const void *k_new_host,
                                   const void *v_new_host, int r, int scope_mode, int step_order, float scale,
