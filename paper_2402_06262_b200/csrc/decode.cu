@@ -193,6 +193,24 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     // ------------------------------------------------------------ policy: scope, victim, in-place overwrite
     const int ptid = tid - kPolicyWarp0 * 32;
     const int t_new = p.t_next[u];  // read by these warps only: they also write the incremented value
+    // What the tail of this branch needs from global memory and does not depend on the victim is requested now,
+    // so that its latency passes during the selection: the 16 bytes of k_new / v_new this thread will write into
+    // the freed slot, and (last warp) the operands of the new token's own score.
+    const bool writes_row = ptid >= 32 && ptid < 32 + 2 * kLanesPerRow;
+    uint4 row_val = make_uint4(0u, 0u, 0u, 0u);
+    if (writes_row) {
+      const int c = ptid - 32;
+      const bool isv = c >= kLanesPerRow;
+      row_val = *((const uint4 *)((isv ? p.v_new : p.k_new) + (size_t)u * kRowBytes) + (isv ? c - kLanesPerRow : c));
+    }
+    float own_q[D / 32], own_k[D / 32];
+    if (evict_first && ptid >= 96) {
+#pragma unroll
+      for (int i = 0; i < D / 32; ++i) {
+        own_q[i] = Elem<T>::load((const T *)p.qv + (size_t)u * D + lane + 32 * i);
+        own_k[i] = Elem<T>::load((const T *)p.k_new + (size_t)u * D + lane + 32 * i);
+      }
+    }
     named_bar_sync(kBarPolicy, kPolicyThreads);
     // statistics of Sec. 4.3 for the slots the query attended over: Acc += p, Acc^square += p^2, Count += 1
     // (a slot that has just received the new token starts from zero)
@@ -288,29 +306,28 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
       sm.ctl[1] = e;
       p.pos[unit_st + e] = t_new;
       p.ev_slot[u] = ev_slot;
-      if (p.ev_pos) p.ev_pos[u] = ev_pos;
       p.live[u] = live_new;
       p.t_next[u] = t_new + 1;
       if (!evict_first) { p.s[unit_st + e] = 0.f; p.q[unit_st + e] = 0.f; p.n[unit_st + e] = 0; }
     }
-    if (ptid >= 32 && ptid < 32 + 2 * kLanesPerRow) {  // in-place overwrite, 16 bytes per thread
+    if (writes_row) {  // in-place overwrite, 16 bytes per thread
       const int c = ptid - 32;
       const bool isv = c >= kLanesPerRow;
-      const int cc = isv ? c - kLanesPerRow : c;
-      const uint4 val = *((const uint4 *)((isv ? p.v_new : p.k_new) + (size_t)u * kRowBytes) + cc);
       char *dst = const_cast<char *>(isv ? p.V : p.K) + unit_kv + (size_t)e * kRowBytes;
-      *((uint4 *)dst + cc) = val;
+      *((uint4 *)dst + (isv ? c - kLanesPerRow : c)) = row_val;
     }
     if (evict_first && ptid >= 96) {  // the new token's own score, from k_new directly
       float acc = 0.f;
-      for (int c = lane; c < D; c += 32)
-        acc = fmaf(Elem<T>::load((const T *)p.qv + (size_t)u * D + c),
-                   Elem<T>::load((const T *)p.k_new + (size_t)u * D + c), acc);
+#pragma unroll
+      for (int i = 0; i < D / 32; ++i) acc = fmaf(own_q[i], own_k[i], acc);
       acc = warp_sum(acc);
       if (lane == 0) *sm.znew = acc * (p.scale * kLog2e);
     }
     named_bar_sync(kBarPolicy, kPolicyThreads);
-    if (ptid == 0) mbar_arrive(sm.policy_done);
+    if (ptid == 0) {
+      mbar_arrive(sm.policy_done);
+      if (p.ev_pos) p.ev_pos[u] = ev_pos;  // waits for the load of the old position: after the signal
+    }
     if (evict_first) update_statistics(e);
     return;
   }
@@ -334,19 +351,28 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     const int st = it % stages;
     mbar_wait(&sm.full[st], (it / stages) & 1, abort_flag, p.status);
     const char *tile = sm.ring + (size_t)st * TILE;
+    // the partial dot products of all the rows this lane touches first, then one butterfly over the lanes of a
+    // row for all of them together (independent shuffles back to back instead of kLoads dependent chains)
+    float acc[kLoads];
 #pragma unroll
     for (int l = 0; l < kLoads; ++l) {
       const int row = warp * kRowsPerWarp + l * kRowsPerLoad + lane_row;
       const uint4 c = *(const uint4 *)(tile + (size_t)row * kRowBytes + lane_chunk * 16);
       float f[kEPC];
       Elem<T>::unpack(c, f);
-      float acc = 0.f;
+      acc[l] = 0.f;
 #pragma unroll
-      for (int i = 0; i < kEPC; ++i) acc = fmaf(f[i], qreg[i], acc);
+      for (int i = 0; i < kEPC; ++i) acc[l] = fmaf(f[i], qreg[i], acc[l]);
+    }
 #pragma unroll
-      for (int o = kLanesPerRow / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      const int j = it * kTileRows + row;
-      if (lane_chunk == 0 && j < live_att) sm.z[j] = acc * zscale;
+    for (int o = kLanesPerRow / 2; o > 0; o >>= 1) {
+#pragma unroll
+      for (int l = 0; l < kLoads; ++l) acc[l] += __shfl_xor_sync(0xffffffffu, acc[l], o);
+    }
+#pragma unroll
+    for (int l = 0; l < kLoads; ++l) {
+      const int j = it * kTileRows + warp * kRowsPerWarp + l * kRowsPerLoad + lane_row;
+      if (lane_chunk == 0 && j < live_att) sm.z[j] = acc[l] * zscale;
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.empty[st]);

@@ -337,16 +337,6 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     v.newtok[slot] = (signed char)ptid;
     gpos[slot] = t_new + ptid;
   }
-#pragma unroll 4
-  for (int w = ptid; w < nb * 2 * kLanesPerRow; w += kMqPolicyThreads) {  // in-place overwrite, 16 bytes each
-    const int i = w / (2 * kLanesPerRow), c = w % (2 * kLanesPerRow);
-    const bool isv = c >= kLanesPerRow;
-    const int cc = isv ? c - kLanesPerRow : c;
-    int slot = tgt[i];
-    if (slot < 0 || slot >= B) slot = 0;
-    const uint4 val = *((const uint4 *)((isv ? p.v_new : p.k_new) + ((size_t)u * p.kv_ustride + i) * kRowBytes) + cc);
-    *((uint4 *)(const_cast<char *>(isv ? p.V : p.K) + unit_kv + (size_t)slot * kRowBytes) + cc) = val;
-  }
   // scores of every query against every new token, from k_new directly (log2 domain)
   const float zscale = p.scale * kLog2e;
   if (v.zn_by_consumers) {
@@ -378,6 +368,18 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
   if (ptid == 0) { p.live[u] = live1; p.t_next[u] = t_new + nb; }
   named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
   if (ptid == 0) mbar_arrive(v.policy_done);
+  // In-place overwrite, 16 bytes per thread and turn.  Nothing in this step reads these rows from the cache (the
+  // scores and values of new tokens come from K_new / V_new), so it is done after the consumers were released.
+#pragma unroll 4
+  for (int w = ptid; w < nb * 2 * kLanesPerRow; w += kMqPolicyThreads) {
+    const int i = w / (2 * kLanesPerRow), c = w % (2 * kLanesPerRow);
+    const bool isv = c >= kLanesPerRow;
+    const int cc = isv ? c - kLanesPerRow : c;
+    int slot = tgt[i];
+    if (slot < 0 || slot >= B) slot = 0;
+    const uint4 val = *((const uint4 *)((isv ? p.v_new : p.k_new) + ((size_t)u * p.kv_ustride + i) * kRowBytes) + cc);
+    *((uint4 *)(const_cast<char *>(isv ? p.V : p.K) + unit_kv + (size_t)slot * kRowBytes) + cc) = val;
+  }
 
   // statistics of Sec. 4.3 once the probabilities are in shared memory
   mbar_wait(v.p_ready, 0, abort_flag, p.status);
