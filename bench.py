@@ -34,7 +34,7 @@ import torch
 import workloads as W
 
 # dram__bytes_read.sum + dram__bytes_write.sum of decode_step_kernel, per unit (profiles/decode_step_kernel_*.md)
-NCU_TRAFFIC = {"kernel_hash": "45ba8bed96d81aa2", "shape": (1024, 128, "bf16"), "dram_bytes_per_unit": 568800}
+NCU_TRAFFIC = {"kernel_hash": "8076960864a82fcd", "shape": (1024, 128, "bf16"), "dram_bytes_per_unit": 568200}
 
 METRIC = "decode_tokens_per_s"
 UNIT = "tokens/s"
