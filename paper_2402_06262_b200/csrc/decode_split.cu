@@ -157,19 +157,27 @@ __global__ void __launch_bounds__(kSpThreads) split_attend_kernel(const SplitPar
     const int st = it % kSpStages;
     mbar_wait(&full[st], (it / kSpStages) & 1, abort_flag, p.status);
     const char *tile = ring + (size_t)st * kSpTile;
+    // partial dot products of all the rows this lane touches, then one butterfly for all of them
+    float acc[kLoads];
 #pragma unroll
     for (int l = 0; l < kLoads; ++l) {
       const int row = warp * kRowsPerWarp + l * kRowsPerLoad + lane_row;
       const uint4 ch = *(const uint4 *)(tile + (size_t)row * kRowBytes + lane_chunk * 16);
       float f[kEPC];
       Elem<T>::unpack(ch, f);
-      float acc = 0.f;
+      acc[l] = 0.f;
 #pragma unroll
-      for (int i = 0; i < kEPC; ++i) acc = fmaf(f[i], qreg[i], acc);
+      for (int i = 0; i < kEPC; ++i) acc[l] = fmaf(f[i], qreg[i], acc[l]);
+    }
 #pragma unroll
-      for (int o = kLanesPerRow / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      const int j = (t0 + it) * kTileRows + row;
-      if (lane_chunk == 0 && j < j1) z[j - j0] = acc * zscale;
+    for (int o = kLanesPerRow / 2; o > 0; o >>= 1) {
+#pragma unroll
+      for (int l = 0; l < kLoads; ++l) acc[l] += __shfl_xor_sync(0xffffffffu, acc[l], o);
+    }
+#pragma unroll
+    for (int l = 0; l < kLoads; ++l) {
+      const int j = (t0 + it) * kTileRows + warp * kRowsPerWarp + l * kRowsPerLoad + lane_row;
+      if (lane_chunk == 0 && j < j1) z[j - j0] = acc[l] * zscale;
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(&empty[st]);

@@ -527,8 +527,11 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
         acc[i] = 0.f;
 #pragma unroll
         for (int e = 0; e < kEPC; ++e) acc[i] = fmaf(f[e], qreg[i][e], acc[i]);
+      }
 #pragma unroll
-        for (int o = kLanesPerRow / 2; o > 0; o >>= 1) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], o);
+      for (int o = kLanesPerRow / 2; o > 0; o >>= 1) {  // one butterfly for the four queries together
+#pragma unroll
+        for (int i = 0; i < kMqQPW; ++i) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], o);
       }
       const int j = it * kTileRows + row;
       if (lane_chunk < kMqQPW && j < live1) {
