@@ -14,6 +14,7 @@
 #include "common.cuh"
 #include "launch.h"
 #include "select.cuh"
+#include "tc.cuh"
 
 namespace roco {
 
@@ -115,6 +116,9 @@ struct PolicyView {
   int *posbuf;  // the unit's positions as they were before the step (with stats_full)
   uint64_t *stats_full;
   bool zn_by_consumers;
+  // Tensor-memory kernel only (else nullptr): per-slot sums over the queries of p and p^2 for the tokens that were
+  // cached before the step, formed by the consumer warps (which keep the probabilities to themselves there).
+  const float *ds, *dq;
 };
 
 // The policy warps' part of a multi-query step: free `need` slots (Sec. 4.3 rule on frozen statistics), insert
@@ -142,7 +146,9 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     const uint4 *gv = reinterpret_cast<const uint4 *>(p.v_new + (size_t)u * p.kv_ustride * kRowBytes);
     const uint4 *gqr = reinterpret_cast<const uint4 *>(p.Q + (size_t)u * p.q_ustride * kRowBytes);
     const int nkv = nb * D / kEPC, nq = v.qf ? M * D / kEPC : 0;
-    if (v.zn_by_consumers) {
+    if (v.zn_by_consumers && !v.vnew) {
+      // the consumers read the new values from global memory themselves
+    } else if (v.zn_by_consumers) {
 #pragma unroll 4
       for (int i = ptid; i < nkv; i += kMqPolicyThreads) {
         float f[kEPC];
@@ -405,7 +411,17 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
       const bool fresh = jn >= 0;
       float ds = 0.f, dq = 0.f;
       int dn;
-      if (p.kind == kMqGqa) {
+      if (v.ds && !fresh) {
+        if (p.kind == kMqGqa) {
+          ds = v.ds[j] / (float)M;  // group-wise averaged attention score
+          dq = ds * ds;
+          dn = 1;
+        } else {
+          ds = v.ds[j];
+          dq = v.dq[j];
+          dn = M;
+        }
+      } else if (p.kind == kMqGqa) {
         for (int i = 0; i < M; ++i) ds += (fresh && v.pn) ? v.pn[i * nb + jn] : v.z[(size_t)i * Bp + j];
         ds /= (float)M;  // group-wise averaged attention score
         dq = ds * ds;
@@ -485,6 +501,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
     v.z = sm.z; v.Bp = Bp; v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok; v.sel = sm.sel;
     v.knew = sm.knew; v.vnew = sm.vnew; v.zn = sm.zn; v.qf = nullptr; v.pn = nullptr; v.ctl = sm.ctl;
     v.nbuf = nullptr; v.posbuf = nullptr; v.stats_full = nullptr; v.zn_by_consumers = false;
+    v.ds = nullptr; v.dq = nullptr;
     v.p_ready = sm.p_ready;
     v.policy_done = sm.policy_done;
     multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
@@ -796,6 +813,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
     v.knew = nullptr; v.vnew = sm.vnew; v.zn = sm.zn; v.qf = nullptr; v.pn = sm.pn; v.ctl = sm.ctl;
     v.nbuf = sm.nbuf; v.posbuf = sm.posbuf; v.stats_full = stats_by_tma ? sm.stats_full : nullptr;
     v.zn_by_consumers = true;
+    v.ds = nullptr; v.dq = nullptr;
     v.p_ready = sm.p_ready;
     v.policy_done = sm.policy_done;
     multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
@@ -966,11 +984,417 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
   }
 }
 
+// ------------------------------------------------------------------------------------------------------------
+// Tensor-memory variant of the kernel above, for more than 8 queries (bf16, d = 128, B <= 2048).  There the M x B
+// fp32 score matrix (64 KiB at M = 16, B = 1024) is what keeps a second CTA off the SM, and with one CTA per SM
+// nothing overlaps the softmax and the selection.  Here every consumer thread keeps the scores its own MMAs
+// produced -- per 64-key tile: rows g and g + 8, keys 2 tq and 2 tq + 1 of the warp's 8 keys -- in four columns of
+// its tensor-memory lane (warps w and w + 4 share lanes and take different column halves), works on them in
+// place (row maxima and sums via quad shuffles and a small shared array), and leaves only what other threads need
+// in shared memory: the probabilities as bf16 for the output MMAs (half the size), and the per-slot sums over the
+// queries of p and p^2 for the statistics (in the key arrays, which the selection no longer needs by then).
+
+struct MultiTmSmem {
+  char *ring;
+  __nv_bfloat16 *pz;  // [16][Bp] probabilities, bf16, rows >= M zero; Bp = multi_tc_row_stride(B)
+  uint32_t *vkey;     // later: ds
+  float *mkey;        // later: dq
+  int *nbuf, *posbuf;
+  signed char *newtok;
+  SelectScratch *sel;
+  float *zn, *pn;
+  float *red;         // [8 warps][16 rows]
+  uint64_t *full, *empty, *p_ready, *policy_done, *stats_full;
+  uint32_t *tmem_base;
+  int *ctl;
+};
+
+__host__ __device__ inline size_t multi_tm_smem_bytes(int B, int stages, int M, int nb) {
+  const size_t Bp = multi_tc_row_stride(B);
+  size_t b = (size_t)stages * kMqTile;
+  b += 16 * Bp * 2 + 4 * Bp * 4 + Bp;
+  b += sizeof(SelectScratch);
+  b += 2 * (size_t)M * nb * 4 + kMqConsumerWarps * 16 * 4;
+  b = align_up(b, 8) + (2 * (size_t)stages + 4) * 8 + 64 * 4;
+  return b + 1024;
+}
+
+__device__ inline MultiTmSmem multi_tm_carve(char *raw, int B, int stages, int M, int nb) {
+  MultiTmSmem m;
+  char *p = smem_align(raw, 1024);
+  const size_t Bp = multi_tc_row_stride(B);
+  m.ring = p; p += (size_t)stages * kMqTile;
+  m.pz = (__nv_bfloat16 *)p; p += 16 * Bp * 2;
+  m.vkey = (uint32_t *)p; p += Bp * 4;
+  m.mkey = (float *)p; p += Bp * 4;
+  m.nbuf = (int *)p; p += Bp * 4;
+  m.posbuf = (int *)p; p += Bp * 4;
+  m.newtok = (signed char *)p; p += Bp;
+  m.sel = (SelectScratch *)p; p += sizeof(SelectScratch);
+  m.zn = (float *)p; p += (size_t)M * nb * 4;
+  m.pn = (float *)p; p += (size_t)M * nb * 4;
+  m.red = (float *)p; p += kMqConsumerWarps * 16 * 4;
+  p = smem_align(p, 8);
+  m.full = (uint64_t *)p; p += stages * 8;
+  m.empty = (uint64_t *)p; p += stages * 8;
+  m.p_ready = (uint64_t *)p; p += 8;
+  m.policy_done = (uint64_t *)p; p += 8;
+  m.stats_full = (uint64_t *)p; p += 8;
+  m.tmem_base = (uint32_t *)p; p += 8;
+  m.ctl = (int *)p;
+  return m;
+}
+
+// Tensor-memory columns of one CTA: two halves (warps 0-3, warps 4-7) of four columns per tile, tiles rounded up
+// to a multiple of four (the in-place passes move 16 columns at a time), a power of two of at least 32.
+__host__ __device__ inline int multi_tm_cols(int B) {
+  const int tiles = ((B + 63) / 64 + 3) / 4 * 4;
+  int c = 32;
+  while (c < 8 * tiles) c <<= 1;
+  return c;
+}
+
+__global__ void __launch_bounds__(kMqThreads, 2) multi_step_tm_kernel(const __grid_constant__ CUtensorMap mapK,
+                                                                      const __grid_constant__ CUtensorMap mapV,
+                                                                      const MultiParams p, int tmem_cols) {
+  using T = __nv_bfloat16;
+  constexpr int D = 128, kTileRows = 64;
+  extern __shared__ char mq_smem_raw[];
+  const int M = p.M, nb = p.nb, B = p.B, stages = p.stages;
+  const MultiTmSmem sm = multi_tm_carve(mq_smem_raw, B, stages, M, nb);
+  volatile int *abort_flag = sm.ctl;
+  const size_t Bp = multi_tc_row_stride(B);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int u = blockIdx.x;
+
+  if (tid == 0) {
+    for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kMqConsumerWarps); }
+    mbar_init(sm.p_ready, kMqConsumerWarps);
+    mbar_init(sm.policy_done, 1);
+    mbar_init(sm.stats_full, 1);
+    sm.ctl[0] = 0;
+    mbar_init_fence();
+  }
+  if (warp == 0) {
+    tmem_alloc(sm.tmem_base, (uint32_t)tmem_cols);
+    tmem_relinquish();
+  }
+  int live0 = p.live[u];
+  if (live0 < 0 || live0 > B) {
+    if (tid == 0) atomicOr(p.status, ROCO_DEV_BAD_LIVE);
+    live0 = live0 < 0 ? 0 : B;
+  }
+  int need = live0 + nb - B;
+  if (need < 0) need = 0;
+  const int live1 = live0 - need + nb;
+  const int n_tiles = (live1 + kTileRows - 1) / kTileRows;
+  const bool stats_by_tma =
+      need > 0 && (B & 3) == 0 &&
+      ((reinterpret_cast<uintptr_t>(p.s) | reinterpret_cast<uintptr_t>(p.q) | reinterpret_cast<uintptr_t>(p.n) |
+        reinterpret_cast<uintptr_t>(p.pos)) & 15) == 0;
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *sm.tmem_base;
+
+  if (warp == kMqProducerWarp) {
+    if (lane == 0) {
+      if (stats_by_tma) {
+        const uint32_t bytes = (uint32_t)align_up((size_t)live0 * 4, 16);  // B % 4 == 0: stays inside the unit
+        mbar_expect_tx(sm.stats_full, 4 * bytes);
+        bulk_g2s(sm.vkey, p.s + (size_t)u * B, bytes, sm.stats_full);
+        bulk_g2s(sm.mkey, p.q + (size_t)u * B, bytes, sm.stats_full);
+        bulk_g2s(sm.nbuf, p.n + (size_t)u * B, bytes, sm.stats_full);
+        bulk_g2s(sm.posbuf, p.pos + (size_t)u * B, bytes, sm.stats_full);
+      }
+      for (int g = 0; g < 2 * n_tiles; ++g) {
+        const int st = g % stages;
+        if (g >= stages) mbar_wait(&sm.empty[st], ((g / stages) - 1) & 1, abort_flag, p.status);
+        const int it = (g < n_tiles) ? g : g - n_tiles;
+        const CUtensorMap *map = (g < n_tiles) ? &mapK : &mapV;
+        char *dst = sm.ring + (size_t)st * kMqTile;
+        const int row = u * B + it * kTileRows;
+        mbar_expect_tx(&sm.full[st], kMqTile);
+        tma_load_2d(dst, map, 0, row, &sm.full[st]);
+        tma_load_2d(dst + 8192, map, 64, row, &sm.full[st]);
+      }
+    }
+    return;
+  }
+
+  if (warp >= kMqPolicyWarp0) {
+    PolicyView v;
+    v.z = nullptr; v.Bp = Bp; v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok; v.sel = sm.sel;
+    v.knew = nullptr; v.vnew = nullptr; v.zn = sm.zn; v.qf = nullptr; v.pn = sm.pn; v.ctl = sm.ctl;
+    v.p_ready = sm.p_ready;
+    v.policy_done = sm.policy_done;
+    v.nbuf = sm.nbuf; v.posbuf = sm.posbuf; v.stats_full = stats_by_tma ? sm.stats_full : nullptr;
+    v.zn_by_consumers = true;
+    v.ds = reinterpret_cast<const float *>(sm.vkey); v.dq = sm.mkey;
+    multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
+    return;
+  }
+
+  // -------------------------------------------------------------- consumers
+  const float zscale = p.scale * kLog2e;
+  const int g = lane >> 2, tq = lane & 3;
+  const bool row_lo = g < M, row_hi = g + 8 < M;
+  const bool block = p.kind == kMqBlock;
+  // this thread's lane of tensor memory and first column: tile `it` occupies the columns 4 it .. 4 it + 3 with
+  // (row g, key 2 tq), (g, 2 tq + 1), (g + 8, 2 tq), (g + 8, 2 tq + 1) of the warp's 8 keys of that tile
+  const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * (tmem_cols / 2));
+  uint32_t qa[8][4];
+  {
+    const T *Qu = (const T *)p.Q + (size_t)u * p.q_ustride * D;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      const int k0 = s * 16 + tq * 2;
+      qa[s][0] = row_lo ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)g * D + k0) : 0u;
+      qa[s][1] = row_hi ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)(g + 8) * D + k0) : 0u;
+      qa[s][2] = row_lo ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)g * D + k0 + 8) : 0u;
+      qa[s][3] = row_hi ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)(g + 8) * D + k0 + 8) : 0u;
+    }
+  }
+
+  // ---- scores: Z[16 x 8] = Q[16 x 128] K^T per warp and tile, into tensor memory (-inf where there is nothing)
+  for (int it = 0; it < n_tiles; ++it) {
+    const int st = it % stages;
+    mbar_wait(&sm.full[st], (it / stages) & 1, abort_flag, p.status);
+    const uint32_t tile = smem_u32(sm.ring + (size_t)st * kMqTile);
+    float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int sp = 0; sp < 4; ++sp) {
+      uint32_t kb[4];
+      ldmatrix_x4(tile + tile_chunk_offset(warp * 8 + (lane & 7), sp * 4 + (lane >> 3)), kb);
+      mma_bf16_16816(c, qa[2 * sp], kb[0], kb[1]);
+      mma_bf16_16816(c, qa[2 * sp + 1], kb[2], kb[3]);
+    }
+    const int j = it * kTileRows + warp * 8 + tq * 2;
+    const float ninf = -INFINITY;
+    tmem_st4(taddr + it * 4, __float_as_uint(row_lo && j < live1 ? c[0] * zscale : ninf),
+             __float_as_uint(row_lo && j + 1 < live1 ? c[1] * zscale : ninf),
+             __float_as_uint(row_hi && j < live1 ? c[2] * zscale : ninf),
+             __float_as_uint(row_hi && j + 1 < live1 ? c[3] * zscale : ninf));
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.empty[st]);
+  }
+  // scores of the queries against the new tokens, from k_new: Zn[16 x 8] per warp, one warp per 8 new tokens
+  if (warp * 8 < nb) {
+    const T *Kn = (const T *)p.k_new + (size_t)u * p.kv_ustride * D;
+    const int jn = warp * 8 + g;
+    float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      const int k0 = s * 16 + tq * 2;
+      const uint32_t b0 = jn < nb ? *reinterpret_cast<const uint32_t *>(Kn + (size_t)jn * D + k0) : 0u;
+      const uint32_t b1 = jn < nb ? *reinterpret_cast<const uint32_t *>(Kn + (size_t)jn * D + k0 + 8) : 0u;
+      mma_bf16_16816(c, qa[s], b0, b1);
+    }
+    const int j0 = warp * 8 + tq * 2;
+    if (row_lo) {
+      if (j0 < nb) sm.zn[g * nb + j0] = c[0] * zscale;
+      if (j0 + 1 < nb) sm.zn[g * nb + j0 + 1] = c[1] * zscale;
+    }
+    if (row_hi) {
+      if (j0 < nb) sm.zn[(g + 8) * nb + j0] = c[2] * zscale;
+      if (j0 + 1 < nb) sm.zn[(g + 8) * nb + j0 + 1] = c[3] * zscale;
+    }
+  }
+  tmem_st_wait();
+  mbar_wait(sm.policy_done, 0, abort_flag, p.status);
+  named_bar_sync(kMqBarConsumers, kMqConsumers);
+
+  // The thread group that owns slot `slot`: its tile, the warp (8 keys of the tile each), the quad lane and the
+  // parity inside the key pair.  All lanes of the owning warp take part in the tensor-memory access.
+  auto for_new_tokens = [&](auto body) {
+    for (int jn = 0; jn < nb; ++jn) {
+      int slot = sm.ctl[1 + jn];
+      if (slot < 0 || slot >= B) slot = 0;
+      const int kk = slot & 63;
+      if (warp != (kk >> 3)) continue;
+      const uint32_t col = taddr + (uint32_t)((slot >> 6) * 4 + (kk & 1));
+      float a = __uint_as_float(tmem_ld1(col)), b = __uint_as_float(tmem_ld1(col + 2));
+      if (tq == ((kk & 7) >> 1)) body(jn, a, b);
+      tmem_st1(col, __float_as_uint(a));
+      tmem_st1(col + 2, __float_as_uint(b));
+    }
+    tmem_st_wait();
+  };
+  // the new tokens' scores replace whatever the stream brought for their slots (causal inside a block)
+  for_new_tokens([&](int jn, float &a, float &b) {
+    a = row_lo ? ((block && jn > g) ? -INFINITY : sm.zn[g * nb + jn]) : -INFINITY;
+    b = row_hi ? ((block && jn > g + 8) ? -INFINITY : sm.zn[(g + 8) * nb + jn]) : -INFINITY;
+  });
+
+  // ---- softmax per query row, in place: maxima, exponentials and sums
+  auto rows_reduce = [&](float &lo, float &hi, bool is_max) {
+#pragma unroll
+    for (int o = 1; o <= 2; o <<= 1) {
+      const float ol = __shfl_xor_sync(0xffffffffu, lo, o), oh = __shfl_xor_sync(0xffffffffu, hi, o);
+      lo = is_max ? fmaxf(lo, ol) : lo + ol;
+      hi = is_max ? fmaxf(hi, oh) : hi + oh;
+    }
+    if (tq == 0) { sm.red[warp * 16 + g] = lo; sm.red[warp * 16 + g + 8] = hi; }
+    named_bar_sync(kMqBarConsumers, kMqConsumers);
+    lo = sm.red[g]; hi = sm.red[g + 8];
+#pragma unroll
+    for (int w = 1; w < kMqConsumerWarps; ++w) {
+      lo = is_max ? fmaxf(lo, sm.red[w * 16 + g]) : lo + sm.red[w * 16 + g];
+      hi = is_max ? fmaxf(hi, sm.red[w * 16 + g + 8]) : hi + sm.red[w * 16 + g + 8];
+    }
+    named_bar_sync(kMqBarConsumers, kMqConsumers);
+  };
+  float mlo = -INFINITY, mhi = -INFINITY;
+  for (int it0 = 0; it0 < n_tiles; it0 += 4) {
+    uint32_t r[16];
+    tmem_ld16(taddr + it0 * 4, r);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      if (it0 + t < n_tiles) {
+        mlo = fmaxf(mlo, fmaxf(__uint_as_float(r[4 * t]), __uint_as_float(r[4 * t + 1])));
+        mhi = fmaxf(mhi, fmaxf(__uint_as_float(r[4 * t + 2]), __uint_as_float(r[4 * t + 3])));
+      }
+    }
+  }
+  rows_reduce(mlo, mhi, true);
+  if (!(mlo > -INFINITY)) mlo = 0.f;  // a row that does not exist
+  if (!(mhi > -INFINITY)) mhi = 0.f;
+  float slo = 0.f, shi = 0.f;
+  for (int it0 = 0; it0 < n_tiles; it0 += 4) {
+    uint32_t r[16];
+    tmem_ld16(taddr + it0 * 4, r);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const bool in = it0 + t < n_tiles;
+      const float e0 = in ? exp2f(__uint_as_float(r[4 * t]) - mlo) : 0.f;
+      const float e1 = in ? exp2f(__uint_as_float(r[4 * t + 1]) - mlo) : 0.f;
+      const float e2 = in ? exp2f(__uint_as_float(r[4 * t + 2]) - mhi) : 0.f;
+      const float e3 = in ? exp2f(__uint_as_float(r[4 * t + 3]) - mhi) : 0.f;
+      slo += e0 + e1;
+      shi += e2 + e3;
+      r[4 * t] = __float_as_uint(e0); r[4 * t + 1] = __float_as_uint(e1);
+      r[4 * t + 2] = __float_as_uint(e2); r[4 * t + 3] = __float_as_uint(e3);
+    }
+    tmem_st16(taddr + it0 * 4, r);
+  }
+  tmem_st_wait();
+  rows_reduce(slo, shi, false);
+  const float inv_lo = row_lo ? 1.f / slo : 0.f, inv_hi = row_hi ? 1.f / shi : 0.f;
+  if (warp == 0 && tq == 0 && p.lse) {
+    if (row_lo) p.lse[(size_t)u * M + g] = (mlo + log2f(slo)) * kLn2;
+    if (row_hi) p.lse[(size_t)u * M + g + 8] = (mhi + log2f(shi)) * kLn2;
+  }
+  // the new tokens' values come from v_new: their probabilities are set aside and cleared in place, so that the
+  // streamed V rows of those slots (possibly read before the overwrite) contribute nothing
+  for_new_tokens([&](int jn, float &a, float &b) {
+    if (row_lo) sm.pn[g * nb + jn] = a * inv_lo;
+    if (row_hi) sm.pn[(g + 8) * nb + jn] = b * inv_hi;
+    a = 0.f;
+    b = 0.f;
+  });
+  // probabilities: bf16 copy for the output MMAs; per-slot sums over the queries of p and p^2 for the statistics
+  {
+    float *ds = reinterpret_cast<float *>(sm.vkey), *dq = sm.mkey;
+    for (int it0 = 0; it0 < n_tiles; it0 += 4) {
+      uint32_t r[16];
+      tmem_ld16(taddr + it0 * 4, r);
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        if (it0 + t < n_tiles) {  // uniform over the warp
+          const int j = (it0 + t) * kTileRows + warp * 8 + tq * 2;
+          const float p0 = __uint_as_float(r[4 * t]) * inv_lo, p1 = __uint_as_float(r[4 * t + 1]) * inv_lo;
+          const float p2 = __uint_as_float(r[4 * t + 2]) * inv_hi, p3 = __uint_as_float(r[4 * t + 3]) * inv_hi;
+          *reinterpret_cast<uint32_t *>(sm.pz + (size_t)g * Bp + j) = pack_bf16x2(p0, p1);
+          *reinterpret_cast<uint32_t *>(sm.pz + (size_t)(g + 8) * Bp + j) = pack_bf16x2(p2, p3);
+          float s0 = p0 + p2, s1 = p1 + p3, q0 = fmaf(p0, p0, p2 * p2), q1 = fmaf(p1, p1, p3 * p3);
+#pragma unroll
+          for (int o = 4; o <= 16; o <<= 1) {  // over the eight row pairs
+            s0 += __shfl_xor_sync(0xffffffffu, s0, o);
+            s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+            q0 += __shfl_xor_sync(0xffffffffu, q0, o);
+            q1 += __shfl_xor_sync(0xffffffffu, q1, o);
+          }
+          if (g == 0) { ds[j] = s0; ds[j + 1] = s1; dq[j] = q0; dq[j + 1] = q1; }
+        }
+      }
+    }
+  }
+  __syncwarp();
+  if (lane == 0) mbar_arrive(sm.p_ready);
+  named_bar_sync(kMqBarConsumers, kMqConsumers);
+
+  // ---- out[16 x 128] += P[16 x 64] V[64 x 128]: each warp owns 16 output columns
+  float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+  for (int it = 0; it < n_tiles; ++it) {
+    const int gg = n_tiles + it;
+    const int st = gg % stages;
+    mbar_wait(&sm.full[st], (gg / stages) & 1, abort_flag, p.status);
+    const uint32_t tile = smem_u32(sm.ring + (size_t)st * kMqTile);
+    if ((it + 1) * kTileRows > live0) {  // slots that were free before the step may hold anything (0 x NaN)
+      const int r0 = live0 > it * kTileRows ? live0 - it * kTileRows : 0;
+      char *tp = sm.ring + (size_t)st * kMqTile;
+      for (int w = lane; w < (kTileRows - r0) * 2; w += 32) {
+        const int row = r0 + (w >> 1);
+        *reinterpret_cast<uint4 *>(tp + tile_chunk_offset(row, warp * 2 + (w & 1))) = make_uint4(0u, 0u, 0u, 0u);
+      }
+      __syncwarp();
+    }
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+      const int j = it * kTileRows + ks * 16 + tq * 2;
+      uint32_t pa[4];
+      const __nv_bfloat16 *zl = sm.pz + (size_t)g * Bp + j, *zh = sm.pz + (size_t)(g + 8) * Bp + j;
+      pa[0] = *reinterpret_cast<const uint32_t *>(zl);
+      pa[1] = *reinterpret_cast<const uint32_t *>(zh);
+      pa[2] = *reinterpret_cast<const uint32_t *>(zl + 8);
+      pa[3] = *reinterpret_cast<const uint32_t *>(zh + 8);
+      uint32_t vb[4];
+      const int mi = lane >> 3;
+      ldmatrix_x4_trans(tile + tile_chunk_offset(ks * 16 + (mi & 1) * 8 + (lane & 7), warp * 2 + (mi >> 1)), vb);
+      mma_bf16_16816(o[0], pa, vb[0], vb[1]);
+      mma_bf16_16816(o[1], pa, vb[2], vb[3]);
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.empty[st]);
+  }
+  const T *Vn = (const T *)p.v_new + (size_t)u * p.kv_ustride * D;
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    const int dcol = warp * 16 + nt * 8 + tq * 2;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int qi = g + 8 * h;
+      if (qi < M) {
+        float o0 = o[nt][2 * h], o1 = o[nt][2 * h + 1];
+        for (int jn = 0; jn < nb; ++jn) {
+          const float pj = sm.pn[qi * nb + jn];
+          const __nv_bfloat162 vv = *reinterpret_cast<const __nv_bfloat162 *>(Vn + (size_t)jn * D + dcol);
+          o0 = fmaf(pj, __bfloat162float(vv.x), o0);
+          o1 = fmaf(pj, __bfloat162float(vv.y), o1);
+        }
+        *reinterpret_cast<uint32_t *>((T *)p.out + ((size_t)u * p.out_ustride + qi) * D + dcol) = pack_bf16x2(o0, o1);
+      }
+    }
+  }
+  tc_fence_before();
+  named_bar_sync(kMqBarConsumers, kMqConsumers);
+  if (warp == 0) tmem_dealloc(tmem, (uint32_t)tmem_cols);
+}
+
 static int multi_tc_pick_stages(int B, int M, int nb) {
   const size_t per_sm = 227 * 1024;
   for (int ctas = 2; ctas >= 1; --ctas)
     for (int st = 6; st >= 3; --st)
       if ((multi_tc_smem_bytes(B, st, M, nb) + 1024) * ctas <= per_sm) return st;
+  return 0;
+}
+
+// Stages for the tensor-memory kernel: two CTAs per SM or nothing (with one it has no advantage).
+static int multi_tm_pick_stages(int B, int M, int nb) {
+  const size_t per_sm = 227 * 1024;
+  if (M <= 8 || multi_tm_cols(B) > 256) return 0;
+  for (int st = 4; st >= 3; --st)
+    if ((multi_tm_smem_bytes(B, st, M, nb) + 1024) * 2 <= per_sm) return st;
   return 0;
 }
 
@@ -1014,9 +1438,17 @@ roco_status launch_multi_step(const roco_cache &c, int kind, int M, int nb, cons
   if (c.kv_dtype == ROCO_BF16 && c.d == 128 && (long long)U * c.B < 0x7fffffffLL) {
     // tensor-core path; falls through to the CUDA-core path if the tensor maps cannot be built
     CUtensorMap mapK, mapV;
-    p.stages = multi_tc_pick_stages(c.B, M, nb);
+    const int tm_stages = multi_tm_pick_stages(c.B, M, nb);
+    p.stages = tm_stages > 0 ? tm_stages : multi_tc_pick_stages(c.B, M, nb);
     if (p.stages > 0 && make_tensor_map_rows128_bf16(&mapK, c.K, (unsigned long long)U * c.B, 64) &&
         make_tensor_map_rows128_bf16(&mapV, c.V, (unsigned long long)U * c.B, 64)) {
+      if (tm_stages > 0) {
+        const size_t smem = multi_tm_smem_bytes(c.B, p.stages, M, nb);
+        err = cudaFuncSetAttribute(multi_step_tm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return ROCO_ERR_CUDA;
+        multi_step_tm_kernel<<<U, kMqThreads, smem, stream>>>(mapK, mapV, p, multi_tm_cols(c.B));
+        return cudaGetLastError() == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
+      }
       const size_t smem = multi_tc_smem_bytes(c.B, p.stages, M, nb);
       err = cudaFuncSetAttribute(multi_step_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (err != cudaSuccess) return ROCO_ERR_CUDA;

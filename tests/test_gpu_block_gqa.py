@@ -30,7 +30,7 @@ def prefilled(w, L, tally, units):
     return cache, st
 
 
-@pytest.mark.parametrize("b", [1, 2, 4, 8, 16])
+@pytest.mark.parametrize("b", [1, 2, 4, 8, 12, 16])
 @pytest.mark.parametrize("dtype,d,B", [("bf16", 128, 300), ("bf16", 128, 302), ("f32", 64, 128)])
 def test_block_steps_fill_then_evict(b, dtype, d, B):
     """Short prompt: the first block steps only fill free slots (some mix freed and free slots), later ones evict
@@ -98,7 +98,7 @@ def test_block_step_argument_checks():
     assert e.value.code == 1
 
 
-@pytest.mark.parametrize("group", [1, 2, 4, 8])
+@pytest.mark.parametrize("group", [1, 2, 4, 8, 16])
 @pytest.mark.parametrize("mode", [R.ROCO_SCOPE_EXCLUDE_TOP_R, R.ROCO_SCOPE_LOWEST_R])
 def test_gqa_decode_steps(group, mode):
     """Zephyr-like grouping: `group` query heads per key-value head, statistics from the group mean."""
