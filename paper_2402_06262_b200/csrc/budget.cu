@@ -15,9 +15,14 @@ constexpr int kBudgetThreads = 512;
 constexpr int kBarAll = 1;
 
 // One CTA per unit.  dst[u][j] = cache slot of token j, or -1 if it is evicted.
+// kCached: the fp64 keys are formed once and kept in dynamic shared memory (16 bytes per token); otherwise every
+// pass of the selects forms them again (two fp64 divisions per token and pass), which is ~5x slower but has no
+// length limit.
+template <bool kCached>
 __global__ void __launch_bounds__(kBudgetThreads) budget_select_kernel(const float *s_full, const float *q_full,
                                                                        const int *lens, int G, int Lmax, int B, int r,
                                                                        int *dst, int *live, int *t_next) {
+  extern __shared__ __align__(16) unsigned char budget_keys_raw[];
   __shared__ SelectScratch sc;
   __shared__ int warp_tot[kBudgetThreads / 32];
   __shared__ int base_sh;
@@ -31,8 +36,19 @@ __global__ void __launch_bounds__(kBudgetThreads) budget_select_kernel(const flo
     return;
   }
   const int E = L - B;  // tokens to evict
-  auto vkey = [&](int j) { return (uint64_t)__double_as_longlong(variance_f64(s[j], q[j], L - j)); };
-  auto mkey = [&](int j) { return (uint64_t)__double_as_longlong(mean_f64(s[j], L - j)); };
+  uint64_t *vk = reinterpret_cast<uint64_t *>(budget_keys_raw), *mk = vk + Lmax;
+  if (kCached) {
+    for (int j = tid; j < L; j += kBudgetThreads) {
+      const float sj = s[j], qj = q[j];
+      vk[j] = (uint64_t)__double_as_longlong(variance_f64(sj, qj, L - j));
+      mk[j] = (uint64_t)__double_as_longlong(mean_f64(sj, L - j));
+    }
+    __syncthreads();
+  }
+  auto vkey = [&](int j) {
+    return kCached ? vk[j] : (uint64_t)__double_as_longlong(variance_f64(s[j], q[j], L - j));
+  };
+  auto mkey = [&](int j) { return kCached ? mk[j] : (uint64_t)__double_as_longlong(mean_f64(s[j], L - j)); };
   uint64_t Tv = ~0ull;
   int Pv = 0x7fffffff;
   if (r > 0) {  // the L-r tokens first in (variance, position) order may be evicted
@@ -246,9 +262,17 @@ roco_status launch_budget_select_gather(const roco_cache &c, int Lmax, const int
   if (scope_mode == ROCO_SCOPE_LOWEST_R && maxlen > c.B)
     budget_lowest_kernel<<<U, kBudgetThreads, 0, stream>>>(s_full, q_full, lens_dev, c.G, Lmax, Lp2max, c.B, r,
                                                            sortbuf, dst, c.live, c.t_next);
-  else
-    budget_select_kernel<<<U, kBudgetThreads, 0, stream>>>(s_full, q_full, lens_dev, c.G, Lmax, c.B, r, dst, c.live,
-                                                           c.t_next);
+  else {
+    const size_t key_bytes = (size_t)Lmax * 16;
+    if (key_bytes <= 200 * 1024 &&
+        cudaFuncSetAttribute(budget_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)key_bytes) == cudaSuccess)
+      budget_select_kernel<true><<<U, kBudgetThreads, key_bytes, stream>>>(s_full, q_full, lens_dev, c.G, Lmax, c.B,
+                                                                           r, dst, c.live, c.t_next);
+    else
+      budget_select_kernel<false><<<U, kBudgetThreads, 0, stream>>>(s_full, q_full, lens_dev, c.G, Lmax, c.B, r, dst,
+                                                                    c.live, c.t_next);
+  }
   const int span = maxlen > c.B ? maxlen : c.B;
   const int chunks = (span + 63) / 64;
   const unsigned grid = (unsigned)U * (unsigned)chunks;
