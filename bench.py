@@ -33,11 +33,14 @@ import torch
 
 import workloads as W
 
-# dram__bytes_read.sum + dram__bytes_write.sum of decode_step_kernel, per unit (profiles/decode_step_kernel_*.md)
+# dram__bytes_read.sum + dram__bytes_write.sum of decode_step_kernel, per unit, from a profiler capture
 NCU_TRAFFIC = {"kernel_hash": "8076960864a82fcd", "shape": (1024, 128, "bf16"), "dram_bytes_per_unit": 568200}
 
 METRIC = "decode_tokens_per_s"
 UNIT = "tokens/s"
+SCOPE_MODES = {"exclude_top_r": 0, "lowest_r": 1}
+STEP_ORDERS = {"evict_first": 0, "attend_first": 1}
+MIN_WARMUP = 10
 
 
 # ----------------------------------------------------------------------------------------- helpers
@@ -140,8 +143,7 @@ def build_cache(w, device, R, seed_offset=0):
 def oracle_sample(w, cache, sample_units, n_steps, first_step, t_pos):
     """Times the fp64 oracle (as it stands) on `sample_units` of the cache for n_steps decode steps."""
     import oracle
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    from harness import unit_view, widen
+    from workloads import unit_view, widen
     st = oracle.State(widen(unit_view(cache.K, sample_units)), widen(unit_view(cache.V, sample_units)),
                       widen(unit_view(cache.s, sample_units)), widen(unit_view(cache.q, sample_units)),
                       unit_view(cache.n, sample_units).cpu().numpy().copy(),
@@ -374,7 +376,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=256)
-    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=MIN_WARMUP)
     ap.add_argument("--impl", default="roco", choices=["roco", "reference"])
     ap.add_argument("--workload", default="llama7b_decode")
     ap.add_argument("--small", action="store_true", help="1/16 of the units (for profiler captures)")
@@ -382,11 +384,16 @@ def main():
     ap.add_argument("--extras", action="store_true", help="also time the block-wise and grouped-query steps")
     ap.add_argument("--prefill-workload", default="llama7b_prefill", help="workload of the prefill measurement")
     ap.add_argument("--scope-r", type=int, default=None, help="override the workload's scope parameter r")
+    ap.add_argument("--scope-mode", default="exclude_top_r", choices=sorted(SCOPE_MODES),
+                    help="reading of the eviction scope (Sec. 4.3: all but the r highest-variance tokens; Sec. 1: "
+                         "the r lowest-variance tokens)")
+    ap.add_argument("--step-order", default="evict_first", choices=sorted(STEP_ORDERS),
+                    help="order inside a decode step (Fig. 1: evict, insert, attend; or attend, then evict and insert)")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
     if args.impl == "reference" and rank != 0:
         return 0
-    steps, warmup = args.steps, max(args.warmup, 3)
+    steps, warmup = args.steps, max(args.warmup, MIN_WARMUP)
 
     if args.impl == "reference":
         return reference_arm(args, steps, warmup)

@@ -53,6 +53,7 @@ struct DecodeSmem {
   uint64_t *p_ready;       // consumers have left the probabilities in shared memory
   uint64_t *policy_done;   // victim chosen, new K/V written
   uint64_t *stats_full;    // the unit's s, q, n have landed in vkey, mkey, nbuf (bulk copies ahead of the K tiles)
+  uint64_t *v_done;        // consumers have read their last V tile (ATTEND_FIRST: the freed V row may be overwritten)
   int *nbuf;
   int *ctl;                // [0] abort flag, [1] slot of the new token
   float *znew;             // score of the new token (EVICT_FIRST)
@@ -66,7 +67,7 @@ __host__ __device__ inline size_t decode_smem_bytes(int B, int d, int stages, in
   b += sizeof(SelectScratch);
   b += (size_t)(2 + kConsumerWarps) * d * 4;  // qf, vnew, outred
   b += 64 * 4;                                // red
-  b += (2 * (size_t)stages + 3) * sizeof(uint64_t);
+  b += (2 * (size_t)stages + 4) * sizeof(uint64_t);
   b += 8 * 4;
   return b + 128;  // slack for aligning the base
 }
@@ -91,6 +92,7 @@ __device__ inline DecodeSmem carve(char *raw, int B, int d, int stages, int stag
   m.p_ready = (uint64_t *)p; p += sizeof(uint64_t);
   m.policy_done = (uint64_t *)p; p += sizeof(uint64_t);
   m.stats_full = (uint64_t *)p; p += sizeof(uint64_t);
+  m.v_done = (uint64_t *)p; p += sizeof(uint64_t);
   m.ctl = (int *)p; p += 4 * 4;
   m.znew = (float *)p;
   return m;
@@ -143,6 +145,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     mbar_init(sm.p_ready, kConsumerWarps);
     mbar_init(sm.policy_done, 1);
     mbar_init(sm.stats_full, 1);
+    mbar_init(sm.v_done, kConsumerWarps);
     sm.ctl[0] = 0;
     mbar_init_fence();
   }
@@ -251,7 +254,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     }
     int e = live0, ev_slot = -1, ev_pos = -1;
     if (full) {
-      // Sec. 4: "when the buffer is full, an eviction policy is executed"
+      // Sec. 4, fixed-budget buffer: eviction runs only once the buffer is full
       const float *gs = p.s + unit_st, *gq = p.q + unit_st;
       const int *gn = p.n + unit_st, *gpos = p.pos + unit_st;
       if (p.policy == ROCO_POLICY_ROCO) {
@@ -313,6 +316,11 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     if (writes_row) {  // in-place overwrite, 16 bytes per thread
       const int c = ptid - 32;
       const bool isv = c >= kLanesPerRow;
+      // ATTEND_FIRST attends over the cache as it stood before the step (Fig. 1, other order), and the victim's
+      // value row is part of what the producer is still streaming: the row is replaced only once every consumer
+      // warp has its last V tile behind it.  (The K pass has ended by p_ready, so the key row can go at once;
+      // under EVICT_FIRST the consumers take the freed slot's score and value from k_new / v_new instead.)
+      if (isv && !evict_first && full) mbar_wait(sm.v_done, 0, abort_flag, p.status);
       char *dst = const_cast<char *>(isv ? p.V : p.K) + unit_kv + (size_t)e * kRowBytes;
       *((uint4 *)dst + (isv ? c - kLanesPerRow : c)) = row_val;
     }
@@ -437,6 +445,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.empty[st]);
   }
+  if (lane == 0) mbar_arrive(sm.v_done);  // this warp has read its share of every V tile
 #pragma unroll
   for (int i = 0; i < kEPC; ++i) {
 #pragma unroll

@@ -15,6 +15,7 @@ import torch
 
 import oracle
 import paper_2402_06262_b200 as R
+from workloads import unit_view, widen
 
 DELTA = 1e-5
 STAT_RTOL = 1e-4
@@ -23,11 +24,6 @@ LSE_ATOL = 1e-4
 
 def out_tol(dtype) -> float:
     return 2e-2 if dtype == torch.bfloat16 else 1e-5
-
-
-def widen(t: torch.Tensor) -> np.ndarray:
-    """Exact widening of device fp32/bf16 values to float64 on the host."""
-    return t.detach().to("cpu").to(torch.float64).numpy()
 
 
 def assert_stats_close(got, want, what):
@@ -45,10 +41,13 @@ class Tally:
     prefill_swapped: int = 0
 
 
-def unit_view(t: torch.Tensor, units: Sequence[int]) -> torch.Tensor:
-    """Rows of a [S][G][...] tensor for flat unit indices."""
-    flat = t.reshape((-1,) + tuple(t.shape[2:]))
-    return flat[torch.as_tensor(list(units), device=t.device)]
+def state_from_cache(cache: R.Cache, units: Sequence[int]) -> oracle.State:
+    """An oracle state that continues from the device cache of the given units (exact widening)."""
+    return oracle.State(widen(unit_view(cache.K, units)), widen(unit_view(cache.V, units)),
+                        widen(unit_view(cache.s, units)), widen(unit_view(cache.q, units)),
+                        unit_view(cache.n, units).cpu().numpy().copy(), unit_view(cache.pos, units).cpu().numpy().copy(),
+                        unit_view(cache.live, units).cpu().numpy().copy(),
+                        unit_view(cache.t_next, units).cpu().numpy().copy())
 
 
 def compare_state(cache: R.Cache, st: oracle.State, units: Sequence[int], what: str, check_kv=True):

@@ -8,18 +8,10 @@ import torch
 import oracle
 import paper_2402_06262_b200 as R
 import workloads as W
-from harness import DecodeParity, Tally, assert_stats_close, prefill_parity, unit_view, widen
+from harness import DecodeParity, Tally, assert_stats_close, prefill_parity, state_from_cache, unit_view, widen
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-
-
-def state_from_cache(cache, units):
-    return oracle.State(widen(unit_view(cache.K, units)), widen(unit_view(cache.V, units)),
-                        widen(unit_view(cache.s, units)), widen(unit_view(cache.q, units)),
-                        unit_view(cache.n, units).cpu().numpy().copy(), unit_view(cache.pos, units).cpu().numpy().copy(),
-                        unit_view(cache.live, units).cpu().numpy().copy(),
-                        unit_view(cache.t_next, units).cpu().numpy().copy())
 
 
 def check_prefill_properties(sf, qf, lens, G):
