@@ -12,13 +12,15 @@
  *     variance              = max(0, q / n - (s / n)^2)      (Sec. 4.3, Std formula; sqrt is monotone)
  *     eviction scope        = the m lowest-variance cached tokens, order (variance, position):
  *                             m = live - r  (EXCLUDE_TOP_R, Sec. 4.3: exclude the r highest-Std tokens)
- *                             m = r         (LOWEST_R, Sec. 1: "tokens with the lowest variance")
+ *                             m = r         (LOWEST_R, Sec. 1 reading: the scope is the r lowest-variance tokens)
  *                             m is clipped to [1, live]
  *     victim                = the in-scope token of lowest mean, order (mean, position)   (Sec. 4.3)
  *
  * Conventions for every entry point
  *   - All array arguments are DEVICE pointers owned by the caller unless the name ends in _host.
- *     The library allocates no device memory and keeps no state between calls.
+ *     The library allocates no device memory, and keeps no state between calls with two exceptions that are
+ *     described at their entry points: the built-in scratch array of roco_prefill_static, and the copy stream
+ *     with its events that the host-buffer decode calls create per device at first use.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls enqueue work
  *     and return; outputs are valid once the stream reaches that point.  The *_host variants
  *     synchronise the stream before returning.
@@ -131,7 +133,10 @@ roco_status roco_prefill(const void *Q, const void *K, const void *V, const int3
  * the library (every GPU that loads the library holds it until the process exits).  The call allocates
  * nothing.
  *   - Limit: roco_prefill_workspace_bytes(cache, Lmax) must not exceed ROCO_PREFILL_STATIC_SCRATCH_BYTES
- *     (S*G*Lmax up to about 524 000 tokens, e.g. 64 units x 8192); larger problems get ROCO_ERR_WORKSPACE.
+ *     (S*G*Lmax up to about 524 000 tokens, e.g. 63 units x 8192); larger problems get ROCO_ERR_WORKSPACE.
+ *     With ROCO_SCOPE_LOWEST_R and a prompt longer than the budget the need is
+ *     roco_prefill_workspace_bytes_lowest_r(cache, Lmax) (8 more bytes per token, Lmax rounded up to a power of
+ *     two: about 349 000 tokens), checked the same way.
  *   - The first call on a device looks up the array's device address (with that device current); make that
  *     first call before starting any stream capture on the device.
  *   - All calls on a device share the one array, which keeps the previous call's contents (no buffer in it
@@ -144,8 +149,8 @@ roco_status roco_prefill_static(const void *Q, const void *K, const void *V, con
                                 float *lse_out, float *s_full, float *q_full, void *stream);
 
 /*
- * One decode step for every unit (Sec. 3 constrained inference; Sec. 4 "when the buffer is full, an
- * eviction policy is executed"; Sec. 4.3 RoCo rule; Fig. 1 ordering).
+ * One decode step for every unit (Sec. 3 constrained inference; Sec. 4, fixed-budget buffer: eviction runs
+ * once the buffer is full; Sec. 4.3 RoCo rule; Fig. 1 ordering).
  *
  * EVICT_FIRST: if live == B the victim's slot is freed, else slot `live` is taken; the new token's
  * K/V are written there with empty statistics and pos = t_next; the query attends over all occupied
@@ -223,7 +228,8 @@ roco_status roco_block_step(roco_cache *cache, const void *Q, const void *K_new,
  *   b              block size 1..16; r as for roco_block_step (EXCLUDE_TOP_R reading, r + b <= B)
  *   attn_out       [S][G][Lmax][d] attention output of every prompt token over the budgeted cache
  *   evicted_slot   [S][G][b] scratch; on return the slots the last block of each sequence freed (-1 padded)
- * Launches sum_s ceil(lens[s] / b) kernels on the stream.
+ * Launches ceil(len / b) kernels per run of consecutive sequences of equal length (one launch advances the whole
+ * run by a block), so a batch of equal-length prompts costs ceil(len / b) launches in all.
  */
 roco_status roco_prefill_blockwise(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax,
                                    int b, int r, float scale, roco_cache *cache, void *attn_out,
@@ -275,6 +281,24 @@ roco_status roco_decode_step_split(roco_cache *cache, const void *q, const void 
                                    int scope_mode, int splits, float scale, void *attn_out, float *lse_out,
                                    int32_t *evicted_slot, int32_t *evicted_pos, void *workspace,
                                    size_t workspace_bytes, void *stream);
+
+/*
+ * Consistency of an importance score under a budget with its full-cache version (Sec. 4.3, preliminary
+ * experiments, set-up): `full` and `budgeted` are two caches of the same units that have been fed the same tokens
+ * with roco_decode_step_policy under `policy`, `full` with a budget large enough never to evict.  For every unit
+ * the call finds the B = budgeted->live[u] most important tokens of the full cache by the policy's own score
+ * (accumulated score for ROCO_POLICY_H2O, accumulated quantised score for ROCO_POLICY_SCISSORHANDS, last score for
+ * ROCO_POLICY_TOVA, mean attention score for ROCO_POLICY_MAS_WINDOW and ROCO_POLICY_ROCO) -- the tokens left when
+ * the policy's eviction order (score asc, position asc) has removed the rest -- and counts how many of them the
+ * budgeted cache retains.  Both sets have B tokens, so the Jaccard similarity is overlap / (2B - overlap).
+ *
+ *   overlap      [S][G] int32: the count of this call (-1 for a unit whose full cache holds fewer than B tokens)
+ *   jaccard_sum  [S][G] fp32, samples [S][G] int32: running sum of the similarity and number of calls that
+ *                added to it (zero both before the first call; mean similarity = sum / samples)
+ *   full->B <= 8192; full and budgeted have the same S and G; device anomalies go to budgeted->status.
+ */
+roco_status roco_consistency_step(const roco_cache *full, const roco_cache *budgeted, int policy, int32_t *overlap,
+                                  float *jaccard_sum, int32_t *samples, void *stream);
 
 /* Bytes of device staging roco_decode_step_host needs (host function). */
 size_t roco_decode_host_staging_bytes(const roco_cache *cache);

@@ -31,6 +31,11 @@ def lib():
         _lib.roco_oracle_select_to_budget_iterated.restype = C.c_int
         _lib.roco_oracle_attention_row.restype = C.c_double
         _lib.roco_oracle_select_to_budget_onepass.restype = C.c_int
+        _lib.roco_oracle_select_to_budget_guided.restype = C.c_int
+        _lib.roco_oracle_policy_score.restype = C.c_double
+        _lib.roco_oracle_policy_score.argtypes = [C.c_int, C.c_double, C.c_double, C.c_int]
+        _lib.roco_oracle_topb_overlap.restype = C.c_int
+        _lib.roco_oracle_jaccard_equal_sets.restype = C.c_double
         _lib.roco_oracle_prefill_unit.restype = C.c_int
         _lib.roco_oracle_prefill_batch.restype = C.c_int
     return _lib
@@ -101,6 +106,27 @@ def select_to_budget_iterated(s, q, n, B, r, mode, delta=0.0):
     lib().roco_oracle_select_to_budget_iterated(_p(s), _p(q), _p(n), C.c_int(len(s)), C.c_int(B), C.c_int(r),
                                                 C.c_int(mode), C.c_double(delta), _p(keep))
     return keep.astype(bool)
+
+
+def admissible_victims(s, q, n, pos, r, mode, delta=1e-5):
+    """Tokens that could be the victim if every statistic were off by at most the relative margin delta: [len] bool."""
+    s, q, n, pos = _f64(s), _f64(q), _i32(n), _i32(pos)
+    adm = np.zeros(len(s), np.int32)
+    lib().roco_oracle_admissible_victims(_p(s), _p(q), _p(n), _p(pos), C.c_int(len(s)), C.c_int(r), C.c_int(mode),
+                                         C.c_double(delta), _p(adm))
+    return adm.astype(bool)
+
+
+def select_to_budget_guided(s, q, n, B, r, mode, guide_keep, delta=1e-5):
+    """The iterated select-to-budget replayed next to another implementation's survivor set.  Returns
+    (followed, keep): followed = number of in-margin iterations where the guide's choice was taken, or
+    -(iteration + 1) at the first disagreement outside the margin; keep = the replayed survivor set."""
+    s, q, n = _f64(s), _f64(q), _i32(n)
+    guide = _i32(np.asarray(guide_keep).astype(np.int32))
+    keep = np.zeros(len(s), np.int32)
+    rc = lib().roco_oracle_select_to_budget_guided(_p(s), _p(q), _p(n), C.c_int(len(s)), C.c_int(B), C.c_int(r),
+                                                   C.c_int(mode), C.c_double(delta), _p(guide), _p(keep))
+    return int(rc), keep.astype(bool)
 
 
 def select_to_budget_onepass(s, q, n, B, r, delta=1e-5):
@@ -256,3 +282,28 @@ def policy_step(st: State, qv, k_new, v_new, policy, r, scale, rnd=None, delta=1
                                         C.c_double(delta), _p(fv), _p(out), _p(lse), _p(es), _p(ep), _p(ch), _p(nt),
                                         _p(qn))
     return StepResult(out, lse, es, ep, ch, nt.astype(bool)), qn.astype(bool)
+
+
+def policy_score(policy, s, q, n) -> np.ndarray:
+    """Importance score of every token under a Table 1 policy, from the statistics its steps keep."""
+    s, q, n = np.asarray(s, np.float64), np.asarray(q, np.float64), np.asarray(n, np.int32)
+    out = np.zeros(s.shape)
+    for idx in np.ndindex(s.shape):
+        out[idx] = lib().roco_oracle_policy_score(int(policy), float(s[idx]), float(q[idx]), int(n[idx]))
+    return out
+
+
+def topb_overlap(score, pos, kept_pos, delta=1e-5, exact_ties_firm=False):
+    """How many of the B = len(kept_pos) most important tokens (by `score`, ties as the eviction order has them)
+    are among kept_pos.  Returns (overlap, slack): slack bounds the change under score errors within delta."""
+    score, pos, kept = _f64(score), _i32(pos), _i32(kept_pos)
+    slack = C.c_int(0)
+    ov = lib().roco_oracle_topb_overlap(_p(score), _p(pos), C.c_int(len(score)), _p(kept), C.c_int(len(kept)),
+                                        C.c_double(delta), C.c_int(int(exact_ties_firm)), C.byref(slack))
+    return int(ov), int(slack.value)
+
+
+def jaccard_from_overlap(overlap: int, B: int) -> float:
+    """Jaccard similarity of two B-sized sets that share `overlap` elements."""
+    return float(lib().roco_oracle_jaccard_equal_sets(int(overlap), int(B)))
+

@@ -19,7 +19,7 @@
  *   Std ............................ Sec. 4.3: sqrt(Acc^square/Count - (Acc/Count)^2); ranking uses the
  *                                    variance (sqrt is monotone), population form (divide by Count)
  *   eviction scope ................. Sec. 4.3: exclude the r tokens of highest Std (EXCLUDE_TOP_R);
- *                                    Sec. 1: "tokens with the lowest variance" read as the r lowest
+ *                                    Sec. 1 describes the scope as the low-variance tokens, read as the r lowest
  *                                    (LOWEST_R).  Both are "the m lowest-variance tokens" with
  *                                    m = live - r or m = r.
  *   victim ......................... Sec. 4.3: the in-scope token of lowest mean attention score
@@ -29,6 +29,11 @@
  *   block-wise evict-and-encode .... Sec. 5.3 "Overhead", App. B (b tokens freed and encoded per eviction step)
  *   grouped-query attention ........ Sec. 5.3 / App. A (group-wise averaged attention score updates the statistics)
  *   other policies ................. Table 1 with Sec. 4.1 (importance scores), Sec. 4.2 (local window), Sec. 5.1
+ *   consistency diagnostic ......... Sec. 4.3 "Preliminary Experiments", set-up (top-B of a full cache against the
+ *                                    tokens a budgeted cache retains; Jaccard similarity)
+ *   margin analysis ................ the parity rule only (not in the paper): which victims are admissible when the
+ *                                    statistics carry a relative error, and a select-to-budget replay guided by
+ *                                    another implementation's survivor set
  *
  * Readings where the paper is silent (stated once here, in words):
  *   - ties: scope membership by (variance asc, position asc); victim by (mean asc, position asc);
@@ -226,6 +231,97 @@ int roco_oracle_select_to_budget_iterated(const double *s, const double *q, cons
   }
   free(cs); free(cq); free(cn); free(cp);
   return n_near;
+}
+
+/* Which tokens could be the victim if every statistic were off by at most the relative margin delta?
+ * With var_j known only to +-delta*(Acc^square/Count + mean^2) (the uncancelled terms, as in roco_oracle_select)
+ * and mean_j to +-delta*mean_j, token u is *admissible* when (a) it may lie in the scope: fewer than m tokens come
+ * certainly before it in (variance, position) order, and (b) no token that lies in the scope whatever the errors
+ * has a certainly lower mean.  Both conditions are necessary for u to be the rule's choice (Sec. 4.3) under some
+ * error within the margin, so adm[] holds every such choice (and, for delta = 0, the choice alone).  "Certainly
+ * before" between two exactly known, equal values falls to the position, like the rule's own ties.
+ * adm: [live] 0/1.  Tokens with Count = 0 are never admissible (they are not evictable). */
+void roco_oracle_admissible_victims(const double *s, const double *q, const int *n, const int *pos, int live, int r,
+                                    int mode, double delta, int *adm) {
+  double *vlo = (double *)malloc(sizeof(double) * (size_t)(live > 0 ? live : 1) * 4);
+  double *vhi = vlo + live, *mlo = vhi + live, *mhi = mlo + live;
+  int nc = 0;
+  for (int j = 0; j < live; ++j) {
+    adm[j] = 0;
+    if (n[j] <= 0) { vlo[j] = vhi[j] = mlo[j] = mhi[j] = NAN; continue; }
+    double mean = s[j] / n[j], a = q[j] / n[j];
+    double var = a - mean * mean;
+    if (var < 0.0) var = 0.0;
+    double ev = delta * (a + mean * mean), em = delta * mean;
+    vlo[j] = var - ev; vhi[j] = var + ev; mlo[j] = mean - em; mhi[j] = mean + em;
+    ++nc;
+  }
+  if (nc == 0) { free(vlo); return; }
+  int m = (mode == ROCO_ORACLE_EXCLUDE_TOP_R) ? nc - r : r;
+  if (m < 1) m = 1;
+  if (m > nc) m = nc;
+#define CERTAINLY_BEFORE(lo, hi, k, u) \
+  ((hi)[k] < (lo)[u] || ((hi)[k] == (lo)[u] && (lo)[k] == (hi)[k] && (lo)[u] == (hi)[u] && pos[k] < pos[u]))
+  int *sure = (int *)malloc(sizeof(int) * (size_t)live); /* in the scope whatever the errors */
+  for (int k = 0; k < live; ++k) {
+    sure[k] = 0;
+    if (n[k] <= 0) continue;
+    int maybe_before = 0; /* tokens that are not certainly after k */
+    for (int j = 0; j < live; ++j)
+      if (j != k && n[j] > 0 && !CERTAINLY_BEFORE(vlo, vhi, k, j)) ++maybe_before;
+    sure[k] = maybe_before < m;
+  }
+  for (int u = 0; u < live; ++u) {
+    if (n[u] <= 0) continue;
+    int before = 0;
+    for (int k = 0; k < live; ++k)
+      if (k != u && n[k] > 0 && CERTAINLY_BEFORE(vlo, vhi, k, u)) ++before;
+    if (before >= m) continue; /* (a) fails */
+    int beaten = 0;
+    for (int k = 0; k < live && !beaten; ++k)
+      if (k != u && sure[k] && CERTAINLY_BEFORE(mlo, mhi, k, u)) beaten = 1;
+    adm[u] = !beaten;
+  }
+#undef CERTAINLY_BEFORE
+  free(sure); free(vlo);
+}
+
+/* Select-to-budget (iterated form) replayed next to another implementation's survivor set guide_keep[L]: at every
+ * iteration the rule's own victim is taken if the guide evicted it too; otherwise the iteration must be a decision
+ * inside the margin delta, and the admissible victim (see above) first in (mean, position) order among those the
+ * guide evicted is taken instead.  Returns the number of iterations where the guide's choice was followed
+ * (0 = the guide's set is the rule's own), or -(iteration + 1) at the first iteration where the guide kept the
+ * rule's victim and evicted no admissible one: a disagreement outside the margin.  keep[L] receives the replayed
+ * survivor set, equal to guide_keep on success when that holds exactly B (or L, if L <= B) tokens. */
+int roco_oracle_select_to_budget_guided(const double *s, const double *q, const int *n, int L, int B, int r,
+                                        int mode, double delta, const int *guide_keep, int *keep) {
+  for (int j = 0; j < L; ++j) keep[j] = 1;
+  if (L <= B) return 0;
+  double *cs = (double *)malloc(sizeof(double) * (size_t)L), *cq = (double *)malloc(sizeof(double) * (size_t)L);
+  int *cn = (int *)malloc(sizeof(int) * (size_t)L), *cp = (int *)malloc(sizeof(int) * (size_t)L);
+  int *adm = (int *)malloc(sizeof(int) * (size_t)L);
+  int followed = 0, rc = 0;
+  for (int alive = L, it = 0; alive > B; --alive, ++it) {
+    int k = 0;
+    for (int j = 0; j < L; ++j)
+      if (keep[j]) { cs[k] = s[j]; cq[k] = q[j]; cn[k] = n[j]; cp[k] = j; ++k; }
+    int c = roco_oracle_select(cs, cq, cn, cp, alive, r, mode, delta, NULL, NULL);
+    if (guide_keep[cp[c]]) { /* the guide kept the rule's victim: look for the admissible one it evicted */
+      roco_oracle_admissible_victims(cs, cq, cn, cp, alive, r, mode, delta, adm);
+      int alt = -1;
+      for (int i = 0; i < alive; ++i) {
+        if (!adm[i] || guide_keep[cp[i]]) continue;
+        double mi = cs[i] / cn[i];
+        if (alt < 0 || mi < cs[alt] / cn[alt] || (mi == cs[alt] / cn[alt] && cp[i] < cp[alt])) alt = i;
+      }
+      if (alt < 0) { rc = -(it + 1); break; }
+      c = alt;
+      ++followed;
+    }
+    keep[cp[c]] = 0;
+  }
+  free(cs); free(cq); free(cn); free(cp); free(adm);
+  return rc ? rc : followed;
 }
 
 typedef struct { double key; double eps; int pos; } rank_t;
@@ -696,3 +792,64 @@ void roco_oracle_policy_step_batch(int U, double *K, double *V, double *s, doubl
                                  evicted_pos + u, choice + u, near_tie + u, quant_near ? quant_near + sb : NULL);
   }
 }
+
+/* ------------------------------ consistency with the full cache (Sec. 4.3 "Preliminary Experiments", set-up) -- */
+
+/* The importance score a policy ranks the cached tokens by (Sec. 4.1; MAS: Sec. 4.3), from the statistics the
+ * policy step keeps: AAS = Acc (H2O), AQAS = the accumulated quantised score (ScissorHands, kept in q), LTAS = the
+ * last query's probability (TOVA, kept in q), MAS = Acc / Count (RoCo and MAS + window; 0 while Count = 0). */
+double roco_oracle_policy_score(int policy, double s, double q, int n) {
+  if (policy == ROCO_ORACLE_POLICY_H2O) return s;
+  if (policy == ROCO_ORACLE_POLICY_SCISSORHANDS || policy == ROCO_ORACLE_POLICY_TOVA) return q;
+  return n > 0 ? s / n : 0.0;
+}
+
+typedef struct { double score; int pos; } scored_t;
+static int cmp_score_pos(const void *a, const void *b) {
+  const scored_t *x = (const scored_t *)a, *y = (const scored_t *)b;
+  if (x->score < y->score) return -1;
+  if (x->score > y->score) return 1;
+  return (x->pos > y->pos) - (x->pos < y->pos);
+}
+
+/* The B most important tokens of a full cache are the ones left when the policy's eviction order -- (score asc,
+ * position asc) -- has removed live - B tokens: the last B in that order.  Returns how many of them are among
+ * kept_pos[B] (the positions a budgeted cache retains); the Jaccard similarity of the two B-sized sets is
+ * overlap / (2B - overlap).  *slack (may be NULL) bounds by how much that count can move if every score is off by
+ * at most the relative margin delta: the smaller of the number of top-B tokens within the margin of the best
+ * excluded score and the number of excluded tokens within the margin of the worst included score (scores exactly
+ * equal to the other side's boundary count as within the margin unless exact_ties_firm, for integer-valued
+ * scores, where equal values are ordered by position on every implementation alike).  live >= B >= 1. */
+int roco_oracle_topb_overlap(const double *score, const int *pos, int live, const int *kept_pos, int B, double delta,
+                             int exact_ties_firm, int *slack) {
+  scored_t *c = (scored_t *)malloc(sizeof(scored_t) * (size_t)live);
+  for (int j = 0; j < live; ++j) { c[j].score = score[j]; c[j].pos = pos[j]; }
+  qsort(c, (size_t)live, sizeof(scored_t), cmp_score_pos);
+  const int cut = live - B; /* c[cut..live) is the top-B set */
+  int overlap = 0;
+  for (int k = cut; k < live; ++k)
+    for (int i = 0; i < B; ++i)
+      if (kept_pos[i] == c[k].pos) { ++overlap; break; }
+  if (slack) {
+    *slack = 0;
+    if (cut > 0) {
+      const double best_out = c[cut - 1].score, worst_in = c[cut].score;
+      int near_in = 0, near_out = 0;
+      for (int k = cut; k < live; ++k) {
+        const double gap = c[k].score - best_out;
+        if (gap <= delta * (fabs(c[k].score) + fabs(best_out)) && !(exact_ties_firm && gap == 0.0)) ++near_in;
+      }
+      for (int k = 0; k < cut; ++k) {
+        const double gap = worst_in - c[k].score;
+        if (gap <= delta * (fabs(c[k].score) + fabs(worst_in)) && !(exact_ties_firm && gap == 0.0)) ++near_out;
+      }
+      *slack = near_in < near_out ? near_in : near_out;
+    }
+  }
+  free(c);
+  return overlap;
+}
+
+/* Jaccard similarity |X and Y| / |X or Y| of two sets of B elements each that share `overlap` elements. */
+double roco_oracle_jaccard_equal_sets(int overlap, int B) { return (double)overlap / (double)(2 * B - overlap); }
+

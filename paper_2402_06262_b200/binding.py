@@ -26,7 +26,8 @@ EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes",
            "roco_block_step", "roco_gqa_decode_step", "roco_decode_step_policy",
            "roco_decode_split_workspace_bytes", "roco_decode_step_split", "roco_prefill_blockwise",
            "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status",
-           "roco_prefill_attend_workspace_bytes", "roco_prefill_attend", "roco_selftest_wait_timeout")
+           "roco_prefill_attend_workspace_bytes", "roco_prefill_attend", "roco_selftest_wait_timeout",
+           "roco_consistency_step")
 
 
 class RocoError(RuntimeError):
@@ -101,6 +102,9 @@ def lib() -> C.CDLL:
         L.roco_decode_step_host.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                             C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_size_t, C.c_void_p]
+        L.roco_consistency_step.restype = C.c_int
+        L.roco_consistency_step.argtypes = [C.POINTER(roco_cache), C.POINTER(roco_cache), C.c_int, C.c_void_p,
+                                            C.c_void_p, C.c_void_p, C.c_void_p]
         L.roco_selftest_wait_timeout.restype = C.c_int
         L.roco_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.roco_device_status.restype = C.c_int
@@ -290,6 +294,15 @@ def roco_gqa_decode_step(cache: Cache, Q, k_new, v_new, r: int, attn_out, evicte
                                     _ptr(evicted_pos), _stream())
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_gqa_decode_step")
+
+
+def roco_consistency_step(full: Cache, budgeted: Cache, policy: int, overlap, jaccard_sum, samples):
+    """Overlap of the budgeted cache's retained tokens with the full cache's top-B by the policy's score, per unit
+    (overlap [S][G] int32), accumulated as Jaccard similarity into jaccard_sum [S][G] fp32 / samples [S][G] int32."""
+    rc = lib().roco_consistency_step(C.byref(full.c), C.byref(budgeted.c), policy, _ptr(overlap), _ptr(jaccard_sum),
+                                     _ptr(samples), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_consistency_step")
 
 
 def roco_decode_host_staging_bytes(cache: Cache) -> int:

@@ -283,23 +283,28 @@ roco_status roco_prefill_blockwise(const void *Q, const void *K, const void *V, 
     if (lens_host[s] < 1 || lens_host[s] > Lmax) return ROCO_ERR_INVALID_ARG;
   const size_t elem = cache->kv_dtype == ROCO_BF16 ? 2 : 4;
   const size_t G = (size_t)cache->G, B = (size_t)cache->B, d = (size_t)cache->d;
-  for (int s = 0; s < cache->S; ++s) {
-    roco_cache sub = *cache;  // the units of sequence s
-    sub.S = 1;
-    sub.K = static_cast<char *>(cache->K) + s * G * B * d * elem;
-    sub.V = static_cast<char *>(cache->V) + s * G * B * d * elem;
-    sub.s = cache->s + s * G * B; sub.q = cache->q + s * G * B;
-    sub.n = cache->n + s * G * B; sub.pos = cache->pos + s * G * B;
-    sub.live = cache->live + s * G; sub.t_next = cache->t_next + s * G;
-    for (int t0 = 0; t0 < lens_host[s]; t0 += b) {
-      const int m = lens_host[s] - t0 < b ? lens_host[s] - t0 : b;
-      const size_t off = ((size_t)s * G * Lmax + t0) * d * elem;
+  // Consecutive sequences of equal length advance together: one launch per block for the whole run.
+  for (int s0 = 0; s0 < cache->S;) {
+    int s1 = s0 + 1;
+    while (s1 < cache->S && lens_host[s1] == lens_host[s0]) ++s1;
+    const int len = lens_host[s0];
+    roco_cache sub = *cache;  // the units of sequences s0 .. s1 - 1
+    sub.S = s1 - s0;
+    sub.K = static_cast<char *>(cache->K) + s0 * G * B * d * elem;
+    sub.V = static_cast<char *>(cache->V) + s0 * G * B * d * elem;
+    sub.s = cache->s + s0 * G * B; sub.q = cache->q + s0 * G * B;
+    sub.n = cache->n + s0 * G * B; sub.pos = cache->pos + s0 * G * B;
+    sub.live = cache->live + s0 * G; sub.t_next = cache->t_next + s0 * G;
+    for (int t0 = 0; t0 < len; t0 += b) {
+      const int m = len - t0 < b ? len - t0 : b;
+      const size_t off = ((size_t)s0 * G * Lmax + t0) * d * elem;
       st = launch_multi_step(sub, 0, m, m, static_cast<const char *>(Q) + off, static_cast<const char *>(K) + off,
                              static_cast<const char *>(V) + off, r, ROCO_SCOPE_EXCLUDE_TOP_R, scale,
-                             static_cast<char *>(attn_out) + off, nullptr, evicted_slot + (size_t)s * G * b, nullptr,
+                             static_cast<char *>(attn_out) + off, nullptr, evicted_slot + (size_t)s0 * G * b, nullptr,
                              static_cast<cudaStream_t>(stream), Lmax);
       if (st != ROCO_OK) return st;
     }
+    s0 = s1;
   }
   return ROCO_OK;
 }
@@ -317,6 +322,21 @@ roco_status roco_gqa_decode_step(roco_cache *cache, const void *Q, const void *k
   if (group > multi_max_queries() || !multi_fits(cache->B, cache->d, group, 1)) return ROCO_ERR_UNSUPPORTED;
   return launch_multi_step(*cache, 1, group, 1, Q, k_new, v_new, r, scope_mode, scale, attn_out, lse_out,
                            evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
+}
+
+roco_status roco_consistency_step(const roco_cache *full, const roco_cache *budgeted, int policy, int32_t *overlap,
+                                  float *jaccard_sum, int32_t *samples, void *stream) {
+  NvtxRange range("roco_consistency_step");
+  roco_status st = check_cache(full);
+  if (st != ROCO_OK) return st;
+  if ((st = check_cache(budgeted)) != ROCO_OK) return st;
+  if (!overlap || !jaccard_sum || !samples) return ROCO_ERR_INVALID_ARG;
+  if (full->S != budgeted->S || full->G != budgeted->G || full->B < budgeted->B) return ROCO_ERR_INVALID_ARG;
+  if (policy != ROCO_POLICY_ROCO && policy != ROCO_POLICY_SCISSORHANDS && policy != ROCO_POLICY_H2O &&
+      policy != ROCO_POLICY_TOVA && policy != ROCO_POLICY_MAS_WINDOW)
+    return ROCO_ERR_INVALID_ARG;  // the other policies have no attention-based score
+  return launch_consistency_step(*full, *budgeted, policy, overlap, jaccard_sum, samples,
+                                 static_cast<cudaStream_t>(stream));
 }
 
 size_t roco_decode_host_staging_bytes(const roco_cache *cache) {

@@ -63,4 +63,9 @@ roco_status launch_multi_step(const roco_cache &c, int kind, int M, int nb, cons
 // unit_stride_rows > 0: Q, k_new, v_new and out are slices of [U][rows][d] tensors with that many rows per unit
 // (used to step through a prompt block by block); 0: dense [U][M][d] / [U][nb][d].
 
+// Overlap of the budgeted cache's retained positions with the full cache's B most important tokens (one CTA per
+// unit; full.B * 8 bytes of shared memory).
+roco_status launch_consistency_step(const roco_cache &full, const roco_cache &budgeted, int policy, int32_t *overlap,
+                                    float *jaccard_sum, int32_t *samples, cudaStream_t stream);
+
 }  // namespace roco

@@ -39,6 +39,8 @@ class Tally:
     near_tie_disagreements: int = 0
     prefill_uncertain: int = 0
     prefill_swapped: int = 0
+    prefill_units_evicting: int = 0     # units whose prompt exceeded the budget
+    prefill_units_firm: int = 0         # ... of which the survivor set equalled the oracle's own, token for token
 
 
 def state_from_cache(cache: R.Cache, units: Sequence[int]) -> oracle.State:
@@ -72,7 +74,7 @@ def compare_state(cache: R.Cache, st: oracle.State, units: Sequence[int], what: 
 
 
 def prefill_parity(cache: R.Cache, Q, K, V, lens: Sequence[int], r: int, scope_mode: int, units: Sequence[int],
-                   tally: Tally, scale: Optional[float] = None) -> oracle.State:
+                   tally: Tally, scale: Optional[float] = None, static: bool = False) -> oracle.State:
     """Runs roco_prefill on the device tensors Q,K,V [S][G][Lmax][d], the oracle on the sampled units, compares,
     and returns the oracle state (continued from the GPU's survivor set where that differs inside the margin)."""
     S, G, Lmax, d = Q.shape
@@ -82,7 +84,8 @@ def prefill_parity(cache: R.Cache, Q, K, V, lens: Sequence[int], r: int, scope_m
     lse = torch.zeros(S, G, Lmax, dtype=torch.float32, device=dev)
     sf = torch.zeros_like(lse)
     qf = torch.zeros_like(lse)
-    R.roco_prefill(Q, K, V, lens, B, r, cache, scope_mode=scope_mode, scale=scale, lse_out=lse, s_full=sf, q_full=qf)
+    (R.roco_prefill_static if static else R.roco_prefill)(Q, K, V, lens, B, r, cache, scope_mode=scope_mode, scale=scale,
+                                                          lse_out=lse, s_full=sf, q_full=qf)
     torch.cuda.synchronize()
     assert R.roco_device_status(cache) == 0
     ulens = [int(lens[u // G]) for u in units]
@@ -102,11 +105,23 @@ def prefill_parity(cache: R.Cache, Q, K, V, lens: Sequence[int], r: int, scope_m
         gkeep = np.zeros(Lmax, bool)
         gkeep[kept] = True
         diff = gkeep[:L] != res.keep[i, :L]
-        tally.prefill_uncertain += int(res.uncertain[i].sum())
-        if diff.any():
+        tally.prefill_units_evicting += int(L > B)
+        tally.prefill_units_firm += int(L > B and not diff.any())
+        if diff.any() and scope_mode == R.ROCO_SCOPE_LOWEST_R:
+            # iterated form: replay the evictions next to the GPU's set; it may be followed only at iterations
+            # inside the margin, and only to a token that could be the victim there
+            followed, keep = oracle.select_to_budget_guided(res.s_full[i, :L], res.q_full[i, :L], res.n_full[i, :L],
+                                                            B, r, scope_mode, gkeep[:L], delta=DELTA)
+            assert followed >= 0, (f"unit {units[i]}: eviction {-followed - 1} of the replay differs outside the "
+                                   f"{DELTA} margin")
+            assert np.array_equal(keep, gkeep[:L])
+            tally.prefill_swapped += followed
+        elif diff.any():
+            tally.prefill_uncertain += int(res.uncertain[i].sum())
             assert np.all(res.uncertain[i, :L][diff]), \
                 f"unit {units[i]}: survivor sets differ outside the {DELTA} margin at {np.nonzero(diff)[0]}"
             tally.prefill_swapped += int(diff.sum())
+        if diff.any():
             if force is None:
                 force = res.keep.copy()
             force[i] = gkeep

@@ -73,7 +73,10 @@ def test_prefill_eviction_structured(kind):
 def test_prefill_eviction_lowest_r(r):
     """LOWEST_R at prefill: the evictions are replayed one by one on frozen statistics (sorted scope order)."""
     w = W.scaled(W.LLAMA7B_PREFILL, S=3, layers=1, heads=3, prompt_lo=700, prompt_hi=700, B=200, r=r, kind="sink")
-    run_workload(w, range(w.U), R.ROCO_SCOPE_LOWEST_R, R.ROCO_EVICT_FIRST, 6, lens=[700, 333, 65], check_every=3)
+    t = run_workload(w, range(w.U), R.ROCO_SCOPE_LOWEST_R, R.ROCO_EVICT_FIRST, 6, lens=[700, 333, 65], check_every=3)
+    # six units evict (prompts of 700 and 333 tokens); most survivor sets equal the oracle's token for token, and
+    # where they do not, each differing eviction was replayed inside the margin
+    assert t.prefill_units_evicting == 6 and t.prefill_units_firm >= 4 and t.prefill_swapped <= 4, t
 
 
 def test_prefill_keeps_everything_when_budget_not_binding():

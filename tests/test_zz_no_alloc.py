@@ -13,6 +13,7 @@ import torch
 
 import paper_2402_06262_b200 as R
 import workloads as W
+from harness import Tally, prefill_parity
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -73,3 +74,39 @@ def test_oversized_problem_is_rejected_with_the_workspace_error():
                                      Lmax, w.B, w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, 1, 0.1, C.byref(cache.c), None, None,
                                      None, None)
     assert rc == 3 and "workspace" in R.status_string(rc)
+
+
+@pytest.mark.parametrize("mode,r", [(R.ROCO_SCOPE_EXCLUDE_TOP_R, 20), (R.ROCO_SCOPE_LOWEST_R, 20)])
+def test_static_call_against_the_oracle_and_allocates_nothing(mode, r):
+    """The built-in-scratch call compared with the fp64 oracle directly (both scope readings; LOWEST_R also needs
+    the sort buffer, which fits here), and a repeat of the call leaves the device's free memory and torch's
+    allocator untouched."""
+    w = W.scaled(W.LLAMA7B_PREFILL, S=2, layers=1, heads=3, prompt_lo=500, prompt_hi=500, B=160, r=r, seed=21)
+    lens = [500, 301]
+    Q, K, V = (torch.stack(x) for x in zip(*[W.prompt_chunk(w, b, 0, w.G, 500, DEV) for b in range(w.S)]))
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    tally = Tally()
+    prefill_parity(cache, Q, K, V, lens, r, mode, range(w.U), tally, scale=w.scale, static=True)
+    assert tally.prefill_units_evicting == w.U
+    torch.cuda.synchronize()
+    free0, alloc0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+    R.roco_prefill_static(Q, K, V, lens, w.B, r, cache, scope_mode=mode, scale=w.scale)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0
+    assert R.roco_device_status(cache) == 0
+
+
+def test_lowest_r_needs_more_scratch_and_is_rejected_earlier():
+    """Under ROCO_SCOPE_LOWEST_R a prompt longer than the budget also needs the sort buffer: a problem that fits
+    under the other reading is rejected with the workspace status."""
+    w = W.scaled(W.LLAMA7B_PREFILL, S=1, layers=1, heads=48, prompt_lo=8192, prompt_hi=8192, B=2048, r=256)
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    assert R.roco_prefill_workspace_bytes(cache, 8192) <= R.binding.PREFILL_STATIC_SCRATCH_BYTES
+    assert R.roco_prefill_workspace_bytes_lowest_r(cache, 8192) > R.binding.PREFILL_STATIC_SCRATCH_BYTES
+    Q, K, V = (t[None] for t in W.prompt_chunk(w, 0, 0, w.G, 8192, DEV))
+    R.roco_prefill_static(Q, K, V, [8192], w.B, w.r, cache, scale=w.scale)            # fits
+    with pytest.raises(R.RocoError) as e:
+        R.roco_prefill_static(Q, K, V, [8192], w.B, w.r, cache, scope_mode=R.ROCO_SCOPE_LOWEST_R, scale=w.scale)
+    assert e.value.code == 3
+    torch.cuda.synchronize()
+    assert R.roco_device_status(cache) == 0
