@@ -8,6 +8,11 @@ evicted to B = 1024).  `value` is decode tokens/s of the attention path (one ste
 all layers*heads units of each sequence).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+                    [--scope-mode exclude_top_r|lowest_r] [--step-order evict_first|attend_first]
+                    [--all-workloads] [--readings] [--extras]
+
+`--readings` adds the three other combinations of scope reading and step order on the same workload, and
+`--all-workloads` the serving-batch and long-context decode workloads, as extra keys of the same line.
 
 N > 1 (under torch.distributed.run): every rank runs the same-sized workload on its own GPU with its own
 seed (units are independent; no data-path collective) and the aggregate is reported: weak scaling.
@@ -34,12 +39,14 @@ import torch
 import workloads as W
 
 # dram__bytes_read.sum + dram__bytes_write.sum of decode_step_kernel, per unit, from a profiler capture
-NCU_TRAFFIC = {"kernel_hash": "8076960864a82fcd", "shape": (1024, 128, "bf16"), "dram_bytes_per_unit": 568200}
+NCU_TRAFFIC = {"kernel_hash": "3bbbd0bf6fecb045", "shape": (1024, 128, "bf16"), "dram_bytes_per_unit": 569470}
 
 METRIC = "decode_tokens_per_s"
 UNIT = "tokens/s"
 SCOPE_MODES = {"exclude_top_r": 0, "lowest_r": 1}
 STEP_ORDERS = {"evict_first": 0, "attend_first": 1}
+MODE_NAMES = {0: "EXCLUDE_TOP_R", 1: "LOWEST_R"}
+ORDER_NAMES = {0: "EVICT_FIRST", 1: "ATTEND_FIRST"}
 MIN_WARMUP = 10
 
 
@@ -117,7 +124,7 @@ def aggregate(tokens_per_rank: float, seconds_this_rank: float, world: int, back
 
 # ----------------------------------------------------------------------------------------- workload
 
-def build_cache(w, device, R, seed_offset=0):
+def build_cache(w, device, R, seed_offset=0, scope_mode=0):
     """Prefill every unit with the library (prompt -> budget B), layer-chunk by layer-chunk."""
     w = W.scaled(w, seed=w.seed + 1000 * seed_offset)
     cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, device)
@@ -129,10 +136,10 @@ def build_cache(w, device, R, seed_offset=0):
             g1 = min(g0 + chunk, w.G)
             Q, K, V = (t[None] for t in W.prompt_chunk(w, b, g0, g1, lens[b], device))
             sub = R.Cache(1, g1 - g0, w.B, w.d, w.torch_dtype, device)
-            need = R.roco_prefill_workspace_bytes(sub, lens[b])
+            need = (R.roco_prefill_workspace_bytes_lowest_r if scope_mode else R.roco_prefill_workspace_bytes)(sub, lens[b])
             if ws is None or ws.numel() < need:
                 ws = torch.empty(need, dtype=torch.uint8, device=device)
-            R.roco_prefill(Q, K, V, [lens[b]], w.B, w.r, sub, scale=w.scale, workspace=ws)
+            R.roco_prefill(Q, K, V, [lens[b]], w.B, w.r, sub, scope_mode=scope_mode, scale=w.scale, workspace=ws)
             for name in ("K", "V", "s", "q", "n", "pos", "live", "t_next"):
                 getattr(cache, name)[b, g0:g1].copy_(getattr(sub, name)[0])
             if R.roco_device_status(sub) != 0:
@@ -140,7 +147,7 @@ def build_cache(w, device, R, seed_offset=0):
     return w, cache, lens
 
 
-def oracle_sample(w, cache, sample_units, n_steps, first_step, t_pos):
+def oracle_sample(w, cache, sample_units, n_steps, first_step, t_pos, scope_mode=0, step_order=0):
     """Times the fp64 oracle (as it stands) on `sample_units` of the cache for n_steps decode steps."""
     import oracle
     from workloads import unit_view, widen
@@ -159,12 +166,25 @@ def oracle_sample(w, cache, sample_units, n_steps, first_step, t_pos):
     per_step = []
     for q, k, v in toks:
         t0 = time.perf_counter()
-        oracle.decode_step(st, q, k, v, w.r, oracle.EXCLUDE_TOP_R, oracle.EVICT_FIRST, w.scale)
+        oracle.decode_step(st, q, k, v, w.r, scope_mode, step_order, w.scale)
         per_step.append(time.perf_counter() - t0)
     return per_step, oracle.threads()
 
 
-def prefill_bench(R, device, small=False, reps=3, workload="llama7b_prefill"):
+def prefill_oracle_baseline(w, L, n_units=16):
+    """The fp64 oracle's prefill (statistics + select-to-budget) on `n_units` units of the prompt workload, timed
+    on the host cores; returns the cpu_baseline block (prompt tokens/s of the whole workload, scaled by U/sample)."""
+    import oracle
+    Q, K, V = (x.to(torch.float64).numpy() for x in W.prompt_chunk(w, 0, 0, n_units, L, "cpu"))
+    t0 = time.perf_counter()
+    oracle.prefill(Q, K, V, [L] * n_units, w.B, w.r, oracle.EXCLUDE_TOP_R, w.scale)
+    sec = time.perf_counter() - t0
+    return {"value": W.ALL[w.name].S * L / (sec * W.ALL[w.name].U / n_units), "unit": "prompt tokens/s",
+            "cores": oracle.threads(), "kind": "oracle", "seconds": sec,
+            "sample": f"{n_units} of {W.ALL[w.name].U} units, whole prompt of {L} tokens each; scaled by U/sample"}
+
+
+def prefill_bench(R, device, small=False, reps=5, workload="llama7b_prefill", with_oracle=False):
     """Prefill-stage statistics + eviction to budget on the Llama-2-7B-shape prompt workload (8192-token causal
     prompt, 32 x 32 heads, evicted to B = 2048 with r = 256): best of `reps` calls of roco_prefill.  Workloads whose
     prompts do not fit at once (long_context: 32768 tokens x 4096 units) are measured on one sequence's first 8
@@ -230,7 +250,23 @@ def prefill_bench(R, device, small=False, reps=3, workload="llama7b_prefill"):
             "frac_executed": executed / best / 1e12 / bf16_peak,
             "frac_algorithmic": algorithmic / best / 1e12 / bf16_peak,
             "launches_per_call": 4, "timing": f"best of {reps} whole roco_prefill calls (both passes, select, gather)",
-            "attention_output": attend}
+            "exp_unit_bound": exp_unit_bound(w.U, T, best), "attention_output": attend,
+            "cpu_baseline": prefill_oracle_baseline(w, L, 64 if L <= 8192 else 8) if with_oracle else None}
+
+
+def exp_unit_bound(U, T, seconds):
+    """What the exponentials alone cost: both passes evaluate one exponential per score, 128 x 128 per tile
+    product; the SM's exponential unit retires 16 per cycle, and the kernels move two of every eight onto the
+    FMA pipe.  At the maximum SM clock, all SMs busy."""
+    p = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(
+        os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+    mhz, sms = float(p.get("sm_max_mhz", 1965.0)), 148
+    tiles = 2 * U * (T * (T + 1) // 2)
+    ms = tiles * (128 * 128 / 16) * 0.75 / (sms * mhz * 1e3)
+    return {"ms": ms, "frac_of_measured_time": ms / (seconds * 1e3),
+            "note": "16384 exponentials per tile product / 16 per cycle per SM x 0.75 (a quarter runs as a "
+                    "polynomial on the FMA pipe), 148 SMs at the maximum SM clock; the MMA work of the same tile "
+                    "is 512 cycles"}
 
 
 def multi_bench(R, cache, w, device, reps=6):
@@ -327,11 +363,11 @@ def multi_bench(R, cache, w, device, reps=6):
     return res
 
 
-def describe(w, world):
+def describe(w, world, scope_mode=0, step_order=0):
     elem = 2 if w.dtype == "bf16" else 4
     return {"workload": f"{w.name}: S={w.S} x {w.layers} layers x {w.heads} heads, d={w.d}, {w.dtype}, "
                         f"prompt {w.prompt_lo}" + (f"-{w.prompt_hi}" if w.prompt_hi != w.prompt_lo else "") +
-                        f" -> B={w.B}, r={w.r}, EXCLUDE_TOP_R, EVICT_FIRST",
+                        f" -> B={w.B}, r={w.r}, {MODE_NAMES[scope_mode]}, {ORDER_NAMES[step_order]}",
             "units": w.U, "budget": w.B, "scope_r": w.r,
             "l2": "inputs larger than L2 (K+V cache per step %.2f GB)" % (w.U * 2 * w.B * w.d * elem / 1e9),
             "parallelism": f"units sharded over {world} GPU(s), no collective" if world > 1 else "1 GPU"}
@@ -345,14 +381,15 @@ def reference_arm(args, steps, warmup):
     n_units = min(w.G, 32)
     lens = W.prompt_lens(w)
     Q, K, V = (x[None].to(torch.float64).numpy() for x in W.prompt_chunk(w, 0, 0, n_units, lens[0], "cpu"))
-    res = oracle.prefill(Q[0], K[0], V[0], [lens[0]] * n_units, w.B, w.r, oracle.EXCLUDE_TOP_R, w.scale)
+    mode, order = SCOPE_MODES[args.scope_mode], STEP_ORDERS[args.step_order]
+    res = oracle.prefill(Q[0], K[0], V[0], [lens[0]] * n_units, w.B, w.r, mode, w.scale)
     st = res.state
     per_step = []
     tp = list(lens)
     for i in range(warmup + steps):
         q, k, v = (x[0, :n_units].to(torch.float64).numpy() for x in W.decode_tokens(w, i, tp, "cpu"))
         t0 = time.perf_counter()
-        oracle.decode_step(st, q, k, v, w.r, oracle.EXCLUDE_TOP_R, oracle.EVICT_FIRST, w.scale)
+        oracle.decode_step(st, q, k, v, w.r, mode, order, w.scale)
         per_step.append(time.perf_counter() - t0)
         tp = [t + 1 for t in tp]
     timed = per_step[warmup:]
@@ -361,13 +398,161 @@ def reference_arm(args, steps, warmup):
     cores = oracle.threads()
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
             "warmup": warmup, "ms_per_step": 1e3 * sec / len(timed) * w.U / n_units, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": describe(w, 1),
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": describe(w, 1, mode, order),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": f"{n_units} of {w.U} units, every step; time scaled by U/sample"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
     return 0
+
+
+
+
+# ----------------------------------------------------------------------------------------- decode measurement
+
+def kernel_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for fn in ("decode.cu", "select.cuh", "common.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_2402_06262_b200", "csrc", fn), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def read_stream_gbs(R, device, gib=4, reps=5):
+    """Read-only streaming rate of this GPU: the library's own sum-over-a-buffer kernel over `gib` GiB, best of reps."""
+    buf = torch.empty(gib << 30, dtype=torch.uint8, device=device)
+    buf.fill_(1)
+    sink = torch.zeros(1, dtype=torch.int64, device=device)
+    R.roco_selftest_read_stream(buf, sink)
+    torch.cuda.synchronize()
+    best = float("inf")
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); R.roco_selftest_read_stream(buf, sink); e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1) / 1e3)
+    n = buf.numel()
+    del buf
+    torch.cuda.empty_cache()
+    return n / best / 1e9
+
+
+def decode_bench(R, w0, device, rank, world, local_rank, steps, warmup, scope_mode, step_order, e2e_steps=32,
+                 clocks=True, read_gbs=None):
+    """Builds the workload's cache with the library's prefill, then times `steps` decode steps (one launch each)
+    after `warmup` untimed ones, device-timed per launch; then the end-to-end rate through the host-buffer entry
+    points.  Returns (result dict, workload, cache, lens, steps consumed)."""
+    w, cache, lens = build_cache(w0, device, R, seed_offset=rank, scope_mode=scope_mode)
+    elem = 2 if w.dtype == "bf16" else 4
+    total = warmup + steps
+    t_pos = list(lens)
+    toks, tp = [], list(t_pos)
+    for i in range(total):                      # inputs of every step resident on the device before the timed region
+        toks.append(W.decode_tokens(w, i, tp, device))
+        tp = [t + 1 for t in tp]
+    out = torch.zeros(w.S, w.G, w.d, dtype=w.torch_dtype, device=device)
+    ev_slot = torch.zeros(w.S, w.G, dtype=torch.int32, device=device)
+    ev_pos = torch.zeros_like(ev_slot)
+
+    def step(i):
+        q, k, v = toks[i]
+        R.roco_decode_step(cache, q, k, v, w.r, out, ev_slot, ev_pos, scope_mode=scope_mode, step_order=step_order,
+                           scale=w.scale)
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+    sampler = None
+    if clocks:
+        visible = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
+        sampler = ClockSampler(visible[local_rank] if local_rank < len(visible) else local_rank)
+        sampler.start()
+        time.sleep(0.3)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    torch.cuda.synchronize()
+    t_wall0 = time.perf_counter()
+    evs[0].record()
+    for i in range(steps):
+        step(warmup + i)
+        evs[i + 1].record()
+    torch.cuda.synchronize()
+    t_wall1 = time.perf_counter()
+    if world > 1:
+        torch.distributed.barrier()
+    clk = sampler.stop(t_wall0, t_wall1) if sampler else None
+    launch_ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
+    sec = evs[0].elapsed_time(evs[steps]) / 1e3
+    if R.roco_device_status(cache) != 0:
+        raise RuntimeError("device status word set during the timed region")
+    value, tmax = aggregate(w.S * steps, sec, world, device)
+    del toks
+
+    # ---- end to end: pinned host tensors in, results out, every step, through the public host-buffer entry points
+    # (two steps in flight: the copies of one step run under the kernel of the other), and through the
+    # synchronising single call beside it
+    h_toks = [tuple(x.cpu().pin_memory() for x in W.decode_tokens(w, total + i, [t + total + i for t in t_pos], device))
+              for i in range(2 * e2e_steps)]
+    h_res = [(torch.zeros(w.S, w.G, w.d, dtype=w.torch_dtype).pin_memory(),
+              torch.zeros(w.S, w.G, dtype=torch.int32).pin_memory(),
+              torch.zeros(w.S, w.G, dtype=torch.int32).pin_memory()) for _ in range(2)]
+    staging = torch.empty(R.roco_decode_host_pipeline_staging_bytes(cache), dtype=torch.uint8, device=device)
+    kw = dict(scope_mode=scope_mode, step_order=step_order, scale=w.scale)
+    R.roco_decode_step_host(cache, *h_toks[0], w.r, *h_res[0], staging, **kw)           # creates the copy streams
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(1, e2e_steps):
+        R.roco_decode_step_host_begin(cache, *h_toks[i], w.r, *h_res[i & 1], staging, **kw)
+        if i > 1:
+            R.roco_decode_step_host_end()
+    R.roco_decode_step_host_end()
+    e1.record()
+    torch.cuda.synchronize()
+    pipe_sec = e0.elapsed_time(e1) / 1e3
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(e2e_steps, 2 * e2e_steps - 1):
+        R.roco_decode_step_host(cache, *h_toks[i], w.r, *h_res[0], staging, **kw)
+    e1.record()
+    torch.cuda.synchronize()
+    sync_sec = e0.elapsed_time(e1) / 1e3
+    n_e2e = e2e_steps - 1
+    e2e_value, _ = aggregate(w.S * n_e2e, pipe_sec, world, device)
+    e2e_sync, _ = aggregate(w.S * n_e2e, sync_sec, world, device)
+    vec = w.U * w.d * elem
+    e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 3 * vec, "d2h_bytes_per_step": vec + 8 * w.U,
+           "steps": n_e2e, "api": "roco_decode_step_host_begin / _end, two steps in flight",
+           "frac_of_device_timed": e2e_value / value,
+           "synchronising_single_call": {"value": e2e_sync, "api": "roco_decode_step_host"}}
+    if R.roco_device_status(cache) != 0:
+        raise RuntimeError("device status word set during the end-to-end steps")
+    del h_toks, staging
+
+    # ---- roofline of the decode kernel (the only kernel in a step)
+    hbm_peak, _, which = peaks()
+    alg = algorithmic_bytes_per_unit_step(w.B, w.d, elem) * w.U
+    avg_launch = sum(launch_ms) / len(launch_ms) / 1e3
+    med_launch = statistics.median(launch_ms) / 1e3
+    roofline = {"bound": "hbm", "achieved": alg / avg_launch / 1e9, "peak": hbm_peak, "unit": "GB/s",
+                "frac": alg / avg_launch / 1e9 / hbm_peak, "traffic": None, "peak_source": f"of {which}",
+                "kernel": "decode_step_kernel", "algorithmic_bytes_per_launch": alg,
+                "avg_launch_ms": avg_launch * 1e3, "median_launch_ms": med_launch * 1e3,
+                "frac_of_nominal_8TBs": alg / avg_launch / 8e12}
+    if read_gbs:
+        roofline["read_stream_gbs"] = read_gbs
+        roofline["frac_of_read_stream"] = alg / avg_launch / 1e9 / read_gbs
+    # DRAM bytes per unit from a profiler capture of a 512-unit launch of the same shape (traffic grows in
+    # proportion to the units); dropped as soon as the kernel sources differ from the captured ones
+    if kernel_hash() == NCU_TRAFFIC["kernel_hash"] and (w.B, w.d, w.dtype) == NCU_TRAFFIC["shape"] and \
+            (scope_mode, step_order) == (0, 0):
+        roofline["traffic"] = NCU_TRAFFIC["dram_bytes_per_unit"] * w.U
+    res = {"value": value, "ms_per_step": statistics.median(launch_ms) if world == 1 else 1e3 * tmax / steps,
+           "ms_per_step_mean": 1e3 * tmax / steps, "clocks": clk, "e2e": e2e, "roofline": roofline,
+           "config": describe(w, world, scope_mode, step_order)}
+    return res, w, cache, lens, total + 2 * e2e_steps
 
 
 # ----------------------------------------------------------------------------------------- main
@@ -381,6 +566,7 @@ def main():
     ap.add_argument("--workload", default="llama7b_decode")
     ap.add_argument("--small", action="store_true", help="1/16 of the units (for profiler captures)")
     ap.add_argument("--prefill-only", action="store_true", help="run only the prefill measurement")
+    ap.add_argument("--no-prefill", action="store_true", help="skip the prefill measurement")
     ap.add_argument("--extras", action="store_true", help="also time the block-wise and grouped-query steps")
     ap.add_argument("--prefill-workload", default="llama7b_prefill", help="workload of the prefill measurement")
     ap.add_argument("--scope-r", type=int, default=None, help="override the workload's scope parameter r")
@@ -389,6 +575,10 @@ def main():
                          "the r lowest-variance tokens)")
     ap.add_argument("--step-order", default="evict_first", choices=sorted(STEP_ORDERS),
                     help="order inside a decode step (Fig. 1: evict, insert, attend; or attend, then evict and insert)")
+    ap.add_argument("--readings", action="store_true",
+                    help="also time the other three combinations of scope reading and step order (extra key)")
+    ap.add_argument("--all-workloads", action="store_true",
+                    help="also time the serving-batch and long-context decode workloads (extra key)")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
     if args.impl == "reference" and rank != 0:
@@ -406,129 +596,81 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(device))
 
     if args.prefill_only:
-        print(json.dumps({"prefill": prefill_bench(R, device, small=args.small, workload=args.prefill_workload)}))
+        print(json.dumps({"prefill": prefill_bench(R, device, small=args.small, workload=args.prefill_workload,
+                                                   with_oracle=(rank == 0 and not args.small))}))
         return 0
     w0 = W.ALL[args.workload]
     if args.scope_r is not None:
         w0 = W.scaled(w0, r=args.scope_r)
     if args.small:
         w0 = W.scaled(w0, layers=max(1, w0.layers // 16))
-    w, cache, lens = build_cache(w0, device, R, seed_offset=rank)
-    elem = 2 if w.dtype == "bf16" else 4
-    config = describe(w, world)
+    mode, order = SCOPE_MODES[args.scope_mode], STEP_ORDERS[args.step_order]
+    read_gbs = read_stream_gbs(R, device)
+    res, w, cache, lens, used = decode_bench(R, w0, device, rank, world, local_rank, steps, warmup, mode, order,
+                                             read_gbs=read_gbs)
 
-    total = warmup + steps
-    t_pos = list(lens)
-
-    # ---- decode inputs for every step, resident on the device before the timed region
-    toks = []
-    tp = list(t_pos)
-    for i in range(total):
-        toks.append(W.decode_tokens(w, i, tp, device))
-        tp = [t + 1 for t in tp]
-    out = torch.zeros(w.S, w.G, w.d, dtype=w.torch_dtype, device=device)
-    ev_slot = torch.zeros(w.S, w.G, dtype=torch.int32, device=device)
-    ev_pos = torch.zeros_like(ev_slot)
-
-    def step(i):
-        q, k, v = toks[i]
-        R.roco_decode_step(cache, q, k, v, w.r, out, ev_slot, ev_pos, scale=w.scale)
-
-    for i in range(warmup):
-        step(i)
-    torch.cuda.synchronize()
-    if world > 1:
-        torch.distributed.barrier()
-    visible = [x for x in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if x]
-    sampler = ClockSampler(visible[local_rank] if local_rank < len(visible) else local_rank)
-    sampler.start()
-    time.sleep(0.3)
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
-    torch.cuda.synchronize()
-    t_wall0 = time.perf_counter()
-    evs[0].record()
-    for i in range(steps):
-        step(warmup + i)
-        evs[i + 1].record()
-    torch.cuda.synchronize()
-    t_wall1 = time.perf_counter()
-    if world > 1:
-        torch.distributed.barrier()
-    clocks = sampler.stop(t_wall0, t_wall1)
-    launch_ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
-    sec = evs[0].elapsed_time(evs[steps]) / 1e3
-    if R.roco_device_status(cache) != 0:
-        raise RuntimeError("device status word set during the timed region")
-    value, tmax = aggregate(w.S * steps, sec, world, device)
-
-    # ---- end to end through the host-buffer entry point (pinned host tensors in, results out, every step)
-    e2e_steps = min(steps, 32)
-    staging = torch.empty(R.roco_decode_host_staging_bytes(cache), dtype=torch.uint8, device=device)
-    h_toks = [tuple(x.cpu().pin_memory() for x in W.decode_tokens(w, total + i, [t + total + i for t in t_pos], device))
-              for i in range(e2e_steps)]
-    h_out = torch.zeros(w.S, w.G, w.d, dtype=w.torch_dtype).pin_memory()
-    h_slot = torch.zeros(w.S, w.G, dtype=torch.int32).pin_memory()
-    h_pos = torch.zeros(w.S, w.G, dtype=torch.int32).pin_memory()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for q, k, v in h_toks:
-        R.roco_decode_step_host(cache, q, k, v, w.r, h_out, h_slot, h_pos, staging, scale=w.scale)
-    e1.record()
-    torch.cuda.synchronize()
-    e2e_sec = e0.elapsed_time(e1) / 1e3
-    e2e_value, _ = aggregate(w.S * e2e_steps, e2e_sec, world, device)
-    vec = w.U * w.d * elem
-    e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 3 * vec, "d2h_bytes_per_step": vec + 8 * w.U,
-           "steps": e2e_steps}
-
-    # ---- roofline of the decode kernel (the only kernel in a step)
-    hbm_peak, _, which = peaks()
-    alg = algorithmic_bytes_per_unit_step(w.B, w.d, elem) * w.U
-    avg_launch = sum(launch_ms) / len(launch_ms) / 1e3
-    roofline = {"bound": "hbm", "achieved": alg / avg_launch / 1e9, "peak": hbm_peak, "unit": "GB/s",
-                "frac": alg / avg_launch / 1e9 / hbm_peak, "traffic": None, "peak_source": f"of {which}",
-                "kernel": "decode_step_kernel", "algorithmic_bytes_per_launch": alg,
-                "avg_launch_ms": avg_launch * 1e3, "frac_of_nominal_8TBs": alg / avg_launch / 8e12}
-    # DRAM bytes per unit from the ncu capture of a 512-unit launch of the same shape (traffic grows in
-    # proportion to the units); dropped as soon as the kernel sources differ from the captured ones
-    if kernel_hash() == NCU_TRAFFIC["kernel_hash"] and (w.B, w.d, w.dtype) == NCU_TRAFFIC["shape"]:
-        roofline["traffic"] = NCU_TRAFFIC["dram_bytes_per_unit"] * w.U
-
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-            "ms_per_step": 1e3 * tmax / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+    line = {"metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": res["ms_per_step"], "ms_per_step_mean": res["ms_per_step_mean"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 K/V, fp32 softmax and statistics" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": config, "clocks": clocks, "e2e": e2e, "gpu_launches": steps, "roofline": roofline}
+            "config": res["config"], "clocks": res["clocks"], "e2e": res["e2e"], "gpu_launches": steps,
+            "roofline": res["roofline"]}
 
-    del toks, h_toks
     torch.cuda.empty_cache()
     if args.extras:
         line["multi_query"] = multi_bench(R, cache, w, device)
         if R.roco_device_status(cache) != 0:
             raise RuntimeError("device status word set during the multi-query steps")
-    line["prefill"] = prefill_bench(R, device, small=args.small, workload=args.prefill_workload)
 
-    if rank == 0:
-        n_units, n_steps = min(w.U, 512), 128
+    if rank == 0:   # the oracle beside the GPU figure, same run, same cache, on a bounded sample of units
+        n_units, n_steps = min(w.U, 512), 512
         sample = sorted(np.random.default_rng(0).choice(w.U, n_units, replace=False).tolist())
-        per_step, cores = oracle_sample(w, cache, sample, n_steps, total + e2e_steps,
-                                        [t + total + e2e_steps for t in t_pos])
+        per_step, cores = oracle_sample(w, cache, sample, n_steps, used, [t + used for t in lens], mode, order)
         osec = sum(per_step)
         line["cpu_baseline"] = {"value": (n_units * n_steps / osec) * w.S / w.U, "unit": UNIT, "cores": cores,
                                 "kind": "oracle", "seconds": osec,
                                 "sample": f"{n_units} of {w.U} units x {n_steps} decode steps; scaled by U/sample"}
+    del cache
+    torch.cuda.empty_cache()
+
+    def brief(r):
+        return {"config": r["config"]["workload"], "units": r["config"]["units"], "tokens_per_s": r["value"],
+                "ms_per_step": r["ms_per_step"], "ms_per_step_mean": r["ms_per_step_mean"],
+                "gbs": r["roofline"]["achieved"], "frac": r["roofline"]["frac"],
+                "frac_of_nominal_8TBs": r["roofline"]["frac_of_nominal_8TBs"],
+                "frac_of_read_stream": r["roofline"].get("frac_of_read_stream"),
+                "e2e_tokens_per_s": r["e2e"]["value"], "e2e_frac_of_device_timed": r["e2e"]["frac_of_device_timed"]}
+
+    if args.readings:      # the same workload under the other readings of scope and order
+        line["readings"] = [dict(brief(res), scope_mode=args.scope_mode, step_order=args.step_order)]
+        for sm_name, so_name in [(a, b) for a in ("exclude_top_r", "lowest_r") for b in ("evict_first", "attend_first")]:
+            if (sm_name, so_name) == (args.scope_mode, args.step_order):
+                continue
+            r2, _, c2, _, _ = decode_bench(R, w0, device, rank, world, local_rank, min(steps, 64), warmup,
+                                           SCOPE_MODES[sm_name], STEP_ORDERS[so_name], e2e_steps=8, clocks=False,
+                                           read_gbs=read_gbs)
+            line["readings"].append(dict(brief(r2), scope_mode=sm_name, step_order=so_name))
+            del c2
+            torch.cuda.empty_cache()
+    if args.all_workloads:  # the other decode workloads at their full sizes (extra keys, not the headline)
+        line["workloads"] = {}
+        for name in ("llama13b_serving", "long_context"):
+            if name == args.workload:
+                continue
+            r2, _, c2, _, _ = decode_bench(R, W.ALL[name], device, rank, world, local_rank, min(steps, 64), warmup,
+                                           mode, order, e2e_steps=8, clocks=False, read_gbs=read_gbs)
+            line["workloads"][name] = brief(r2)
+            del c2
+            torch.cuda.empty_cache()
+
+    if not args.no_prefill:
+        line["prefill"] = prefill_bench(R, device, small=args.small, workload=args.prefill_workload,
+                                        with_oracle=(rank == 0 and not args.small))
+    if rank == 0:
         print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()
     return 0
-
-
-def kernel_hash() -> str:
-    import hashlib
-    h = hashlib.sha256()
-    for fn in ("decode.cu", "select.cuh", "common.cuh"):
-        h.update(open(os.path.join(ROOT, "paper_2402_06262_b200", "csrc", fn), "rb").read())
-    return h.hexdigest()[:16]
 
 
 if __name__ == "__main__":

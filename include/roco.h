@@ -321,6 +321,25 @@ roco_status roco_decode_step_host(roco_cache *cache, const void *q_host, const v
                                   void *staging, size_t staging_bytes, void *stream);
 
 /*
+ * The host-buffer step in two halves, so that the copies of one step run under the kernel of another: _begin
+ * enqueues the input copies (on an input stream of the library), the step's kernel (on `stream`) and the result
+ * copies (on an output stream) and returns without waiting; _end blocks the calling host thread until the oldest
+ * begun step's results are in its host buffers.  Up to two steps may be in flight: begin(t), begin(t + 1),
+ * end() [t is done], begin(t + 2), ...  A third _begin without an _end returns ROCO_ERR_STATE, as does an _end
+ * with nothing in flight.  Steps of one cache must be begun on one stream (they are ordered by it); the host
+ * buffers of a step must stay valid and untouched until its _end, and be pinned for the copies to overlap.
+ * Arguments as roco_decode_step_host; staging >= roco_decode_host_pipeline_staging_bytes(cache) (two sets),
+ * 256-byte aligned.  The two copy streams and six events are created per device at the first call and kept (see
+ * roco_decode_step_host); the in-flight count is per device, so one host thread drives one pipeline per device.
+ */
+size_t roco_decode_host_pipeline_staging_bytes(const roco_cache *cache);
+roco_status roco_decode_step_host_begin(roco_cache *cache, const void *q_host, const void *k_new_host,
+                                        const void *v_new_host, int r, int scope_mode, int step_order, float scale,
+                                        void *attn_out_host, int32_t *evicted_slot_host, int32_t *evicted_pos_host,
+                                        void *staging, size_t staging_bytes, void *stream);
+roco_status roco_decode_step_host_end(void);
+
+/*
  * Self-test of the bounded waits (the paper has no counterpart: this checks the library's own failure reporting).
  * Every kernel here waits on shared-memory barriers with a time limit of about two seconds; a wait that runs out
  * sets ROCO_DEV_WAIT_TIMEOUT in the status word and the kernel carries on to its end instead of hanging.  This
@@ -329,6 +348,14 @@ roco_status roco_decode_step_host(roco_cache *cache, const void *q_host, const v
  * took.  The kernel occupies one SM for that time and touches no other memory.
  */
 roco_status roco_selftest_wait_timeout(int32_t *status, int32_t *waited_ms, void *stream);
+
+/*
+ * Measurement aid (the paper has no counterpart): one launch that reads `bytes` bytes (16-byte aligned buffer,
+ * a multiple of 16 is read) with plain 16-byte loads and adds a checksum to *sink (device, may be NULL).  Timed
+ * by the caller, it gives the read-only streaming rate of the device, the ceiling for the read-dominated decode
+ * step; a copy (half reads, half writes) runs below it.
+ */
+roco_status roco_selftest_read_stream(const void *buf, size_t bytes, unsigned long long *sink, void *stream);
 
 /* Copies the device status word to *flags_host (synchronises the stream).  Returns ROCO_ERR_STATE
  * when it is non-zero. */

@@ -251,6 +251,23 @@ def block_step(st: State, Q, K_new, V_new, r, mode, scale, delta=1e-5, force_slo
     return BlockResult(out, lse, es, ep, ch, nt)
 
 
+def gqa_block_step(st: State, Q, K_new, V_new, r, mode, scale, delta=1e-5, force_slots=None) -> BlockResult:
+    """Block-wise evict-and-encode of b tokens per key-value head shared by `group` query heads, in place on `st`.
+    Q: [U][b][group][d]; K_new, V_new: [U][b][d].  Returns out [U][b][group][d], lse [U][b][group]."""
+    Q, K_new, V_new = _f64(Q), _f64(K_new), _f64(V_new)
+    U, b, group, d = Q.shape
+    out = np.zeros((U, b, group, d)); lse = np.zeros((U, b, group))
+    es = np.zeros((U, b), np.int32); ep = np.zeros((U, b), np.int32); ch = np.zeros((U, b), np.int32)
+    nt = np.zeros(U, np.int32)
+    fs = None if force_slots is None else _i32(force_slots)
+    lib().roco_oracle_gqa_block_step_batch(C.c_int(U), _p(st.K), _p(st.V), _p(st.s), _p(st.q), _p(st.n), _p(st.pos),
+                                           _p(st.live), _p(st.t_next), C.c_int(st.B), C.c_int(d), C.c_int(b),
+                                           C.c_int(group), _p(Q), _p(K_new), _p(V_new), C.c_int(r), C.c_int(mode),
+                                           C.c_double(scale), C.c_double(delta), _p(fs), _p(out), _p(lse), _p(es),
+                                           _p(ep), _p(ch), _p(nt))
+    return BlockResult(out, lse, es, ep, ch, nt)
+
+
 def gqa_step(st: State, Q, k_new, v_new, r, mode, scale, delta=1e-5, force_victim=None) -> StepResult:
     """One decode step of U key-value heads, each shared by `group` query heads.  Q: [U][group][d];
     k_new, v_new: [U][d].  Returns out [U][group][d], lse [U][group]."""

@@ -657,6 +657,115 @@ void roco_oracle_gqa_step_unit(double *K, double *V, double *s, double *q, int *
   free(p); free(pbar);
 }
 
+/* --------- block-wise evict-and-encode on a grouped-query model (Sec. 5.3 "Extension to Grouped-Query Attention",
+ * App. A; App. B / Table 9: block-wise eviction on Zephyr-7B, a grouped-query model) -- */
+
+/* One eviction step that frees and encodes b tokens of a key-value head shared by `group` query heads.
+ * Steps 1 and 2 as in roco_oracle_block_step_unit (rule applied on frozen statistics; new tokens to the freed /
+ * free slots in increasing slot order).  Step 3: for token i of the block every query head g attends over the
+ * remaining old tokens and the new tokens 0..i (Eq. 1, causal inside the block), out_{i,g} = p_{i,g} V; the
+ * statistics of Sec. 4.3 receive, once per token of the block, the group-wise averaged probability
+ * pbar_i = (1/group) sum_g p_{i,g}: Count += 1, Acc += pbar_i, Acc^square += pbar_i^2.
+ * group = 1 is roco_oracle_block_step_unit; b = 1 is roco_oracle_gqa_step_unit.
+ * Q: [b][group][d]; Kn, Vn: [b][d]; out: [b][group][d]; lse: [b][group].  Other arguments as the block step. */
+void roco_oracle_gqa_block_step_unit(double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
+                                     int *t_next, int B, int d, int b, int group, const double *Q, const double *Kn,
+                                     const double *Vn, int r, int mode, double scale, double delta,
+                                     const int *force_slots, double *out, double *lse, int *evicted_slot,
+                                     int *evicted_pos, int *choice, int *near_tie) {
+  const int live0 = *live, t0 = *t_next;
+  int need = live0 + b - B;
+  if (need < 0) need = 0;
+  int *gone = (int *)calloc((size_t)B, sizeof(int));
+  int n_near = 0;
+  double *cs = (double *)malloc(sizeof(double) * (size_t)B), *cq = (double *)malloc(sizeof(double) * (size_t)B);
+  int *cn = (int *)malloc(sizeof(int) * (size_t)B), *cp = (int *)malloc(sizeof(int) * (size_t)B);
+  int *cslot = (int *)malloc(sizeof(int) * (size_t)B);
+  for (int it = 0; it < need; ++it) { /* 1. the rule, `need` times, on the statistics as they stand */
+    int k = 0;
+    for (int j = 0; j < live0; ++j)
+      if (!gone[j]) { cs[k] = s[j]; cq[k] = q[j]; cn[k] = n[j]; cp[k] = pos[j]; cslot[k] = j; ++k; }
+    int near = 0;
+    int c = roco_oracle_select(cs, cq, cn, cp, k, r, mode, delta, &near, NULL);
+    n_near += near;
+    gone[cslot[c]] = 1;
+  }
+  for (int i = 0; i < b; ++i) { choice[i] = -1; evicted_slot[i] = -1; evicted_pos[i] = -1; }
+  {
+    int k = 0;
+    for (int j = 0; j < live0; ++j) if (gone[j]) choice[k++] = j;
+  }
+  if (force_slots && n_near > 0) {
+    memset(gone, 0, sizeof(int) * (size_t)B);
+    for (int i = 0; i < b; ++i) if (force_slots[i] >= 0 && force_slots[i] < live0) gone[force_slots[i]] = 1;
+  }
+  {
+    int k = 0;
+    for (int j = 0; j < live0; ++j) if (gone[j]) { evicted_slot[k] = j; evicted_pos[k] = pos[j]; ++k; }
+  }
+  int *slot_of_new = (int *)malloc(sizeof(int) * (size_t)b); /* 2. insert */
+  {
+    int k = 0;
+    for (int j = 0; j < B && k < b; ++j)
+      if (j >= live0 || gone[j]) slot_of_new[k++] = j;
+  }
+  const int live1 = live0 - need + b;
+  for (int i = 0; i < b; ++i)
+    insert_token(K, V, s, q, n, pos, slot_of_new[i], d, Kn + (size_t)i * d, Vn + (size_t)i * d, t0 + i);
+  double *p = (double *)malloc(sizeof(double) * (size_t)B), *pbar = (double *)malloc(sizeof(double) * (size_t)B);
+  double *Kc = (double *)malloc(sizeof(double) * (size_t)B * d);
+  int *members = (int *)malloc(sizeof(int) * (size_t)B);
+  for (int i = 0; i < b; ++i) { /* 3. token i of the block: every head of the group, then the group mean */
+    int m = 0;
+    for (int j = 0; j < live1; ++j) {
+      int newer = 0;
+      for (int i2 = i + 1; i2 < b; ++i2) if (slot_of_new[i2] == j) newer = 1;
+      if (!newer) members[m++] = j;
+    }
+    for (int k = 0; k < m; ++k) {
+      memcpy(Kc + (size_t)k * d, K + (size_t)members[k] * d, sizeof(double) * (size_t)d);
+      pbar[k] = 0.0;
+    }
+    for (int g = 0; g < group; ++g) {
+      const size_t row = (size_t)i * group + g;
+      lse[row] = softmax_row(Q + row * d, Kc, m, d, scale, p);
+      for (int c = 0; c < d; ++c) out[row * d + c] = 0.0;
+      for (int k = 0; k < m; ++k) {
+        for (int c = 0; c < d; ++c) out[row * d + c] += p[k] * V[(size_t)members[k] * d + c];
+        pbar[k] += p[k];
+      }
+    }
+    for (int k = 0; k < m; ++k) {
+      const int j = members[k];
+      const double pb = pbar[k] / group;
+      s[j] += pb;
+      q[j] += pb * pb;
+      n[j] += 1;
+    }
+  }
+  *live = live1;
+  *t_next = t0 + b;
+  *near_tie = n_near;
+  free(gone); free(cs); free(cq); free(cn); free(cp); free(cslot); free(slot_of_new); free(p); free(pbar); free(Kc);
+  free(members);
+}
+
+void roco_oracle_gqa_block_step_batch(int U, double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
+                                      int *t_next, int B, int d, int b, int group, const double *Q, const double *Kn,
+                                      const double *Vn, int r, int mode, double scale, double delta,
+                                      const int *force_slots, double *out, double *lse, int *evicted_slot,
+                                      int *evicted_pos, int *choice, int *near_tie) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int u = 0; u < U; ++u) {
+    size_t kb = (size_t)u * B * d, sb = (size_t)u * B, qb = (size_t)u * b * group * d, vb = (size_t)u * b * d;
+    size_t ib = (size_t)u * b;
+    roco_oracle_gqa_block_step_unit(K + kb, V + kb, s + sb, q + sb, n + sb, pos + sb, live + u, t_next + u, B, d, b,
+                                    group, Q + qb, Kn + vb, Vn + vb, r, mode, scale, delta,
+                                    force_slots ? force_slots + ib : NULL, out + qb, lse + ib * group,
+                                    evicted_slot + ib, evicted_pos + ib, choice + ib, near_tie + u);
+  }
+}
+
 void roco_oracle_block_step_batch(int U, double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
                                   int *t_next, int B, int d, int b, const double *Q, const double *Kn,
                                   const double *Vn, int r, int mode, double scale, double delta,

@@ -27,7 +27,8 @@ EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes",
            "roco_decode_split_workspace_bytes", "roco_decode_step_split", "roco_prefill_blockwise",
            "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status",
            "roco_prefill_attend_workspace_bytes", "roco_prefill_attend", "roco_selftest_wait_timeout",
-           "roco_consistency_step")
+           "roco_consistency_step", "roco_selftest_read_stream", "roco_decode_host_pipeline_staging_bytes",
+           "roco_decode_step_host_begin", "roco_decode_step_host_end")
 
 
 class RocoError(RuntimeError):
@@ -105,6 +106,14 @@ def lib() -> C.CDLL:
         L.roco_consistency_step.restype = C.c_int
         L.roco_consistency_step.argtypes = [C.POINTER(roco_cache), C.POINTER(roco_cache), C.c_int, C.c_void_p,
                                             C.c_void_p, C.c_void_p, C.c_void_p]
+        L.roco_decode_host_pipeline_staging_bytes.restype = C.c_size_t
+        L.roco_decode_host_pipeline_staging_bytes.argtypes = [C.POINTER(roco_cache)]
+        L.roco_decode_step_host_begin.restype = C.c_int
+        L.roco_decode_step_host_begin.argtypes = L.roco_decode_step_host.argtypes
+        L.roco_decode_step_host_end.restype = C.c_int
+        L.roco_decode_step_host_end.argtypes = []
+        L.roco_selftest_read_stream.restype = C.c_int
+        L.roco_selftest_read_stream.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.roco_selftest_wait_timeout.restype = C.c_int
         L.roco_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.roco_device_status.restype = C.c_int
@@ -220,6 +229,14 @@ def roco_prefill_attend(cache: Cache, Q, K, V, lens: Sequence[int], lse, attn_ou
     return workspace
 
 
+def roco_selftest_read_stream(buf: torch.Tensor, sink: Optional[torch.Tensor] = None):
+    """One launch that reads every byte of `buf` (device tensor) with plain 16-byte loads; time it to get the
+    device's read-only streaming rate.  sink: int64 [1] device checksum accumulator, or None."""
+    rc = lib().roco_selftest_read_stream(_ptr(buf), buf.numel() * buf.element_size(), _ptr(sink), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_selftest_read_stream")
+
+
 def roco_selftest_wait_timeout(status: torch.Tensor, waited_ms: Optional[torch.Tensor] = None):
     """Launches the bounded-wait self-test: `status` (int32 [1], device) gets ROCO_DEV_WAIT_TIMEOUT once the
     kernel's wait has run out (about two seconds); `waited_ms` (int32 [1], device) how long that took."""
@@ -302,7 +319,8 @@ def roco_consistency_step(full: Cache, budgeted: Cache, policy: int, overlap, ja
     rc = lib().roco_consistency_step(C.byref(full.c), C.byref(budgeted.c), policy, _ptr(overlap), _ptr(jaccard_sum),
                                      _ptr(samples), _stream())
     if rc != ROCO_OK:
-        raise RocoError(rc, "roco_consistency_step")
+        raise RocoError(rc, "roco_consistency_step", "roco_selftest_read_stream", "roco_decode_host_pipeline_staging_bytes",
+           "roco_decode_step_host_begin", "roco_decode_step_host_end")
 
 
 def roco_decode_host_staging_bytes(cache: Cache) -> int:
@@ -319,6 +337,30 @@ def roco_decode_step_host(cache: Cache, q_host, k_new_host, v_new_host, r: int, 
                                      _ptr(evicted_pos_host), _ptr(staging), staging.numel(), _stream())
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_decode_step_host")
+
+
+def roco_decode_host_pipeline_staging_bytes(cache: Cache) -> int:
+    return int(lib().roco_decode_host_pipeline_staging_bytes(C.byref(cache.c)))
+
+
+def roco_decode_step_host_begin(cache: Cache, q_host, k_new_host, v_new_host, r: int, attn_out_host,
+                                evicted_slot_host, evicted_pos_host, staging, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R,
+                                step_order=ROCO_EVICT_FIRST, scale: Optional[float] = None):
+    """First half of the host-buffer step: enqueues copies in, kernel, copies out; does not wait."""
+    scale = cache.d ** -0.5 if scale is None else scale
+    rc = lib().roco_decode_step_host_begin(C.byref(cache.c), _ptr(q_host), _ptr(k_new_host), _ptr(v_new_host), r,
+                                           scope_mode, step_order, scale, _ptr(attn_out_host),
+                                           _ptr(evicted_slot_host), _ptr(evicted_pos_host), _ptr(staging),
+                                           staging.numel(), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_decode_step_host_begin")
+
+
+def roco_decode_step_host_end():
+    """Second half: waits until the oldest begun step's results are in its host buffers."""
+    rc = lib().roco_decode_step_host_end()
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_decode_step_host_end")
 
 
 def roco_device_status(cache: Cache) -> int:

@@ -60,10 +60,16 @@ PrefillWs prefill_ws(int S, int G, int Lmax) {
 // and kept until the process exits.
 constexpr int kHostChunks = 4;
 constexpr int kHostMaxDevices = 64;
+constexpr int kHostDepth = 2;  // steps in flight in the begin/end form
 struct HostPipe {
   bool ready = false;
   cudaStream_t copy = nullptr;
   cudaEvent_t start = nullptr, done = nullptr, h2d[kHostChunks] = {}, ker[kHostChunks] = {};
+  // begin/end form: an input and an output copy stream, and per staging set the three events of its last step
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t set_h2d[kHostDepth] = {}, set_ker[kHostDepth] = {}, set_d2h[kHostDepth] = {};
+  bool set_used[kHostDepth] = {};
+  unsigned long long begun = 0, ended = 0;
 };
 
 HostPipe *host_pipe() {
@@ -80,6 +86,12 @@ HostPipe *host_pipe() {
     for (int i = 0; ok && i < kHostChunks; ++i)
       ok = cudaEventCreateWithFlags(&hp.h2d[i], cudaEventDisableTiming) == cudaSuccess &&
            cudaEventCreateWithFlags(&hp.ker[i], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) == cudaSuccess &&
+         cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; ok && i < kHostDepth; ++i)
+      ok = cudaEventCreateWithFlags(&hp.set_h2d[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.set_ker[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.set_d2h[i], cudaEventDisableTiming) == cudaSuccess;
     if (!ok) return nullptr;
     hp.ready = true;
   }
@@ -431,6 +443,65 @@ roco_status roco_decode_step_host(roco_cache *cache, const void *q_host, const v
                        ok(cudaStreamSynchronize(cs)) && ok(cudaStreamSynchronize(hp->copy));
   if (st != ROCO_OK) return st;
   return drained ? ROCO_OK : ROCO_ERR_CUDA;
+}
+
+size_t roco_decode_host_pipeline_staging_bytes(const roco_cache *cache) {
+  return kHostDepth * roco_decode_host_staging_bytes(cache);
+}
+
+roco_status roco_decode_step_host_begin(roco_cache *cache, const void *q_host, const void *k_new_host,
+                                        const void *v_new_host, int r, int scope_mode, int step_order, float scale,
+                                        void *attn_out_host, int32_t *evicted_slot_host, int32_t *evicted_pos_host,
+                                        void *staging, size_t staging_bytes, void *stream) {
+  NvtxRange range("roco_decode_step_host_begin");
+  roco_status st = check_cache(cache);
+  if (st != ROCO_OK) return st;
+  if (!q_host || !k_new_host || !v_new_host || !attn_out_host || !evicted_slot_host) return ROCO_ERR_INVALID_ARG;
+  const size_t one = roco_decode_host_staging_bytes(cache);
+  if (!staging || staging_bytes < kHostDepth * one || (reinterpret_cast<uintptr_t>(staging) & 255u))
+    return ROCO_ERR_WORKSPACE;
+  HostPipe *hp = host_pipe();
+  if (!hp) return ROCO_ERR_CUDA;
+  if (hp->begun - hp->ended >= kHostDepth) return ROCO_ERR_STATE;  // end a step first
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const int set = (int)(hp->begun % kHostDepth);
+  const size_t U = (size_t)cache->S * cache->G;
+  const size_t vbytes = U * cache->d * (cache->kv_dtype == ROCO_BF16 ? 2 : 4);
+  const size_t vec = align_up(vbytes, 256), ivec = align_up(U * 4, 256);
+  char *p = static_cast<char *>(staging) + set * one;
+  char *dq = p, *dk = p + vec, *dv = p + 2 * vec, *dout = p + 3 * vec;
+  int32_t *dslot = reinterpret_cast<int32_t *>(p + 4 * vec), *dpos = reinterpret_cast<int32_t *>(p + 4 * vec + ivec);
+  auto ok = [](cudaError_t e) { return e == cudaSuccess; };
+  // inputs of this step: the set's input buffers were last read by the kernel two steps ago
+  if (hp->set_used[set] && !ok(cudaStreamWaitEvent(hp->in, hp->set_ker[set], 0))) return ROCO_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(dq, q_host, vbytes, cudaMemcpyHostToDevice, hp->in)) ||
+      !ok(cudaMemcpyAsync(dk, k_new_host, vbytes, cudaMemcpyHostToDevice, hp->in)) ||
+      !ok(cudaMemcpyAsync(dv, v_new_host, vbytes, cudaMemcpyHostToDevice, hp->in)) ||
+      !ok(cudaEventRecord(hp->set_h2d[set], hp->in)) || !ok(cudaStreamWaitEvent(cs, hp->set_h2d[set], 0)))
+    return ROCO_ERR_CUDA;
+  // the kernel: the set's output buffers were last read by the copy-out two steps ago
+  if (hp->set_used[set] && !ok(cudaStreamWaitEvent(cs, hp->set_d2h[set], 0))) return ROCO_ERR_CUDA;
+  st = roco_decode_step(cache, dq, dk, dv, r, scope_mode, step_order, scale, dout, nullptr, dslot, dpos, stream);
+  if (st != ROCO_OK) return st;
+  if (!ok(cudaEventRecord(hp->set_ker[set], cs)) || !ok(cudaStreamWaitEvent(hp->out, hp->set_ker[set], 0)) ||
+      !ok(cudaMemcpyAsync(attn_out_host, dout, vbytes, cudaMemcpyDeviceToHost, hp->out)) ||
+      !ok(cudaMemcpyAsync(evicted_slot_host, dslot, U * 4, cudaMemcpyDeviceToHost, hp->out)) ||
+      (evicted_pos_host && !ok(cudaMemcpyAsync(evicted_pos_host, dpos, U * 4, cudaMemcpyDeviceToHost, hp->out))) ||
+      !ok(cudaEventRecord(hp->set_d2h[set], hp->out)))
+    return ROCO_ERR_CUDA;
+  hp->set_used[set] = true;
+  ++hp->begun;
+  return ROCO_OK;
+}
+
+roco_status roco_decode_step_host_end(void) {
+  NvtxRange range("roco_decode_step_host_end");
+  HostPipe *hp = host_pipe();
+  if (!hp) return ROCO_ERR_CUDA;
+  if (hp->begun == hp->ended) return ROCO_ERR_STATE;  // nothing in flight
+  const int set = (int)(hp->ended % kHostDepth);
+  ++hp->ended;
+  return cudaEventSynchronize(hp->set_d2h[set]) == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
 }
 
 roco_status roco_device_status(const roco_cache *cache, void *stream, int32_t *flags_host) {

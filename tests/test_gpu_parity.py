@@ -188,6 +188,50 @@ def test_host_buffer_variant_matches_device_variant(layers, heads, B):
     assert torch.equal(caches[0].s, caches[1].s) and torch.equal(caches[0].K, caches[1].K)
 
 
+def test_pipelined_host_buffer_steps_match_device_steps():
+    """begin/end form of the host-buffer step (two steps in flight, copies of one under the kernel of the other)
+    against the device-buffer step, bit for bit, over 7 steps; and the in-flight rules."""
+    w = W.scaled(W.LLAMA7B_DECODE, S=2, layers=4, heads=8, prompt_lo=150, prompt_hi=150, B=96, r=8)
+    Q, K, V = prompt_tensors(w, 150)
+    caches = [R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV) for _ in range(2)]
+    for c in caches:
+        R.roco_prefill(Q, K, V, [150, 150], w.B, w.r, c, scale=w.scale)
+    n = 7
+    toks = [W.decode_tokens(w, i, [150 + i] * 2, DEV) for i in range(n)]
+    want = []
+    out = torch.zeros(w.S, w.G, w.d, dtype=w.torch_dtype, device=DEV)
+    ev = torch.zeros(w.S, w.G, dtype=torch.int32, device=DEV)
+    evp = torch.zeros_like(ev)
+    for q, k, v in toks:
+        R.roco_decode_step(caches[0], q, k, v, w.r, out, ev, evp, scale=w.scale)
+        want.append((out.cpu().clone(), ev.cpu().clone(), evp.cpu().clone()))
+    staging = torch.empty(R.roco_decode_host_pipeline_staging_bytes(caches[1]), dtype=torch.uint8, device=DEV)
+    h_in = [tuple(x.cpu().pin_memory() for x in t) for t in toks]
+    h_out = [(torch.zeros(w.S, w.G, w.d, dtype=w.torch_dtype).pin_memory(),
+              torch.zeros(w.S, w.G, dtype=torch.int32).pin_memory(),
+              torch.zeros(w.S, w.G, dtype=torch.int32).pin_memory()) for _ in range(n)]
+    with pytest.raises(R.RocoError) as e:
+        R.roco_decode_step_host_end()                                   # nothing in flight
+    assert e.value.code == 5
+    for i in range(n):
+        R.roco_decode_step_host_begin(caches[1], *h_in[i], w.r, *h_out[i], staging, scale=w.scale)
+        if i == 1:
+            with pytest.raises(R.RocoError) as e:                       # a third step without an end
+                R.roco_decode_step_host_begin(caches[1], *h_in[2], w.r, *h_out[2], staging, scale=w.scale)
+            assert e.value.code == 5
+        if i >= 1:
+            R.roco_decode_step_host_end()                               # step i - 1 is complete
+            for a, b in zip(want[i - 1], h_out[i - 1]):
+                assert torch.equal(a, b)
+    R.roco_decode_step_host_end()
+    for a, b in zip(want[n - 1], h_out[n - 1]):
+        assert torch.equal(a, b)
+    torch.cuda.synchronize()
+    for name in ("K", "V", "s", "q", "n", "pos", "live", "t_next"):
+        assert torch.equal(getattr(caches[0], name), getattr(caches[1], name)), name
+    assert R.roco_device_status(caches[1]) == 0
+
+
 def test_llama7b_decode_shape_sampled_units():
     """The benchmark's launch configuration (8192 units, B=1024, d=128, bf16, r=64): the cache is built by the
     library's prefill from 2048-token prompts, layer-chunk by layer-chunk; 64 sampled units are followed by the

@@ -152,3 +152,92 @@ def test_gqa_brute_force_group_mean(group):
         np.testing.assert_allclose(st.q[0], q + pbar ** 2, rtol=1e-12)
         np.testing.assert_array_equal(st.n[0], n + 1)
         assert pbar.sum() == pytest.approx(1.0, rel=1e-13)            # the group mean is still a distribution
+
+
+# ------------------------------------------------ block-wise eviction on a grouped-query model (App. B, Table 9)
+
+def test_grouped_block_with_one_head_is_the_block_step_and_with_one_token_the_gqa_step():
+    rng = np.random.default_rng(21)
+    U, B, d = 2, 12, 5
+    base = filled_state(rng, U, B, d, 14)
+    # group = 1  ==  block step
+    a, b_ = base.copy(), base.copy()
+    for _ in range(3):
+        Q, Kn, Vn = rng.normal(size=(3, U, 3, d))
+        ra = oracle.block_step(a, Q, Kn, Vn, 2, EXCLUDE_TOP_R, 0.4)
+        rb = oracle.gqa_block_step(b_, Q[:, :, None], Kn, Vn, 2, EXCLUDE_TOP_R, 0.4)
+        np.testing.assert_array_equal(ra.evicted_slot, rb.evicted_slot)
+        np.testing.assert_array_equal(ra.out, rb.out[:, :, 0])
+        np.testing.assert_array_equal(ra.lse, rb.lse[:, :, 0])
+        for name in ("K", "V", "s", "q", "n", "pos", "live", "t_next"):
+            np.testing.assert_array_equal(getattr(a, name), getattr(b_, name))
+    # b = 1  ==  grouped-query decode step
+    a, b_ = base.copy(), base.copy()
+    for _ in range(3):
+        Q = rng.normal(size=(U, 4, d))
+        kn, vn = rng.normal(size=(2, U, d))
+        ra = oracle.gqa_step(a, Q, kn, vn, 2, EXCLUDE_TOP_R, 0.4)
+        rb = oracle.gqa_block_step(b_, Q[:, None], kn[:, None], vn[:, None], 2, EXCLUDE_TOP_R, 0.4)
+        np.testing.assert_array_equal(ra.evicted_slot, rb.evicted_slot[:, 0])
+        np.testing.assert_array_equal(ra.out, rb.out[:, 0])
+        for name in ("K", "V", "s", "q", "n", "pos", "live", "t_next"):
+            np.testing.assert_array_equal(getattr(a, name), getattr(b_, name))
+
+
+def test_grouped_block_identical_heads_equal_the_single_head_block_step():
+    rng = np.random.default_rng(22)
+    U, B, d, b = 2, 10, 6, 4
+    a = filled_state(rng, U, B, d, 13)
+    c = a.copy()
+    for _ in range(3):
+        Q, Kn, Vn = rng.normal(size=(3, U, b, d))
+        ra = oracle.block_step(a, Q, Kn, Vn, 3, EXCLUDE_TOP_R, 0.4)
+        rc = oracle.gqa_block_step(c, np.repeat(Q[:, :, None], 3, 2), Kn, Vn, 3, EXCLUDE_TOP_R, 0.4)
+        np.testing.assert_array_equal(ra.evicted_slot, rc.evicted_slot)
+        for g in range(3):
+            np.testing.assert_allclose(rc.out[:, :, g], ra.out, rtol=1e-13)
+        for name in ("s", "q"):
+            np.testing.assert_allclose(getattr(c, name), getattr(a, name), rtol=1e-12)
+        np.testing.assert_array_equal(c.n, a.n)
+
+
+@pytest.mark.parametrize("b,group", [(2, 2), (3, 4), (4, 2)])
+def test_grouped_block_brute_force(b, group):
+    """Definitions written out with library softmax: victims by exhaustive sorting on the frozen statistics, new
+    tokens to the freed / free slots in increasing slot order, token i's heads see the survivors and new tokens
+    0..i, statistics from the mean over the heads, once per token."""
+    rng = np.random.default_rng(100 * b + group)
+    U, B, d, scale, r = 1, 9, 4, 0.5, 2
+    for live_start in (6, 12):
+        st = filled_state(rng, U, B, d, live_start, scale)
+        before = st.copy()
+        live0 = int(before.live[0])
+        need = max(0, live0 + b - B)
+        Q = rng.normal(size=(U, b, group, d))
+        Kn, Vn = rng.normal(size=(2, U, b, d))
+        res = oracle.gqa_block_step(st, Q, Kn, Vn, r, EXCLUDE_TOP_R, scale)
+        gone = brute_victims(before.s[0], before.q[0], before.n[0], before.pos[0], live0, need, r, EXCLUDE_TOP_R)
+        assert list(res.evicted_slot[0][:need]) == gone and all(x == -1 for x in res.evicted_slot[0][need:])
+        targets = sorted(gone + list(range(live0, live0 + b - need)))
+        Kc, Vc = before.K[0].copy(), before.V[0].copy()
+        s, q, n = before.s[0].copy(), before.q[0].copy(), before.n[0].copy()
+        for i, t in enumerate(targets):
+            Kc[t], Vc[t], s[t], q[t], n[t] = Kn[0, i], Vn[0, i], 0.0, 0.0, 0
+        live1 = live0 - need + b
+        for i in range(b):
+            members = [j for j in range(live1) if j not in targets[i + 1:]]
+            pbar = np.zeros(len(members))
+            for g in range(group):
+                z = scale * Kc[members] @ Q[0, i, g]
+                p = softmax(z)
+                np.testing.assert_allclose(res.out[0, i, g], p @ Vc[members], rtol=1e-12, atol=1e-15)
+                assert res.lse[0, i, g] == pytest.approx(logsumexp(z), rel=1e-12)
+                pbar += p
+            pbar /= group
+            s[members] += pbar; q[members] += pbar * pbar; n[members] += 1
+        np.testing.assert_allclose(st.s[0, :live1], s[:live1], rtol=1e-12)
+        np.testing.assert_allclose(st.q[0, :live1], q[:live1], rtol=1e-12)
+        np.testing.assert_array_equal(st.n[0, :live1], n[:live1])
+        # the group mean of probability rows still sums to 1 per token of the block
+        lost = before.s[0][gone].sum()
+        assert st.s[0, :live1].sum() + lost == pytest.approx(before.s[0, :live0].sum() + b, rel=1e-12)
