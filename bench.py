@@ -353,6 +353,16 @@ def multi_bench(R, cache, w, device, reps=6):
         res["blockwise_prefill"].append({"b": b, "prompt": Lp, "ms": ms, "prompt_tokens_per_s": w.S * Lp / ms * 1e3,
                                          "speedup_vs_b1": t_b1 / ms})
     del Qp, Kp, Vp, outp, pc
+    # block-wise evict-and-encode on key-value heads shared by `group` query heads (b x group <= 16 query rows)
+    res["gqa_block"] = []
+    for b, g in ((4, 4), (8, 2), (2, 8)):
+        Q = torch.randn(w.S, w.G, b, g, w.d, device=device, generator=gen).to(dt)
+        K, V = (torch.randn(w.S, w.G, b, w.d, device=device, generator=gen).to(dt) for _ in range(2))
+        out = torch.zeros(w.S, w.G, b, g, w.d, dtype=dt, device=device)
+        ev = torch.zeros(w.S, w.G, b, dtype=torch.int32, device=device)
+        ms = timed(lambda: R.roco_gqa_block_step(cache, Q, K, V, w.r, out, ev, scale=w.scale))
+        res["gqa_block"].append({"b": b, "group": g, "ms_per_step": ms, "tokens_per_s": w.S * b / ms * 1e3,
+                                 "hbm_frac": alg / ms / 1e6 / hbm_peak})
     for g in (4, 8):
         Q = torch.randn(w.S, w.G, g, w.d, device=device, generator=gen).to(dt)
         k, v = (torch.randn(w.S, w.G, w.d, device=device, generator=gen).to(dt) for _ in range(2))

@@ -255,6 +255,28 @@ roco_status roco_prefill_attend(const roco_cache *cache, const void *Q, const vo
                                 void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Block-wise evict-and-encode on a grouped-query model (Sec. 5.3 "Extension to Grouped-Query Attention", App. A;
+ * App. B / Table 9 run block-wise eviction on such a model): the cache belongs to a key-value head that `group`
+ * query heads share.  Steps 1 and 2 as roco_block_step.  Step 3: for token i of the block each of its query heads
+ * attends over the remaining old tokens and the new tokens 0..i; the statistics receive, once per token of the
+ * block, the group-wise averaged probability: Count += 1, Acc += pbar_i, Acc^square += pbar_i^2.
+ * group = 1 is roco_block_step; b = 1 is roco_gqa_decode_step.
+ *
+ *   Q            [S][G][b][group][d];   K_new, V_new [S][G][b][d]
+ *   b, group     b * group <= 16 query rows per pass; other limits as roco_block_step
+ *   attn_out     [S][G][b][group][d];   lse_out [S][G][b][group] or NULL;   evicted_slot, evicted_pos [S][G][b]
+ *
+ * roco_prefill_blockwise_gqa is roco_prefill_blockwise for such a model: Q and attn_out are
+ * [S][G][Lmax][group][d], K and V [S][G][Lmax][d].
+ */
+roco_status roco_gqa_block_step(roco_cache *cache, const void *Q, const void *K_new, const void *V_new, int b,
+                                int group, int r, int scope_mode, float scale, void *attn_out, float *lse_out,
+                                int32_t *evicted_slot, int32_t *evicted_pos, void *stream);
+roco_status roco_prefill_blockwise_gqa(const void *Q, const void *K, const void *V, const int32_t *lens_host,
+                                       int Lmax, int b, int group, int r, float scale, roco_cache *cache,
+                                       void *attn_out, int32_t *evicted_slot, void *stream);
+
+/*
  * Decode step for grouped-query attention (Sec. 5.3 "Extension to Grouped-Query Attention", App. A): the cache
  * belongs to a key-value head that `group` query heads share.  Order as ROCO_EVICT_FIRST.  Each query head g
  * attends over the same cache, out_g = Softmax(scale * q_g K^T) V; the statistics receive the group-wise

@@ -28,7 +28,8 @@ EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes",
            "roco_decode_step", "roco_decode_host_staging_bytes", "roco_decode_step_host", "roco_device_status",
            "roco_prefill_attend_workspace_bytes", "roco_prefill_attend", "roco_selftest_wait_timeout",
            "roco_consistency_step", "roco_selftest_read_stream", "roco_decode_host_pipeline_staging_bytes",
-           "roco_decode_step_host_begin", "roco_decode_step_host_end")
+           "roco_decode_step_host_begin", "roco_decode_step_host_end", "roco_gqa_block_step",
+           "roco_prefill_blockwise_gqa")
 
 
 class RocoError(RuntimeError):
@@ -86,6 +87,14 @@ def lib() -> C.CDLL:
             fn.restype = C.c_int
             fn.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                            C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.roco_gqa_block_step.restype = C.c_int
+        L.roco_gqa_block_step.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                          C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p]
+        L.roco_prefill_blockwise_gqa.restype = C.c_int
+        L.roco_prefill_blockwise_gqa.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                                 C.c_int, C.c_int, C.c_float, C.POINTER(roco_cache), C.c_void_p,
+                                                 C.c_void_p, C.c_void_p]
         L.roco_prefill_blockwise.restype = C.c_int
         L.roco_prefill_blockwise.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                              C.c_float, C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p]
@@ -302,6 +311,30 @@ def roco_block_step(cache: Cache, Q, K_new, V_new, r: int, attn_out, evicted_slo
         raise RocoError(rc, "roco_block_step")
 
 
+def roco_gqa_block_step(cache: Cache, Q, K_new, V_new, r: int, attn_out, evicted_slot, evicted_pos=None,
+                        lse_out=None, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R, scale: Optional[float] = None):
+    """Block-wise evict-and-encode of b = Q.shape[2] tokens per key-value head shared by group = Q.shape[3] query
+    heads.  Q: [S][G][b][group][d]; K_new, V_new: [S][G][b][d]."""
+    scale = cache.d ** -0.5 if scale is None else scale
+    rc = lib().roco_gqa_block_step(C.byref(cache.c), _ptr(Q), _ptr(K_new), _ptr(V_new), int(Q.shape[2]),
+                                   int(Q.shape[3]), r, scope_mode, scale, _ptr(attn_out), _ptr(lse_out),
+                                   _ptr(evicted_slot), _ptr(evicted_pos), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_gqa_block_step")
+
+
+def roco_prefill_blockwise_gqa(Q, K, V, lens: Sequence[int], b: int, r: int, cache: Cache, attn_out, evicted_slot,
+                               scale: Optional[float] = None):
+    """roco_prefill_blockwise for a grouped-query model.  Q, attn_out: [S][G][Lmax][group][d]; K, V: [S][G][Lmax][d]."""
+    scale = cache.d ** -0.5 if scale is None else scale
+    lens_arr = (C.c_int32 * len(lens))(*[int(x) for x in lens])
+    rc = lib().roco_prefill_blockwise_gqa(_ptr(Q), _ptr(K), _ptr(V), C.cast(lens_arr, C.c_void_p), int(K.shape[2]), b,
+                                          int(Q.shape[3]), r, scale, C.byref(cache.c), _ptr(attn_out),
+                                          _ptr(evicted_slot), _stream())
+    if rc != ROCO_OK:
+        raise RocoError(rc, "roco_prefill_blockwise_gqa")
+
+
 def roco_gqa_decode_step(cache: Cache, Q, k_new, v_new, r: int, attn_out, evicted_slot, evicted_pos=None,
                          lse_out=None, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R, scale: Optional[float] = None):
     """Decode step of key-value heads shared by group = Q.shape[2] query heads.  Q: [S][G][group][d]."""
@@ -320,7 +353,8 @@ def roco_consistency_step(full: Cache, budgeted: Cache, policy: int, overlap, ja
                                      _ptr(samples), _stream())
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_consistency_step", "roco_selftest_read_stream", "roco_decode_host_pipeline_staging_bytes",
-           "roco_decode_step_host_begin", "roco_decode_step_host_end")
+           "roco_decode_step_host_begin", "roco_decode_step_host_end", "roco_gqa_block_step",
+           "roco_prefill_blockwise_gqa")
 
 
 def roco_decode_host_staging_bytes(cache: Cache) -> int:

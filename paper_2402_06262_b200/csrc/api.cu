@@ -261,36 +261,44 @@ roco_status roco_decode_step_policy(roco_cache *cache, const void *q, const void
                             attn_out, lse_out, evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
 }
 
-roco_status roco_block_step(roco_cache *cache, const void *Q, const void *K_new, const void *V_new, int b, int r,
-                            int scope_mode, float scale, void *attn_out, float *lse_out, int32_t *evicted_slot,
-                            int32_t *evicted_pos, void *stream) {
-  NvtxRange range("roco_block_step");
+roco_status roco_gqa_block_step(roco_cache *cache, const void *Q, const void *K_new, const void *V_new, int b,
+                                int group, int r, int scope_mode, float scale, void *attn_out, float *lse_out,
+                                int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {
+  NvtxRange range("roco_gqa_block_step");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
   if (!Q || !K_new || !V_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K_new) || !aligned16(V_new) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
-  if (b < 1) return ROCO_ERR_INVALID_ARG;
+  if (b < 1 || group < 1) return ROCO_ERR_INVALID_ARG;
   if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
-  if (b > multi_max_queries()) return ROCO_ERR_UNSUPPORTED;
+  if ((long long)b * group > multi_max_queries()) return ROCO_ERR_UNSUPPORTED;
   if (b > 1 && scope_mode != ROCO_SCOPE_EXCLUDE_TOP_R) return ROCO_ERR_UNSUPPORTED;  // the scope would refill
   if (b > 1 && r + b > cache->B) return ROCO_ERR_INVALID_ARG;  // the scope must hold the b victims
-  if (!multi_fits(cache->B, cache->d, b, b)) return ROCO_ERR_UNSUPPORTED;
-  return launch_multi_step(*cache, 0, b, b, Q, K_new, V_new, r, scope_mode, scale, attn_out, lse_out, evicted_slot,
-                           evicted_pos, static_cast<cudaStream_t>(stream));
+  if (!multi_fits(cache->B, cache->d, b * group, b)) return ROCO_ERR_UNSUPPORTED;
+  return launch_multi_step(*cache, b * group, b, Q, K_new, V_new, r, scope_mode, scale, attn_out, lse_out,
+                           evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
 }
 
-roco_status roco_prefill_blockwise(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax,
-                                   int b, int r, float scale, roco_cache *cache, void *attn_out,
-                                   int32_t *evicted_slot, void *stream) {
+roco_status roco_block_step(roco_cache *cache, const void *Q, const void *K_new, const void *V_new, int b, int r,
+                            int scope_mode, float scale, void *attn_out, float *lse_out, int32_t *evicted_slot,
+                            int32_t *evicted_pos, void *stream) {
+  return roco_gqa_block_step(cache, Q, K_new, V_new, b, 1, r, scope_mode, scale, attn_out, lse_out, evicted_slot,
+                             evicted_pos, stream);
+}
+
+roco_status roco_prefill_blockwise_gqa(const void *Q, const void *K, const void *V, const int32_t *lens_host,
+                                       int Lmax, int b, int group, int r, float scale, roco_cache *cache,
+                                       void *attn_out, int32_t *evicted_slot, void *stream) {
   NvtxRange range("roco_prefill_blockwise");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
-  if (!Q || !K || !V || !lens_host || !attn_out || !evicted_slot || Lmax < 1 || b < 1) return ROCO_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !lens_host || !attn_out || !evicted_slot || Lmax < 1 || b < 1 || group < 1)
+    return ROCO_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
   if ((st = check_scope(r, ROCO_SCOPE_EXCLUDE_TOP_R, cache->B, true)) != ROCO_OK) return st;
-  if (b > multi_max_queries()) return ROCO_ERR_UNSUPPORTED;
+  if ((long long)b * group > multi_max_queries()) return ROCO_ERR_UNSUPPORTED;
   if (b > 1 && r + b > cache->B) return ROCO_ERR_INVALID_ARG;
-  if (!multi_fits(cache->B, cache->d, b, b)) return ROCO_ERR_UNSUPPORTED;
+  if (!multi_fits(cache->B, cache->d, b * group, b)) return ROCO_ERR_UNSUPPORTED;
   for (int s = 0; s < cache->S; ++s)
     if (lens_host[s] < 1 || lens_host[s] > Lmax) return ROCO_ERR_INVALID_ARG;
   const size_t elem = cache->kv_dtype == ROCO_BF16 ? 2 : 4;
@@ -309,16 +317,22 @@ roco_status roco_prefill_blockwise(const void *Q, const void *K, const void *V, 
     sub.live = cache->live + s0 * G; sub.t_next = cache->t_next + s0 * G;
     for (int t0 = 0; t0 < len; t0 += b) {
       const int m = len - t0 < b ? len - t0 : b;
-      const size_t off = ((size_t)s0 * G * Lmax + t0) * d * elem;
-      st = launch_multi_step(sub, 0, m, m, static_cast<const char *>(Q) + off, static_cast<const char *>(K) + off,
-                             static_cast<const char *>(V) + off, r, ROCO_SCOPE_EXCLUDE_TOP_R, scale,
-                             static_cast<char *>(attn_out) + off, nullptr, evicted_slot + (size_t)s0 * G * b, nullptr,
-                             static_cast<cudaStream_t>(stream), Lmax);
+      const size_t off = ((size_t)s0 * G * Lmax + t0) * d * elem;  // K, V: one row per token; Q, out: `group` rows
+      st = launch_multi_step(sub, m * group, m, static_cast<const char *>(Q) + off * group,
+                             static_cast<const char *>(K) + off, static_cast<const char *>(V) + off, r,
+                             ROCO_SCOPE_EXCLUDE_TOP_R, scale, static_cast<char *>(attn_out) + off * group, nullptr,
+                             evicted_slot + (size_t)s0 * G * b, nullptr, static_cast<cudaStream_t>(stream), Lmax);
       if (st != ROCO_OK) return st;
     }
     s0 = s1;
   }
   return ROCO_OK;
+}
+
+roco_status roco_prefill_blockwise(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax,
+                                   int b, int r, float scale, roco_cache *cache, void *attn_out,
+                                   int32_t *evicted_slot, void *stream) {
+  return roco_prefill_blockwise_gqa(Q, K, V, lens_host, Lmax, b, 1, r, scale, cache, attn_out, evicted_slot, stream);
 }
 
 roco_status roco_gqa_decode_step(roco_cache *cache, const void *Q, const void *k_new, const void *v_new, int group,
@@ -332,7 +346,7 @@ roco_status roco_gqa_decode_step(roco_cache *cache, const void *Q, const void *k
   if (group < 1) return ROCO_ERR_INVALID_ARG;
   if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
   if (group > multi_max_queries() || !multi_fits(cache->B, cache->d, group, 1)) return ROCO_ERR_UNSUPPORTED;
-  return launch_multi_step(*cache, 1, group, 1, Q, k_new, v_new, r, scope_mode, scale, attn_out, lse_out,
+  return launch_multi_step(*cache, group, 1, Q, k_new, v_new, r, scope_mode, scale, attn_out, lse_out,
                            evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
 }
 

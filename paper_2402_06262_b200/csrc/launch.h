@@ -54,14 +54,16 @@ roco_status launch_budget_select_gather(const roco_cache &c, int Lmax, const int
 // box_rows rows and the 128-byte swizzle; false when the driver entry point is unavailable or the encode fails.
 bool make_tensor_map_rows128_bf16(void *map, const void *base, unsigned long long rows, unsigned box_rows);
 
-// Multi-query steps (block-wise evict-and-encode: kind 0, nb == M; grouped-query decode: kind 1, nb == 1).
+// Multi-query steps: nb new tokens per unit, each with M / nb query heads (M = nb * group query rows, row
+// t * group + g = head g of token t).  Block-wise evict-and-encode: group 1; grouped-query decode: nb 1.
 int multi_max_queries();
 bool multi_fits(int B, int d, int M, int nb);
-roco_status launch_multi_step(const roco_cache &c, int kind, int M, int nb, const void *Q, const void *k_new,
+roco_status launch_multi_step(const roco_cache &c, int M, int nb, const void *Q, const void *k_new,
                               const void *v_new, int r, int scope_mode, float scale, void *out, float *lse,
                               int32_t *ev_slot, int32_t *ev_pos, cudaStream_t stream, long long unit_stride_rows = 0);
-// unit_stride_rows > 0: Q, k_new, v_new and out are slices of [U][rows][d] tensors with that many rows per unit
-// (used to step through a prompt block by block); 0: dense [U][M][d] / [U][nb][d].
+// unit_stride_rows > 0: k_new and v_new are slices of [U][rows][d] tensors with that many rows (tokens) per unit,
+// Q and out of [U][rows][group][d] tensors (used to step through a prompt block by block); 0: dense [U][M][d] /
+// [U][nb][d].
 
 // Overlap of the budgeted cache's retained positions with the full cache's B most important tokens (one CTA per
 // unit; full.B * 8 bytes of shared memory).

@@ -30,8 +30,6 @@ constexpr int kMqTile = 16384;
 constexpr int kMqMaxQ = 16;  // queries per step
 constexpr int kMqQPW = 4;    // queries per consumer warp
 
-enum { kMqBlock = 0, kMqGqa = 1 };
-
 struct MultiParams {
   const char *K, *V;
   float *s, *q;
@@ -40,7 +38,8 @@ struct MultiParams {
   char *out;
   float *lse;
   int *ev_slot, *ev_pos;
-  int B, r, scope_mode, stages, M, nb, kind;
+  int B, r, scope_mode, stages, M, nb;
+  int group;  // query heads per new token: M = nb * group, query row i belongs to token i / group of the block
   float scale;
   long long q_ustride, kv_ustride, out_ustride;  // rows (tokens) between consecutive units in Q, K_new/V_new, out
 };
@@ -412,8 +411,8 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
       float ds = 0.f, dq = 0.f;
       int dn;
       if (v.ds && !fresh) {
-        if (p.kind == kMqGqa) {
-          ds = v.ds[j] / (float)M;  // group-wise averaged attention score
+        if (nb == 1) {
+          ds = v.ds[j] / (float)M;  // one token, M heads: group-wise averaged attention score
           dq = ds * ds;
           dn = 1;
         } else {
@@ -421,19 +420,21 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
           dq = v.dq[j];
           dn = M;
         }
-      } else if (p.kind == kMqGqa) {
-        for (int i = 0; i < M; ++i) ds += (fresh && v.pn) ? v.pn[i * nb + jn] : v.z[(size_t)i * Bp + j];
-        ds /= (float)M;  // group-wise averaged attention score
-        dq = ds * ds;
-        dn = 1;
       } else {
-        const int i0 = fresh ? jn : 0;  // query i sees new token jn only if i >= jn
-        for (int i = i0; i < M; ++i) {
-          const float pij = (fresh && v.pn) ? v.pn[i * nb + jn] : v.z[(size_t)i * Bp + j];
-          ds += pij;
-          dq = fmaf(pij, pij, dq);
+        // token t of the block (its `group` query heads) sees new token jn only if t >= jn; the statistics take
+        // the group-wise averaged probability once per token (Sec. 5.3, App. A), which for one head is p itself
+        const int t0 = fresh ? jn : 0, group = p.group;
+        for (int t = t0; t < nb; ++t) {
+          float pb = 0.f;
+          for (int g = 0; g < group; ++g) {
+            const int i = t * group + g;
+            pb += (fresh && v.pn) ? v.pn[i * nb + jn] : v.z[(size_t)i * Bp + j];
+          }
+          if (group > 1) pb = pb / (float)group;
+          ds += pb;
+          dq = fmaf(pb, pb, dq);
         }
-        dn = M - i0;
+        dn = nb - t0;
       }
       p.s[unit_st + j] = s0v[k] + ds;
       p.q[unit_st + j] = q0v[k] + dq;
@@ -572,7 +573,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
     const int i = w / nb, jn = w % nb;
     int slot = sm.ctl[1 + jn];
     if (slot < 0 || slot >= B) slot = 0;
-    sm.z[(size_t)i * Bp + slot] = (p.kind == kMqBlock && jn > i) ? -INFINITY : sm.zn[w];
+    sm.z[(size_t)i * Bp + slot] = (jn > i / p.group) ? -INFINITY : sm.zn[w];
   }
   named_bar_sync(kMqBarConsumers, kMqConsumers);
 
@@ -893,7 +894,7 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
     const int i = w / nb, jn = w % nb;
     int slot = sm.ctl[1 + jn];
     if (slot < 0 || slot >= B) slot = 0;
-    sm.z[(size_t)i * Bp + slot] = (p.kind == kMqBlock && jn > i) ? -INFINITY : sm.zn[w];
+    sm.z[(size_t)i * Bp + slot] = (jn > i / p.group) ? -INFINITY : sm.zn[w];
   }
   named_bar_sync(kMqBarConsumers, kMqConsumers);
 
@@ -1139,7 +1140,7 @@ __global__ void __launch_bounds__(kMqThreads, 2) multi_step_tm_kernel(const __gr
   const float zscale = p.scale * kLog2e;
   const int g = lane >> 2, tq = lane & 3;
   const bool row_lo = g < M, row_hi = g + 8 < M;
-  const bool block = p.kind == kMqBlock;
+  const int grp = p.group;
   // this thread's lane of tensor memory and first column: tile `it` occupies the columns 4 it .. 4 it + 3 with
   // (row g, key 2 tq), (g, 2 tq + 1), (g + 8, 2 tq), (g + 8, 2 tq + 1) of the warp's 8 keys of that tile
   const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * (tmem_cols / 2));
@@ -1222,8 +1223,8 @@ __global__ void __launch_bounds__(kMqThreads, 2) multi_step_tm_kernel(const __gr
   };
   // the new tokens' scores replace whatever the stream brought for their slots (causal inside a block)
   for_new_tokens([&](int jn, float &a, float &b) {
-    a = row_lo ? ((block && jn > g) ? -INFINITY : sm.zn[g * nb + jn]) : -INFINITY;
-    b = row_hi ? ((block && jn > g + 8) ? -INFINITY : sm.zn[(g + 8) * nb + jn]) : -INFINITY;
+    a = row_lo ? ((jn > g / grp) ? -INFINITY : sm.zn[g * nb + jn]) : -INFINITY;
+    b = row_hi ? ((jn > (g + 8) / grp) ? -INFINITY : sm.zn[(g + 8) * nb + jn]) : -INFINITY;
   });
 
   // ---- softmax per query row, in place: maxima, exponentials and sums
@@ -1421,7 +1422,7 @@ bool multi_fits(int B, int d, int M, int nb) {
   return multi_pick_stages(B, d, M, nb) > 0 || (d == 128 && multi_tc_pick_stages(B, M, nb) > 0);
 }
 
-roco_status launch_multi_step(const roco_cache &c, int kind, int M, int nb, const void *Q, const void *k_new,
+roco_status launch_multi_step(const roco_cache &c, int M, int nb, const void *Q, const void *k_new,
                               const void *v_new, int r, int scope_mode, float scale, void *out, float *lse,
                               int32_t *ev_slot, int32_t *ev_pos, cudaStream_t stream, long long unit_stride_rows) {
   MultiParams p;
@@ -1429,16 +1430,19 @@ roco_status launch_multi_step(const roco_cache &c, int kind, int M, int nb, cons
   p.s = c.s; p.q = c.q; p.n = c.n; p.pos = c.pos; p.live = c.live; p.t_next = c.t_next; p.status = c.status;
   p.Q = (const char *)Q; p.k_new = (const char *)k_new; p.v_new = (const char *)v_new;
   p.out = (char *)out; p.lse = lse; p.ev_slot = ev_slot; p.ev_pos = ev_pos;
-  p.B = c.B; p.r = r; p.scope_mode = scope_mode; p.M = M; p.nb = nb; p.kind = kind; p.scale = scale;
-  p.q_ustride = unit_stride_rows > 0 ? unit_stride_rows : M;
+  p.B = c.B; p.r = r; p.scope_mode = scope_mode; p.M = M; p.nb = nb; p.scale = scale;
+  p.group = M / nb;
+  p.q_ustride = unit_stride_rows > 0 ? unit_stride_rows * p.group : M;
   p.kv_ustride = unit_stride_rows > 0 ? unit_stride_rows : nb;
-  p.out_ustride = unit_stride_rows > 0 ? unit_stride_rows : M;
+  p.out_ustride = unit_stride_rows > 0 ? unit_stride_rows * p.group : M;
   const int U = c.S * c.G;
   cudaError_t err;
   if (c.kv_dtype == ROCO_BF16 && c.d == 128 && (long long)U * c.B < 0x7fffffffLL) {
     // tensor-core path; falls through to the CUDA-core path if the tensor maps cannot be built
     CUtensorMap mapK, mapV;
-    const int tm_stages = multi_tm_pick_stages(c.B, M, nb);
+    // the tensor-memory kernel forms per-slot sums over all query rows, which is the statistic only when the rows
+    // are all tokens (one head) or all heads (one token)
+    const int tm_stages = (nb == 1 || nb == M) ? multi_tm_pick_stages(c.B, M, nb) : 0;
     p.stages = tm_stages > 0 ? tm_stages : multi_tc_pick_stages(c.B, M, nb);
     if (p.stages > 0 && make_tensor_map_rows128_bf16(&mapK, c.K, (unsigned long long)U * c.B, 64) &&
         make_tensor_map_rows128_bf16(&mapV, c.V, (unsigned long long)U * c.B, 64)) {

@@ -226,6 +226,43 @@ class BlockParity:
         return res
 
 
+class GqaBlockParity:
+    """Steps key-value-head caches shared by `group` query heads, b tokens per step, on the GPU and in the oracle."""
+
+    def __init__(self, cache: R.Cache, st: oracle.State, units: Sequence[int], b: int, group: int, r: int, tally: Tally,
+                 scale: Optional[float] = None):
+        self.cache, self.st, self.units, self.b, self.group, self.r, self.tally = cache, st, list(units), b, group, r, tally
+        self.scale = cache.d ** -0.5 if scale is None else scale
+        dev = cache.K.device
+        self.out = torch.zeros(cache.S, cache.G, b, group, cache.d, dtype=cache.dtype, device=dev)
+        self.lse = torch.zeros(cache.S, cache.G, b, group, dtype=torch.float32, device=dev)
+        self.ev_slot = torch.zeros(cache.S, cache.G, b, dtype=torch.int32, device=dev)
+        self.ev_pos = torch.zeros(cache.S, cache.G, b, dtype=torch.int32, device=dev)
+
+    def step(self, Q, K_new, V_new, check_state=False):
+        c = self.cache
+        R.roco_gqa_block_step(c, Q, K_new, V_new, self.r, self.out, self.ev_slot, self.ev_pos, self.lse, scale=self.scale)
+        torch.cuda.synchronize()
+        g_slot = unit_view(self.ev_slot, self.units).cpu().numpy()
+        g_pos = unit_view(self.ev_pos, self.units).cpu().numpy()
+        res = oracle.gqa_block_step(self.st, widen(unit_view(Q, self.units)), widen(unit_view(K_new, self.units)),
+                                    widen(unit_view(V_new, self.units)), self.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, self.scale,
+                                    delta=DELTA, force_slots=g_slot)
+        firm = res.near_tie == 0
+        np.testing.assert_array_equal(g_slot[firm], res.choice[firm], err_msg="freed slots differ outside the margin")
+        self.tally.near_ties += int((~firm).sum())
+        np.testing.assert_array_equal(g_slot, res.evicted_slot)
+        np.testing.assert_array_equal(g_pos, res.evicted_pos)
+        self.tally.steps += 1
+        self.tally.decisions += int((res.choice >= 0).sum())
+        g_out = widen(unit_view(self.out, self.units))
+        assert np.abs(g_out - res.out).max() <= out_tol(c.dtype), f"attention output off by {np.abs(g_out - res.out).max()}"
+        np.testing.assert_allclose(widen(unit_view(self.lse, self.units)), res.lse, rtol=0, atol=LSE_ATOL)
+        if check_state:
+            compare_state(c, self.st, self.units, f"after grouped block step {self.tally.steps}")
+        return res
+
+
 class GqaParity:
     """Steps key-value-head caches shared by `group` query heads on the GPU and in the oracle."""
 

@@ -7,7 +7,7 @@ import torch
 import oracle
 import paper_2402_06262_b200 as R
 import workloads as W
-from harness import BlockParity, DecodeParity, GqaParity, Tally, prefill_parity, unit_view, widen
+from harness import BlockParity, DecodeParity, GqaBlockParity, GqaParity, Tally, prefill_parity, unit_view, widen
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -159,3 +159,69 @@ def test_blockwise_prompt_encoding(b, lens):
         assert R.roco_device_status(sub) == 0
     assert tally.decisions >= sum(max(0, L - w.B) for L in lens) * w.G
     assert tally.near_ties <= tally.decisions // 10, tally
+
+
+def grouped_block_tokens(w, step0, b, group, t_pos):
+    """Q [S][G][b][group][d] (head g of token i drawn as an independent query), K_new, V_new [S][G][b][d]."""
+    toks = [W.decode_tokens(w, step0 + i, [t + i for t in t_pos], DEV) for i in range(b)]
+    K = torch.stack([t[1] for t in toks], dim=2).contiguous()
+    V = torch.stack([t[2] for t in toks], dim=2).contiguous()
+    Q = torch.stack([torch.stack([W.decode_tokens(w, 1000 * (g + 1) + step0 + i, [t + i for t in t_pos], DEV)[0]
+                                  for g in range(group)], dim=2) for i in range(b)], dim=2).contiguous()
+    return Q, K, V
+
+
+@pytest.mark.parametrize("b,group", [(2, 2), (4, 4), (2, 8), (8, 2), (3, 5), (4, 1), (1, 4)])
+@pytest.mark.parametrize("dtype,d,B", [("bf16", 128, 300), ("bf16", 128, 302), ("f32", 64, 128)])
+def test_grouped_block_steps_fill_then_evict(b, group, dtype, d, B):
+    """Block-wise evict-and-encode on key-value heads shared by `group` query heads (the paper's block-wise
+    experiment on a grouped-query model): fill phase, mixed phase, eviction of b tokens per step; tensor-core
+    kernel with staged and with plainly loaded statistics, and the CUDA-core kernel."""
+    w = W.scaled(W.LLAMA7B_DECODE, S=2, layers=1, heads=3, d=d, dtype=dtype, prompt_lo=B - 21, prompt_hi=B - 21,
+                 B=B, r=9)
+    tally = Tally()
+    cache, st = prefilled(w, B - 21, tally, range(w.U))
+    par = GqaBlockParity(cache, st, range(w.U), b, group, w.r, tally, scale=w.scale)
+    t = B - 21
+    for i in range(max(4, 40 // b)):
+        par.step(*grouped_block_tokens(w, i * b, b, group, [t] * w.S), check_state=True)
+        t += b
+    assert R.roco_device_status(cache) == 0 and tally.decisions > 0
+
+
+def test_grouped_block_step_llama_shape():
+    """B = 1024, d = 128, bf16 after prefill eviction: 4 tokens x 4 heads per step (16 query rows)."""
+    w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=8, prompt_lo=1500, prompt_hi=1500)
+    tally = Tally()
+    cache, st = prefilled(w, 1500, tally, range(w.U))
+    par = GqaBlockParity(cache, st, range(w.U), 4, 4, w.r, tally, scale=w.scale)
+    for i in range(3):
+        par.step(*grouped_block_tokens(w, 4 * i, 4, 4, [1500 + 4 * i]), check_state=(i == 2))
+    assert tally.decisions == 3 * 4 * w.U
+
+
+def test_grouped_blockwise_prompt_encoding_equals_grouped_block_steps():
+    """roco_prefill_blockwise_gqa (strided prompt tensors, ragged lengths) against the same blocks fed one by one
+    through roco_gqa_block_step, which the tests above hold against the oracle: bit-equal caches and outputs."""
+    b, group = 4, 2
+    w = W.scaled(W.LLAMA7B_DECODE, S=2, layers=1, heads=3, prompt_lo=90, prompt_hi=90, B=48, r=5)
+    lens = [90, 61]
+    _, K, V = prompt_tensors(w, 90)
+    g = torch.Generator(device=DEV); g.manual_seed(3)
+    Q = torch.randn(w.S, w.G, 90, group, w.d, device=DEV, generator=g).to(w.torch_dtype)
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    out = torch.zeros_like(Q)
+    ev = torch.zeros(w.S, w.G, b, dtype=torch.int32, device=DEV)
+    R.roco_prefill_blockwise_gqa(Q, K, V, lens, b, w.r, cache, out, ev, scale=w.scale)
+    for s, L in enumerate(lens):
+        sub = R.Cache(1, w.G, w.B, w.d, w.torch_dtype, DEV)
+        for t0 in range(0, L, b):
+            m = min(b, L - t0)
+            o1 = torch.zeros(1, w.G, m, group, w.d, dtype=w.torch_dtype, device=DEV)
+            e1 = torch.zeros(1, w.G, m, dtype=torch.int32, device=DEV)
+            R.roco_gqa_block_step(sub, Q[s:s + 1, :, t0:t0 + m].contiguous(), K[s:s + 1, :, t0:t0 + m].contiguous(),
+                                  V[s:s + 1, :, t0:t0 + m].contiguous(), w.r, o1, e1, scale=w.scale)
+            assert torch.equal(o1[0], out[s, :, t0:t0 + m])
+        for name in ("K", "V", "s", "q", "n", "pos", "live", "t_next"):
+            assert torch.equal(getattr(sub, name)[0], getattr(cache, name)[s]), name
+    assert R.roco_device_status(cache) == 0
