@@ -233,6 +233,24 @@ def prefill_bench(R, device, small=False, reps=5, workload="llama7b_prefill", wi
         ex_a = w.U * (Tt * (Tt + 1) // 2) * 2 * 2 * 128 ** 3      # Q K^T and P V per tile
         attend = {"ms": best_a * 1e3, "ms_whole_workload": best_a * 1e3 * scale_units,
                   "tflops_executed": ex_a / best_a / 1e12, "frac_executed": ex_a / best_a / 1e12 / bf16_peak}
+        # the same outputs from one call: the sweep that yields the row log-sum-exp also accumulates P.V
+        best_f = float("inf")
+        R.roco_prefill(Q, K, V, [L], w.B, w.r, cache, scale=w.scale, workspace=ws, attn_out=out)
+        torch.cuda.synchronize()
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            R.roco_prefill(Q, K, V, [L], w.B, w.r, cache, scale=w.scale, workspace=ws, attn_out=out)
+            e1.record()
+            torch.cuda.synchronize()
+            best_f = min(best_f, e0.elapsed_time(e1) / 1e3)
+        ex_f = w.U * (Tt * (Tt + 1) // 2) * 3 * 2 * 128 ** 3      # scores + P V in the sweep, scores again for the statistics
+        attend["fused_call"] = {"ms": best_f * 1e3, "ms_whole_workload": best_f * 1e3 * scale_units,
+                                "what": "roco_prefill_with_output: statistics + eviction to budget + attention output, "
+                                        "three L x L contractions",
+                                "ms_separate_calls": (best + best_a) * 1e3,
+                                "tflops_executed": ex_f / best_f / 1e12,
+                                "frac_executed": ex_f / best_f / 1e12 / bf16_peak}
         del out, lse
     if R.roco_device_status(cache) != 0:
         raise RuntimeError("device status word set during prefill")

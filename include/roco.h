@@ -125,6 +125,22 @@ roco_status roco_prefill(const void *Q, const void *K, const void *V, const int3
                          size_t workspace_bytes, void *stream);
 
 /*
+ * roco_prefill that also returns the prompt's attention output (Eq. 1 with the causal mask of Sec. 2.1), for
+ * callers that need the layer's output and not only the budgeted cache:
+ *     attn_out_i = sum_{j<=i} softmax_j(scale * Q_i.K_j) V_j,      i < lens
+ * The output comes from the same sweep over the score tiles that yields the row log-sum-exp (running row maximum,
+ * output accumulator rescaled when the maximum moves), so the whole call costs three L x L contractions (scores
+ * and P.V in the sweep, scores again for the column statistics) instead of the four of roco_prefill followed by
+ * roco_prefill_attend.  Tensor cores only: kv_dtype ROCO_BF16 and d = 128, else ROCO_ERR_UNSUPPORTED; scale > 0.
+ *   attn_out     [S][G][Lmax][d] device, 16-byte aligned; rows >= lens are left untouched; NULL: roco_prefill
+ * All other arguments, results and errors as roco_prefill.
+ */
+roco_status roco_prefill_with_output(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax,
+                                     int B, int r, int scope_mode, int count_self, float scale, roco_cache *cache,
+                                     float *lse_out, float *s_full, float *q_full, void *attn_out, void *workspace,
+                                     size_t workspace_bytes, void *stream);
+
+/*
  * roco_prefill without a caller-provided workspace.  The paper has no counterpart: this exists for callers
  * that cannot allocate device memory at call time -- code running inside a serving runtime whose memory
  * pool already owns the GPU (cudaMalloc fails there), or a latency-critical loop that must not call

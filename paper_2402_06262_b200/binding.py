@@ -29,7 +29,7 @@ EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes",
            "roco_prefill_attend_workspace_bytes", "roco_prefill_attend", "roco_selftest_wait_timeout",
            "roco_consistency_step", "roco_selftest_read_stream", "roco_decode_host_pipeline_staging_bytes",
            "roco_decode_step_host_begin", "roco_decode_step_host_end", "roco_gqa_block_step",
-           "roco_prefill_blockwise_gqa")
+           "roco_prefill_blockwise_gqa", "roco_prefill_with_output")
 
 
 class RocoError(RuntimeError):
@@ -70,6 +70,10 @@ def lib() -> C.CDLL:
         L.roco_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
                                    C.c_int, C.c_float, C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_void_p, C.c_size_t, C.c_void_p]
+        L.roco_prefill_with_output.restype = C.c_int
+        L.roco_prefill_with_output.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                               C.c_int, C.c_int, C.c_int, C.c_float, C.POINTER(roco_cache), C.c_void_p,
+                                               C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.roco_prefill_static.restype = C.c_int
         L.roco_prefill_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                           C.c_int, C.c_int, C.c_float, C.POINTER(roco_cache), C.c_void_p, C.c_void_p,
@@ -182,8 +186,9 @@ def roco_prefill_uses_tensor_cores(cache: Cache) -> bool:
 
 def roco_prefill(Q, K, V, lens: Sequence[int], B: int, r: int, cache: Cache, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R,
                  count_self=1, scale: Optional[float] = None, lse_out=None, s_full=None, q_full=None,
-                 workspace: Optional[torch.Tensor] = None):
-    """Q, K, V: [S][G][Lmax][d] device tensors.  Fills `cache`."""
+                 workspace: Optional[torch.Tensor] = None, attn_out=None):
+    """Q, K, V: [S][G][Lmax][d] device tensors.  Fills `cache`.  attn_out ([S][G][Lmax][d], bf16, d = 128): also
+    the prompt's causal attention output (roco_prefill_with_output)."""
     Lmax = Q.shape[2]
     scale = cache.d ** -0.5 if scale is None else scale
     if workspace is None:
@@ -191,9 +196,15 @@ def roco_prefill(Q, K, V, lens: Sequence[int], B: int, r: int, cache: Cache, sco
                   else roco_prefill_workspace_bytes)(cache, Lmax)
         workspace = torch.empty(nbytes, dtype=torch.uint8, device=Q.device)
     lens_arr = (C.c_int32 * len(lens))(*[int(x) for x in lens])
-    rc = lib().roco_prefill(_ptr(Q), _ptr(K), _ptr(V), C.cast(lens_arr, C.c_void_p), Lmax, B, r, scope_mode,
-                            count_self, scale, C.byref(cache.c), _ptr(lse_out), _ptr(s_full), _ptr(q_full),
-                            _ptr(workspace), workspace.numel(), _stream())
+    if attn_out is not None:
+        rc = lib().roco_prefill_with_output(_ptr(Q), _ptr(K), _ptr(V), C.cast(lens_arr, C.c_void_p), Lmax, B, r,
+                                            scope_mode, count_self, scale, C.byref(cache.c), _ptr(lse_out),
+                                            _ptr(s_full), _ptr(q_full), _ptr(attn_out), _ptr(workspace),
+                                            workspace.numel(), _stream())
+    else:
+        rc = lib().roco_prefill(_ptr(Q), _ptr(K), _ptr(V), C.cast(lens_arr, C.c_void_p), Lmax, B, r, scope_mode,
+                                count_self, scale, C.byref(cache.c), _ptr(lse_out), _ptr(s_full), _ptr(q_full),
+                                _ptr(workspace), workspace.numel(), _stream())
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_prefill")
     return workspace
@@ -332,7 +343,7 @@ def roco_prefill_blockwise_gqa(Q, K, V, lens: Sequence[int], b: int, r: int, cac
                                           int(Q.shape[3]), r, scale, C.byref(cache.c), _ptr(attn_out),
                                           _ptr(evicted_slot), _stream())
     if rc != ROCO_OK:
-        raise RocoError(rc, "roco_prefill_blockwise_gqa")
+        raise RocoError(rc, "roco_prefill_blockwise_gqa", "roco_prefill_with_output")
 
 
 def roco_gqa_decode_step(cache: Cache, Q, k_new, v_new, r: int, attn_out, evicted_slot, evicted_pos=None,
@@ -354,7 +365,7 @@ def roco_consistency_step(full: Cache, budgeted: Cache, policy: int, overlap, ja
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_consistency_step", "roco_selftest_read_stream", "roco_decode_host_pipeline_staging_bytes",
            "roco_decode_step_host_begin", "roco_decode_step_host_end", "roco_gqa_block_step",
-           "roco_prefill_blockwise_gqa")
+           "roco_prefill_blockwise_gqa", "roco_prefill_with_output")
 
 
 def roco_decode_host_staging_bytes(cache: Cache) -> int:

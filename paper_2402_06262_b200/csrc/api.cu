@@ -139,6 +139,14 @@ int roco_prefill_uses_tensor_cores(const roco_cache *cache) {
 roco_status roco_prefill(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax, int B,
                          int r, int scope_mode, int count_self, float scale, roco_cache *cache, float *lse_out,
                          float *s_full, float *q_full, void *workspace, size_t workspace_bytes, void *stream) {
+  return roco_prefill_with_output(Q, K, V, lens_host, Lmax, B, r, scope_mode, count_self, scale, cache, lse_out,
+                                  s_full, q_full, nullptr, workspace, workspace_bytes, stream);
+}
+
+roco_status roco_prefill_with_output(const void *Q, const void *K, const void *V, const int32_t *lens_host, int Lmax,
+                                     int B, int r, int scope_mode, int count_self, float scale, roco_cache *cache,
+                                     float *lse_out, float *s_full, float *q_full, void *attn_out, void *workspace,
+                                     size_t workspace_bytes, void *stream) {
   NvtxRange range("roco_prefill");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
@@ -146,6 +154,10 @@ roco_status roco_prefill(const void *Q, const void *K, const void *V, const int3
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V)) return ROCO_ERR_INVALID_ARG;
   if ((st = check_scope(r, scope_mode, B, false)) != ROCO_OK) return st;
   if (count_self != 1) return ROCO_ERR_UNSUPPORTED;
+  if (attn_out) {  // the prompt's attention output from the same sweep that yields the row log-sum-exp
+    if (!prefill_tc_supported(cache->kv_dtype, cache->d)) return ROCO_ERR_UNSUPPORTED;
+    if (!aligned16(attn_out) || !(scale > 0.f)) return ROCO_ERR_INVALID_ARG;
+  }
   int maxlen = 0;
   for (int b = 0; b < cache->S; ++b) {
     if (lens_host[b] < 1 || lens_host[b] > Lmax) return ROCO_ERR_INVALID_ARG;
@@ -167,7 +179,13 @@ roco_status roco_prefill(const void *Q, const void *K, const void *V, const int3
   int *dst = reinterpret_cast<int *>(ws + w.dst_off);
   if (cudaMemcpyAsync(lens_dev, lens_host, (size_t)cache->S * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess)
     return ROCO_ERR_CUDA;
-  if (prefill_tc_supported(cache->kv_dtype, cache->d))
+  if (attn_out) {
+    st = launch_prefill_attend_tc(cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, V, scale, nullptr, lse, attn_out,
+                                  cache->status, cs);
+    if (st == ROCO_OK)
+      st = launch_prefill_stats_tc(cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, scale, lse, sf, qf,
+                                   cache->status, cs, true);
+  } else if (prefill_tc_supported(cache->kv_dtype, cache->d))
     st = launch_prefill_stats_tc(cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, scale, lse, sf, qf, cache->status,
                                  cs);
   else
@@ -204,7 +222,7 @@ roco_status roco_prefill_attend(const roco_cache *cache, const void *Q, const vo
   int *lens_dev = static_cast<int *>(workspace);
   if (cudaMemcpyAsync(lens_dev, lens_host, (size_t)cache->S * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess)
     return ROCO_ERR_CUDA;
-  return launch_prefill_attend_tc(cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, V, scale, lse, attn_out,
+  return launch_prefill_attend_tc(cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, V, scale, lse, nullptr, attn_out,
                                   cache->status, cs);
 }
 

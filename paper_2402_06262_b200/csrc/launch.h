@@ -25,21 +25,24 @@ roco_status launch_prefill_stats_simt(int kv_dtype, int d, int S, int G, int Lma
                                       const void *Q, const void *K, float scale, float *lse, float *s_full,
                                       float *q_full, cudaStream_t stream);
 
-// The same two passes on tcgen05 tensor cores with TMA-fed operands (bf16, d = 128 only).
+// The same two passes on tcgen05 tensor cores with TMA-fed operands (bf16, d = 128 only).  lse_ready: `lse`
+// already holds the row log-sum-exp (from the one-sweep attention kernel), so only the statistics pass runs.
 bool prefill_tc_supported(int kv_dtype, int d);
 roco_status launch_prefill_stats_tc(int S, int G, int Lmax, const int *lens_dev, int maxlen, const void *Q,
                                     const void *K, float scale, float *lse, float *s_full, float *q_full, int *status,
-                                    cudaStream_t stream);
+                                    cudaStream_t stream, bool lse_ready = false);
 
 // Tensor map (CUtensorMap, 128 bytes, passed as void*) over a [U][Lmax][128] bf16 prompt tensor with boxes of
 // 64 columns x 128 rows x 1 unit and the 128-byte swizzle; rows past Lmax read as zero.
 bool make_tensor_map_prompt_bf16(void *map, const void *base, int U, int Lmax);
 
 // Causal attention output of the prompt pass on the tensor cores (bf16, d = 128): out_i = sum_{j<=i}
-// exp(scale Q_i.K_j - lse_i) V_j with the row log-sum-exp `lse` the statistics pass produced.  out: [U][Lmax][128].
+// exp(scale Q_i.K_j - lse_i) V_j.  out: [U][Lmax][128].  With lse_in the row log-sum-exp is taken from there
+// (lse_out unused); with lse_in == nullptr one sweep with a running row maximum produces both the output and
+// lse_out [U][Lmax] (scale > 0).
 roco_status launch_prefill_attend_tc(int S, int G, int Lmax, const int *lens_dev, int maxlen, const void *Q,
-                                     const void *K, const void *V, float scale, const float *lse, void *out,
-                                     int *status, cudaStream_t stream);
+                                     const void *K, const void *V, float scale, const float *lse_in, float *lse_out,
+                                     void *out, int *status, cudaStream_t stream);
 
 // Select-to-budget on frozen statistics and gather of the survivors into the cache.
 // dst: [U][Lmax] int32 scratch (destination slot per token, -1 = evicted).  LOWEST_R with eviction also needs

@@ -66,6 +66,13 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
       : "memory");
 }
 
+// max of three in one instruction
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 struct AtSmem {
@@ -110,10 +117,24 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t *>(&v);
 }
 
+// kOnline: a row is moved to a new reference when the sum of one 32-column chunk of its unnormalised
+// probabilities 2^(z - reference) reaches 2^60 (or is not finite).  Up to there bf16 and fp32 hold the values with
+// their full relative precision, and whatever an fp32 sum drops beside such a term is below its last bit anyway.
+constexpr float kAtRescaleLimit = 1152921504606846976.f;  // 2^60
+
+// kOnline = false: the row log-sum-exp comes from `lse_in` (computed earlier for the same Q, K).
+// kOnline = true:  one sweep yields both: every softmax thread keeps a reference maximum m and the running sum
+//   l = sum_j 2^(z_j - m) of its query row (m = the maximum over the row's first key tile, to begin with); P =
+//   2^(z - m) goes to the output contraction unnormalised; when a chunk of P grows past kAtRescaleLimit, m moves to
+//   that chunk's maximum and the row of the output accumulator, l and the part of the current P tile already
+//   written are scaled by 2^(m_old - m_new) (the accumulator is idle at
+//   that point: S_h(j) complete implies PV_h(j-1) complete, and PV_h(j) is issued only after this thread's
+//   arrival).  At the end out = O / l and lse = (m + log2 l) ln 2 is written to `lse_out`.  Needs scale > 0.
+template <bool kOnline>
 __global__ void __launch_bounds__(kAtThreads, 1)
     prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                              const __grid_constant__ CUtensorMap mapV, const int *lens, int G, int Lmax, int npairs,
-                             float scale, const float *lse, __nv_bfloat16 *out, int *status) {
+                             float scale, const float *lse_in, float *lse_out, __nv_bfloat16 *out, int *status) {
   extern __shared__ char at_smem_raw[];
   const AtSmem sm = at_carve(at_smem_raw);
   volatile int *abort_flag = sm.abort_flag;
@@ -244,29 +265,106 @@ __global__ void __launch_bounds__(kAtThreads, 1)
       if (h < nq) {
         const int a = 2 * A + h;  // this group's 128-row query tile; its diagonal key tile
         const int grow = a * kTcTile + row;
-        const float nl2 = (grow < L) ? -lse[(size_t)u * Lmax + grow] * kLog2e : 0.f;
-        const f32x2 nl22 = pack2(nl2, nl2), zs2 = pack2(zscale, zscale);
+        float nl2 = 0.f, m_ref = -INFINITY, lsum = 0.f;
+        if constexpr (!kOnline) nl2 = (grow < L) ? -lse_in[(size_t)u * Lmax + grow] * kLog2e : 0.f;
+        f32x2 nl22 = pack2(nl2, nl2);
+        const f32x2 zs2 = pack2(zscale, zscale);
+        const uint32_t oaddr = tmem + lane_addr + (uint32_t)(kAtColO + h * kTcTile);
         for (int j = 0; j <= a; ++j, ++mine) {
           mbar_wait(&sm.s_full[h], mine & 1, abort_flag, status);
           tc_fence_after();
           const int col0 = j * kTcTile;
           uint32_t ra[32], rb[32];
+          if constexpr (kOnline) {
+            if (j == 0) {  // the row's reference maximum starts as the maximum over its first key tile
+              float mx = -INFINITY;
+#pragma unroll 1
+              for (int c = 0; c < 4; ++c) {
+                tmem_ld32_issue(taddr + c * 32, ra);
+                tmem_ld_wait(ra);
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  mx = fmaxf(mx, (a > 0 || c * 32 + i <= grow) ? __uint_as_float(ra[i]) : -INFINITY);
+              }
+              m_ref = mx * zscale;
+              nl22 = pack2(-m_ref, -m_ref);
+            }
+          }
+          // kOnline: move the row's reference maximum up to `cz` (where `need`) before chunk c of this tile
+          auto rescale_row = [&](int c, bool need, float cz) {
+            const float m_new = need ? cz : m_ref;
+            const float f = need ? exp2f(m_ref - m_new) : 1.f;
+            lsum *= f;
+            uint32_t t16[16];
+#pragma unroll 1
+            for (int cc = 0; cc < kTcD / 16; ++cc) {  // the output accumulator's row (j > 0 here: it is valid)
+              tmem_ld16(oaddr + cc * 16, t16);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) t16[i] = __float_as_uint(__uint_as_float(t16[i]) * f);
+              tmem_st16(oaddr + cc * 16, t16);
+            }
+#pragma unroll 1
+            for (int c2 = 0; c2 < c; ++c2) {  // the chunks of this tile's P written so far (packed bf16 pairs)
+              tmem_ld16(taddr + c2 * 16, t16);
+#pragma unroll
+              for (int i = 0; i < 16; ++i)
+                t16[i] = pack_bf16x2(__uint_as_float(t16[i] << 16) * f, __uint_as_float(t16[i] & 0xffff0000u) * f);
+              tmem_st16(taddr + c2 * 16, t16);
+            }
+            tmem_st_wait();
+            m_ref = m_new;
+            nl22 = pack2(-m_ref, -m_ref);
+          };
 
           auto chunk = [&](const uint32_t (&r)[32], int c, auto masked_tag) {
             constexpr bool kMasked = decltype(masked_tag)::value;
             uint32_t pk[16];
+            float ls = 0.f;
+            // P of the chunk against the current reference (packed bf16 pairs in pk, their fp32 sum in ls)
+            auto exponentials = [&]() {
+              ls = 0.f;
+              [[maybe_unused]] f32x2 ls2 = pack2(0.f, 0.f);
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              f32x2 p2 = ((i >> 1) & 7) < kAtPolyPairsPer8 ? exp2_poly2(fma2(pack2u(r[i], r[i + 1]), zs2, nl22))
-                                                         : exp2_mufu2(fma2(pack2u(r[i], r[i + 1]), zs2, nl22));
-              float pa, pb;
-              unpack2(p2, pa, pb);
-              if (kMasked) {
-                const int kj = col0 + c * 32 + i;
-                pa = (kj <= grow) ? pa : 0.f;
-                pb = (kj + 1 <= grow) ? pb : 0.f;
+              for (int i = 0; i < 32; i += 2) {
+                f32x2 p2 = ((i >> 1) & 7) < kAtPolyPairsPer8 ? exp2_poly2(fma2(pack2u(r[i], r[i + 1]), zs2, nl22))
+                                                           : exp2_mufu2(fma2(pack2u(r[i], r[i + 1]), zs2, nl22));
+                float pa, pb;
+                unpack2(p2, pa, pb);
+                if (kMasked) {
+                  const int kj = col0 + c * 32 + i;
+                  pa = (kj <= grow) ? pa : 0.f;
+                  pb = (kj + 1 <= grow) ? pb : 0.f;
+                }
+                if constexpr (kOnline) {
+                  if constexpr (kMasked) ls += pa + pb; else ls2 = add2(ls2, p2);
+                }
+                pk[i >> 1] = pack_bf16x2(pa, pb);
               }
-              pk[i >> 1] = pack_bf16x2(pa, pb);
+              if constexpr (kOnline) {
+                float la, lb;
+                unpack2(ls2, la, lb);
+                ls += la + lb;
+              }
+            };
+            if constexpr (!kOnline) {
+              exponentials();
+            } else {
+              // No maximum is formed ahead of the exponentials: a score far above the row's reference shows in
+              // the chunk's sum (beyond 2^kAtRescaleLog2, or not finite).  Only then is the chunk's maximum
+              // taken, the row moved to it, and the chunk done again -- once, since its maximum is then the
+              // reference.
+#pragma unroll 1
+              for (int pass = 0; pass < 2; ++pass) {
+                exponentials();
+                const bool need = !(ls < kAtRescaleLimit);
+                if (pass == 1 || j == 0 || !__any_sync(0xffffffffu, need)) break;
+                float cm = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  cm = fmaxf(cm, (!kMasked || col0 + c * 32 + i <= grow) ? __uint_as_float(r[i]) : -INFINITY);
+                rescale_row(c, need, cm * zscale);
+              }
+              lsum += ls;
             }
             tmem_st16(taddr + c * 16, pk);  // behind the columns already read
           };
@@ -306,12 +404,20 @@ __global__ void __launch_bounds__(kAtThreads, 1)
         // the finished output accumulator of this query tile: one row per thread
         mbar_wait(&sm.o_full[h], k & 1, abort_flag, status);
         tc_fence_after();
-        const uint32_t oaddr = tmem + lane_addr + (uint32_t)(kAtColO + h * kTcTile);
         uint32_t r[32];
+        float inv = 1.f;
+        if constexpr (kOnline) {
+          inv = 1.f / lsum;
+          if (grow < L) lse_out[(size_t)u * Lmax + grow] = (m_ref + log2f(lsum)) * kLn2;
+        }
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           tmem_ld32_issue(oaddr + c * 32, r);
           tmem_ld_wait(r);
+          if constexpr (kOnline) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * inv);
+          }
           if (grow < L) {
             uint4 *dst = reinterpret_cast<uint4 *>(out + ((size_t)u * Lmax + grow) * kTcD + c * 32);
 #pragma unroll
@@ -335,8 +441,8 @@ __global__ void __launch_bounds__(kAtThreads, 1)
 }
 
 roco_status launch_prefill_attend_tc(int S, int G, int Lmax, const int *lens_dev, int maxlen, const void *Q,
-                                     const void *K, const void *V, float scale, const float *lse, void *out,
-                                     int *status, cudaStream_t stream) {
+                                     const void *K, const void *V, float scale, const float *lse_in, float *lse_out,
+                                     void *out, int *status, cudaStream_t stream) {
   CUtensorMap mapQ, mapK, mapV;
   const int U = S * G;
   if (!make_tensor_map_prompt_bf16(&mapQ, Q, U, Lmax) || !make_tensor_map_prompt_bf16(&mapK, K, U, Lmax) ||
@@ -346,12 +452,15 @@ roco_status launch_prefill_attend_tc(int S, int G, int Lmax, const int *lens_dev
   const int T2 = (T + 1) / 2;
   const int npairs = (T2 + 1) / 2;
   const unsigned grid = (unsigned)U * (unsigned)npairs;
-  if (cudaFuncSetAttribute(prefill_attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)kAtSmemBytes) != cudaSuccess)
-    return ROCO_ERR_CUDA;
-  prefill_attend_tc_kernel<<<grid, kAtThreads, kAtSmemBytes, stream>>>(
-      mapQ, mapK, mapV, lens_dev, G, Lmax, npairs, scale, lse, static_cast<__nv_bfloat16 *>(out), status);
-  return cudaGetLastError() == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
+  auto launch = [&](auto kernel) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtSmemBytes) != cudaSuccess)
+      return ROCO_ERR_CUDA;
+    kernel<<<grid, kAtThreads, kAtSmemBytes, stream>>>(mapQ, mapK, mapV, lens_dev, G, Lmax, npairs, scale, lse_in,
+                                                      lse_out, static_cast<__nv_bfloat16 *>(out), status);
+    return cudaGetLastError() == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
+  };
+  // lse_in given: the output alone from a known row log-sum-exp; else one sweep that also produces lse_out
+  return lse_in ? launch(prefill_attend_tc_kernel<false>) : launch(prefill_attend_tc_kernel<true>);
 }
 
 }  // namespace roco

@@ -341,7 +341,7 @@ bool prefill_tc_supported(int kv_dtype, int d) { return kv_dtype == ROCO_BF16 &&
 
 roco_status launch_prefill_stats_tc(int S, int G, int Lmax, const int *lens_dev, int maxlen, const void *Q,
                                     const void *K, float scale, float *lse, float *s_full, float *q_full, int *status,
-                                    cudaStream_t stream) {
+                                    cudaStream_t stream, bool lse_ready) {
   CUtensorMap mapQ, mapK;
   const int U = S * G;
   if (!make_tensor_map_prompt_bf16(&mapQ, Q, U, Lmax) || !make_tensor_map_prompt_bf16(&mapK, K, U, Lmax))
@@ -354,8 +354,9 @@ roco_status launch_prefill_stats_tc(int S, int G, int Lmax, const int *lens_dev,
   if (err == cudaSuccess)
     err = cudaFuncSetAttribute(prefill_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes);
   if (err != cudaSuccess) return ROCO_ERR_CUDA;
-  prefill_tc_kernel<0><<<grid, kTcThreads, kTcSmemBytes, stream>>>(mapQ, mapK, lens_dev, G, Lmax, npairs, scale, lse,
-                                                                  s_full, q_full, status);
+  if (!lse_ready)
+    prefill_tc_kernel<0><<<grid, kTcThreads, kTcSmemBytes, stream>>>(mapQ, mapK, lens_dev, G, Lmax, npairs, scale, lse,
+                                                                    s_full, q_full, status);
   prefill_tc_kernel<1><<<grid, kTcThreads, kTcSmemBytes, stream>>>(mapQ, mapK, lens_dev, G, Lmax, npairs, scale, lse,
                                                                   s_full, q_full, status);
   return cudaGetLastError() == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;

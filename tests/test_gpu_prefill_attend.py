@@ -80,3 +80,95 @@ def test_attend_rejects_unsupported_shapes():
     lse = torch.zeros(w.S, w.G, 128, device=DEV)
     with pytest.raises(R.RocoError):
         R.roco_prefill_attend(cache, Q, Q, Q, [128], lse, torch.zeros_like(Q))
+
+
+# ------------------------------------------------ one sweep: output and row log-sum-exp together (running maximum)
+
+def run_fused(w, lens, Lmax, edit=None, poison_padding=False):
+    Q, K, V = prompt_tensors(w, Lmax)
+    if edit is not None:
+        edit(Q, K, V)
+    if poison_padding:
+        for b, L in enumerate(lens):
+            for X in (Q, K, V):
+                X[b, :, L:] = float("nan")
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    lse = torch.zeros(w.S, w.G, Lmax, dtype=torch.float32, device=DEV)
+    sf = torch.zeros_like(lse); qf = torch.zeros_like(lse)
+    out = torch.full((w.S, w.G, Lmax, w.d), 7.0, dtype=w.torch_dtype, device=DEV)
+    R.roco_prefill(Q, K, V, lens, w.B, w.r, cache, scale=w.scale, lse_out=lse, s_full=sf, q_full=qf, attn_out=out)
+    torch.cuda.synchronize()
+    assert R.roco_device_status(cache) == 0
+    return Q, K, V, lse, out, cache, sf, qf
+
+
+def plain_prefill(w, Q, K, V, lens, Lmax):
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    lse = torch.zeros(w.S, w.G, Lmax, dtype=torch.float32, device=DEV)
+    sf = torch.zeros_like(lse); qf = torch.zeros_like(lse)
+    R.roco_prefill(Q, K, V, lens, w.B, w.r, cache, scale=w.scale, lse_out=lse, s_full=sf, q_full=qf)
+    torch.cuda.synchronize()
+    return cache, lse, sf, qf
+
+
+@pytest.mark.parametrize("kind", ["iid", "sink", "lowrank"])
+def test_fused_prompt_pass_every_row_ragged(kind):
+    """roco_prefill with attn_out: output and log-sum-exp of every row against the oracle, and the statistics and
+    the budgeted cache against the call without the output (which the other tests hold against the oracle)."""
+    w = W.scaled(W.LLAMA7B_PREFILL, S=4, layers=1, heads=3, prompt_lo=520, prompt_hi=520, B=64, r=8, kind=kind)
+    lens = [520, 333, 128, 7]
+    Q, K, V, lse, out, cache, sf, qf = run_fused(w, lens, 520, poison_padding=True)
+    check_rows(w, Q, K, V, lse, out, lens, range(w.U), lambda L: list(range(L)))
+    ref, lse0, sf0, qf0 = plain_prefill(w, Q, K, V, lens, 520)
+    for b, L in enumerate(lens):
+        np.testing.assert_allclose(lse[b, :, :L].cpu().numpy(), lse0[b, :, :L].cpu().numpy(), rtol=0, atol=2e-5)
+        np.testing.assert_allclose(sf[b, :, :L].cpu().numpy(), sf0[b, :, :L].cpu().numpy(), rtol=1e-4)
+        np.testing.assert_allclose(qf[b, :, :L].cpu().numpy(), qf0[b, :, :L].cpu().numpy(), rtol=1e-4)
+    assert torch.equal(cache.live, ref.live) and torch.equal(cache.n, ref.n)
+    assert (cache.pos != ref.pos).float().mean().item() <= 0.01      # survivors equal up to decisions inside the margin
+
+
+def test_fused_prompt_pass_moves_the_row_maximum():
+    """Keys planted late in the prompt that beat every earlier score by far: the reference maximum of all later
+    rows has to move (several times, in different 32-column chunks of a tile), which rescales the output
+    accumulator, the running sum and the part of the current P tile already written."""
+    w = W.scaled(W.LLAMA7B_PREFILL, S=1, layers=1, heads=4, prompt_lo=900, prompt_hi=900, B=128, r=8, kind="iid")
+    # position -> strength: logits of about 3 x strength, each ~48 nats (69 powers of two) above the one before,
+    # past the 2^60 at which a row moves its reference; chunks 3, 1, 0, 2 of their key tiles
+    planted = {230: 16.0, 417: 32.0, 640: 48.0, 705: 64.0}
+
+    def edit(Q, K, V):
+        g = torch.Generator(device=DEV); g.manual_seed(7)
+        u = torch.randn(w.S, w.G, 1, w.d, device=DEV, generator=g)
+        u = u / u.norm(dim=-1, keepdim=True)
+        Q += (3.0 * u).to(Q.dtype)                               # every query has a component along u
+        for pos, strength in planted.items():
+            K[:, :, pos] = (strength * w.d ** 0.5 * u[:, :, 0]).to(K.dtype)
+            V[:, :, pos] = float(pos) / 100.0
+
+    Q, K, V, lse, out, cache, _, _ = run_fused(w, [900], 900, edit=edit)
+    check_rows(w, Q, K, V, lse, out, [900], range(w.U), lambda L: list(range(L)))
+    # the planted keys dominate: rows after the last one return (nearly) its value, so the rescaling was exercised
+    assert abs(float(out[0, 0, 899, 0]) - 7.05) < 0.1
+
+
+def test_fused_prompt_pass_long_prompt_sampled_rows():
+    w = W.scaled(W.LLAMA7B_PREFILL, S=1, layers=1, heads=8, prompt_lo=4096, prompt_hi=4096, B=1024, r=64)
+    Q, K, V, lse, out, cache, _, _ = run_fused(w, [4096], 4096)
+    rows = [0, 1, 127, 128, 129, 2047, 2048, 3000, 3967, 3968, 4095]
+    check_rows(w, Q, K, V, lse, out, [4096], [0, 3, 7], lambda L: rows)
+
+
+def test_fused_prompt_pass_argument_checks():
+    w = W.scaled(W.LLAMA7B_PREFILL, S=1, layers=1, heads=1, prompt_lo=128, prompt_hi=128, B=64, r=8)
+    Q, K, V = prompt_tensors(w, 128)
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    with pytest.raises(R.RocoError) as e:                        # the running-maximum sweep needs scale > 0
+        R.roco_prefill(Q, K, V, [128], w.B, w.r, cache, scale=-0.1, attn_out=torch.zeros_like(Q))
+    assert e.value.code == 1
+    t = W.TOY                                                    # fp32, d = 64: no tensor-core path
+    c2 = R.Cache(t.S, t.G, t.B, t.d, t.torch_dtype, DEV)
+    X = torch.zeros(t.S, t.G, 128, t.d, device=DEV)
+    with pytest.raises(R.RocoError) as e:
+        R.roco_prefill(X, X, X, [128], t.B, t.r, c2, attn_out=torch.zeros_like(X))
+    assert e.value.code == 2
