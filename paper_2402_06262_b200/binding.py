@@ -343,7 +343,7 @@ def roco_prefill_blockwise_gqa(Q, K, V, lens: Sequence[int], b: int, r: int, cac
                                           int(Q.shape[3]), r, scale, C.byref(cache.c), _ptr(attn_out),
                                           _ptr(evicted_slot), _stream())
     if rc != ROCO_OK:
-        raise RocoError(rc, "roco_prefill_blockwise_gqa", "roco_prefill_with_output")
+        raise RocoError(rc, "roco_prefill_blockwise_gqa")
 
 
 def roco_gqa_decode_step(cache: Cache, Q, k_new, v_new, r: int, attn_out, evicted_slot, evicted_pos=None,
@@ -363,9 +363,7 @@ def roco_consistency_step(full: Cache, budgeted: Cache, policy: int, overlap, ja
     rc = lib().roco_consistency_step(C.byref(full.c), C.byref(budgeted.c), policy, _ptr(overlap), _ptr(jaccard_sum),
                                      _ptr(samples), _stream())
     if rc != ROCO_OK:
-        raise RocoError(rc, "roco_consistency_step", "roco_selftest_read_stream", "roco_decode_host_pipeline_staging_bytes",
-           "roco_decode_step_host_begin", "roco_decode_step_host_end", "roco_gqa_block_step",
-           "roco_prefill_blockwise_gqa", "roco_prefill_with_output")
+        raise RocoError(rc, "roco_consistency_step")
 
 
 def roco_decode_host_staging_bytes(cache: Cache) -> int:
