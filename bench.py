@@ -315,39 +315,7 @@ def multi_bench(R, cache, w, device, reps=6):
         base = base or ms
         res["block"].append({"b": b, "ms_per_step": ms, "tokens_per_s": w.S * b / ms * 1e3,
                              "speedup_vs_b1_per_token": base * b / ms, "hbm_frac": alg / ms / 1e6 / hbm_peak})
-    # calls with few units (one layer at a time, what a transformer's decode loop does): the same step with each
-    # unit's slots divided among several CTAs.  Two cases: one layer of the decode workload, and one layer of a
-    # single long-context sequence (32 units, B = 8192).  L2 is flushed between launches (the caches are small).
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
-    def timed_cold(fn):
-        ts = []
-        for _ in range(reps + 2):
-            flush.zero_()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(); fn(); e1.record(); torch.cuda.synchronize()
-            ts.append(e0.elapsed_time(e1))
-        return statistics.median(ts[2:])
-    sub = R.Cache(w.S, w.heads, w.B, w.d, dt, device)
-    for name in ("K", "V", "s", "q", "n", "pos", "live", "t_next"):
-        getattr(sub, name).copy_(getattr(cache, name)[:, :w.heads])
-    wl = W.scaled(W.LONG_CONTEXT, S=1, layers=1, prompt_lo=8192, prompt_hi=8192, B=8192)
-    _, long_cache, _ = build_cache(wl, device, R)
-    res["few_units"] = []
-    for label, cch, rr in ((f"{sub.U} units, B={sub.B}", sub, w.r), (f"{long_cache.U} units, B={long_cache.B}", long_cache, wl.r)):
-        algb = algorithmic_bytes_per_unit_step(cch.B, cch.d, elem) * cch.U
-        q1, k1, v1 = (torch.randn(cch.S, cch.G, cch.d, device=device, generator=gen).to(dt) for _ in range(3))
-        out1 = torch.zeros(cch.S, cch.G, cch.d, dtype=dt, device=device)
-        ev1 = torch.zeros(cch.S, cch.G, dtype=torch.int32, device=device)
-        rows = []
-        ms = timed_cold(lambda: R.roco_decode_step(cch, q1, k1, v1, rr, out1, ev1, scale=cch.d ** -0.5))
-        rows.append({"splits": 0, "us_per_step": ms * 1e3, "hbm_frac": algb / ms / 1e6 / hbm_peak})
-        for sp in (2, 4, 8):
-            ws = torch.empty(R.roco_decode_split_workspace_bytes(cch, sp), dtype=torch.uint8, device=device)
-            ms = timed_cold(lambda: R.roco_decode_step_split(cch, q1, k1, v1, rr, sp, out1, ev1, ws,
-                                                             scale=cch.d ** -0.5))
-            rows.append({"splits": sp, "us_per_step": ms * 1e3, "hbm_frac": algb / ms / 1e6 / hbm_peak})
-        res["few_units"].append({"case": label, "rows": rows})
-    del flush, long_cache
+    res["few_units"] = few_units_bench(R, cache, w, device, reps)
     # the paper's prefill scheme: the whole prompt through the budgeted cache, b tokens per evict-and-encode step
     # (its Table "block-wise eviction" reports the speed-up over b = 1)
     Lp = w.prompt_lo
@@ -389,6 +357,98 @@ def multi_bench(R, cache, w, device, reps=6):
         ms = timed(lambda: R.roco_gqa_decode_step(cache, Q, k, v, w.r, out, ev, scale=w.scale))
         res["gqa"].append({"group": g, "ms_per_step": ms, "hbm_frac": alg / ms / 1e6 / hbm_peak})
     return res
+
+
+def few_units_bench(R, cache, w, device, reps=6):
+    """Decode calls with few units (one layer at a time, what a transformer's decode loop issues): one layer of the
+    decode workload, and one layer of a single long sequence (32 units, B = 8192).  Paths: one CTA per unit, the
+    three-launch split, the one-launch persistent kernel, and a bare read of the same number of bytes.  Two timings
+    each: a single launch between two events with L2 flushed before it (includes the launch and event overhead of a
+    lone call), and a sweep over 8 distinct caches back to back (every call still reads cold rows)."""
+    hbm_peak, _, which = peaks()
+    elem = 2 if w.dtype == "bf16" else 4
+    dt = w.torch_dtype
+    gen = torch.Generator(device=device); gen.manual_seed(98)
+    # calls with few units (one layer at a time, what a transformer's decode loop does): the same step with each
+    # unit's slots divided among several CTAs.  Two cases: one layer of the decode workload, and one layer of a
+    # single long-context sequence (32 units, B = 8192).  L2 is flushed between launches (the caches are small).
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    def timed_cold(fn):
+        ts = []
+        for _ in range(reps + 2):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts[2:])
+    sub = R.Cache(w.S, w.heads, w.B, w.d, dt, device)
+    for name in ("K", "V", "s", "q", "n", "pos", "live", "t_next"):
+        getattr(sub, name).copy_(getattr(cache, name)[:, :w.heads])
+    wl = W.scaled(W.LONG_CONTEXT, S=1, layers=1, prompt_lo=8192, prompt_hi=8192, B=8192)
+    _, long_cache, _ = build_cache(wl, device, R)
+    out_rows = []
+    n_layers = 8   # distinct caches swept back to back: together far larger than L2, so every call reads cold rows
+
+    def clone_cache(src):
+        c = R.Cache(src.S, src.G, src.B, src.d, dt, device)
+        for name in ("K", "V", "s", "q", "n", "pos", "live", "t_next"):
+            getattr(c, name).copy_(getattr(src, name))
+        return c
+
+    def timed_sweep(fns):
+        """One call per cache of the sweep, back to back on the stream (what a decode loop over layers issues);
+        median over repetitions of the time per call."""
+        ts = []
+        for _ in range(reps + 2):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for fn in fns:
+                fn()
+            e1.record(); torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) / len(fns))
+        return statistics.median(ts[2:])
+
+    for label, cch, rr in ((f"{sub.U} units, B={sub.B}", sub, w.r), (f"{long_cache.U} units, B={long_cache.B}", long_cache, wl.r)):
+        algb = algorithmic_bytes_per_unit_step(cch.B, cch.d, elem) * cch.U
+        q1, k1, v1 = (torch.randn(cch.S, cch.G, cch.d, device=device, generator=gen).to(dt) for _ in range(3))
+        out1 = torch.zeros(cch.S, cch.G, cch.d, dtype=dt, device=device)
+        ev1 = torch.zeros(cch.S, cch.G, dtype=torch.int32, device=device)
+        layers = [clone_cache(cch) for _ in range(n_layers)]
+        sc = cch.d ** -0.5
+
+        def row(name, make):
+            """make(cache) -> callable of one step on that cache."""
+            iso = timed_cold(make(cch))
+            sweep = timed_sweep([make(c) for c in layers])
+            return {"path": name, "us_per_step": iso * 1e3, "hbm_frac": algb / iso / 1e6 / hbm_peak,
+                    "us_per_step_layer_sweep": sweep * 1e3, "hbm_frac_layer_sweep": algb / sweep / 1e6 / hbm_peak}
+
+        rows = [row("one CTA per unit", lambda c: (lambda: R.roco_decode_step(c, q1, k1, v1, rr, out1, ev1, scale=sc)))]
+        rows[-1]["splits"] = 0
+        for sp in (2, 4, 8):
+            ws = torch.empty(R.roco_decode_split_workspace_bytes(cch, sp), dtype=torch.uint8, device=device)
+            rows.append(row(f"three launches, {sp} splits",
+                            lambda c, sp=sp, ws=ws: (lambda: R.roco_decode_step_split(c, q1, k1, v1, rr, sp, out1, ev1, ws, scale=sc))))
+            rows[-1]["splits"] = sp
+        pws = torch.empty(R.roco_decode_persistent_workspace_bytes(cch), dtype=torch.uint8, device=device)
+        R.roco_decode_persistent_workspace_init(cch, pws)
+        for order, oname in ((0, "EVICT_FIRST"), (1, "ATTEND_FIRST")):
+            rows.append(row(f"one launch, persistent CTAs, {oname}",
+                            lambda c, order=order: (lambda: R.roco_decode_step_persistent(c, q1, k1, v1, rr, out1, ev1, pws,
+                                                                                          step_order=order, scale=sc))))
+        # what a bare read of the same number of bytes takes, launched the same two ways (own streaming kernel)
+        n_bytes = (algb // 16) * 16
+        bufs = [torch.empty(n_bytes, dtype=torch.uint8, device=device) for _ in range(n_layers)]
+        sink = torch.zeros(1, dtype=torch.int64, device=device)
+        buf_of = {id(c): b for c, b in zip(layers, bufs)}
+        buf_of[id(cch)] = bufs[0]
+        rows.append(row("bare read of the same bytes",
+                        lambda c: (lambda b=buf_of[id(c)]: R.roco_selftest_read_stream(b, sink))))
+        out_rows.append({"case": label, "algorithmic_bytes": algb, "layers_in_sweep": n_layers, "rows": rows})
+        del layers, bufs
+    del flush, long_cache
+    return out_rows
 
 
 def describe(w, world, scope_mode=0, step_order=0):
@@ -596,6 +656,7 @@ def main():
     ap.add_argument("--prefill-only", action="store_true", help="run only the prefill measurement")
     ap.add_argument("--no-prefill", action="store_true", help="skip the prefill measurement")
     ap.add_argument("--extras", action="store_true", help="also time the block-wise and grouped-query steps")
+    ap.add_argument("--no-few-units", action="store_true", help="skip the calls with few units (one layer at a time)")
     ap.add_argument("--prefill-workload", default="llama7b_prefill", help="workload of the prefill measurement")
     ap.add_argument("--scope-r", type=int, default=None, help="override the workload's scope parameter r")
     ap.add_argument("--scope-mode", default="exclude_top_r", choices=sorted(SCOPE_MODES),
@@ -647,6 +708,9 @@ def main():
     torch.cuda.empty_cache()
     if args.extras:
         line["multi_query"] = multi_bench(R, cache, w, device)
+        line["few_units"] = line["multi_query"].pop("few_units")
+    elif not args.no_few_units and not args.small and w.dtype == "bf16":
+        line["few_units"] = few_units_bench(R, cache, w, device)
         if R.roco_device_status(cache) != 0:
             raise RuntimeError("device status word set during the multi-query steps")
 

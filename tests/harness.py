@@ -136,8 +136,15 @@ class DecodeParity:
     """Steps the GPU cache and the oracle state of the sampled units together."""
 
     def __init__(self, cache: R.Cache, st: oracle.State, units: Sequence[int], r: int, scope_mode: int, order: int,
-                 tally: Tally, scale: Optional[float] = None, strict: bool = False, splits: int = 0):
+                 tally: Tally, scale: Optional[float] = None, strict: bool = False, splits: int = 0,
+                 persistent: bool = False):
         self.splits = splits
+        self.persistent = persistent
+        self.pws = None
+        if persistent:   # one launch of persistent CTAs; the workspace is initialised once
+            self.pws = torch.empty(R.roco_decode_persistent_workspace_bytes(cache), dtype=torch.uint8,
+                                   device=cache.K.device)
+            R.roco_decode_persistent_workspace_init(cache, self.pws)
         self.ws = (torch.empty(R.roco_decode_split_workspace_bytes(cache, splits), dtype=torch.uint8,
                                device=cache.K.device) if splits else None)
         self.cache, self.st, self.units = cache, st, list(units)
@@ -151,7 +158,10 @@ class DecodeParity:
 
     def step(self, q, k_new, v_new, check_state: bool = False):
         c = self.cache
-        if self.splits:
+        if self.persistent:
+            R.roco_decode_step_persistent(c, q, k_new, v_new, self.r, self.out, self.ev_slot, self.pws, self.ev_pos,
+                                          self.lse, scope_mode=self.mode, step_order=self.order, scale=self.scale)
+        elif self.splits:
             R.roco_decode_step_split(c, q, k_new, v_new, self.r, self.splits, self.out, self.ev_slot, self.ws,
                                      self.ev_pos, self.lse, scope_mode=self.mode, scale=self.scale)
         else:
