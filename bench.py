@@ -362,7 +362,7 @@ def multi_bench(R, cache, w, device, reps=6):
 def few_units_bench(R, cache, w, device, reps=6):
     """Decode calls with few units (one layer at a time, what a transformer's decode loop issues): one layer of the
     decode workload, and one layer of a single long sequence (32 units, B = 8192).  Paths: one CTA per unit, the
-    three-launch split, the one-launch persistent kernel, and a bare read of the same number of bytes.  Two timings
+    three-launch split, the one-launch cluster kernel, and a bare read of the same number of bytes.  Two timings
     each: a single launch between two events with L2 flushed before it (includes the launch and event overhead of a
     lone call), and a sweep over 8 distinct caches back to back (every call still reads cold rows)."""
     hbm_peak, _, which = peaks()
@@ -431,12 +431,13 @@ def few_units_bench(R, cache, w, device, reps=6):
             rows.append(row(f"three launches, {sp} splits",
                             lambda c, sp=sp, ws=ws: (lambda: R.roco_decode_step_split(c, q1, k1, v1, rr, sp, out1, ev1, ws, scale=sc))))
             rows[-1]["splits"] = sp
-        pws = torch.empty(R.roco_decode_persistent_workspace_bytes(cch), dtype=torch.uint8, device=device)
-        R.roco_decode_persistent_workspace_init(cch, pws)
+        kr = R.roco_decode_cluster_ranks(cch)
         for order, oname in ((0, "EVICT_FIRST"), (1, "ATTEND_FIRST")):
-            rows.append(row(f"one launch, persistent CTAs, {oname}",
-                            lambda c, order=order: (lambda: R.roco_decode_step_persistent(c, q1, k1, v1, rr, out1, ev1, pws,
-                                                                                          step_order=order, scale=sc))))
+            if kr > 1:
+                rows.append(row(f"one launch, cluster of {kr} CTAs per unit, {oname}",
+                                lambda c, order=order: (lambda: R.roco_decode_step_cluster(c, q1, k1, v1, rr, out1, ev1,
+                                                                                           step_order=order, ranks=kr, scale=sc))))
+                rows[-1]["ranks"] = kr
         # what a bare read of the same number of bytes takes, launched the same two ways (own streaming kernel)
         n_bytes = (algb // 16) * 16
         bufs = [torch.empty(n_bytes, dtype=torch.uint8, device=device) for _ in range(n_layers)]

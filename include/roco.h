@@ -321,32 +321,26 @@ roco_status roco_decode_step_split(roco_cache *cache, const void *q, const void 
                                    size_t workspace_bytes, void *stream);
 
 /*
- * roco_decode_step (either step order, both scope readings) for calls with few units in ONE launch: persistent
- * CTAs, one or two per SM, divide the cache rows of all units evenly among themselves, so a call of a few dozen
- * units keeps every SM streaming.  A CTA's share is a few pieces (unit, row range); each piece leaves its partial
- * (max, sum, sum of p*V) triple of Eq. 1 and its scores in the workspace and draws a ticket for its unit; the
- * contributor that draws a unit's last ticket merges the triples (log-sum-exp merge), adds the new token from
- * k_new / v_new, overwrites the freed slot in place (Fig. 1) and accumulates the statistics of Sec. 4.3 from the
- * saved scores.  No CTA waits for another.  Under ROCO_EVICT_FIRST the eviction scope and the victim (Sec. 4.3)
- * are found while the rows stream, and the victim's stale row is taken out of the merged sums afterwards (by
- * subtraction, or -- when that row holds more than a quarter of the softmax mass -- by an exact second pass);
- * under ROCO_ATTEND_FIRST the selection follows the statistics update.  Same arguments, results and parity
- * bounds as roco_decode_step; the output differs from it by fp32 rounding of the merge only.
+ * roco_decode_step (either step order, both scope readings) for calls with few units -- one layer of a small
+ * batch, a few long sequences -- with a thread-block cluster of `ranks` CTAs per unit: every rank streams the K/V
+ * rows of its own slot range exactly once and keeps that range's scores and statistics; the ranks agree on the
+ * softmax maximum and denominator of Eq. 1, on the eviction scope and on the victim (Sec. 4.3; a radix select and
+ * an argmin that run on all ranks in lockstep) by exchanging a few words through distributed shared memory, the
+ * partial outputs are added up on the first rank, the rank that owns the freed slot overwrites it in place
+ * (Fig. 1), and each rank updates the statistics of its own slots.  One launch, no workspace, no global-memory
+ * traffic besides what roco_decode_step has.  Same arguments, results and parity bounds as roco_decode_step.
  *
- *   workspace   >= roco_decode_persistent_workspace_bytes(cache) (0: shape not supported), 256-byte aligned,
- *               device.  It holds the ticket counters, which must be zero when a call starts: call
- *               roco_decode_persistent_workspace_init once after allocating it (it clears them on `stream`);
- *               every call that completes leaves them zero again.  After a call that reported a device status
- *               (a wait that ran out), initialise the workspace again.
- * Calls that share a workspace must not overlap on the GPU.
+ *   ranks   2, 4 or 8 CTAs per unit; 1: the one-CTA-per-unit kernel; 0: roco_decode_cluster_ranks(cache)
+ * Needs B a multiple of 4 and 16-byte aligned statistics arrays (else ROCO_ERR_UNSUPPORTED for ranks > 1).
+ * roco_decode_cluster_ranks: the cluster size that suits this cache's shape on the current device -- the
+ * largest whose CTAs fit the GPU in one wave of two per SM while every rank keeps at least two 16 KiB tiles;
+ * 1 when one CTA per unit already fills the GPU (host function; 0 on error).
  */
-size_t roco_decode_persistent_workspace_bytes(const roco_cache *cache);
-roco_status roco_decode_persistent_workspace_init(const roco_cache *cache, void *workspace, size_t workspace_bytes,
-                                                  void *stream);
-roco_status roco_decode_step_persistent(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,
-                                        int scope_mode, int step_order, float scale, void *attn_out, float *lse_out,
-                                        int32_t *evicted_slot, int32_t *evicted_pos, void *workspace,
-                                        size_t workspace_bytes, void *stream);
+int roco_decode_cluster_ranks(const roco_cache *cache);
+roco_status roco_decode_step_cluster(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,
+                                     int scope_mode, int step_order, int ranks, float scale, void *attn_out,
+                                     float *lse_out, int32_t *evicted_slot, int32_t *evicted_pos, void *stream);
+
 
 /*
  * Consistency of an importance score under a budget with its full-cache version (Sec. 4.3, preliminary

@@ -29,8 +29,8 @@ EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes",
            "roco_prefill_attend_workspace_bytes", "roco_prefill_attend", "roco_selftest_wait_timeout",
            "roco_consistency_step", "roco_selftest_read_stream", "roco_decode_host_pipeline_staging_bytes",
            "roco_decode_step_host_begin", "roco_decode_step_host_end", "roco_gqa_block_step",
-           "roco_prefill_blockwise_gqa", "roco_prefill_with_output", "roco_decode_persistent_workspace_bytes",
-           "roco_decode_persistent_workspace_init", "roco_decode_step_persistent")
+           "roco_prefill_blockwise_gqa", "roco_prefill_with_output", "roco_decode_cluster_ranks",
+           "roco_decode_step_cluster")
 
 
 class RocoError(RuntimeError):
@@ -109,14 +109,12 @@ def lib() -> C.CDLL:
         L.roco_decode_step_split.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                              C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
-        L.roco_decode_persistent_workspace_bytes.restype = C.c_size_t
-        L.roco_decode_persistent_workspace_bytes.argtypes = [C.POINTER(roco_cache)]
-        L.roco_decode_persistent_workspace_init.restype = C.c_int
-        L.roco_decode_persistent_workspace_init.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_size_t, C.c_void_p]
-        L.roco_decode_step_persistent.restype = C.c_int
-        L.roco_decode_step_persistent.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
-                                                  C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
-                                                  C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.roco_decode_cluster_ranks.restype = C.c_int
+        L.roco_decode_cluster_ranks.argtypes = [C.POINTER(roco_cache)]
+        L.roco_decode_step_cluster.restype = C.c_int
+        L.roco_decode_step_cluster.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                               C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p,
+                                               C.c_void_p, C.c_void_p, C.c_void_p]
         L.roco_decode_step_policy.restype = C.c_int
         L.roco_decode_step_policy.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                               C.c_int, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -310,28 +308,21 @@ def roco_decode_step_split(cache: Cache, q, k_new, v_new, r: int, splits: int, a
         raise RocoError(rc, "roco_decode_step_split")
 
 
-def roco_decode_persistent_workspace_bytes(cache: Cache) -> int:
-    return int(lib().roco_decode_persistent_workspace_bytes(C.byref(cache.c)))
+def roco_decode_cluster_ranks(cache: Cache) -> int:
+    """CTAs per unit that suit this cache's shape on the current device (1: one CTA per unit)."""
+    return int(lib().roco_decode_cluster_ranks(C.byref(cache.c)))
 
 
-def roco_decode_persistent_workspace_init(cache: Cache, workspace):
-    """Clears the ticket counters of a freshly allocated workspace (once; every completed call leaves them clear)."""
-    rc = lib().roco_decode_persistent_workspace_init(C.byref(cache.c), _ptr(workspace), workspace.numel(), _stream())
-    if rc != ROCO_OK:
-        raise RocoError(rc, "roco_decode_persistent_workspace_init")
-
-
-def roco_decode_step_persistent(cache: Cache, q, k_new, v_new, r: int, attn_out, evicted_slot, workspace,
-                                evicted_pos=None, lse_out=None, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R,
-                                step_order=ROCO_EVICT_FIRST, scale: Optional[float] = None):
-    """roco_decode_step in one launch of persistent CTAs that divide the cache rows of all units evenly (calls with
-    few units).  workspace: uint8 tensor of roco_decode_persistent_workspace_bytes(cache), initialised once."""
+def roco_decode_step_cluster(cache: Cache, q, k_new, v_new, r: int, attn_out, evicted_slot, evicted_pos=None,
+                             lse_out=None, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R, step_order=ROCO_EVICT_FIRST,
+                             ranks: int = 0, scale: Optional[float] = None):
+    """roco_decode_step with a cluster of `ranks` CTAs per unit (0: chosen from the shape; 1: one CTA per unit)."""
     scale = cache.d ** -0.5 if scale is None else scale
-    rc = lib().roco_decode_step_persistent(C.byref(cache.c), _ptr(q), _ptr(k_new), _ptr(v_new), r, scope_mode,
-                                           step_order, scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot),
-                                           _ptr(evicted_pos), _ptr(workspace), workspace.numel(), _stream())
+    rc = lib().roco_decode_step_cluster(C.byref(cache.c), _ptr(q), _ptr(k_new), _ptr(v_new), r, scope_mode,
+                                        step_order, ranks, scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot),
+                                        _ptr(evicted_pos), _stream())
     if rc != ROCO_OK:
-        raise RocoError(rc, "roco_decode_step_persistent")
+        raise RocoError(rc, "roco_decode_step_cluster")
 
 
 def roco_decode_step_policy(cache: Cache, q, k_new, v_new, policy: int, r: int, attn_out, evicted_slot,

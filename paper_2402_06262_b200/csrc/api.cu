@@ -263,40 +263,35 @@ roco_status roco_decode_step_split(roco_cache *cache, const void *q, const void 
                                   evicted_slot, evicted_pos, workspace, static_cast<cudaStream_t>(stream));
 }
 
-size_t roco_decode_persistent_workspace_bytes(const roco_cache *cache) {
+int roco_decode_cluster_ranks(const roco_cache *cache) {
   if (check_cache(cache) != ROCO_OK) return 0;
-  return decode_persist_workspace_bytes(cache->S * cache->G, cache->B, cache->d, cache->kv_dtype == ROCO_BF16 ? 2 : 4);
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return 0;
+  if (((reinterpret_cast<uintptr_t>(cache->s) | reinterpret_cast<uintptr_t>(cache->q) |
+        reinterpret_cast<uintptr_t>(cache->n) | reinterpret_cast<uintptr_t>(cache->pos)) & 15) != 0)
+    return 1;
+  return decode_cluster_ranks(cache->S * cache->G, cache->B, cache->d, cache->kv_dtype == ROCO_BF16 ? 2 : 4, sms);
 }
 
-roco_status roco_decode_persistent_workspace_init(const roco_cache *cache, void *workspace, size_t workspace_bytes,
-                                                  void *stream) {
-  const size_t need = roco_decode_persistent_workspace_bytes(cache);
-  if (need == 0) return ROCO_ERR_INVALID_ARG;
-  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
-    return ROCO_ERR_WORKSPACE;
-  return cudaMemsetAsync(workspace, 0, decode_persist_ticket_bytes(cache->S * cache->G),
-                         static_cast<cudaStream_t>(stream)) == cudaSuccess
-             ? ROCO_OK
-             : ROCO_ERR_CUDA;
-}
-
-roco_status roco_decode_step_persistent(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,
-                                        int scope_mode, int step_order, float scale, void *attn_out, float *lse_out,
-                                        int32_t *evicted_slot, int32_t *evicted_pos, void *workspace,
-                                        size_t workspace_bytes, void *stream) {
-  NvtxRange range("roco_decode_step_persistent");
+roco_status roco_decode_step_cluster(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,
+                                     int scope_mode, int step_order, int ranks, float scale, void *attn_out,
+                                     float *lse_out, int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {
+  NvtxRange range("roco_decode_step_cluster");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
   if (!q || !k_new || !v_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
   if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
   if (step_order != ROCO_EVICT_FIRST && step_order != ROCO_ATTEND_FIRST) return ROCO_ERR_INVALID_ARG;
-  const size_t need = roco_decode_persistent_workspace_bytes(cache);
-  if (need == 0) return ROCO_ERR_UNSUPPORTED;
-  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
-    return ROCO_ERR_WORKSPACE;
-  return launch_decode_step_persistent(*cache, q, k_new, v_new, r, scope_mode, step_order, scale, attn_out, lse_out,
-                                       evicted_slot, evicted_pos, workspace, static_cast<cudaStream_t>(stream));
+  if (ranks == 0) ranks = roco_decode_cluster_ranks(cache);
+  if (ranks == 1)
+    return launch_decode_step(*cache, q, k_new, v_new, r, scope_mode, step_order, ROCO_POLICY_ROCO, nullptr, scale,
+                              attn_out, lse_out, evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
+  if (ranks != 2 && ranks != 4 && ranks != 8) return ROCO_ERR_INVALID_ARG;
+  return launch_decode_step_cluster(*cache, ranks, q, k_new, v_new, r, scope_mode, step_order, scale, attn_out,
+                                    lse_out, evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
 }
 
 roco_status roco_decode_step_policy(roco_cache *cache, const void *q, const void *k_new, const void *v_new,

@@ -19,14 +19,13 @@ roco_status launch_decode_step_split(const roco_cache &c, const void *q, const v
                                      int scope_mode, int splits, float scale, void *out, float *lse, int32_t *ev_slot,
                                      int32_t *ev_pos, void *workspace, cudaStream_t stream);
 
-// The same step (either order) in one launch of persistent CTAs that divide the cache rows of all units evenly
-// among themselves; partial results, saved scores, tickets and victim slots live in `workspace`
-// (decode_persist_workspace_bytes; its first decode_persist_ticket_bytes bytes are zero between calls).
-size_t decode_persist_workspace_bytes(int U, int B, int d, int elem);
-size_t decode_persist_ticket_bytes(int U);
-roco_status launch_decode_step_persistent(const roco_cache &c, const void *q, const void *k_new, const void *v_new,
-                                          int r, int scope_mode, int step_order, float scale, void *out, float *lse,
-                                          int32_t *ev_slot, int32_t *ev_pos, void *workspace, cudaStream_t stream);
+// The same step (either order) with a thread-block cluster of `ranks` CTAs (2, 4 or 8) per unit that exchange
+// partial results through distributed shared memory; no workspace.  decode_cluster_ranks: the cluster size that
+// suits a call of U units (1 = one CTA per unit is the better shape).
+int decode_cluster_ranks(int U, int B, int d, int elem, int sms);
+roco_status launch_decode_step_cluster(const roco_cache &c, int ranks, const void *q, const void *k_new,
+                                       const void *v_new, int r, int scope_mode, int step_order, float scale,
+                                       void *out, float *lse, int32_t *ev_slot, int32_t *ev_pos, cudaStream_t stream);
 
 // Row log-sum-exp and column statistics of the causal softmax, CUDA-core path (any supported dtype/d).
 // lens_dev: [S] device copy of the prompt lengths.  lse, s_full, q_full: [U][Lmax].

@@ -137,14 +137,9 @@ class DecodeParity:
 
     def __init__(self, cache: R.Cache, st: oracle.State, units: Sequence[int], r: int, scope_mode: int, order: int,
                  tally: Tally, scale: Optional[float] = None, strict: bool = False, splits: int = 0,
-                 persistent: bool = False):
+                 ranks: int = 0):
         self.splits = splits
-        self.persistent = persistent
-        self.pws = None
-        if persistent:   # one launch of persistent CTAs; the workspace is initialised once
-            self.pws = torch.empty(R.roco_decode_persistent_workspace_bytes(cache), dtype=torch.uint8,
-                                   device=cache.K.device)
-            R.roco_decode_persistent_workspace_init(cache, self.pws)
+        self.ranks = ranks      # > 1: a cluster of that many CTAs per unit
         self.ws = (torch.empty(R.roco_decode_split_workspace_bytes(cache, splits), dtype=torch.uint8,
                                device=cache.K.device) if splits else None)
         self.cache, self.st, self.units = cache, st, list(units)
@@ -158,9 +153,9 @@ class DecodeParity:
 
     def step(self, q, k_new, v_new, check_state: bool = False):
         c = self.cache
-        if self.persistent:
-            R.roco_decode_step_persistent(c, q, k_new, v_new, self.r, self.out, self.ev_slot, self.pws, self.ev_pos,
-                                          self.lse, scope_mode=self.mode, step_order=self.order, scale=self.scale)
+        if self.ranks > 1:
+            R.roco_decode_step_cluster(c, q, k_new, v_new, self.r, self.out, self.ev_slot, self.ev_pos, self.lse,
+                                       scope_mode=self.mode, step_order=self.order, ranks=self.ranks, scale=self.scale)
         elif self.splits:
             R.roco_decode_step_split(c, q, k_new, v_new, self.r, self.splits, self.out, self.ev_slot, self.ws,
                                      self.ev_pos, self.lse, scope_mode=self.mode, scale=self.scale)
