@@ -201,134 +201,184 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     }
     group_and_or(k_and, k_or, *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy);  // publishes vkey / mkey too
     const int m = scope_size(live0, p.r, p.scope_mode);
-    uint32_t Tv = 0xffffffffu;
-    int Pv = 0x7fffffff;
-    uint32_t rank, ties;
-    if (m < live0) {
-      Tv = radix_select<uint32_t>([&](int j) { return v.vkey[j]; }, [&](int) { return true; }, live0,
-                                  (uint32_t)(m - 1), *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &rank, &ties,
-                                  k_and, k_or);
-      if (ties != rank + 1) {
-        uint32_t r2, t2;
-        Pv = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)opos[j]; },
-                                         [&](int j) { return v.vkey[j] == Tv; }, live0, rank, *v.sel, ptid,
-                                         kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
-      }
-    }
-    auto in_scope = [&](int j) {
-      const uint32_t k = v.vkey[j];
-      return k < Tv || (k == Tv && (Pv == 0x7fffffff || opos[j] <= Pv));
-    };
     int *list = v.ctl + 24;  // freed slots, in the order they were chosen
-    if (need == 1) {
-      // one victim: the in-scope token first in (mean, position) order
-      float bm = INFINITY;
-      int bs = -1;
-      for (int j = ptid; j < live0; j += kMqPolicyThreads) {
-        if (!in_scope(j)) continue;
-        const float mean = v.mkey[j];
-        if (mean < bm) { bm = mean; bs = j; }
-        else if (mean == bm && bs >= 0 && opos[j] < opos[bs]) bs = j;
-      }
-      int bp = bs >= 0 ? opos[bs] : 0x7fffffff;
+    int *cnt = v.ctl + 20;
+    uint32_t rank, ties;
+    // `rounds` times the token first in (mean, position) order over mkey; a chosen token is masked by the thread
+    // that scans it, which keeps the mean it had in keep[] (about 2 000 cycles a round)
+    float keep[4] = {0.f, 0.f, 0.f, 0.f};
+    auto argmin_rounds = [&](int rounds) {
+      bool ok = true;
+#pragma unroll 1
+      for (int e = 0; e < rounds; ++e) {
+        float bm = INFINITY;
+        int bs = -1;
+#pragma unroll 4
+        for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+          const float mean = v.mkey[j];
+          if (mean < bm) { bm = mean; bs = j; }
+          else if (mean == bm && bs >= 0 && opos[j] < opos[bs]) bs = j;
+        }
+        // a thread's candidates come in increasing slot order but ties go to the lower *position*
+        int bp = bs >= 0 ? opos[bs] : 0x7fffffff;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float om = __shfl_xor_sync(0xffffffffu, bm, o);
-        const int op = __shfl_xor_sync(0xffffffffu, bp, o);
-        const int os = __shfl_xor_sync(0xffffffffu, bs, o);
-        if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
-      }
-      if (plane == 0) { v.sel->red_mean[pwarp] = bm; v.sel->red_pos[pwarp] = bp; v.sel->red_slot[pwarp] = bs; }
-      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      if (ptid == 0) {
-        bm = v.sel->red_mean[0]; bp = v.sel->red_pos[0]; bs = v.sel->red_slot[0];
-        for (int w = 1; w < kMqPolicyThreads / 32; ++w) {
-          const float om = v.sel->red_mean[w];
-          const int op = v.sel->red_pos[w], os = v.sel->red_slot[w];
+        for (int o = 16; o > 0; o >>= 1) {
+          const float om = __shfl_xor_sync(0xffffffffu, bm, o);
+          const int op = __shfl_xor_sync(0xffffffffu, bp, o);
+          const int os = __shfl_xor_sync(0xffffffffu, bs, o);
           if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
         }
-        if (bs < 0) { atomicOr(p.status, ROCO_DEV_BAD_VICTIM); bs = 0; }
-        tgt[0] = bs;
+        float *rm = v.sel->red_mean + (e & 1) * 4;  // double-buffered: one barrier per round
+        int *rp = v.sel->red_pos + (e & 1) * 4, *rs = v.sel->red_slot + (e & 1) * 4;
+        if (plane == 0) { rm[pwarp] = bm; rp[pwarp] = bp; rs[pwarp] = bs; }
+        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+        bm = rm[0]; bp = rp[0]; bs = rs[0];
+#pragma unroll
+        for (int w = 1; w < kMqPolicyThreads / 32; ++w) {
+          const float om = rm[w];
+          const int op = rp[w], os = rs[w];
+          if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+        }
+        if (bs < 0) {
+          ok = false;
+          bs = e;  // keeps the slots distinct
+        }
+        if (ptid == 0) list[e] = bs;
+        if (ok && (bs % kMqPolicyThreads) == ptid) {  // only this thread ever scans slot bs
+          if (e < 4) keep[e] = v.mkey[bs];
+          v.mkey[bs] = INFINITY;
+        }
       }
-    } else {
+      return ok;
+    };
+    // the `need` smallest of mkey by radix select on the need-th, then one pass that collects everything up to it
+    auto collect_lowest = [&](uint32_t m_and, uint32_t m_or) {
+      const uint32_t Tm = radix_select<uint32_t>([&](int j) { return __float_as_uint(v.mkey[j]); },
+                                                 [&](int) { return true; }, live0, (uint32_t)(need - 1), *v.sel, ptid,
+                                                 kMqPolicyThreads, kMqBarPolicy, &rank, &ties, m_and, m_or);
+      int Pm = 0x7fffffff;
+      if (ties != rank + 1) {
+        uint32_t r2, t2;
+        Pm = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)opos[j]; },
+                                         [&](int j) { return __float_as_uint(v.mkey[j]) == Tm; }, live0, rank,
+                                         *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
+      }
+      if (ptid == 0) *cnt = 0;
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+        const uint32_t k = __float_as_uint(v.mkey[j]);
+        if (k < 0x7f800000u && (k < Tm || (k == Tm && (Pm == 0x7fffffff || opos[j] <= Pm)))) {
+          const int at = atomicAdd(cnt, 1);
+          if (at < kMqMaxQ) list[at] = j;
+        }
+      }
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      return *cnt == need;
+    };
+
+    // A scope that leaves out only a few tokens almost always contains the `need` tokens of lowest mean.  So
+    // those are picked first, over all cached tokens, and then tested: the one of them that comes last in
+    // (variance, position) order is in scope iff fewer than m tokens come before it, and then so are the others
+    // (they come before it too) -- one counting pass in place of the radix select for the scope threshold.
+    bool done = false;
+    if (2 * m >= live0) {
+      bool ok;
+      if (need <= 4) {
+        ok = argmin_rounds(need);
+      } else {
+        uint32_t m_and = 0xffffffffu, m_or = 0u;
+#pragma unroll 8
+        for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+          const uint32_t k = __float_as_uint(v.mkey[j]);
+          m_and &= k;
+          m_or |= k;
+        }
+        group_and_or(m_and, m_or, *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy);
+        ok = collect_lowest(m_and, m_or);
+      }
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);  // list[] is complete
+      // the candidate last in (variance, position) order
+      uint32_t cv = 0u;
+      int cp = -1;
+      if (ptid < need) {
+        const int c = list[ptid];
+        cv = v.vkey[c];
+        cp = opos[c];
+      }
+      if (pwarp == 0) {  // need <= 16: the first warp holds all candidates
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const uint32_t ov = __shfl_xor_sync(0xffffffffu, cv, o);
+          const int op = __shfl_xor_sync(0xffffffffu, cp, o);
+          if (ov > cv || (ov == cv && op > cp)) { cv = ov; cp = op; }
+        }
+        if (plane == 0) { v.sel->digit = cv; v.sel->rank = (uint32_t)cp; }
+      }
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      cv = v.sel->digit;
+      cp = (int)v.sel->rank;
+      uint32_t before = 0;
+#pragma unroll 8
+      for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+        const uint32_t k = v.vkey[j];
+        before += (k < cv || (k == cv && opos[j] < cp)) ? 1u : 0u;
+      }
+      before = __reduce_add_sync(0xffffffffu, before);
+      if (plane == 0) v.sel->hist[pwarp] = before;
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      before = 0;
+#pragma unroll
+      for (int w = 0; w < kMqPolicyThreads / 32; ++w) before += v.sel->hist[w];
+      done = ok && before < (uint32_t)m;
+      if (done) {
+        if (need == 1 && ptid == 0) tgt[0] = list[0];
+      } else if (need <= 4) {  // the general rule below needs the means as they were
+        for (int e = 0; e < need; ++e) {
+          const int c = list[e];
+          if (c >= 0 && c < live0 && (c % kMqPolicyThreads) == ptid && v.mkey[c] == INFINITY) v.mkey[c] = keep[e];
+        }
+      }
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+    }
+    if (!done) {
+      uint32_t Tv = 0xffffffffu;
+      int Pv = 0x7fffffff;
+      if (m < live0) {
+        Tv = radix_select<uint32_t>([&](int j) { return v.vkey[j]; }, [&](int) { return true; }, live0,
+                                    (uint32_t)(m - 1), *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &rank, &ties,
+                                    k_and, k_or);
+        if (ties != rank + 1) {
+          uint32_t r2, t2;
+          Pv = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)opos[j]; },
+                                           [&](int j) { return v.vkey[j] == Tv; }, live0, rank, *v.sel, ptid,
+                                           kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
+        }
+      }
+      auto in_scope = [&](int j) {
+        const uint32_t k = v.vkey[j];
+        return k < Tv || (k == Tv && (Pv == 0x7fffffff || opos[j] <= Pv));
+      };
       // the `need` (at most 16) in-scope tokens first in (mean, position) order; out-of-scope tokens are masked
       // once, which leaves a plain selection over mkey
       for (int j = ptid; j < live0; j += kMqPolicyThreads)
         if (!in_scope(j)) v.mkey[j] = INFINITY;
       named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      if (need <= 4) {
-        // few victims: one argmin after the other (about 2 000 cycles each, against ~20 000 for the threshold
-        // search below); a chosen token is masked by the thread that scans it
-        for (int e = 0; e < need; ++e) {
-          float bm = INFINITY;
-          int bs = -1;
-#pragma unroll 4
-          for (int j = ptid; j < live0; j += kMqPolicyThreads) {
-            const float mean = v.mkey[j];
-            if (mean < bm) { bm = mean; bs = j; }
-            else if (mean == bm && bs >= 0 && opos[j] < opos[bs]) bs = j;
-          }
-          // a thread's candidates come in increasing slot order but ties go to the lower *position*
-          int bp = bs >= 0 ? opos[bs] : 0x7fffffff;
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            const float om = __shfl_xor_sync(0xffffffffu, bm, o);
-            const int op = __shfl_xor_sync(0xffffffffu, bp, o);
-            const int os = __shfl_xor_sync(0xffffffffu, bs, o);
-            if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
-          }
-          float *rm = v.sel->red_mean + (e & 1) * 4;  // double-buffered: one barrier per round
-          int *rp = v.sel->red_pos + (e & 1) * 4, *rs = v.sel->red_slot + (e & 1) * 4;
-          if (plane == 0) { rm[pwarp] = bm; rp[pwarp] = bp; rs[pwarp] = bs; }
-          named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-          bm = rm[0]; bp = rp[0]; bs = rs[0];
-#pragma unroll
-          for (int w = 1; w < kMqPolicyThreads / 32; ++w) {
-            const float om = rm[w];
-            const int op = rp[w], os = rs[w];
-            if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
-          }
-          if (bs < 0) {
-            if (ptid == 0) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
-            bs = e;  // keeps the slots distinct; the step's results are void
-          }
-          if (ptid == 0) list[e] = bs;
-          if ((bs % kMqPolicyThreads) == ptid) v.mkey[bs] = INFINITY;  // only this thread ever scans slot bs
-        }
-      } else {
-        // many victims: the need-th smallest mean by radix select, then one pass that collects everything up to it
-        const uint32_t Tm = radix_select<uint32_t>([&](int j) { return __float_as_uint(v.mkey[j]); },
-                                                   [&](int) { return true; }, live0, (uint32_t)(need - 1), *v.sel, ptid,
-                                                   kMqPolicyThreads, kMqBarPolicy, &rank, &ties);
-        int Pm = 0x7fffffff;
-        if (ties != rank + 1) {
-          uint32_t r2, t2;
-          Pm = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)opos[j]; },
-                                           [&](int j) { return __float_as_uint(v.mkey[j]) == Tm; }, live0, rank,
-                                           *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
-        }
-        int *cnt = v.ctl + 20;
-        if (ptid == 0) *cnt = 0;
-        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-        for (int j = ptid; j < live0; j += kMqPolicyThreads) {
-          const uint32_t k = __float_as_uint(v.mkey[j]);
-          if (k < 0x7f800000u && (k < Tm || (k == Tm && (Pm == 0x7fffffff || opos[j] <= Pm)))) {
-            const int at = atomicAdd(cnt, 1);
-            if (at < kMqMaxQ) list[at] = j;
-          }
-        }
-        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-        if (ptid == 0 && *cnt != need) {  // only after corrupt statistics
-          atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
-          for (int x = *cnt < 0 ? 0 : *cnt; x < need; ++x) list[x] = x;
-        }
-      }
+      bool ok;
+      if (need <= 4) ok = argmin_rounds(need);  // few victims: one argmin after the other
+      else ok = collect_lowest(0u, 0xffffffffu);
       named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      if (ptid < need) {  // order the freed slots by slot index
-        int rk = 0;
-        for (int x = 0; x < need; ++x) rk += list[x] < list[ptid];
-        if (rk < nb) tgt[rk] = list[ptid];
+      if (!ok && ptid == 0) {  // only after corrupt statistics; the step's results are void
+        atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
+        if (need > 4)
+          for (int x = *cnt < 0 ? 0 : (*cnt > need ? need : *cnt); x < need; ++x) list[x] = x;
       }
+      if (need == 1 && ptid == 0) tgt[0] = list[0];
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+    }
+    if (need > 1 && ptid < need) {  // order the freed slots by slot index
+      int rk = 0;
+      for (int x = 0; x < need; ++x) rk += list[x] < list[ptid];
+      if (rk < nb) tgt[rk] = list[ptid];
     }
   }
   if (ptid < nb - need) tgt[need + ptid] = live0 + ptid;  // free slots behind the occupied ones
