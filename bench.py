@@ -710,7 +710,7 @@ def main():
     if args.extras:
         line["multi_query"] = multi_bench(R, cache, w, device)
         line["few_units"] = line["multi_query"].pop("few_units")
-    elif not args.no_few_units and not args.small and w.dtype == "bf16":
+    elif not args.no_few_units and w.dtype == "bf16":
         line["few_units"] = few_units_bench(R, cache, w, device)
         if R.roco_device_status(cache) != 0:
             raise RuntimeError("device status word set during the multi-query steps")
