@@ -48,24 +48,24 @@ struct DecodeSmem {
   uint32_t *vkey;      // policy warps: variance keys
   float *mkey;         // policy warps: mean keys
   SelectScratch *sel;  // policy warps: histogram and reduction scratch
-  float *qf, *vnew, *outred, *red;
+  float *qf, *vnew, *knew, *outred, *red;
   uint64_t *full, *empty;  // ring barriers
   uint64_t *p_ready;       // consumers have left the probabilities in shared memory
   uint64_t *policy_done;   // victim chosen, new K/V written
   uint64_t *stats_full;    // the unit's s, q, n have landed in vkey, mkey, nbuf (bulk copies ahead of the K tiles)
   uint64_t *v_done;        // consumers have read their last V tile (ATTEND_FIRST: the freed V row may be overwritten)
-  int *nbuf;
+  int *nbuf;               // staged Count array
+  int *posb;               // staged positions
   int *ctl;                // [0] abort flag, [1] slot of the new token
-  float *znew;             // score of the new token (EVICT_FIRST)
 };
 
 template <int TILE>
 __host__ __device__ inline size_t decode_smem_bytes(int B, int d, int stages, int stage_stats) {
   const size_t Bp = align_up((size_t)B, 4);
   size_t b = (size_t)stages * TILE;
-  b += (stage_stats ? 4 : 3) * Bp * 4;  // z, vkey, mkey (, nbuf)
+  b += (stage_stats ? 5 : 3) * Bp * 4;  // z, vkey, mkey (, nbuf, posb)
   b += sizeof(SelectScratch);
-  b += (size_t)(2 + kConsumerWarps) * d * 4;  // qf, vnew, outred
+  b += (size_t)3 * d * 4;  // qf, vnew, knew (outred reuses the ring once the V pass is over)
   b += 64 * 4;                                // red
   b += (2 * (size_t)stages + 4) * sizeof(uint64_t);
   b += 8 * 4;
@@ -82,10 +82,12 @@ __device__ inline DecodeSmem carve(char *raw, int B, int d, int stages, int stag
   m.vkey = (uint32_t *)p; p += Bp * 4;
   m.mkey = (float *)p; p += Bp * 4;
   m.nbuf = (int *)p; p += stage_stats ? Bp * 4 : 0;
+  m.posb = (int *)p; p += stage_stats ? Bp * 4 : 0;
   m.sel = (SelectScratch *)p; p += sizeof(SelectScratch);
   m.qf = (float *)p; p += d * 4;
   m.vnew = (float *)p; p += d * 4;
-  m.outred = (float *)p; p += (size_t)kConsumerWarps * d * 4;
+  m.knew = (float *)p; p += d * 4;
+  m.outred = (float *)m.ring;  // kConsumerWarps * d floats, written after every warp's last V tile
   m.red = (float *)p; p += 64 * 4;
   m.full = (uint64_t *)p; p += stages * sizeof(uint64_t);
   m.empty = (uint64_t *)p; p += stages * sizeof(uint64_t);
@@ -93,8 +95,7 @@ __device__ inline DecodeSmem carve(char *raw, int B, int d, int stages, int stag
   m.policy_done = (uint64_t *)p; p += sizeof(uint64_t);
   m.stats_full = (uint64_t *)p; p += sizeof(uint64_t);
   m.v_done = (uint64_t *)p; p += sizeof(uint64_t);
-  m.ctl = (int *)p; p += 4 * 4;
-  m.znew = (float *)p;
+  m.ctl = (int *)p;
   return m;
 }
 
@@ -164,7 +165,8 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
   // at the start of the step, and the unit's arrays start on 16-byte boundaries.
   const bool stats_staged =
       p.stage_stats && full && evict_first && p.policy == ROCO_POLICY_ROCO && (B & 3) == 0 &&
-      ((reinterpret_cast<uintptr_t>(p.s) | reinterpret_cast<uintptr_t>(p.q) | reinterpret_cast<uintptr_t>(p.n)) & 15) == 0;
+      ((reinterpret_cast<uintptr_t>(p.s) | reinterpret_cast<uintptr_t>(p.q) | reinterpret_cast<uintptr_t>(p.n) |
+        reinterpret_cast<uintptr_t>(p.pos)) & 15) == 0;
   __syncthreads();
 
   if (warp == kProducerWarp) {
@@ -172,10 +174,11 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     if (lane == 0) {
       if (stats_staged) {
         const uint32_t bytes = (uint32_t)B * 4;
-        mbar_expect_tx(sm.stats_full, 3 * bytes);
+        mbar_expect_tx(sm.stats_full, 4 * bytes);
         bulk_g2s(sm.vkey, p.s + unit_st, bytes, sm.stats_full);
         bulk_g2s(sm.mkey, p.q + unit_st, bytes, sm.stats_full);
         bulk_g2s(sm.nbuf, p.n + unit_st, bytes, sm.stats_full);
+        bulk_g2s(sm.posb, p.pos + unit_st, bytes, sm.stats_full);
       }
       for (int g = 0; g < 2 * n_tiles; ++g) {
         const int st = g % stages;
@@ -198,21 +201,15 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     const int t_new = p.t_next[u];  // read by these warps only: they also write the incremented value
     // What the tail of this branch needs from global memory and does not depend on the victim is requested now,
     // so that its latency passes during the selection: the 16 bytes of k_new / v_new this thread will write into
-    // the freed slot, and (last warp) the operands of the new token's own score.
+    // the freed slot (raw bytes: nothing waits for them before the store; a load whose value is converted at once
+    // would hold its warp, and with it the group's next barrier, until the reply has made its way through the
+    // queue of streamed tiles).
     const bool writes_row = ptid >= 32 && ptid < 32 + 2 * kLanesPerRow;
     uint4 row_val = make_uint4(0u, 0u, 0u, 0u);
     if (writes_row) {
       const int c = ptid - 32;
       const bool isv = c >= kLanesPerRow;
       row_val = *((const uint4 *)((isv ? p.v_new : p.k_new) + (size_t)u * kRowBytes) + (isv ? c - kLanesPerRow : c));
-    }
-    float own_q[D / 32], own_k[D / 32];
-    if (evict_first && ptid >= 96) {
-#pragma unroll
-      for (int i = 0; i < D / 32; ++i) {
-        own_q[i] = Elem<T>::load((const T *)p.qv + (size_t)u * D + lane + 32 * i);
-        own_k[i] = Elem<T>::load((const T *)p.k_new + (size_t)u * D + lane + 32 * i);
-      }
     }
     named_bar_sync(kBarPolicy, kPolicyThreads);
     // statistics of Sec. 4.3 for the slots the query attended over: Acc += p, Acc^square += p^2, Count += 1
@@ -271,7 +268,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
             k_and &= vk;
             k_or |= vk;
           }
-          e = group_select_from_keys(gpos, B, m, sm.vkey, sm.mkey, k_and, k_or, *sm.sel, ptid, kPolicyThreads,
+          e = group_select_from_keys(sm.posb, B, m, sm.vkey, sm.mkey, k_and, k_or, *sm.sel, ptid, kPolicyThreads,
                                      kBarPolicy);
         } else {
           e = group_select_victim(gs, gq, gn, gpos, B, m, sm.vkey, sm.mkey, *sm.sel, ptid, kPolicyThreads,
@@ -302,7 +299,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
         e = 0;
       }
       ev_slot = e;
-      if (ptid == 0) ev_pos = p.pos[unit_st + e];
+      if (ptid == 0) ev_pos = stats_staged ? sm.posb[e] : p.pos[unit_st + e];
     }
     // the new token takes the slot with empty statistics
     if (ptid == 0) {
@@ -324,13 +321,6 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
       char *dst = const_cast<char *>(isv ? p.V : p.K) + unit_kv + (size_t)e * kRowBytes;
       *((uint4 *)dst + (isv ? c - kLanesPerRow : c)) = row_val;
     }
-    if (evict_first && ptid >= 96) {  // the new token's own score, from k_new directly
-      float acc = 0.f;
-#pragma unroll
-      for (int i = 0; i < D / 32; ++i) acc = fmaf(own_q[i], own_k[i], acc);
-      acc = warp_sum(acc);
-      if (lane == 0) *sm.znew = acc * (p.scale * kLog2e);
-    }
     named_bar_sync(kBarPolicy, kPolicyThreads);
     if (ptid == 0) {
       mbar_arrive(sm.policy_done);
@@ -344,7 +334,10 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
   if (tid < D) {
     const size_t o = (size_t)u * D + tid;
     sm.qf[tid] = Elem<T>::load((const T *)p.qv + o);
-    if (evict_first) sm.vnew[tid] = Elem<T>::load((const T *)p.v_new + o);
+    if (evict_first) {
+      sm.vnew[tid] = Elem<T>::load((const T *)p.v_new + o);
+      sm.knew[tid] = Elem<T>::load((const T *)p.k_new + o);
+    }
   }
   named_bar_sync(kBarConsumers, kConsumers);
 
@@ -395,7 +388,13 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     if (e_sub < 0 || e_sub >= B) e_sub = 0;  // only after an aborted wait
   }
   named_bar_sync(kBarConsumers, kConsumers);  // all scores are in shared memory
-  if (tid == 0 && e_sub >= 0) sm.z[e_sub] = *sm.znew;
+  if (warp == 0 && e_sub >= 0) {  // the new token's own score, from k_new directly
+    float a = 0.f;
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) a = fmaf(sm.qf[lane + 32 * i], sm.knew[lane + 32 * i], a);
+    a = warp_sum(a);
+    if (lane == 0) sm.z[e_sub] = a * zscale;
+  }
   named_bar_sync(kBarConsumers, kConsumers);
 
   // ---- softmax over the occupied slots
@@ -446,6 +445,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     if (lane == 0) mbar_arrive(&sm.empty[st]);
   }
   if (lane == 0) mbar_arrive(sm.v_done);  // this warp has read its share of every V tile
+  named_bar_sync(kBarConsumers, kConsumers);  // ... and so have the others: the ring is free for the partial sums
 #pragma unroll
   for (int i = 0; i < kEPC; ++i) {
 #pragma unroll

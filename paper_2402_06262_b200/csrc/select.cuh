@@ -134,6 +134,64 @@ __device__ __forceinline__ void group_and_or(uint32_t &k_and, uint32_t &k_or, Se
 __device__ __forceinline__ int group_select_from_keys(const int *pos, int live, int m, const uint32_t *vkey,
                                                       const float *mkey, uint32_t k_and, uint32_t k_or,
                                                       SelectScratch &sc, int tid, int nthreads, int bar_id) {
+  const int warp = tid >> 5, nwarps = nthreads >> 5;
+  // (mean, position, slot) of the group's best candidate from each thread's own; every thread gets it
+  auto reduce_best = [&](float &bm, int &bp, int &bs) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float om = __shfl_xor_sync(0xffffffffu, bm, o);
+      const int op = __shfl_xor_sync(0xffffffffu, bp, o);
+      const int os = __shfl_xor_sync(0xffffffffu, bs, o);
+      if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+    }
+    if ((tid & 31) == 0) { sc.red_mean[warp] = bm; sc.red_pos[warp] = bp; sc.red_slot[warp] = bs; }
+    named_bar_sync(bar_id, nthreads);
+    bm = sc.red_mean[0]; bp = sc.red_pos[0]; bs = sc.red_slot[0];
+    for (int w = 1; w < nwarps; ++w) {
+      const float om = sc.red_mean[w];
+      const int op = sc.red_pos[w], os = sc.red_slot[w];
+      if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+    }
+    named_bar_sync(bar_id, nthreads);  // the scratch may be reused right away
+  };
+  named_bar_sync(bar_id, nthreads);  // publishes the keys
+  // A scope that leaves out only a few tokens almost always contains the token of lowest mean.  So: take the
+  // tokens in (mean, position) order and test each for membership -- it is in scope iff fewer than m tokens come
+  // before it in (variance, position) order -- which costs two passes over the keys per candidate where the radix
+  // select below costs two per digit.  After three candidates outside the scope the radix select takes over.
+  if (2 * m >= live) {
+    int excl0 = -1, excl1 = -1, excl2 = -1;
+#pragma unroll 1
+    for (int attempt = 0; attempt < 3; ++attempt) {
+      float bm = INFINITY;
+      int bs = -1;
+#pragma unroll 4
+      for (int j = tid; j < live; j += nthreads) {
+        if (j == excl0 || j == excl1 || j == excl2) continue;
+        const float mean = mkey[j];
+        if (mean < bm) { bm = mean; bs = j; }
+        else if (mean == bm && bs >= 0 && pos[j] < pos[bs]) bs = j;
+      }
+      int bp = (bs >= 0) ? pos[bs] : 0x7fffffff;
+      reduce_best(bm, bp, bs);
+      if (bs < 0) return -1;  // no candidate left (NaN statistics)
+      const uint32_t cv = vkey[bs];
+      uint32_t cnt = 0;
+#pragma unroll 4
+      for (int j = tid; j < live; j += nthreads) {
+        const uint32_t k = vkey[j];
+        cnt += (k < cv || (k == cv && pos[j] < bp)) ? 1u : 0u;
+      }
+      cnt = __reduce_add_sync(0xffffffffu, cnt);
+      if ((tid & 31) == 0) sc.red_slot[warp] = (int)cnt;
+      named_bar_sync(bar_id, nthreads);
+      cnt = 0;
+      for (int w = 0; w < nwarps; ++w) cnt += (uint32_t)sc.red_slot[w];
+      named_bar_sync(bar_id, nthreads);
+      if (cnt < (uint32_t)m) return bs;
+      if (attempt == 0) excl0 = bs; else if (attempt == 1) excl1 = bs; else excl2 = bs;
+    }
+  }
   group_and_or(k_and, k_or, sc, tid, nthreads, bar_id);
   uint32_t T = 0xffffffffu;
   int P = 0x7fffffff;
@@ -159,23 +217,7 @@ __device__ __forceinline__ int group_select_from_keys(const int *pos, int live, 
     else if (mean == bm && bs >= 0 && pos[j] < pos[bs]) bs = j;
   }
   int bp = (bs >= 0) ? pos[bs] : 0x7fffffff;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float om = __shfl_xor_sync(0xffffffffu, bm, o);
-    const int op = __shfl_xor_sync(0xffffffffu, bp, o);
-    const int os = __shfl_xor_sync(0xffffffffu, bs, o);
-    if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
-  }
-  const int warp = tid >> 5, nwarps = nthreads >> 5;
-  if ((tid & 31) == 0) { sc.red_mean[warp] = bm; sc.red_pos[warp] = bp; sc.red_slot[warp] = bs; }
-  named_bar_sync(bar_id, nthreads);
-  bm = sc.red_mean[0]; bp = sc.red_pos[0]; bs = sc.red_slot[0];
-  for (int w = 1; w < nwarps; ++w) {
-    const float om = sc.red_mean[w];
-    const int op = sc.red_pos[w], os = sc.red_slot[w];
-    if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
-  }
-  named_bar_sync(bar_id, nthreads);
+  reduce_best(bm, bp, bs);
   return bs;
 }
 
