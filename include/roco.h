@@ -131,7 +131,9 @@ roco_status roco_prefill(const void *Q, const void *K, const void *V, const int3
  * The output comes from the same sweep over the score tiles that yields the row log-sum-exp (running row maximum,
  * output accumulator rescaled when the maximum moves), so the whole call costs three L x L contractions (scores
  * and P.V in the sweep, scores again for the column statistics) instead of the four of roco_prefill followed by
- * roco_prefill_attend.  Tensor cores only: kv_dtype ROCO_BF16 and d = 128, else ROCO_ERR_UNSUPPORTED; scale > 0.
+ * roco_prefill_attend.  That is the tensor-core path (kv_dtype ROCO_BF16, d = 128; it needs scale > 0); for the other
+ * dtypes and head dimensions the output comes from a CUDA-core pass over the row log-sum-exp, after the two
+ * statistics passes.
  *   attn_out     [S][G][Lmax][d] device, 16-byte aligned; rows >= lens are left untouched; NULL: roco_prefill
  * All other arguments, results and errors as roco_prefill.
  */
@@ -256,8 +258,8 @@ roco_status roco_prefill_blockwise(const void *Q, const void *K, const void *V, 
  * also need the layer's output and not only the budgeted cache:
  *     out_i = sum_{j<=i} exp(scale * Q_i.K_j - lse_i) V_j,      i < lens
  * where lse is the row log-sum-exp roco_prefill returned in lse_out for the same Q, K, lens, Lmax and scale
- * (call roco_prefill first, on the same stream).  Tensor cores only: kv_dtype ROCO_BF16 and d = 128, else
- * ROCO_ERR_UNSUPPORTED.  Only S, G, d, kv_dtype and status of `cache` are read.
+ * (call roco_prefill first, on the same stream).  On the tensor cores for kv_dtype ROCO_BF16 and d = 128, on the
+ * CUDA cores otherwise.  Only S, G, d, kv_dtype and status of `cache` are read.
  *
  *   Q, K, V      [S][G][Lmax][d] device; rows >= lens may hold anything
  *   lens_host    [S] HOST array, 1 <= lens <= Lmax

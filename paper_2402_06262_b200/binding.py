@@ -194,8 +194,8 @@ def roco_prefill_uses_tensor_cores(cache: Cache) -> bool:
 def roco_prefill(Q, K, V, lens: Sequence[int], B: int, r: int, cache: Cache, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R,
                  count_self=1, scale: Optional[float] = None, lse_out=None, s_full=None, q_full=None,
                  workspace: Optional[torch.Tensor] = None, attn_out=None):
-    """Q, K, V: [S][G][Lmax][d] device tensors.  Fills `cache`.  attn_out ([S][G][Lmax][d], bf16, d = 128): also
-    the prompt's causal attention output (roco_prefill_with_output)."""
+    """Q, K, V: [S][G][Lmax][d] device tensors.  Fills `cache`.  attn_out ([S][G][Lmax][d]): also the prompt's
+    causal attention output (roco_prefill_with_output)."""
     Lmax = Q.shape[2]
     scale = cache.d ** -0.5 if scale is None else scale
     if workspace is None:

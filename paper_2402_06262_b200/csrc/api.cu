@@ -154,9 +154,9 @@ roco_status roco_prefill_with_output(const void *Q, const void *K, const void *V
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V)) return ROCO_ERR_INVALID_ARG;
   if ((st = check_scope(r, scope_mode, B, false)) != ROCO_OK) return st;
   if (count_self != 1) return ROCO_ERR_UNSUPPORTED;
-  if (attn_out) {  // the prompt's attention output from the same sweep that yields the row log-sum-exp
-    if (!prefill_tc_supported(cache->kv_dtype, cache->d)) return ROCO_ERR_UNSUPPORTED;
-    if (!aligned16(attn_out) || !(scale > 0.f)) return ROCO_ERR_INVALID_ARG;
+  const bool tc = prefill_tc_supported(cache->kv_dtype, cache->d);
+  if (attn_out) {  // tensor cores: from the same sweep that yields the row log-sum-exp (needs a positive scale)
+    if (!aligned16(attn_out) || (tc && !(scale > 0.f))) return ROCO_ERR_INVALID_ARG;
   }
   int maxlen = 0;
   for (int b = 0; b < cache->S; ++b) {
@@ -179,18 +179,22 @@ roco_status roco_prefill_with_output(const void *Q, const void *K, const void *V
   int *dst = reinterpret_cast<int *>(ws + w.dst_off);
   if (cudaMemcpyAsync(lens_dev, lens_host, (size_t)cache->S * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess)
     return ROCO_ERR_CUDA;
-  if (attn_out) {
+  if (attn_out && tc) {
     st = launch_prefill_attend_tc(cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, V, scale, nullptr, lse, attn_out,
                                   cache->status, cs);
     if (st == ROCO_OK)
       st = launch_prefill_stats_tc(cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, scale, lse, sf, qf,
                                    cache->status, cs, true);
-  } else if (prefill_tc_supported(cache->kv_dtype, cache->d))
+  } else if (tc) {
     st = launch_prefill_stats_tc(cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, scale, lse, sf, qf, cache->status,
                                  cs);
-  else
+  } else {  // CUDA cores: log-sum-exp pass, statistics pass, and -- if asked for -- the output from that log-sum-exp
     st = launch_prefill_stats_simt(cache->kv_dtype, cache->d, cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, scale,
                                    lse, sf, qf, cs);
+    if (st == ROCO_OK && attn_out)
+      st = launch_prefill_attend_simt(cache->kv_dtype, cache->d, cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, V,
+                                      scale, lse, attn_out, cs);
+  }
   if (st != ROCO_OK) return st;
   return launch_budget_select_gather(*cache, Lmax, lens_dev, maxlen, r, scope_mode, K, V, sf, qf, dst,
                                      reinterpret_cast<unsigned long long *>(ws + w.total), pow2_at_least(Lmax), cs);
@@ -208,13 +212,14 @@ roco_status roco_prefill_attend(const roco_cache *cache, const void *Q, const vo
   if (!cache || !cache->status || cache->S < 1 || cache->G < 1) return ROCO_ERR_INVALID_ARG;
   if (!Q || !K || !V || !lens_host || !lse || !attn_out || Lmax < 1) return ROCO_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
-  if (!prefill_tc_supported(cache->kv_dtype, cache->d)) return ROCO_ERR_UNSUPPORTED;
+  if ((cache->kv_dtype != ROCO_F32 && cache->kv_dtype != ROCO_BF16) || (cache->d != 64 && cache->d != 128))
+    return ROCO_ERR_UNSUPPORTED;
   int maxlen = 0;
   for (int b = 0; b < cache->S; ++b) {
     if (lens_host[b] < 1 || lens_host[b] > Lmax) return ROCO_ERR_INVALID_ARG;
     if (lens_host[b] > maxlen) maxlen = lens_host[b];
   }
-  if ((long long)cache->S * cache->G * ((maxlen + 255) / 256 + 1) > 0x7fffffffLL) return ROCO_ERR_UNSUPPORTED;
+  if ((long long)cache->S * cache->G * ((maxlen + 63) / 64 + 1) > 0x7fffffffLL) return ROCO_ERR_UNSUPPORTED;
   if (!workspace || workspace_bytes < roco_prefill_attend_workspace_bytes(cache) ||
       (reinterpret_cast<uintptr_t>(workspace) & 255u))
     return ROCO_ERR_WORKSPACE;
@@ -222,6 +227,9 @@ roco_status roco_prefill_attend(const roco_cache *cache, const void *Q, const vo
   int *lens_dev = static_cast<int *>(workspace);
   if (cudaMemcpyAsync(lens_dev, lens_host, (size_t)cache->S * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess)
     return ROCO_ERR_CUDA;
+  if (!prefill_tc_supported(cache->kv_dtype, cache->d))
+    return launch_prefill_attend_simt(cache->kv_dtype, cache->d, cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, V,
+                                      scale, lse, attn_out, cs);
   return launch_prefill_attend_tc(cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, V, scale, lse, nullptr, attn_out,
                                   cache->status, cs);
 }

@@ -33,6 +33,12 @@ roco_status launch_prefill_stats_simt(int kv_dtype, int d, int S, int G, int Lma
                                       const void *Q, const void *K, float scale, float *lse, float *s_full,
                                       float *q_full, cudaStream_t stream);
 
+// Causal attention output of the prompt pass on CUDA cores from the row log-sum-exp (any supported dtype/d):
+// out_i = sum_{j<=i} exp(scale Q_i.K_j - lse_i) V_j.  out: [U][Lmax][d], rows >= lens untouched.
+roco_status launch_prefill_attend_simt(int kv_dtype, int d, int S, int G, int Lmax, const int *lens_dev, int maxlen,
+                                       const void *Q, const void *K, const void *V, float scale, const float *lse,
+                                       void *out, cudaStream_t stream);
+
 // The same two passes on tcgen05 tensor cores with TMA-fed operands (bf16, d = 128 only).  lse_ready: `lse`
 // already holds the row log-sum-exp (from the one-sweep attention kernel), so only the statistics pass runs.
 bool prefill_tc_supported(int kv_dtype, int d);

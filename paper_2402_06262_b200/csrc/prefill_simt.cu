@@ -152,6 +152,101 @@ __global__ void __launch_bounds__(kPThreads) prefill_colstats_kernel(const T *Q,
   }
 }
 
+// grid U * tiles, unit-major; heavy (late) row tiles first.  out[u][i] = sum_{j<=i} exp(scale * Q_i.K_j - lse_i) V_j
+// (Eq. 1 with the causal mask of Sec. 2.1) from the row log-sum-exp of prefill_lse_kernel: per key tile the 64 x 64
+// block of probabilities goes through shared memory, and each thread keeps 4 rows x D/16 columns of the output.
+template <typename T, int D>
+__global__ void __launch_bounds__(kPThreads) prefill_attend_simt_kernel(const T *Q, const T *K, const T *V,
+                                                                        const int *lens, int G, int Lmax, int tiles,
+                                                                        float scale, const float *lse, T *out) {
+  extern __shared__ float psm[];
+  float *Qs = psm, *Ks = psm + kPT * (D + 1), *Ps = Ks + kPT * (D + 1), *lse2 = Ps + kPT * (kPT + 1);
+  const int u = blockIdx.x / tiles, L = lens[u / G];
+  const int row0 = (tiles - 1 - (int)(blockIdx.x % tiles)) * kPT;
+  if (row0 >= L) return;
+  const int tid = threadIdx.x, ty = tid / 16, tx = tid % 16;
+  const T *Qu = Q + (size_t)u * Lmax * D, *Ku = K + (size_t)u * Lmax * D, *Vu = V + (size_t)u * Lmax * D;
+  const float zscale = scale * kLog2e;
+  load_tile<T, D>(Qs, Qu, row0, L, tid);
+  if (tid < kPT) lse2[tid] = (row0 + tid < L) ? lse[(size_t)u * Lmax + row0 + tid] * kLog2e : 0.f;
+  float o[4][D / 16];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int c = 0; c < D / 16; ++c) o[i][c] = 0.f;
+  for (int col0 = 0; col0 <= row0; col0 += kPT) {
+    __syncthreads();  // the previous tile's values (in Ks) and probabilities have been used
+    load_tile<T, D>(Ks, Ku, col0, L, tid);
+    __syncthreads();
+    float acc[4][4];
+    score_tile<D>(Qs, Ks, ty, tx, acc);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int gi = row0 + ty * 4 + i;
+      const float li = lse2[ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int gj = col0 + tx * 4 + j;
+        Ps[(ty * 4 + i) * (kPT + 1) + tx * 4 + j] = (gj <= gi && gi < L) ? exp2f(fmaf(acc[i][j], zscale, -li)) : 0.f;
+      }
+    }
+    __syncthreads();  // scores done with the keys: their place takes the values (rows past L read as zero)
+    load_tile<T, D>(Ks, Vu, col0, L, tid);
+    __syncthreads();
+#pragma unroll 4
+    for (int j = 0; j < kPT; ++j) {
+      float pr[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) pr[i] = Ps[(ty * 4 + i) * (kPT + 1) + j];
+#pragma unroll
+      for (int c = 0; c < D / 16; ++c) {
+        const float v = Ks[j * (D + 1) + tx + 16 * c];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o[i][c] = fmaf(pr[i], v, o[i][c]);
+      }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int gi = row0 + ty * 4 + i;
+    if (gi < L) {
+#pragma unroll
+      for (int c = 0; c < D / 16; ++c) Elem<T>::store(out + ((size_t)u * Lmax + gi) * D + tx + 16 * c, o[i][c]);
+    }
+  }
+}
+
+template <typename T, int D>
+static cudaError_t launch_attend_t(int S, int G, int Lmax, const int *lens, int maxlen, const void *Q, const void *K,
+                                   const void *V, float scale, const float *lse, void *out, cudaStream_t stream) {
+  const size_t smem = (2 * kPT * (D + 1) + kPT * (kPT + 1) + kPT) * sizeof(float);
+  cudaError_t err = cudaFuncSetAttribute(prefill_attend_simt_kernel<T, D>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  const int tiles = (maxlen + kPT - 1) / kPT;
+  const unsigned grid = (unsigned)(S * G) * (unsigned)tiles;
+  prefill_attend_simt_kernel<T, D><<<grid, kPThreads, smem, stream>>>((const T *)Q, (const T *)K, (const T *)V, lens, G,
+                                                                     Lmax, tiles, scale, lse, (T *)out);
+  return cudaGetLastError();
+}
+
+roco_status launch_prefill_attend_simt(int kv_dtype, int d, int S, int G, int Lmax, const int *lens_dev, int maxlen,
+                                       const void *Q, const void *K, const void *V, float scale, const float *lse,
+                                       void *out, cudaStream_t stream) {
+  cudaError_t err;
+  if (kv_dtype == ROCO_BF16 && d == 128)
+    err = launch_attend_t<__nv_bfloat16, 128>(S, G, Lmax, lens_dev, maxlen, Q, K, V, scale, lse, out, stream);
+  else if (kv_dtype == ROCO_BF16 && d == 64)
+    err = launch_attend_t<__nv_bfloat16, 64>(S, G, Lmax, lens_dev, maxlen, Q, K, V, scale, lse, out, stream);
+  else if (kv_dtype == ROCO_F32 && d == 128)
+    err = launch_attend_t<float, 128>(S, G, Lmax, lens_dev, maxlen, Q, K, V, scale, lse, out, stream);
+  else if (kv_dtype == ROCO_F32 && d == 64)
+    err = launch_attend_t<float, 64>(S, G, Lmax, lens_dev, maxlen, Q, K, V, scale, lse, out, stream);
+  else
+    return ROCO_ERR_UNSUPPORTED;
+  return err == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
+}
+
 template <typename T, int D>
 static cudaError_t launch_t(int S, int G, int Lmax, const int *lens, int maxlen, const void *Q, const void *K,
                             float scale, float *lse, float *s_full, float *q_full, cudaStream_t stream) {

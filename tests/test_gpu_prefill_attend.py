@@ -1,4 +1,5 @@
-"""GPU parity of the prompt pass's attention output (roco_prefill_attend, tensor cores) against the fp64 oracle."""
+"""GPU parity of the prompt pass's attention output (roco_prefill_attend, roco_prefill_with_output; tensor cores and
+the CUDA-core path) against the fp64 oracle."""
 import numpy as np
 import pytest
 import torch
@@ -73,13 +74,38 @@ def test_attend_long_prompt_sampled_rows():
     check_rows(w, Q, K, V, lse, out, lens, [0, 3, 7], lambda L: rows)
 
 
-def test_attend_rejects_unsupported_shapes():
-    w = W.TOY   # fp32, d = 64
+@pytest.mark.parametrize("dtype,d", [("f32", 64), ("bf16", 64), ("f32", 128)])
+@pytest.mark.parametrize("fused", [False, True])
+def test_attend_on_cuda_cores(dtype, d, fused):
+    """Dtypes and head dimensions the tensor-core path does not take (the toy configuration is fp32, d = 64): the
+    output comes from a CUDA-core pass over the row log-sum-exp, through roco_prefill_attend and through
+    roco_prefill_with_output alike.  Every row of every unit, ragged lengths, NaN in the padding rows."""
+    w = W.scaled(W.TOY, S=3, heads=2, d=d, dtype=dtype, prompt_lo=200, prompt_hi=200, B=64, r=8)
+    lens = [200, 129, 5]
+    Q, K, V = prompt_tensors(w, 200)
+    for b, L in enumerate(lens):
+        for X in (Q, K, V):
+            X[b, :, L:] = float("nan")
     cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
-    Q = torch.zeros(w.S, w.G, 128, w.d, device=DEV)
-    lse = torch.zeros(w.S, w.G, 128, device=DEV)
-    with pytest.raises(R.RocoError):
-        R.roco_prefill_attend(cache, Q, Q, Q, [128], lse, torch.zeros_like(Q))
+    assert not R.roco_prefill_uses_tensor_cores(cache)
+    lse = torch.zeros(w.S, w.G, 200, dtype=torch.float32, device=DEV)
+    out = torch.full((w.S, w.G, 200, w.d), 7.0, dtype=w.torch_dtype, device=DEV)
+    if fused:
+        R.roco_prefill(Q, K, V, lens, w.B, w.r, cache, scale=w.scale, lse_out=lse, attn_out=out)
+    else:
+        R.roco_prefill(Q, K, V, lens, w.B, w.r, cache, scale=w.scale, lse_out=lse)
+        R.roco_prefill_attend(cache, Q, K, V, lens, lse, out, scale=w.scale)
+    torch.cuda.synchronize()
+    assert R.roco_device_status(cache) == 0
+    tol = 2e-2 if dtype == "bf16" else 1e-5
+    for u in range(w.U):
+        L = lens[u // w.G]
+        q, k, v = (widen(unit_view(X, [u]))[0, :L] for X in (Q, K, V))
+        want, want_lse = oracle.prompt_attention_rows(q, k, v, list(range(L)), w.scale)
+        got = widen(unit_view(out, [u]))[0]
+        np.testing.assert_allclose(widen(unit_view(lse, [u]))[0, :L], want_lse, rtol=0, atol=1e-4)
+        np.testing.assert_allclose(got[:L], want, rtol=tol, atol=tol, err_msg=f"unit {u}")
+        assert np.all(got[L:] == 7.0), "rows past the prompt must be left untouched"
 
 
 # ------------------------------------------------ one sweep: output and row log-sum-exp together (running maximum)
@@ -166,9 +192,7 @@ def test_fused_prompt_pass_argument_checks():
     with pytest.raises(R.RocoError) as e:                        # the running-maximum sweep needs scale > 0
         R.roco_prefill(Q, K, V, [128], w.B, w.r, cache, scale=-0.1, attn_out=torch.zeros_like(Q))
     assert e.value.code == 1
-    t = W.TOY                                                    # fp32, d = 64: no tensor-core path
-    c2 = R.Cache(t.S, t.G, t.B, t.d, t.torch_dtype, DEV)
-    X = torch.zeros(t.S, t.G, 128, t.d, device=DEV)
-    with pytest.raises(R.RocoError) as e:
-        R.roco_prefill(X, X, X, [128], t.B, t.r, c2, attn_out=torch.zeros_like(X))
-    assert e.value.code == 2
+    misaligned = torch.zeros(Q.numel() + 8, dtype=Q.dtype, device=DEV)[1:1 + Q.numel()].view_as(Q)
+    with pytest.raises(R.RocoError) as e:                        # the output must be 16-byte aligned
+        R.roco_prefill(Q, K, V, [128], w.B, w.r, cache, attn_out=misaligned)
+    assert e.value.code == 1
