@@ -225,7 +225,9 @@ roco_status roco_decode_step_policy(roco_cache *cache, const void *q, const void
  * b = 1 is roco_decode_step with ROCO_EVICT_FIRST.
  *
  *   Q, K_new, V_new  [S][G][b][d], cache->kv_dtype
- *   b                1..16; b > 1 needs ROCO_SCOPE_EXCLUDE_TOP_R (else ROCO_ERR_UNSUPPORTED) and r + b <= B;
+ *   b                1..16, r + b <= B.  Under ROCO_SCOPE_LOWEST_R the scope refills after each of the step's
+ *                    evictions (the token next in (variance, position) order is admitted before the next victim
+ *                    is taken), all on the statistics as they stand before the step;
  *                    b * B floats of scores must fit in shared memory (else ROCO_ERR_UNSUPPORTED)
  *   attn_out         [S][G][b][d];   lse_out [S][G][b] or NULL
  *   evicted_slot     [S][G][b] freed slots in increasing order, padded with -1;  evicted_pos likewise, or NULL

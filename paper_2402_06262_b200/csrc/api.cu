@@ -329,7 +329,6 @@ roco_status roco_gqa_block_step(roco_cache *cache, const void *Q, const void *K_
   if (b < 1 || group < 1) return ROCO_ERR_INVALID_ARG;
   if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
   if ((long long)b * group > multi_max_queries()) return ROCO_ERR_UNSUPPORTED;
-  if (b > 1 && scope_mode != ROCO_SCOPE_EXCLUDE_TOP_R) return ROCO_ERR_UNSUPPORTED;  // the scope would refill
   if (b > 1 && r + b > cache->B) return ROCO_ERR_INVALID_ARG;  // the scope must hold the b victims
   if (!multi_fits(cache->B, cache->d, b * group, b)) return ROCO_ERR_UNSUPPORTED;
   return launch_multi_step(*cache, b * group, b, Q, K_new, V_new, r, scope_mode, scale, attn_out, lse_out,

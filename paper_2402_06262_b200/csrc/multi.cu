@@ -281,7 +281,92 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     // (variance, position) order is in scope iff fewer than m tokens come before it, and then so are the others
     // (they come before it too) -- one counting pass in place of the radix select for the scope threshold.
     bool done = false;
-    if (2 * m >= live0) {
+    if (need > 1 && p.scope_mode == ROCO_SCOPE_LOWEST_R && m < live0) {
+      // The scope is the r lowest-variance tokens still cached (Sec. 1 reading), so it refills after every
+      // eviction: one radix select gives the scope of the first eviction, and each later one admits the token
+      // next in (variance, position) order before the in-scope token of lowest mean leaves.  The state of a
+      // token is kept in newtok for the duration: -1 outside the scope, -2 in scope, -3 evicted.
+      uint32_t Tv = radix_select<uint32_t>([&](int j) { return v.vkey[j]; }, [&](int) { return true; }, live0,
+                                           (uint32_t)(m - 1), *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &rank, &ties,
+                                           k_and, k_or);
+      int Pv = 0x7fffffff;
+      if (ties != rank + 1) {
+        uint32_t r2, t2;
+        Pv = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)opos[j]; },
+                                         [&](int j) { return v.vkey[j] == Tv; }, live0, rank, *v.sel, ptid,
+                                         kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
+      }
+      for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+        const uint32_t k = v.vkey[j];
+        if (k < Tv || (k == Tv && (Pv == 0x7fffffff || opos[j] <= Pv))) v.newtok[j] = -2;
+      }
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      bool ok = true;
+#pragma unroll 1
+      for (int it = 0; it < need; ++it) {
+        if (it > 0 && p.r <= live0 - it) {  // the scope has lost a token and the cache still holds one to admit
+          uint32_t bk = 0xffffffffu;
+          int bs = -1, bp = 0x7fffffff;
+          for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+            if (v.newtok[j] != -1) continue;
+            const uint32_t k = v.vkey[j];
+            const int pj = opos[j];
+            if (bs < 0 || k < bk || (k == bk && pj < bp)) { bk = k; bs = j; bp = pj; }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const uint32_t ok2 = __shfl_xor_sync(0xffffffffu, bk, o);
+            const int op = __shfl_xor_sync(0xffffffffu, bp, o);
+            const int os = __shfl_xor_sync(0xffffffffu, bs, o);
+            if (os >= 0 && (bs < 0 || ok2 < bk || (ok2 == bk && op < bp))) { bk = ok2; bp = op; bs = os; }
+          }
+          if (plane == 0) { v.sel->hist[pwarp] = bk; v.sel->red_pos[pwarp] = bp; v.sel->red_slot[pwarp] = bs; }
+          named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+          bk = v.sel->hist[0]; bp = v.sel->red_pos[0]; bs = v.sel->red_slot[0];
+#pragma unroll
+          for (int w = 1; w < kMqPolicyThreads / 32; ++w) {
+            const uint32_t ok2 = v.sel->hist[w];
+            const int op = v.sel->red_pos[w], os = v.sel->red_slot[w];
+            if (os >= 0 && (bs < 0 || ok2 < bk || (ok2 == bk && op < bp))) { bk = ok2; bp = op; bs = os; }
+          }
+          named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+          if (bs >= 0 && ptid == 0) v.newtok[bs] = -2;
+          named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+        }
+        float bm = INFINITY;
+        int bs = -1, bp = 0x7fffffff;
+        for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+          if (v.newtok[j] != -2) continue;
+          const float mean = v.mkey[j];
+          const int pj = opos[j];
+          if (mean < bm || (mean == bm && pj < bp)) { bm = mean; bs = j; bp = pj; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float om = __shfl_xor_sync(0xffffffffu, bm, o);
+          const int op = __shfl_xor_sync(0xffffffffu, bp, o);
+          const int os = __shfl_xor_sync(0xffffffffu, bs, o);
+          if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+        }
+        if (plane == 0) { v.sel->red_mean[pwarp] = bm; v.sel->red_pos[pwarp] = bp; v.sel->red_slot[pwarp] = bs; }
+        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+        bm = v.sel->red_mean[0]; bp = v.sel->red_pos[0]; bs = v.sel->red_slot[0];
+#pragma unroll
+        for (int w = 1; w < kMqPolicyThreads / 32; ++w) {
+          const float om = v.sel->red_mean[w];
+          const int op = v.sel->red_pos[w], os = v.sel->red_slot[w];
+          if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+        }
+        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+        if (bs < 0) { ok = false; bs = it; }  // only after corrupt statistics; keeps the slots distinct
+        if (ptid == 0) { list[it] = bs; v.newtok[bs] = -3; }
+        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      }
+      for (int j = ptid; j < live0; j += kMqPolicyThreads) v.newtok[j] = -1;
+      if (!ok && ptid == 0) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
+      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      done = true;
+    } else if (2 * m >= live0) {
       bool ok;
       if (need <= 4) {
         ok = argmin_rounds(need);

@@ -49,6 +49,27 @@ def test_block_steps_fill_then_evict(b, dtype, d, B):
     assert tally.decisions > 0
 
 
+@pytest.mark.parametrize("b", [2, 5, 16])
+@pytest.mark.parametrize("r", [1, 9, 150, 290])
+@pytest.mark.parametrize("dtype,d,B", [("bf16", 128, 300), ("f32", 64, 128)])
+def test_block_steps_lowest_r_scope_refills(b, r, dtype, d, B):
+    """The other reading of the scope (the r lowest-variance tokens): within one block step the scope refills
+    after every eviction.  r = 1 (each victim is the lowest-variance token left), a small scope, one that is half
+    the cache, and one larger than what is left after a few evictions (the scope is then everything)."""
+    r = min(r, B - b)
+    w = W.scaled(W.LLAMA7B_DECODE, S=2, layers=1, heads=3, d=d, dtype=dtype, prompt_lo=B - 21, prompt_hi=B - 21,
+                 B=B, r=r)
+    tally = Tally()
+    cache, st = prefilled(w, B - 21, tally, range(w.U))
+    par = BlockParity(cache, st, range(w.U), b, r, R.ROCO_SCOPE_LOWEST_R, tally, scale=w.scale)
+    t = B - 21
+    for i in range(max(4, 48 // b)):
+        par.step(*block_tokens(w, i * b, b, [t] * w.S), check_state=True)
+        t += b
+    assert R.roco_device_status(cache) == 0
+    assert tally.decisions > 0 and tally.near_ties <= max(4, tally.decisions // 4), tally
+
+
 def test_block_step_after_eviction_prefill_llama_shape():
     """Evict-and-encode with b = 16 on a cache built by prefill eviction (B = 1024, d = 128, bf16, sinks)."""
     w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=8, prompt_lo=1500, prompt_hi=1500)
@@ -89,9 +110,6 @@ def test_block_step_argument_checks():
     out = lambda b: (torch.zeros(w.S, w.G, b, w.d, device=DEV), torch.zeros(w.S, w.G, b, dtype=torch.int32, device=DEV))
     with pytest.raises(R.RocoError) as e:
         R.roco_block_step(cache, mk(17), mk(17), mk(17), 4, *out(17))
-    assert e.value.code == 2
-    with pytest.raises(R.RocoError) as e:
-        R.roco_block_step(cache, mk(4), mk(4), mk(4), 4, *out(4), scope_mode=R.ROCO_SCOPE_LOWEST_R)
     assert e.value.code == 2
     with pytest.raises(R.RocoError) as e:
         R.roco_block_step(cache, mk(8), mk(8), mk(8), 25, *out(8))        # r + b > B
