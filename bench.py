@@ -424,7 +424,8 @@ def few_units_bench(R, cache, w, device, reps=6):
             return {"path": name, "us_per_step": iso * 1e3, "hbm_frac": algb / iso / 1e6 / hbm_peak,
                     "us_per_step_layer_sweep": sweep * 1e3, "hbm_frac_layer_sweep": algb / sweep / 1e6 / hbm_peak}
 
-        rows = [row("one CTA per unit", lambda c: (lambda: R.roco_decode_step(c, q1, k1, v1, rr, out1, ev1, scale=sc)))]
+        rows = [row("one CTA per unit", lambda c: (lambda: R.roco_decode_step_cluster(c, q1, k1, v1, rr, out1, ev1, ranks=1,
+                                                                                      scale=sc)))]
         rows[-1]["splits"] = 0
         for sp in (2, 4, 8):
             ws = torch.empty(R.roco_decode_split_workspace_bytes(cch, sp), dtype=torch.uint8, device=device)
@@ -434,7 +435,7 @@ def few_units_bench(R, cache, w, device, reps=6):
         kr = R.roco_decode_cluster_ranks(cch)
         for order, oname in ((0, "EVICT_FIRST"), (1, "ATTEND_FIRST")):
             if kr > 1:
-                rows.append(row(f"one launch, cluster of {kr} CTAs per unit, {oname}",
+                rows.append(row(f"one launch, cluster of {kr} CTAs per unit (what roco_decode_step picks), {oname}",
                                 lambda c, order=order: (lambda: R.roco_decode_step_cluster(c, q1, k1, v1, rr, out1, ev1,
                                                                                            step_order=order, ranks=kr, scale=sc))))
                 rows[-1]["ranks"] = kr

@@ -175,6 +175,8 @@ roco_status roco_prefill_static(const void *Q, const void *K, const void *V, con
  * slots (Eq. 1); every occupied slot gets n += 1, s += p, q += p^2.  ATTEND_FIRST: attention and the
  * statistics update run over the cache as it stands, then the eviction and the in-place write.
  * The cache is never compacted: only the freed slot is overwritten.
+ * One launch.  Its shape follows the call's size: one CTA per unit when the units fill the GPU, a cluster of
+ * 2, 4 or 8 CTAs per unit when they are few (roco_decode_step_cluster with ranks = 0, below).
  *
  *   q, k_new, v_new  [S][G][d], cache->kv_dtype
  *   r                EXCLUDE_TOP_R: 0 <= r < B;  LOWEST_R: 1 <= r <= B
@@ -334,7 +336,8 @@ roco_status roco_decode_step_split(roco_cache *cache, const void *q, const void 
  * (Fig. 1), and each rank updates the statistics of its own slots.  One launch, no workspace, no global-memory
  * traffic besides what roco_decode_step has.  Same arguments, results and parity bounds as roco_decode_step.
  *
- *   ranks   2, 4 or 8 CTAs per unit; 1: the one-CTA-per-unit kernel; 0: roco_decode_cluster_ranks(cache)
+ *   ranks   2, 4 or 8 CTAs per unit; 1: the one-CTA-per-unit kernel; 0: roco_decode_cluster_ranks(cache), which is
+ *           what roco_decode_step does
  * Needs B a multiple of 4 and 16-byte aligned statistics arrays (else ROCO_ERR_UNSUPPORTED for ranks > 1).
  * roco_decode_cluster_ranks: the cluster size that suits this cache's shape on the current device -- the
  * largest whose CTAs fit the GPU in one wave of two per SM while every rank keeps at least two 16 KiB tiles;

@@ -237,15 +237,9 @@ roco_status roco_prefill_attend(const roco_cache *cache, const void *Q, const vo
 roco_status roco_decode_step(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,
                              int scope_mode, int step_order, float scale, void *attn_out, float *lse_out,
                              int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {
-  NvtxRange range("roco_decode_step");
-  roco_status st = check_cache(cache);
-  if (st != ROCO_OK) return st;
-  if (!q || !k_new || !v_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
-  if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
-  if (step_order != ROCO_EVICT_FIRST && step_order != ROCO_ATTEND_FIRST) return ROCO_ERR_INVALID_ARG;
-  return launch_decode_step(*cache, q, k_new, v_new, r, scope_mode, step_order, ROCO_POLICY_ROCO, nullptr, scale,
-                            attn_out, lse_out, evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
+  // the launch shape follows the call's size: one CTA per unit, or a cluster of CTAs per unit when the units are few
+  return roco_decode_step_cluster(cache, q, k_new, v_new, r, scope_mode, step_order, 0, scale, attn_out, lse_out,
+                                  evicted_slot, evicted_pos, stream);
 }
 
 size_t roco_decode_split_workspace_bytes(const roco_cache *cache, int splits) {
@@ -273,10 +267,15 @@ roco_status roco_decode_step_split(roco_cache *cache, const void *q, const void 
 
 int roco_decode_cluster_ranks(const roco_cache *cache) {
   if (check_cache(cache) != ROCO_OK) return 0;
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return 0;
+  static int sm_count[kHostMaxDevices] = {};  // per device, asked once (racing first calls write the same value)
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kHostMaxDevices) return 0;
+  if (sm_count[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 0;
+    sm_count[dev] = n;
+  }
+  const int sms = sm_count[dev];
   if (((reinterpret_cast<uintptr_t>(cache->s) | reinterpret_cast<uintptr_t>(cache->q) |
         reinterpret_cast<uintptr_t>(cache->n) | reinterpret_cast<uintptr_t>(cache->pos)) & 15) != 0)
     return 1;
@@ -286,7 +285,7 @@ int roco_decode_cluster_ranks(const roco_cache *cache) {
 roco_status roco_decode_step_cluster(roco_cache *cache, const void *q, const void *k_new, const void *v_new, int r,
                                      int scope_mode, int step_order, int ranks, float scale, void *attn_out,
                                      float *lse_out, int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {
-  NvtxRange range("roco_decode_step_cluster");
+  NvtxRange range("roco_decode_step");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
   if (!q || !k_new || !v_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;

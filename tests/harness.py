@@ -139,7 +139,7 @@ class DecodeParity:
                  tally: Tally, scale: Optional[float] = None, strict: bool = False, splits: int = 0,
                  ranks: int = 0):
         self.splits = splits
-        self.ranks = ranks      # > 1: a cluster of that many CTAs per unit
+        self.ranks = ranks      # 0: roco_decode_step picks the launch shape; 1: one CTA per unit; > 1: that cluster
         self.ws = (torch.empty(R.roco_decode_split_workspace_bytes(cache, splits), dtype=torch.uint8,
                                device=cache.K.device) if splits else None)
         self.cache, self.st, self.units = cache, st, list(units)
@@ -153,7 +153,7 @@ class DecodeParity:
 
     def step(self, q, k_new, v_new, check_state: bool = False):
         c = self.cache
-        if self.ranks > 1:
+        if self.ranks >= 1:
             R.roco_decode_step_cluster(c, q, k_new, v_new, self.r, self.out, self.ev_slot, self.ev_pos, self.lse,
                                        scope_mode=self.mode, step_order=self.order, ranks=self.ranks, scale=self.scale)
         elif self.splits:

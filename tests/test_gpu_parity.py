@@ -22,7 +22,7 @@ def prompt_tensors(w, L, device=DEV):
     return torch.stack(qs), torch.stack(ks), torch.stack(vs)
 
 
-def run_workload(w, units, mode, order, steps, lens=None, check_every=8, Lmax=None):
+def run_workload(w, units, mode, order, steps, lens=None, check_every=8, Lmax=None, ranks=0):
     """prefill + `steps` decode steps of workload w on the GPU, compared with the oracle on `units`."""
     tally = Tally()
     lens = W.prompt_lens(w) if lens is None else lens
@@ -30,7 +30,7 @@ def run_workload(w, units, mode, order, steps, lens=None, check_every=8, Lmax=No
     Q, K, V = prompt_tensors(w, Lmax)
     cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
     st = prefill_parity(cache, Q, K, V, lens, w.r, mode, units, tally, scale=w.scale)
-    par = DecodeParity(cache, st, units, w.r, mode, order, tally, scale=w.scale)
+    par = DecodeParity(cache, st, units, w.r, mode, order, tally, scale=w.scale, ranks=ranks)
     t_pos = list(lens)
     for i in range(steps):
         q, k, v = W.decode_tokens(w, i, t_pos, DEV)
@@ -51,12 +51,14 @@ def test_toy_config_whole(mode, order):
 
 @pytest.mark.parametrize("mode,order", MODES)
 @pytest.mark.parametrize("dtype,d,B", [("bf16", 128, 300), ("bf16", 64, 333), ("f32", 128, 100)])
-def test_fill_then_evict_ragged_tiles(mode, order, dtype, d, B):
+@pytest.mark.parametrize("ranks", [0, 1])     # the shape roco_decode_step picks for so few units, and one CTA per unit
+def test_fill_then_evict_ragged_tiles(mode, order, dtype, d, B, ranks):
     """Short prompts (cache not full): slots are appended until the buffer fills, then eviction starts.
     B is not a multiple of the tile height, and the live count crosses tile boundaries on the way."""
     w = W.scaled(W.LLAMA7B_DECODE, S=2, layers=1, heads=5, d=d, dtype=dtype, prompt_lo=B - 40, prompt_hi=B - 40,
                  B=B, r=7, steps=60)
-    t = run_workload(w, range(w.U), mode, order, w.steps, lens=[B - 40, B - 55], check_every=10, Lmax=B - 40)
+    t = run_workload(w, range(w.U), mode, order, w.steps, lens=[B - 40, B - 55], check_every=10, Lmax=B - 40,
+                     ranks=ranks)
     assert t.decisions >= 2 * 5 * 5
 
 
