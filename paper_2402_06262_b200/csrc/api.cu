@@ -292,7 +292,19 @@ roco_status roco_decode_step_cluster(roco_cache *cache, const void *q, const voi
   if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
   if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
   if (step_order != ROCO_EVICT_FIRST && step_order != ROCO_ATTEND_FIRST) return ROCO_ERR_INVALID_ARG;
-  if (ranks == 0) ranks = roco_decode_cluster_ranks(cache);
+  const bool automatic = ranks == 0;
+  if (automatic) {
+    ranks = roco_decode_cluster_ranks(cache);
+    if (ranks > 1) {
+      // a cluster launch can be refused where the device cannot co-schedule that many CTAs (a partitioned GPU):
+      // nothing has been enqueued then, and the step still runs with one CTA per unit
+      st = launch_decode_step_cluster(*cache, ranks, q, k_new, v_new, r, scope_mode, step_order, scale, attn_out,
+                                      lse_out, evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
+      if (st == ROCO_OK) return st;
+      (void)cudaGetLastError();
+      ranks = 1;
+    }
+  }
   if (ranks == 1)
     return launch_decode_step(*cache, q, k_new, v_new, r, scope_mode, step_order, ROCO_POLICY_ROCO, nullptr, scale,
                               attn_out, lse_out, evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));

@@ -551,9 +551,9 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
           dq = ds * ds;
           dn = 1;
         } else {
-          ds = v.ds[j];
+          ds = v.ds[j];  // sums over the block's tokens of the (group-wise averaged) probability and its square
           dq = v.dq[j];
-          dn = M;
+          dn = nb;
         }
       } else {
         // token t of the block (its `group` query heads) sees new token jn only if t >= jn; the statistics take
@@ -1190,6 +1190,9 @@ __host__ __device__ inline int multi_tm_cols(int B) {
   return c;
 }
 
+// kGroupedTokens: several tokens per step, each with several query heads (the statistics then take the heads'
+// mean per token); false: every query row is a token of its own, or all rows are the heads of one token.
+template <bool kGroupedTokens>
 __global__ void __launch_bounds__(kMqThreads, 2) multi_step_tm_kernel(const __grid_constant__ CUtensorMap mapK,
                                                                       const __grid_constant__ CUtensorMap mapV,
                                                                       const MultiParams p, int tmem_cols) {
@@ -1442,13 +1445,34 @@ __global__ void __launch_bounds__(kMqThreads, 2) multi_step_tm_kernel(const __gr
           const float p2 = __uint_as_float(r[4 * t + 2]) * inv_hi, p3 = __uint_as_float(r[4 * t + 3]) * inv_hi;
           *reinterpret_cast<uint32_t *>(sm.pz + (size_t)g * Bp + j) = pack_bf16x2(p0, p1);
           *reinterpret_cast<uint32_t *>(sm.pz + (size_t)(g + 8) * Bp + j) = pack_bf16x2(p2, p3);
-          float s0 = p0 + p2, s1 = p1 + p3, q0 = fmaf(p0, p0, p2 * p2), q1 = fmaf(p1, p1, p3 * p3);
+          // Rows g and g + 8 of this thread are query heads g % grp and (g + 8) % grp of two different tokens
+          // (grp divides 8 here; one token with all its heads when nb = 1, summed as a whole).  First the heads
+          // of a token are added up (the lanes that differ in the low bits of g), which gives the group-wise
+          // averaged probability of Sec. 5.3 / App. A; then p and p^2 of the tokens (the remaining bits).
+          float a0 = p0, a1 = p1, a2 = p2, a3 = p3;
+          if (kGroupedTokens) {
 #pragma unroll
-          for (int o = 4; o <= 16; o <<= 1) {  // over the eight row pairs
-            s0 += __shfl_xor_sync(0xffffffffu, s0, o);
-            s1 += __shfl_xor_sync(0xffffffffu, s1, o);
-            q0 += __shfl_xor_sync(0xffffffffu, q0, o);
-            q1 += __shfl_xor_sync(0xffffffffu, q1, o);
+            for (int o = 4; o <= 16; o <<= 1) {
+              if (o < 4 * grp) {
+                a0 += __shfl_xor_sync(0xffffffffu, a0, o);
+                a1 += __shfl_xor_sync(0xffffffffu, a1, o);
+                a2 += __shfl_xor_sync(0xffffffffu, a2, o);
+                a3 += __shfl_xor_sync(0xffffffffu, a3, o);
+              }
+            }
+            const float ig = 1.f / (float)grp;
+            a0 *= ig; a1 *= ig; a2 *= ig; a3 *= ig;
+          }
+          float s0 = a0 + a2, s1 = a1 + a3, q0 = fmaf(a0, a0, a2 * a2), q1 = fmaf(a1, a1, a3 * a3);
+          const int o_first = kGroupedTokens ? 4 * grp : 4;
+#pragma unroll
+          for (int o = 4; o <= 16; o <<= 1) {  // over the tokens (all eight row pairs when every row is a token)
+            if (o >= o_first) {
+              s0 += __shfl_xor_sync(0xffffffffu, s0, o);
+              s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+              q0 += __shfl_xor_sync(0xffffffffu, q0, o);
+              q1 += __shfl_xor_sync(0xffffffffu, q1, o);
+            }
           }
           if (g == 0) { ds[j] = s0; ds[j + 1] = s1; dq[j] = q0; dq[j + 1] = q1; }
         }
@@ -1577,15 +1601,21 @@ roco_status launch_multi_step(const roco_cache &c, int M, int nb, const void *Q,
     CUtensorMap mapK, mapV;
     // the tensor-memory kernel forms per-slot sums over all query rows, which is the statistic only when the rows
     // are all tokens (one head) or all heads (one token)
-    const int tm_stages = (nb == 1 || nb == M) ? multi_tm_pick_stages(c.B, M, nb) : 0;
+    // the tensor-memory kernel sums the heads of a token with lane shuffles: group sizes that divide 8
+    const int grp_of = M / nb;
+    const bool tm_group = nb == 1 || grp_of == 1 || grp_of == 2 || grp_of == 4 || grp_of == 8;
+    const int tm_stages = tm_group ? multi_tm_pick_stages(c.B, M, nb) : 0;
     p.stages = tm_stages > 0 ? tm_stages : multi_tc_pick_stages(c.B, M, nb);
     if (p.stages > 0 && make_tensor_map_rows128_bf16(&mapK, c.K, (unsigned long long)U * c.B, 64) &&
         make_tensor_map_rows128_bf16(&mapV, c.V, (unsigned long long)U * c.B, 64)) {
       if (tm_stages > 0) {
         const size_t smem = multi_tm_smem_bytes(c.B, p.stages, M, nb);
-        err = cudaFuncSetAttribute(multi_step_tm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const bool grouped = nb > 1 && grp_of > 1;
+        err = grouped ? cudaFuncSetAttribute(multi_step_tm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                      : cudaFuncSetAttribute(multi_step_tm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return ROCO_ERR_CUDA;
-        multi_step_tm_kernel<<<U, kMqThreads, smem, stream>>>(mapK, mapV, p, multi_tm_cols(c.B));
+        if (grouped) multi_step_tm_kernel<true><<<U, kMqThreads, smem, stream>>>(mapK, mapV, p, multi_tm_cols(c.B));
+        else multi_step_tm_kernel<false><<<U, kMqThreads, smem, stream>>>(mapK, mapV, p, multi_tm_cols(c.B));
         return cudaGetLastError() == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
       }
       const size_t smem = multi_tc_smem_bytes(c.B, p.stages, M, nb);
