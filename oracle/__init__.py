@@ -283,8 +283,10 @@ def gqa_step(st: State, Q, k_new, v_new, r, mode, scale, delta=1e-5, force_victi
     return StepResult(out, lse, es, ep, ch, nt.astype(bool))
 
 
-def policy_step(st: State, qv, k_new, v_new, policy, r, scale, rnd=None, delta=1e-5, force_victim=None):
-    """One decode step (evict, insert, attend) under one of the Table 1 policies, in place on `st`.
+def policy_step(st: State, qv, k_new, v_new, policy, r, scale, rnd=None, delta=1e-5, force_victim=None,
+                order=EVICT_FIRST):
+    """One decode step under one of the Table 1 policies, in place on `st`; order: EVICT_FIRST (evict, insert,
+    attend) or ATTEND_FIRST (attend and update, then evict and insert).
     Returns (StepResult, quant_near [U][B] bool).  rnd: [U] uint32 draws for POLICY_RANDOM."""
     qv, k_new, v_new = _f64(qv), _f64(k_new), _f64(v_new)
     U, B, d = st.U, st.B, st.d
@@ -295,7 +297,7 @@ def policy_step(st: State, qv, k_new, v_new, policy, r, scale, rnd=None, delta=1
     rn = None if rnd is None else np.ascontiguousarray(rnd, dtype=np.uint32)
     lib().roco_oracle_policy_step_batch(C.c_int(U), _p(st.K), _p(st.V), _p(st.s), _p(st.q), _p(st.n), _p(st.pos),
                                         _p(st.live), _p(st.t_next), C.c_int(B), C.c_int(d), _p(qv), _p(k_new),
-                                        _p(v_new), C.c_int(policy), C.c_int(r), _p(rn), C.c_double(scale),
+                                        _p(v_new), C.c_int(policy), C.c_int(r), C.c_int(order), _p(rn), C.c_double(scale),
                                         C.c_double(delta), _p(fv), _p(out), _p(lse), _p(es), _p(ep), _p(ch), _p(nt),
                                         _p(qn))
     return StepResult(out, lse, es, ep, ch, nt.astype(bool)), qn.astype(bool)

@@ -809,63 +809,46 @@ enum {
   ROCO_ORACLE_POLICY_MAS_WINDOW = 7    /* Sec. 4.3 preliminary experiment: MAS + local window of size r            */
 };
 
-/* One decode step (evict, insert, attend: Fig. 1) under one of the policies above.
- * State: s = accumulated probability (Acc), n = Count for every policy; q = Acc^square, except under
- * SCISSORHANDS, where it accumulates the quantised score (1 if the token's probability exceeds the average
- * 1/live of this query, else 0), and under TOVA, where it holds the last query's probability.
- * Local window (Sec. 4.2): tokens outside a window of the r most recent positions are evictable, i.e. pos < t - r
- * with t the position of the incoming token.  Ties: (score asc, position asc).
- * rnd: the random draw for RANDOM (victim = rnd mod live).  quant_near [B] (may be NULL): set to 1 where a
- * SCISSORHANDS quantisation falls within delta (relative) of the average. */
-void roco_oracle_policy_step_unit(double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
-                                  int *t_next, int B, int d, const double *qv, const double *k_new,
-                                  const double *v_new, int policy, int r, unsigned rnd, double scale, double delta,
-                                  int force_victim, double *out, double *lse, int *evicted_slot, int *evicted_pos,
-                                  int *choice, int *near_tie, int *quant_near) {
-  const int t = *t_next;
-  int slot, own = -1, near = 0;
-  *evicted_slot = -1;
-  *evicted_pos = -1;
-  if (*live == B) {
-    if (policy == ROCO_ORACLE_POLICY_ROCO) {
-      own = roco_oracle_select(s, q, n, pos, B, r, ROCO_ORACLE_EXCLUDE_TOP_R, delta, &near, NULL);
-    } else if (policy == ROCO_ORACLE_POLICY_RANDOM) {
-      own = (int)(rnd % (unsigned)B);
-    } else {
-      const int windowed = policy == ROCO_ORACLE_POLICY_SCISSORHANDS || policy == ROCO_ORACLE_POLICY_H2O ||
-                           policy == ROCO_ORACLE_POLICY_MAS_WINDOW;
-      int any = 0;
-      for (int j = 0; j < B; ++j) if (!windowed || pos[j] < t - r) any = 1;
-      double best = 0.0, second = INFINITY;
-      for (int j = 0; j < B; ++j) {
-        if (windowed && any && !(pos[j] < t - r)) continue;
-        if (policy == ROCO_ORACLE_POLICY_STREAMLLM && pos[j] < 4) continue;
-        double sc = 0.0; /* RECENCY, STREAMLLM: position alone decides */
-        if (policy == ROCO_ORACLE_POLICY_H2O) sc = s[j];
-        if (policy == ROCO_ORACLE_POLICY_SCISSORHANDS || policy == ROCO_ORACLE_POLICY_TOVA) sc = q[j];
-        if (policy == ROCO_ORACLE_POLICY_MAS_WINDOW) sc = s[j] / n[j];
-        if (own < 0 || sc < best || (sc == best && pos[j] < pos[own])) {
-          if (own >= 0) second = best < second ? best : second;
-          best = sc; own = j;
-        } else if (sc < second) {
-          second = sc;
-        }
-      }
-      if (own < 0) { own = 0; for (int j = 1; j < B; ++j) if (pos[j] < pos[own]) own = j; } /* all sinks */
-      const int real_valued = policy == ROCO_ORACLE_POLICY_H2O || policy == ROCO_ORACLE_POLICY_TOVA ||
-                              policy == ROCO_ORACLE_POLICY_MAS_WINDOW;
-      if (real_valued && second - best <= delta * (second + best)) near = 1;
+/* The token a policy evicts from a full buffer (Sec. 4.1, 4.2, 5.1), given the state arrays described at
+ * roco_oracle_policy_step_unit and t, the position of the incoming token.  *near: the decision is inside the
+ * margin delta. */
+static int policy_pick(const double *s, const double *q, const int *n, const int *pos, int B, int policy, int r,
+                       unsigned rnd, int t, double delta, int *near) {
+  int own = -1;
+  *near = 0;
+  if (policy == ROCO_ORACLE_POLICY_ROCO) return roco_oracle_select(s, q, n, pos, B, r, ROCO_ORACLE_EXCLUDE_TOP_R, delta, near, NULL);
+  if (policy == ROCO_ORACLE_POLICY_RANDOM) return (int)(rnd % (unsigned)B);
+  const int windowed = policy == ROCO_ORACLE_POLICY_SCISSORHANDS || policy == ROCO_ORACLE_POLICY_H2O ||
+                       policy == ROCO_ORACLE_POLICY_MAS_WINDOW;
+  int any = 0;
+  for (int j = 0; j < B; ++j) if (!windowed || pos[j] < t - r) any = 1;
+  double best = 0.0, second = INFINITY;
+  for (int j = 0; j < B; ++j) {
+    if (windowed && any && !(pos[j] < t - r)) continue;
+    if (policy == ROCO_ORACLE_POLICY_STREAMLLM && pos[j] < 4) continue;
+    double sc = 0.0; /* RECENCY, STREAMLLM: position alone decides */
+    if (policy == ROCO_ORACLE_POLICY_H2O) sc = s[j];
+    if (policy == ROCO_ORACLE_POLICY_SCISSORHANDS || policy == ROCO_ORACLE_POLICY_TOVA) sc = q[j];
+    if (policy == ROCO_ORACLE_POLICY_MAS_WINDOW) sc = s[j] / n[j];
+    if (own < 0 || sc < best || (sc == best && pos[j] < pos[own])) {
+      if (own >= 0) second = best < second ? best : second;
+      best = sc; own = j;
+    } else if (sc < second) {
+      second = sc;
     }
-    slot = (force_victim >= 0 && force_victim < B && near) ? force_victim : own;
-    *evicted_slot = slot;
-    *evicted_pos = pos[slot];
-  } else {
-    slot = (*live)++;
   }
-  insert_token(K, V, s, q, n, pos, slot, d, k_new, v_new, t);
-  const int m = *live;
-  double *p = (double *)malloc(sizeof(double) * (size_t)m);
-  *lse = softmax_row(qv, K, m, d, scale, p);
+  if (own < 0) { own = 0; for (int j = 1; j < B; ++j) if (pos[j] < pos[own]) own = j; } /* all sinks */
+  const int real_valued = policy == ROCO_ORACLE_POLICY_H2O || policy == ROCO_ORACLE_POLICY_TOVA ||
+                          policy == ROCO_ORACLE_POLICY_MAS_WINDOW;
+  if (real_valued && second - best <= delta * (second + best)) *near = 1;
+  return own;
+}
+
+/* Eq. 1 over the m occupied slots and the policy's statistics update; returns the log-sum-exp. */
+static double policy_attend(const double *K, const double *V, double *s, double *q, int *n, int m, int d,
+                            const double *qv, double scale, int policy, double delta, double *out, int *quant_near) {
+  double *p = (double *)malloc(sizeof(double) * (size_t)(m > 0 ? m : 1));
+  const double lse = softmax_row(qv, K, m, d, scale, p);
   for (int c = 0; c < d; ++c) out[c] = 0.0;
   for (int j = 0; j < m; ++j) {
     for (int c = 0; c < d; ++c) out[c] += p[j] * V[(size_t)j * d + c];
@@ -882,6 +865,40 @@ void roco_oracle_policy_step_unit(double *K, double *V, double *s, double *q, in
     }
   }
   free(p);
+  return lse;
+}
+
+/* One decode step under one of the policies above, in either order of Fig. 1 / its alternative: EVICT_FIRST
+ * (evict, insert, attend) or ATTEND_FIRST (attend over the cache as it stands, update, then evict and insert).
+ * State: s = accumulated probability (Acc), n = Count for every policy; q = Acc^square, except under
+ * SCISSORHANDS, where it accumulates the quantised score (1 if the token's probability exceeds the average
+ * 1/live of this query, else 0), and under TOVA, where it holds the last query's probability.
+ * Local window (Sec. 4.2): tokens outside a window of the r most recent positions are evictable, i.e. pos < t - r
+ * with t the position of the incoming token.  Ties: (score asc, position asc).
+ * rnd: the random draw for RANDOM (victim = rnd mod live).  quant_near [B] (may be NULL): set to 1 where a
+ * SCISSORHANDS quantisation falls within delta (relative) of the average. */
+void roco_oracle_policy_step_unit(double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
+                                  int *t_next, int B, int d, const double *qv, const double *k_new,
+                                  const double *v_new, int policy, int r, int order, unsigned rnd, double scale,
+                                  double delta, int force_victim, double *out, double *lse, int *evicted_slot,
+                                  int *evicted_pos, int *choice, int *near_tie, int *quant_near) {
+  const int t = *t_next;
+  int slot, own = -1, near = 0;
+  *evicted_slot = -1;
+  *evicted_pos = -1;
+  if (order == ROCO_ORACLE_ATTEND_FIRST)
+    *lse = policy_attend(K, V, s, q, n, *live, d, qv, scale, policy, delta, out, quant_near);
+  if (*live == B) {
+    own = policy_pick(s, q, n, pos, B, policy, r, rnd, t, delta, &near);
+    slot = (force_victim >= 0 && force_victim < B && near) ? force_victim : own;
+    *evicted_slot = slot;
+    *evicted_pos = pos[slot];
+  } else {
+    slot = (*live)++;
+  }
+  insert_token(K, V, s, q, n, pos, slot, d, k_new, v_new, t);
+  if (order == ROCO_ORACLE_EVICT_FIRST)
+    *lse = policy_attend(K, V, s, q, n, *live, d, qv, scale, policy, delta, out, quant_near);
   *choice = own;
   *near_tie = near;
   *t_next = t + 1;
@@ -889,14 +906,15 @@ void roco_oracle_policy_step_unit(double *K, double *V, double *s, double *q, in
 
 void roco_oracle_policy_step_batch(int U, double *K, double *V, double *s, double *q, int *n, int *pos, int *live,
                                    int *t_next, int B, int d, const double *qv, const double *k_new,
-                                   const double *v_new, int policy, int r, const unsigned *rnd, double scale,
-                                   double delta, const int *force_victim, double *out, double *lse, int *evicted_slot,
+                                   const double *v_new, int policy, int r, int order, const unsigned *rnd,
+                                   double scale, double delta, const int *force_victim, double *out, double *lse,
+                                   int *evicted_slot,
                                    int *evicted_pos, int *choice, int *near_tie, int *quant_near) {
 #pragma omp parallel for schedule(dynamic, 1)
   for (int u = 0; u < U; ++u) {
     size_t kb = (size_t)u * B * d, sb = (size_t)u * B, vb = (size_t)u * d;
     roco_oracle_policy_step_unit(K + kb, V + kb, s + sb, q + sb, n + sb, pos + sb, live + u, t_next + u, B, d, qv + vb,
-                                 k_new + vb, v_new + vb, policy, r, rnd ? rnd[u] : 0u, scale, delta,
+                                 k_new + vb, v_new + vb, policy, r, order, rnd ? rnd[u] : 0u, scale, delta,
                                  force_victim ? force_victim[u] : -1, out + vb, lse + u, evicted_slot + u,
                                  evicted_pos + u, choice + u, near_tie + u, quant_near ? quant_near + sb : NULL);
   }
