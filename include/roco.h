@@ -214,10 +214,17 @@ typedef enum {
 roco_status roco_decode_step_policy(roco_cache *cache, const void *q, const void *k_new, const void *v_new,
                                     int policy, int r, const uint32_t *rnd, float scale, void *attn_out,
                                     float *lse_out, int32_t *evicted_slot, int32_t *evicted_pos, void *stream);
+/* The same in either order of a step (roco_step_order): under ROCO_ATTEND_FIRST the query attends over the cache as
+ * it stands, the policy's statistics are updated, and the eviction is decided on the updated statistics (the last
+ * score of ROCO_POLICY_TOVA is then this step's own query's). */
+roco_status roco_decode_step_policy_ordered(roco_cache *cache, const void *q, const void *k_new, const void *v_new,
+                                            int policy, int r, int step_order, const uint32_t *rnd, float scale,
+                                            void *attn_out, float *lse_out, int32_t *evicted_slot,
+                                            int32_t *evicted_pos, void *stream);
 
 /*
- * Block-wise evict-and-encode (Sec. 5.3 "Overhead", App. B: "the block size b controls the number of tokens being
- * freed and encoded within one eviction step"): b new tokens per unit in one pass over the cache.
+ * Block-wise evict-and-encode (Sec. 5.3 "Overhead", App. B, where one eviction step frees and encodes a block of
+ * b tokens): b new tokens per unit in one pass over the cache.
  *   1. live + b - B tokens (if positive) leave: the rule of Sec. 4.3 applied that many times on the statistics as
  *      they stand (frozen), each time on the tokens still cached.
  *   2. The new tokens (positions t_next .. t_next + b - 1) take, in order, the freed slots and -- while the buffer

@@ -30,7 +30,7 @@ EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes",
            "roco_consistency_step", "roco_selftest_read_stream", "roco_decode_host_pipeline_staging_bytes",
            "roco_decode_step_host_begin", "roco_decode_step_host_end", "roco_gqa_block_step",
            "roco_prefill_blockwise_gqa", "roco_prefill_with_output", "roco_decode_cluster_ranks",
-           "roco_decode_step_cluster")
+           "roco_decode_step_cluster", "roco_decode_step_policy_ordered")
 
 
 class RocoError(RuntimeError):
@@ -115,6 +115,10 @@ def lib() -> C.CDLL:
         L.roco_decode_step_cluster.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                                C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p,
                                                C.c_void_p, C.c_void_p, C.c_void_p]
+        L.roco_decode_step_policy_ordered.restype = C.c_int
+        L.roco_decode_step_policy_ordered.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p,
+                                                      C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_float, C.c_void_p,
+                                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.roco_decode_step_policy.restype = C.c_int
         L.roco_decode_step_policy.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                               C.c_int, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -326,12 +330,19 @@ def roco_decode_step_cluster(cache: Cache, q, k_new, v_new, r: int, attn_out, ev
 
 
 def roco_decode_step_policy(cache: Cache, q, k_new, v_new, policy: int, r: int, attn_out, evicted_slot,
-                            evicted_pos=None, lse_out=None, rnd=None, scale: Optional[float] = None):
-    """Decode step (evict, insert, attend) under one of the Table 1 policies; rnd: [S][G] int32/uint32 draws."""
+                            evicted_pos=None, lse_out=None, rnd=None, scale: Optional[float] = None,
+                            step_order: Optional[int] = None):
+    """Decode step under one of the Table 1 policies; rnd: [S][G] int32/uint32 draws.  step_order None: the entry
+    point with the order of Fig. 1 (evict, insert, attend); else roco_decode_step_policy_ordered."""
     scale = cache.d ** -0.5 if scale is None else scale
-    rc = lib().roco_decode_step_policy(C.byref(cache.c), _ptr(q), _ptr(k_new), _ptr(v_new), policy, r, _ptr(rnd),
-                                       scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot), _ptr(evicted_pos),
-                                       _stream())
+    if step_order is None:
+        rc = lib().roco_decode_step_policy(C.byref(cache.c), _ptr(q), _ptr(k_new), _ptr(v_new), policy, r, _ptr(rnd),
+                                           scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot),
+                                           _ptr(evicted_pos), _stream())
+    else:
+        rc = lib().roco_decode_step_policy_ordered(C.byref(cache.c), _ptr(q), _ptr(k_new), _ptr(v_new), policy, r,
+                                                   step_order, _ptr(rnd), scale, _ptr(attn_out), _ptr(lse_out),
+                                                   _ptr(evicted_slot), _ptr(evicted_pos), _stream())
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_decode_step_policy")
 

@@ -313,20 +313,29 @@ roco_status roco_decode_step_cluster(roco_cache *cache, const void *q, const voi
                                     lse_out, evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
 }
 
-roco_status roco_decode_step_policy(roco_cache *cache, const void *q, const void *k_new, const void *v_new,
-                                    int policy, int r, const uint32_t *rnd, float scale, void *attn_out,
-                                    float *lse_out, int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {
+roco_status roco_decode_step_policy_ordered(roco_cache *cache, const void *q, const void *k_new, const void *v_new,
+                                            int policy, int r, int step_order, const uint32_t *rnd, float scale,
+                                            void *attn_out, float *lse_out, int32_t *evicted_slot,
+                                            int32_t *evicted_pos, void *stream) {
   NvtxRange range("roco_decode_step_policy");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
   if (!q || !k_new || !v_new || !attn_out || !evicted_slot) return ROCO_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
   if (policy < ROCO_POLICY_ROCO || policy > ROCO_POLICY_MAS_WINDOW) return ROCO_ERR_INVALID_ARG;
+  if (step_order != ROCO_EVICT_FIRST && step_order != ROCO_ATTEND_FIRST) return ROCO_ERR_INVALID_ARG;
   if (r < 0 || r >= cache->B) return ROCO_ERR_INVALID_ARG;
   if (policy == ROCO_POLICY_RANDOM && !rnd) return ROCO_ERR_INVALID_ARG;
   if (policy == ROCO_POLICY_STREAMLLM && cache->B <= 4) return ROCO_ERR_INVALID_ARG;  // room for the four sinks
-  return launch_decode_step(*cache, q, k_new, v_new, r, ROCO_SCOPE_EXCLUDE_TOP_R, ROCO_EVICT_FIRST, policy, rnd, scale,
+  return launch_decode_step(*cache, q, k_new, v_new, r, ROCO_SCOPE_EXCLUDE_TOP_R, step_order, policy, rnd, scale,
                             attn_out, lse_out, evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
+}
+
+roco_status roco_decode_step_policy(roco_cache *cache, const void *q, const void *k_new, const void *v_new,
+                                    int policy, int r, const uint32_t *rnd, float scale, void *attn_out,
+                                    float *lse_out, int32_t *evicted_slot, int32_t *evicted_pos, void *stream) {
+  return roco_decode_step_policy_ordered(cache, q, k_new, v_new, policy, r, ROCO_EVICT_FIRST, rnd, scale, attn_out,
+                                         lse_out, evicted_slot, evicted_pos, stream);
 }
 
 roco_status roco_gqa_block_step(roco_cache *cache, const void *Q, const void *K_new, const void *V_new, int b,

@@ -311,8 +311,9 @@ class PolicyParity:
     """Steps the GPU cache and the oracle state together under one of the Table 1 policies."""
 
     def __init__(self, cache: R.Cache, st: oracle.State, units: Sequence[int], policy: int, r: int, tally: Tally,
-                 scale: Optional[float] = None):
+                 scale: Optional[float] = None, order: Optional[int] = None):
         self.cache, self.st, self.units, self.policy, self.r, self.tally = cache, st, list(units), policy, r, tally
+        self.order = order      # None: roco_decode_step_policy (evict, insert, attend); else the ordered entry point
         self.scale = cache.d ** -0.5 if scale is None else scale
         dev = cache.K.device
         self.out = torch.zeros(cache.S, cache.G, cache.d, dtype=cache.dtype, device=dev)
@@ -324,14 +325,15 @@ class PolicyParity:
     def step(self, q, k_new, v_new, rnd=None, check_state=False):
         c = self.cache
         R.roco_decode_step_policy(c, q, k_new, v_new, self.policy, self.r, self.out, self.ev_slot, self.ev_pos,
-                                  self.lse, rnd=rnd, scale=self.scale)
+                                  self.lse, rnd=rnd, scale=self.scale, step_order=self.order)
         torch.cuda.synchronize()
         g_slot = unit_view(self.ev_slot, self.units).cpu().numpy()
         g_pos = unit_view(self.ev_pos, self.units).cpu().numpy()
         rn = None if rnd is None else unit_view(rnd, self.units).cpu().numpy().astype(np.uint32)
         res, qn = oracle.policy_step(self.st, widen(unit_view(q, self.units)), widen(unit_view(k_new, self.units)),
                                      widen(unit_view(v_new, self.units)), self.policy, self.r, self.scale, rnd=rn,
-                                     delta=DELTA, force_victim=g_slot)
+                                     delta=DELTA, force_victim=g_slot,
+                                     order=R.ROCO_EVICT_FIRST if self.order is None else self.order)
         firm = ~res.near_tie
         np.testing.assert_array_equal(g_slot[firm], res.choice[firm], err_msg="victim differs outside the margin")
         self.tally.near_ties += int(res.near_tie.sum())
@@ -345,7 +347,10 @@ class PolicyParity:
             self.quant_fixups += int(qn.sum())
         g_out = widen(unit_view(self.out, self.units))
         assert np.abs(g_out - res.out).max() <= out_tol(c.dtype)
-        np.testing.assert_allclose(widen(unit_view(self.lse, self.units)), res.lse, rtol=0, atol=LSE_ATOL)
+        g_lse = widen(unit_view(self.lse, self.units))
+        fin = np.isfinite(res.lse)      # ATTEND_FIRST on an empty cache attends over nothing
+        np.testing.assert_allclose(g_lse[fin], res.lse[fin], rtol=0, atol=LSE_ATOL)
+        assert np.all(np.isneginf(g_lse[~fin]))
         if check_state:
             compare_state(c, self.st, self.units, f"after policy step {self.tally.steps}")
         return res

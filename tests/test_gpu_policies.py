@@ -16,13 +16,15 @@ POLICIES = [R.ROCO_POLICY_ROCO, R.ROCO_POLICY_RANDOM, R.ROCO_POLICY_RECENCY, R.R
 
 @pytest.mark.parametrize("policy", POLICIES)
 @pytest.mark.parametrize("dtype,d,B", [("bf16", 128, 200), ("f32", 64, 96)])
-def test_policy_decode_from_empty_cache(policy, dtype, d, B):
-    """From an empty cache: B fill steps, then 60 steps that each evict under the policy (sink-structured inputs)."""
+@pytest.mark.parametrize("order", [None, R.ROCO_EVICT_FIRST, R.ROCO_ATTEND_FIRST])
+def test_policy_decode_from_empty_cache(policy, dtype, d, B, order):
+    """From an empty cache: B fill steps, then 60 steps that each evict under the policy (sink-structured inputs),
+    through the entry point with the order of Fig. 1 and through the ordered one in both orders."""
     w = W.scaled(W.LLAMA7B_DECODE, S=2, layers=1, heads=3, d=d, dtype=dtype, B=B, r=B // 4)
     cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
     st = oracle.empty_state(w.U, B, d)
     tally = Tally()
-    par = PolicyParity(cache, st, range(w.U), policy, w.r, tally, scale=w.scale)
+    par = PolicyParity(cache, st, range(w.U), policy, w.r, tally, scale=w.scale, order=order)
     g = torch.Generator(device=DEV); g.manual_seed(policy)
     for i in range(B + 60):
         rnd = torch.randint(0, 2 ** 31 - 1, (w.S, w.G), generator=g, device=DEV, dtype=torch.int32)
