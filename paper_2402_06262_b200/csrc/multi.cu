@@ -115,9 +115,8 @@ struct PolicyView {
   int *posbuf;  // the unit's positions as they were before the step (with stats_full)
   uint64_t *stats_full;
   bool zn_by_consumers;
-  // Tensor-memory kernel only (else nullptr): per-slot sums over the queries of p and p^2 for the tokens that were
-  // cached before the step, formed by the consumer warps (which keep the probabilities to themselves there).
-  const float *ds, *dq;
+  // tcgen05 kernel only: the consumer threads own a slot each and apply the statistics update themselves
+  bool stats_by_consumers = false;
 };
 
 // The policy warps' part of a multi-query step: free `need` slots (Sec. 4.3 rule on frozen statistics), insert
@@ -521,6 +520,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     *((uint4 *)(const_cast<char *>(isv ? p.V : p.K) + unit_kv + (size_t)slot * kRowBytes) + cc) = val;
   }
 
+  if (v.stats_by_consumers) return;
   // statistics of Sec. 4.3 once the probabilities are in shared memory
   mbar_wait(v.p_ready, 0, abort_flag, p.status);
   // four slots per turn, their old statistics loaded before the first store (the arrays are updated in place,
@@ -545,17 +545,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
       const bool fresh = jn >= 0;
       float ds = 0.f, dq = 0.f;
       int dn;
-      if (v.ds && !fresh) {
-        if (nb == 1) {
-          ds = v.ds[j] / (float)M;  // one token, M heads: group-wise averaged attention score
-          dq = ds * ds;
-          dn = 1;
-        } else {
-          ds = v.ds[j];  // sums over the block's tokens of the (group-wise averaged) probability and its square
-          dq = v.dq[j];
-          dn = nb;
-        }
-      } else {
+      {
         // token t of the block (its `group` query heads) sees new token jn only if t >= jn; the statistics take
         // the group-wise averaged probability once per token (Sec. 5.3, App. A), which for one head is p itself
         const int t0 = fresh ? jn : 0, group = p.group;
@@ -637,7 +627,6 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_kernel(const MultiParam
     v.z = sm.z; v.Bp = Bp; v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok; v.sel = sm.sel;
     v.knew = sm.knew; v.vnew = sm.vnew; v.zn = sm.zn; v.qf = nullptr; v.pn = nullptr; v.ctl = sm.ctl;
     v.nbuf = nullptr; v.posbuf = nullptr; v.stats_full = nullptr; v.zn_by_consumers = false;
-    v.ds = nullptr; v.dq = nullptr;
     v.p_ready = sm.p_ready;
     v.policy_done = sm.policy_done;
     multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
@@ -949,7 +938,6 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
     v.knew = nullptr; v.vnew = sm.vnew; v.zn = sm.zn; v.qf = nullptr; v.pn = sm.pn; v.ctl = sm.ctl;
     v.nbuf = sm.nbuf; v.posbuf = sm.posbuf; v.stats_full = stats_by_tma ? sm.stats_full : nullptr;
     v.zn_by_consumers = true;
-    v.ds = nullptr; v.dq = nullptr;
     v.p_ready = sm.p_ready;
     v.policy_done = sm.policy_done;
     multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
@@ -1121,59 +1109,89 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
 }
 
 // ------------------------------------------------------------------------------------------------------------
-// Tensor-memory variant of the kernel above, for more than 8 queries (bf16, d = 128, B <= 2048).  There the M x B
-// fp32 score matrix (64 KiB at M = 16, B = 1024) is what keeps a second CTA off the SM, and with one CTA per SM
-// nothing overlaps the softmax and the selection.  Here every consumer thread keeps the scores its own MMAs
-// produced -- per 64-key tile: rows g and g + 8, keys 2 tq and 2 tq + 1 of the warp's 8 keys -- in four columns of
-// its tensor-memory lane (warps w and w + 4 share lanes and take different column halves), works on them in
-// place (row maxima and sums via quad shuffles and a small shared array), and leaves only what other threads need
-// in shared memory: the probabilities as bf16 for the output MMAs (half the size), and the per-slot sums over the
-// queries of p and p^2 for the statistics (in the key arrays, which the selection no longer needs by then).
+// tcgen05 variant for up to 16 queries (bf16, d = 128): both contractions of the step run on the fifth-generation
+// tensor cores, issued by one thread, with the key index on the accumulator's lanes:
+//
+//   scores   S^T[128 keys x 16 queries] = K_tile[128 x 128] Q^T        (A: streamed tile, B: the queries, K-major)
+//   output   O^T[128 dims x 16 queries] += V_tile^T[128 x 16 keys] P^T (A: streamed tile, B: probabilities, both
+//                                                                       with the M / N index contiguous)
+//
+// A consumer thread then owns one key of a tile with its 16 scores side by side in the columns of its
+// tensor-memory lane: the softmax works on them in place (the row maxima and sums are sums over lanes: one
+// transposing shuffle reduction per pass), the per-slot sums over the queries of p and p^2 that the statistics
+// need (Sec. 4.3) are sums inside a thread, and the 16 probabilities of a key are 32 contiguous bytes of the
+// operand P^T.  The consumer warps issue no MMA, no matrix load and no per-tile barrier; what they execute per
+// score is one maximum, two fused multiply-adds, two exponentials, the two statistics sums and half a conversion.
+// The new tokens' values enter through one more MMA (V_new as a 16-key tile), their scores through a small
+// warp-level MMA as before.
 
-struct MultiTmSmem {
+constexpr int kUmTile = 128;                    // keys per streamed tile
+constexpr int kUmTileBytes = kUmTile * 256;     // two 64-column halves of 16 KiB
+constexpr int kUmHalfBytes = kUmTileBytes / 2;
+constexpr int kUmStages = 2;
+constexpr int kUmMmaWarp = kMqPolicyWarp0 + kMqPolicyThreads / 32;
+constexpr int kUmThreads = (kUmMmaWarp + 1) * 32;
+constexpr int kUmBarStaged = 3;                 // consumers + MMA warp: the query operand is in shared memory
+constexpr int kUmPBlock = 16384;                // P^T of four tiles: 128 key rows of 128 bytes (4 x 16 queries)
+// kind::f16 instruction descriptors: fp32 accumulator, bf16 operands, M = 128, N = 16
+constexpr uint32_t kIdescUmS = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescUmO = kIdescUmS | (1u << 15) | (1u << 16);  // A and B with the M / N index contiguous
+
+struct MultiUmSmem {
   char *ring;
-  __nv_bfloat16 *pz;  // [16][Bp] probabilities, bf16, rows >= M zero; Bp = multi_tc_row_stride(B)
-  uint32_t *vkey;     // later: ds
-  float *mkey;        // later: dq
+  char *pbuf;  // P^T blocks; until the selection is done its first 16 Bp bytes hold vkey | mkey | nbuf | posbuf
+  uint32_t *vkey;
+  float *mkey;
   int *nbuf, *posbuf;
+  char *qv;    // 4 KiB: the queries (B operand of the score MMAs), afterwards V_new (A operand of the last MMA)
+  char *pn;    // 2 KiB: P^T of the new tokens, 16 key rows of 128 bytes
   signed char *newtok;
   SelectScratch *sel;
-  float *zn, *pn;
-  float *red;         // [8 warps][16 rows]
-  uint64_t *full, *empty, *p_ready, *policy_done, *stats_full;
+  float *zn;   // [M][nb] raw scores of the queries against the new tokens
+  float *red;  // [2][8 warps][16 queries]
+  uint64_t *full, *empty, *s_full, *p_ready, *o_full, *policy_done, *stats_full;
   uint32_t *tmem_base;
   int *ctl;
 };
 
-__host__ __device__ inline size_t multi_tm_smem_bytes(int B, int stages, int M, int nb) {
-  const size_t Bp = multi_tc_row_stride(B);
-  size_t b = (size_t)stages * kMqTile;
-  b += 16 * Bp * 2 + 4 * Bp * 4 + Bp;
-  b += sizeof(SelectScratch);
-  b += 2 * (size_t)M * nb * 4 + kMqConsumerWarps * 16 * 4;
-  b = align_up(b, 8) + (2 * (size_t)stages + 4) * 8 + 64 * 4;
+__host__ __device__ inline size_t multi_um_pbuf_bytes(int B) {
+  const size_t tiles = ((size_t)B + kUmTile - 1) / kUmTile;
+  return (tiles + 3) / 4 * kUmPBlock;
+}
+
+__host__ __device__ inline size_t multi_um_smem_bytes(int B, int M, int nb) {
+  const size_t Bp = align_up((size_t)B, 64);
+  size_t b = (size_t)kUmStages * kUmTileBytes + multi_um_pbuf_bytes(B) + 4096 + 2048;
+  b += Bp + sizeof(SelectScratch);
+  b = align_up(b, 16) + (size_t)M * nb * 4 + 2 * kMqConsumerWarps * 16 * 4;
+  b = align_up(b, 8) + (2 * (size_t)kUmStages + 6) * 8 + 64 * 4;
   return b + 1024;
 }
 
-__device__ inline MultiTmSmem multi_tm_carve(char *raw, int B, int stages, int M, int nb) {
-  MultiTmSmem m;
+__device__ inline MultiUmSmem multi_um_carve(char *raw, int B, int M, int nb) {
+  MultiUmSmem m;
   char *p = smem_align(raw, 1024);
-  const size_t Bp = multi_tc_row_stride(B);
-  m.ring = p; p += (size_t)stages * kMqTile;
-  m.pz = (__nv_bfloat16 *)p; p += 16 * Bp * 2;
-  m.vkey = (uint32_t *)p; p += Bp * 4;
-  m.mkey = (float *)p; p += Bp * 4;
-  m.nbuf = (int *)p; p += Bp * 4;
-  m.posbuf = (int *)p; p += Bp * 4;
+  const size_t Bp = align_up((size_t)B, 64);
+  m.ring = p; p += (size_t)kUmStages * kUmTileBytes;
+  m.pbuf = p;
+  m.vkey = (uint32_t *)p;
+  m.mkey = (float *)(p + 4 * Bp);
+  m.nbuf = (int *)(p + 8 * Bp);
+  m.posbuf = (int *)(p + 12 * Bp);
+  p += multi_um_pbuf_bytes(B);
+  m.qv = p; p += 4096;
+  m.pn = p; p += 2048;
   m.newtok = (signed char *)p; p += Bp;
   m.sel = (SelectScratch *)p; p += sizeof(SelectScratch);
+  p = smem_align(p, 16);
   m.zn = (float *)p; p += (size_t)M * nb * 4;
-  m.pn = (float *)p; p += (size_t)M * nb * 4;
-  m.red = (float *)p; p += kMqConsumerWarps * 16 * 4;
+  m.red = (float *)p; p += 2 * kMqConsumerWarps * 16 * 4;
   p = smem_align(p, 8);
-  m.full = (uint64_t *)p; p += stages * 8;
-  m.empty = (uint64_t *)p; p += stages * 8;
+  m.full = (uint64_t *)p; p += kUmStages * 8;
+  m.empty = (uint64_t *)p; p += kUmStages * 8;
+  m.s_full = (uint64_t *)p; p += 8;
   m.p_ready = (uint64_t *)p; p += 8;
+  m.o_full = (uint64_t *)p; p += 8;
   m.policy_done = (uint64_t *)p; p += 8;
   m.stats_full = (uint64_t *)p; p += 8;
   m.tmem_base = (uint32_t *)p; p += 8;
@@ -1181,34 +1199,52 @@ __device__ inline MultiTmSmem multi_tm_carve(char *raw, int B, int stages, int M
   return m;
 }
 
-// Tensor-memory columns of one CTA: two halves (warps 0-3, warps 4-7) of four columns per tile, tiles rounded up
-// to a multiple of four (the in-place passes move 16 columns at a time), a power of two of at least 32.
-__host__ __device__ inline int multi_tm_cols(int B) {
-  const int tiles = ((B + 63) / 64 + 3) / 4 * 4;
+// Tensor-memory columns of one CTA: 16 per tile of 128 keys, a power of two of at least 32.  The output
+// accumulator takes the columns of tile 0 once the probabilities have been formed.
+__host__ __device__ inline int multi_um_cols(int B) {
+  const int tiles = (B + kUmTile - 1) / kUmTile;
   int c = 32;
-  while (c < 8 * tiles) c <<= 1;
+  while (c < 16 * tiles) c <<= 1;
   return c;
 }
 
-// kGroupedTokens: several tokens per step, each with several query heads (the statistics then take the heads'
-// mean per token); false: every query row is a token of its own, or all rows are the heads of one token.
-template <bool kGroupedTokens>
-__global__ void __launch_bounds__(kMqThreads, 2) multi_step_tm_kernel(const __grid_constant__ CUtensorMap mapK,
-                                                                      const __grid_constant__ CUtensorMap mapV,
-                                                                      const MultiParams p, int tmem_cols) {
+// v[i] (i = query) reduced over the 32 lanes; lane l returns the result for query l >> 1.  The exchange halves
+// the number of live values at every step (16 shuffles in all instead of 80).
+template <bool kMax>
+__device__ __forceinline__ float lanes_reduce16(float (&v)[16], int lane) {
+#pragma unroll
+  for (int step = 0; step < 4; ++step) {
+    const int w = 8 >> step, o = 16 >> step;
+    const bool up = (lane & o) != 0;
+#pragma unroll
+    for (int k = 0; k < w; ++k) {
+      const float send = up ? v[k] : v[k + w];
+      const float keep = up ? v[k + w] : v[k];
+      const float got = __shfl_xor_sync(0xffffffffu, send, o);
+      v[k] = kMax ? fmaxf(keep, got) : keep + got;
+    }
+  }
+  const float got = __shfl_xor_sync(0xffffffffu, v[0], 1);
+  return kMax ? fmaxf(v[0], got) : v[0] + got;
+}
+
+__global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __grid_constant__ CUtensorMap mapK,
+                                                                        const __grid_constant__ CUtensorMap mapV,
+                                                                        const MultiParams p, int tmem_cols) {
   using T = __nv_bfloat16;
-  constexpr int D = 128, kTileRows = 64;
+  constexpr int D = 128;
   extern __shared__ char mq_smem_raw[];
-  const int M = p.M, nb = p.nb, B = p.B, stages = p.stages;
-  const MultiTmSmem sm = multi_tm_carve(mq_smem_raw, B, stages, M, nb);
+  const int M = p.M, nb = p.nb, B = p.B;
+  const MultiUmSmem sm = multi_um_carve(mq_smem_raw, B, M, nb);
   volatile int *abort_flag = sm.ctl;
-  const size_t Bp = multi_tc_row_stride(B);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int u = blockIdx.x;
 
   if (tid == 0) {
-    for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kMqConsumerWarps); }
+    for (int i = 0; i < kUmStages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
+    mbar_init(sm.s_full, 1);
     mbar_init(sm.p_ready, kMqConsumerWarps);
+    mbar_init(sm.o_full, 1);
     mbar_init(sm.policy_done, 1);
     mbar_init(sm.stats_full, 1);
     sm.ctl[0] = 0;
@@ -1226,7 +1262,7 @@ __global__ void __launch_bounds__(kMqThreads, 2) multi_step_tm_kernel(const __gr
   int need = live0 + nb - B;
   if (need < 0) need = 0;
   const int live1 = live0 - need + nb;
-  const int n_tiles = (live1 + kTileRows - 1) / kTileRows;
+  const int n_tiles = (live1 + kUmTile - 1) / kUmTile;
   const bool stats_by_tma =
       need > 0 && (B & 3) == 0 &&
       ((reinterpret_cast<uintptr_t>(p.s) | reinterpret_cast<uintptr_t>(p.q) | reinterpret_cast<uintptr_t>(p.n) |
@@ -1247,293 +1283,317 @@ __global__ void __launch_bounds__(kMqThreads, 2) multi_step_tm_kernel(const __gr
         bulk_g2s(sm.posbuf, p.pos + (size_t)u * B, bytes, sm.stats_full);
       }
       for (int g = 0; g < 2 * n_tiles; ++g) {
-        const int st = g % stages;
-        if (g >= stages) mbar_wait(&sm.empty[st], ((g / stages) - 1) & 1, abort_flag, p.status);
+        const int st = g % kUmStages;
+        if (g >= kUmStages) mbar_wait(&sm.empty[st], ((g / kUmStages) - 1) & 1, abort_flag, p.status);
         const int it = (g < n_tiles) ? g : g - n_tiles;
         const CUtensorMap *map = (g < n_tiles) ? &mapK : &mapV;
-        char *dst = sm.ring + (size_t)st * kMqTile;
-        const int row = u * B + it * kTileRows;
-        mbar_expect_tx(&sm.full[st], kMqTile);
+        char *dst = sm.ring + (size_t)st * kUmTileBytes;
+        const int row = u * B + it * kUmTile;
+        mbar_expect_tx(&sm.full[st], kUmTileBytes);
         tma_load_2d(dst, map, 0, row, &sm.full[st]);
-        tma_load_2d(dst + 8192, map, 64, row, &sm.full[st]);
+        tma_load_2d(dst + kUmHalfBytes, map, 64, row, &sm.full[st]);
       }
     }
     return;
   }
 
-  if (warp >= kMqPolicyWarp0) {
+  if (warp >= kMqPolicyWarp0 && warp < kUmMmaWarp) {
     PolicyView v;
-    v.z = nullptr; v.Bp = Bp; v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok; v.sel = sm.sel;
-    v.knew = nullptr; v.vnew = nullptr; v.zn = sm.zn; v.qf = nullptr; v.pn = sm.pn; v.ctl = sm.ctl;
+    v.z = nullptr; v.Bp = align_up((size_t)B, 64); v.vkey = sm.vkey; v.mkey = sm.mkey; v.newtok = sm.newtok;
+    v.sel = sm.sel; v.knew = nullptr; v.vnew = nullptr; v.zn = sm.zn; v.qf = nullptr; v.pn = nullptr; v.ctl = sm.ctl;
     v.p_ready = sm.p_ready;
     v.policy_done = sm.policy_done;
     v.nbuf = sm.nbuf; v.posbuf = sm.posbuf; v.stats_full = stats_by_tma ? sm.stats_full : nullptr;
     v.zn_by_consumers = true;
-    v.ds = reinterpret_cast<const float *>(sm.vkey); v.dq = sm.mkey;
+    v.stats_by_consumers = true;
     multi_policy<T, D>(p, v, u, tid - kMqPolicyWarp0 * 32, live0, need, live1);
+    return;
+  }
+
+  if (warp == kUmMmaWarp) {
+    // ---------------------------------------------------------- MMA issue: one thread, the warp helps with zeroing
+    named_bar_sync(kUmBarStaged, kMqConsumers + 32);
+    for (int it = 0; it < n_tiles; ++it) {
+      const int st = it % kUmStages;
+      mbar_wait(&sm.full[st], (it / kUmStages) & 1, abort_flag, p.status);
+      tc_fence_after();
+      if (lane == 0) {
+        const char *tile = sm.ring + (size_t)st * kUmTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const int off = (kk >> 2) * kUmHalfBytes + (kk & 3) * 32, qoff = (kk >> 2) * 2048 + (kk & 3) * 32;
+          umma_bf16(tmem + (uint32_t)(16 * it), smem_desc_sw128(tile + off), smem_desc_sw128(sm.qv + qoff), kIdescUmS,
+                    kk > 0 ? 1u : 0u);
+        }
+        umma_commit(&sm.empty[st]);
+        if (it == n_tiles - 1) umma_commit(sm.s_full);
+      }
+      __syncwarp();
+    }
+    mbar_wait(sm.p_ready, 0, abort_flag, p.status);
+    tc_fence_after();
+    for (int it = 0; it < n_tiles; ++it) {
+      const int g = n_tiles + it;
+      const int st = g % kUmStages;
+      mbar_wait(&sm.full[st], (g / kUmStages) & 1, abort_flag, p.status);
+      char *tile = sm.ring + (size_t)st * kUmTileBytes;
+      if ((it + 1) * kUmTile > live0) {
+        // slots that were free before the step may hold anything (their probabilities are zero, but 0 x NaN)
+        const int r0 = live0 > it * kUmTile ? live0 - it * kUmTile : 0;
+        for (int w = lane; w < (kUmTile - r0) * 8; w += 32) {
+          *reinterpret_cast<uint4 *>(tile + (size_t)r0 * 128 + (size_t)w * 16) = make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4 *>(tile + kUmHalfBytes + (size_t)r0 * 128 + (size_t)w * 16) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        fence_async_smem();
+        __syncwarp();
+      }
+      tc_fence_after();
+      if (lane == 0) {
+        const char *pb = sm.pbuf + (size_t)(it >> 2) * kUmPBlock + (it & 3) * 32;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          umma_bf16(tmem, smem_desc_sw128_mn(tile + kk * 2048, kUmHalfBytes), smem_desc_sw128_mn(pb + kk * 2048, 16),
+                    kIdescUmO, (it > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(&sm.empty[st]);
+      }
+      __syncwarp();
+    }
+    if (lane == 0) {
+      umma_bf16(tmem, smem_desc_sw128_mn(sm.qv, 2048), smem_desc_sw128_mn(sm.pn, 16), kIdescUmO, 1u);
+      umma_commit(sm.o_full);
+    }
     return;
   }
 
   // -------------------------------------------------------------- consumers
   const float zscale = p.scale * kLog2e;
-  const int g = lane >> 2, tq = lane & 3;
-  const bool row_lo = g < M, row_hi = g + 8 < M;
   const int grp = p.group;
-  // this thread's lane of tensor memory and first column: tile `it` occupies the columns 4 it .. 4 it + 3 with
-  // (row g, key 2 tq), (g, 2 tq + 1), (g + 8, 2 tq), (g + 8, 2 tq + 1) of the warp's 8 keys of that tile
-  const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * (tmem_cols / 2));
-  uint32_t qa[8][4];
+  const T *Qu = (const T *)p.Q + (size_t)u * p.q_ustride * D;
+  // the queries as the K-major B operand of the score MMAs: row i = 128 bytes per 64-column half, 128-byte swizzle
   {
-    const T *Qu = (const T *)p.Q + (size_t)u * p.q_ustride * D;
-#pragma unroll
-    for (int s = 0; s < 8; ++s) {
-      const int k0 = s * 16 + tq * 2;
-      qa[s][0] = row_lo ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)g * D + k0) : 0u;
-      qa[s][1] = row_hi ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)(g + 8) * D + k0) : 0u;
-      qa[s][2] = row_lo ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)g * D + k0 + 8) : 0u;
-      qa[s][3] = row_hi ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)(g + 8) * D + k0 + 8) : 0u;
-    }
+    const int i = tid >> 4, chunk = tid & 15;
+    uint4 val = make_uint4(0u, 0u, 0u, 0u);
+    if (i < M) val = *(reinterpret_cast<const uint4 *>(Qu + (size_t)i * D) + chunk);
+    *reinterpret_cast<uint4 *>(sm.qv + (chunk >> 3) * 2048 + i * 128 + (((chunk & 7) ^ (i & 7)) << 4)) = val;
+    fence_async_smem();
   }
+  named_bar_sync(kUmBarStaged, kMqConsumers + 32);
 
-  // ---- scores: Z[16 x 8] = Q[16 x 128] K^T per warp and tile, into tensor memory (-inf where there is nothing)
-  for (int it = 0; it < n_tiles; ++it) {
-    const int st = it % stages;
-    mbar_wait(&sm.full[st], (it / stages) & 1, abort_flag, p.status);
-    const uint32_t tile = smem_u32(sm.ring + (size_t)st * kMqTile);
-    float c[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int sp = 0; sp < 4; ++sp) {
-      uint32_t kb[4];
-      ldmatrix_x4(tile + tile_chunk_offset(warp * 8 + (lane & 7), sp * 4 + (lane >> 3)), kb);
-      mma_bf16_16816(c, qa[2 * sp], kb[0], kb[1]);
-      mma_bf16_16816(c, qa[2 * sp + 1], kb[2], kb[3]);
-    }
-    const int j = it * kTileRows + warp * 8 + tq * 2;
-    const float ninf = -INFINITY;
-    tmem_st4(taddr + it * 4, __float_as_uint(row_lo && j < live1 ? c[0] * zscale : ninf),
-             __float_as_uint(row_lo && j + 1 < live1 ? c[1] * zscale : ninf),
-             __float_as_uint(row_hi && j < live1 ? c[2] * zscale : ninf),
-             __float_as_uint(row_hi && j + 1 < live1 ? c[3] * zscale : ninf));
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&sm.empty[st]);
-  }
-  // scores of the queries against the new tokens, from k_new: Zn[16 x 8] per warp, one warp per 8 new tokens
+  // raw scores of the queries against the new tokens, from k_new: Zn[16 x 8] per warp, one warp per 8 new tokens
   if (warp * 8 < nb) {
+    const int g = lane >> 2, tq = lane & 3;
+    const bool row_lo = g < M, row_hi = g + 8 < M;
     const T *Kn = (const T *)p.k_new + (size_t)u * p.kv_ustride * D;
     const int jn = warp * 8 + g;
     float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
       const int k0 = s * 16 + tq * 2;
+      uint32_t qa[4];
+      qa[0] = row_lo ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)g * D + k0) : 0u;
+      qa[1] = row_hi ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)(g + 8) * D + k0) : 0u;
+      qa[2] = row_lo ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)g * D + k0 + 8) : 0u;
+      qa[3] = row_hi ? *reinterpret_cast<const uint32_t *>(Qu + (size_t)(g + 8) * D + k0 + 8) : 0u;
       const uint32_t b0 = jn < nb ? *reinterpret_cast<const uint32_t *>(Kn + (size_t)jn * D + k0) : 0u;
       const uint32_t b1 = jn < nb ? *reinterpret_cast<const uint32_t *>(Kn + (size_t)jn * D + k0 + 8) : 0u;
-      mma_bf16_16816(c, qa[s], b0, b1);
+      mma_bf16_16816(c, qa, b0, b1);
     }
     const int j0 = warp * 8 + tq * 2;
     if (row_lo) {
-      if (j0 < nb) sm.zn[g * nb + j0] = c[0] * zscale;
-      if (j0 + 1 < nb) sm.zn[g * nb + j0 + 1] = c[1] * zscale;
+      if (j0 < nb) sm.zn[g * nb + j0] = c[0];
+      if (j0 + 1 < nb) sm.zn[g * nb + j0 + 1] = c[1];
     }
     if (row_hi) {
-      if (j0 < nb) sm.zn[(g + 8) * nb + j0] = c[2] * zscale;
-      if (j0 + 1 < nb) sm.zn[(g + 8) * nb + j0 + 1] = c[3] * zscale;
+      if (j0 < nb) sm.zn[(g + 8) * nb + j0] = c[2];
+      if (j0 + 1 < nb) sm.zn[(g + 8) * nb + j0 + 1] = c[3];
     }
   }
-  tmem_st_wait();
+
+  mbar_wait(sm.s_full, 0, abort_flag, p.status);
+  tc_fence_after();
+  // the score MMAs are done with the query operand: V_new takes its place as a 16-key tile with the dimension
+  // index contiguous (rows of new tokens that do not exist are zero), and the new tokens' P^T block is cleared
+  {
+    const T *Vn = (const T *)p.v_new + (size_t)u * p.kv_ustride * D;
+    const int jn = tid >> 4, chunk = tid & 15;
+    uint4 val = make_uint4(0u, 0u, 0u, 0u);
+    if (jn < nb) val = *(reinterpret_cast<const uint4 *>(Vn + (size_t)jn * D) + chunk);
+    *reinterpret_cast<uint4 *>(sm.qv + (chunk >> 3) * 2048 + jn * 128 + (((chunk & 7) ^ (jn & 7)) << 4)) = val;
+    if (tid < 128) *reinterpret_cast<uint4 *>(sm.pn + tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+  }
   mbar_wait(sm.policy_done, 0, abort_flag, p.status);
   named_bar_sync(kMqBarConsumers, kMqConsumers);
 
-  // The thread group that owns slot `slot`: its tile, the warp (8 keys of the tile each), the quad lane and the
-  // parity inside the key pair.  All lanes of the owning warp take part in the tensor-memory access.
-  auto for_new_tokens = [&](auto body) {
-    for (int jn = 0; jn < nb; ++jn) {
-      int slot = sm.ctl[1 + jn];
-      if (slot < 0 || slot >= B) slot = 0;
-      const int kk = slot & 63;
-      if (warp != (kk >> 3)) continue;
-      const uint32_t col = taddr + (uint32_t)((slot >> 6) * 4 + (kk & 1));
-      float a = __uint_as_float(tmem_ld1(col)), b = __uint_as_float(tmem_ld1(col + 2));
-      if (tq == ((kk & 7) >> 1)) body(jn, a, b);
-      tmem_st1(col, __float_as_uint(a));
-      tmem_st1(col + 2, __float_as_uint(b));
-    }
-    tmem_st_wait();
-  };
-  // the new tokens' scores replace whatever the stream brought for their slots (causal inside a block)
-  for_new_tokens([&](int jn, float &a, float &b) {
-    a = row_lo ? ((jn > g / grp) ? -INFINITY : sm.zn[g * nb + jn]) : -INFINITY;
-    b = row_hi ? ((jn > (g + 8) / grp) ? -INFINITY : sm.zn[(g + 8) * nb + jn]) : -INFINITY;
-  });
+  // this thread: key kl of the tiles wg, wg + 2, ...; tensor-memory lane kl, columns 16 it .. 16 it + 15
+  const int wq = warp & 3, wg = warp >> 2;
+  const int kl = wq * 32 + lane;
+  const uint32_t tlane = tmem + ((uint32_t)(wq * 32) << 16);
+  const int gshift = nb == 1 ? 4 : (grp >= 8 ? 3 : (grp >= 4 ? 2 : (grp >= 2 ? 1 : 0)));  // token of row i: i >> gshift
+  const uint32_t ninf = 0xff800000u;
 
-  // ---- softmax per query row, in place: maxima, exponentials and sums
-  auto rows_reduce = [&](float &lo, float &hi, bool is_max) {
-#pragma unroll
-    for (int o = 1; o <= 2; o <<= 1) {
-      const float ol = __shfl_xor_sync(0xffffffffu, lo, o), oh = __shfl_xor_sync(0xffffffffu, hi, o);
-      lo = is_max ? fmaxf(lo, ol) : lo + ol;
-      hi = is_max ? fmaxf(hi, oh) : hi + oh;
-    }
-    if (tq == 0) { sm.red[warp * 16 + g] = lo; sm.red[warp * 16 + g + 8] = hi; }
+  // over the 256 consumer threads; returns the result for query (lane & 15) and leaves all 16 in v
+  auto all_reduce16 = [&](float (&v)[16], bool is_max, float *red) {
+    const float x = is_max ? lanes_reduce16<true>(v, lane) : lanes_reduce16<false>(v, lane);
+    if (!(lane & 1)) red[warp * 16 + (lane >> 1)] = x;
     named_bar_sync(kMqBarConsumers, kMqConsumers);
-    lo = sm.red[g]; hi = sm.red[g + 8];
+    float acc = red[lane & 15];
 #pragma unroll
     for (int w = 1; w < kMqConsumerWarps; ++w) {
-      lo = is_max ? fmaxf(lo, sm.red[w * 16 + g]) : lo + sm.red[w * 16 + g];
-      hi = is_max ? fmaxf(hi, sm.red[w * 16 + g + 8]) : hi + sm.red[w * 16 + g + 8];
+      const float o = red[w * 16 + (lane & 15)];
+      acc = is_max ? fmaxf(acc, o) : acc + o;
     }
-    named_bar_sync(kMqBarConsumers, kMqConsumers);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __shfl_sync(0xffffffffu, acc, i);
+    return acc;
   };
-  float mlo = -INFINITY, mhi = -INFINITY;
-  for (int it0 = 0; it0 < n_tiles; it0 += 4) {
-    uint32_t r[16];
-    tmem_ld16(taddr + it0 * 4, r);
+
+  // ---- pass 1: masks and the new tokens' scores in place, row maxima
+  float a[16];
 #pragma unroll
-    for (int t = 0; t < 4; ++t) {
-      if (it0 + t < n_tiles) {
-        mlo = fmaxf(mlo, fmaxf(__uint_as_float(r[4 * t]), __uint_as_float(r[4 * t + 1])));
-        mhi = fmaxf(mhi, fmaxf(__uint_as_float(r[4 * t + 2]), __uint_as_float(r[4 * t + 3])));
+  for (int i = 0; i < 16; ++i) a[i] = -INFINITY;
+  for (int it = wg; it < n_tiles; it += 2) {
+    const int j = it * kUmTile + kl;
+    uint32_t r[16];
+    tmem_ld16(tlane + (uint32_t)(it * 16), r);
+    const int nt = j < live1 ? (int)sm.newtok[j] : -1;
+    if (__any_sync(0xffffffffu, nt >= 0 || j >= live1)) {
+      if (j >= live1) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) r[i] = ninf;
+      } else if (nt >= 0) {  // causal inside the block: the token of row i sees new token nt only if it is not later
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          r[i] = (i < M && nt <= (i >> gshift)) ? __float_as_uint(sm.zn[i * nb + nt]) : ninf;
       }
+      tmem_st16(tlane + (uint32_t)(it * 16), r);
     }
-  }
-  rows_reduce(mlo, mhi, true);
-  if (!(mlo > -INFINITY)) mlo = 0.f;  // a row that does not exist
-  if (!(mhi > -INFINITY)) mhi = 0.f;
-  float slo = 0.f, shi = 0.f;
-  for (int it0 = 0; it0 < n_tiles; it0 += 4) {
-    uint32_t r[16];
-    tmem_ld16(taddr + it0 * 4, r);
 #pragma unroll
-    for (int t = 0; t < 4; ++t) {
-      const bool in = it0 + t < n_tiles;
-      const float e0 = in ? exp2f(__uint_as_float(r[4 * t]) - mlo) : 0.f;
-      const float e1 = in ? exp2f(__uint_as_float(r[4 * t + 1]) - mlo) : 0.f;
-      const float e2 = in ? exp2f(__uint_as_float(r[4 * t + 2]) - mhi) : 0.f;
-      const float e3 = in ? exp2f(__uint_as_float(r[4 * t + 3]) - mhi) : 0.f;
-      slo += e0 + e1;
-      shi += e2 + e3;
-      r[4 * t] = __float_as_uint(e0); r[4 * t + 1] = __float_as_uint(e1);
-      r[4 * t + 2] = __float_as_uint(e2); r[4 * t + 3] = __float_as_uint(e3);
-    }
-    tmem_st16(taddr + it0 * 4, r);
+    for (int i = 0; i < 16; ++i) a[i] = fmaxf(a[i], __uint_as_float(r[i]));
   }
   tmem_st_wait();
-  rows_reduce(slo, shi, false);
-  const float inv_lo = row_lo ? 1.f / slo : 0.f, inv_hi = row_hi ? 1.f / shi : 0.f;
-  if (warp == 0 && tq == 0 && p.lse) {
-    if (row_lo) p.lse[(size_t)u * M + g] = (mlo + log2f(slo)) * kLn2;
-    if (row_hi) p.lse[(size_t)u * M + g + 8] = (mhi + log2f(shi)) * kLn2;
+  const float my_max = all_reduce16(a, true, sm.red);
+  // a[i] <- -(row maximum in the log2 domain); rows that do not exist hold zeros
+#pragma unroll
+  for (int i = 0; i < 16; ++i) a[i] = (a[i] > -INFINITY) ? -a[i] * zscale : 0.f;
+
+  // ---- pass 2: row sums of 2^(z - max)
+  float sums[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) sums[i] = 0.f;
+  for (int it = wg; it < n_tiles; it += 2) {
+    uint32_t r[16];
+    tmem_ld16(tlane + (uint32_t)(it * 16), r);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) sums[i] += ex2_approx(fmaf(__uint_as_float(r[i]), zscale, a[i]));
   }
-  // the new tokens' values come from v_new: their probabilities are set aside and cleared in place, so that the
-  // streamed V rows of those slots (possibly read before the overwrite) contribute nothing
-  for_new_tokens([&](int jn, float &a, float &b) {
-    if (row_lo) sm.pn[g * nb + jn] = a * inv_lo;
-    if (row_hi) sm.pn[(g + 8) * nb + jn] = b * inv_hi;
-    a = 0.f;
-    b = 0.f;
-  });
-  // probabilities: bf16 copy for the output MMAs; per-slot sums over the queries of p and p^2 for the statistics
+  const float my_sum = all_reduce16(sums, false, sm.red + kMqConsumerWarps * 16);
+  if (warp == 0 && lane < M && p.lse) {
+    const float mz = (my_max > -INFINITY) ? my_max * zscale : 0.f;
+    p.lse[(size_t)u * M + lane] = (mz + log2f(my_sum)) * kLn2;
+  }
+  // a[i] <- -(log2 of the row's normaliser): p = 2^(z * zscale + a[i]); rows that do not exist give p = 0
+#pragma unroll
+  for (int i = 0; i < 16; ++i) a[i] = (i < M) ? a[i] - __log2f(sums[i]) : -INFINITY;
+
+  // ---- pass 3: probabilities; P^T as bf16 operand blocks; the statistics of Sec. 4.3 for this thread's slots
   {
-    float *ds = reinterpret_cast<float *>(sm.vkey), *dq = sm.mkey;
-    for (int it0 = 0; it0 < n_tiles; it0 += 4) {
+    const size_t unit_st = (size_t)u * B;
+    int it = wg;
+    int j = it * kUmTile + kl;
+    // the old statistics of a tile's slot are loaded one tile ahead of their use
+    float s_old = 0.f, q_old = 0.f;
+    int n_old = 0;
+    if (it < n_tiles && j < live1) { s_old = p.s[unit_st + j]; q_old = p.q[unit_st + j]; n_old = p.n[unit_st + j]; }
+    for (; it < n_tiles; it += 2) {
+      j = it * kUmTile + kl;
+      const int jx = j + 2 * kUmTile;
+      float s_nx = 0.f, q_nx = 0.f;
+      int n_nx = 0;
+      if (it + 2 < n_tiles && jx < live1) { s_nx = p.s[unit_st + jx]; q_nx = p.q[unit_st + jx]; n_nx = p.n[unit_st + jx]; }
       uint32_t r[16];
-      tmem_ld16(taddr + it0 * 4, r);
+      tmem_ld16(tlane + (uint32_t)(it * 16), r);
+      float pr[16];
 #pragma unroll
-      for (int t = 0; t < 4; ++t) {
-        if (it0 + t < n_tiles) {  // uniform over the warp
-          const int j = (it0 + t) * kTileRows + warp * 8 + tq * 2;
-          const float p0 = __uint_as_float(r[4 * t]) * inv_lo, p1 = __uint_as_float(r[4 * t + 1]) * inv_lo;
-          const float p2 = __uint_as_float(r[4 * t + 2]) * inv_hi, p3 = __uint_as_float(r[4 * t + 3]) * inv_hi;
-          *reinterpret_cast<uint32_t *>(sm.pz + (size_t)g * Bp + j) = pack_bf16x2(p0, p1);
-          *reinterpret_cast<uint32_t *>(sm.pz + (size_t)(g + 8) * Bp + j) = pack_bf16x2(p2, p3);
-          // Rows g and g + 8 of this thread are query heads g % grp and (g + 8) % grp of two different tokens
-          // (grp divides 8 here; one token with all its heads when nb = 1, summed as a whole).  First the heads
-          // of a token are added up (the lanes that differ in the low bits of g), which gives the group-wise
-          // averaged probability of Sec. 5.3 / App. A; then p and p^2 of the tokens (the remaining bits).
-          float a0 = p0, a1 = p1, a2 = p2, a3 = p3;
-          if (kGroupedTokens) {
+      for (int i = 0; i < 16; ++i) pr[i] = ex2_approx(fmaf(__uint_as_float(r[i]), zscale, a[i]));
+      const int nt = j < live1 ? (int)sm.newtok[j] : -1;
+      // per token of the block the group-wise averaged probability (Sec. 5.3, App. A; one head: p itself), then its
+      // sum and sum of squares over the tokens; one token with all rows as its heads when nb = 1
+      float ds = 0.f, dq = 0.f;
+      if (nb == 1) {
+        float t = 0.f;
 #pragma unroll
-            for (int o = 4; o <= 16; o <<= 1) {
-              if (o < 4 * grp) {
-                a0 += __shfl_xor_sync(0xffffffffu, a0, o);
-                a1 += __shfl_xor_sync(0xffffffffu, a1, o);
-                a2 += __shfl_xor_sync(0xffffffffu, a2, o);
-                a3 += __shfl_xor_sync(0xffffffffu, a3, o);
-              }
-            }
-            const float ig = 1.f / (float)grp;
-            a0 *= ig; a1 *= ig; a2 *= ig; a3 *= ig;
-          }
-          float s0 = a0 + a2, s1 = a1 + a3, q0 = fmaf(a0, a0, a2 * a2), q1 = fmaf(a1, a1, a3 * a3);
-          const int o_first = kGroupedTokens ? 4 * grp : 4;
+        for (int i = 0; i < 16; ++i) t += pr[i];
+        ds = t / (float)M;
+        dq = ds * ds;
+      } else if (gshift == 0) {
 #pragma unroll
-          for (int o = 4; o <= 16; o <<= 1) {  // over the tokens (all eight row pairs when every row is a token)
-            if (o >= o_first) {
-              s0 += __shfl_xor_sync(0xffffffffu, s0, o);
-              s1 += __shfl_xor_sync(0xffffffffu, s1, o);
-              q0 += __shfl_xor_sync(0xffffffffu, q0, o);
-              q1 += __shfl_xor_sync(0xffffffffu, q1, o);
-            }
-          }
-          if (g == 0) { ds[j] = s0; ds[j + 1] = s1; dq[j] = q0; dq[j + 1] = q1; }
+        for (int i = 0; i < 16; ++i) { ds += pr[i]; dq = fmaf(pr[i], pr[i], dq); }
+      } else if (gshift == 1) {
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          const float m2 = (pr[2 * t] + pr[2 * t + 1]) * 0.5f;
+          ds += m2; dq = fmaf(m2, m2, dq);
+        }
+      } else if (gshift == 2) {
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const float m4 = ((pr[4 * t] + pr[4 * t + 1]) + (pr[4 * t + 2] + pr[4 * t + 3])) * 0.25f;
+          ds += m4; dq = fmaf(m4, m4, dq);
+        }
+      } else {
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          float m8 = 0.f;
+#pragma unroll
+          for (int h = 0; h < 8; ++h) m8 += pr[8 * t + h];
+          m8 *= 0.125f;
+          ds += m8; dq = fmaf(m8, m8, dq);
         }
       }
+      if (j < live1) {
+        const bool fresh = nt >= 0;
+        const int dn = nb == 1 ? 1 : (fresh ? nb - nt : nb);
+        p.s[unit_st + j] = (fresh ? 0.f : s_old) + ds;
+        p.q[unit_st + j] = (fresh ? 0.f : q_old) + dq;
+        p.n[unit_st + j] = (fresh ? 0 : n_old) + dn;
+      }
+      uint4 w0, w1;
+      w0.x = pack_bf16x2(pr[0], pr[1]); w0.y = pack_bf16x2(pr[2], pr[3]);
+      w0.z = pack_bf16x2(pr[4], pr[5]); w0.w = pack_bf16x2(pr[6], pr[7]);
+      w1.x = pack_bf16x2(pr[8], pr[9]); w1.y = pack_bf16x2(pr[10], pr[11]);
+      w1.z = pack_bf16x2(pr[12], pr[13]); w1.w = pack_bf16x2(pr[14], pr[15]);
+      if (nt >= 0) {
+        // a new token's value comes from V_new: its probabilities go to the new tokens' block, and the streamed
+        // row of its slot (possibly read before the overwrite) gets zeros
+        char *row = sm.pn + nt * 128;
+        *reinterpret_cast<uint4 *>(row + ((0 ^ (nt & 7)) << 4)) = w0;
+        *reinterpret_cast<uint4 *>(row + ((1 ^ (nt & 7)) << 4)) = w1;
+        w0 = make_uint4(0u, 0u, 0u, 0u);
+        w1 = w0;
+      }
+      char *row = sm.pbuf + (size_t)(it >> 2) * kUmPBlock + kl * 128;
+      const int c0 = 2 * (it & 3);
+      *reinterpret_cast<uint4 *>(row + ((c0 ^ (kl & 7)) << 4)) = w0;
+      *reinterpret_cast<uint4 *>(row + (((c0 + 1) ^ (kl & 7)) << 4)) = w1;
+      s_old = s_nx; q_old = q_nx; n_old = n_nx;
     }
   }
+  fence_async_smem();
+  tc_fence_before();
   __syncwarp();
   if (lane == 0) mbar_arrive(sm.p_ready);
-  named_bar_sync(kMqBarConsumers, kMqConsumers);
 
-  // ---- out[16 x 128] += P[16 x 64] V[64 x 128]: each warp owns 16 output columns
-  float o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-  for (int it = 0; it < n_tiles; ++it) {
-    const int gg = n_tiles + it;
-    const int st = gg % stages;
-    mbar_wait(&sm.full[st], (gg / stages) & 1, abort_flag, p.status);
-    const uint32_t tile = smem_u32(sm.ring + (size_t)st * kMqTile);
-    if ((it + 1) * kTileRows > live0) {  // slots that were free before the step may hold anything (0 x NaN)
-      const int r0 = live0 > it * kTileRows ? live0 - it * kTileRows : 0;
-      char *tp = sm.ring + (size_t)st * kMqTile;
-      for (int w = lane; w < (kTileRows - r0) * 2; w += 32) {
-        const int row = r0 + (w >> 1);
-        *reinterpret_cast<uint4 *>(tp + tile_chunk_offset(row, warp * 2 + (w & 1))) = make_uint4(0u, 0u, 0u, 0u);
-      }
-      __syncwarp();
-    }
+  // ---- output: O^T[dim][query] from tensor memory, this thread's dimension wq * 32 + lane, queries 8 wg .. 8 wg + 7
+  mbar_wait(sm.o_full, 0, abort_flag, p.status);
+  tc_fence_after();
+  {
+    uint32_t o[8];
+    tmem_ld8(tlane + (uint32_t)(8 * wg), o);
+    T *outp = (T *)p.out + (size_t)u * p.out_ustride * D + kl;
 #pragma unroll
-    for (int ks = 0; ks < 4; ++ks) {
-      const int j = it * kTileRows + ks * 16 + tq * 2;
-      uint32_t pa[4];
-      const __nv_bfloat16 *zl = sm.pz + (size_t)g * Bp + j, *zh = sm.pz + (size_t)(g + 8) * Bp + j;
-      pa[0] = *reinterpret_cast<const uint32_t *>(zl);
-      pa[1] = *reinterpret_cast<const uint32_t *>(zh);
-      pa[2] = *reinterpret_cast<const uint32_t *>(zl + 8);
-      pa[3] = *reinterpret_cast<const uint32_t *>(zh + 8);
-      uint32_t vb[4];
-      const int mi = lane >> 3;
-      ldmatrix_x4_trans(tile + tile_chunk_offset(ks * 16 + (mi & 1) * 8 + (lane & 7), warp * 2 + (mi >> 1)), vb);
-      mma_bf16_16816(o[0], pa, vb[0], vb[1]);
-      mma_bf16_16816(o[1], pa, vb[2], vb[3]);
-    }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&sm.empty[st]);
-  }
-  const T *Vn = (const T *)p.v_new + (size_t)u * p.kv_ustride * D;
-#pragma unroll
-  for (int nt = 0; nt < 2; ++nt) {
-    const int dcol = warp * 16 + nt * 8 + tq * 2;
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int qi = g + 8 * h;
-      if (qi < M) {
-        float o0 = o[nt][2 * h], o1 = o[nt][2 * h + 1];
-        for (int jn = 0; jn < nb; ++jn) {
-          const float pj = sm.pn[qi * nb + jn];
-          const __nv_bfloat162 vv = *reinterpret_cast<const __nv_bfloat162 *>(Vn + (size_t)jn * D + dcol);
-          o0 = fmaf(pj, __bfloat162float(vv.x), o0);
-          o1 = fmaf(pj, __bfloat162float(vv.y), o1);
-        }
-        *reinterpret_cast<uint32_t *>((T *)p.out + ((size_t)u * p.out_ustride + qi) * D + dcol) = pack_bf16x2(o0, o1);
-      }
+    for (int k = 0; k < 8; ++k) {
+      const int i = 8 * wg + k;
+      if (i < M) outp[(size_t)i * D] = __float2bfloat16(__uint_as_float(o[k]));
     }
   }
   tc_fence_before();
@@ -1549,13 +1609,9 @@ static int multi_tc_pick_stages(int B, int M, int nb) {
   return 0;
 }
 
-// Stages for the tensor-memory kernel: two CTAs per SM or nothing (with one it has no advantage).
-static int multi_tm_pick_stages(int B, int M, int nb) {
-  const size_t per_sm = 227 * 1024;
-  if (M <= 8 || multi_tm_cols(B) > 256) return 0;
-  for (int st = 4; st >= 3; --st)
-    if ((multi_tm_smem_bytes(B, st, M, nb) + 1024) * 2 <= per_sm) return st;
-  return 0;
+// The tcgen05 kernel runs with two CTAs per SM or not at all (with one, nothing covers a CTA's softmax phase).
+static bool multi_um_fits(int B, int M, int nb) {
+  return multi_um_cols(B) <= 256 && (multi_um_smem_bytes(B, M, nb) + 1024) * 2 <= (size_t)227 * 1024;
 }
 
 static int multi_pick_stages(int B, int d, int M, int nb) {
@@ -1599,25 +1655,23 @@ roco_status launch_multi_step(const roco_cache &c, int M, int nb, const void *Q,
   if (c.kv_dtype == ROCO_BF16 && c.d == 128 && (long long)U * c.B < 0x7fffffffLL) {
     // tensor-core path; falls through to the CUDA-core path if the tensor maps cannot be built
     CUtensorMap mapK, mapV;
-    // the tensor-memory kernel forms per-slot sums over all query rows, which is the statistic only when the rows
-    // are all tokens (one head) or all heads (one token)
-    // the tensor-memory kernel sums the heads of a token with lane shuffles: group sizes that divide 8
+    // the tcgen05 kernel averages the heads of a token inside a thread: group sizes that are powers of two, or one
+    // token with any number of heads
     const int grp_of = M / nb;
-    const bool tm_group = nb == 1 || grp_of == 1 || grp_of == 2 || grp_of == 4 || grp_of == 8;
-    const int tm_stages = tm_group ? multi_tm_pick_stages(c.B, M, nb) : 0;
-    p.stages = tm_stages > 0 ? tm_stages : multi_tc_pick_stages(c.B, M, nb);
+    const bool um_group = nb == 1 || grp_of == 1 || grp_of == 2 || grp_of == 4 || grp_of == 8;
+    if (M > 8 && um_group && multi_um_fits(c.B, M, nb) &&
+        make_tensor_map_rows128_bf16(&mapK, c.K, (unsigned long long)U * c.B, kUmTile) &&
+        make_tensor_map_rows128_bf16(&mapV, c.V, (unsigned long long)U * c.B, kUmTile)) {
+      const size_t smem = multi_um_smem_bytes(c.B, M, nb);
+      err = cudaFuncSetAttribute(multi_step_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (err != cudaSuccess) return ROCO_ERR_CUDA;
+      p.stages = kUmStages;
+      multi_step_umma_kernel<<<U, kUmThreads, smem, stream>>>(mapK, mapV, p, multi_um_cols(c.B));
+      return cudaGetLastError() == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
+    }
+    p.stages = multi_tc_pick_stages(c.B, M, nb);
     if (p.stages > 0 && make_tensor_map_rows128_bf16(&mapK, c.K, (unsigned long long)U * c.B, 64) &&
         make_tensor_map_rows128_bf16(&mapV, c.V, (unsigned long long)U * c.B, 64)) {
-      if (tm_stages > 0) {
-        const size_t smem = multi_tm_smem_bytes(c.B, p.stages, M, nb);
-        const bool grouped = nb > 1 && grp_of > 1;
-        err = grouped ? cudaFuncSetAttribute(multi_step_tm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                      : cudaFuncSetAttribute(multi_step_tm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (err != cudaSuccess) return ROCO_ERR_CUDA;
-        if (grouped) multi_step_tm_kernel<true><<<U, kMqThreads, smem, stream>>>(mapK, mapV, p, multi_tm_cols(c.B));
-        else multi_step_tm_kernel<false><<<U, kMqThreads, smem, stream>>>(mapK, mapV, p, multi_tm_cols(c.B));
-        return cudaGetLastError() == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
-      }
       const size_t smem = multi_tc_smem_bytes(c.B, p.stages, M, nb);
       err = cudaFuncSetAttribute(multi_step_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (err != cudaSuccess) return ROCO_ERR_CUDA;

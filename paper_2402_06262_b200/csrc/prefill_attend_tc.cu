@@ -44,16 +44,6 @@ constexpr int kAtPolyPairsPer8 = ROCO_ATTEND_POLY_PAIRS_PER_8;
 // (MN-major).  The tile sits as two halves of 64 dims, each 128 rows (keys) of 128 bytes, 128-byte swizzle:
 // 8-key groups are 1024 bytes apart (stride offset), the second 64-dim block is one half further (leading
 // offset).
-__device__ __forceinline__ uint64_t smem_desc_sw128_mn(const void *p) {
-  uint64_t d = 0;
-  d |= (uint64_t)((smem_u32(p) >> 4) & 0x3fffu);
-  d |= (uint64_t)(kTcHalfBytes >> 4) << 16;
-  d |= (uint64_t)(1024 >> 4) << 32;
-  d |= (uint64_t)1 << 46;
-  d |= (uint64_t)2 << 61;
-  return d;
-}
-
 constexpr uint32_t kIdescPV = kIdescBf16M128N128 | (1u << 16);  // B operand MN-major
 
 // D[tmem] (+)= A[tmem] * B[smem]: A is 128 lanes (rows) x 8 columns of packed bf16 pairs (K = 16)
@@ -73,7 +63,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return d;
 }
 
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 struct AtSmem {
   char *qt;     // two query tiles
@@ -226,7 +215,7 @@ __global__ void __launch_bounds__(kAtThreads, 1)
 #pragma unroll
               for (int kk = 0; kk < kTcTile / 16; ++kk)  // 16 keys per instruction
                 umma_bf16_ts(tmem + (uint32_t)(kAtColO + h * kTcTile), tmem + (uint32_t)(h * kTcTile + kk * 8),
-                             smem_desc_sw128_mn(vt + kk * 2048), kIdescPV, (kk > 0 || j - 1 > 0) ? 1u : 0u);
+                             smem_desc_sw128_mn(vt + kk * 2048, kTcHalfBytes), kIdescPV, (kk > 0 || j - 1 > 0) ? 1u : 0u);
               if (last_user(h, j - 1)) umma_commit(&sm.v_empty[vs]);
               if (!active(h, j)) umma_commit(&sm.o_full[h]);  // that was this query tile's last key tile
             }
