@@ -237,7 +237,9 @@ roco_status roco_decode_step_policy_ordered(roco_cache *cache, const void *q, co
  *   b                1..16, r + b <= B.  Under ROCO_SCOPE_LOWEST_R the scope refills after each of the step's
  *                    evictions (the token next in (variance, position) order is admitted before the next victim
  *                    is taken), all on the statistics as they stand before the step;
- *                    b * B floats of scores must fit in shared memory (else ROCO_ERR_UNSUPPORTED)
+ *                    the step's working set must fit on an SM, else ROCO_ERR_UNSUPPORTED: for bf16, d = 128 and 4 or
+ *                    more query rows B <= 3968 (scores in tensor memory), otherwise b * B floats of scores in
+ *                    shared memory
  *   attn_out         [S][G][b][d];   lse_out [S][G][b] or NULL
  *   evicted_slot     [S][G][b] freed slots in increasing order, padded with -1;  evicted_pos likewise, or NULL
  */
@@ -312,7 +314,7 @@ roco_status roco_prefill_blockwise_gqa(const void *Q, const void *K, const void 
  * averaged probability pbar = (1/group) sum_g p_g: Count += 1, Acc += pbar, Acc^square += pbar^2.
  *
  *   Q            [S][G][group][d]  (G counts key-value heads);  k_new, v_new [S][G][d]
- *   group        1..16 (group * B floats of scores must fit in shared memory)
+ *   group        1..16 (the working set must fit on an SM as for roco_block_step, with group query rows)
  *   attn_out     [S][G][group][d];  lse_out [S][G][group] or NULL;  evicted_slot, evicted_pos [S][G]
  */
 roco_status roco_gqa_decode_step(roco_cache *cache, const void *Q, const void *k_new, const void *v_new, int group,

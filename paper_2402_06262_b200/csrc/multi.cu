@@ -1128,12 +1128,11 @@ __global__ void __launch_bounds__(kMqThreads) multi_step_tc_kernel(const __grid_
 constexpr int kUmTile = 128;                    // keys per streamed tile
 constexpr int kUmTileBytes = kUmTile * 256;     // two 64-column halves of 16 KiB
 constexpr int kUmHalfBytes = kUmTileBytes / 2;
-constexpr int kUmStages = 2;
 constexpr int kUmMmaWarp = kMqPolicyWarp0 + kMqPolicyThreads / 32;
 constexpr int kUmThreads = (kUmMmaWarp + 1) * 32;
 constexpr int kUmBarStaged = 3;                 // consumers + MMA warp: the query operand is in shared memory
 constexpr int kUmBarDone = 4;                   // consumers + policy warps: nobody reads tensor memory any more
-constexpr int kUmMaxTiles = 16;                // tensor-memory columns / 16 at one CTA per SM
+constexpr int kUmMaxTiles = 31;                 // 16 tensor-memory columns each, and 16 for the output
 constexpr int kUmPBlock = 16384;                // P^T of four tiles: 128 key rows of 128 bytes (4 x 16 queries)
 // kind::f16 instruction descriptors: fp32 accumulator, bf16 operands, M = 128, N = 16
 constexpr uint32_t kIdescUmS = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
@@ -1161,20 +1160,20 @@ __host__ __device__ inline size_t multi_um_pbuf_bytes(int B) {
   return (tiles + 3) / 4 * kUmPBlock;
 }
 
-__host__ __device__ inline size_t multi_um_smem_bytes(int B, int M, int nb) {
+__host__ __device__ inline size_t multi_um_smem_bytes(int B, int stages, int nb) {
   const size_t Bp = align_up((size_t)B, 64);
-  size_t b = (size_t)kUmStages * kUmTileBytes + multi_um_pbuf_bytes(B) + 4096 + 2048;
+  size_t b = (size_t)stages * kUmTileBytes + multi_um_pbuf_bytes(B) + 4096 + 2048;
   b += Bp + sizeof(SelectScratch);
   b = align_up(b, 16) + (size_t)16 * nb * 4 + (2 * kMqConsumerWarps + 2) * 16 * 4;
-  b = align_up(b, 8) + (2 * (size_t)kUmStages + 6 + kUmMaxTiles) * 8 + 64 * 4;
+  b = align_up(b, 8) + (2 * (size_t)stages + 6 + kUmMaxTiles) * 8 + 64 * 4;
   return b + 1024;
 }
 
-__device__ inline MultiUmSmem multi_um_carve(char *raw, int B, int M, int nb) {
+__device__ inline MultiUmSmem multi_um_carve(char *raw, int B, int stages, int nb) {
   MultiUmSmem m;
   char *p = smem_align(raw, 1024);
   const size_t Bp = align_up((size_t)B, 64);
-  m.ring = p; p += (size_t)kUmStages * kUmTileBytes;
+  m.ring = p; p += (size_t)stages * kUmTileBytes;
   m.pbuf = p;
   m.vkey = (uint32_t *)p;
   m.mkey = (float *)(p + 4 * Bp);
@@ -1189,8 +1188,8 @@ __device__ inline MultiUmSmem multi_um_carve(char *raw, int B, int M, int nb) {
   m.zn = (float *)p; p += (size_t)16 * nb * 4;
   m.red = (float *)p; p += (2 * kMqConsumerWarps + 2) * 16 * 4;
   p = smem_align(p, 8);
-  m.full = (uint64_t *)p; p += kUmStages * 8;
-  m.empty = (uint64_t *)p; p += kUmStages * 8;
+  m.full = (uint64_t *)p; p += stages * 8;
+  m.empty = (uint64_t *)p; p += stages * 8;
   m.s_full = (uint64_t *)p; p += 8;
   m.p_tile = (uint64_t *)p; p += kUmMaxTiles * 8;
   m.d_ready = (uint64_t *)p; p += 8;
@@ -1237,14 +1236,14 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
   using T = __nv_bfloat16;
   constexpr int D = 128;
   extern __shared__ char mq_smem_raw[];
-  const int M = p.M, nb = p.nb, B = p.B;
-  const MultiUmSmem sm = multi_um_carve(mq_smem_raw, B, M, nb);
+  const int M = p.M, nb = p.nb, B = p.B, stages = p.stages;
+  const MultiUmSmem sm = multi_um_carve(mq_smem_raw, B, stages, nb);
   volatile int *abort_flag = sm.ctl;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int u = blockIdx.x;
 
   if (tid == 0) {
-    for (int i = 0; i < kUmStages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
+    for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
     mbar_init(sm.s_full, 1);
     for (int i = 0; i < kUmMaxTiles; ++i) mbar_init(&sm.p_tile[i], kMqConsumerWarps / 2);
     mbar_init(sm.d_ready, kMqConsumerWarps);
@@ -1288,8 +1287,8 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
         bulk_g2s(sm.posbuf, p.pos + (size_t)u * B, bytes, sm.stats_full);
       }
       for (int g = 0; g < 2 * n_tiles; ++g) {
-        const int st = g % kUmStages;
-        if (g >= kUmStages) mbar_wait(&sm.empty[st], ((g / kUmStages) - 1) & 1, abort_flag, p.status);
+        const int st = g % stages;
+        if (g >= stages) mbar_wait(&sm.empty[st], ((g / stages) - 1) & 1, abort_flag, p.status);
         const int it = (g < n_tiles) ? g : g - n_tiles;
         const CUtensorMap *map = (g < n_tiles) ? &mapK : &mapV;
         char *dst = sm.ring + (size_t)st * kUmTileBytes;
@@ -1356,8 +1355,8 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
     // ---------------------------------------------------------- MMA issue: one thread, the warp helps with zeroing
     named_bar_sync(kUmBarStaged, kMqConsumers + 32);
     for (int it = 0; it < n_tiles; ++it) {
-      const int st = it % kUmStages;
-      mbar_wait(&sm.full[st], (it / kUmStages) & 1, abort_flag, p.status);
+      const int st = it % stages;
+      mbar_wait(&sm.full[st], (it / stages) & 1, abort_flag, p.status);
       tc_fence_after();
       if (lane == 0) {
         const char *tile = sm.ring + (size_t)st * kUmTileBytes;
@@ -1374,9 +1373,9 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
     }
     for (int it = 0; it < n_tiles; ++it) {
       const int g = n_tiles + it;
-      const int st = g % kUmStages;
+      const int st = g % stages;
       mbar_wait(&sm.p_tile[it], 0, abort_flag, p.status);  // this tile's P^T block
-      mbar_wait(&sm.full[st], (g / kUmStages) & 1, abort_flag, p.status);
+      mbar_wait(&sm.full[st], (g / stages) & 1, abort_flag, p.status);
       char *tile = sm.ring + (size_t)st * kUmTileBytes;
       if ((it + 1) * kUmTile > live0) {
         // slots that were free before the step may hold anything (their probabilities are zero, but 0 x NaN)
@@ -1675,9 +1674,22 @@ static int multi_tc_pick_stages(int B, int M, int nb) {
   return 0;
 }
 
-// The tcgen05 kernel runs with two CTAs per SM or not at all (with one, nothing covers a CTA's softmax phase).
-static bool multi_um_fits(int B, int M, int nb) {
-  return multi_um_cols(B) <= 256 && (multi_um_smem_bytes(B, M, nb) + 1024) * 2 <= (size_t)227 * 1024;
+// Ring stages of the tcgen05 kernel: two (of 32 KiB) where two CTAs then share an SM, which covers a CTA's softmax
+// phase with the other's stream; else one CTA per SM with as many stages as fit.  0: the budget does not fit.
+static int multi_um_pick_stages(int B, int nb) {
+  const size_t per_sm = 227 * 1024;
+  if (multi_um_cols(B) > 512) return 0;
+  if (multi_um_cols(B) <= 256 && (multi_um_smem_bytes(B, 2, nb) + 1024) * 2 <= per_sm) return 2;
+  for (int st = 4; st >= 2; --st)
+    if (multi_um_smem_bytes(B, st, nb) + 1024 <= per_sm) return st;
+  return 0;
+}
+
+// Row layouts the tcgen05 kernel takes: from 4 rows up (below that the warp-level kernel is as fast), the heads of
+// a token averaged inside a thread -- group sizes that are powers of two, or one token with any number of heads.
+static bool multi_um_rows(int M, int nb) {
+  const int grp = M / nb;
+  return M >= 4 && (nb == 1 || grp == 1 || grp == 2 || grp == 4 || grp == 8);
 }
 
 static int multi_pick_stages(int B, int d, int M, int nb) {
@@ -1700,7 +1712,8 @@ static cudaError_t launch_multi_t(MultiParams &p, int U, cudaStream_t stream) {
 int multi_max_queries() { return kMqMaxQ; }
 
 bool multi_fits(int B, int d, int M, int nb) {
-  return multi_pick_stages(B, d, M, nb) > 0 || (d == 128 && multi_tc_pick_stages(B, M, nb) > 0);
+  return multi_pick_stages(B, d, M, nb) > 0 || (d == 128 && multi_tc_pick_stages(B, M, nb) > 0) ||
+         (d == 128 && multi_um_rows(M, nb) && multi_um_pick_stages(B, nb) > 0);
 }
 
 roco_status launch_multi_step(const roco_cache &c, int M, int nb, const void *Q, const void *k_new,
@@ -1721,17 +1734,17 @@ roco_status launch_multi_step(const roco_cache &c, int M, int nb, const void *Q,
   if (c.kv_dtype == ROCO_BF16 && c.d == 128 && (long long)U * c.B < 0x7fffffffLL) {
     // tensor-core path; falls through to the CUDA-core path if the tensor maps cannot be built
     CUtensorMap mapK, mapV;
-    // the tcgen05 kernel averages the heads of a token inside a thread: group sizes that are powers of two, or one
-    // token with any number of heads
-    const int grp_of = M / nb;
-    const bool um_group = nb == 1 || grp_of == 1 || grp_of == 2 || grp_of == 4 || grp_of == 8;
-    if (M > 8 && um_group && multi_um_fits(c.B, M, nb) &&
+    const int um_stages = multi_um_rows(M, nb) ? multi_um_pick_stages(c.B, nb) : 0;
+    // with one CTA per SM either way, the tcgen05 kernel keeps more bytes in flight; with two of the warp-level
+    // kernel against one of this, the two win
+    const bool tc_two = (multi_tc_smem_bytes(c.B, 3, M, nb) + 1024) * 2 <= (size_t)227 * 1024;
+    if (um_stages > 0 && (um_stages == 2 || !tc_two) &&
         make_tensor_map_rows128_bf16(&mapK, c.K, (unsigned long long)U * c.B, kUmTile) &&
         make_tensor_map_rows128_bf16(&mapV, c.V, (unsigned long long)U * c.B, kUmTile)) {
-      const size_t smem = multi_um_smem_bytes(c.B, M, nb);
+      const size_t smem = multi_um_smem_bytes(c.B, um_stages, nb);
       err = cudaFuncSetAttribute(multi_step_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (err != cudaSuccess) return ROCO_ERR_CUDA;
-      p.stages = kUmStages;
+      p.stages = um_stages;
       multi_step_umma_kernel<<<U, kUmThreads, smem, stream>>>(mapK, mapV, p, multi_um_cols(c.B));
       return cudaGetLastError() == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
     }

@@ -81,6 +81,20 @@ def test_block_step_after_eviction_prefill_llama_shape():
     assert tally.decisions == 3 * 16 * w.U
 
 
+@pytest.mark.parametrize("B,b", [(2048, 16), (3000, 8), (3968, 16)])
+def test_block_step_large_budget(B, b):
+    """Budgets that leave room for one CTA per SM only (more ring stages, up to 31 tiles of 128 keys)."""
+    L = B + 300
+    w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=4, prompt_lo=L, prompt_hi=L, B=B, r=64)
+    tally = Tally()
+    cache, st = prefilled(w, L, tally, range(w.U))
+    par = BlockParity(cache, st, range(w.U), b, w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, tally, scale=w.scale)
+    for i in range(3):
+        par.step(*block_tokens(w, b * i, b, [L + b * i]), check_state=(i == 2))
+    assert R.roco_device_status(cache) == 0
+    assert tally.decisions == 3 * b * w.U
+
+
 def test_block_of_one_equals_decode_step_bitwise():
     w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=4, prompt_lo=200, prompt_hi=200, B=128, r=8)
     Q, K, V = prompt_tensors(w, 200)
