@@ -26,7 +26,7 @@ constexpr int kUmMmaWarp = kMqPolicyWarp0 + kMqPolicyThreads / 32;
 constexpr int kUmThreads = (kUmMmaWarp + 1) * 32;
 constexpr int kUmBarStaged = 3;                 // consumers + MMA warp: the query operand is in shared memory
 constexpr int kUmBarDone = 4;                   // consumers + policy warps: nobody reads tensor memory any more
-constexpr int kUmMaxTiles = 31;                 // 16 tensor-memory columns each, and 16 for the output
+constexpr int kUmMaxTiles = 32;                 // 16 tensor-memory columns each
 constexpr int kUmPBlock = 16384;                // P^T of four tiles: 128 key rows of 128 bytes (4 x 16 queries)
 // kind::f16 instruction descriptors: fp32 accumulator, bf16 operands, M = 128, N = 16
 constexpr uint32_t kIdescUmS = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
@@ -96,13 +96,19 @@ __device__ inline MultiUmSmem multi_um_carve(char *raw, int B, int stages, int n
 }
 
 // Tensor-memory columns of one CTA: 16 per tile of 128 keys and 16 for the output accumulator behind them, a
-// power of two of at least 32.
+// power of two of at least 32.  With 32 tiles (3968 < B <= 4096) all 512 columns hold scores: the output
+// accumulator then takes the columns of tile 0 once that tile's probabilities have been formed, and the per-slot
+// sums of tile 0, which would lie there, go to two columns of tile 30 (by then read for the last time, by the
+// same thread, or not used at all).
+__host__ __device__ inline bool multi_um_o_aliases(int B) { return (B + kUmTile - 1) / kUmTile == kUmMaxTiles; }
 __host__ __device__ inline int multi_um_cols(int B) {
   const int tiles = (B + kUmTile - 1) / kUmTile;
+  const int need = multi_um_o_aliases(B) ? 16 * tiles : 16 * tiles + 16;
   int c = 32;
-  while (c < 16 * tiles + 16) c <<= 1;
+  while (c < need) c <<= 1;
   return c;
 }
+constexpr int kUmSumsColOfTile0 = 16 * 30 + 2;
 
 // v[i] (i = query) reduced over the 32 lanes; lane l returns the result for query l >> 1.  The exchange halves
 // the number of live values at every step (16 shuffles in all instead of 80).
@@ -168,7 +174,8 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *sm.tmem_base;
-  const uint32_t tmem_o = tmem + (uint32_t)(16 * ((B + kUmTile - 1) / kUmTile));
+  const bool o_aliases = multi_um_o_aliases(B);
+  const uint32_t tmem_o = o_aliases ? tmem : tmem + (uint32_t)(16 * ((B + kUmTile - 1) / kUmTile));
 
   if (warp == kMqProducerWarp) {
     if (lane == 0) {
@@ -231,7 +238,7 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
         if (it0 + k < n_tiles) {  // uniform over the warp
           const int j = (it0 + k) * kUmTile + kq;
           uint32_t d2[2];
-          tmem_ld2(tl + (uint32_t)(16 * (it0 + k)), d2);
+          tmem_ld2(tl + (uint32_t)((o_aliases && it0 + k == 0) ? kUmSumsColOfTile0 : 16 * (it0 + k)), d2);
           if (nt[k] > -2) {
             p.s[unit_st + j] = so[k] + __uint_as_float(d2[0]);
             p.q[unit_st + j] = qo[k] + __uint_as_float(d2[1]);
@@ -268,7 +275,7 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
     for (int it = 0; it < n_tiles; ++it) {
       const int g = n_tiles + it;
       const int st = g % stages;
-      mbar_wait(&sm.p_tile[it], 0, abort_flag, p.status);  // this tile's P^T block
+      mbar_wait(&sm.p_tile[it], 0, abort_flag, p.status);  // this tile's P^T block (at it = 0 also: its columns are free)
       mbar_wait(&sm.full[st], (g / stages) & 1, abort_flag, p.status);
       char *tile = sm.ring + (size_t)st * kUmTileBytes;
       if ((it + 1) * kUmTile > live0) {
@@ -467,6 +474,7 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
     p.lse[(size_t)u * M + lane] = (mz + log2f(my_sum)) * kLn2;
   }
 
+  float ds_tile0 = 0.f, dq_tile0 = 0.f;
   // ---- pass 3: probabilities; P^T as bf16 operand blocks, tile by tile (the output MMAs of a tile start as soon
   // as its block is complete); the statistics of Sec. 4.3 for this thread's slots
   for (int it = wg; it < n_tiles; it += 2) {
@@ -535,8 +543,11 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
         ds += m8; dq = fmaf(m8, m8, dq);
       }
     }
-    tmem_st2(tlane + (uint32_t)(it * 16), __float_as_uint(ds), __float_as_uint(dq));  // for the policy warps
+    // for the policy warps
+    if (o_aliases && it == 0) { ds_tile0 = ds; dq_tile0 = dq; }
+    else tmem_st2(tlane + (uint32_t)(it * 16), __float_as_uint(ds), __float_as_uint(dq));
   }
+  if (o_aliases && wg == 0) tmem_st2(tlane + (uint32_t)kUmSumsColOfTile0, __float_as_uint(ds_tile0), __float_as_uint(dq_tile0));
   tmem_st_wait();
   tc_fence_before();
   __syncwarp();

@@ -81,9 +81,9 @@ def test_block_step_after_eviction_prefill_llama_shape():
     assert tally.decisions == 3 * 16 * w.U
 
 
-@pytest.mark.parametrize("B,b", [(2048, 16), (3000, 8), (3968, 16)])
+@pytest.mark.parametrize("B,b", [(2048, 16), (3000, 8), (3968, 16), (4000, 12), (4096, 16)])
 def test_block_step_large_budget(B, b):
-    """Budgets that leave room for one CTA per SM only (more ring stages, up to 31 tiles of 128 keys)."""
+    """Budgets that leave room for one CTA per SM only (more ring stages, up to 32 tiles of 128 keys; with 32 the output accumulator shares tensor-memory columns with the first tile)."""
     L = B + 300
     w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=4, prompt_lo=L, prompt_hi=L, B=B, r=64)
     tally = Tally()
