@@ -119,7 +119,9 @@ __device__ __forceinline__ float consumers_sum(float v, float *red, int tid) {
   return r;
 }
 
-template <typename T, int D, int TILE>
+// kEvictFirst: the order of the step (Fig. 1: evict, insert, attend; or attend, update, then evict and insert) is a
+// compile-time choice, so that neither order carries the other's registers.
+template <typename T, int D, int TILE, bool kEvictFirst>
 __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const DecodeParams p) {
   constexpr int kRowBytes = D * (int)sizeof(T);
   constexpr int kLanesPerRow = kRowBytes / 16;
@@ -156,15 +158,15 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
     live0 = live0 < 0 ? 0 : B;
   }
   const bool full = (live0 == B);
-  const bool evict_first = (p.order == ROCO_EVICT_FIRST);
+  constexpr bool evict_first = kEvictFirst;
   const int live_att = evict_first ? (full ? B : live0 + 1) : live0;  // slots the query attends over
   const int live_new = full ? B : live0 + 1;
   const int n_tiles = (live_att + kTileRows - 1) / kTileRows;
   // The statistics the selection reads are fetched by bulk copies issued ahead of the K tiles (plain loads would
-  // queue behind the tile stream for microseconds).  Only where the selection sees the statistics as they stand
-  // at the start of the step, and the unit's arrays start on 16-byte boundaries.
+  // queue behind the tile stream for microseconds).  Under ATTEND_FIRST the copies are brought up to date in shared
+  // memory once the probabilities are there.  Only where the unit's arrays start on 16-byte boundaries.
   const bool stats_staged =
-      p.stage_stats && full && evict_first && p.policy == ROCO_POLICY_ROCO && (B & 3) == 0 &&
+      p.stage_stats && full && p.policy == ROCO_POLICY_ROCO && (B & 3) == 0 &&
       ((reinterpret_cast<uintptr_t>(p.s) | reinterpret_cast<uintptr_t>(p.q) | reinterpret_cast<uintptr_t>(p.n) |
         reinterpret_cast<uintptr_t>(p.pos)) & 15) == 0;
   __syncthreads();
@@ -212,9 +214,11 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
       row_val = *((const uint4 *)((isv ? p.v_new : p.k_new) + (size_t)u * kRowBytes) + (isv ? c - kLanesPerRow : c));
     }
     named_bar_sync(kBarPolicy, kPolicyThreads);
+    uint32_t k_and = 0xffffffffu, k_or = 0u;
     // statistics of Sec. 4.3 for the slots the query attended over: Acc += p, Acc^square += p^2, Count += 1
-    // (a slot that has just received the new token starts from zero)
-    auto update_statistics = [&](int fresh_slot) {
+    // (a slot that has just received the new token starts from zero).  form_keys: the selection follows on the
+    // new values, so its keys are formed here instead of from a second round of loads.
+    auto update_statistics = [&](int fresh_slot, bool form_keys) {
       mbar_wait(sm.p_ready, 0, abort_flag, p.status);
       // four slots per turn: all loads are issued before the first store (the compiler cannot move a load of
       // one array above a store to another, and the arrays are read-modify-written in place)
@@ -242,12 +246,41 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
           if (p.policy == ROCO_POLICY_TOVA) q1 = pj;                                                       // LTAS
           p.q[unit_st + j] = q1;
           p.n[unit_st + j] = n0[k] + 1;
+          if (form_keys) {
+            const uint32_t vk = variance_key_fast(s0[k] + pj, q1, n0[k] + 1);
+            sm.mkey[j] = mean_fast(s0[k] + pj, n0[k] + 1);
+            sm.vkey[j] = vk;
+            k_and &= vk;
+            k_or |= vk;
+          }
         }
       }
     };
+    const bool keys_with_update = !evict_first && full && p.policy == ROCO_POLICY_ROCO;
     if (!evict_first) {  // select on the updated statistics
-      update_statistics(-1);
-      named_bar_sync(kBarPolicy, kPolicyThreads);
+      if (stats_staged) {
+        // the staged copies plus this step's probabilities: the new values go to global memory (stores only) and
+        // the selection's keys are formed from them in place, so nothing here waits for a reply from global memory
+        mbar_wait(sm.p_ready, 0, abort_flag, p.status);
+        mbar_wait(sm.stats_full, 0, abort_flag, p.status);
+#pragma unroll 4
+        for (int j = ptid; j < B; j += kPolicyThreads) {
+          const float pj = sm.z[j];
+          const float s1 = __uint_as_float(sm.vkey[j]) + pj, q1 = fmaf(pj, pj, sm.mkey[j]);
+          const int n1 = sm.nbuf[j] + 1;
+          p.s[unit_st + j] = s1;
+          p.q[unit_st + j] = q1;
+          p.n[unit_st + j] = n1;
+          const uint32_t vk = variance_key_fast(s1, q1, n1);
+          sm.mkey[j] = mean_fast(s1, n1);
+          sm.vkey[j] = vk;
+          k_and &= vk;
+          k_or |= vk;
+        }
+      } else {
+        update_statistics(-1, keys_with_update);
+        named_bar_sync(kBarPolicy, kPolicyThreads);
+      }
     }
     int e = live0, ev_slot = -1, ev_pos = -1;
     if (full) {
@@ -257,18 +290,22 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
       if (p.policy == ROCO_POLICY_ROCO) {
         const int m = scope_size(B, p.r, p.scope_mode);
         if (stats_staged) {  // s, q, n sit in vkey, mkey, nbuf: form the keys in place
-          mbar_wait(sm.stats_full, 0, abort_flag, p.status);
-          uint32_t k_and = 0xffffffffu, k_or = 0u;
+          if (evict_first) {
+            mbar_wait(sm.stats_full, 0, abort_flag, p.status);
 #pragma unroll 4
-          for (int j = ptid; j < B; j += kPolicyThreads) {
-            const float sj = __uint_as_float(sm.vkey[j]);
-            const uint32_t vk = variance_key_fast(sj, sm.mkey[j], sm.nbuf[j]);
-            sm.mkey[j] = mean_fast(sj, sm.nbuf[j]);
-            sm.vkey[j] = vk;
-            k_and &= vk;
-            k_or |= vk;
+            for (int j = ptid; j < B; j += kPolicyThreads) {
+              const float sj = __uint_as_float(sm.vkey[j]);
+              const uint32_t vk = variance_key_fast(sj, sm.mkey[j], sm.nbuf[j]);
+              sm.mkey[j] = mean_fast(sj, sm.nbuf[j]);
+              sm.vkey[j] = vk;
+              k_and &= vk;
+              k_or |= vk;
+            }
           }
           e = group_select_from_keys(sm.posb, B, m, sm.vkey, sm.mkey, k_and, k_or, *sm.sel, ptid, kPolicyThreads,
+                                     kBarPolicy);
+        } else if (keys_with_update) {
+          e = group_select_from_keys(gpos, B, m, sm.vkey, sm.mkey, k_and, k_or, *sm.sel, ptid, kPolicyThreads,
                                      kBarPolicy);
         } else {
           e = group_select_victim(gs, gq, gn, gpos, B, m, sm.vkey, sm.mkey, *sm.sel, ptid, kPolicyThreads,
@@ -326,7 +363,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
       mbar_arrive(sm.policy_done);
       if (p.ev_pos) p.ev_pos[u] = ev_pos;  // waits for the load of the old position: after the signal
     }
-    if (evict_first) update_statistics(e);
+    if (evict_first) update_statistics(e, false);
     return;
   }
 
@@ -468,10 +505,10 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
 template <typename T, int D, int TILE>
 static cudaError_t launch_decode_t(const DecodeParams &p, int U, cudaStream_t stream) {
   const size_t smem = decode_smem_bytes<TILE>(p.B, D, p.stages, p.stage_stats);
-  cudaError_t err = cudaFuncSetAttribute(decode_step_kernel<T, D, TILE>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  auto kernel = p.order == ROCO_EVICT_FIRST ? decode_step_kernel<T, D, TILE, true> : decode_step_kernel<T, D, TILE, false>;
+  cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
-  decode_step_kernel<T, D, TILE><<<U, kDecodeThreads, smem, stream>>>(p);
+  kernel<<<U, kDecodeThreads, smem, stream>>>(p);
   return cudaGetLastError();
 }
 
