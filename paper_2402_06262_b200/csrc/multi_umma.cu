@@ -110,13 +110,14 @@ __host__ __device__ inline int multi_um_cols(int B) {
 }
 constexpr int kUmSumsColOfTile0 = 16 * 30 + 2;
 
-// v[i] (i = query) reduced over the 32 lanes; lane l returns the result for query l >> 1.  The exchange halves
-// the number of live values at every step (16 shuffles in all instead of 80).
-template <bool kMax>
-__device__ __forceinline__ float lanes_reduce16(float (&v)[16], int lane) {
+// v[i] (i = query, N = 8 or 16 of them) reduced over the 32 lanes; lane l returns the result for query l / (32 / N).
+// The exchange halves the number of live values at every step (N shuffles in all instead of 5 N).
+template <bool kMax, int N>
+__device__ __forceinline__ float lanes_reduce(float (&v)[N], int lane) {
+  constexpr int kSteps = N == 16 ? 4 : 3;
 #pragma unroll
-  for (int step = 0; step < 4; ++step) {
-    const int w = 8 >> step, o = 16 >> step;
+  for (int step = 0; step < kSteps; ++step) {
+    const int w = N >> (step + 1), o = 16 >> step;
     const bool up = (lane & o) != 0;
 #pragma unroll
     for (int k = 0; k < w; ++k) {
@@ -126,10 +127,47 @@ __device__ __forceinline__ float lanes_reduce16(float (&v)[16], int lane) {
       v[k] = kMax ? fmaxf(keep, got) : keep + got;
     }
   }
-  const float got = __shfl_xor_sync(0xffffffffu, v[0], 1);
-  return kMax ? fmaxf(v[0], got) : v[0] + got;
+#pragma unroll
+  for (int o = 16 >> kSteps; o >= 1; o >>= 1) {
+    const float got = __shfl_xor_sync(0xffffffffu, v[0], o);
+    v[0] = kMax ? fmaxf(v[0], got) : v[0] + got;
+  }
+  return v[0];
 }
 
+// kQ consecutive columns of this thread's tensor-memory lane
+template <int kQ>
+__device__ __forceinline__ void tmem_ldq(uint32_t taddr, uint32_t (&r)[kQ]) {
+  if constexpr (kQ == 16) tmem_ld16(taddr, r);
+  else tmem_ld8(taddr, r);
+}
+template <int kQ>
+__device__ __forceinline__ void tmem_stq(uint32_t taddr, const uint32_t (&r)[kQ]) {
+  if constexpr (kQ == 16) tmem_st16(taddr, r);
+  else tmem_st8(taddr, r);
+}
+
+// Per token of the block (1 << GS query heads each) the group-wise averaged probability (Sec. 5.3, App. A; one
+// head: p itself); ds and dq receive its sum and sum of squares over the tokens.
+template <int kQ, int GS>
+__device__ __forceinline__ void token_sums(const float (&pr)[kQ], float &ds, float &dq) {
+  constexpr int G = 1 << GS;
+  if constexpr (G <= kQ) {
+#pragma unroll
+    for (int t = 0; t < kQ / G; ++t) {
+      float m = pr[t * G];
+#pragma unroll
+      for (int h = 1; h < G; ++h) m += pr[t * G + h];
+      m *= 1.f / (float)G;
+      ds += m;
+      dq = fmaf(m, m, dq);
+    }
+  }
+}
+
+// kQ: query columns the consumer threads work on (8 when the step has at most 8 query rows, else 16; the MMAs
+// always carry 16, the rows that do not exist being zero)
+template <int kQ>
 __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __grid_constant__ CUtensorMap mapK,
                                                                         const __grid_constant__ CUtensorMap mapV,
                                                                         const MultiParams p, int tmem_cols) {
@@ -373,21 +411,21 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
   const int kl = wq * 32 + lane;
   const uint32_t tlane = tmem + ((uint32_t)(wq * 32) << 16);
   const uint32_t ninf = 0xff800000u;
-  // over the 256 consumer threads; returns the result for query (lane & 15) and leaves in v the maxima of all 16
-  // queries, or the reciprocals of their sums (0 for rows that do not exist)
-  auto all_reduce16 = [&](float (&v)[16], bool is_max, float *red) {
-    const float x = is_max ? lanes_reduce16<true>(v, lane) : lanes_reduce16<false>(v, lane);
-    if (!(lane & 1)) red[warp * 16 + (lane >> 1)] = x;
+  // over the 256 consumer threads; returns the result for query (lane & (kQ - 1)) and leaves in v the maxima of
+  // all kQ queries, or the reciprocals of their sums (0 for rows that do not exist)
+  auto all_reduce = [&](float (&v)[kQ], bool is_max, float *red) {
+    const float x = is_max ? lanes_reduce<true, kQ>(v, lane) : lanes_reduce<false, kQ>(v, lane);
+    if ((lane & (32 / kQ - 1)) == 0) red[warp * kQ + lane / (32 / kQ)] = x;
     named_bar_sync(kMqBarConsumers, kMqConsumers);
-    float acc = red[lane & 15];
+    float acc = red[lane & (kQ - 1)];
 #pragma unroll
     for (int w = 1; w < kMqConsumerWarps; ++w) {
-      const float o = red[w * 16 + (lane & 15)];
+      const float o = red[w * kQ + (lane & (kQ - 1))];
       acc = is_max ? fmaxf(acc, o) : acc + o;
     }
-    const float give = is_max ? acc : ((lane & 15) < M ? 1.f / acc : 0.f);
+    const float give = is_max ? acc : ((lane & (kQ - 1)) < M ? 1.f / acc : 0.f);
 #pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __shfl_sync(0xffffffffu, give, i);
+    for (int i = 0; i < kQ; ++i) v[i] = __shfl_sync(0xffffffffu, give, i);
     return acc;
   };
 
@@ -404,29 +442,29 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
   // ---- pass 1, while the selection may still be running: row maxima over the slots that held a token before
   // the step.  The slots that the new tokens will take still count with the score of the token they held, which
   // only makes the maximum an upper bound (it is the stabiliser of the exponentials, nothing else).
-  float a[16];
+  float a[kQ];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) a[i] = -INFINITY;
+  for (int i = 0; i < kQ; ++i) a[i] = -INFINITY;
   for (int it = wg; it < n_tiles; it += 2) {
     const int j = it * kUmTile + kl;
-    uint32_t r[16];
-    tmem_ld16(tlane + (uint32_t)(it * 16), r);
+    uint32_t r[kQ];
+    tmem_ldq<kQ>(tlane + (uint32_t)(it * 16), r);
     const bool held = j < live0;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) a[i] = fmaxf(a[i], held ? __uint_as_float(r[i]) : -INFINITY);
+    for (int i = 0; i < kQ; ++i) a[i] = fmaxf(a[i], held ? __uint_as_float(r[i]) : -INFINITY);
   }
-  float my_max = all_reduce16(a, true, sm.red);  // its barrier also publishes zn, V_new and the cleared block
+  float my_max = all_reduce(a, true, sm.red);  // its barrier also publishes zn, V_new and the cleared block
   {
     // the new tokens' scores join the maxima
     const float *znmax = sm.red + 2 * kMqConsumerWarps * 16;
-    const float zm = fmaxf(znmax[lane & 15], znmax[16 + (lane & 15)]);
+    const float zm = fmaxf(znmax[lane & (kQ - 1)], znmax[16 + (lane & (kQ - 1))]);
     my_max = fmaxf(my_max, zm);
 #pragma unroll
-    for (int k = 0; k < 16; ++k) a[k] = fmaxf(a[k], __shfl_sync(0xffffffffu, zm, k));
+    for (int k = 0; k < kQ; ++k) a[k] = fmaxf(a[k], __shfl_sync(0xffffffffu, zm, k));
   }
   // a[i] <- -(row maximum in the log2 domain); rows that do not exist hold zeros
 #pragma unroll
-  for (int i = 0; i < 16; ++i) a[i] = (a[i] > -INFINITY) ? -a[i] * zscale : 0.f;
+  for (int i = 0; i < kQ; ++i) a[i] = (a[i] > -INFINITY) ? -a[i] * zscale : 0.f;
 
   // ---- the selection's result: masks and the new tokens' scores in place
   mbar_wait(sm.policy_done, 0, abort_flag, p.status);
@@ -434,42 +472,42 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
     const int j = it * kUmTile + kl;
     const int nt = j < live1 ? (int)sm.newtok[j] : -1;
     if (__any_sync(0xffffffffu, nt >= 0 || j >= live1)) {
-      uint32_t r[16];
-      tmem_ld16(tlane + (uint32_t)(it * 16), r);
+      uint32_t r[kQ];
+      tmem_ldq<kQ>(tlane + (uint32_t)(it * 16), r);
       if (j >= live1) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) r[i] = ninf;
+        for (int i = 0; i < kQ; ++i) r[i] = ninf;
       } else if (nt >= 0) {  // the new token's scores, -inf where the block's causal mask hides it
         const uint4 *zr = reinterpret_cast<const uint4 *>(sm.zn + nt * 16);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
+        for (int k = 0; k < kQ / 4; ++k) {
           const uint4 z4 = zr[k];
           r[4 * k] = z4.x; r[4 * k + 1] = z4.y; r[4 * k + 2] = z4.z; r[4 * k + 3] = z4.w;
         }
       }
-      tmem_st16(tlane + (uint32_t)(it * 16), r);
+      tmem_stq<kQ>(tlane + (uint32_t)(it * 16), r);
     }
   }
   tmem_st_wait();
 
   // ---- pass 2: e = 2^(z - max) in place, row sums
-  float sums[16];
+  float sums[kQ];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) sums[i] = 0.f;
+  for (int i = 0; i < kQ; ++i) sums[i] = 0.f;
   for (int it = wg; it < n_tiles; it += 2) {
-    uint32_t r[16];
-    tmem_ld16(tlane + (uint32_t)(it * 16), r);
+    uint32_t r[kQ];
+    tmem_ldq<kQ>(tlane + (uint32_t)(it * 16), r);
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
+    for (int i = 0; i < kQ; ++i) {
       const float e = ex2_approx(fmaf(__uint_as_float(r[i]), zscale, a[i]));
       sums[i] += e;
       r[i] = __float_as_uint(e);
     }
-    tmem_st16(tlane + (uint32_t)(it * 16), r);
+    tmem_stq<kQ>(tlane + (uint32_t)(it * 16), r);
   }
   tmem_st_wait();
-  const float my_sum = all_reduce16(sums, false, sm.red + kMqConsumerWarps * 16);
-  if (warp == 0 && lane < M && p.lse) {
+  const float my_sum = all_reduce(sums, false, sm.red + kMqConsumerWarps * 16);
+  if (warp == 0 && lane < kQ && lane < M && p.lse) {
     const float mz = (my_max > -INFINITY) ? my_max * zscale : 0.f;
     p.lse[(size_t)u * M + lane] = (mz + log2f(my_sum)) * kLn2;
   }
@@ -479,18 +517,22 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
   // as its block is complete); the statistics of Sec. 4.3 for this thread's slots
   for (int it = wg; it < n_tiles; it += 2) {
     const int j = it * kUmTile + kl;
-    uint32_t r[16];
-    tmem_ld16(tlane + (uint32_t)(it * 16), r);
-    float pr[16];
+    uint32_t r[kQ];
+    tmem_ldq<kQ>(tlane + (uint32_t)(it * 16), r);
+    float pr[kQ];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) pr[i] = __uint_as_float(r[i]) * sums[i];  // sums[] holds the reciprocals by now
+    for (int i = 0; i < kQ; ++i) pr[i] = __uint_as_float(r[i]) * sums[i];  // sums[] holds the reciprocals by now
     const int nt = j < live1 ? (int)sm.newtok[j] : -1;
     {
       uint4 w0, w1;
       w0.x = pack_bf16x2(pr[0], pr[1]); w0.y = pack_bf16x2(pr[2], pr[3]);
       w0.z = pack_bf16x2(pr[4], pr[5]); w0.w = pack_bf16x2(pr[6], pr[7]);
-      w1.x = pack_bf16x2(pr[8], pr[9]); w1.y = pack_bf16x2(pr[10], pr[11]);
-      w1.z = pack_bf16x2(pr[12], pr[13]); w1.w = pack_bf16x2(pr[14], pr[15]);
+      if constexpr (kQ == 16) {
+        w1.x = pack_bf16x2(pr[8], pr[9]); w1.y = pack_bf16x2(pr[10], pr[11]);
+        w1.z = pack_bf16x2(pr[12], pr[13]); w1.w = pack_bf16x2(pr[14], pr[15]);
+      } else {
+        w1 = make_uint4(0u, 0u, 0u, 0u);  // the operand carries 16 queries: the upper eight do not exist
+      }
       if (nt >= 0) {
         // a new token's value comes from V_new: its probabilities go to the new tokens' block, and the streamed
         // row of its slot (possibly read before the overwrite) gets zeros
@@ -512,36 +554,20 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
     // per token of the block the group-wise averaged probability (Sec. 5.3, App. A; one head: p itself), then its
     // sum and sum of squares over the tokens; one token with all rows as its heads when nb = 1
     float ds = 0.f, dq = 0.f;
-    if (nb == 1) {
+    if (nb == 1) {  // one token with all rows as its heads
       float t = 0.f;
 #pragma unroll
-      for (int i = 0; i < 16; ++i) t += pr[i];
+      for (int i = 0; i < kQ; ++i) t += pr[i];
       ds = t / (float)M;
       dq = ds * ds;
     } else if (gshift == 0) {
-#pragma unroll
-      for (int i = 0; i < 16; ++i) { ds += pr[i]; dq = fmaf(pr[i], pr[i], dq); }
+      token_sums<kQ, 0>(pr, ds, dq);
     } else if (gshift == 1) {
-#pragma unroll
-      for (int t = 0; t < 8; ++t) {
-        const float m2 = (pr[2 * t] + pr[2 * t + 1]) * 0.5f;
-        ds += m2; dq = fmaf(m2, m2, dq);
-      }
+      token_sums<kQ, 1>(pr, ds, dq);
     } else if (gshift == 2) {
-#pragma unroll
-      for (int t = 0; t < 4; ++t) {
-        const float m4 = ((pr[4 * t] + pr[4 * t + 1]) + (pr[4 * t + 2] + pr[4 * t + 3])) * 0.25f;
-        ds += m4; dq = fmaf(m4, m4, dq);
-      }
+      token_sums<kQ, 2>(pr, ds, dq);
     } else {
-#pragma unroll
-      for (int t = 0; t < 2; ++t) {
-        float m8 = 0.f;
-#pragma unroll
-        for (int h = 0; h < 8; ++h) m8 += pr[8 * t + h];
-        m8 *= 0.125f;
-        ds += m8; dq = fmaf(m8, m8, dq);
-      }
+      token_sums<kQ, 3>(pr, ds, dq);
     }
     // for the policy warps
     if (o_aliases && it == 0) { ds_tile0 = ds; dq_tile0 = dq; }
@@ -595,9 +621,10 @@ int launch_multi_step_umma(const MultiParams &p, const roco_cache &c, int U, cud
       !make_tensor_map_rows128_bf16(&mapV, c.V, (unsigned long long)U * c.B, kUmTile))
     return -1;
   const size_t smem = multi_um_smem_bytes(c.B, p.stages, p.nb);
-  if (cudaFuncSetAttribute(multi_step_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+  auto kernel = p.M <= 8 ? multi_step_umma_kernel<8> : multi_step_umma_kernel<16>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return ROCO_ERR_CUDA;
-  multi_step_umma_kernel<<<U, kUmThreads, smem, stream>>>(mapK, mapV, p, multi_um_cols(c.B));
+  kernel<<<U, kUmThreads, smem, stream>>>(mapK, mapV, p, multi_um_cols(c.B));
   return cudaGetLastError() == cudaSuccess ? ROCO_OK : ROCO_ERR_CUDA;
 }
 
