@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
   // queue behind the tile stream for microseconds).  Under ATTEND_FIRST the copies are brought up to date in shared
   // memory once the probabilities are there.  Only where the unit's arrays start on 16-byte boundaries.
   const bool stats_staged =
-      p.stage_stats && full && p.policy == ROCO_POLICY_ROCO && (B & 3) == 0 &&
+      p.stage_stats && full && p.policy != ROCO_POLICY_RANDOM && (B & 3) == 0 &&
       ((reinterpret_cast<uintptr_t>(p.s) | reinterpret_cast<uintptr_t>(p.q) | reinterpret_cast<uintptr_t>(p.n) |
         reinterpret_cast<uintptr_t>(p.pos)) & 15) == 0;
   __syncthreads();
@@ -265,17 +265,26 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
         mbar_wait(sm.stats_full, 0, abort_flag, p.status);
 #pragma unroll 4
         for (int j = ptid; j < B; j += kPolicyThreads) {
-          const float pj = sm.z[j];
-          const float s1 = __uint_as_float(sm.vkey[j]) + pj, q1 = fmaf(pj, pj, sm.mkey[j]);
+          const float pj = sm.z[j], q0 = sm.mkey[j];
+          const float s1 = __uint_as_float(sm.vkey[j]) + pj;
+          float q1 = fmaf(pj, pj, q0);
+          if (p.policy == ROCO_POLICY_SCISSORHANDS) q1 = q0 + (pj * (float)live_att > 1.f ? 1.f : 0.f);  // AQAS
+          if (p.policy == ROCO_POLICY_TOVA) q1 = pj;                                                    // LTAS
           const int n1 = sm.nbuf[j] + 1;
           p.s[unit_st + j] = s1;
           p.q[unit_st + j] = q1;
           p.n[unit_st + j] = n1;
-          const uint32_t vk = variance_key_fast(s1, q1, n1);
-          sm.mkey[j] = mean_fast(s1, n1);
-          sm.vkey[j] = vk;
-          k_and &= vk;
-          k_or |= vk;
+          if (p.policy == ROCO_POLICY_ROCO) {
+            const uint32_t vk = variance_key_fast(s1, q1, n1);
+            sm.mkey[j] = mean_fast(s1, n1);
+            sm.vkey[j] = vk;
+            k_and &= vk;
+            k_or |= vk;
+          } else {  // the other policies of Table 1 read the new values themselves
+            sm.vkey[j] = __float_as_uint(s1);
+            sm.mkey[j] = q1;
+            sm.nbuf[j] = n1;
+          }
         }
       } else {
         update_statistics(-1, keys_with_update);
@@ -317,19 +326,28 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_step_kernel(const Decod
         // Table 1: importance score (Sec. 4.1) and local window of the r most recent positions (Sec. 4.2)
         const int pol = p.policy, horizon = t_new - p.r;
         const bool windowed = pol == ROCO_POLICY_SCISSORHANDS || pol == ROCO_POLICY_H2O || pol == ROCO_POLICY_MAS_WINDOW;
+        // the statistics as the selection has to see them: the staged copies (brought up to date above under
+        // ATTEND_FIRST) where there are any, else global memory
+        if (stats_staged) {
+          if (evict_first) mbar_wait(sm.stats_full, 0, abort_flag, p.status);
+          else named_bar_sync(kBarPolicy, kPolicyThreads);
+        }
+        const float *ss = stats_staged ? reinterpret_cast<const float *>(sm.vkey) : gs;
+        const float *qq = stats_staged ? sm.mkey : gq;
+        const int *nn = stats_staged ? sm.nbuf : gn, *pp = stats_staged ? sm.posb : gpos;
         e = group_argmin(
             [&](int j) {
-              if (pol == ROCO_POLICY_H2O) return gs[j];
-              if (pol == ROCO_POLICY_SCISSORHANDS || pol == ROCO_POLICY_TOVA) return gq[j];
-              if (pol == ROCO_POLICY_MAS_WINDOW) return mean_fast(gs[j], gn[j]);
+              if (pol == ROCO_POLICY_H2O) return ss[j];
+              if (pol == ROCO_POLICY_SCISSORHANDS || pol == ROCO_POLICY_TOVA) return qq[j];
+              if (pol == ROCO_POLICY_MAS_WINDOW) return mean_fast(ss[j], nn[j]);
               return 0.f;  // recency, StreamLLM: the position alone decides
             },
             [&](int j) {
-              if (windowed) return gpos[j] < horizon;
-              if (pol == ROCO_POLICY_STREAMLLM) return gpos[j] >= 4;
+              if (windowed) return pp[j] < horizon;
+              if (pol == ROCO_POLICY_STREAMLLM) return pp[j] >= 4;
               return true;
             },
-            gpos, B, *sm.sel, ptid, kPolicyThreads, kBarPolicy);
+            pp, B, *sm.sel, ptid, kPolicyThreads, kBarPolicy);
       }
       if (e < 0) {
         if (ptid == 0) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
