@@ -202,10 +202,13 @@ __global__ void __launch_bounds__(kTcThreads, 2) prefill_tc_kernel(const __grid_
           if (PASS == 0) {
             // online softmax, one rescale per chunk
             float cmax = -INFINITY;
+            if (kMasked) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const bool ok = !kMasked || (col0 + c * 32 + i <= grow);
-              cmax = fmaxf(cmax, ok ? __uint_as_float(r[i]) : -INFINITY);
+              for (int i = 0; i < 32; ++i)
+                cmax = fmaxf(cmax, (col0 + c * 32 + i <= grow) ? __uint_as_float(r[i]) : -INFINITY);
+            } else {  // three-input maxima: two elements per instruction
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) cmax = max3(cmax, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
             }
             const float m_new = fmaxf(run0, cmax * zscale);
             if (m_new > -INFINITY) {
