@@ -334,6 +334,13 @@ roco_status roco_decode_step_split(roco_cache *cache, const void *q, const void 
                                    int scope_mode, int splits, float scale, void *attn_out, float *lse_out,
                                    int32_t *evicted_slot, int32_t *evicted_pos, void *workspace,
                                    size_t workspace_bytes, void *stream);
+/* The same in either order of a step (roco_step_order): under ROCO_ATTEND_FIRST the attention and merge launches
+ * run first, over the cache as it stands, and the selection launch last, on the updated statistics. */
+roco_status roco_decode_step_split_ordered(roco_cache *cache, const void *q, const void *k_new, const void *v_new,
+                                           int r, int scope_mode, int step_order, int splits, float scale,
+                                           void *attn_out, float *lse_out, int32_t *evicted_slot,
+                                           int32_t *evicted_pos, void *workspace, size_t workspace_bytes,
+                                           void *stream);
 
 /*
  * roco_decode_step (either step order, both scope readings) for calls with few units -- one layer of a small

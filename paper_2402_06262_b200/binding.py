@@ -30,7 +30,7 @@ EXPORTS = ("roco_version", "roco_status_string", "roco_prefill_workspace_bytes",
            "roco_consistency_step", "roco_selftest_read_stream", "roco_decode_host_pipeline_staging_bytes",
            "roco_decode_step_host_begin", "roco_decode_step_host_end", "roco_gqa_block_step",
            "roco_prefill_blockwise_gqa", "roco_prefill_with_output", "roco_decode_cluster_ranks",
-           "roco_decode_step_cluster", "roco_decode_step_policy_ordered")
+           "roco_decode_step_cluster", "roco_decode_step_policy_ordered", "roco_decode_step_split_ordered")
 
 
 class RocoError(RuntimeError):
@@ -105,6 +105,10 @@ def lib() -> C.CDLL:
                                              C.c_float, C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p]
         L.roco_decode_split_workspace_bytes.restype = C.c_size_t
         L.roco_decode_split_workspace_bytes.argtypes = [C.POINTER(roco_cache), C.c_int]
+        L.roco_decode_step_split_ordered.restype = C.c_int
+        L.roco_decode_step_split_ordered.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                                     C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p,
+                                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.roco_decode_step_split.restype = C.c_int
         L.roco_decode_step_split.argtypes = [C.POINTER(roco_cache), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                              C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -302,12 +306,19 @@ def roco_decode_split_workspace_bytes(cache: Cache, splits: int) -> int:
 
 def roco_decode_step_split(cache: Cache, q, k_new, v_new, r: int, splits: int, attn_out, evicted_slot, workspace,
                            evicted_pos=None, lse_out=None, scope_mode=ROCO_SCOPE_EXCLUDE_TOP_R,
-                           scale: Optional[float] = None):
-    """roco_decode_step (evict, insert, attend) with every unit's slots divided among `splits` CTAs."""
+                           scale: Optional[float] = None, step_order: Optional[int] = None):
+    """roco_decode_step with every unit's slots divided among `splits` CTAs.  step_order None: the entry point with
+    the order of Fig. 1 (evict, insert, attend); else roco_decode_step_split_ordered."""
     scale = cache.d ** -0.5 if scale is None else scale
-    rc = lib().roco_decode_step_split(C.byref(cache.c), _ptr(q), _ptr(k_new), _ptr(v_new), r, scope_mode, splits,
-                                      scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot), _ptr(evicted_pos),
-                                      _ptr(workspace), workspace.numel(), _stream())
+    if step_order is None:
+        rc = lib().roco_decode_step_split(C.byref(cache.c), _ptr(q), _ptr(k_new), _ptr(v_new), r, scope_mode, splits,
+                                          scale, _ptr(attn_out), _ptr(lse_out), _ptr(evicted_slot),
+                                          _ptr(evicted_pos), _ptr(workspace), workspace.numel(), _stream())
+    else:
+        rc = lib().roco_decode_step_split_ordered(C.byref(cache.c), _ptr(q), _ptr(k_new), _ptr(v_new), r, scope_mode,
+                                                  step_order, splits, scale, _ptr(attn_out), _ptr(lse_out),
+                                                  _ptr(evicted_slot), _ptr(evicted_pos), _ptr(workspace),
+                                                  workspace.numel(), _stream())
     if rc != ROCO_OK:
         raise RocoError(rc, "roco_decode_step_split")
 

@@ -251,6 +251,16 @@ roco_status roco_decode_step_split(roco_cache *cache, const void *q, const void 
                                    int scope_mode, int splits, float scale, void *attn_out, float *lse_out,
                                    int32_t *evicted_slot, int32_t *evicted_pos, void *workspace,
                                    size_t workspace_bytes, void *stream) {
+  return roco_decode_step_split_ordered(cache, q, k_new, v_new, r, scope_mode, ROCO_EVICT_FIRST, splits, scale,
+                                        attn_out, lse_out, evicted_slot, evicted_pos, workspace, workspace_bytes,
+                                        stream);
+}
+
+roco_status roco_decode_step_split_ordered(roco_cache *cache, const void *q, const void *k_new, const void *v_new,
+                                           int r, int scope_mode, int step_order, int splits, float scale,
+                                           void *attn_out, float *lse_out, int32_t *evicted_slot,
+                                           int32_t *evicted_pos, void *workspace, size_t workspace_bytes,
+                                           void *stream) {
   NvtxRange range("roco_decode_step_split");
   roco_status st = check_cache(cache);
   if (st != ROCO_OK) return st;
@@ -258,11 +268,12 @@ roco_status roco_decode_step_split(roco_cache *cache, const void *q, const void 
   if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
   if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
   if (splits < 1 || splits > 64) return ROCO_ERR_INVALID_ARG;
+  if (step_order != ROCO_EVICT_FIRST && step_order != ROCO_ATTEND_FIRST) return ROCO_ERR_INVALID_ARG;
   const size_t need = roco_decode_split_workspace_bytes(cache, splits);
   if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
     return ROCO_ERR_WORKSPACE;
-  return launch_decode_step_split(*cache, q, k_new, v_new, r, scope_mode, splits, scale, attn_out, lse_out,
-                                  evicted_slot, evicted_pos, workspace, static_cast<cudaStream_t>(stream));
+  return launch_decode_step_split(*cache, q, k_new, v_new, r, scope_mode, step_order, splits, scale, attn_out,
+                                  lse_out, evicted_slot, evicted_pos, workspace, static_cast<cudaStream_t>(stream));
 }
 
 int roco_decode_cluster_ranks(const roco_cache *cache) {

@@ -1,6 +1,7 @@
 // Decode step split over the cache slots, for calls with few units (one layer of a small batch): with one CTA per
 // unit such a call cannot fill the GPU, so each unit's slots are divided among `splits` CTAs.  Three launches on
-// one stream (order as Fig. 1: evict, insert, attend):
+// one stream (in the order of Fig. 1: evict, insert, attend; under ROCO_ATTEND_FIRST launches 2 and 3 come first, over
+// the cache as it stands, and launch 1 then selects on the updated statistics and inserts with empty ones):
 //   1. split_policy_kernel   one CTA per unit: scope + victim (Sec. 4.3), in-place overwrite with the new K/V;
 //   2. split_attend_kernel   one CTA per (unit, slot range): scores, local (max, sum), local sum of p*V; the
 //                            log2-domain scores and the partial results go to the caller's workspace;
@@ -31,7 +32,7 @@ struct SplitParams {
   char *out;
   float *lse;
   int *ev_slot, *ev_pos;
-  int B, r, scope_mode, splits;
+  int B, r, scope_mode, splits, order;
   float scale;
   // workspace
   float *zbuf;   // [U][B]        log2-domain scores
@@ -76,6 +77,11 @@ __global__ void __launch_bounds__(kSpPolicyThreads) split_policy_kernel(const Sp
     if (p.ev_pos) p.ev_pos[u] = ev_pos;
     p.live[u] = live0 == B ? B : live0 + 1;
     p.t_next[u] = t_new + 1;
+    if (p.order == ROCO_ATTEND_FIRST) {  // the new token was not attended over: its statistics start empty
+      p.s[unit_st + e] = 0.f;
+      p.q[unit_st + e] = 0.f;
+      p.n[unit_st + e] = 0;
+    }
   }
   if (tid >= 32 && tid < 32 + 2 * kLanesPerRow) {  // in-place overwrite, 16 bytes per thread
     const int c = tid - 32;
@@ -111,7 +117,7 @@ __global__ void __launch_bounds__(kSpThreads) split_attend_kernel(const SplitPar
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int c = blockIdx.x, u = blockIdx.y, B = p.B, splits = p.splits;
   const size_t unit_kv = (size_t)u * B * kRowBytes;
-  const int live = p.live[u];  // already incremented by the policy kernel: slots the query attends over
+  const int live = p.live[u];  // slots the query attends over (EVICT_FIRST: the policy kernel has added the new one)
   // slot range of this CTA: whole tiles
   const int tiles_total = (live + kTileRows - 1) / kTileRows;
   const int tiles_per = (tiles_total + splits - 1) / splits;
@@ -284,7 +290,7 @@ __global__ void __launch_bounds__(kSpMergeThreads) split_merge_kernel(const Spli
     Elem<T>::store((T *)p.out + (size_t)u * D + tid, o * inv);
   }
   // statistics of Sec. 4.3 from the saved scores and the merged log-sum-exp
-  const int e = p.slot_new[u];
+  const int e = p.order == ROCO_EVICT_FIRST ? p.slot_new[u] : -1;  // the slot whose statistics start from zero
 #pragma unroll 4
   for (int j = tid; j < live; j += kSpMergeThreads) {
     const float pj = exp2f(p.zbuf[unit_st + j] - M) * inv;
@@ -315,22 +321,23 @@ static cudaError_t launch_split_t(SplitParams &p, int U, cudaStream_t stream) {
   if (err == cudaSuccess)
     err = cudaFuncSetAttribute(split_attend_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
   if (err != cudaSuccess) return err;
-  split_policy_kernel<T, D><<<U, kSpPolicyThreads, smem1, stream>>>(p);
+  if (p.order == ROCO_EVICT_FIRST) split_policy_kernel<T, D><<<U, kSpPolicyThreads, smem1, stream>>>(p);
   split_attend_kernel<T, D><<<dim3(p.splits, U), kSpThreads, smem2, stream>>>(p);
   split_merge_kernel<T, D><<<U, kSpMergeThreads, 0, stream>>>(p);
+  if (p.order != ROCO_EVICT_FIRST) split_policy_kernel<T, D><<<U, kSpPolicyThreads, smem1, stream>>>(p);
   return cudaGetLastError();
 }
 
 roco_status launch_decode_step_split(const roco_cache &c, const void *q, const void *k_new, const void *v_new, int r,
-                                     int scope_mode, int splits, float scale, void *out, float *lse, int32_t *ev_slot,
-                                     int32_t *ev_pos, void *workspace, cudaStream_t stream) {
+                                     int scope_mode, int step_order, int splits, float scale, void *out, float *lse,
+                                     int32_t *ev_slot, int32_t *ev_pos, void *workspace, cudaStream_t stream) {
   SplitParams p;
   const int U = c.S * c.G;
   p.K = (const char *)c.K; p.V = (const char *)c.V;
   p.s = c.s; p.q = c.q; p.n = c.n; p.pos = c.pos; p.live = c.live; p.t_next = c.t_next; p.status = c.status;
   p.qv = (const char *)q; p.k_new = (const char *)k_new; p.v_new = (const char *)v_new;
   p.out = (char *)out; p.lse = lse; p.ev_slot = ev_slot; p.ev_pos = ev_pos;
-  p.B = c.B; p.r = r; p.scope_mode = scope_mode; p.splits = splits; p.scale = scale;
+  p.B = c.B; p.r = r; p.scope_mode = scope_mode; p.splits = splits; p.order = step_order; p.scale = scale;
   char *ws = (char *)workspace;
   p.zbuf = (float *)ws;
   ws += align_up((size_t)U * c.B * 4, 256);

@@ -16,8 +16,8 @@ roco_status launch_decode_step(const roco_cache &c, const void *q, const void *k
 // partial results and saved scores in `workspace` (decode_split_workspace_bytes).
 size_t decode_split_workspace_bytes(int U, int B, int d, int splits);
 roco_status launch_decode_step_split(const roco_cache &c, const void *q, const void *k_new, const void *v_new, int r,
-                                     int scope_mode, int splits, float scale, void *out, float *lse, int32_t *ev_slot,
-                                     int32_t *ev_pos, void *workspace, cudaStream_t stream);
+                                     int scope_mode, int step_order, int splits, float scale, void *out, float *lse,
+                                     int32_t *ev_slot, int32_t *ev_pos, void *workspace, cudaStream_t stream);
 
 // The same step (either order) with a thread-block cluster of `ranks` CTAs (2, 4 or 8) per unit that exchange
 // partial results through distributed shared memory; no workspace.  decode_cluster_ranks: the cluster size that

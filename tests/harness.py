@@ -158,7 +158,8 @@ class DecodeParity:
                                        scope_mode=self.mode, step_order=self.order, ranks=self.ranks, scale=self.scale)
         elif self.splits:
             R.roco_decode_step_split(c, q, k_new, v_new, self.r, self.splits, self.out, self.ev_slot, self.ws,
-                                     self.ev_pos, self.lse, scope_mode=self.mode, scale=self.scale)
+                                     self.ev_pos, self.lse, scope_mode=self.mode, scale=self.scale,
+                                     step_order=(None if self.order == R.ROCO_EVICT_FIRST else self.order))
         else:
             R.roco_decode_step(c, q, k_new, v_new, self.r, self.out, self.ev_slot, self.ev_pos, self.lse,
                                scope_mode=self.mode, step_order=self.order, scale=self.scale)

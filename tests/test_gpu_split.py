@@ -11,16 +11,17 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
+@pytest.mark.parametrize("order", [R.ROCO_EVICT_FIRST, R.ROCO_ATTEND_FIRST])
 @pytest.mark.parametrize("splits", [1, 2, 3, 8])
 @pytest.mark.parametrize("mode", [R.ROCO_SCOPE_EXCLUDE_TOP_R, R.ROCO_SCOPE_LOWEST_R])
 @pytest.mark.parametrize("dtype,d,B", [("bf16", 128, 300), ("f32", 64, 100)])
-def test_split_decode_from_empty_cache(splits, mode, dtype, d, B):
+def test_split_decode_from_empty_cache(splits, mode, dtype, d, B, order):
     """Fill from empty (ranges that are still empty for some CTAs), then evict; B is not a multiple of the tile."""
     w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=5, d=d, dtype=dtype, B=B, r=11)
     cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
     st = oracle.empty_state(w.U, B, d)
     tally = Tally()
-    par = DecodeParity(cache, st, range(w.U), w.r, mode, R.ROCO_EVICT_FIRST, tally, scale=w.scale, splits=splits)
+    par = DecodeParity(cache, st, range(w.U), w.r, mode, order, tally, scale=w.scale, splits=splits)
     for i in range(B + 40):
         par.step(*W.decode_tokens(w, i, [i], DEV), check_state=(i % 25 == 24) or i == B + 39)
     assert R.roco_device_status(cache) == 0 and tally.decisions == 40 * w.U
