@@ -44,22 +44,29 @@ struct MultiUmSmem {
   SelectScratch *sel;
   float *zn;   // [nb][16] raw scores of the queries (second index) against the new tokens
   float *red;  // [2][8 warps][16 queries], then [2][16]: row maxima of zn from the two warps that form it
-  uint64_t *full, *empty, *s_full, *p_tile, *d_ready, *o_full, *policy_done, *stats_full;
+  uint64_t *full, *empty, *s_full, *p_tile, *p_free, *d_ready, *o_full, *policy_done, *stats_full;
   uint32_t *tmem_base;
   int *ctl;
 };
 
+// The P^T buffer holds up to eight tiles' blocks (32 KiB) and is reused as a ring beyond that: a block is free again
+// once the output MMAs of its tile have completed.  Until the selection is done the same memory holds the staged
+// s, q, n and pos (16 bytes per slot), which sets its size for budgets above 2048.
 __host__ __device__ inline size_t multi_um_pbuf_bytes(int B) {
   const size_t tiles = ((size_t)B + kUmTile - 1) / kUmTile;
-  return (tiles + 3) / 4 * kUmPBlock;
+  const size_t all = (tiles + 3) / 4 * kUmPBlock, ring = all < 2 * (size_t)kUmPBlock ? all : 2 * (size_t)kUmPBlock;
+  const size_t stats = align_up(16 * align_up((size_t)B, 64), kUmPBlock);
+  return ring > stats ? ring : stats;
 }
+// tiles of P^T in flight at once: four or eight (a power of two, so that a tile's place is a mask of its index)
+__host__ __device__ inline int multi_um_ptiles(int B) { return B <= 4 * kUmTile ? 4 : 8; }
 
 __host__ __device__ inline size_t multi_um_smem_bytes(int B, int stages, int nb) {
   const size_t Bp = align_up((size_t)B, 64);
   size_t b = (size_t)stages * kUmTileBytes + multi_um_pbuf_bytes(B) + 4096 + 2048;
   b += Bp + sizeof(SelectScratch);
   b = align_up(b, 16) + (size_t)16 * nb * 4 + (2 * kMqConsumerWarps + 2) * 16 * 4;
-  b = align_up(b, 8) + (2 * (size_t)stages + 6 + kUmMaxTiles) * 8 + 64 * 4;
+  b = align_up(b, 8) + (2 * (size_t)stages + 6 + 2 * kUmMaxTiles) * 8 + 64 * 4;
   return b + 1024;
 }
 
@@ -86,6 +93,7 @@ __device__ inline MultiUmSmem multi_um_carve(char *raw, int B, int stages, int n
   m.empty = (uint64_t *)p; p += stages * 8;
   m.s_full = (uint64_t *)p; p += 8;
   m.p_tile = (uint64_t *)p; p += kUmMaxTiles * 8;
+  m.p_free = (uint64_t *)p; p += kUmMaxTiles * 8;
   m.d_ready = (uint64_t *)p; p += 8;
   m.o_full = (uint64_t *)p; p += 8;
   m.policy_done = (uint64_t *)p; p += 8;
@@ -96,11 +104,14 @@ __device__ inline MultiUmSmem multi_um_carve(char *raw, int B, int stages, int n
 }
 
 // Tensor-memory columns of one CTA: 16 per tile of 128 keys and 16 for the output accumulator behind them, a
-// power of two of at least 32.  With 32 tiles (3968 < B <= 4096) all 512 columns hold scores: the output
-// accumulator then takes the columns of tile 0 once that tile's probabilities have been formed, and the per-slot
-// sums of tile 0, which would lie there, go to two columns of tile 30 (by then read for the last time, by the
-// same thread, or not used at all).
-__host__ __device__ inline bool multi_um_o_aliases(int B) { return (B + kUmTile - 1) / kUmTile == kUmMaxTiles; }
+// power of two of at least 32.  With 16 or 32 tiles the scores alone fill 256 or 512 columns (what two CTAs per SM,
+// or one, can have): the output accumulator then takes the columns of tile 0 once that tile's probabilities have
+// been formed, and the per-slot sums of tile 0, which would lie there, go to two columns of the last even tile but
+// one (by then read for the last time, by the same thread, or not used at all).
+__host__ __device__ inline bool multi_um_o_aliases(int B) {
+  const int tiles = (B + kUmTile - 1) / kUmTile;
+  return tiles == 16 || tiles == 32;
+}
 __host__ __device__ inline int multi_um_cols(int B) {
   const int tiles = (B + kUmTile - 1) / kUmTile;
   const int need = multi_um_o_aliases(B) ? 16 * tiles : 16 * tiles + 16;
@@ -108,7 +119,7 @@ __host__ __device__ inline int multi_um_cols(int B) {
   while (c < need) c <<= 1;
   return c;
 }
-constexpr int kUmSumsColOfTile0 = 16 * 30 + 2;
+__host__ __device__ inline int multi_um_sums_col_of_tile0(int B) { return 16 * ((B + kUmTile - 1) / kUmTile - 2) + 2; }
 
 // v[i] (i = query, N = 8 or 16 of them) reduced over the 32 lanes; lane l returns the result for query l / (32 / N).
 // The exchange halves the number of live values at every step (N shuffles in all instead of 5 N).
@@ -166,8 +177,9 @@ __device__ __forceinline__ void token_sums(const float (&pr)[kQ], float &ds, flo
 }
 
 // kQ: query columns the consumer threads work on (8 when the step has at most 8 query rows, else 16; the MMAs
-// always carry 16, the rows that do not exist being zero)
-template <int kQ>
+// always carry 16, the rows that do not exist being zero).  kRing: the budget has more tiles than the P^T buffer
+// holds, so a tile's block is reused once the output MMAs of the tile that held it have completed.
+template <int kQ, bool kRing>
 __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __grid_constant__ CUtensorMap mapK,
                                                                         const __grid_constant__ CUtensorMap mapV,
                                                                         const MultiParams p, int tmem_cols) {
@@ -183,7 +195,7 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
   if (tid == 0) {
     for (int i = 0; i < stages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
     mbar_init(sm.s_full, 1);
-    for (int i = 0; i < kUmMaxTiles; ++i) mbar_init(&sm.p_tile[i], kMqConsumerWarps / 2);
+    for (int i = 0; i < kUmMaxTiles; ++i) { mbar_init(&sm.p_tile[i], kMqConsumerWarps / 2); mbar_init(&sm.p_free[i], 1); }
     mbar_init(sm.d_ready, kMqConsumerWarps);
     mbar_init(sm.o_full, 1);
     mbar_init(sm.policy_done, 1);
@@ -213,6 +225,7 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
   tc_fence_after();
   const uint32_t tmem = *sm.tmem_base;
   const bool o_aliases = multi_um_o_aliases(B);
+  const int ptiles = multi_um_ptiles(B), pshift = ptiles == 4 ? 2 : 3;
   const uint32_t tmem_o = o_aliases ? tmem : tmem + (uint32_t)(16 * ((B + kUmTile - 1) / kUmTile));
 
   if (warp == kMqProducerWarp) {
@@ -253,6 +266,8 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
     // The statistics of Sec. 4.3: the consumer that owns a slot leaves the slot's sums over the block's tokens of
     // the (group-wise averaged) probability and of its square in the first two columns of the slot's tile; the
     // four policy warps cover the four lane quarters of tensor memory.  Old values are loaded four tiles at a time.
+    // (Following the consumers group by group instead of waiting for all of them cost more in the consumers' pass
+    // than it saved here.)
     const int kq = (warp & 3) * 32 + lane;
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const size_t unit_st = (size_t)u * B;
@@ -276,7 +291,7 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
         if (it0 + k < n_tiles) {  // uniform over the warp
           const int j = (it0 + k) * kUmTile + kq;
           uint32_t d2[2];
-          tmem_ld2(tl + (uint32_t)((o_aliases && it0 + k == 0) ? kUmSumsColOfTile0 : 16 * (it0 + k)), d2);
+          tmem_ld2(tl + (uint32_t)((o_aliases && it0 + k == 0) ? multi_um_sums_col_of_tile0(B) : 16 * (it0 + k)), d2);
           if (nt[k] > -2) {
             p.s[unit_st + j] = so[k] + __uint_as_float(d2[0]);
             p.q[unit_st + j] = qo[k] + __uint_as_float(d2[1]);
@@ -328,12 +343,14 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
       }
       tc_fence_after();
       if (lane == 0) {
-        const char *pb = sm.pbuf + (size_t)(it >> 2) * kUmPBlock + (it & 3) * 32;
+        const int ps = kRing ? (it & (ptiles - 1)) : it;  // this tile's place in the P^T buffer
+        const char *pb = sm.pbuf + (size_t)(ps >> 2) * kUmPBlock + (ps & 3) * 32;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
           umma_bf16(tmem_o, smem_desc_sw128_mn(tile + kk * 2048, kUmHalfBytes), smem_desc_sw128_mn(pb + kk * 2048, 16),
                     kIdescUmO, (it > 0 || kk > 0) ? 1u : 0u);
         umma_commit(&sm.empty[st]);
+        if (kRing && it + ptiles < n_tiles) umma_commit(&sm.p_free[ps]);  // a later tile waits for this place
       }
       __syncwarp();
     }
@@ -542,8 +559,10 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
         w0 = make_uint4(0u, 0u, 0u, 0u);
         w1 = w0;
       }
-      char *row = sm.pbuf + (size_t)(it >> 2) * kUmPBlock + kl * 128;
-      const int c0 = 2 * (it & 3);
+      const int ps = kRing ? (it & (ptiles - 1)) : it;
+      if (kRing && it >= ptiles) mbar_wait(&sm.p_free[ps], ((it >> pshift) - 1) & 1, abort_flag, p.status);
+      char *row = sm.pbuf + (size_t)(ps >> 2) * kUmPBlock + kl * 128;
+      const int c0 = 2 * (ps & 3);
       *reinterpret_cast<uint4 *>(row + ((c0 ^ (kl & 7)) << 4)) = w0;
       *reinterpret_cast<uint4 *>(row + (((c0 + 1) ^ (kl & 7)) << 4)) = w1;
     }
@@ -573,7 +592,8 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
     if (o_aliases && it == 0) { ds_tile0 = ds; dq_tile0 = dq; }
     else tmem_st2(tlane + (uint32_t)(it * 16), __float_as_uint(ds), __float_as_uint(dq));
   }
-  if (o_aliases && wg == 0) tmem_st2(tlane + (uint32_t)kUmSumsColOfTile0, __float_as_uint(ds_tile0), __float_as_uint(dq_tile0));
+  if (o_aliases && wg == 0)
+    tmem_st2(tlane + (uint32_t)multi_um_sums_col_of_tile0(B), __float_as_uint(ds_tile0), __float_as_uint(dq_tile0));
   tmem_st_wait();
   tc_fence_before();
   __syncwarp();
@@ -621,7 +641,9 @@ int launch_multi_step_umma(const MultiParams &p, const roco_cache &c, int U, cud
       !make_tensor_map_rows128_bf16(&mapV, c.V, (unsigned long long)U * c.B, kUmTile))
     return -1;
   const size_t smem = multi_um_smem_bytes(c.B, p.stages, p.nb);
-  auto kernel = p.M <= 8 ? multi_step_umma_kernel<8> : multi_step_umma_kernel<16>;
+  const bool ring = (c.B + kUmTile - 1) / kUmTile > multi_um_ptiles(c.B);
+  auto kernel = p.M <= 8 ? (ring ? multi_step_umma_kernel<8, true> : multi_step_umma_kernel<8, false>)
+                         : (ring ? multi_step_umma_kernel<16, true> : multi_step_umma_kernel<16, false>);
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return ROCO_ERR_CUDA;
   kernel<<<U, kUmThreads, smem, stream>>>(mapK, mapV, p, multi_um_cols(c.B));
