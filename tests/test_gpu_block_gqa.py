@@ -7,7 +7,8 @@ import torch
 import oracle
 import paper_2402_06262_b200 as R
 import workloads as W
-from harness import BlockParity, DecodeParity, GqaBlockParity, GqaParity, Tally, prefill_parity, unit_view, widen
+from harness import (BlockParity, DecodeParity, GqaBlockParity, GqaParity, Tally, prefill_parity, state_from_cache, unit_view,
+                     widen)
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -230,6 +231,41 @@ def test_grouped_block_step_llama_shape():
     for i in range(3):
         par.step(*grouped_block_tokens(w, 4 * i, 4, 4, [1500 + 4 * i]), check_state=(i == 2))
     assert tally.decisions == 3 * 4 * w.U
+
+
+def test_block_steps_at_the_benchmark_size():
+    """The launch configuration the bench times: all 8192 units of the Llama-7B decode shape (B = 1024, d = 128,
+    bf16) in one call, b = 16 and then 4 tokens x 4 heads; sampled units (first, last, some between) follow the
+    oracle from the cache the prefill left, every unit obeys the invariants."""
+    w = W.LLAMA7B_DECODE
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    L = 1500
+    for s in range(w.S):
+        for g0 in range(0, w.G, 256):
+            Q, K, V = (t[None] for t in W.prompt_chunk(w, s, g0, g0 + 256, L, DEV))
+            sub = R.Cache(1, 256, w.B, w.d, w.torch_dtype, DEV)
+            R.roco_prefill(Q, K, V, [L], w.B, w.r, sub, scale=w.scale)
+            for name in ("K", "V", "s", "q", "n", "pos", "live", "t_next"):
+                getattr(cache, name)[s, g0:g0 + 256].copy_(getattr(sub, name)[0])
+    units = [0, 1, 777, 4095, 4096, 8190, 8191]
+    tally = Tally()
+    par = BlockParity(cache, state_from_cache(cache, units), units, 16, w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, tally,
+                      scale=w.scale)
+    t = L
+    for i in range(2):
+        par.step(*block_tokens(w, 16 * i, 16, [t] * w.S), check_state=(i == 1))
+        t += 16
+    assert tally.decisions == 2 * 16 * len(units)
+    gpar = GqaBlockParity(cache, state_from_cache(cache, units), units, 4, 4, w.r, tally, scale=w.scale)
+    for i in range(2):
+        gpar.step(*grouped_block_tokens(w, 100 + 4 * i, 4, 4, [t] * w.S), check_state=(i == 1))
+        t += 4
+    assert R.roco_device_status(cache) == 0
+    assert int(cache.live.min()) == w.B == int(cache.live.max())
+    assert int(cache.t_next.min()) == t == int(cache.t_next.max())
+    assert bool((cache.n == (t - cache.pos)).all())           # Count = age for every slot of every unit
+    srt = cache.pos.sort(-1).values
+    assert bool((srt[..., 1:] > srt[..., :-1]).all())          # live positions distinct
 
 
 def test_grouped_blockwise_prompt_encoding_equals_grouped_block_steps():
