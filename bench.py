@@ -364,7 +364,8 @@ def few_units_bench(R, cache, w, device, reps=6):
     decode workload, and one layer of a single long sequence (32 units, B = 8192).  Paths: one CTA per unit, the
     three-launch split, the one-launch cluster kernel, and a bare read of the same number of bytes.  Two timings
     each: a single launch between two events with L2 flushed before it (includes the launch and event overhead of a
-    lone call), and a sweep over 8 distinct caches back to back (every call still reads cold rows)."""
+    lone call), and a sweep over 8 distinct caches back to back (every call still reads cold rows); the sweep is also
+    timed as one replay of a CUDA graph that holds its 8 calls."""
     hbm_peak, _, which = peaks()
     elem = 2 if w.dtype == "bf16" else 4
     dt = w.torch_dtype
@@ -409,6 +410,22 @@ def few_units_bench(R, cache, w, device, reps=6):
             ts.append(e0.elapsed_time(e1) / len(fns))
         return statistics.median(ts[2:])
 
+    def timed_graph(fns):
+        """The same sweep captured once in a CUDA graph and replayed: what a decode loop pays per call when it does
+        not launch from the host every time."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for fn in fns:
+                fn()
+        ts = []
+        for _ in range(reps + 2):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); g.replay(); e1.record(); torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) / len(fns))
+        del g
+        return statistics.median(ts[2:])
+
     for label, cch, rr in ((f"{sub.U} units, B={sub.B}", sub, w.r), (f"{long_cache.U} units, B={long_cache.B}", long_cache, wl.r)):
         algb = algorithmic_bytes_per_unit_step(cch.B, cch.d, elem) * cch.U
         q1, k1, v1 = (torch.randn(cch.S, cch.G, cch.d, device=device, generator=gen).to(dt) for _ in range(3))
@@ -421,8 +438,10 @@ def few_units_bench(R, cache, w, device, reps=6):
             """make(cache) -> callable of one step on that cache."""
             iso = timed_cold(make(cch))
             sweep = timed_sweep([make(c) for c in layers])
+            graph = timed_graph([make(c) for c in layers])
             return {"path": name, "us_per_step": iso * 1e3, "hbm_frac": algb / iso / 1e6 / hbm_peak,
-                    "us_per_step_layer_sweep": sweep * 1e3, "hbm_frac_layer_sweep": algb / sweep / 1e6 / hbm_peak}
+                    "us_per_step_layer_sweep": sweep * 1e3, "hbm_frac_layer_sweep": algb / sweep / 1e6 / hbm_peak,
+                    "us_per_step_graph": graph * 1e3, "hbm_frac_graph": algb / graph / 1e6 / hbm_peak}
 
         rows = [row("one CTA per unit", lambda c: (lambda: R.roco_decode_step_cluster(c, q1, k1, v1, rr, out1, ev1, ranks=1,
                                                                                       scale=sc)))]
