@@ -625,9 +625,9 @@ roco_status launch_multi_step(const roco_cache &c, int M, int nb, const void *Q,
   if (c.kv_dtype == ROCO_BF16 && c.d == 128 && (long long)U * c.B < 0x7fffffffLL) {
     // tensor-core path; falls through to the CUDA-core path if the tensor maps cannot be built
     CUtensorMap mapK, mapV;
-    // (the tcgen05 kernel takes its row maxima on the raw scores, which is the maximum of the scaled ones only for
-    // a scale that is not negative)
-    const int um_stages = (multi_um_rows(M, nb) && scale >= 0.f) ? multi_um_pick_stages(c.B, nb) : 0;
+    // (the tcgen05 kernel takes its row maxima on the raw scores and masks with -inf before scaling: right only
+    // for a positive scale)
+    const int um_stages = (multi_um_rows(M, nb) && scale > 0.f) ? multi_um_pick_stages(c.B, nb) : 0;
     // with one CTA per SM either way, the tcgen05 kernel keeps more bytes in flight; with two of the warp-level
     // kernel against one of this, the two win
     const bool tc_two = (multi_tc_smem_bytes(c.B, 3, M, nb) + 1024) * 2 <= (size_t)227 * 1024;

@@ -71,6 +71,25 @@ def test_block_steps_lowest_r_scope_refills(b, r, dtype, d, B):
     assert tally.decisions > 0 and tally.near_ties <= max(4, tally.decisions // 4), tally
 
 
+@pytest.mark.parametrize("scale", [0.0, -0.05])
+def test_block_steps_with_a_scale_that_is_not_positive(scale):
+    """Eq. 1 with scale 0 (uniform attention over what a query may see) and with a negative scale (the largest raw
+    score is then the smallest scaled one, which the tensor-memory kernel's row maxima do not cover: the step must
+    take another kernel and still match)."""
+    B, b = 300, 8
+    w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=3, prompt_lo=B - 10, prompt_hi=B - 10, B=B, r=9)
+    tally = Tally()
+    Q, K, V = prompt_tensors(w, B - 10)
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    st = prefill_parity(cache, Q, K, V, [B - 10], w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, range(w.U), tally, scale=w.scale)
+    par = BlockParity(cache, st, range(w.U), b, w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, tally, scale=scale)
+    t = B - 10
+    for i in range(4):
+        par.step(*block_tokens(w, i * b, b, [t]), check_state=True)
+        t += b
+    assert R.roco_device_status(cache) == 0
+
+
 def test_block_step_after_eviction_prefill_llama_shape():
     """Evict-and-encode with b = 16 on a cache built by prefill eviction (B = 1024, d = 128, bf16, sinks)."""
     w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=8, prompt_lo=1500, prompt_hi=1500)
