@@ -95,7 +95,8 @@ size_t roco_prefill_workspace_bytes(const roco_cache *cache, int Lmax);
 size_t roco_prefill_workspace_bytes_lowest_r(const roco_cache *cache, int Lmax);
 
 /* 1 if roco_prefill will run the score contraction of Eq. 1 on the tensor cores for this cache's dtype and
- * head dimension (bf16, d = 128), 0 if it will use the CUDA-core path (host function). */
+ * head dimension (bf16, d = 128; and a positive scale -- zero or negative scales always take the CUDA-core path),
+ * 0 if it will use the CUDA-core path (host function). */
 int roco_prefill_uses_tensor_cores(const roco_cache *cache);
 
 /*
@@ -131,9 +132,9 @@ roco_status roco_prefill(const void *Q, const void *K, const void *V, const int3
  * The output comes from the same sweep over the score tiles that yields the row log-sum-exp (running row maximum,
  * output accumulator rescaled when the maximum moves), so the whole call costs three L x L contractions (scores
  * and P.V in the sweep, scores again for the column statistics) instead of the four of roco_prefill followed by
- * roco_prefill_attend.  That is the tensor-core path (kv_dtype ROCO_BF16, d = 128; it needs scale > 0); for the other
- * dtypes and head dimensions the output comes from a CUDA-core pass over the row log-sum-exp, after the two
- * statistics passes.
+ * roco_prefill_attend.  That is the tensor-core path (kv_dtype ROCO_BF16, d = 128, scale > 0); for the other
+ * dtypes and head dimensions, and for a scale that is not positive, the output comes from a CUDA-core pass over
+ * the row log-sum-exp, after the two statistics passes.
  *   attn_out     [S][G][Lmax][d] device, 16-byte aligned; rows >= lens are left untouched; NULL: roco_prefill
  * All other arguments, results and errors as roco_prefill.
  */

@@ -154,10 +154,10 @@ roco_status roco_prefill_with_output(const void *Q, const void *K, const void *V
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V)) return ROCO_ERR_INVALID_ARG;
   if ((st = check_scope(r, scope_mode, B, false)) != ROCO_OK) return st;
   if (count_self != 1) return ROCO_ERR_UNSUPPORTED;
-  const bool tc = prefill_tc_supported(cache->kv_dtype, cache->d);
-  if (attn_out) {  // tensor cores: from the same sweep that yields the row log-sum-exp (needs a positive scale)
-    if (!aligned16(attn_out) || (tc && !(scale > 0.f))) return ROCO_ERR_INVALID_ARG;
-  }
+  // The tensor-core kernels take maxima on the raw scores and mask before scaling: right for a positive scale only
+  // (any other goes to the CUDA-core path).
+  const bool tc = prefill_tc_supported(cache->kv_dtype, cache->d) && scale > 0.f;
+  if (attn_out && !aligned16(attn_out)) return ROCO_ERR_INVALID_ARG;
   int maxlen = 0;
   for (int b = 0; b < cache->S; ++b) {
     if (lens_host[b] < 1 || lens_host[b] > Lmax) return ROCO_ERR_INVALID_ARG;
@@ -227,7 +227,7 @@ roco_status roco_prefill_attend(const roco_cache *cache, const void *Q, const vo
   int *lens_dev = static_cast<int *>(workspace);
   if (cudaMemcpyAsync(lens_dev, lens_host, (size_t)cache->S * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess)
     return ROCO_ERR_CUDA;
-  if (!prefill_tc_supported(cache->kv_dtype, cache->d))
+  if (!prefill_tc_supported(cache->kv_dtype, cache->d) || !(scale > 0.f))
     return launch_prefill_attend_simt(cache->kv_dtype, cache->d, cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, V,
                                       scale, lse, attn_out, cs);
   return launch_prefill_attend_tc(cache->S, cache->G, Lmax, lens_dev, maxlen, Q, K, V, scale, lse, nullptr, attn_out,

@@ -62,6 +62,24 @@ def test_fill_then_evict_ragged_tiles(mode, order, dtype, d, B, ranks):
     assert t.decisions >= 2 * 5 * 5
 
 
+@pytest.mark.parametrize("scale", [0.0, -0.07])
+@pytest.mark.parametrize("ranks,splits", [(1, 0), (2, 0), (0, 3)])   # one CTA per unit, a cluster of two, the split
+@pytest.mark.parametrize("order", [R.ROCO_EVICT_FIRST, R.ROCO_ATTEND_FIRST])
+def test_decode_with_a_scale_that_is_not_positive(scale, ranks, splits, order):
+    """Eq. 1 with scale 0 (uniform attention) and with a negative scale: masks and maxima must act on the scaled
+    scores."""
+    B = 200
+    w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=3, B=B, r=7)
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    st = oracle.empty_state(w.U, B, w.d)
+    tally = Tally()
+    par = DecodeParity(cache, st, range(w.U), w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, order, tally, scale=scale,
+                       ranks=ranks, splits=splits)
+    for i in range(B + 12):
+        par.step(*W.decode_tokens(w, i, [i], DEV), check_state=(i == B + 11))
+    assert R.roco_device_status(cache) == 0
+
+
 @pytest.mark.parametrize("kind", ["sink", "lowrank", "burst"])
 def test_prefill_eviction_structured(kind):
     """Prefill with eviction to budget on the structured generators, ragged lengths, several column tiles."""

@@ -7,7 +7,7 @@ import torch
 import oracle
 import paper_2402_06262_b200 as R
 import workloads as W
-from harness import unit_view, widen
+from harness import Tally, prefill_parity, unit_view, widen
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -185,13 +185,37 @@ def test_fused_prompt_pass_long_prompt_sampled_rows():
     check_rows(w, Q, K, V, lse, out, [4096], [0, 3, 7], lambda L: rows)
 
 
+@pytest.mark.parametrize("scale", [0.0, -0.06])
+def test_prompt_pass_with_a_scale_that_is_not_positive(scale):
+    """The tensor-core sweeps need a positive scale; zero and negative ones take the CUDA-core path and must still
+    give Eq. 1: log-sum-exp and output of every row, statistics and survivors against the oracle."""
+    w = W.scaled(W.LLAMA7B_PREFILL, S=1, layers=1, heads=2, prompt_lo=300, prompt_hi=300, B=128, r=16)
+    Q, K, V = prompt_tensors(w, 300)
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    lse = torch.zeros(w.S, w.G, 300, dtype=torch.float32, device=DEV)
+    out = torch.full((w.S, w.G, 300, w.d), 7.0, dtype=w.torch_dtype, device=DEV)
+    R.roco_prefill(Q, K, V, [300], w.B, w.r, cache, scale=scale, lse_out=lse, attn_out=out)
+    torch.cuda.synchronize()
+    assert R.roco_device_status(cache) == 0
+    for u in range(w.U):
+        q, k, v = (widen(unit_view(X, [u]))[0] for X in (Q, K, V))
+        want, want_lse = oracle.prompt_attention_rows(q, k, v, list(range(300)), scale)
+        np.testing.assert_allclose(widen(unit_view(lse, [u]))[0], want_lse, rtol=0, atol=1e-4)
+        np.testing.assert_allclose(widen(unit_view(out, [u]))[0], want, rtol=OUT_TOL, atol=OUT_TOL)
+    tally = Tally()
+    prefill_parity(R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV), Q, K, V, [300], w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R,
+                   range(w.U), tally, scale=scale)
+    # the second, separate call for the output takes the same path
+    out2 = torch.full_like(out, 7.0)
+    R.roco_prefill_attend(cache, Q, K, V, [300], lse, out2, scale=scale)
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+
+
 def test_fused_prompt_pass_argument_checks():
     w = W.scaled(W.LLAMA7B_PREFILL, S=1, layers=1, heads=1, prompt_lo=128, prompt_hi=128, B=64, r=8)
     Q, K, V = prompt_tensors(w, 128)
     cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
-    with pytest.raises(R.RocoError) as e:                        # the running-maximum sweep needs scale > 0
-        R.roco_prefill(Q, K, V, [128], w.B, w.r, cache, scale=-0.1, attn_out=torch.zeros_like(Q))
-    assert e.value.code == 1
     misaligned = torch.zeros(Q.numel() + 8, dtype=Q.dtype, device=DEV)[1:1 + Q.numel()].view_as(Q)
     with pytest.raises(R.RocoError) as e:                        # the output must be 16-byte aligned
         R.roco_prefill(Q, K, V, [128], w.B, w.r, cache, attn_out=misaligned)
