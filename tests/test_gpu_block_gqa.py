@@ -90,6 +90,33 @@ def test_block_steps_with_a_scale_that_is_not_positive(scale):
     assert R.roco_device_status(cache) == 0
 
 
+@pytest.mark.parametrize("b,group", [(16, 1), (4, 4), (1, 8), (2, 1)])
+@pytest.mark.parametrize("B", [300, 1000])
+def test_free_slots_may_hold_anything(b, group, B):
+    """Slots past `live` are not part of the cache (the caller's buffers need not be cleared): with NaN in their K
+    and V rows and in their statistics, steps that fill them must give what they give on a clean buffer."""
+    L = B - 150
+    w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=2, prompt_lo=L, prompt_hi=L, B=B, r=9)
+    tally = Tally()
+    cache, st = prefilled(w, L, tally, range(w.U))
+    cache.K[:, :, L:] = float("nan"); cache.V[:, :, L:] = float("nan")
+    cache.s[:, :, L:] = float("nan"); cache.q[:, :, L:] = float("nan"); cache.n[:, :, L:] = -7; cache.pos[:, :, L:] = 123456
+    par = (GqaBlockParity(cache, st, range(w.U), b, group, w.r, tally, scale=w.scale) if group > 1 else
+           BlockParity(cache, st, range(w.U), b, w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, tally, scale=w.scale))
+    t = L
+    for i in range(3):
+        toks = grouped_block_tokens(w, i * b, b, group, [t]) if group > 1 else block_tokens(w, i * b, b, [t])
+        par.step(*toks, check_state=False)
+        t += b
+    assert R.roco_device_status(cache) == 0
+    assert bool(torch.isfinite(par.out.float()).all())
+    live = int(cache.live[0, 0])
+    assert live == L + 3 * b
+    for name in ("s", "q"):
+        assert bool(torch.isfinite(getattr(cache, name)[:, :, :live]).all())
+    assert bool(torch.isfinite(cache.K[:, :, :live].float()).all()) and bool(torch.isfinite(cache.V[:, :, :live].float()).all())
+
+
 def test_block_step_after_eviction_prefill_llama_shape():
     """Evict-and-encode with b = 16 on a cache built by prefill eviction (B = 1024, d = 128, bf16, sinks)."""
     w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=8, prompt_lo=1500, prompt_hi=1500)

@@ -80,6 +80,26 @@ def test_decode_with_a_scale_that_is_not_positive(scale, ranks, splits, order):
     assert R.roco_device_status(cache) == 0
 
 
+@pytest.mark.parametrize("ranks,splits", [(1, 0), (2, 0), (0, 3)])   # one CTA per unit, a cluster of two, the split
+@pytest.mark.parametrize("order", [R.ROCO_EVICT_FIRST, R.ROCO_ATTEND_FIRST])
+def test_free_slots_may_hold_anything(ranks, splits, order):
+    """Slots past `live` are not part of the cache: NaN in their K, V and statistics changes nothing."""
+    B, fill = 400, 170
+    w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=3, B=B, r=7)
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    st = oracle.empty_state(w.U, B, w.d)
+    tally = Tally()
+    par = DecodeParity(cache, st, range(w.U), w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, order, tally, scale=w.scale,
+                       ranks=ranks, splits=splits)
+    for i in range(fill):
+        par.step(*W.decode_tokens(w, i, [i], DEV))
+    cache.K[:, :, fill:] = float("nan"); cache.V[:, :, fill:] = float("nan")
+    cache.s[:, :, fill:] = float("nan"); cache.q[:, :, fill:] = float("nan"); cache.n[:, :, fill:] = -7
+    for i in range(fill, fill + 40):
+        par.step(*W.decode_tokens(w, i, [i], DEV), check_state=(i == fill + 39))
+    assert R.roco_device_status(cache) == 0 and bool(torch.isfinite(par.out.float()).all())
+
+
 @pytest.mark.parametrize("kind", ["sink", "lowrank", "burst"])
 def test_prefill_eviction_structured(kind):
     """Prefill with eviction to budget on the structured generators, ragged lengths, several column tiles."""
