@@ -27,6 +27,7 @@ constexpr int kUmThreads = (kUmMmaWarp + 1) * 32;
 constexpr int kUmBarStaged = 3;                 // consumers + MMA warp: the query operand is in shared memory
 constexpr int kUmBarDone = 4;                   // consumers + policy warps: nobody reads tensor memory any more
 constexpr int kUmMaxTiles = 32;                 // 16 tensor-memory columns each
+constexpr int kUmCtlStaleMax = 60;              // ctl word: a replaced slot held a row's maximum
 constexpr int kUmPBlock = 16384;                // P^T of four tiles: 128 key rows of 128 bytes (4 x 16 queries)
 // kind::f16 instruction descriptors: fp32 accumulator, bf16 operands, M = 128, N = 16
 constexpr uint32_t kIdescUmS = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
@@ -201,6 +202,7 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
     mbar_init(sm.policy_done, 1);
     mbar_init(sm.stats_full, 1);
     sm.ctl[0] = 0;
+    sm.ctl[kUmCtlStaleMax] = 0;
     mbar_init_fence();
   }
   if (warp == 0) {
@@ -458,54 +460,69 @@ __global__ void __launch_bounds__(kUmThreads, 2) multi_step_umma_kernel(const __
 
   // ---- pass 1, while the selection may still be running: row maxima over the slots that held a token before
   // the step.  The slots that the new tokens will take still count with the score of the token they held, which
-  // only makes the maximum an upper bound (it is the stabiliser of the exponentials, nothing else).
+  // only makes the maximum an upper bound (it is the stabiliser of the exponentials, nothing else) -- unless that
+  // score was the row's maximum: far above the others it would push every exponential of the row below the
+  // smallest float.  Then (rare) a second turn takes the maxima again, over the scores as they stand by then.
   float a[kQ];
+  float my_max;
+#pragma unroll 1
+  for (int turn = 0;; ++turn) {
 #pragma unroll
-  for (int i = 0; i < kQ; ++i) a[i] = -INFINITY;
-  for (int it = wg; it < n_tiles; it += 2) {
-    const int j = it * kUmTile + kl;
-    uint32_t r[kQ];
-    tmem_ldq<kQ>(tlane + (uint32_t)(it * 16), r);
-    const bool held = j < live0;
-#pragma unroll
-    for (int i = 0; i < kQ; ++i) a[i] = fmaxf(a[i], held ? __uint_as_float(r[i]) : -INFINITY);
-  }
-  float my_max = all_reduce(a, true, sm.red);  // its barrier also publishes zn, V_new and the cleared block
-  {
-    // the new tokens' scores join the maxima
-    const float *znmax = sm.red + 2 * kMqConsumerWarps * 16;
-    const float zm = fmaxf(znmax[lane & (kQ - 1)], znmax[16 + (lane & (kQ - 1))]);
-    my_max = fmaxf(my_max, zm);
-#pragma unroll
-    for (int k = 0; k < kQ; ++k) a[k] = fmaxf(a[k], __shfl_sync(0xffffffffu, zm, k));
-  }
-  // a[i] <- -(row maximum in the log2 domain); rows that do not exist hold zeros
-#pragma unroll
-  for (int i = 0; i < kQ; ++i) a[i] = (a[i] > -INFINITY) ? -a[i] * zscale : 0.f;
-
-  // ---- the selection's result: masks and the new tokens' scores in place
-  mbar_wait(sm.policy_done, 0, abort_flag, p.status);
-  for (int it = wg; it < n_tiles; it += 2) {
-    const int j = it * kUmTile + kl;
-    const int nt = j < live1 ? (int)sm.newtok[j] : -1;
-    if (__any_sync(0xffffffffu, nt >= 0 || j >= live1)) {
+    for (int i = 0; i < kQ; ++i) a[i] = -INFINITY;
+    for (int it = wg; it < n_tiles; it += 2) {
+      const int j = it * kUmTile + kl;
       uint32_t r[kQ];
       tmem_ldq<kQ>(tlane + (uint32_t)(it * 16), r);
-      if (j >= live1) {
+      const bool counts = turn > 0 || j < live0;  // second turn: the masks are in place
 #pragma unroll
-        for (int i = 0; i < kQ; ++i) r[i] = ninf;
-      } else if (nt >= 0) {  // the new token's scores, -inf where the block's causal mask hides it
-        const uint4 *zr = reinterpret_cast<const uint4 *>(sm.zn + nt * 16);
-#pragma unroll
-        for (int k = 0; k < kQ / 4; ++k) {
-          const uint4 z4 = zr[k];
-          r[4 * k] = z4.x; r[4 * k + 1] = z4.y; r[4 * k + 2] = z4.z; r[4 * k + 3] = z4.w;
-        }
-      }
-      tmem_stq<kQ>(tlane + (uint32_t)(it * 16), r);
+      for (int i = 0; i < kQ; ++i) a[i] = fmaxf(a[i], counts ? __uint_as_float(r[i]) : -INFINITY);
     }
+    my_max = all_reduce(a, true, sm.red);  // its barrier also publishes zn, V_new and the cleared block
+    {
+      // the new tokens' scores join the maxima
+      const float *znmax = sm.red + 2 * kMqConsumerWarps * 16;
+      const float zm = fmaxf(znmax[lane & (kQ - 1)], znmax[16 + (lane & (kQ - 1))]);
+      my_max = fmaxf(my_max, zm);
+#pragma unroll
+      for (int k = 0; k < kQ; ++k) a[k] = fmaxf(a[k], __shfl_sync(0xffffffffu, zm, k));
+    }
+    // a[i] <- -(row maximum in the log2 domain); rows that do not exist hold zeros
+#pragma unroll
+    for (int i = 0; i < kQ; ++i) a[i] = (a[i] > -INFINITY) ? -a[i] * zscale : 0.f;
+    if (turn > 0) break;
+
+    // ---- the selection's result: masks and the new tokens' scores in place
+    mbar_wait(sm.policy_done, 0, abort_flag, p.status);
+    for (int it = wg; it < n_tiles; it += 2) {
+      const int j = it * kUmTile + kl;
+      const int nt = j < live1 ? (int)sm.newtok[j] : -1;
+      if (__any_sync(0xffffffffu, nt >= 0 || j >= live1)) {
+        uint32_t r[kQ];
+        tmem_ldq<kQ>(tlane + (uint32_t)(it * 16), r);
+        if (j >= live1) {
+#pragma unroll
+          for (int i = 0; i < kQ; ++i) r[i] = ninf;
+        } else if (nt >= 0) {  // the new token's scores, -inf where the block's causal mask hides it
+          // (did the score this slot held set a row's maximum?  Within a binary order counts, which also covers
+          // the rounding of the comparison.)
+          bool held_max = false;
+#pragma unroll
+          for (int i = 0; i < kQ; ++i) held_max |= i < M && fmaf(__uint_as_float(r[i]), zscale, a[i]) >= -1.f;
+          if (held_max && j < live0) sm.ctl[kUmCtlStaleMax] = 1;  // (a slot that was free counted for nothing)
+          const uint4 *zr = reinterpret_cast<const uint4 *>(sm.zn + nt * 16);
+#pragma unroll
+          for (int k = 0; k < kQ / 4; ++k) {
+            const uint4 z4 = zr[k];
+            r[4 * k] = z4.x; r[4 * k + 1] = z4.y; r[4 * k + 2] = z4.z; r[4 * k + 3] = z4.w;
+          }
+        }
+        tmem_stq<kQ>(tlane + (uint32_t)(it * 16), r);
+      }
+    }
+    tmem_st_wait();
+    named_bar_sync(kMqBarConsumers, kMqConsumers);
+    if (!sm.ctl[kUmCtlStaleMax]) break;
   }
-  tmem_st_wait();
 
   // ---- pass 2: e = 2^(z - max) in place, row sums
   float sums[kQ];

@@ -117,6 +117,29 @@ def test_free_slots_may_hold_anything(b, group, B):
     assert bool(torch.isfinite(cache.K[:, :, :live].float()).all()) and bool(torch.isfinite(cache.V[:, :, :live].float()).all())
 
 
+def test_evicted_tokens_held_the_row_maxima():
+    """The tokens that leave in this step have, by construction, by far the largest scores of every row (keys 30
+    times the first new query) and the lowest means: a row maximum taken before the selection is known would sit
+    hundreds of binary orders above every score that remains, and the exponentials of the row would all vanish."""
+    B, L, b = 300, 330, 4
+    w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=2, prompt_lo=L, prompt_hi=L, B=B, r=9)
+    tally = Tally()
+    cache, _ = prefilled(w, L, tally, range(w.U))
+    toks = block_tokens(w, 0, b, [L])
+    slots = [5, 77, 150, 290]
+    for u in range(w.U):
+        for sl in slots:
+            n = float(cache.n[0, u, sl])
+            cache.s[0, u, sl] = 1e-6
+            cache.q[0, u, sl] = 1e-12 / n          # variance 0, mean the lowest: in scope and first to go
+            cache.K[0, u, sl] = (30.0 * toks[0][0, u, 0].float()).to(cache.K.dtype)
+    par = BlockParity(cache, state_from_cache(cache, range(w.U)), range(w.U), b, w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R, tally,
+                      scale=w.scale)
+    par.step(*toks, check_state=True)
+    assert sorted(par.ev_slot[0, 0].tolist()) == slots and sorted(par.ev_slot[0, 1].tolist()) == slots
+    assert bool(torch.isfinite(par.out.float()).all()) and R.roco_device_status(cache) == 0
+
+
 def test_block_step_after_eviction_prefill_llama_shape():
     """Evict-and-encode with b = 16 on a cache built by prefill eviction (B = 1024, d = 128, bf16, sinks)."""
     w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=8, prompt_lo=1500, prompt_hi=1500)
