@@ -117,16 +117,18 @@ def test_free_slots_may_hold_anything(b, group, B):
     assert bool(torch.isfinite(cache.K[:, :, :live].float()).all()) and bool(torch.isfinite(cache.V[:, :, :live].float()).all())
 
 
-def test_evicted_tokens_held_the_row_maxima():
+@pytest.mark.parametrize("b", [2, 4, 16])   # warp-level-MMA kernel; tcgen05 kernel with 8 and with 16 query columns
+def test_evicted_tokens_held_the_row_maxima(b):
     """The tokens that leave in this step have, by construction, by far the largest scores of every row (keys 30
     times the first new query) and the lowest means: a row maximum taken before the selection is known would sit
     hundreds of binary orders above every score that remains, and the exponentials of the row would all vanish."""
-    B, L, b = 300, 330, 4
+    B, L = 300, 330
     w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=2, prompt_lo=L, prompt_hi=L, B=B, r=9)
     tally = Tally()
     cache, _ = prefilled(w, L, tally, range(w.U))
     toks = block_tokens(w, 0, b, [L])
-    slots = [5, 77, 150, 290]
+    slots = [5, 77, 150, 290, 11, 23, 35, 47, 59, 61, 83, 95, 107, 119, 131, 143][:b]
+    slots.sort()
     for u in range(w.U):
         for sl in slots:
             n = float(cache.n[0, u, sl])

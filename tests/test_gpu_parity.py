@@ -8,7 +8,7 @@ import torch
 import oracle
 import paper_2402_06262_b200 as R
 import workloads as W
-from harness import DecodeParity, Tally, compare_state, prefill_parity, unit_view, widen
+from harness import DecodeParity, Tally, compare_state, prefill_parity, unit_view, widen, state_from_cache
 
 pytestmark = pytest.mark.gpu
 
@@ -98,6 +98,29 @@ def test_free_slots_may_hold_anything(ranks, splits, order):
     for i in range(fill, fill + 40):
         par.step(*W.decode_tokens(w, i, [i], DEV), check_state=(i == fill + 39))
     assert R.roco_device_status(cache) == 0 and bool(torch.isfinite(par.out.float()).all())
+
+
+@pytest.mark.parametrize("ranks,splits", [(1, 0), (2, 0), (0, 3)])   # one CTA per unit, a cluster of two, the split
+def test_evicted_token_would_have_held_the_maximum(ranks, splits):
+    """The token that leaves in this step (lowest mean, no variance) has a key 30 times the query: under
+    EVICT_FIRST its score is no part of the row, and a maximum that still saw it would wipe out the row."""
+    B, L = 300, 330
+    w = W.scaled(W.LLAMA7B_DECODE, S=1, layers=1, heads=3, prompt_lo=L, prompt_hi=L, B=B, r=9)
+    Q, K, V = (torch.stack(x) for x in zip(*[W.prompt_chunk(w, b, 0, w.G, L, DEV) for b in range(w.S)]))
+    cache = R.Cache(w.S, w.G, w.B, w.d, w.torch_dtype, DEV)
+    R.roco_prefill(Q, K, V, [L], w.B, w.r, cache, scale=w.scale)
+    q, k, v = W.decode_tokens(w, 0, [L], DEV)
+    for u in range(w.U):
+        sl = 40 + 50 * u
+        cache.s[0, u, sl] = 1e-6
+        cache.q[0, u, sl] = 1e-12 / float(cache.n[0, u, sl])
+        cache.K[0, u, sl] = (30.0 * q[0, u].float()).to(cache.K.dtype)
+    tally = Tally()
+    par = DecodeParity(cache, state_from_cache(cache, range(w.U)), range(w.U), w.r, R.ROCO_SCOPE_EXCLUDE_TOP_R,
+                       R.ROCO_EVICT_FIRST, tally, scale=w.scale, ranks=ranks, splits=splits)
+    par.step(q, k, v, check_state=True)
+    assert par.ev_slot[0].tolist() == [40, 90, 140]
+    assert bool(torch.isfinite(par.out.float()).all()) and R.roco_device_status(cache) == 0
 
 
 @pytest.mark.parametrize("kind", ["sink", "lowrank", "burst"])
