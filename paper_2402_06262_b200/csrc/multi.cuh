@@ -61,6 +61,129 @@ struct PolicyView {
   bool stats_by_consumers = false;
 };
 
+// Victims of a block step under ROCO_SCOPE_LOWEST_R when more than one token leaves.  The scope is the r
+// lowest-variance tokens still cached (Sec. 1 reading), so it refills after every eviction: before each eviction but
+// the first the token next in (variance, position) order is admitted, then the in-scope token of lowest mean
+// leaves.  Everything that can take part is known up front: the first scope S (rank m - 1 in variance order), the
+// at most need - 1 tokens that follow it in that order (the admits), and -- since a victim from S is always the
+// lowest-mean token left in S -- the `need` lowest means of S.  Three threshold searches find them; one warp then
+// plays the evictions on those at most 31 tokens.  The freed slots go to ctl[24 ..] in the order they were chosen;
+// mkey is left masked.  Called by the kMqPolicyThreads policy threads.  (Not inlined: it is the rarer reading, and
+// inlined its registers weigh on every kernel that contains the policy warps' code.)
+static __device__ __noinline__ void lowest_r_block_victims(const uint32_t *vkey, float *mkey, SelectScratch *sel, int *ctl,
+                                                    const int *opos, int *status, int r, int live0, int need, int m,
+                                                    uint32_t k_and, uint32_t k_or, int ptid) {
+  const int plane = ptid & 31, pwarp = ptid >> 5;
+  int *list = ctl + 24, *cnt = ctl + 20;
+  uint32_t rank, ties;
+  auto variance_threshold = [&](int rk, uint32_t &T, int &P) {
+    T = radix_select<uint32_t>([&](int j) { return vkey[j]; }, [&](int) { return true; }, live0, (uint32_t)rk, *sel,
+                               ptid, kMqPolicyThreads, kMqBarPolicy, &rank, &ties, k_and, k_or);
+    P = 0x7fffffff;
+    if (ties != rank + 1) {
+      uint32_t r2, t2;
+      P = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)opos[j]; }, [&](int j) { return vkey[j] == T; },
+                                      live0, rank, *sel, ptid, kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
+    }
+  };
+  auto up_to = [&](int j, uint32_t T, int P) {
+    const uint32_t k = vkey[j];
+    return k < T || (k == T && (P == 0x7fffffff || opos[j] <= P));
+  };
+  uint32_t Tv, Tw;
+  int Pv, Pw;
+  variance_threshold(m - 1, Tv, Pv);
+  const int wsize = live0 < m + need - 1 ? live0 : m + need - 1;  // first scope and admits together
+  Tw = Tv; Pw = Pv;
+  if (wsize > m) variance_threshold(wsize - 1, Tw, Pw);
+  int *adm_slot = sel->red_slot;  // the admits (unordered), with the means they had
+  float *adm_mean = sel->red_mean;
+  if (ptid == 0) *cnt = 0;
+  named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+  for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+    if (up_to(j, Tv, Pv)) continue;
+    if (wsize > m && up_to(j, Tw, Pw)) {
+      const int at = atomicAdd(cnt, 1);
+      if (at < kMqMaxQ) { adm_slot[at] = j; adm_mean[at] = mkey[j]; }
+    }
+    mkey[j] = INFINITY;  // outside the first scope: no candidate below
+  }
+  named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+  int n_adm = *cnt;
+  if (n_adm > kMqMaxQ - 1) n_adm = kMqMaxQ - 1;
+  named_bar_sync(kMqBarPolicy, kMqPolicyThreads);  // cnt is reused below
+  // the n_cand lowest means of the first scope: threshold search on the n_cand-th, then everything up to it
+  const int n_cand = need < m ? need : m;
+  const uint32_t Tm = radix_select<uint32_t>([&](int j) { return __float_as_uint(mkey[j]); }, [&](int) { return true; },
+                                             live0, (uint32_t)(n_cand - 1), *sel, ptid, kMqPolicyThreads, kMqBarPolicy,
+                                             &rank, &ties);
+  int Pm = 0x7fffffff;
+  if (ties != rank + 1) {
+    uint32_t r2, t2;
+    Pm = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)opos[j]; },
+                                     [&](int j) { return __float_as_uint(mkey[j]) == Tm; }, live0, rank, *sel, ptid,
+                                     kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
+  }
+  if (ptid == 0) *cnt = 0;
+  named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+  for (int j = ptid; j < live0; j += kMqPolicyThreads) {
+    const uint32_t k = __float_as_uint(mkey[j]);
+    if (k < 0x7f800000u && (k < Tm || (k == Tm && (Pm == 0x7fffffff || opos[j] <= Pm)))) {
+      const int at = atomicAdd(cnt, 1);
+      if (at < kMqMaxQ) list[at] = j;
+    }
+  }
+  named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+  bool ok = *cnt == n_cand;
+  if (pwarp == 0) {
+    // lanes 0-15: the candidates of the first scope; lanes 16-31: the admits, ranked in (variance, position) order
+    const bool is_adm = plane >= 16;
+    const int idx = is_adm ? plane - 16 : plane;
+    const bool has = is_adm ? idx < n_adm : idx < n_cand;
+    int slot = -1, pj = 0x7fffffff;
+    float mean = INFINITY;
+    uint32_t vk = 0xffffffffu;
+    if (has) {
+      slot = is_adm ? adm_slot[idx] : list[idx];
+      if (slot < 0 || slot >= live0) slot = 0;  // only after corrupt statistics
+      mean = is_adm ? adm_mean[idx] : mkey[slot];
+      pj = opos[slot];
+      vk = vkey[slot];
+    }
+    int ord = 0;
+#pragma unroll
+    for (int i = 16; i < 32; ++i) {
+      const uint32_t ovk = __shfl_sync(0xffffffffu, vk, i);
+      const int op = __shfl_sync(0xffffffffu, pj, i);
+      const bool oh = __shfl_sync(0xffffffffu, (int)has, i) != 0;
+      if (oh && (ovk < vk || (ovk == vk && op < pj))) ++ord;
+    }
+    bool in_scope = has && !is_adm, gone = false;
+    int n_admitted = 0;
+#pragma unroll 1
+    for (int it = 0; it < need; ++it) {
+      if (it > 0 && r <= live0 - it && n_admitted < n_adm) {  // the scope has lost a token: the next one enters
+        if (has && is_adm && ord == n_admitted) in_scope = true;
+        ++n_admitted;
+      }
+      float bm = (in_scope && !gone) ? mean : INFINITY;
+      int bp = pj, bs = (in_scope && !gone) ? slot : -1;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, bm, o);
+        const int op = __shfl_xor_sync(0xffffffffu, bp, o);
+        const int os = __shfl_xor_sync(0xffffffffu, bs, o);
+        if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
+      }
+      if (bs < 0) { ok = false; bs = it; }  // only after corrupt statistics; keeps the slots distinct
+      else if (in_scope && !gone && slot == bs) gone = true;
+      if (plane == 0) list[it] = bs;
+    }
+    if (!ok && plane == 0) atomicOr(status, ROCO_DEV_BAD_VICTIM);
+  }
+  named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+}
+
 // The policy warps' part of a multi-query step: free `need` slots (Sec. 4.3 rule on frozen statistics), insert
 // the new tokens in increasing slot order, score the queries against the new keys, and -- once the consumers
 // have normalised -- apply the statistics update.  Called by the kMqPolicyThreads policy threads.
@@ -192,10 +315,10 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
       }
       return ok;
     };
-    // the `need` smallest of mkey by radix select on the need-th, then one pass that collects everything up to it
-    auto collect_lowest = [&](uint32_t m_and, uint32_t m_or) {
+    // the kn smallest of mkey by radix select on the kn-th, then one pass that collects everything up to it
+    auto collect_lowest = [&](int kn, uint32_t m_and, uint32_t m_or) {
       const uint32_t Tm = radix_select<uint32_t>([&](int j) { return __float_as_uint(v.mkey[j]); },
-                                                 [&](int) { return true; }, live0, (uint32_t)(need - 1), *v.sel, ptid,
+                                                 [&](int) { return true; }, live0, (uint32_t)(kn - 1), *v.sel, ptid,
                                                  kMqPolicyThreads, kMqBarPolicy, &rank, &ties, m_and, m_or);
       int Pm = 0x7fffffff;
       if (ties != rank + 1) {
@@ -214,7 +337,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
         }
       }
       named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      return *cnt == need;
+      return *cnt == kn;
     };
 
     // A scope that leaves out only a few tokens almost always contains the `need` tokens of lowest mean.  So
@@ -223,89 +346,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
     // (they come before it too) -- one counting pass in place of the radix select for the scope threshold.
     bool done = false;
     if (need > 1 && p.scope_mode == ROCO_SCOPE_LOWEST_R && m < live0) {
-      // The scope is the r lowest-variance tokens still cached (Sec. 1 reading), so it refills after every
-      // eviction: one radix select gives the scope of the first eviction, and each later one admits the token
-      // next in (variance, position) order before the in-scope token of lowest mean leaves.  The state of a
-      // token is kept in newtok for the duration: -1 outside the scope, -2 in scope, -3 evicted.
-      uint32_t Tv = radix_select<uint32_t>([&](int j) { return v.vkey[j]; }, [&](int) { return true; }, live0,
-                                           (uint32_t)(m - 1), *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy, &rank, &ties,
-                                           k_and, k_or);
-      int Pv = 0x7fffffff;
-      if (ties != rank + 1) {
-        uint32_t r2, t2;
-        Pv = (int)radix_select<uint32_t>([&](int j) { return (uint32_t)opos[j]; },
-                                         [&](int j) { return v.vkey[j] == Tv; }, live0, rank, *v.sel, ptid,
-                                         kMqPolicyThreads, kMqBarPolicy, &r2, &t2);
-      }
-      for (int j = ptid; j < live0; j += kMqPolicyThreads) {
-        const uint32_t k = v.vkey[j];
-        if (k < Tv || (k == Tv && (Pv == 0x7fffffff || opos[j] <= Pv))) v.newtok[j] = -2;
-      }
-      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      bool ok = true;
-#pragma unroll 1
-      for (int it = 0; it < need; ++it) {
-        if (it > 0 && p.r <= live0 - it) {  // the scope has lost a token and the cache still holds one to admit
-          uint32_t bk = 0xffffffffu;
-          int bs = -1, bp = 0x7fffffff;
-          for (int j = ptid; j < live0; j += kMqPolicyThreads) {
-            if (v.newtok[j] != -1) continue;
-            const uint32_t k = v.vkey[j];
-            const int pj = opos[j];
-            if (bs < 0 || k < bk || (k == bk && pj < bp)) { bk = k; bs = j; bp = pj; }
-          }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            const uint32_t ok2 = __shfl_xor_sync(0xffffffffu, bk, o);
-            const int op = __shfl_xor_sync(0xffffffffu, bp, o);
-            const int os = __shfl_xor_sync(0xffffffffu, bs, o);
-            if (os >= 0 && (bs < 0 || ok2 < bk || (ok2 == bk && op < bp))) { bk = ok2; bp = op; bs = os; }
-          }
-          if (plane == 0) { v.sel->hist[pwarp] = bk; v.sel->red_pos[pwarp] = bp; v.sel->red_slot[pwarp] = bs; }
-          named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-          bk = v.sel->hist[0]; bp = v.sel->red_pos[0]; bs = v.sel->red_slot[0];
-#pragma unroll
-          for (int w = 1; w < kMqPolicyThreads / 32; ++w) {
-            const uint32_t ok2 = v.sel->hist[w];
-            const int op = v.sel->red_pos[w], os = v.sel->red_slot[w];
-            if (os >= 0 && (bs < 0 || ok2 < bk || (ok2 == bk && op < bp))) { bk = ok2; bp = op; bs = os; }
-          }
-          named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-          if (bs >= 0 && ptid == 0) v.newtok[bs] = -2;
-          named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-        }
-        float bm = INFINITY;
-        int bs = -1, bp = 0x7fffffff;
-        for (int j = ptid; j < live0; j += kMqPolicyThreads) {
-          if (v.newtok[j] != -2) continue;
-          const float mean = v.mkey[j];
-          const int pj = opos[j];
-          if (mean < bm || (mean == bm && pj < bp)) { bm = mean; bs = j; bp = pj; }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          const float om = __shfl_xor_sync(0xffffffffu, bm, o);
-          const int op = __shfl_xor_sync(0xffffffffu, bp, o);
-          const int os = __shfl_xor_sync(0xffffffffu, bs, o);
-          if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
-        }
-        if (plane == 0) { v.sel->red_mean[pwarp] = bm; v.sel->red_pos[pwarp] = bp; v.sel->red_slot[pwarp] = bs; }
-        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-        bm = v.sel->red_mean[0]; bp = v.sel->red_pos[0]; bs = v.sel->red_slot[0];
-#pragma unroll
-        for (int w = 1; w < kMqPolicyThreads / 32; ++w) {
-          const float om = v.sel->red_mean[w];
-          const int op = v.sel->red_pos[w], os = v.sel->red_slot[w];
-          if (os >= 0 && (bs < 0 || om < bm || (om == bm && op < bp))) { bm = om; bp = op; bs = os; }
-        }
-        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-        if (bs < 0) { ok = false; bs = it; }  // only after corrupt statistics; keeps the slots distinct
-        if (ptid == 0) { list[it] = bs; v.newtok[bs] = -3; }
-        named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
-      }
-      for (int j = ptid; j < live0; j += kMqPolicyThreads) v.newtok[j] = -1;
-      if (!ok && ptid == 0) atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
-      named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
+      lowest_r_block_victims(v.vkey, v.mkey, v.sel, v.ctl, opos, p.status, p.r, live0, need, m, k_and, k_or, ptid);
       done = true;
     } else if (2 * m >= live0) {
       bool ok;
@@ -320,7 +361,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
           m_or |= k;
         }
         group_and_or(m_and, m_or, *v.sel, ptid, kMqPolicyThreads, kMqBarPolicy);
-        ok = collect_lowest(m_and, m_or);
+        ok = collect_lowest(need, m_and, m_or);
       }
       named_bar_sync(kMqBarPolicy, kMqPolicyThreads);  // list[] is complete
       // the candidate last in (variance, position) order
@@ -391,7 +432,7 @@ __device__ __forceinline__ void multi_policy(const MultiParams &p, const PolicyV
       named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
       bool ok;
       if (need <= 4) ok = argmin_rounds(need);  // few victims: one argmin after the other
-      else ok = collect_lowest(0u, 0xffffffffu);
+      else ok = collect_lowest(need, 0u, 0xffffffffu);
       named_bar_sync(kMqBarPolicy, kMqPolicyThreads);
       if (!ok && ptid == 0) {  // only after corrupt statistics; the step's results are void
         atomicOr(p.status, ROCO_DEV_BAD_VICTIM);
