@@ -9,9 +9,10 @@ all layers*heads units of each sequence).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
                     [--scope-mode exclude_top_r|lowest_r] [--step-order evict_first|attend_first]
-                    [--all-workloads] [--readings] [--extras]
+                    [--all-workloads] [--readings] [--no-extras]
 
-`--readings` adds the three other combinations of scope reading and step order on the same workload, and
+On one GPU the line also carries the calls with few units (`few_units`), the block-wise and grouped-query steps
+(`multi_query`) and the prompt pass (`prefill`).  `--readings` adds the three other combinations of scope reading and step order on the same workload, and
 `--all-workloads` the serving-batch and long-context decode workloads, as extra keys of the same line.
 
 N > 1 (under torch.distributed.run): every rank runs the same-sized workload on its own GPU with its own
@@ -676,7 +677,10 @@ def main():
     ap.add_argument("--small", action="store_true", help="1/16 of the units (for profiler captures)")
     ap.add_argument("--prefill-only", action="store_true", help="run only the prefill measurement")
     ap.add_argument("--no-prefill", action="store_true", help="skip the prefill measurement")
-    ap.add_argument("--extras", action="store_true", help="also time the block-wise and grouped-query steps")
+    ap.add_argument("--extras", action="store_true",
+                    help="time the block-wise and grouped-query steps too (the default on one GPU; with several, only "
+                         "when asked)")
+    ap.add_argument("--no-extras", action="store_true", help="skip the block-wise and grouped-query steps")
     ap.add_argument("--no-few-units", action="store_true", help="skip the calls with few units (one layer at a time)")
     ap.add_argument("--prefill-workload", default="llama7b_prefill", help="workload of the prefill measurement")
     ap.add_argument("--scope-r", type=int, default=None, help="override the workload's scope parameter r")
@@ -727,9 +731,17 @@ def main():
             "roofline": res["roofline"]}
 
     torch.cuda.empty_cache()
-    if args.extras:
-        line["multi_query"] = multi_bench(R, cache, w, device)
-        line["few_units"] = line["multi_query"].pop("few_units")
+    extras = (args.extras or world == 1) and not args.no_extras and w.dtype == "bf16"
+    if extras and args.no_few_units and not args.extras:
+        extras = False   # a run trimmed to the decode step alone
+    if extras:
+        try:
+            line["multi_query"] = multi_bench(R, cache, w, device)
+            line["few_units"] = line["multi_query"].pop("few_units")
+        except Exception as e:   # the headline must not depend on the extra rows
+            line["multi_query"] = {"error": f"{type(e).__name__}: {e}"}
+        if R.roco_device_status(cache) != 0:
+            raise RuntimeError("device status word set during the multi-query steps")
     elif not args.no_few_units and w.dtype == "bf16":
         line["few_units"] = few_units_bench(R, cache, w, device)
         if R.roco_device_status(cache) != 0:
