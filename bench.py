@@ -12,7 +12,8 @@ all layers*heads units of each sequence).
                     [--all-workloads] [--readings] [--no-extras]
 
 On one GPU the line also carries the calls with few units (`few_units`), the block-wise and grouped-query steps
-(`multi_query`) and the prompt pass (`prefill`).  `--readings` adds the three other combinations of scope reading and step order on the same workload, and
+(`multi_query`), the four readings (`readings`), the two other decode workloads (`workloads`) and the prompt pass
+(`prefill`); `--no-extras` trims it to the decode step, the calls with few units and the prompt pass.  `--readings` adds the three other combinations of scope reading and step order on the same workload, and
 `--all-workloads` the serving-batch and long-context decode workloads, as extra keys of the same line.
 
 N > 1 (under torch.distributed.run): every rank runs the same-sized workload on its own GPU with its own
@@ -766,7 +767,10 @@ def main():
                 "frac_of_read_stream": r["roofline"].get("frac_of_read_stream"),
                 "e2e_tokens_per_s": r["e2e"]["value"], "e2e_frac_of_device_timed": r["e2e"]["frac_of_device_timed"]}
 
-    if args.readings:      # the same workload under the other readings of scope and order
+    # on one GPU the plain run carries the extra keys too (they take about 20 s)
+    full_line = (world == 1 and not args.no_extras and not args.no_few_units and not args.small and
+                 not args.no_prefill and args.workload == "llama7b_decode")
+    if args.readings or full_line:      # the same workload under the other readings of scope and order
         line["readings"] = [dict(brief(res), scope_mode=args.scope_mode, step_order=args.step_order)]
         for sm_name, so_name in [(a, b) for a in ("exclude_top_r", "lowest_r") for b in ("evict_first", "attend_first")]:
             if (sm_name, so_name) == (args.scope_mode, args.step_order):
@@ -777,7 +781,7 @@ def main():
             line["readings"].append(dict(brief(r2), scope_mode=sm_name, step_order=so_name))
             del c2
             torch.cuda.empty_cache()
-    if args.all_workloads:  # the other decode workloads at their full sizes (extra keys, not the headline)
+    if args.all_workloads or full_line:  # the other decode workloads at their full sizes (extra keys, not the headline)
         line["workloads"] = {}
         for name in ("llama13b_serving", "long_context"):
             if name == args.workload:
