@@ -238,9 +238,9 @@ roco_status roco_decode_step_policy_ordered(roco_cache *cache, const void *q, co
  *   b                1..16, r + b <= B.  Under ROCO_SCOPE_LOWEST_R the scope refills after each of the step's
  *                    evictions (the token next in (variance, position) order is admitted before the next victim
  *                    is taken), all on the statistics as they stand before the step;
- *                    the step's working set must fit on an SM, else ROCO_ERR_UNSUPPORTED: for bf16, d = 128, 4 or
- *                    more query rows and scale > 0: B <= 4096 (scores in tensor memory), otherwise b * B floats of
- *                    scores in shared memory
+ *                    the step's working set must fit on an SM, else ROCO_ERR_UNSUPPORTED: for bf16, d = 128 and
+ *                    scale > 0: B <= 4096 (scores in tensor memory), otherwise b * B floats of scores in shared
+ *                    memory
  *   attn_out         [S][G][b][d];   lse_out [S][G][b] or NULL
  *   evicted_slot     [S][G][b] freed slots in increasing order, padded with -1;  evicted_pos likewise, or NULL
  */

@@ -645,11 +645,11 @@ int multi_um_pick_stages(int B, int nb) {
   return 0;
 }
 
-// Row layouts the tcgen05 kernel takes: from 4 rows up (below that the warp-level kernel is as fast), the heads of
-// a token averaged inside a thread -- group sizes that are powers of two, or one token with any number of heads.
+// Row layouts the tcgen05 kernel takes: the heads of a token are averaged inside a thread -- group sizes that are
+// powers of two, or one token with any number of heads.
 bool multi_um_rows(int M, int nb) {
   const int grp = M / nb;
-  return M >= 4 && (nb == 1 || grp == 1 || grp == 2 || grp == 4 || grp == 8);
+  return M >= 1 && (nb == 1 || grp == 1 || grp == 2 || grp == 4 || grp == 8);
 }
 
 int launch_multi_step_umma(const MultiParams &p, const roco_cache &c, int U, cudaStream_t stream) {
