@@ -361,6 +361,10 @@ roco_status roco_gqa_block_step(roco_cache *cache, const void *Q, const void *K_
   if ((st = check_scope(r, scope_mode, cache->B, true)) != ROCO_OK) return st;
   if ((long long)b * group > multi_max_queries()) return ROCO_ERR_UNSUPPORTED;
   if (b > 1 && r + b > cache->B) return ROCO_ERR_INVALID_ARG;  // the scope must hold the b victims
+  if (b == 1 && group == 1)  // one token, one head: the decode step in the order of Fig. 1 (same layouts), which
+                             // also picks its launch shape from the number of units
+    return roco_decode_step(cache, Q, K_new, V_new, r, scope_mode, ROCO_EVICT_FIRST, scale, attn_out, lse_out,
+                            evicted_slot, evicted_pos, stream);
   if (!multi_fits(cache->B, cache->d, b * group, b)) return ROCO_ERR_UNSUPPORTED;
   return launch_multi_step(*cache, b * group, b, Q, K_new, V_new, r, scope_mode, scale, attn_out, lse_out,
                            evicted_slot, evicted_pos, static_cast<cudaStream_t>(stream));
