@@ -16,3 +16,10 @@ def pytest_configure(config):
 def _oracle_built():
     from oracle.build import build
     build()
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _library_built():
+    """libroco.so is built in-tree (and rebuilt when a source is newer); the binding itself never builds."""
+    from paper_2402_06262_b200.build import build
+    build()
